@@ -1,0 +1,243 @@
+"""fp64 CPU oracle for the MtPC head: TEST INFRASTRUCTURE, not a product path.
+
+Plain, slow, step-by-step numpy (float64) statement of what the head computes, written from the paper's
+definitions. It shares no code with the CUDA library and must never be imported by it; only the tests,
+the smoke check and the benchmark's CPU-baseline leg call it.
+
+What follows which passage:
+  emission_logphi   Sec. 3.3 "Input unit distributions": phi_tij = softmax(W_ij e_t)
+  sum_unit_logw     Sec. 3.3 "Sum unit parameters":      omega_ti = softmax(R_i e_t)
+  evidence          Sec. 3.1 (input units) + App. B.1 (a marginalised input unit integrates to 1)
+  cp_eval           Eq. (CP)
+  hmm_eval          Eq. (HMM), evaluated layer by layer (one sum + one product layer per window step)
+  btree_eval        Eq. (BTree), recursive halving with a latent per internal node
+  draft_sample      App. B.2, Algorithm 1 (ancestral sampling), with inverse-CDF categorical draws
+  circuit_counts    App. C, Table 3 (sizes of the circuits and of the linear head)
+
+Readings taken where the paper is silent or garbled (each is listed in the design notes too):
+  * BTree: the left half is the first floor(n/2) tokens; a child latent depends on its parent's latent
+    only; products are element-wise in the latent; n must be a power of two here. Internal nodes are in
+    heap order (root 0, children 2j+1 and 2j+2); the deepest internal node n/2-1+m owns tokens 2m, 2m+1.
+    Table 3's parameter counts fix the number of sum units at 1 + (n-2) r, each of fan-in r.
+  * HMM: T_static[i-1, a, b] is the logit of z_i = b given z_{i-1} = a (softmax over b); only the initial
+    distribution is contextual here (the paper's "non-contextual" transition variant).
+  * sampleCategorical is inverse-CDF: the smallest index j with u < p_0 + ... + p_j (last index if none).
+  * The draft log-prob is the joint marginal log q(x_1..x_n) (latents summed out), as verification needs.
+  * No bias and no temperature in either projection.
+
+Pins (tests/test_oracle_*.py): brute-force normalisation over all v^n strings; CP with r=1 equals the
+product of marginals; CP/HMM/BTree equal literal enumeration over latent assignments; HMM with identity
+transitions equals CP; BTree with n=2 equals CP; masked targets equal brute-force marginals; closed-form
+softmax cases; sampled frequencies match the exact joint (chi-squared); Table 3 counts. No function here
+is left unpinned.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+CP, HMM, BTREE = 0, 1, 2
+
+
+# ----------------------------------------------------------------------------------------------------
+# elementary pieces
+# ----------------------------------------------------------------------------------------------------
+def logsumexp(x: np.ndarray, axis: int = -1) -> np.ndarray:
+    m = np.max(x, axis=axis, keepdims=True)
+    return np.squeeze(m, axis=axis) + np.log(np.sum(np.exp(x - m), axis=axis))
+
+
+def log_softmax(x: np.ndarray, axis: int = -1) -> np.ndarray:
+    return x - np.expand_dims(logsumexp(x, axis=axis), axis)
+
+
+def num_sum_units(family: int, n: int, r: int, contextual_transitions: bool = False) -> int:
+    """How many sum units the head parameterises from the hidden state (the z of R in R^{z x r x d})."""
+    if family == CP:
+        return 1
+    if family == HMM:
+        return 1 + (n - 1) * r if contextual_transitions else 1
+    if family == BTREE:
+        return 1 + (n - 2) * r
+    raise ValueError(family)
+
+
+def circuit_counts(family: str, n: int, r: int, v: int, d: int) -> dict:
+    """Parameter and FLOP counts in the convention of Table 3 (contextual HMM transitions, as the paper's
+    experiments use). A sum unit of fan-in r costs 2r FLOPs; FF is n input units and one product."""
+    if family == "ff":
+        return dict(circuit_params=n * v, circuit_flops=n - 1, head_params=n * v * d, head_flops=2 * n * v * d)
+    fam = {"cp": CP, "hmm": HMM, "btree": BTREE}[family]
+    S = num_sum_units(fam, n, r, contextual_transitions=True)
+    circuit_params = n * r * v + S * r
+    head_params = circuit_params * d
+    return dict(circuit_params=circuit_params, circuit_flops=2 * r * S, head_params=head_params,
+                head_flops=2 * head_params)
+
+
+# ----------------------------------------------------------------------------------------------------
+# head: hidden state -> circuit parameters (Sec. 3.3)
+# ----------------------------------------------------------------------------------------------------
+def emission_logphi(h: np.ndarray, W_emit: np.ndarray) -> np.ndarray:
+    """log phi[t, i, k, :] = log softmax(W_emit[i, k] @ h[t]);  h [T, d], W_emit [n, r, v, d] -> [T, n, r, v]."""
+    h = np.asarray(h, dtype=np.float64)
+    W = np.asarray(W_emit, dtype=np.float64)
+    n, r, v, d = W.shape
+    logits = (h @ W.reshape(n * r * v, d).T).reshape(h.shape[0], n, r, v)
+    return log_softmax(logits, axis=-1)
+
+
+def sum_unit_logw(h: np.ndarray, W_sum: np.ndarray, r: int) -> np.ndarray:
+    """log omega[t, s, :] = log softmax(W_sum[s*r:(s+1)*r] @ h[t]);  -> [T, S, r]."""
+    h = np.asarray(h, dtype=np.float64)
+    R = np.asarray(W_sum, dtype=np.float64)
+    logits = (h @ R.T).reshape(h.shape[0], R.shape[0] // r, r)
+    return log_softmax(logits, axis=-1)
+
+
+def evidence(logphi: np.ndarray, targets: np.ndarray, pos: np.ndarray | None = None) -> np.ndarray:
+    """g[w, i, k] = log phi[pos[w], i, k, x_wi]; a negative target marginalises the byte: the unit
+    outputs 1 (log 0 = 0 contribution). `pos` maps each window to its position (identity if None)."""
+    T, n, r, v = logphi.shape
+    x = np.asarray(targets).reshape(-1, n)
+    if pos is None:
+        pos = np.arange(T)
+    safe = np.where(x < 0, 0, x)
+    g = logphi[pos[:, None, None], np.arange(n)[None, :, None], np.arange(r)[None, None, :], safe[:, :, None]]
+    return np.where((x < 0)[:, :, None], 0.0, g)
+
+
+# ----------------------------------------------------------------------------------------------------
+# circuit evaluation (log space)
+# ----------------------------------------------------------------------------------------------------
+def cp_eval(logw: np.ndarray, g: np.ndarray) -> np.ndarray:
+    """Eq. (CP): sum_z q(z) prod_i q(x_i | z);  logw [T, r], g [T, n, r] -> [T]."""
+    return logsumexp(logw + g.sum(axis=1), axis=-1)
+
+
+def hmm_eval(logpi: np.ndarray, logA: np.ndarray, g: np.ndarray) -> np.ndarray:
+    """Eq. (HMM). logpi [T, r]; logA [n-1, r, r] with logA[i-1, a, b] = log q(z_i = b | z_{i-1} = a);
+    g [T, n, r]. alpha_1(z) = q(z) q(x_1|z); alpha_i(b) = q(x_i|b) sum_a alpha_{i-1}(a) q(b|a)."""
+    T, n, r = g.shape
+    alpha = logpi + g[:, 0, :]
+    for i in range(1, n):
+        alpha = g[:, i, :] + logsumexp(alpha[:, :, None] + logA[i - 1][None, :, :], axis=1)
+    return logsumexp(alpha, axis=-1)
+
+
+def _btree_product(j: int, lo: int, hi: int, logw: np.ndarray, g: np.ndarray, r: int) -> np.ndarray:
+    """log of the product unit under latent z_j over tokens [lo, hi): [T, r] indexed by the value of z_j."""
+    mid = lo + (hi - lo) // 2
+    out = 0.0
+    for child, (a, b) in ((2 * j + 1, (lo, mid)), (2 * j + 2, (mid, hi))):
+        if b - a == 1:
+            out = out + g[:, a, :]                       # input units of token a, one per value of z_j
+        else:
+            below = _btree_product(child, a, b, logw, g, r)            # [T, r] over z_child
+            rows = 1 + (child - 1) * r                                  # sum units of node `child`
+            logOmega = logw[:, rows:rows + r, :]                        # [T, z_j, z_child]
+            out = out + logsumexp(logOmega + below[:, None, :], axis=-1)
+    return out
+
+
+def btree_eval(logw: np.ndarray, g: np.ndarray) -> np.ndarray:
+    """Eq. (BTree). logw [T, 1 + (n-2) r, r]: group 0 = root weights; group 1 + (j-1) r + a = weights of
+    node j's latent given its parent's latent = a.  g [T, n, r]."""
+    T, n, r = g.shape
+    if n < 2 or (n & (n - 1)):
+        raise ValueError("binary-tree head: n must be a power of two >= 2")
+    return logsumexp(logw[:, 0, :] + _btree_product(0, 0, n, logw, g, r), axis=-1)
+
+
+def static_log_transitions(T_static: np.ndarray) -> np.ndarray:
+    return log_softmax(np.asarray(T_static, dtype=np.float64), axis=-1)
+
+
+def circuit_eval(family: int, logw: np.ndarray, g: np.ndarray, T_static: np.ndarray | None = None) -> np.ndarray:
+    if family == CP:
+        return cp_eval(logw[:, 0, :], g)
+    if family == HMM:
+        return hmm_eval(logw[:, 0, :], static_log_transitions(T_static), g)
+    if family == BTREE:
+        return btree_eval(logw, g)
+    raise ValueError(family)
+
+
+def window_logprob(family: int, h, W_emit, W_sum, T_static, targets) -> np.ndarray:
+    """log q(x_{t+1..t+n} | context) in nats for every position: [T]."""
+    r = np.asarray(W_emit).shape[1]
+    logphi = emission_logphi(h, W_emit)
+    logw = sum_unit_logw(h, W_sum, r)
+    return circuit_eval(family, logw, evidence(logphi, targets), T_static)
+
+
+# ----------------------------------------------------------------------------------------------------
+# ancestral sampling (Algorithm 1) from pre-generated uniforms
+# ----------------------------------------------------------------------------------------------------
+def inv_cdf(logp: np.ndarray, u: np.ndarray):
+    """Rows of log-probabilities [M, c] and uniforms [M] -> (index [M], margin [M]).
+    index = smallest j with u < p_0 + ... + p_j, or c-1 if rounding leaves none.
+    margin = distance from u to the nearest interior CDF boundary (how close the draw is to flipping)."""
+    cdf = np.cumsum(np.exp(logp), axis=-1)
+    u = np.asarray(u, dtype=np.float64)
+    idx = np.minimum((cdf <= u[:, None]).sum(axis=-1), logp.shape[-1] - 1)
+    if logp.shape[-1] > 1:
+        margin = np.abs(cdf[:, :-1] - u[:, None]).min(axis=-1)
+    else:
+        margin = np.full(u.shape, np.inf)
+    return idx.astype(np.int64), margin
+
+
+def sample_latents(family: int, logw: np.ndarray, T_static, wpp: int, u: np.ndarray, n: int):
+    """Top-down draws at the sum units. logw [P, S, r]; u [P*wpp, 2n] (latent draws use columns 0..n-1:
+    CP column 0; HMM column i for z_i; BTree column j for internal node j). Returns
+    (unit [W, n]: the input unit selected for every token, margin [W]: smallest latent-draw margin)."""
+    P, S, r = logw.shape
+    W = P * wpp
+    pos = np.repeat(np.arange(P), wpp)
+    unit = np.zeros((W, n), dtype=np.int64)
+    margin = np.full(W, np.inf)
+    if family == CP:
+        z, m = inv_cdf(logw[pos, 0, :], u[:, 0])
+        unit[:] = z[:, None]
+        margin = m
+    elif family == HMM:
+        logA = static_log_transitions(T_static)
+        z, margin = inv_cdf(logw[pos, 0, :], u[:, 0])
+        unit[:, 0] = z
+        for i in range(1, n):
+            z, m = inv_cdf(logA[i - 1][z, :], u[:, i])
+            unit[:, i] = z
+            margin = np.minimum(margin, m)
+    elif family == BTREE:
+        zs = np.zeros((W, n - 1), dtype=np.int64)
+        zs[:, 0], margin = inv_cdf(logw[pos, 0, :], u[:, 0])
+        for j in range(1, n - 1):
+            parent = (j - 1) // 2
+            zs[:, j], m = inv_cdf(logw[pos, 1 + (j - 1) * r + zs[:, parent], :], u[:, j])
+            margin = np.minimum(margin, m)
+        for i in range(n):
+            unit[:, i] = zs[:, n // 2 - 1 + i // 2]
+    else:
+        raise ValueError(family)
+    return unit, margin
+
+
+def draft_sample(family: int, h, W_emit, W_sum, T_static, wpp: int, u: np.ndarray):
+    """Algorithm 1 for wpp windows per position. Window w = p*wpp + j uses uniforms u[w]: latent draws in
+    columns 0..n-1, the byte of token i in column n+i. Returns dict(bytes [W, n], logprob [W] = joint
+    marginal log q of the drafted bytes, unit [W, n], margin [W] = smallest |u - CDF boundary| of any draw
+    the window made)."""
+    W_emit = np.asarray(W_emit)
+    n, r, v, d = W_emit.shape
+    logphi = emission_logphi(h, W_emit)                     # [P, n, r, v]
+    logw = sum_unit_logw(h, W_sum, r)
+    P = logphi.shape[0]
+    pos = np.repeat(np.arange(P), wpp)
+    unit, margin = sample_latents(family, logw, T_static, wpp, u, n)
+    x = np.zeros((P * wpp, n), dtype=np.int64)
+    for i in range(n):
+        x[:, i], m = inv_cdf(logphi[pos, i, unit[:, i], :], u[:, n + i])
+        margin = np.minimum(margin, m)
+    g = evidence(logphi, x, pos)
+    logprob = circuit_eval(family, logw[pos], g, T_static)
+    return dict(bytes=x, logprob=logprob, unit=unit, margin=margin)

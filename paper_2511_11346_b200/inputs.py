@@ -1,0 +1,176 @@
+"""Seeded synthetic inputs for the MtPC head (shared by the tests, the bench and the CPU oracle's callers).
+
+This module holds NONE of the method's arithmetic: it only draws random tensors with the shapes, dtypes
+and value distributions of the five workloads and quantises them to bf16 (round-to-nearest-even) so that
+the CUDA path and the fp64 oracle read bit-identical values.
+
+Workloads (stand-ins for the paper's EvaByte / Llama-byte features and trained unembeddings, which need
+weights and data that are not available offline):
+  0  CP tiny            T=256  d=256  n=4  r=8  v=256  fp32 io, uniform targets, + 256 draft windows
+  1  CP training-shaped T=8192 d=4096 n=8  r=16 v=320  bf16, Zipf(1.1) targets
+  2  HMM                T=8192 d=4096 n=8  r=32 v=320  bf16, static transitions ~N(0,1), Zipf(1.1) targets
+  3  BTree              T=4096 d=3072 n=16 r=32 v=256  bf16, uniform targets, + draft wpp=1
+  4  decode sweep cells P in {1,8,64}, d=4096, v=320, CP r=16 / HMM r=32, n in {8,16}, wpp=16
+Hidden states ~N(0,1); every weight ~N(0, std=0.02); uniforms in [0,1) as fp32.
+"""
+from __future__ import annotations
+
+import dataclasses
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+CP, HMM, BTREE = 0, 1, 2
+F32, BF16 = 0, 1
+FAMILY_NAMES = {CP: "cp", HMM: "hmm", BTREE: "btree"}
+BASE_SEED = 2511113460
+
+
+@dataclasses.dataclass(frozen=True)
+class HeadShape:
+    family: int
+    n: int
+    r: int
+    v: int
+    d: int
+    io_dtype: int = BF16
+
+    @property
+    def num_sum_groups(self) -> int:
+        """Number of contextual sum units S (each has r weights produced from the hidden state)."""
+        if self.family == BTREE:
+            return 1 + (self.n - 2) * self.r
+        return 1
+
+    @property
+    def sum_rows(self) -> int:
+        return self.num_sum_groups * self.r
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round fp32 values to the nearest bf16 (ties to even); returns fp32 holding bf16-representable values."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    bits = x.view(np.uint32)
+    lsb = (bits >> np.uint32(16)) & np.uint32(1)
+    rounded = (bits + np.uint32(0x7FFF) + lsb) & np.uint32(0xFFFF0000)
+    return rounded.view(np.float32)
+
+
+def bf16_bits(x_rounded: np.ndarray) -> np.ndarray:
+    """The uint16 bf16 bit patterns of values that are already bf16-representable."""
+    x = np.ascontiguousarray(x_rounded, dtype=np.float32)
+    return (x.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+
+
+_CHUNK = 1 << 22
+
+
+def _normal(seed: int, stream: int, shape, std: float) -> np.ndarray:
+    """N(0, std) fp32 tensor; chunk c of stream s comes from Philox(key=[seed, s * 2^20 + c]), so the
+    values do not depend on how many threads fill the buffer."""
+    total = int(np.prod(shape))
+    out = np.empty(total, dtype=np.float32)
+    nchunks = (total + _CHUNK - 1) // _CHUNK
+
+    def fill(c):
+        lo = c * _CHUNK
+        hi = min(total, lo + _CHUNK)
+        g = np.random.Generator(np.random.Philox(key=[seed, stream * (1 << 20) + c]))
+        out[lo:hi] = g.standard_normal(hi - lo, dtype=np.float32) * np.float32(std)
+
+    if nchunks == 1:
+        fill(0)
+    else:
+        with ThreadPoolExecutor(max_workers=8) as ex:
+            list(ex.map(fill, range(nchunks)))
+    return out.reshape(shape)
+
+
+def _gen(seed: int, stream: int) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[seed, stream * (1 << 20)]))
+
+
+def zipf_targets(seed: int, stream: int, shape, v: int, a: float = 1.1) -> np.ndarray:
+    """Symbols whose RANKS follow a Zipf(a) law truncated to v; rank -> symbol by a seeded permutation."""
+    g = _gen(seed, stream)
+    pmf = 1.0 / np.arange(1, v + 1, dtype=np.float64) ** a
+    pmf /= pmf.sum()
+    ranks = g.choice(v, size=shape, p=pmf)
+    perm = g.permutation(v)
+    return perm[ranks].astype(np.int32)
+
+
+def uniform_targets(seed: int, stream: int, shape, v: int) -> np.ndarray:
+    return _gen(seed, stream).integers(0, v, size=shape, dtype=np.int32)
+
+
+def uniforms(seed: int, stream: int, shape) -> np.ndarray:
+    """fp32 uniforms in [0,1) on a 2^-24 grid (exactly representable, never 1.0)."""
+    k = _gen(seed, stream).integers(0, 1 << 24, size=shape, dtype=np.int64)
+    return (k.astype(np.float64) / float(1 << 24)).astype(np.float32)
+
+
+@dataclasses.dataclass
+class Workload:
+    """Everything one call needs. `*_q` arrays are fp32 holding the bf16-rounded values both sides compute
+    on; `hidden_raw` / `W_*_raw` are the un-rounded fp32 tensors, handed to the library only when io_dtype is F32."""
+    name: str
+    shape: HeadShape
+    T: int
+    hidden_q: np.ndarray
+    W_emit_q: np.ndarray
+    W_sum_q: np.ndarray
+    T_static: np.ndarray | None
+    targets: np.ndarray | None
+    wpp: int = 0
+    uniforms: np.ndarray | None = None
+    hidden_raw: np.ndarray | None = None
+    W_emit_raw: np.ndarray | None = None
+    W_sum_raw: np.ndarray | None = None
+
+
+def make_workload(name: str, shape: HeadShape, T: int, seed: int, *, target_kind: str | None = "uniform",
+                  wpp: int = 0, weight_std: float = 0.02, trans_std: float = 1.0) -> Workload:
+    hidden = _normal(seed, 1, (T, shape.d), 1.0)
+    W_emit = _normal(seed, 2, (shape.n, shape.r, shape.v, shape.d), weight_std)
+    W_sum = _normal(seed, 3, (shape.sum_rows, shape.d), weight_std)
+    T_static = None
+    if shape.family == HMM:
+        T_static = _normal(seed, 4, (max(shape.n - 1, 1), shape.r, shape.r), trans_std)[: shape.n - 1]
+    targets = None
+    if target_kind == "uniform":
+        targets = uniform_targets(seed, 5, (T, shape.n), shape.v)
+    elif target_kind == "zipf":
+        targets = zipf_targets(seed, 5, (T, shape.n), shape.v)
+    u = uniforms(seed, 6, (T * wpp, 2 * shape.n)) if wpp > 0 else None
+    wl = Workload(name, shape, T, bf16_round(hidden), bf16_round(W_emit), bf16_round(W_sum), T_static,
+                  targets, wpp, u)
+    if shape.io_dtype == F32:
+        wl.hidden_raw, wl.W_emit_raw, wl.W_sum_raw = hidden, W_emit, W_sum
+    return wl
+
+
+DECODE_CELLS = [(fam, n, P) for fam in (CP, HMM) for n in (8, 16) for P in (1, 8, 64)]
+
+
+def config_workload(idx: int, *, cell: tuple[int, int, int] | None = None, T: int | None = None) -> Workload:
+    """The five named workloads. `T` overrides the number of positions (used for scaled-down captures);
+    for idx 4 `cell` = (family, n, P) picks one cell of the decode sweep."""
+    seed = BASE_SEED + idx
+    if idx == 0:
+        return make_workload("cp_tiny", HeadShape(CP, 4, 8, 256, 256, F32), T or 256, seed,
+                             target_kind="uniform", wpp=1)
+    if idx == 1:
+        return make_workload("cp_train", HeadShape(CP, 8, 16, 320, 4096), T or 8192, seed, target_kind="zipf")
+    if idx == 2:
+        return make_workload("hmm_train", HeadShape(HMM, 8, 32, 320, 4096), T or 8192, seed, target_kind="zipf")
+    if idx == 3:
+        return make_workload("btree_train", HeadShape(BTREE, 16, 32, 256, 3072), T or 4096, seed,
+                             target_kind="uniform", wpp=1)
+    if idx == 4:
+        fam, n, P = cell or (CP, 8, 8)
+        r = 16 if fam == CP else 32
+        cseed = seed + 1000 * (fam * 2 + (n // 8 - 1))   # weights shared by the three P of a (family, n)
+        return make_workload(f"decode_{FAMILY_NAMES[fam]}_n{n}_P{P}", HeadShape(fam, n, r, 320, 4096), T or P,
+                             cseed, target_kind=None, wpp=16)
+    raise ValueError(f"no such config {idx}")
