@@ -1,0 +1,164 @@
+/*
+ * mtpc.h - C ABI of the B200 (sm_100a) MtPC head: the probabilistic-circuit multi-byte prediction head of
+ * "MtPC" (arXiv 2511.11346).
+ *
+ * For every context position the head maps the LLM hidden state h (the paper's e_t) to a circuit over the
+ * next n bytes (Sec. 3.3: phi = softmax(W_ij e_t) for the input units, omega = softmax(R_i e_t) for the sum
+ * units) and then either
+ *   - evaluates the exact joint log-likelihood of n observed bytes (Eq. 1 through Eq. CP / HMM / BTree), or
+ *   - draws n-byte draft windows by ancestral sampling (App. B.2, Algorithm 1) and returns their joint
+ *     log-probability (the quantity Algorithm 3 needs for verification).
+ *
+ * Conventions
+ *   - All indices are 0-based. Window slot i in [0,n), unit k in [0,r), byte b in [0,v).
+ *   - "dev" = device (HBM) pointer, "host" = host pointer. Every device buffer is allocated and owned by the
+ *     caller and must stay valid until the work that uses it has finished on the stream. The library
+ *     allocates no device memory: all scratch lives in the caller's workspace.
+ *   - Calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*) and return without
+ *     waiting, except where stated. A head must not be used from two streams at once: its workspace is shared.
+ *   - Return value: MTPC_OK (0) or a negative MTPC_ERR_* code. Nothing throws or aborts across this ABI and
+ *     the device code never traps: data errors only the device can see (target >= v, uniform outside [0,1),
+ *     a bounded wait that ran out) set bits in a device status word, read with mtpc_get_status, and put
+ *     NaN / -1 in the affected outputs.
+ *   - There is no CPU fallback: without a CUDA device every compute call returns MTPC_ERR_CUDA.
+ */
+#ifndef MTPC_H_
+#define MTPC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mtpc_head mtpc_head; /* opaque; created by mtpc_create_head, freed by mtpc_destroy */
+
+/* Circuit family (Sec. 3.2). The fully factorised head (Eq. FF) is MTPC_CP with r = 1. */
+enum { MTPC_CP = 0, MTPC_HMM = 1, MTPC_BTREE = 2 };
+/* dtype of the hidden states and of the weight buffers handed to the library. Arithmetic is always
+ * bf16 x bf16 -> fp32 on the tensor cores; MTPC_F32 inputs are rounded to bf16 (nearest-even) first. */
+enum { MTPC_F32 = 0, MTPC_BF16 = 1 };
+
+enum {
+  MTPC_OK = 0,
+  MTPC_ERR_NULL = -1,        /* a required pointer is NULL                                            */
+  MTPC_ERR_SHAPE = -2,       /* a size is out of range (T > max_positions, n < 1, ...)                */
+  MTPC_ERR_UNSUPPORTED = -3, /* a valid request this version does not implement (see mtpc_config)     */
+  MTPC_ERR_WORKSPACE = -4,   /* workspace too small or misaligned                                     */
+  MTPC_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed (includes: no device)               */
+  MTPC_ERR_TIMEOUT = -6      /* mtpc_get_status: a device-side bounded wait gave up                   */
+};
+
+/* Bits of the device status word. */
+enum {
+  MTPC_STATUS_BAD_TARGET = 1u,  /* a target >= v was seen; that window's log-prob is NaN               */
+  MTPC_STATUS_BAD_UNIFORM = 2u, /* a uniform outside [0,1) was seen; that draw returned -1             */
+  MTPC_STATUS_TIMEOUT = 4u      /* a bounded barrier wait expired; the outputs of that call are invalid */
+};
+
+typedef struct {
+  int32_t family;              /* MTPC_CP | MTPC_HMM | MTPC_BTREE                                      */
+  int32_t n;                   /* window length. BTREE: a power of two >= 2                            */
+  int32_t r;                   /* units per layer (mixture components / hidden states): a power of two,
+                                  <= 128 for CP, <= 32 for HMM and BTREE                               */
+  int32_t v;                   /* vocabulary: a multiple of 16, <= 512, splittable into equal chunks of
+                                  <= 256 columns that are multiples of 16 (256 and 320 are)            */
+  int32_t d;                   /* hidden size: a multiple of 64                                        */
+  int32_t io_dtype;            /* MTPC_F32 | MTPC_BF16: dtype of hidden, W_emit and W_sum              */
+  int32_t max_positions;       /* upper bound on T (log-prob) and P (draft) per call                   */
+  int32_t max_windows_per_pos; /* upper bound on wpp (>= 1; <= 64)                                     */
+  uint32_t flags;              /* must be 0 (bit 0 is reserved for contextual HMM transitions)         */
+} mtpc_config;
+
+/* Bytes of device workspace a head with this configuration needs (a multiple of 256). */
+int mtpc_workspace_bytes(const mtpc_config* cfg, size_t* out_bytes);
+
+/*
+ * Build a head (Sec. 3.3). Enqueues, on `stream`, the one-off preparation (bf16 rounding of F32 weights into
+ * the workspace; log-softmax of the static HMM transition logits) and encodes the TMA descriptors.
+ *   W_emit   dev [n, r, v, d] io_dtype, row-major: the unembedding tensor W of Sec. 3.3; row ((i*r+k)*v+b).
+ *   W_sum    dev [S*r, d] io_dtype: the sum-unit projection R of Sec. 3.3. CP: S=1, the mixture logits
+ *            (W_mix). HMM: S=1, the initial-state logits (W_init). BTREE: S = 1+(n-2)*r; rows [0,r) are the
+ *            root's weights; for internal node j >= 1 (heap order: root 0, children 2j+1, 2j+2; node
+ *            n/2-1+m owns tokens 2m and 2m+1) row r + (j-1)*r*r + a*r + b is the logit of
+ *            z_j = b given z_parent(j) = a (softmax over b).
+ *   T_static dev [n-1, r, r] fp32, HMM only (else NULL): logit of z_i = b given z_{i-1} = a at
+ *            [i-1, a, b], softmax over b (Eq. HMM with input-independent transitions, App. H).
+ *   workspace dev, 256-byte aligned, >= mtpc_workspace_bytes(cfg); owned by the caller, used by every call
+ *            on this head, and must outlive it. With MTPC_BF16 the head keeps the W_emit / W_sum pointers
+ *            (they must outlive it too); with MTPC_F32 it keeps rounded copies in the workspace.
+ */
+int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_sum, const float* T_static,
+                     void* workspace, size_t workspace_bytes, void* stream, mtpc_head** out);
+
+/*
+ * Window log-likelihood (Eq. 1 evaluated through Eq. CP / Eq. HMM / Eq. BTree):
+ *   out_logprob[t] = log q(x_{t,0..n-1} | h_t), natural log, for t in [0,T).
+ *   hidden  dev [T, d] io_dtype, row-major.
+ *   targets dev [T, n] int32. A negative target marginalises that byte (App. B.1: any subset of the
+ *           variables can be summed out in one pass); a target >= v sets MTPC_STATUS_BAD_TARGET and yields NaN.
+ *   T       0 <= T <= max_positions (T == 0 is a no-op).
+ *   out_logprob dev [T] fp32.
+ * The [T, n, r, v] logit tensor is never written to memory: the GEMM epilogue reduces it on chip.
+ */
+int mtpc_window_logprob(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t T,
+                        float* out_logprob, void* stream);
+
+/*
+ * Draft sampling (App. B.2, Algorithm 1) of wpp windows for each of P positions, then the joint log-prob of
+ * every drafted window (latents summed out), as speculative verification needs (Algorithm 3).
+ *   hidden   dev [P, d] io_dtype.
+ *   uniforms dev [P*wpp, 2n] fp32 in [0,1). Window w = p*wpp + j uses row w: columns 0..n-1 drive the latent
+ *            draws (CP: column 0; HMM: column i for z_i; BTREE: column j for internal node j, column n-1
+ *            unused), column n+i drives the byte of slot i. Every categorical draw is inverse-CDF: the
+ *            smallest index j with u < p_0 + ... + p_j (the last index if rounding leaves none).
+ *   out_bytes   dev [P*wpp, n] int32.
+ *   out_logprob dev [P*wpp] fp32, natural log.
+ *   1 <= wpp <= max_windows_per_pos, 0 <= P <= max_positions.
+ */
+int mtpc_draft_sample(mtpc_head* head, const void* hidden, int32_t P, int32_t wpp, const float* uniforms,
+                      int32_t* out_bytes, float* out_logprob, void* stream);
+
+/*
+ * Host-buffer variants: same results, but hidden / targets / uniforms are HOST pointers (pinned memory for
+ * full copy speed) and the outputs are written to HOST buffers. The copies to and from the device go through
+ * staging areas in the workspace on `stream`; the call returns after the stream has been synchronised, so
+ * the outputs are ready on return.
+ */
+int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int32_t* targets_host, int32_t T,
+                             float* out_logprob_host, void* stream);
+int mtpc_draft_sample_host(mtpc_head* head, const void* hidden_host, int32_t P, int32_t wpp,
+                           const float* uniforms_host, int32_t* out_bytes_host, float* out_logprob_host,
+                           void* stream);
+
+/*
+ * Read and clear the device status word. Synchronises `stream` first. *out_flags receives the MTPC_STATUS_*
+ * bits; returns MTPC_ERR_TIMEOUT if MTPC_STATUS_TIMEOUT is set, MTPC_ERR_CUDA on a CUDA error, else MTPC_OK.
+ */
+int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags);
+
+/*
+ * Per-kernel device timing of the most recent call (CUDA events recorded on the call's stream around each
+ * launch). Off by default. mtpc_get_timing synchronises on the events and writes up to `capacity` phase
+ * durations in milliseconds, *out_count = number of phases of the last call:
+ *   mtpc_window_logprob: [0] projection GEMM + fused epilogue, [1] circuit evaluation.
+ *   mtpc_draft_sample:   [0] sum-unit GEMM, [1] latent sampling, [2] GEMM + inverse-CDF epilogue,
+ *                        [3] GEMM + gather epilogue on the drafted bytes, [4] circuit evaluation.
+ */
+int mtpc_set_timing(mtpc_head* head, int32_t enabled);
+int mtpc_get_timing(mtpc_head* head, float* out_ms, int32_t capacity, int32_t* out_count);
+
+/* Number of kernels the library launched on behalf of this head since creation (preparation included). */
+int mtpc_launch_count(mtpc_head* head, uint64_t* out_count);
+
+/* Frees the host-side object (the workspace and the weights stay the caller's). Synchronises nothing. */
+int mtpc_destroy(mtpc_head* head);
+
+/* Static, NUL-terminated description of a return code. */
+const char* mtpc_status_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MTPC_H_ */

@@ -1,0 +1,166 @@
+"""ctypes binding of libmtpc.so with the same names as the C ABI (include/mtpc.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels. PyTorch appears here
+solely as the owner of device memory and streams. There is no fallback: if the library is missing or cannot
+be loaded, importing a symbol from it raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+from . import build as _build
+
+MTPC_CP, MTPC_HMM, MTPC_BTREE = 0, 1, 2
+MTPC_F32, MTPC_BF16 = 0, 1
+MTPC_OK = 0
+STATUS_BAD_TARGET, STATUS_BAD_UNIFORM, STATUS_TIMEOUT = 1, 2, 4
+
+EXPORTS = [
+    "mtpc_workspace_bytes", "mtpc_create_head", "mtpc_window_logprob", "mtpc_draft_sample",
+    "mtpc_window_logprob_host", "mtpc_draft_sample_host", "mtpc_get_status", "mtpc_set_timing", "mtpc_get_timing",
+    "mtpc_launch_count", "mtpc_destroy", "mtpc_status_string",
+]
+
+
+class MtpcConfig(ctypes.Structure):
+    _fields_ = [("family", ctypes.c_int32), ("n", ctypes.c_int32), ("r", ctypes.c_int32), ("v", ctypes.c_int32),
+                ("d", ctypes.c_int32), ("io_dtype", ctypes.c_int32), ("max_positions", ctypes.c_int32),
+                ("max_windows_per_pos", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class MtpcError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {status_string(code)} ({code})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load (building first if the sources are newer) the CUDA library. Raises if that is impossible."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if _build.is_stale():
+        path = _build.build()
+    L = ctypes.CDLL(path)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+    L.mtpc_workspace_bytes.argtypes = [ctypes.POINTER(MtpcConfig), ctypes.POINTER(sz)]
+    L.mtpc_create_head.argtypes = [ctypes.POINTER(MtpcConfig), vp, vp, vp, vp, sz, vp, ctypes.POINTER(vp)]
+    L.mtpc_window_logprob.argtypes = [vp, vp, vp, i32, vp, vp]
+    L.mtpc_draft_sample.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    L.mtpc_window_logprob_host.argtypes = [vp, vp, vp, i32, vp, vp]
+    L.mtpc_draft_sample_host.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    L.mtpc_get_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    L.mtpc_set_timing.argtypes = [vp, i32]
+    L.mtpc_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), i32, ctypes.POINTER(i32)]
+    L.mtpc_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
+    L.mtpc_destroy.argtypes = [vp]
+    L.mtpc_status_string.argtypes = [ctypes.c_int]
+    L.mtpc_status_string.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name != "mtpc_status_string":
+            getattr(L, name).restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+def status_string(code: int) -> str:
+    return lib().mtpc_status_string(code).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != MTPC_OK:
+        raise MtpcError(code, what)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def mtpc_workspace_bytes(cfg: MtpcConfig) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().mtpc_workspace_bytes(ctypes.byref(cfg), ctypes.byref(out)), "mtpc_workspace_bytes")
+    return out.value
+
+
+class MtpcHead:
+    """Owns the opaque head handle and keeps the tensors the head points into alive."""
+
+    def __init__(self, family: int, n: int, r: int, v: int, d: int, io_dtype: int, max_positions: int,
+                 max_windows_per_pos: int, W_emit, W_sum, T_static=None, stream=None):
+        import torch
+        self.cfg = MtpcConfig(family, n, r, v, d, io_dtype, max_positions, max_windows_per_pos, 0)
+        nbytes = mtpc_workspace_bytes(self.cfg)
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=W_emit.device)
+        self._keep = (W_emit, W_sum, T_static)
+        handle = ctypes.c_void_p(0)
+        _check(lib().mtpc_create_head(ctypes.byref(self.cfg), _ptr(W_emit), _ptr(W_sum), _ptr(T_static),
+                                      self.workspace.data_ptr(), nbytes, _stream(stream), ctypes.byref(handle)),
+               "mtpc_create_head")
+        self.handle = handle
+
+    # -- device-buffer calls
+    def mtpc_window_logprob(self, hidden, targets, out_logprob, stream=None) -> None:
+        T = hidden.shape[0]
+        _check(lib().mtpc_window_logprob(self.handle, _ptr(hidden), _ptr(targets), T, _ptr(out_logprob),
+                                         _stream(stream)), "mtpc_window_logprob")
+
+    def mtpc_draft_sample(self, hidden, wpp: int, uniforms, out_bytes, out_logprob, stream=None) -> None:
+        P = hidden.shape[0]
+        _check(lib().mtpc_draft_sample(self.handle, _ptr(hidden), P, wpp, _ptr(uniforms), _ptr(out_bytes),
+                                       _ptr(out_logprob), _stream(stream)), "mtpc_draft_sample")
+
+    # -- host-buffer calls (copies inside; outputs ready on return)
+    def mtpc_window_logprob_host(self, hidden_host, targets_host, out_logprob_host, stream=None) -> None:
+        T = hidden_host.shape[0]
+        _check(lib().mtpc_window_logprob_host(self.handle, _ptr(hidden_host), _ptr(targets_host), T,
+                                              _ptr(out_logprob_host), _stream(stream)), "mtpc_window_logprob_host")
+
+    def mtpc_draft_sample_host(self, hidden_host, wpp: int, uniforms_host, out_bytes_host, out_logprob_host,
+                               stream=None) -> None:
+        P = hidden_host.shape[0]
+        _check(lib().mtpc_draft_sample_host(self.handle, _ptr(hidden_host), P, wpp, _ptr(uniforms_host),
+                                            _ptr(out_bytes_host), _ptr(out_logprob_host), _stream(stream)),
+               "mtpc_draft_sample_host")
+
+    def mtpc_get_status(self, stream=None) -> int:
+        flags = ctypes.c_uint32(0)
+        code = lib().mtpc_get_status(self.handle, _stream(stream), ctypes.byref(flags))
+        if code not in (MTPC_OK, -6):
+            raise MtpcError(code, "mtpc_get_status")
+        return flags.value
+
+    def mtpc_set_timing(self, enabled: bool) -> None:
+        _check(lib().mtpc_set_timing(self.handle, 1 if enabled else 0), "mtpc_set_timing")
+
+    def mtpc_get_timing(self) -> list[float]:
+        buf = (ctypes.c_float * 8)()
+        cnt = ctypes.c_int32(0)
+        _check(lib().mtpc_get_timing(self.handle, buf, 8, ctypes.byref(cnt)), "mtpc_get_timing")
+        return [buf[i] for i in range(cnt.value)]
+
+    def mtpc_launch_count(self) -> int:
+        out = ctypes.c_uint64(0)
+        _check(lib().mtpc_launch_count(self.handle, ctypes.byref(out)), "mtpc_launch_count")
+        return out.value
+
+    def mtpc_destroy(self) -> None:
+        if self.handle:
+            lib().mtpc_destroy(self.handle)
+            self.handle = ctypes.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.mtpc_destroy()
+        except Exception:
+            pass

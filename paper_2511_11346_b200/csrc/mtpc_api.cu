@@ -1,0 +1,520 @@
+// Host side of the C ABI declared in include/mtpc.h: argument checks, workspace carving, TMA descriptor
+// encoding and kernel launches. Every step of the path runs in the kernels of this library; there is no CPU
+// or library fallback.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/mtpc.h"
+#include "mtpc_circuit.cuh"
+#include "mtpc_gemm.cuh"
+
+namespace {
+
+using namespace mtpc;
+
+constexpr size_t kAlign = 256;
+constexpr int kMaxPhases = 5;
+constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA on sm_100
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
+struct Layout {
+  // derived sizes
+  int S, sum_rows, chunk_cols, chunks_per_unit, sum_cols, sum_tiles, slot_stride, num_slots, stages, stage_bytes;
+  size_t max_windows;
+  // workspace offsets (bytes)
+  size_t off_status, off_wemit, off_wsum, off_hidden, off_logA, off_G, off_logw, off_sel;
+  size_t off_h_hidden, off_h_targets, off_h_uniforms, off_h_bytes, off_h_out;
+  size_t total;
+};
+
+int plan(const mtpc_config& c, Layout* L) {
+  if (c.family < MTPC_CP || c.family > MTPC_BTREE) return MTPC_ERR_SHAPE;
+  if (c.io_dtype != MTPC_F32 && c.io_dtype != MTPC_BF16) return MTPC_ERR_SHAPE;
+  if (c.n < 1 || c.r < 1 || c.v < 1 || c.d < 1 || c.max_positions < 1 || c.max_windows_per_pos < 1)
+    return MTPC_ERR_SHAPE;
+  if (c.flags != 0) return MTPC_ERR_UNSUPPORTED;
+  if (c.n > 64 || c.max_windows_per_pos > 64) return MTPC_ERR_UNSUPPORTED;
+  if (!is_pow2(c.r) || c.r > 128) return MTPC_ERR_UNSUPPORTED;
+  if (c.family != MTPC_CP && c.r > 32) return MTPC_ERR_UNSUPPORTED;
+  if (c.family == MTPC_BTREE && (c.n < 2 || !is_pow2(c.n))) return MTPC_ERR_UNSUPPORTED;
+  if (c.d % kBlockK != 0) return MTPC_ERR_UNSUPPORTED;
+  if (c.v % 16 != 0 || c.v > 512) return MTPC_ERR_UNSUPPORTED;
+  if (static_cast<int64_t>(c.n) * c.r * c.v > (1ll << 30)) return MTPC_ERR_SHAPE;
+
+  L->S = (c.family == MTPC_BTREE) ? 1 + (c.n - 2) * c.r : 1;
+  L->sum_rows = L->S * c.r;
+  // emission unit -> equal chunks of <= 256 columns, each a multiple of 16
+  int chunks = (c.v + 255) / 256;
+  while (c.v % chunks != 0 || (c.v / chunks) % 16 != 0) ++chunks;
+  L->chunks_per_unit = chunks;
+  L->chunk_cols = c.v / chunks;
+  // sum tile: a multiple of both r and 16, at most 256 columns
+  const int unit = c.r > 16 ? c.r : 16;
+  int sum_cols = (L->sum_rows + unit - 1) / unit * unit;
+  if (sum_cols > 256) sum_cols = 256 / unit * unit;
+  L->sum_cols = sum_cols;
+  L->sum_tiles = (L->sum_rows + sum_cols - 1) / sum_cols;
+  int widest = L->chunk_cols > sum_cols ? L->chunk_cols : sum_cols;
+  L->slot_stride = (widest + 31) / 32 * 32;
+  L->num_slots = kTmemCols / L->slot_stride;
+  if (L->num_slots > kMaxSlots) L->num_slots = kMaxSlots;
+  if (L->num_slots < chunks) return MTPC_ERR_UNSUPPORTED;
+  const int brows = chunks * L->chunk_cols > sum_cols ? chunks * L->chunk_cols : sum_cols;
+  L->stage_bytes = kABytes + brows * kBlockK * 2;          // multiples of 1024 (rows are multiples of 16)
+  L->stage_bytes = (L->stage_bytes + 1023) / 1024 * 1024;
+  int stages = (kSmemLimit - 1024 - static_cast<int>(sizeof(GemmControl))) / L->stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) return MTPC_ERR_UNSUPPORTED;
+  L->stages = stages;
+
+  L->max_windows = static_cast<size_t>(c.max_positions) * c.max_windows_per_pos;
+  const size_t elt = c.io_dtype == MTPC_F32 ? 4 : 2;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  L->off_status = take(256);
+  const bool f32 = c.io_dtype == MTPC_F32;
+  L->off_wemit = take(f32 ? static_cast<size_t>(c.n) * c.r * c.v * c.d * 2 : 0);
+  L->off_wsum = take(f32 ? static_cast<size_t>(L->sum_rows) * c.d * 2 : 0);
+  L->off_hidden = take(f32 ? static_cast<size_t>(c.max_positions) * c.d * 2 : 0);
+  L->off_logA = take(c.family == MTPC_HMM ? static_cast<size_t>(c.n - 1) * c.r * c.r * 4 : 0);
+  L->off_G = take(L->max_windows * c.n * c.r * 4);
+  L->off_logw = take(static_cast<size_t>(c.max_positions) * L->sum_rows * 4);
+  L->off_sel = take(L->max_windows * c.n * 4);
+  L->off_h_hidden = take(static_cast<size_t>(c.max_positions) * c.d * elt);
+  L->off_h_targets = take(static_cast<size_t>(c.max_positions) * c.n * 4);
+  L->off_h_uniforms = take(L->max_windows * 2 * c.n * 4);
+  L->off_h_bytes = take(L->max_windows * c.n * 4);
+  L->off_h_out = take(L->max_windows * 4);
+  L->total = off;
+  return MTPC_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows, cols] row-major -> tiles of box_rows x 64 elements, 128-byte swizzle, zero fill outside.
+int make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return MTPC_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0) return MTPC_ERR_WORKSPACE;
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstride[1] = {cols * 2};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MTPC_OK : MTPC_ERR_CUDA;
+}
+
+}  // namespace
+
+struct mtpc_head {
+  mtpc_config cfg;
+  Layout L;
+  uint8_t* ws;
+  const void* W_emit_bf16;
+  const void* W_sum_bf16;
+  CUtensorMap tm_emit, tm_sum;
+  int num_sms;
+  int gemm_smem;
+  bool timing;
+  cudaEvent_t ev[2 * kMaxPhases];
+  bool ev_ready;
+  int last_phases;
+  uint64_t launches;
+};
+
+namespace {
+
+template <typename T>
+T* at(mtpc_head* h, size_t off) { return reinterpret_cast<T*>(h->ws + off); }
+
+struct PhaseTimer {
+  mtpc_head* h;
+  cudaStream_t st;
+  int idx;
+  PhaseTimer(mtpc_head* head, cudaStream_t s) : h(head), st(s), idx(0) { h->last_phases = 0; }
+  void begin() { if (h->timing && idx < kMaxPhases) cudaEventRecord(h->ev[2 * idx], st); }
+  void end() {
+    if (h->timing && idx < kMaxPhases) cudaEventRecord(h->ev[2 * idx + 1], st);
+    ++idx;
+    h->last_phases = idx;
+  }
+};
+
+int check_launch() { return cudaGetLastError() == cudaSuccess ? MTPC_OK : MTPC_ERR_CUDA; }
+
+// Launch the projection kernel over units [unit_begin, unit_begin + unit_count) for `rows` positions.
+int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int wpp, int unit_begin, int unit_count,
+                const int* targets, const float* uniforms, int* out_bytes, cudaStream_t st) {
+  if (rows <= 0 || unit_count <= 0) return MTPC_OK;
+  const mtpc_config& c = h->cfg;
+  const Layout& L = h->L;
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  int rc = make_tmap(&p.tm_a, hidden_bf16, static_cast<uint64_t>(rows), static_cast<uint64_t>(c.d), kBlockM);
+  if (rc != MTPC_OK) return rc;
+  p.tm_emit = h->tm_emit;
+  p.tm_sum = h->tm_sum;
+  p.T = rows;
+  p.m_tiles = (rows + kBlockM - 1) / kBlockM;
+  p.kblocks = c.d / kBlockK;
+  p.n = c.n; p.r = c.r; p.v = c.v;
+  p.emit_units = c.n * c.r;
+  p.unit_begin = unit_begin;
+  p.unit_count = unit_count;
+  p.chunk_cols = L.chunk_cols;
+  p.chunks_per_unit = L.chunks_per_unit;
+  p.sum_cols = L.sum_cols;
+  p.sum_rows = L.sum_rows;
+  p.slot_stride = L.slot_stride;
+  p.num_slots = L.num_slots;
+  p.stages = L.stages;
+  p.stage_bytes = L.stage_bytes;
+  p.wpp = wpp;
+  p.targets = targets;
+  p.G = at<float>(h, L.off_G);
+  p.logw = at<float>(h, L.off_logw);
+  p.unit_sel = at<int>(h, L.off_sel);
+  p.uniforms = uniforms;
+  p.out_bytes = out_bytes;
+  p.status = at<unsigned>(h, L.off_status);
+  const long long tiles = static_cast<long long>(p.m_tiles) * unit_count;
+  const int grid = static_cast<int>(tiles < h->num_sms ? tiles : h->num_sms);
+  if (mode == kModeLogprob)
+    mtpc_gemm_kernel<kModeLogprob><<<grid, kGemmThreads, h->gemm_smem, st>>>(p);
+  else
+    mtpc_gemm_kernel<kModeSample><<<grid, kGemmThreads, h->gemm_smem, st>>>(p);
+  h->launches++;
+  return check_launch();
+}
+
+int launch_circuit(mtpc_head* h, int W, int wpp, float* out, cudaStream_t st) {
+  if (W <= 0) return MTPC_OK;
+  const mtpc_config& c = h->cfg;
+  const Layout& L = h->L;
+  const float* G = at<float>(h, L.off_G);
+  const float* logw = at<float>(h, L.off_logw);
+  const int blocks = (W + kCircuitWarps - 1) / kCircuitWarps;
+  const int threads = kCircuitWarps * 32;
+  if (c.family == MTPC_CP) {
+    circuit_cp_kernel<<<blocks, threads, 0, st>>>(G, logw, out, W, wpp, c.n, c.r, L.sum_rows);
+  } else if (c.family == MTPC_HMM) {
+    circuit_hmm_kernel<<<blocks, threads, 0, st>>>(G, logw, at<float>(h, L.off_logA), out, W, wpp, c.n, c.r,
+                                                   L.sum_rows);
+  } else {
+    const size_t smem = static_cast<size_t>(kCircuitWarps) * ((c.n - 1) * c.r + c.r * (c.r + 1)) * 4;
+    circuit_btree_kernel<<<blocks, threads, smem, st>>>(G, logw, out, W, wpp, c.n, c.r, L.sum_rows);
+  }
+  h->launches++;
+  return check_launch();
+}
+
+// hidden (io_dtype, device) -> bf16 device pointer the GEMM reads
+int stage_hidden(mtpc_head* h, const void* hidden, int rows, const void** out_bf16, cudaStream_t st) {
+  if (h->cfg.io_dtype == MTPC_BF16) { *out_bf16 = hidden; return MTPC_OK; }
+  __nv_bfloat16* dst = at<__nv_bfloat16>(h, h->L.off_hidden);
+  const size_t count = static_cast<size_t>(rows) * h->cfg.d;
+  if (count) {
+    const int blocks = static_cast<int>((count + 255) / 256 < 4096 ? (count + 255) / 256 : 4096);
+    f32_to_bf16_kernel<<<blocks, 256, 0, st>>>(static_cast<const float*>(hidden), dst, count);
+    h->launches++;
+    if (check_launch() != MTPC_OK) return MTPC_ERR_CUDA;
+  }
+  *out_bf16 = dst;
+  return MTPC_OK;
+}
+
+int window_logprob_impl(mtpc_head* h, const void* hidden, const int32_t* targets, int32_t T, float* out,
+                        cudaStream_t st) {
+  const void* hb = nullptr;
+  int rc = stage_hidden(h, hidden, T, &hb, st);
+  if (rc != MTPC_OK) return rc;
+  PhaseTimer pt(h, st);
+  pt.begin();
+  rc = launch_gemm(h, kModeLogprob, hb, T, 1, 0, h->cfg.n * h->cfg.r + h->L.sum_tiles, targets, nullptr, nullptr, st);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  pt.begin();
+  rc = launch_circuit(h, T, 1, out, st);
+  pt.end();
+  return rc;
+}
+
+int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, const float* uniforms,
+                      int32_t* out_bytes, float* out_logprob, cudaStream_t st) {
+  const mtpc_config& c = h->cfg;
+  const Layout& L = h->L;
+  const int W = P * wpp;
+  const void* hb = nullptr;
+  int rc = stage_hidden(h, hidden, P, &hb, st);
+  if (rc != MTPC_OK) return rc;
+  const int emit_units = c.n * c.r;
+  PhaseTimer pt(h, st);
+  // 1. sum-unit weights (Sec. 3.3) -> 2. latent draws at the sum units (Algorithm 1)
+  pt.begin();
+  rc = launch_gemm(h, kModeLogprob, hb, P, 1, emit_units, L.sum_tiles, nullptr, nullptr, nullptr, st);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  pt.begin();
+  latent_sample_kernel<<<(W + 127) / 128, 128, 0, st>>>(c.family, at<float>(h, L.off_logw), at<float>(h, L.off_logA),
+                                                        uniforms, at<int>(h, L.off_sel), out_bytes,
+                                                        at<unsigned>(h, L.off_status), W, wpp, c.n, c.r, L.sum_rows);
+  h->launches++;
+  pt.end();
+  if ((rc = check_launch()) != MTPC_OK) return rc;
+  // 3. byte draws at the selected input units
+  pt.begin();
+  rc = launch_gemm(h, kModeSample, hb, P, wpp, 0, emit_units, nullptr, uniforms, out_bytes, st);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  // 4. evidence of the drafted bytes under every unit -> 5. joint log-prob with the latents summed out
+  pt.begin();
+  rc = launch_gemm(h, kModeLogprob, hb, P, wpp, 0, emit_units, out_bytes, nullptr, nullptr, st);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  pt.begin();
+  rc = launch_circuit(h, W, wpp, out_logprob, st);
+  pt.end();
+  return rc;
+}
+
+int check_call(mtpc_head* h, int32_t rows) {
+  if (!h) return MTPC_ERR_NULL;
+  if (rows < 0 || rows > h->cfg.max_positions) return MTPC_ERR_SHAPE;
+  return MTPC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mtpc_workspace_bytes(const mtpc_config* cfg, size_t* out_bytes) {
+  if (!cfg || !out_bytes) return MTPC_ERR_NULL;
+  Layout L;
+  int rc = plan(*cfg, &L);
+  if (rc != MTPC_OK) return rc;
+  *out_bytes = L.total;
+  return MTPC_OK;
+}
+
+int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_sum, const float* T_static,
+                     void* workspace, size_t workspace_bytes, void* stream, mtpc_head** out) {
+  if (!cfg || !W_emit || !W_sum || !workspace || !out) return MTPC_ERR_NULL;
+  *out = nullptr;
+  Layout L;
+  int rc = plan(*cfg, &L);
+  if (rc != MTPC_OK) return rc;
+  if (cfg->family == MTPC_HMM && cfg->n > 1 && !T_static) return MTPC_ERR_NULL;
+  if (workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0) return MTPC_ERR_WORKSPACE;
+  int dev = 0, cc_major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MTPC_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || cc_major != 10)
+    return MTPC_ERR_CUDA;   // tcgen05 / TMEM code: sm_100 only
+  mtpc_head* h = new (std::nothrow) mtpc_head;
+  if (!h) return MTPC_ERR_CUDA;
+  memset(h, 0, sizeof(*h));
+  h->cfg = *cfg;
+  h->L = L;
+  h->ws = static_cast<uint8_t*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bool fail = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess;
+  h->gemm_smem = L.stages * L.stage_bytes + 1024 + static_cast<int>(sizeof(GemmControl));
+  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               h->gemm_smem) != cudaSuccess;
+  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeSample>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               h->gemm_smem) != cudaSuccess;
+  if (cfg->family == MTPC_BTREE) {
+    const int smem = kCircuitWarps * ((cfg->n - 1) * cfg->r + cfg->r * (cfg->r + 1)) * 4;
+    if (smem > 48 * 1024)
+      fail |= cudaFuncSetAttribute(circuit_btree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+              cudaSuccess;
+  }
+  fail |= cudaMemsetAsync(h->ws + L.off_status, 0, 256, st) != cudaSuccess;
+  if (fail) { delete h; return MTPC_ERR_CUDA; }
+
+  const size_t emit_count = static_cast<size_t>(cfg->n) * cfg->r * cfg->v * cfg->d;
+  const size_t sum_count = static_cast<size_t>(L.sum_rows) * cfg->d;
+  if (cfg->io_dtype == MTPC_F32) {
+    f32_to_bf16_kernel<<<2048, 256, 0, st>>>(static_cast<const float*>(W_emit), at<__nv_bfloat16>(h, L.off_wemit),
+                                             emit_count);
+    f32_to_bf16_kernel<<<256, 256, 0, st>>>(static_cast<const float*>(W_sum), at<__nv_bfloat16>(h, L.off_wsum),
+                                            sum_count);
+    h->launches += 2;
+    h->W_emit_bf16 = h->ws + L.off_wemit;
+    h->W_sum_bf16 = h->ws + L.off_wsum;
+  } else {
+    h->W_emit_bf16 = W_emit;
+    h->W_sum_bf16 = W_sum;
+  }
+  if (cfg->family == MTPC_HMM && cfg->n > 1) {
+    const int rows = (cfg->n - 1) * cfg->r;
+    log_softmax_rows_kernel<<<(rows + 127) / 128, 128, 0, st>>>(T_static, at<float>(h, L.off_logA), rows, cfg->r);
+    h->launches++;
+  }
+  if (check_launch() != MTPC_OK) { delete h; return MTPC_ERR_CUDA; }
+  rc = make_tmap(&h->tm_emit, h->W_emit_bf16, static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v, cfg->d, L.chunk_cols);
+  if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols);
+  if (rc != MTPC_OK) { delete h; return rc; }
+  *out = h;
+  return MTPC_OK;
+}
+
+int mtpc_window_logprob(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t T, float* out_logprob,
+                        void* stream) {
+  int rc = check_call(head, T);
+  if (rc != MTPC_OK) return rc;
+  if (T == 0) return MTPC_OK;
+  if (!hidden || !targets || !out_logprob) return MTPC_ERR_NULL;
+  return window_logprob_impl(head, hidden, targets, T, out_logprob, static_cast<cudaStream_t>(stream));
+}
+
+int mtpc_draft_sample(mtpc_head* head, const void* hidden, int32_t P, int32_t wpp, const float* uniforms,
+                      int32_t* out_bytes, float* out_logprob, void* stream) {
+  int rc = check_call(head, P);
+  if (rc != MTPC_OK) return rc;
+  if (wpp < 1 || wpp > head->cfg.max_windows_per_pos) return MTPC_ERR_SHAPE;
+  if (P == 0) return MTPC_OK;
+  if (!hidden || !uniforms || !out_bytes || !out_logprob) return MTPC_ERR_NULL;
+  return draft_sample_impl(head, hidden, P, wpp, uniforms, out_bytes, out_logprob, static_cast<cudaStream_t>(stream));
+}
+
+int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int32_t* targets_host, int32_t T,
+                             float* out_logprob_host, void* stream) {
+  int rc = check_call(head, T);
+  if (rc != MTPC_OK) return rc;
+  if (T == 0) return MTPC_OK;
+  if (!hidden_host || !targets_host || !out_logprob_host) return MTPC_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Layout& L = head->L;
+  const size_t elt = head->cfg.io_dtype == MTPC_F32 ? 4 : 2;
+  void* dh = head->ws + L.off_h_hidden;
+  int32_t* dt = at<int32_t>(head, L.off_h_targets);
+  float* dout = at<float>(head, L.off_h_out);
+  bool fail = cudaMemcpyAsync(dh, hidden_host, static_cast<size_t>(T) * head->cfg.d * elt, cudaMemcpyHostToDevice, st) !=
+              cudaSuccess;
+  fail |= cudaMemcpyAsync(dt, targets_host, static_cast<size_t>(T) * head->cfg.n * 4, cudaMemcpyHostToDevice, st) !=
+          cudaSuccess;
+  if (fail) return MTPC_ERR_CUDA;
+  rc = window_logprob_impl(head, dh, dt, T, dout, st);
+  if (rc != MTPC_OK) return rc;
+  fail = cudaMemcpyAsync(out_logprob_host, dout, static_cast<size_t>(T) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess;
+  fail |= cudaStreamSynchronize(st) != cudaSuccess;
+  return fail ? MTPC_ERR_CUDA : MTPC_OK;
+}
+
+int mtpc_draft_sample_host(mtpc_head* head, const void* hidden_host, int32_t P, int32_t wpp,
+                           const float* uniforms_host, int32_t* out_bytes_host, float* out_logprob_host,
+                           void* stream) {
+  int rc = check_call(head, P);
+  if (rc != MTPC_OK) return rc;
+  if (wpp < 1 || wpp > head->cfg.max_windows_per_pos) return MTPC_ERR_SHAPE;
+  if (P == 0) return MTPC_OK;
+  if (!hidden_host || !uniforms_host || !out_bytes_host || !out_logprob_host) return MTPC_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Layout& L = head->L;
+  const mtpc_config& c = head->cfg;
+  const size_t elt = c.io_dtype == MTPC_F32 ? 4 : 2;
+  const size_t W = static_cast<size_t>(P) * wpp;
+  void* dh = head->ws + L.off_h_hidden;
+  float* du = at<float>(head, L.off_h_uniforms);
+  int32_t* db = at<int32_t>(head, L.off_h_bytes);
+  float* dout = at<float>(head, L.off_h_out);
+  bool fail = cudaMemcpyAsync(dh, hidden_host, static_cast<size_t>(P) * c.d * elt, cudaMemcpyHostToDevice, st) !=
+              cudaSuccess;
+  fail |= cudaMemcpyAsync(du, uniforms_host, W * 2 * c.n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess;
+  if (fail) return MTPC_ERR_CUDA;
+  rc = draft_sample_impl(head, dh, P, wpp, du, db, dout, st);
+  if (rc != MTPC_OK) return rc;
+  fail = cudaMemcpyAsync(out_bytes_host, db, W * c.n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess;
+  fail |= cudaMemcpyAsync(out_logprob_host, dout, W * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess;
+  fail |= cudaStreamSynchronize(st) != cudaSuccess;
+  return fail ? MTPC_ERR_CUDA : MTPC_OK;
+}
+
+int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags) {
+  if (!head || !out_flags) return MTPC_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t flags = 0;
+  void* dev = head->ws + head->L.off_status;
+  if (cudaMemcpyAsync(&flags, dev, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MTPC_ERR_CUDA;
+  if (cudaMemsetAsync(dev, 0, 4, st) != cudaSuccess) return MTPC_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MTPC_ERR_CUDA;
+  *out_flags = flags;
+  return (flags & MTPC_STATUS_TIMEOUT) ? MTPC_ERR_TIMEOUT : MTPC_OK;
+}
+
+int mtpc_set_timing(mtpc_head* head, int32_t enabled) {
+  if (!head) return MTPC_ERR_NULL;
+  if (enabled && !head->ev_ready) {
+    for (int i = 0; i < 2 * kMaxPhases; ++i)
+      if (cudaEventCreate(&head->ev[i]) != cudaSuccess) return MTPC_ERR_CUDA;
+    head->ev_ready = true;
+  }
+  head->timing = enabled != 0;
+  head->last_phases = 0;
+  return MTPC_OK;
+}
+
+int mtpc_get_timing(mtpc_head* head, float* out_ms, int32_t capacity, int32_t* out_count) {
+  if (!head || !out_ms || !out_count) return MTPC_ERR_NULL;
+  *out_count = 0;
+  if (!head->timing) return MTPC_OK;
+  const int nph = head->last_phases < kMaxPhases ? head->last_phases : kMaxPhases;
+  for (int i = 0; i < nph && i < capacity; ++i) {
+    if (cudaEventSynchronize(head->ev[2 * i + 1]) != cudaSuccess) return MTPC_ERR_CUDA;
+    if (cudaEventElapsedTime(&out_ms[i], head->ev[2 * i], head->ev[2 * i + 1]) != cudaSuccess) return MTPC_ERR_CUDA;
+    *out_count = i + 1;
+  }
+  return MTPC_OK;
+}
+
+int mtpc_launch_count(mtpc_head* head, uint64_t* out_count) {
+  if (!head || !out_count) return MTPC_ERR_NULL;
+  *out_count = head->launches;
+  return MTPC_OK;
+}
+
+int mtpc_destroy(mtpc_head* head) {
+  if (!head) return MTPC_ERR_NULL;
+  if (head->ev_ready)
+    for (int i = 0; i < 2 * kMaxPhases; ++i) cudaEventDestroy(head->ev[i]);
+  delete head;
+  return MTPC_OK;
+}
+
+const char* mtpc_status_string(int code) {
+  switch (code) {
+    case MTPC_OK: return "ok";
+    case MTPC_ERR_NULL: return "a required pointer is NULL";
+    case MTPC_ERR_SHAPE: return "a size argument is out of range";
+    case MTPC_ERR_UNSUPPORTED: return "configuration not supported by this version";
+    case MTPC_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case MTPC_ERR_CUDA: return "a CUDA call failed (no sm_100 device, launch error, or driver entry point missing)";
+    case MTPC_ERR_TIMEOUT: return "a device-side bounded wait expired";
+    default: return "unknown status code";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,207 @@
+// Circuit evaluation in log space (Eq. CP, Eq. HMM, Eq. BTree), latent ancestral sampling (Algorithm 1, sum
+// units) and the small preparation kernels. One warp evaluates one window; lane = latent value.
+#pragma once
+#include <cuda_bf16.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+namespace mtpc {
+
+constexpr int kCircuitWarps = 8;
+constexpr unsigned kFull = 0xffffffffu;
+
+// (m, s) represents log-sum-exp = m + log s. Merging tolerates empty operands (m = -inf, s = 0).
+__device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2) {
+  const float mn = fmaxf(m, m2);
+  if (mn == -CUDART_INF_F) { m = mn; s = 0.f; return; }
+  s = s * __expf(m - mn) + s2 * __expf(m2 - mn);
+  m = mn;
+}
+__device__ __forceinline__ float warp_lse(float val, bool has) {
+  float m = has ? val : -CUDART_INF_F;
+  float s = has ? 1.f : 0.f;
+  if (has && val != val) { m = 0.f; s = val; }   // NaN must survive the max
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float m2 = __shfl_xor_sync(kFull, m, off);
+    const float s2 = __shfl_xor_sync(kFull, s, off);
+    lse_merge(m, s, m2, s2);
+  }
+  return m + __logf(s);
+}
+
+// Eq. (CP): out[w] = LSE_k( log omega[p, k] + sum_i G[w, i, k] ),  p = w / wpp.
+__global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __restrict__ logw,
+                                  float* __restrict__ out, int W, int wpp, int n, int r, int sum_rows) {
+  const int w = blockIdx.x * kCircuitWarps + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (w >= W) return;
+  const float* g = G + static_cast<size_t>(w) * n * r;
+  const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
+  float m = -CUDART_INF_F, s = 0.f;
+  for (int k = lane; k < r; k += 32) {
+    float a = lw[k];
+    for (int i = 0; i < n; ++i) a += g[i * r + k];
+    if (a != a) { m = 0.f; s = a; continue; }
+    lse_merge(m, s, a, 1.f);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float m2 = __shfl_xor_sync(kFull, m, off);
+    const float s2 = __shfl_xor_sync(kFull, s, off);
+    lse_merge(m, s, m2, s2);
+  }
+  if (lane == 0) out[w] = m + __logf(s);
+}
+
+// Eq. (HMM), forward recursion over the window: alpha_0[k] = log pi[k] + G[0,k];
+// alpha_i[k] = G[i,k] + LSE_a(alpha_{i-1}[a] + logA[i-1][a][k]); out = LSE_k alpha_{n-1}[k].  r <= 32.
+__global__ void circuit_hmm_kernel(const float* __restrict__ G, const float* __restrict__ logw,
+                                   const float* __restrict__ logA, float* __restrict__ out, int W, int wpp, int n,
+                                   int r, int sum_rows) {
+  const int w = blockIdx.x * kCircuitWarps + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (w >= W) return;
+  const float* g = G + static_cast<size_t>(w) * n * r;
+  const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
+  const bool has = lane < r;
+  float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
+  for (int i = 1; i < n; ++i) {
+    const float* A = logA + static_cast<size_t>(i - 1) * r * r;
+    float m = -CUDART_INF_F;
+    for (int a = 0; a < r; ++a) {
+      const float prev = __shfl_sync(kFull, alpha, a);
+      if (has) m = fmaxf(m, prev + __ldg(A + a * r + lane));
+    }
+    float s = 0.f;
+    for (int a = 0; a < r; ++a) {
+      const float prev = __shfl_sync(kFull, alpha, a);
+      if (has) s += __expf(prev + __ldg(A + a * r + lane) - m);
+    }
+    if (has) alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : g[i * r + lane] + m + __logf(s);
+  }
+  const float res = warp_lse(alpha, has);
+  if (lane == 0) out[w] = res;
+}
+
+// Eq. (BTree), bottom-up over the heap-ordered latent tree. Node j >= 1 has the table
+// logOmega_j[a][b] = logw[p, r + (j-1) r^2 + a r + b] (parent's value a, own value b); the deepest internal node
+// n/2-1+m multiplies the input units of tokens 2m and 2m+1. prod[j][z] is the product unit under z_j = z.
+// Shared memory per warp: (n-1) * r floats of prod + r * (r+1) floats of one staged table.  r <= 32.
+__global__ void circuit_btree_kernel(const float* __restrict__ G, const float* __restrict__ logw,
+                                     float* __restrict__ out, int W, int wpp, int n, int r, int sum_rows) {
+  extern __shared__ float sm[];
+  const int wib = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int w = blockIdx.x * kCircuitWarps + wib;
+  float* prod = sm + static_cast<size_t>(wib) * ((n - 1) * r + r * (r + 1));
+  float* table = prod + (n - 1) * r;
+  if (w >= W) return;
+  const float* g = G + static_cast<size_t>(w) * n * r;
+  const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
+  const bool has = lane < r;
+  const int first_leaf_node = n / 2 - 1;
+  for (int j = n - 2; j >= first_leaf_node; --j) {
+    const int m = j - first_leaf_node;
+    if (has) prod[j * r + lane] = g[(2 * m) * r + lane] + g[(2 * m + 1) * r + lane];
+  }
+  __syncwarp();
+  for (int j = first_leaf_node - 1; j >= 0; --j) {
+    float acc = 0.f;
+    for (int side = 0; side < 2; ++side) {
+      const int c = 2 * j + 1 + side;
+      const float* tab = lw + r + static_cast<size_t>(c - 1) * r * r;
+      for (int a = 0; a < r; ++a)                      // coalesced rows -> padded shared tile
+        if (has) table[a * (r + 1) + lane] = tab[a * r + lane];
+      __syncwarp();
+      if (has) {
+        const float* row = table + lane * (r + 1);     // row z_j = lane, over the child's values b
+        const float* pc = prod + c * r;
+        float m = -CUDART_INF_F;
+        for (int b = 0; b < r; ++b) m = fmaxf(m, row[b] + pc[b]);
+        float s = 0.f;
+        for (int b = 0; b < r; ++b) s += __expf(row[b] + pc[b] - m);
+        acc += (m == -CUDART_INF_F) ? -CUDART_INF_F : m + __logf(s);
+        if (s != s) acc = s;
+      }
+      __syncwarp();
+    }
+    if (has) prod[j * r + lane] = acc;
+    __syncwarp();
+  }
+  const float res = warp_lse(has ? lw[lane] + prod[lane] : 0.f, has);
+  if (lane == 0) out[w] = res;
+}
+
+// ---------------------------------------------------------------- latent draws (Algorithm 1, sum units)
+// Inverse CDF over r log-probabilities: the smallest j with u < p_0 + ... + p_j, else r - 1.
+__device__ __forceinline__ int inv_cdf_logp(const float* __restrict__ logp, int r, float u) {
+  float cum = 0.f;
+  int found = r - 1;
+  bool hit = false;
+  for (int j = 0; j < r; ++j) {
+    cum += expf(logp[j]);
+    if (!hit && u < cum) { hit = true; found = j; }
+  }
+  return found;
+}
+
+// One thread per window. Writes unit_sel[w, i] = the input unit chosen for token i and presets out_bytes to -1.
+__global__ void latent_sample_kernel(int family, const float* __restrict__ logw, const float* __restrict__ logA,
+                                     const float* __restrict__ uniforms, int* __restrict__ unit_sel,
+                                     int* __restrict__ out_bytes, unsigned* status, int W, int wpp, int n, int r,
+                                     int sum_rows) {
+  const int w = blockIdx.x * blockDim.x + threadIdx.x;
+  if (w >= W) return;
+  const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
+  const float* u = uniforms + static_cast<size_t>(w) * 2 * n;
+  int* sel = unit_sel + static_cast<size_t>(w) * n;
+  bool bad = false;
+  for (int i = 0; i < n; ++i) out_bytes[static_cast<size_t>(w) * n + i] = -1;
+  const int nlat = (family == 0) ? 1 : (family == 1 ? n : n - 1);
+  for (int i = 0; i < nlat; ++i) bad |= !(u[i] >= 0.f && u[i] < 1.f);
+  if (bad) {
+    atomicOr(status, 2u);
+    for (int i = 0; i < n; ++i) sel[i] = -1;
+    return;
+  }
+  if (family == 0) {
+    const int z = inv_cdf_logp(lw, r, u[0]);
+    for (int i = 0; i < n; ++i) sel[i] = z;
+  } else if (family == 1) {
+    int z = inv_cdf_logp(lw, r, u[0]);
+    sel[0] = z;
+    for (int i = 1; i < n; ++i) {
+      z = inv_cdf_logp(logA + (static_cast<size_t>(i - 1) * r + z) * r, r, u[i]);
+      sel[i] = z;
+    }
+  } else {
+    int zs[63];
+    zs[0] = inv_cdf_logp(lw, r, u[0]);
+    for (int j = 1; j < n - 1; ++j)
+      zs[j] = inv_cdf_logp(lw + r + (static_cast<size_t>(j - 1) * r + zs[(j - 1) >> 1]) * r, r, u[j]);
+    for (int i = 0; i < n; ++i) sel[i] = zs[n / 2 - 1 + (i >> 1)];
+  }
+}
+
+// ---------------------------------------------------------------- preparation
+__global__ void f32_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t count) {
+  size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  for (; i < count; i += stride) dst[i] = __float2bfloat16_rn(src[i]);
+}
+
+// Row-wise log-softmax of the static transition logits: one thread per row of r entries.
+__global__ void log_softmax_rows_kernel(const float* __restrict__ src, float* __restrict__ dst, int rows, int r) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= rows) return;
+  const float* x = src + static_cast<size_t>(row) * r;
+  float m = x[0];
+  for (int j = 1; j < r; ++j) m = fmaxf(m, x[j]);
+  float s = 0.f;
+  for (int j = 0; j < r; ++j) s += expf(x[j] - m);
+  const float lse = m + logf(s);
+  for (int j = 0; j < r; ++j) dst[static_cast<size_t>(row) * r + j] = x[j] - lse;
+}
+
+}  // namespace mtpc

@@ -1,0 +1,481 @@
+// Projection kernel of the MtPC head (Sec. 3.3): logits = h W^T on the tcgen05 tensor cores, with the softmax
+// over the vocabulary, the evidence gather (log phi at the target byte) or the inverse-CDF byte draw
+// (Algorithm 1, input units), and the log-softmax of the sum-unit logits all done in the epilogue straight
+// out of tensor memory. The [positions, n, r, v] logit tensor never exists in HBM.
+//
+// One persistent CTA per SM, 6 warps:
+//   warp 0      TMA producer: per 64-wide K block, one 128-row tile of h and the v rows of one emission unit
+//               (or one tile of sum-unit rows) into a ring of shared-memory stages (128-byte swizzle).
+//   warp 1      allocates the 512 TMEM columns, issues tcgen05.mma (M=128, N=chunk, K=16) from one thread.
+//   warps 2..5  epilogue; warp w reads TMEM lanes 32*(w%4)..+31, one thread per position (row), so every
+//               row-wise reduction over the vocabulary is a plain in-thread loop.
+// A work item ("tile") is 128 positions x one unit: emission unit (i,k) = v logit columns, split into
+// `chunks_per_unit` accumulators of `chunk_cols` columns (v=320 -> 2 x 160, v=256 -> 1 x 256), or one tile
+// of `sum_cols` sum-unit columns. Accumulators live in a ring of TMEM slots, so the epilogue of one tile
+// overlaps the MMAs of the next. Every barrier wait is bounded: when one runs out the CTA raises
+// MTPC_STATUS_TIMEOUT in the status word, drains its copies, frees its TMEM and returns.
+#pragma once
+#include <math_constants.h>
+
+#include "mtpc_ptx.cuh"
+
+namespace mtpc {
+
+constexpr int kBlockM = 128;         // positions per tile (= TMEM lanes)
+constexpr int kBlockK = 64;          // bf16 elements per 128-byte swizzled row
+constexpr int kMaxStages = 8;
+constexpr int kMaxSlots = 16;
+constexpr int kTmemCols = 512;
+constexpr int kGemmThreads = 192;
+constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per barrier wait
+constexpr int kABytes = kBlockM * kBlockK * 2;                   // 16 KB
+constexpr uint32_t kStatusBadTarget = 1u, kStatusBadUniform = 2u, kStatusTimeout = 4u;
+
+enum { kModeLogprob = 0, kModeSample = 1 };
+
+struct GemmParams {
+  CUtensorMap tm_a;      // hidden  [T, d]        box 64 x 128
+  CUtensorMap tm_emit;   // W_emit  [n*r*v, d]    box 64 x chunk_cols
+  CUtensorMap tm_sum;    // W_sum   [S*r, d]      box 64 x sum_cols
+  int T, m_tiles, kblocks;
+  int n, r, v;
+  int emit_units;                    // n * r
+  int unit_begin, unit_count;        // units [unit_begin, unit_begin + unit_count); >= emit_units = sum tiles
+  int chunk_cols, chunks_per_unit;
+  int sum_cols, sum_rows;            // sum tile width; S * r
+  int slot_stride, num_slots;
+  int stages, stage_bytes;
+  int wpp;                           // windows (target rows) per position
+  const int* targets;                // [T*wpp, n]
+  float* G;                          // [T*wpp, n, r]   log phi at the target
+  float* logw;                       // [T, S*r]        log-softmaxed sum-unit weights
+  const int* unit_sel;               // [T*wpp, n]      selected input unit per token (sample mode)
+  const float* uniforms;             // [T*wpp, 2n]
+  int* out_bytes;                    // [T*wpp, n]
+  unsigned* status;
+};
+
+struct GemmControl {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t tfull[kMaxSlots];
+  uint64_t tempty[kMaxSlots];
+  uint64_t drain;
+  uint32_t tmem_base;
+  volatile int abort;
+};
+
+__device__ __forceinline__ float fast_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float fast_lg2(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, GemmControl* ctl, unsigned* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  uint32_t it = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++it & 63u) == 0) {
+      if (ctl->abort) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        ctl->abort = 1;
+        atomicOr(status, kStatusTimeout);
+        return false;
+      }
+    }
+  }
+}
+// Lane 0 waits, the whole warp learns the outcome (keeps the warp converged for the .sync.aligned TMEM loads).
+__device__ __forceinline__ bool bounded_wait_warp(uint32_t bar, uint32_t parity, GemmControl* ctl, unsigned* status,
+                                                  int lane) {
+  int ok = 1;
+  if (lane == 0) ok = bounded_wait(bar, parity, ctl, status) ? 1 : 0;
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+struct TileCoord {
+  int unit, mt, is_sum, chunks, cols, brow0;
+};
+__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile) {
+  TileCoord c;
+  c.unit = p.unit_begin + tile / p.m_tiles;
+  c.mt = tile % p.m_tiles;
+  c.is_sum = c.unit >= p.emit_units;
+  c.chunks = c.is_sum ? 1 : p.chunks_per_unit;
+  c.cols = c.is_sum ? p.sum_cols : p.chunk_cols;
+  c.brow0 = c.is_sum ? (c.unit - p.emit_units) * p.sum_cols : c.unit * p.v;
+  return c;
+}
+
+// log-softmax over groups of R adjacent columns inside one 16-column batch (R in {1,2,4,8,16}).
+template <int R>
+__device__ __forceinline__ void sum_groups_in_batch(const float (&x)[16], float* dst, int col0, int sum_rows) {
+#pragma unroll
+  for (int g = 0; g < 16 / R; ++g) {
+    float m = x[g * R];
+#pragma unroll
+    for (int q = 1; q < R; ++q) m = fmaxf(m, x[g * R + q]);
+    float s = 0.f;
+#pragma unroll
+    for (int q = 0; q < R; ++q) s += fast_ex2((x[g * R + q] - m) * kLog2e);
+    const float lse = m + fast_lg2(s) * kLn2;
+    if (col0 + g * R < sum_rows) {
+#pragma unroll
+      for (int q = 0; q < R; ++q) dst[col0 + g * R + q] = x[g * R + q] - lse;
+    }
+  }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
+  uint8_t* tiles = smem_raw + (tiles_addr - raw_addr);
+  GemmControl* ctl = reinterpret_cast<GemmControl*>(tiles + static_cast<size_t>(p.stages) * p.stage_bytes);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int num_tiles = p.unit_count * p.m_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(smem_u32(&ctl->full[s]), 1);
+      mbar_init(smem_u32(&ctl->empty[s]), 1);
+    }
+    for (int s = 0; s < p.num_slots; ++s) {
+      mbar_init(smem_u32(&ctl->tfull[s]), 1);
+      mbar_init(smem_u32(&ctl->tempty[s]), 4);
+    }
+    mbar_init(smem_u32(&ctl->drain), 1);
+    ctl->abort = 0;
+    fence_mbar_init();
+    tma_prefetch_desc(&p.tm_a);
+    tma_prefetch_desc(&p.tm_emit);
+    tma_prefetch_desc(&p.tm_sum);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const TileCoord tc = tile_coord(p, tile);
+        const CUtensorMap* tmb = tc.is_sum ? &p.tm_sum : &p.tm_emit;
+        const uint32_t bytes = kABytes + tc.chunks * tc.cols * (kBlockK * 2);
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
+          const uint32_t full = smem_u32(&ctl->full[stage]);
+          const uint32_t a_dst = tiles_addr + stage * p.stage_bytes;
+          mbar_arrive_expect_tx(full, bytes);
+          tma_load_2d(a_dst, &p.tm_a, full, kb * kBlockK, tc.mt * kBlockM);
+          for (int c = 0; c < tc.chunks; ++c)
+            tma_load_2d(a_dst + kABytes + c * tc.cols * (kBlockK * 2), tmb, full, kb * kBlockK,
+                        tc.brow0 + c * tc.cols);
+          issued_mask |= 1u << stage;
+          phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
+          if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {   // give the copies still in flight a bounded chance to land before the CTA goes away
+        for (int s = 0; s < p.stages; ++s)
+          if (issued_mask & (1u << s)) {
+            const uint32_t bar = smem_u32(&ctl->full[s]);
+            const uint32_t par = (phase_mask >> s) & 1u;
+            const uint64_t t0 = global_timer_ns();
+            while (!mbar_try_wait(bar, par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, use = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const TileCoord tc = tile_coord(p, tile);
+        const uint32_t idesc = umma_idesc_bf16(kBlockM, tc.cols);
+        for (int kb = 0; kb < p.kblocks && ok; ++kb) {
+          if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = tiles_addr + stage * p.stage_bytes;
+          const uint64_t a_desc = umma_smem_desc_sw128(a_addr);
+          for (int c = 0; c < tc.chunks; ++c) {
+            const uint32_t u = use + c;
+            const uint32_t slot = u % p.num_slots;
+            if (kb == 0) {
+              const uint32_t sphase = (u / p.num_slots) & 1u;
+              if (!bounded_wait(smem_u32(&ctl->tempty[slot]), sphase ^ 1u, ctl, p.status)) { ok = false; break; }
+              tc_fence_after();
+            }
+            const uint64_t b_desc = umma_smem_desc_sw128(a_addr + kABytes + c * tc.cols * (kBlockK * 2));
+            const uint32_t d_tmem = tmem_base + slot * p.slot_stride;
+#pragma unroll
+            for (int kk = 0; kk < kBlockK / 16; ++kk)   // +32 bytes per K=16 step inside the swizzled row
+              umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+          }
+          if (!ok) break;
+          umma_commit(smem_u32(&ctl->empty[stage]));
+          if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        for (int c = 0; c < tc.chunks; ++c) umma_commit(smem_u32(&ctl->tfull[(use + c) % p.num_slots]));
+        use += tc.chunks;
+      }
+      if (!ok) {   // wait (bounded) for the MMAs already issued before TMEM is freed
+        umma_commit(smem_u32(&ctl->drain));
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int quarter = warp & 3;
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    uint32_t use = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      const TileCoord tc = tile_coord(p, tile);
+      const int row = tc.mt * kBlockM + quarter * 32 + lane;
+      const bool valid = row < p.T;
+      const int nbatch = tc.cols / 16;
+
+      if (tc.is_sum) {
+        // ---- sum-unit logits -> log omega (Sec. 3.3): log-softmax over groups of r adjacent columns
+        const uint32_t slot = use % p.num_slots;
+        if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (use / p.num_slots) & 1u, ctl, p.status, lane)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t tcol = lane_base + slot * p.slot_stride;
+        const int col_base = (tc.unit - p.emit_units) * p.sum_cols;
+        float* dst = p.logw + static_cast<size_t>(valid ? row : 0) * p.sum_rows;
+        if (p.r <= 16) {
+          for (int b = 0; b < nbatch; ++b) {
+            float x[16];
+            tmem_ld16(tcol + b * 16, x);
+            if (valid) {
+              const int col0 = col_base + b * 16;
+              switch (p.r) {
+                case 1: sum_groups_in_batch<1>(x, dst, col0, p.sum_rows); break;
+                case 2: sum_groups_in_batch<2>(x, dst, col0, p.sum_rows); break;
+                case 4: sum_groups_in_batch<4>(x, dst, col0, p.sum_rows); break;
+                case 8: sum_groups_in_batch<8>(x, dst, col0, p.sum_rows); break;
+                default: sum_groups_in_batch<16>(x, dst, col0, p.sum_rows); break;
+              }
+            }
+          }
+        } else {
+          const int bpg = p.r / 16;   // batches per group
+          for (int g = 0; g < tc.cols / p.r; ++g) {
+            float m = -CUDART_INF_F, s = 0.f;
+            for (int b = 0; b < bpg; ++b) {
+              float x[16];
+              tmem_ld16(tcol + (g * bpg + b) * 16, x);
+              float bm = x[0];
+#pragma unroll
+              for (int q = 1; q < 16; ++q) bm = fmaxf(bm, x[q]);
+              const float mn = fmaxf(m, bm);
+              s *= fast_ex2((m - mn) * kLog2e);
+#pragma unroll
+              for (int q = 0; q < 16; ++q) s += fast_ex2((x[q] - mn) * kLog2e);
+              m = mn;
+            }
+            const float lse = m + fast_lg2(s) * kLn2;
+            const int gcol = col_base + g * p.r;
+            for (int b = 0; b < bpg; ++b) {
+              float x[16];
+              tmem_ld16(tcol + (g * bpg + b) * 16, x);
+              if (valid && gcol < p.sum_rows) {
+                float4* d4 = reinterpret_cast<float4*>(dst + gcol + b * 16);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                  d4[q] = make_float4(x[4 * q] - lse, x[4 * q + 1] - lse, x[4 * q + 2] - lse, x[4 * q + 3] - lse);
+              }
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctl->tempty[slot]));
+        use += 1;
+        continue;
+      }
+
+      const int slot_i = tc.unit / p.r;   // window slot i
+      const int k = tc.unit % p.r;        // input unit k
+
+      if (MODE == kModeLogprob) {
+        // ---- log phi at the target byte: online log-sum-exp over the v columns + gather
+        float m = -CUDART_INF_F, s = 0.f, tval = 0.f;
+        int tgt = -1;
+        const size_t wrow0 = static_cast<size_t>(valid ? row : 0) * p.wpp;
+        if (p.wpp == 1 && valid) tgt = p.targets[wrow0 * p.n + slot_i];
+        for (int c = 0; c < tc.chunks && ok; ++c) {
+          const uint32_t u = use + c;
+          const uint32_t slot = u % p.num_slots;
+          if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (u / p.num_slots) & 1u, ctl, p.status, lane)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t tcol = lane_base + slot * p.slot_stride;
+          for (int b = 0; b < nbatch; ++b) {
+            float x[16];
+            tmem_ld16(tcol + b * 16, x);
+            const int col0 = c * tc.cols + b * 16;
+            float bm = x[0];
+#pragma unroll
+            for (int q = 1; q < 16; ++q) bm = fmaxf(bm, x[q]);
+            const float mn = fmaxf(m, bm);
+            const float mn2 = mn * kLog2e;
+            s *= fast_ex2((m - mn) * kLog2e);
+#pragma unroll
+            for (int q = 0; q < 16; ++q) s += fast_ex2(fmaf(x[q], kLog2e, -mn2));
+            m = mn;
+            if (p.wpp == 1) {
+              const int rel = tgt - col0;
+              if (static_cast<unsigned>(rel) < 16u) {
+#pragma unroll
+                for (int q = 0; q < 16; ++q)
+                  if (rel == q) tval = x[q];
+              }
+            } else if (valid) {
+              for (int j = 0; j < p.wpp; ++j) {
+                const int rel = p.targets[(wrow0 + j) * p.n + slot_i] - col0;
+                if (static_cast<unsigned>(rel) < 16u) {
+                  float val = 0.f;
+#pragma unroll
+                  for (int q = 0; q < 16; ++q)
+                    if (rel == q) val = x[q];
+                  p.G[((wrow0 + j) * p.n + slot_i) * p.r + k] = val;   // raw logit; normalised below
+                }
+              }
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&ctl->tempty[slot]));
+        }
+        if (!ok) break;
+        const float lse = m + fast_lg2(s) * kLn2;
+        if (valid) {
+          for (int j = 0; j < p.wpp; ++j) {
+            const int t = (p.wpp == 1) ? tgt : p.targets[(wrow0 + j) * p.n + slot_i];
+            float* g = p.G + ((wrow0 + j) * p.n + slot_i) * p.r + k;
+            if (t < 0) {
+              *g = 0.f;                                  // marginalised byte: the input unit sums to 1
+            } else if (t >= p.v) {
+              *g = CUDART_NAN_F;
+              atomicOr(p.status, kStatusBadTarget);
+            } else {
+              *g = ((p.wpp == 1) ? tval : *g) - lse;
+            }
+          }
+        }
+      } else {
+        // ---- byte draws (Algorithm 1, input units): inverse CDF of softmax(logits) for every window of this
+        // row whose selected unit for this slot is k. All chunks of the unit stay in TMEM until the end.
+        unsigned long long pending = 0ull;
+        const size_t wrow0 = static_cast<size_t>(valid ? row : 0) * p.wpp;
+        if (valid)
+          for (int j = 0; j < p.wpp; ++j)
+            if (p.unit_sel[(wrow0 + j) * p.n + slot_i] == k) pending |= 1ull << j;
+        for (int c = 0; c < tc.chunks && ok; ++c) {
+          const uint32_t u = use + c;
+          if (!bounded_wait_warp(smem_u32(&ctl->tfull[u % p.num_slots]), (u / p.num_slots) & 1u, ctl, p.status,
+                                 lane))
+            ok = false;
+        }
+        if (!ok) break;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, pending != 0ull)) {
+          float m = -CUDART_INF_F;
+          for (int c = 0; c < tc.chunks; ++c) {
+            const uint32_t tcol = lane_base + ((use + c) % p.num_slots) * p.slot_stride;
+            for (int b = 0; b < nbatch; ++b) {
+              float x[16];
+              tmem_ld16(tcol + b * 16, x);
+#pragma unroll
+              for (int q = 0; q < 16; ++q) m = fmaxf(m, x[q]);
+            }
+          }
+          const float m2 = m * kLog2e;
+          float total = 0.f;   // same terms in the same order as the running sum of the scan below
+          for (int c = 0; c < tc.chunks; ++c) {
+            const uint32_t tcol = lane_base + ((use + c) % p.num_slots) * p.slot_stride;
+            for (int b = 0; b < nbatch; ++b) {
+              float x[16];
+              tmem_ld16(tcol + b * 16, x);
+#pragma unroll
+              for (int q = 0; q < 16; ++q) total += fast_ex2(fmaf(x[q], kLog2e, -m2));
+            }
+          }
+          while (__any_sync(0xffffffffu, pending != 0ull)) {
+            const int j = pending ? __ffsll(static_cast<long long>(pending)) - 1 : -1;
+            float uval = 0.f;
+            if (j >= 0) uval = p.uniforms[(wrow0 + j) * (2 * p.n) + p.n + slot_i];
+            const float thr = uval * total;
+            float cum = 0.f;
+            int found = p.v - 1;   // rounding may leave no index: the last one
+            bool hit = false;
+            for (int c = 0; c < tc.chunks; ++c) {
+              const uint32_t tcol = lane_base + ((use + c) % p.num_slots) * p.slot_stride;
+              for (int b = 0; b < nbatch; ++b) {
+                float x[16];
+                tmem_ld16(tcol + b * 16, x);
+                const int col0 = c * tc.cols + b * 16;
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                  cum += fast_ex2(fmaf(x[q], kLog2e, -m2));
+                  if (!hit && thr < cum) { hit = true; found = col0 + q; }
+                }
+              }
+            }
+            if (j >= 0) {
+              if (!(uval >= 0.f && uval < 1.f)) {
+                found = -1;
+                atomicOr(p.status, kStatusBadUniform);
+              }
+              p.out_bytes[(wrow0 + j) * p.n + slot_i] = found;
+              pending &= pending - 1ull;
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0)
+          for (int c = 0; c < tc.chunks; ++c) mbar_arrive(smem_u32(&ctl->tempty[(use + c) % p.num_slots]));
+      }
+      use += tc.chunks;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace mtpc
