@@ -1,0 +1,78 @@
+"""Moves a synthetic workload onto the device and drives the head through the C-ABI binding.
+Used by the GPU tests, the smoke check and the benchmark; holds no arithmetic of the method."""
+from __future__ import annotations
+
+import numpy as np
+
+from . import binding as B
+from . import inputs as I
+
+
+def to_device_bf16(x_q: np.ndarray, device="cuda"):
+    """fp32 array of bf16-representable values -> torch.bfloat16 tensor with the same bit patterns."""
+    import torch
+    return torch.from_numpy(I.bf16_bits(x_q).view(np.int16)).to(device).view(torch.bfloat16).reshape(x_q.shape)
+
+
+def to_host_bf16(x_q: np.ndarray, pinned: bool = True):
+    import torch
+    t = torch.from_numpy(I.bf16_bits(x_q).view(np.int16)).view(torch.bfloat16).reshape(x_q.shape)
+    return t.pin_memory() if pinned else t
+
+
+class DeviceHead:
+    """Weights of a workload resident in HBM plus a head created on them."""
+
+    def __init__(self, wl: I.Workload, max_positions: int | None = None, max_wpp: int | None = None, device="cuda"):
+        import torch
+        s = wl.shape
+        self.wl = wl
+        self.device = device
+        if s.io_dtype == I.F32:
+            self.W_emit = torch.from_numpy(wl.W_emit_raw).to(device)
+            self.W_sum = torch.from_numpy(wl.W_sum_raw).to(device)
+        else:
+            self.W_emit = to_device_bf16(wl.W_emit_q, device)
+            self.W_sum = to_device_bf16(wl.W_sum_q, device)
+        self.T_static = torch.from_numpy(np.ascontiguousarray(wl.T_static)).to(device) if wl.T_static is not None else None
+        self.head = B.MtpcHead(s.family, s.n, s.r, s.v, s.d, s.io_dtype, max_positions or max(wl.T, 1),
+                               max_wpp or max(wl.wpp, 1), self.W_emit, self.W_sum, self.T_static)
+
+    def hidden_device(self, rows=None):
+        import torch
+        wl = self.wl
+        sl = slice(None) if rows is None else rows
+        if wl.shape.io_dtype == I.F32:
+            return torch.from_numpy(np.ascontiguousarray(wl.hidden_raw[sl])).to(self.device)
+        return to_device_bf16(np.ascontiguousarray(wl.hidden_q[sl]), self.device)
+
+    def hidden_host(self, rows=None):
+        import torch
+        wl = self.wl
+        sl = slice(None) if rows is None else rows
+        if wl.shape.io_dtype == I.F32:
+            return torch.from_numpy(np.ascontiguousarray(wl.hidden_raw[sl])).pin_memory()
+        return to_host_bf16(np.ascontiguousarray(wl.hidden_q[sl]))
+
+    def window_logprob(self, hidden=None, targets=None):
+        """Device-buffer call on the workload's own hidden states / targets (or the given device tensors)."""
+        import torch
+        h = self.hidden_device() if hidden is None else hidden
+        t = torch.from_numpy(self.wl.targets).to(self.device) if targets is None else targets
+        out = torch.empty(h.shape[0], dtype=torch.float32, device=self.device)
+        self.head.mtpc_window_logprob(h, t, out)
+        return out
+
+    def draft_sample(self, wpp=None, hidden=None, uniforms=None):
+        import torch
+        wpp = wpp or self.wl.wpp
+        h = self.hidden_device() if hidden is None else hidden
+        u = torch.from_numpy(self.wl.uniforms).to(self.device) if uniforms is None else uniforms
+        W = h.shape[0] * wpp
+        out_bytes = torch.empty((W, self.wl.shape.n), dtype=torch.int32, device=self.device)
+        out_lp = torch.empty(W, dtype=torch.float32, device=self.device)
+        self.head.mtpc_draft_sample(h, wpp, u, out_bytes, out_lp)
+        return out_bytes, out_lp
+
+    def close(self):
+        self.head.mtpc_destroy()
