@@ -1,0 +1,334 @@
+#!/usr/bin/env python
+"""Benchmark of the MtPC head on B200: window log-likelihood positions/s on the training-shaped CP workload
+(8192 positions, d=4096, n=8, r=16, v=320), plus draft windows/s on one decode cell.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3] [--impl reference]
+
+One step = one mtpc_window_logprob call over the whole batch (projection GEMM with fused softmax/gather
+epilogue + circuit evaluation). Prints ONE JSON line on rank 0. With N > 1 (launched by torchrun, one process
+per GPU) every rank runs an independent replica: the head has no exchange step, so there is no collective on
+the data path; ranks meet only at the timing barrier and `value` sums the replicas' work over the slowest
+rank's time. `--impl reference` times the fp64 CPU oracle on the host cores instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2511_11346_b200 import inputs as I          # noqa: E402
+from paper_2511_11346_b200 import replicas             # noqa: E402
+
+METRIC = "window_loglik_positions_per_s"
+UNIT = "positions/s"
+FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one projection-kernel launch, from the ncu capture
+# summarised in profiles/ (captured at a quarter of the positions and scaled). None = not captured.
+NCU_TRAFFIC_BYTES = {1: None, 2: None, 3: None}
+
+
+def workload_name(idx: int, wl) -> str:
+    s = wl.shape
+    return (f"configs[{idx}] {wl.name}: T={wl.T} d={s.d} n={s.n} r={s.r} v={s.v} "
+            f"{'bf16' if s.io_dtype == I.BF16 else 'fp32'} io")
+
+
+def algorithmic_flops(wl) -> float:
+    """2 d (n r v + S r) per position: the method's own projection work (Table 3's 'MTP head linear')."""
+    s = wl.shape
+    return 2.0 * s.d * (s.n * s.r * s.v + s.sum_rows) * wl.T
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+                 "hw_power_brake_slowdown": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_positions_per_s(wl, sample_positions: int, chunk: int = 256):
+    """The oracle as it stands, on the first `sample_positions` positions, in chunks (memory)."""
+    from oracle import mtpc_oracle as orc
+    s = wl.shape
+    t0 = time.perf_counter()
+    done = 0
+    while done < sample_positions:
+        rows = slice(done, min(done + chunk, sample_positions))
+        orc.window_logprob(s.family, wl.hidden_q[rows], wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets[rows])
+        done = rows.stop
+    dt = time.perf_counter() - t0
+    return sample_positions / dt, dt
+
+
+def host_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank, _, world = replicas.rank_env()
+    if rank != 0:
+        return
+    wl = I.config_workload(args.workload)
+    for _ in range(max(args.warmup, 1)):
+        rate, _ = oracle_positions_per_s(wl, 64, chunk=64)
+    # bounded sample: the whole run should take about two minutes whatever K is
+    budget_s = 120.0
+    sample = int(max(16, min(wl.T, args.ref_positions, rate * budget_s / max(args.steps, 1))))
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_positions_per_s(wl, sample)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    cores = host_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(args.workload, wl),
+                   "sample": f"each step = the fp64 numpy oracle on the first {sample} of {wl.T} positions"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"first {sample} of {wl.T} positions per step, {args.steps} steps"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def measure_decode_cell(torch, cell, steps: int, warmup: int):
+    """Draft windows/s and p50 latency on one decode cell (family, n, P) with 16 windows per position."""
+    from paper_2511_11346_b200.runner import DeviceHead
+    wl = I.config_workload(4, cell=cell)
+    dh = DeviceHead(wl)
+    h = dh.hidden_device()
+    u = torch.from_numpy(wl.uniforms).cuda()
+    W = wl.T * wl.wpp
+    ob = torch.empty((W, wl.shape.n), dtype=torch.int32, device="cuda")
+    ol = torch.empty(W, dtype=torch.float32, device="cuda")
+    for _ in range(warmup):
+        dh.head.mtpc_draft_sample(h, wl.wpp, u, ob, ol)
+    torch.cuda.synchronize()
+    lat = []
+    for _ in range(steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        dh.head.mtpc_draft_sample(h, wl.wpp, u, ob, ol)
+        e1.record()
+        e1.synchronize()
+        lat.append(e0.elapsed_time(e1))
+    p50 = statistics.median(lat)
+    s = wl.shape
+    weight_bytes = (s.n * s.r * s.v + s.sum_rows) * s.d * 2
+    peaks, src = load_peaks()
+    out = {"workload": f"configs[4] {wl.name}: P={wl.T} wpp={wl.wpp} d={s.d} n={s.n} r={s.r} v={s.v}",
+           "windows_per_s": W / (p50 * 1e-3), "p50_ms": p50, "calls": steps,
+           "hbm_roofline": {"algorithmic_bytes": weight_bytes, "note": "one pass over the weights",
+                            "achieved_gbs": weight_bytes / (p50 * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
+                            "frac": weight_bytes / (p50 * 1e-3) / 1e9 / peaks["hbm_gbs"], "peak_source": src}}
+    dh.close()
+    return out
+
+
+def run_ours(args):
+    import torch
+    from paper_2511_11346_b200.runner import DeviceHead
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the MtPC head has no CPU path (use --impl reference for the oracle)")
+    rank, local_rank, world = replicas.rank_env()
+    torch.cuda.set_device(local_rank if world > 1 else 0)
+    replicas.init_process_group("nccl")
+    dev_index = torch.cuda.current_device()
+
+    wl = I.config_workload(args.workload, T=args.positions)
+    s = wl.shape
+    dh = DeviceHead(wl)
+    head = dh.head
+    hidden = dh.hidden_device()
+    targets = torch.from_numpy(wl.targets).cuda()
+    out = torch.empty(wl.T, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    # ---------------- device-resident throughput: K steps back to back, per-kernel events kept by the library
+    for _ in range(args.warmup):
+        head.mtpc_window_logprob(hidden, targets, out)
+    torch.cuda.synchronize()
+    head.mtpc_set_timing(min(args.steps, 4096))
+    launches0 = head.mtpc_launch_count()
+    sampler = ClockSampler(dev_index)
+    replicas.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        head.mtpc_window_logprob(hidden, targets, out)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    replicas.barrier()
+    clocks = sampler.stop()
+    elapsed_s = replicas.max_over_ranks(e0.elapsed_time(e1) * 1e-3, device="cuda")
+    launches = head.mtpc_launch_count() - launches0
+    kept = min(args.steps, 4096)
+    phases = [head.mtpc_get_timing(i) for i in range(kept)]
+    gemm_ms = statistics.mean(p[0] for p in phases)
+    circuit_ms = statistics.mean(p[1] for p in phases)
+    head.mtpc_set_timing(0)
+    status = head.mtpc_get_status()
+    value = replicas.aggregate_throughput(wl.T, args.steps, world, elapsed_s)
+
+    # ---------------- end to end through the host-buffer entry point (pinned host memory, copies timed)
+    hh = dh.hidden_host()
+    th = torch.from_numpy(wl.targets).pin_memory()
+    oh = torch.empty(wl.T, dtype=torch.float32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 50))
+    for _ in range(3):
+        head.mtpc_window_logprob_host(hh, th, oh)
+    replicas.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        head.mtpc_window_logprob_host(hh, th, oh)      # returns after the result is in host memory
+    torch.cuda.synchronize()
+    e2e_s = replicas.max_over_ranks(time.perf_counter() - t0, device="cuda")
+    e2e_value = replicas.aggregate_throughput(wl.T, e2e_steps, world, e2e_s)
+    h2d = hh.numel() * hh.element_size() + th.numel() * 4
+    d2h = oh.numel() * 4
+
+    if rank != 0:
+        return
+
+    peaks, peak_src = load_peaks()
+    flops = algorithmic_flops(wl)
+    achieved = flops / (gemm_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    traffic = NCU_TRAFFIC_BYTES.get(args.workload)
+    roofline = {"bound": "tensor", "kernel": "mtpc_gemm_kernel<logprob>", "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic,
+                "peak_source": f"{peak_src}: bf16_tflops_sustained (kernel timed inside a {elapsed_s:.2f} s back-to-back loop)",
+                "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "burst_peak": peaks["bf16_tflops"],
+                "flops_per_launch": flops, "avg_launch_ms": gemm_ms, "circuit_kernel_avg_ms": circuit_ms,
+                "timed_launches": kept}
+
+    # CPU baseline: the oracle as it stands on a bounded sample of the same workload
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        sample = min(wl.T, args.ref_positions)
+        cpu_value, cpu_s = oracle_positions_per_s(wl, sample)
+        cpu_baseline = {"value": cpu_value, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                        "sample": f"first {sample} of {wl.T} positions, one pass, {cpu_s:.1f} s"}
+
+    draft = None
+    if not args.no_draft and world == 1:
+        draft = measure_decode_cell(torch, (I.CP, 8, 64), steps=200, warmup=5)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": elapsed_s / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(args.workload, wl), "parallelism": f"replicas x{world} (no collective)",
+                   "l2": "inputs larger than L2 (336 MB of weights + 67 MB of hidden states per step vs 126 MB)"
+                   if args.workload == 1 else "inputs larger than L2",
+                   "step": "one mtpc_window_logprob call: projection GEMM + fused epilogue, then circuit evaluation"},
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3,
+                "call": "mtpc_window_logprob_host (pinned host buffers, copies inside the call)"},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": cpu_baseline,
+        "device_status": status,
+    }
+    if draft is not None:
+        line["draft"] = draft
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3])
+    ap.add_argument("--ref-positions", type=int, default=None,
+                    help="positions the CPU oracle processes per step / for the cpu_baseline sample")
+    ap.add_argument("--no-draft", action="store_true", help="skip the decode-cell draft measurement")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiling runs)")
+    ap.add_argument("--positions", type=int, default=None,
+                    help="override the number of positions (scaled-down profiler captures; not a bench value)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        args.ref_positions = args.ref_positions or 1024
+        run_reference(args)
+    else:
+        args.steps = 400 if args.steps is None else args.steps
+        args.warmup = max(3, 5 if args.warmup is None else args.warmup)
+        args.ref_positions = args.ref_positions or 4096
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

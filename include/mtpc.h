@@ -139,15 +139,17 @@ int mtpc_draft_sample_host(mtpc_head* head, const void* hidden_host, int32_t P, 
 int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags);
 
 /*
- * Per-kernel device timing of the most recent call (CUDA events recorded on the call's stream around each
- * launch). Off by default. mtpc_get_timing synchronises on the events and writes up to `capacity` phase
- * durations in milliseconds, *out_count = number of phases of the last call:
+ * Per-kernel device timing (CUDA events recorded on the call's stream around each launch). Off by default.
+ * mtpc_set_timing(head, ring): keep the events of the `ring` most recent calls (0 <= ring <= 4096; 0 = off;
+ * changing it discards what was recorded). mtpc_get_timing(head, calls_back, ...) synchronises on the events
+ * of the call made `calls_back` calls ago (0 = the most recent) and writes up to `capacity` phase durations
+ * in milliseconds, *out_count = number of phases that call had:
  *   mtpc_window_logprob: [0] projection GEMM + fused epilogue, [1] circuit evaluation.
  *   mtpc_draft_sample:   [0] sum-unit GEMM, [1] latent sampling, [2] GEMM + inverse-CDF epilogue,
  *                        [3] GEMM + gather epilogue on the drafted bytes, [4] circuit evaluation.
  */
-int mtpc_set_timing(mtpc_head* head, int32_t enabled);
-int mtpc_get_timing(mtpc_head* head, float* out_ms, int32_t capacity, int32_t* out_count);
+int mtpc_set_timing(mtpc_head* head, int32_t ring);
+int mtpc_get_timing(mtpc_head* head, int32_t calls_back, float* out_ms, int32_t capacity, int32_t* out_count);
 
 /* Number of kernels the library launched on behalf of this head since creation (preparation included). */
 int mtpc_launch_count(mtpc_head* head, uint64_t* out_count);

@@ -56,7 +56,7 @@ def lib() -> ctypes.CDLL:
     L.mtpc_draft_sample_host.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
     L.mtpc_get_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     L.mtpc_set_timing.argtypes = [vp, i32]
-    L.mtpc_get_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), i32, ctypes.POINTER(i32)]
+    L.mtpc_get_timing.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_float), i32, ctypes.POINTER(i32)]
     L.mtpc_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
     L.mtpc_destroy.argtypes = [vp]
     L.mtpc_status_string.argtypes = [ctypes.c_int]
@@ -140,13 +140,13 @@ class MtpcHead:
             raise MtpcError(code, "mtpc_get_status")
         return flags.value
 
-    def mtpc_set_timing(self, enabled: bool) -> None:
-        _check(lib().mtpc_set_timing(self.handle, 1 if enabled else 0), "mtpc_set_timing")
+    def mtpc_set_timing(self, ring: int) -> None:
+        _check(lib().mtpc_set_timing(self.handle, int(ring)), "mtpc_set_timing")
 
-    def mtpc_get_timing(self) -> list[float]:
+    def mtpc_get_timing(self, calls_back: int = 0) -> list[float]:
         buf = (ctypes.c_float * 8)()
         cnt = ctypes.c_int32(0)
-        _check(lib().mtpc_get_timing(self.handle, buf, 8, ctypes.byref(cnt)), "mtpc_get_timing")
+        _check(lib().mtpc_get_timing(self.handle, calls_back, buf, 8, ctypes.byref(cnt)), "mtpc_get_timing")
         return [buf[i] for i in range(cnt.value)]
 
     def mtpc_launch_count(self) -> int:

@@ -138,10 +138,10 @@ struct mtpc_head {
   CUtensorMap tm_emit, tm_sum;
   int num_sms;
   int gemm_smem;
-  bool timing;
-  cudaEvent_t ev[2 * kMaxPhases];
-  bool ev_ready;
-  int last_phases;
+  int ring;                 // calls whose per-kernel events are retained (0 = timing off)
+  cudaEvent_t* ev;          // [ring][kMaxPhases][2]
+  int* ring_phases;         // [ring] phases recorded by the call in that slot
+  uint64_t calls;           // timed calls so far
   uint64_t launches;
 };
 
@@ -153,13 +153,22 @@ T* at(mtpc_head* h, size_t off) { return reinterpret_cast<T*>(h->ws + off); }
 struct PhaseTimer {
   mtpc_head* h;
   cudaStream_t st;
-  int idx;
-  PhaseTimer(mtpc_head* head, cudaStream_t s) : h(head), st(s), idx(0) { h->last_phases = 0; }
-  void begin() { if (h->timing && idx < kMaxPhases) cudaEventRecord(h->ev[2 * idx], st); }
+  int idx, slot;
+  PhaseTimer(mtpc_head* head, cudaStream_t s) : h(head), st(s), idx(0), slot(0) {
+    if (h->ring > 0) {
+      slot = static_cast<int>(h->calls % h->ring);
+      h->ring_phases[slot] = 0;
+      h->calls++;
+    }
+  }
+  cudaEvent_t* pair() { return h->ev + (static_cast<size_t>(slot) * kMaxPhases + idx) * 2; }
+  void begin() { if (h->ring > 0 && idx < kMaxPhases) cudaEventRecord(pair()[0], st); }
   void end() {
-    if (h->timing && idx < kMaxPhases) cudaEventRecord(h->ev[2 * idx + 1], st);
+    if (h->ring > 0 && idx < kMaxPhases) {
+      cudaEventRecord(pair()[1], st);
+      h->ring_phases[slot] = idx + 1;
+    }
     ++idx;
-    h->last_phases = idx;
   }
 };
 
@@ -465,26 +474,45 @@ int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags) {
   return (flags & MTPC_STATUS_TIMEOUT) ? MTPC_ERR_TIMEOUT : MTPC_OK;
 }
 
-int mtpc_set_timing(mtpc_head* head, int32_t enabled) {
-  if (!head) return MTPC_ERR_NULL;
-  if (enabled && !head->ev_ready) {
-    for (int i = 0; i < 2 * kMaxPhases; ++i)
-      if (cudaEventCreate(&head->ev[i]) != cudaSuccess) return MTPC_ERR_CUDA;
-    head->ev_ready = true;
+static void free_timing(mtpc_head* head) {
+  if (head->ev) {
+    for (size_t i = 0; i < static_cast<size_t>(head->ring) * kMaxPhases * 2; ++i) cudaEventDestroy(head->ev[i]);
+    free(head->ev);
+    free(head->ring_phases);
   }
-  head->timing = enabled != 0;
-  head->last_phases = 0;
+  head->ev = nullptr;
+  head->ring_phases = nullptr;
+  head->ring = 0;
+  head->calls = 0;
+}
+
+int mtpc_set_timing(mtpc_head* head, int32_t ring) {
+  if (!head) return MTPC_ERR_NULL;
+  if (ring < 0 || ring > 4096) return MTPC_ERR_SHAPE;
+  free_timing(head);
+  if (ring == 0) return MTPC_OK;
+  const size_t count = static_cast<size_t>(ring) * kMaxPhases * 2;
+  head->ev = static_cast<cudaEvent_t*>(calloc(count, sizeof(cudaEvent_t)));
+  head->ring_phases = static_cast<int*>(calloc(ring, sizeof(int)));
+  if (!head->ev || !head->ring_phases) { free(head->ev); free(head->ring_phases); head->ev = nullptr; return MTPC_ERR_CUDA; }
+  head->ring = ring;
+  for (size_t i = 0; i < count; ++i)
+    if (cudaEventCreate(&head->ev[i]) != cudaSuccess) { head->ring = 0; return MTPC_ERR_CUDA; }
   return MTPC_OK;
 }
 
-int mtpc_get_timing(mtpc_head* head, float* out_ms, int32_t capacity, int32_t* out_count) {
+int mtpc_get_timing(mtpc_head* head, int32_t calls_back, float* out_ms, int32_t capacity, int32_t* out_count) {
   if (!head || !out_ms || !out_count) return MTPC_ERR_NULL;
   *out_count = 0;
-  if (!head->timing) return MTPC_OK;
-  const int nph = head->last_phases < kMaxPhases ? head->last_phases : kMaxPhases;
+  if (head->ring == 0) return MTPC_OK;
+  if (calls_back < 0 || calls_back >= head->ring || static_cast<uint64_t>(calls_back) >= head->calls)
+    return MTPC_ERR_SHAPE;
+  const int slot = static_cast<int>((head->calls - 1 - calls_back) % head->ring);
+  const int nph = head->ring_phases[slot];
   for (int i = 0; i < nph && i < capacity; ++i) {
-    if (cudaEventSynchronize(head->ev[2 * i + 1]) != cudaSuccess) return MTPC_ERR_CUDA;
-    if (cudaEventElapsedTime(&out_ms[i], head->ev[2 * i], head->ev[2 * i + 1]) != cudaSuccess) return MTPC_ERR_CUDA;
+    cudaEvent_t* pair = head->ev + (static_cast<size_t>(slot) * kMaxPhases + i) * 2;
+    if (cudaEventSynchronize(pair[1]) != cudaSuccess) return MTPC_ERR_CUDA;
+    if (cudaEventElapsedTime(&out_ms[i], pair[0], pair[1]) != cudaSuccess) return MTPC_ERR_CUDA;
     *out_count = i + 1;
   }
   return MTPC_OK;
@@ -498,8 +526,7 @@ int mtpc_launch_count(mtpc_head* head, uint64_t* out_count) {
 
 int mtpc_destroy(mtpc_head* head) {
   if (!head) return MTPC_ERR_NULL;
-  if (head->ev_ready)
-    for (int i = 0; i < 2 * kMaxPhases; ++i) cudaEventDestroy(head->ev[i]);
+  free_timing(head);
   delete head;
   return MTPC_OK;
 }
