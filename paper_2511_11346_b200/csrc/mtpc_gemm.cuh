@@ -205,6 +205,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
           }
       }
     }
+    __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
@@ -246,6 +247,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
         while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
       }
     }
+    __syncwarp();
   } else {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;
