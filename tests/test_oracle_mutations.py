@@ -1,0 +1,154 @@
+"""The pins must be sharp: a plausible mistake planted in the oracle (a transposed table, a dropped term, a wrong
+child or slot index, a non-strict comparison) has to break at least one of them. Each mutant is the oracle's
+own source with one textual edit, executed as a throw-away module on the CPU; the pin is a literal enumeration
+or a closed form from test_oracle_pins.py, never the oracle itself."""
+import importlib.util
+import itertools
+import math
+import os
+import types
+
+import numpy as np
+import pytest
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+ORACLE_SRC = os.path.join(os.path.dirname(HERE), "oracle", "mtpc_oracle.py")
+
+_spec = importlib.util.spec_from_file_location("pins_for_mutants", os.path.join(HERE, "test_oracle_pins.py"))
+pins = importlib.util.module_from_spec(_spec)
+_spec.loader.exec_module(pins)
+
+
+def mutant(old: str, new: str) -> types.ModuleType:
+    src = open(ORACLE_SRC).read()
+    assert src.count(old) == 1, f"mutation site not unique or missing: {old!r}"
+    mod = types.ModuleType("oracle_mutant")
+    exec(compile(src.replace(old, new), "oracle_mutant", "exec"), mod.__dict__)
+    return mod
+
+
+def cp_gap(orc):
+    rng = np.random.default_rng(1)
+    n, r, v = 3, 3, 3
+    omega, phi = pins.rand_simplex(rng, r), pins.rand_simplex(rng, n, r, v)
+    gap = 0.0
+    for x in itertools.product(range(v), repeat=n):
+        g = orc.evidence(np.log(phi)[None], np.array([x]))
+        gap = max(gap, abs(orc.cp_eval(np.log(omega)[None], g)[0] - math.log(pins.enum_cp(omega, phi, x))))
+    return gap
+
+
+def hmm_gap(orc):
+    rng = np.random.default_rng(2)
+    n, r, v = 3, 3, 3
+    pi, A, phi = pins.rand_simplex(rng, r), pins.rand_simplex(rng, n - 1, r, r), pins.rand_simplex(rng, n, r, v)
+    gap = 0.0
+    for x in itertools.product(range(v), repeat=n):
+        g = orc.evidence(np.log(phi)[None], np.array([x]))
+        gap = max(gap, abs(orc.hmm_eval(np.log(pi)[None], np.log(A), g)[0] - math.log(pins.enum_hmm(pi, A, phi, x))))
+    return gap
+
+
+def btree_gap(orc, n=8, r=2, v=2):
+    rng = np.random.default_rng(3)
+    omega_root = pins.rand_simplex(rng, r)
+    Omega = {j: pins.rand_simplex(rng, r, r) for j in range(1, n - 1)}
+    phi = pins.rand_simplex(rng, n, r, v)
+    logw = pins.btree_logw(omega_root, Omega, n, r)[None]
+    gap = 0.0
+    for x in list(itertools.product(range(v), repeat=n))[::7]:
+        g = orc.evidence(np.log(phi)[None], np.array([x]))
+        gap = max(gap, abs(orc.btree_eval(logw, g)[0] - math.log(pins.enum_btree(omega_root, Omega, phi, x))))
+    return gap
+
+
+def emission_gap(orc):
+    rng = np.random.default_rng(4)
+    T, n, r, v = 3, 2, 3, 5
+    d = n * r * v
+    W = np.eye(d).reshape(n, r, v, d)
+    h = rng.normal(size=(T, d))
+    import scipy.special
+    want = scipy.special.log_softmax(h.reshape(T, n, r, v), axis=-1)
+    return float(np.abs(orc.emission_logphi(h, W) - want).max())
+
+
+def inv_cdf_wrong(orc):
+    idx, _ = orc.inv_cdf(np.log(np.array([[0.25, 0.5, 0.25]] * 3)), np.array([0.25, 0.75, 0.1]))
+    return 0.0 if idx.tolist() == [1, 2, 0] else 1.0
+
+
+def hmm_sampler_wrong(orc):
+    r, n = 3, 4
+    Ts = np.full((n - 1, r, r), -1e5)
+    for a in range(r):
+        Ts[:, a, (a + 1) % r] = 0.0
+    logw = np.log(np.array([[[1.0 - 2e-9, 1e-9, 1e-9]]]))
+    unit, _ = orc.sample_latents(orc.HMM, logw, Ts, 1, np.full((1, 2 * n), 0.5), n)
+    return 0.0 if unit.tolist() == [[0, 1, 2, 0]] else 1.0
+
+
+def btree_sampler_wrong(orc):
+    n, r = 8, 3
+    Omega = {}
+    for j in range(1, n - 1):
+        t = np.zeros((r, r))
+        for a in range(r):
+            t[a, (a + j) % r] = 1.0
+        Omega[j] = t
+    with np.errstate(divide="ignore"):
+        logw = pins.btree_logw(np.array([1.0, 0.0, 0.0]), Omega, n, r)[None]
+    unit, _ = orc.sample_latents(orc.BTREE, logw, None, 1, np.full((1, 16), 0.5), n)
+    parent, owner = pins.tree_structure(n)
+    z = {0: 0}
+    for j in range(1, n - 1):
+        z[j] = (z[parent[j]] + j) % r
+    return 0.0 if unit[0].tolist() == [z[owner[i]] for i in range(n)] else 1.0
+
+
+def masked_gap(orc):
+    rng = np.random.default_rng(5)
+    logphi = np.log(pins.rand_simplex(rng, 1, 2, 2, 3))
+    g = orc.evidence(logphi, np.array([[-1, 2]]))
+    return float(np.abs(g[0, 0]).max() + np.abs(g[0, 1] - logphi[0, 1, :, 2]).max())
+
+
+MUTANTS = [
+    # (what is planted, old text, new text, pin that must notice)
+    ("mixture weights dropped from Eq. CP", "logsumexp(logw + g.sum(axis=1), axis=-1)", "logsumexp(g.sum(axis=1), axis=-1)", cp_gap),
+    ("product over slots replaced by the first slot", "logw + g.sum(axis=1)", "logw + g[:, 0, :]", cp_gap),
+    ("transition table transposed", "alpha[:, :, None] + logA[i - 1][None, :, :], axis=1)",
+     "alpha[:, :, None] + logA[i - 1].T[None, :, :], axis=1)", hmm_gap),
+    ("forward sum taken over the new state", "logA[i - 1][None, :, :], axis=1)", "logA[i - 1][None, :, :], axis=2)", hmm_gap),
+    ("transition of the wrong step", "alpha[:, :, None] + logA[i - 1]", "alpha[:, :, None] + logA[(i - 1) // 2]", hmm_gap),
+    ("initial weights forgotten", "alpha = logpi + g[:, 0, :]", "alpha = g[:, 0, :]", hmm_gap),
+    ("right child uses the left child's table", "rows = 1 + (child - 1) * r", "rows = 1 + (2 * j + 1 - 1) * r", btree_gap),
+    ("child table transposed", "logsumexp(logOmega + below[:, None, :], axis=-1)",
+     "logsumexp(logOmega + below[:, :, None], axis=1)", btree_gap),
+    ("halves split off centre", "mid = lo + (hi - lo) // 2", "mid = lo + max((hi - lo) // 2 - 1, 1)", btree_gap),
+    ("root weights forgotten", "logsumexp(logw[:, 0, :] + _btree_product", "logsumexp(_btree_product", btree_gap),
+    ("softmax over the units instead of the vocabulary", "return log_softmax(logits, axis=-1)\n\n\ndef sum_unit_logw",
+     "return log_softmax(logits, axis=-2)\n\n\ndef sum_unit_logw", emission_gap),
+    ("non-strict CDF comparison", "(cdf <= u[:, None])", "(cdf < u[:, None])", inv_cdf_wrong),
+    ("sampler walks the transposed chain", "inv_cdf(logA[i - 1][z, :], u[:, i])", "inv_cdf(logA[i - 1][:, z].T, u[:, i])",
+     hmm_sampler_wrong),
+    ("tree sampler conditions on the wrong parent", "parent = (j - 1) // 2", "parent = max(j - 2, 0) // 2", btree_sampler_wrong),
+    ("tree sampler gives tokens to the wrong node", "zs[:, n // 2 - 1 + i // 2]", "zs[:, n // 2 - 1 + (i + 1) // 2 % (n // 2)]",
+     btree_sampler_wrong),
+    ("marginalised byte not set to one", "return np.where((x < 0)[:, :, None], 0.0, g)", "return g", masked_gap),
+]
+
+
+def test_every_pin_passes_on_the_real_oracle():
+    orc = mutant("CP, HMM, BTREE = 0, 1, 2", "CP, HMM, BTREE = 0, 1, 2")        # unmodified copy
+    for pin in {m[3] for m in MUTANTS}:
+        assert pin(orc) < 1e-12, pin.__name__
+
+
+@pytest.mark.parametrize("what,old,new,pin", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_planted_mistake_breaks_a_pin(what, old, new, pin):
+    try:
+        gap = pin(mutant(old, new))
+    except Exception:
+        return                      # a mutant that cannot even run is caught too
+    assert gap > 1e-6, f"the pins do not notice: {what}"
