@@ -47,7 +47,8 @@ enum {
   MTPC_ERR_UNSUPPORTED = -3, /* a valid request this version does not implement (see mtpc_config)     */
   MTPC_ERR_WORKSPACE = -4,   /* workspace too small or misaligned                                     */
   MTPC_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed (includes: no device)               */
-  MTPC_ERR_TIMEOUT = -6      /* mtpc_get_status: a device-side bounded wait gave up                   */
+  MTPC_ERR_TIMEOUT = -6,     /* mtpc_get_status: a device-side bounded wait gave up                   */
+  MTPC_ERR_STATIC_SCRATCH = -7 /* mtpc_window_logprob_static: the call needs more than the built-in array */
 };
 
 /* Bits of the device status word. */
@@ -153,6 +154,42 @@ int mtpc_get_timing(mtpc_head* head, int32_t calls_back, float* out_ms, int32_t 
 
 /* Number of kernels the library launched on behalf of this head since creation (preparation included). */
 int mtpc_launch_count(mtpc_head* head, uint64_t* out_count);
+
+/*
+ * Window log-likelihood without any allocation (the paper has no counterpart: this is a packaging variant of
+ * mtpc_window_logprob, same arithmetic, same kernels, same results).
+ *
+ * Who needs it: code that must not, or cannot, allocate device memory at the point where it wants a
+ * log-likelihood - a plug-in running inside somebody else's memory pool, a callback on a serving thread that
+ * is forbidden to call cudaMalloc because that call synchronises the device, a process whose memory budget was
+ * handed out in full at start-up. mtpc_window_logprob asks such callers for a workspace they have no way to
+ * obtain. This entry point needs neither a head nor a workspace: its scratch (a status word, the
+ * log-softmaxed HMM transitions, G [T, n, r] and log omega [T, S*r], all fp32) lives in one static device array
+ * of MTPC_STATIC_SCRATCH_BYTES that is part of the library image. Every GPU that loads the library therefore
+ * holds those bytes until the process exits, whether or not this function is ever called. It calls no
+ * cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   cfg        family, n, r, v, d as for mtpc_create_head; io_dtype must be MTPC_BF16 (MTPC_ERR_UNSUPPORTED
+ *              otherwise: fp32 inputs would need a rounded copy of the weights); max_positions,
+ *              max_windows_per_pos are ignored; flags must be 0.
+ *   W_emit, W_sum, T_static, hidden, targets, out_logprob: dev, exactly as for mtpc_create_head and
+ *              mtpc_window_logprob; all caller-owned, read or written only by the work this call enqueues.
+ *   out_status dev uint32 or NULL: receives this call's MTPC_STATUS_* bits (stream-ordered, like the outputs).
+ *   T          T == 0 is a no-op. If 256 + 4*(n-1)*r*r (HMM) + 4*T*n*r + 4*T*S*r bytes (each term rounded up
+ *              to 256) exceed MTPC_STATIC_SCRATCH_BYTES the call returns MTPC_ERR_STATIC_SCRATCH and
+ *              enqueues nothing; split the positions over several calls then.
+ *
+ * First call on a device: it looks up the array's device address (once per device, with that device current)
+ * and may make the CUDA runtime load the library's kernels. Make that first call outside any stream capture.
+ * All calls on one device share the one array, and the array keeps the previous call's contents; the call
+ * clears the part that has to start at zero (the status word) itself. Two calls whose work overlaps on the
+ * GPU (different streams, or different threads without ordering) race on the array: order them on one stream
+ * or with events. Asynchronous like mtpc_window_logprob: the outputs are ready when `stream` reaches them.
+ */
+#define MTPC_STATIC_SCRATCH_BYTES (16u << 20) /* 16 MiB: configs up to T*(n*r + S*r) = 4.19 M fp32 entries */
+int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_emit, const void* W_sum,
+                               const float* T_static, const void* hidden, const int32_t* targets, int32_t T,
+                               float* out_logprob, uint32_t* out_status, void* stream);
 
 /* Frees the host-side object (the workspace and the weights stay the caller's). Synchronises nothing. */
 int mtpc_destroy(mtpc_head* head);

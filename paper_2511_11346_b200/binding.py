@@ -19,8 +19,10 @@ STATUS_BAD_TARGET, STATUS_BAD_UNIFORM, STATUS_TIMEOUT = 1, 2, 4
 EXPORTS = [
     "mtpc_workspace_bytes", "mtpc_create_head", "mtpc_window_logprob", "mtpc_draft_sample",
     "mtpc_window_logprob_host", "mtpc_draft_sample_host", "mtpc_get_status", "mtpc_set_timing", "mtpc_get_timing",
-    "mtpc_launch_count", "mtpc_destroy", "mtpc_status_string",
+    "mtpc_launch_count", "mtpc_destroy", "mtpc_status_string", "mtpc_window_logprob_static",
 ]
+STATIC_SCRATCH_BYTES = 16 << 20
+ERR_STATIC_SCRATCH = -7
 
 
 class MtpcConfig(ctypes.Structure):
@@ -59,6 +61,7 @@ def lib() -> ctypes.CDLL:
     L.mtpc_get_timing.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_float), i32, ctypes.POINTER(i32)]
     L.mtpc_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
     L.mtpc_destroy.argtypes = [vp]
+    L.mtpc_window_logprob_static.argtypes = [ctypes.POINTER(MtpcConfig), vp, vp, vp, vp, vp, i32, vp, vp, vp]
     L.mtpc_status_string.argtypes = [ctypes.c_int]
     L.mtpc_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -91,6 +94,20 @@ def mtpc_workspace_bytes(cfg: MtpcConfig) -> int:
     out = ctypes.c_size_t(0)
     _check(lib().mtpc_workspace_bytes(ctypes.byref(cfg), ctypes.byref(out)), "mtpc_workspace_bytes")
     return out.value
+
+
+def mtpc_window_logprob_static(family: int, n: int, r: int, v: int, d: int, W_emit, W_sum, T_static, hidden, targets,
+                               out_logprob, out_status=None, stream=None) -> None:
+    """Window log-likelihood through the entry point that allocates nothing: no head, no workspace. For callers
+    that cannot allocate device memory where they need the result (inside another component's memory pool, on
+    a thread where a synchronising cudaMalloc is forbidden). The library's one static scratch array per device is
+    shared by all such calls, so do not let two of them overlap on the GPU. bf16 tensors only; raises MtpcError
+    with code ERR_STATIC_SCRATCH when the positions do not fit the array (split them over several calls)."""
+    cfg = MtpcConfig(family, n, r, v, d, MTPC_BF16, 1, 1, 0)
+    T = hidden.shape[0]
+    _check(lib().mtpc_window_logprob_static(ctypes.byref(cfg), _ptr(W_emit), _ptr(W_sum), _ptr(T_static), _ptr(hidden),
+                                            _ptr(targets), T, _ptr(out_logprob), _ptr(out_status), _stream(stream)),
+           "mtpc_window_logprob_static")
 
 
 class MtpcHead:

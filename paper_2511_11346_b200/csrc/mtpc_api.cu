@@ -540,8 +540,111 @@ const char* mtpc_status_string(int code) {
     case MTPC_ERR_WORKSPACE: return "workspace too small or misaligned";
     case MTPC_ERR_CUDA: return "a CUDA call failed (no sm_100 device, launch error, or driver entry point missing)";
     case MTPC_ERR_TIMEOUT: return "a device-side bounded wait expired";
+    case MTPC_ERR_STATIC_SCRATCH:
+      return "the call needs more scratch than the library's built-in static array holds (mtpc_window_logprob_static)";
     default: return "unknown status code";
   }
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------------------
+// mtpc_window_logprob_static: the window log-likelihood for callers that have no device allocator at hand.
+// All scratch (status word, log-softmaxed HMM transitions, G, log omega) is carved out of one file-scope device
+// array, so the call needs neither a head nor a caller-made workspace and allocates nothing.
+// ------------------------------------------------------------------------------------------------------------
+namespace {
+
+// Every GPU that loads the library holds this array until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[MTPC_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices];   // device address of the array on each device, 0 = not looked up yet
+
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address: the address the
+// kernels need comes from cudaGetSymbolAddress, asked once per device with that device current.
+int static_scratch_address(unsigned char** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MTPC_ERR_CUDA;
+  void* p = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return MTPC_ERR_CUDA;
+    __atomic_store_n(&g_static_scratch_addr[dev], p, __ATOMIC_RELEASE);   // every thread gets the same answer
+  }
+  *out = static_cast<unsigned char*>(p);
+  return MTPC_OK;
+}
+
+}  // namespace
+
+extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_emit, const void* W_sum,
+                                          const float* T_static, const void* hidden, const int32_t* targets,
+                                          int32_t T, float* out_logprob, uint32_t* out_status, void* stream) {
+  if (!cfg) return MTPC_ERR_NULL;
+  if (cfg->io_dtype != MTPC_BF16) return MTPC_ERR_UNSUPPORTED;   // fp32 inputs would need rounded copies of the weights
+  if (T < 0) return MTPC_ERR_SHAPE;
+  mtpc_config c = *cfg;
+  c.max_positions = T > 0 ? T : 1;
+  c.max_windows_per_pos = 1;
+  Layout L;
+  int rc = plan(c, &L);
+  if (rc != MTPC_OK) return rc;
+  // Carve only what this call needs: [status | logA (HMM) | G | log omega].
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  L.off_status = take(256);
+  L.off_logA = take(c.family == MTPC_HMM ? static_cast<size_t>(c.n - 1) * c.r * c.r * 4 : 0);
+  L.off_G = take(static_cast<size_t>(c.max_positions) * c.n * c.r * 4);
+  L.off_logw = take(static_cast<size_t>(c.max_positions) * L.sum_rows * 4);
+  L.off_sel = L.off_wemit = L.off_wsum = L.off_hidden = 0;                               // unused by this call
+  L.off_h_hidden = L.off_h_targets = L.off_h_uniforms = L.off_h_bytes = L.off_h_out = 0;
+  L.total = off;
+  if (L.total > static_cast<size_t>(MTPC_STATIC_SCRATCH_BYTES)) return MTPC_ERR_STATIC_SCRATCH;
+  if (T == 0) return MTPC_OK;
+  if (!W_emit || !W_sum || !hidden || !targets || !out_logprob) return MTPC_ERR_NULL;
+  if (c.family == MTPC_HMM && c.n > 1 && !T_static) return MTPC_ERR_NULL;
+
+  int dev = 0, cc_major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MTPC_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || cc_major != 10)
+    return MTPC_ERR_CUDA;
+  unsigned char* scratch = nullptr;
+  if ((rc = static_scratch_address(&scratch)) != MTPC_OK) return rc;
+
+  mtpc_head h;                       // host-side bookkeeping only, lives for the duration of this call
+  memset(&h, 0, sizeof(h));
+  h.cfg = c;
+  h.L = L;
+  h.ws = scratch;
+  h.W_emit_bf16 = W_emit;
+  h.W_sum_bf16 = W_sum;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bool fail = cudaDeviceGetAttribute(&h.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess;
+  h.gemm_smem = L.stages * L.stage_bytes + 1024 + static_cast<int>(sizeof(GemmControl));
+  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               h.gemm_smem) != cudaSuccess;
+  if (c.family == MTPC_BTREE) {
+    const int smem = kCircuitWarps * ((c.n - 1) * c.r + c.r * (c.r + 1)) * 4;
+    if (smem > 48 * 1024)
+      fail |= cudaFuncSetAttribute(circuit_btree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+              cudaSuccess;
+  }
+  // The array keeps whatever the previous call left in it. Only the status word has to start at zero; G, log omega
+  // and logA are fully rewritten for the rows this call reads.
+  fail |= cudaMemsetAsync(scratch + L.off_status, 0, 256, st) != cudaSuccess;
+  if (fail) return MTPC_ERR_CUDA;
+  if (c.family == MTPC_HMM && c.n > 1) {
+    const int rows = (c.n - 1) * c.r;
+    log_softmax_rows_kernel<<<(rows + 127) / 128, 128, 0, st>>>(T_static, at<float>(&h, L.off_logA), rows, c.r);
+    if (check_launch() != MTPC_OK) return MTPC_ERR_CUDA;
+  }
+  rc = make_tmap(&h.tm_emit, W_emit, static_cast<uint64_t>(c.n) * c.r * c.v, c.d, L.chunk_cols);
+  if (rc == MTPC_OK) rc = make_tmap(&h.tm_sum, W_sum, L.sum_rows, c.d, L.sum_cols);
+  if (rc != MTPC_OK) return rc;
+  rc = window_logprob_impl(&h, hidden, targets, T, out_logprob, st);
+  if (rc != MTPC_OK) return rc;
+  if (out_status &&
+      cudaMemcpyAsync(out_status, scratch + L.off_status, 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return MTPC_ERR_CUDA;
+  return MTPC_OK;
+}
