@@ -24,15 +24,43 @@ constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 
+// How one launch of the projection kernel tiles the N axis and uses shared / tensor memory.
+struct Tiling {
+  int tile_cols;        // accumulator width of an emission tile
+  int group_units;      // emission units per work group
+  int group_tiles;      // tiles of a full group
+  int num_groups;       // groups covering all n*r units
+  int slot_stride, num_slots, stages, stage_bytes, smem;
+};
+
 struct Layout {
   // derived sizes
-  int S, sum_rows, chunk_cols, chunks_per_unit, sum_cols, sum_tiles, slot_stride, num_slots, stages, stage_bytes;
+  int S, sum_rows, sum_cols, sum_tiles;
+  Tiling lp;            // log-likelihood mode: 256-column tiles over the flattened (i,k,b) axis
+  Tiling sm;            // sampling mode: one unit per group, equal tiles of <= 256 columns
   size_t max_windows;
   // workspace offsets (bytes)
   size_t off_status, off_wemit, off_wsum, off_hidden, off_logA, off_G, off_logw, off_sel;
   size_t off_h_hidden, off_h_targets, off_h_uniforms, off_h_bytes, off_h_out;
   size_t total;
 };
+
+int gcd_int(int a, int b) { while (b) { int t = a % b; a = b; b = t; } return a; }
+
+// Shared-memory ring and TMEM slots for tiles of `tile_cols` emission columns and `sum_cols` sum columns.
+bool fit_tiling(Tiling* t, int sum_cols) {
+  const int widest = t->tile_cols > sum_cols ? t->tile_cols : sum_cols;
+  t->slot_stride = (widest + 31) / 32 * 32;
+  t->num_slots = kTmemCols / t->slot_stride;
+  if (t->num_slots > kMaxSlots) t->num_slots = kMaxSlots;
+  t->stage_bytes = (kABytes + widest * kBlockK * 2 + 1023) / 1024 * 1024;   // A tile + one B tile
+  const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
+  int stages = (kSmemLimit - ctl) / t->stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  t->stages = stages;
+  t->smem = stages * t->stage_bytes + ctl;
+  return stages >= 2 && t->num_slots >= 2;
+}
 
 int plan(const mtpc_config& c, Layout* L) {
   if (c.family < MTPC_CP || c.family > MTPC_BTREE) return MTPC_ERR_SHAPE;
@@ -50,29 +78,32 @@ int plan(const mtpc_config& c, Layout* L) {
 
   L->S = (c.family == MTPC_BTREE) ? 1 + (c.n - 2) * c.r : 1;
   L->sum_rows = L->S * c.r;
-  // emission unit -> equal chunks of <= 256 columns, each a multiple of 16
-  int chunks = (c.v + 255) / 256;
-  while (c.v % chunks != 0 || (c.v / chunks) % 16 != 0) ++chunks;
-  L->chunks_per_unit = chunks;
-  L->chunk_cols = c.v / chunks;
   // sum tile: a multiple of both r and 16, at most 256 columns
   const int unit = c.r > 16 ? c.r : 16;
   int sum_cols = (L->sum_rows + unit - 1) / unit * unit;
   if (sum_cols > 256) sum_cols = 256 / unit * unit;
   L->sum_cols = sum_cols;
   L->sum_tiles = (L->sum_rows + sum_cols - 1) / sum_cols;
-  int widest = L->chunk_cols > sum_cols ? L->chunk_cols : sum_cols;
-  L->slot_stride = (widest + 31) / 32 * 32;
-  L->num_slots = kTmemCols / L->slot_stride;
-  if (L->num_slots > kMaxSlots) L->num_slots = kMaxSlots;
-  if (L->num_slots < chunks) return MTPC_ERR_UNSUPPORTED;
-  const int brows = chunks * L->chunk_cols > sum_cols ? chunks * L->chunk_cols : sum_cols;
-  L->stage_bytes = kABytes + brows * kBlockK * 2;          // multiples of 1024 (rows are multiples of 16)
-  L->stage_bytes = (L->stage_bytes + 1023) / 1024 * 1024;
-  int stages = (kSmemLimit - 1024 - static_cast<int>(sizeof(GemmControl))) / L->stage_bytes;
-  if (stages > kMaxStages) stages = kMaxStages;
-  if (stages < 2) return MTPC_ERR_UNSUPPORTED;
-  L->stages = stages;
+  const int emit_units = c.n * c.r;
+  // sampling: emission unit -> equal tiles of <= 256 columns, each a multiple of 16, all in TMEM at once
+  int chunks = (c.v + 255) / 256;
+  while (c.v % chunks != 0 || (c.v / chunks) % 16 != 0) ++chunks;
+  L->sm.tile_cols = c.v / chunks;
+  L->sm.group_units = 1;
+  L->sm.group_tiles = chunks;
+  L->sm.num_groups = emit_units;
+  if (!fit_tiling(&L->sm, sum_cols) || L->sm.num_slots < chunks) return MTPC_ERR_UNSUPPORTED;
+  // log-likelihood: 256-column tiles; a group is the shortest run of whole units that is a whole number of tiles
+  const int lcm = c.v / gcd_int(c.v, 256) * 256;
+  L->lp.tile_cols = 256;
+  L->lp.group_units = lcm / c.v;
+  L->lp.group_tiles = lcm / 256;
+  if (L->lp.group_units > emit_units) {   // fewer units than one full group: a single, partial group
+    L->lp.group_units = emit_units;
+    L->lp.group_tiles = (emit_units * c.v + 255) / 256;
+  }
+  L->lp.num_groups = (emit_units + L->lp.group_units - 1) / L->lp.group_units;
+  if (!fit_tiling(&L->lp, sum_cols)) return MTPC_ERR_UNSUPPORTED;
 
   L->max_windows = static_cast<size_t>(c.max_positions) * c.max_windows_per_pos;
   const size_t elt = c.io_dtype == MTPC_F32 ? 4 : 2;
@@ -135,9 +166,8 @@ struct mtpc_head {
   uint8_t* ws;
   const void* W_emit_bf16;
   const void* W_sum_bf16;
-  CUtensorMap tm_emit, tm_sum;
+  CUtensorMap tm_emit_lp, tm_emit_sm, tm_sum;   // W_emit with the box of either tiling; W_sum
   int num_sms;
-  int gemm_smem;
   int ring;                 // calls whose per-kernel events are retained (0 = timing off)
   cudaEvent_t* ev;          // [ring][kMaxPhases][2]
   int* ring_phases;         // [ring] phases recorded by the call in that slot
@@ -174,33 +204,34 @@ struct PhaseTimer {
 
 int check_launch() { return cudaGetLastError() == cudaSuccess ? MTPC_OK : MTPC_ERR_CUDA; }
 
-// Launch the projection kernel over units [unit_begin, unit_begin + unit_count) for `rows` positions.
-int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int wpp, int unit_begin, int unit_count,
+// Launch the projection kernel for `rows` positions over the emission groups (with_emit) and / or the sum tiles.
+int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int wpp, bool with_emit, bool with_sum,
                 const int* targets, const float* uniforms, int* out_bytes, cudaStream_t st) {
-  if (rows <= 0 || unit_count <= 0) return MTPC_OK;
+  if (rows <= 0 || (!with_emit && !with_sum)) return MTPC_OK;
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
+  const Tiling& tl = mode == kModeSample ? L.sm : L.lp;
   GemmParams p;
   memset(&p, 0, sizeof(p));
   int rc = make_tmap(&p.tm_a, hidden_bf16, static_cast<uint64_t>(rows), static_cast<uint64_t>(c.d), kBlockM);
   if (rc != MTPC_OK) return rc;
-  p.tm_emit = h->tm_emit;
+  p.tm_emit = mode == kModeSample ? h->tm_emit_sm : h->tm_emit_lp;
   p.tm_sum = h->tm_sum;
   p.T = rows;
   p.m_tiles = (rows + kBlockM - 1) / kBlockM;
   p.kblocks = c.d / kBlockK;
   p.n = c.n; p.r = c.r; p.v = c.v;
   p.emit_units = c.n * c.r;
-  p.unit_begin = unit_begin;
-  p.unit_count = unit_count;
-  p.chunk_cols = L.chunk_cols;
-  p.chunks_per_unit = L.chunks_per_unit;
+  p.num_groups = with_emit ? tl.num_groups : 0;
+  p.group_units = tl.group_units;
+  p.tile_cols = tl.tile_cols;
+  p.num_sum_tiles = with_sum ? L.sum_tiles : 0;
   p.sum_cols = L.sum_cols;
   p.sum_rows = L.sum_rows;
-  p.slot_stride = L.slot_stride;
-  p.num_slots = L.num_slots;
-  p.stages = L.stages;
-  p.stage_bytes = L.stage_bytes;
+  p.slot_stride = tl.slot_stride;
+  p.num_slots = tl.num_slots;
+  p.stages = tl.stages;
+  p.stage_bytes = tl.stage_bytes;
   p.wpp = wpp;
   p.targets = targets;
   p.G = at<float>(h, L.off_G);
@@ -209,12 +240,12 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   p.uniforms = uniforms;
   p.out_bytes = out_bytes;
   p.status = at<unsigned>(h, L.off_status);
-  const long long tiles = static_cast<long long>(p.m_tiles) * unit_count;
-  const int grid = static_cast<int>(tiles < h->num_sms ? tiles : h->num_sms);
+  const long long items = static_cast<long long>(p.m_tiles) * (p.num_groups + p.num_sum_tiles);
+  const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
   if (mode == kModeLogprob)
-    mtpc_gemm_kernel<kModeLogprob><<<grid, kGemmThreads, h->gemm_smem, st>>>(p);
+    mtpc_gemm_kernel<kModeLogprob><<<grid, kGemmThreads, tl.smem, st>>>(p);
   else
-    mtpc_gemm_kernel<kModeSample><<<grid, kGemmThreads, h->gemm_smem, st>>>(p);
+    mtpc_gemm_kernel<kModeSample><<<grid, kGemmThreads, tl.smem, st>>>(p);
   h->launches++;
   return check_launch();
 }
@@ -262,7 +293,7 @@ int window_logprob_impl(mtpc_head* h, const void* hidden, const int32_t* targets
   if (rc != MTPC_OK) return rc;
   PhaseTimer pt(h, st);
   pt.begin();
-  rc = launch_gemm(h, kModeLogprob, hb, T, 1, 0, h->cfg.n * h->cfg.r + h->L.sum_tiles, targets, nullptr, nullptr, st);
+  rc = launch_gemm(h, kModeLogprob, hb, T, 1, true, true, targets, nullptr, nullptr, st);
   pt.end();
   if (rc != MTPC_OK) return rc;
   pt.begin();
@@ -279,11 +310,10 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   const void* hb = nullptr;
   int rc = stage_hidden(h, hidden, P, &hb, st);
   if (rc != MTPC_OK) return rc;
-  const int emit_units = c.n * c.r;
   PhaseTimer pt(h, st);
   // 1. sum-unit weights (Sec. 3.3) -> 2. latent draws at the sum units (Algorithm 1)
   pt.begin();
-  rc = launch_gemm(h, kModeLogprob, hb, P, 1, emit_units, L.sum_tiles, nullptr, nullptr, nullptr, st);
+  rc = launch_gemm(h, kModeLogprob, hb, P, 1, false, true, nullptr, nullptr, nullptr, st);
   pt.end();
   if (rc != MTPC_OK) return rc;
   pt.begin();
@@ -295,12 +325,12 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   if ((rc = check_launch()) != MTPC_OK) return rc;
   // 3. byte draws at the selected input units
   pt.begin();
-  rc = launch_gemm(h, kModeSample, hb, P, wpp, 0, emit_units, nullptr, uniforms, out_bytes, st);
+  rc = launch_gemm(h, kModeSample, hb, P, wpp, true, false, nullptr, uniforms, out_bytes, st);
   pt.end();
   if (rc != MTPC_OK) return rc;
   // 4. evidence of the drafted bytes under every unit -> 5. joint log-prob with the latents summed out
   pt.begin();
-  rc = launch_gemm(h, kModeLogprob, hb, P, wpp, 0, emit_units, out_bytes, nullptr, nullptr, st);
+  rc = launch_gemm(h, kModeLogprob, hb, P, wpp, true, false, out_bytes, nullptr, nullptr, st);
   pt.end();
   if (rc != MTPC_OK) return rc;
   pt.begin();
@@ -349,11 +379,11 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   h->ws = static_cast<uint8_t*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   bool fail = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess;
-  h->gemm_smem = L.stages * L.stage_bytes + 1024 + static_cast<int>(sizeof(GemmControl));
+  // the attribute is per function, not per head: always ask for the full 227 KB so that heads do not undo each other
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               h->gemm_smem) != cudaSuccess;
+                               kSmemLimit) != cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeSample>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               h->gemm_smem) != cudaSuccess;
+                               kSmemLimit) != cudaSuccess;
   if (cfg->family == MTPC_BTREE) {
     const int smem = kCircuitWarps * ((cfg->n - 1) * cfg->r + cfg->r * (cfg->r + 1)) * 4;
     if (smem > 48 * 1024)
@@ -383,7 +413,9 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
     h->launches++;
   }
   if (check_launch() != MTPC_OK) { delete h; return MTPC_ERR_CUDA; }
-  rc = make_tmap(&h->tm_emit, h->W_emit_bf16, static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v, cfg->d, L.chunk_cols);
+  const uint64_t emit_rows = static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v;
+  rc = make_tmap(&h->tm_emit_lp, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols);
+  if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols);
   if (rc != MTPC_OK) { delete h; return rc; }
   *out = h;
@@ -620,9 +652,8 @@ extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_
   h.W_sum_bf16 = W_sum;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   bool fail = cudaDeviceGetAttribute(&h.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess;
-  h.gemm_smem = L.stages * L.stage_bytes + 1024 + static_cast<int>(sizeof(GemmControl));
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               h.gemm_smem) != cudaSuccess;
+                               kSmemLimit) != cudaSuccess;
   if (c.family == MTPC_BTREE) {
     const int smem = kCircuitWarps * ((c.n - 1) * c.r + c.r * (c.r + 1)) * 4;
     if (smem > 48 * 1024)
@@ -638,7 +669,7 @@ extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_
     log_softmax_rows_kernel<<<(rows + 127) / 128, 128, 0, st>>>(T_static, at<float>(&h, L.off_logA), rows, c.r);
     if (check_launch() != MTPC_OK) return MTPC_ERR_CUDA;
   }
-  rc = make_tmap(&h.tm_emit, W_emit, static_cast<uint64_t>(c.n) * c.r * c.v, c.d, L.chunk_cols);
+  rc = make_tmap(&h.tm_emit_lp, W_emit, static_cast<uint64_t>(c.n) * c.r * c.v, c.d, L.lp.tile_cols);
   if (rc == MTPC_OK) rc = make_tmap(&h.tm_sum, W_sum, L.sum_rows, c.d, L.sum_cols);
   if (rc != MTPC_OK) return rc;
   rc = window_logprob_impl(&h, hidden, targets, T, out_logprob, st);

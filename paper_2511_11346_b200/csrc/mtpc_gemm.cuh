@@ -9,9 +9,14 @@
 //   warp 1      allocates the 512 TMEM columns, issues tcgen05.mma (M=128, N=chunk, K=16) from one thread.
 //   warps 2..5  epilogue; warp w reads TMEM lanes 32*(w%4)..+31, one thread per position (row), so every
 //               row-wise reduction over the vocabulary is a plain in-thread loop.
-// A work item ("tile") is 128 positions x one unit: emission unit (i,k) = v logit columns, split into
-// `chunks_per_unit` accumulators of `chunk_cols` columns (v=320 -> 2 x 160, v=256 -> 1 x 256), or one tile
-// of `sum_cols` sum-unit columns. Accumulators live in a ring of TMEM slots, so the epilogue of one tile
+// The N axis of the GEMM is the flattened (slot i, unit k, byte b) row index of W_emit. A work item is 128
+// positions x one "group": `group_units` consecutive emission units = a run of rows that starts at a unit
+// boundary, covered by accumulator tiles of `tile_cols` columns. The log-likelihood mode uses 256-column tiles
+// whatever v is (v=320: 4 units = 1280 rows = 5 tiles; v=256: 1 unit = 1 tile): a tile may then hold the end
+// of one unit and the start of the next, and the epilogue carries its running max / sum across tiles and
+// closes a unit whenever its v-th column has been consumed. The sampling mode needs a whole unit on chip at
+// once and uses one unit per group (v=320 -> 2 tiles of 160). Sum-unit rows form work items of their own
+// (one tile of `sum_cols` columns). Accumulators live in a ring of TMEM slots, so the epilogue of one tile
 // overlaps the MMAs of the next. Every barrier wait is bounded: when one runs out the CTA raises
 // MTPC_STATUS_TIMEOUT in the status word, drains its copies, frees its TMEM and returns.
 #pragma once
@@ -35,13 +40,15 @@ enum { kModeLogprob = 0, kModeSample = 1 };
 
 struct GemmParams {
   CUtensorMap tm_a;      // hidden  [T, d]        box 64 x 128
-  CUtensorMap tm_emit;   // W_emit  [n*r*v, d]    box 64 x chunk_cols
+  CUtensorMap tm_emit;   // W_emit  [n*r*v, d]    box 64 x tile_cols
   CUtensorMap tm_sum;    // W_sum   [S*r, d]      box 64 x sum_cols
   int T, m_tiles, kblocks;
   int n, r, v;
   int emit_units;                    // n * r
-  int unit_begin, unit_count;        // units [unit_begin, unit_begin + unit_count); >= emit_units = sum tiles
-  int chunk_cols, chunks_per_unit;
+  int num_groups;                    // emission groups in this launch (0: sum tiles only)
+  int group_units;                   // emission units per full group (the last group may hold fewer)
+  int tile_cols;                     // accumulator width of an emission tile
+  int num_sum_tiles;                 // sum tiles in this launch (0: emission groups only)
   int sum_cols, sum_rows;            // sum tile width; S * r
   int slot_stride, num_slots;
   int stages, stage_bytes;
@@ -103,16 +110,27 @@ __device__ __forceinline__ bool bounded_wait_warp(uint32_t bar, uint32_t parity,
 }
 
 struct TileCoord {
-  int unit, mt, is_sum, chunks, cols, brow0;
+  int mt, is_sum, ntiles, cols, brow0, unit0, nunits;
 };
-__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile) {
+// Work items: m-tile fastest, so the CTAs that run at the same time share one group's weights through L2.
+__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int item) {
   TileCoord c;
-  c.unit = p.unit_begin + tile / p.m_tiles;
-  c.mt = tile % p.m_tiles;
-  c.is_sum = c.unit >= p.emit_units;
-  c.chunks = c.is_sum ? 1 : p.chunks_per_unit;
-  c.cols = c.is_sum ? p.sum_cols : p.chunk_cols;
-  c.brow0 = c.is_sum ? (c.unit - p.emit_units) * p.sum_cols : c.unit * p.v;
+  const int g = item / p.m_tiles;
+  c.mt = item % p.m_tiles;
+  c.is_sum = g >= p.num_groups;
+  if (c.is_sum) {
+    c.ntiles = 1;
+    c.cols = p.sum_cols;
+    c.brow0 = (g - p.num_groups) * p.sum_cols;
+    c.unit0 = g - p.num_groups;   // index of the sum tile
+    c.nunits = 0;
+  } else {
+    c.unit0 = g * p.group_units;
+    c.nunits = min(p.group_units, p.emit_units - c.unit0);
+    c.cols = p.tile_cols;
+    c.brow0 = c.unit0 * p.v;
+    c.ntiles = (c.nunits * p.v + p.tile_cols - 1) / p.tile_cols;
+  }
   return c;
 }
 
@@ -145,7 +163,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int num_tiles = p.unit_count * p.m_tiles;
+  const int num_items = (p.num_groups + p.num_sum_tiles) * p.m_tiles;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -177,22 +195,22 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const TileCoord tc = tile_coord(p, tile);
+      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+        const TileCoord tc = tile_coord(p, item);
         const CUtensorMap* tmb = tc.is_sum ? &p.tm_sum : &p.tm_emit;
-        const uint32_t bytes = kABytes + tc.chunks * tc.cols * (kBlockK * 2);
-        for (int kb = 0; kb < p.kblocks; ++kb) {
-          if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
-          const uint32_t full = smem_u32(&ctl->full[stage]);
-          const uint32_t a_dst = tiles_addr + stage * p.stage_bytes;
-          mbar_arrive_expect_tx(full, bytes);
-          tma_load_2d(a_dst, &p.tm_a, full, kb * kBlockK, tc.mt * kBlockM);
-          for (int c = 0; c < tc.chunks; ++c)
-            tma_load_2d(a_dst + kABytes + c * tc.cols * (kBlockK * 2), tmb, full, kb * kBlockK,
-                        tc.brow0 + c * tc.cols);
-          issued_mask |= 1u << stage;
-          phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
-          if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
+        const uint32_t bytes = kABytes + tc.cols * (kBlockK * 2);
+        for (int t = 0; t < tc.ntiles && ok; ++t) {
+          for (int kb = 0; kb < p.kblocks; ++kb) {
+            if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
+            const uint32_t full = smem_u32(&ctl->full[stage]);
+            const uint32_t a_dst = tiles_addr + stage * p.stage_bytes;
+            mbar_arrive_expect_tx(full, bytes);
+            tma_load_2d(a_dst, &p.tm_a, full, kb * kBlockK, tc.mt * kBlockM);
+            tma_load_2d(a_dst + kABytes, tmb, full, kb * kBlockK, tc.brow0 + t * tc.cols);
+            issued_mask |= 1u << stage;
+            phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
+            if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
+          }
         }
       }
       if (!ok) {   // give the copies still in flight a bounded chance to land before the CTA goes away
@@ -211,35 +229,32 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, use = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const TileCoord tc = tile_coord(p, tile);
+      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+        const TileCoord tc = tile_coord(p, item);
         const uint32_t idesc = umma_idesc_bf16(kBlockM, tc.cols);
-        for (int kb = 0; kb < p.kblocks && ok; ++kb) {
-          if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
+        for (int t = 0; t < tc.ntiles && ok; ++t, ++use) {
+          const uint32_t slot = use % p.num_slots;
+          if (!bounded_wait(smem_u32(&ctl->tempty[slot]), ((use / p.num_slots) & 1u) ^ 1u, ctl, p.status)) {
+            ok = false;
+            break;
+          }
           tc_fence_after();
-          const uint32_t a_addr = tiles_addr + stage * p.stage_bytes;
-          const uint64_t a_desc = umma_smem_desc_sw128(a_addr);
-          for (int c = 0; c < tc.chunks; ++c) {
-            const uint32_t u = use + c;
-            const uint32_t slot = u % p.num_slots;
-            if (kb == 0) {
-              const uint32_t sphase = (u / p.num_slots) & 1u;
-              if (!bounded_wait(smem_u32(&ctl->tempty[slot]), sphase ^ 1u, ctl, p.status)) { ok = false; break; }
-              tc_fence_after();
-            }
-            const uint64_t b_desc = umma_smem_desc_sw128(a_addr + kABytes + c * tc.cols * (kBlockK * 2));
-            const uint32_t d_tmem = tmem_base + slot * p.slot_stride;
+          const uint32_t d_tmem = tmem_base + slot * p.slot_stride;
+          for (int kb = 0; kb < p.kblocks; ++kb) {
+            if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_addr = tiles_addr + stage * p.stage_bytes;
+            const uint64_t a_desc = umma_smem_desc_sw128(a_addr);
+            const uint64_t b_desc = umma_smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
             for (int kk = 0; kk < kBlockK / 16; ++kk)   // +32 bytes per K=16 step inside the swizzled row
               umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+            umma_commit(smem_u32(&ctl->empty[stage]));
+            if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
           }
           if (!ok) break;
-          umma_commit(smem_u32(&ctl->empty[stage]));
-          if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
+          umma_commit(smem_u32(&ctl->tfull[slot]));
         }
-        if (!ok) break;
-        for (int c = 0; c < tc.chunks; ++c) umma_commit(smem_u32(&ctl->tfull[(use + c) % p.num_slots]));
-        use += tc.chunks;
       }
       if (!ok) {   // wait (bounded) for the MMAs already issued before TMEM is freed
         umma_commit(smem_u32(&ctl->drain));
@@ -254,8 +269,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     uint32_t use = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-      const TileCoord tc = tile_coord(p, tile);
+    for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+      const TileCoord tc = tile_coord(p, item);
       const int row = tc.mt * kBlockM + quarter * 32 + lane;
       const bool valid = row < p.T;
       const int nbatch = tc.cols / 16;
@@ -269,7 +284,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
         }
         tc_fence_after();
         const uint32_t tcol = lane_base + slot * p.slot_stride;
-        const int col_base = (tc.unit - p.emit_units) * p.sum_cols;
+        const int col_base = tc.unit0 * p.sum_cols;
         float* dst = p.logw + static_cast<size_t>(valid ? row : 0) * p.sum_rows;
         if (p.r <= 16) {
           for (int b = 0; b < nbatch; ++b) {
@@ -323,28 +338,27 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
         continue;
       }
 
-      const int slot_i = tc.unit / p.r;   // window slot i
-      const int k = tc.unit % p.r;        // input unit k
-
       if (MODE == kModeLogprob) {
-        // ---- log phi at the target byte: online log-sum-exp over the v columns + gather
-        float m = -CUDART_INF_F, s = 0.f, tval = 0.f;
-        int tgt = -1;
+        // ---- log phi at the target byte: online log-sum-exp over the v columns of each unit + gather. The
+        // running (m, s) and the gathered logit live across tile boundaries; a unit is closed when its v-th
+        // column has been consumed.
         const size_t wrow0 = static_cast<size_t>(valid ? row : 0) * p.wpp;
-        if (p.wpp == 1 && valid) tgt = p.targets[wrow0 * p.n + slot_i];
-        for (int c = 0; c < tc.chunks && ok; ++c) {
-          const uint32_t u = use + c;
-          const uint32_t slot = u % p.num_slots;
-          if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (u / p.num_slots) & 1u, ctl, p.status, lane)) {
+        const int units_end = tc.unit0 + tc.nunits;
+        int unit = tc.unit0, col_in_unit = 0;
+        int slot_i = unit / p.r, k = unit - slot_i * p.r;
+        float m = -CUDART_INF_F, s = 0.f, tval = 0.f;
+        int tgt = (p.wpp == 1 && valid) ? p.targets[wrow0 * p.n + slot_i] : -1;
+        for (int t = 0; t < tc.ntiles && ok; ++t, ++use) {
+          const uint32_t slot = use % p.num_slots;
+          if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (use / p.num_slots) & 1u, ctl, p.status, lane)) {
             ok = false;
             break;
           }
           tc_fence_after();
           const uint32_t tcol = lane_base + slot * p.slot_stride;
-          for (int b = 0; b < nbatch; ++b) {
+          for (int b = 0; b < nbatch && unit < units_end; ++b) {
             float x[16];
             tmem_ld16(tcol + b * 16, x);
-            const int col0 = c * tc.cols + b * 16;
             float bm = x[0];
 #pragma unroll
             for (int q = 1; q < 16; ++q) bm = fmaxf(bm, x[q]);
@@ -355,7 +369,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
             for (int q = 0; q < 16; ++q) s += fast_ex2(fmaf(x[q], kLog2e, -mn2));
             m = mn;
             if (p.wpp == 1) {
-              const int rel = tgt - col0;
+              const int rel = tgt - col_in_unit;
               if (static_cast<unsigned>(rel) < 16u) {
 #pragma unroll
                 for (int q = 0; q < 16; ++q)
@@ -363,7 +377,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
               }
             } else if (valid) {
               for (int j = 0; j < p.wpp; ++j) {
-                const int rel = p.targets[(wrow0 + j) * p.n + slot_i] - col0;
+                const int rel = p.targets[(wrow0 + j) * p.n + slot_i] - col_in_unit;
                 if (static_cast<unsigned>(rel) < 16u) {
                   float val = 0.f;
 #pragma unroll
@@ -373,36 +387,50 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
                 }
               }
             }
+            col_in_unit += 16;
+            if (col_in_unit == p.v) {
+              // ---- unit (slot_i, k) complete
+              const float lse = m + fast_lg2(s) * kLn2;
+              if (valid) {
+                for (int j = 0; j < p.wpp; ++j) {
+                  const int tj = (p.wpp == 1) ? tgt : p.targets[(wrow0 + j) * p.n + slot_i];
+                  float* g = p.G + ((wrow0 + j) * p.n + slot_i) * p.r + k;
+                  if (tj < 0) {
+                    *g = 0.f;                                  // marginalised byte: the input unit sums to 1
+                  } else if (tj >= p.v) {
+                    *g = CUDART_NAN_F;
+                    atomicOr(p.status, kStatusBadTarget);
+                  } else {
+                    *g = ((p.wpp == 1) ? tval : *g) - lse;
+                  }
+                }
+              }
+              ++unit;
+              col_in_unit = 0;
+              m = -CUDART_INF_F; s = 0.f; tval = 0.f;
+              if (unit < units_end) {
+                slot_i = unit / p.r;
+                k = unit - slot_i * p.r;
+                tgt = (p.wpp == 1 && valid) ? p.targets[wrow0 * p.n + slot_i] : -1;
+              }
+            }
           }
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&ctl->tempty[slot]));
         }
         if (!ok) break;
-        const float lse = m + fast_lg2(s) * kLn2;
-        if (valid) {
-          for (int j = 0; j < p.wpp; ++j) {
-            const int t = (p.wpp == 1) ? tgt : p.targets[(wrow0 + j) * p.n + slot_i];
-            float* g = p.G + ((wrow0 + j) * p.n + slot_i) * p.r + k;
-            if (t < 0) {
-              *g = 0.f;                                  // marginalised byte: the input unit sums to 1
-            } else if (t >= p.v) {
-              *g = CUDART_NAN_F;
-              atomicOr(p.status, kStatusBadTarget);
-            } else {
-              *g = ((p.wpp == 1) ? tval : *g) - lse;
-            }
-          }
-        }
       } else {
         // ---- byte draws (Algorithm 1, input units): inverse CDF of softmax(logits) for every window of this
-        // row whose selected unit for this slot is k. All chunks of the unit stay in TMEM until the end.
+        // row whose selected unit for this slot is k. One unit per group: all its tiles stay in TMEM until the end.
+        const int slot_i = tc.unit0 / p.r;
+        const int k = tc.unit0 - slot_i * p.r;
         unsigned long long pending = 0ull;
         const size_t wrow0 = static_cast<size_t>(valid ? row : 0) * p.wpp;
         if (valid)
           for (int j = 0; j < p.wpp; ++j)
             if (p.unit_sel[(wrow0 + j) * p.n + slot_i] == k) pending |= 1ull << j;
-        for (int c = 0; c < tc.chunks && ok; ++c) {
+        for (int c = 0; c < tc.ntiles && ok; ++c) {
           const uint32_t u = use + c;
           if (!bounded_wait_warp(smem_u32(&ctl->tfull[u % p.num_slots]), (u / p.num_slots) & 1u, ctl, p.status,
                                  lane))
@@ -412,7 +440,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
         tc_fence_after();
         if (__any_sync(0xffffffffu, pending != 0ull)) {
           float m = -CUDART_INF_F;
-          for (int c = 0; c < tc.chunks; ++c) {
+          for (int c = 0; c < tc.ntiles; ++c) {
             const uint32_t tcol = lane_base + ((use + c) % p.num_slots) * p.slot_stride;
             for (int b = 0; b < nbatch; ++b) {
               float x[16];
@@ -423,7 +451,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
           }
           const float m2 = m * kLog2e;
           float total = 0.f;   // same terms in the same order as the running sum of the scan below
-          for (int c = 0; c < tc.chunks; ++c) {
+          for (int c = 0; c < tc.ntiles; ++c) {
             const uint32_t tcol = lane_base + ((use + c) % p.num_slots) * p.slot_stride;
             for (int b = 0; b < nbatch; ++b) {
               float x[16];
@@ -440,7 +468,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
             float cum = 0.f;
             int found = p.v - 1;   // rounding may leave no index: the last one
             bool hit = false;
-            for (int c = 0; c < tc.chunks; ++c) {
+            for (int c = 0; c < tc.ntiles; ++c) {
               const uint32_t tcol = lane_base + ((use + c) % p.num_slots) * p.slot_stride;
               for (int b = 0; b < nbatch; ++b) {
                 float x[16];
@@ -466,9 +494,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
         tc_fence_before();
         __syncwarp();
         if (lane == 0)
-          for (int c = 0; c < tc.chunks; ++c) mbar_arrive(smem_u32(&ctl->tempty[(use + c) % p.num_slots]));
+          for (int c = 0; c < tc.ntiles; ++c) mbar_arrive(smem_u32(&ctl->tempty[(use + c) % p.num_slots]));
+        use += tc.ntiles;
       }
-      use += tc.chunks;
     }
   }
 
