@@ -155,7 +155,8 @@ def run_reference(args):
 
 
 def measure_decode_cell(torch, cell, steps: int, warmup: int):
-    """Draft windows/s and p50 latency on one decode cell (family, n, P) with 16 windows per position."""
+    """Draft windows/s and p50 latency on one decode cell (family, n, P) with 16 windows per position. Every call
+    is timed on its own (CUDA events on the launching stream); the library's event ring gives the per-kernel split."""
     from paper_2511_11346_b200.runner import DeviceHead
     wl = I.config_workload(4, cell=cell)
     dh = DeviceHead(wl)
@@ -167,6 +168,7 @@ def measure_decode_cell(torch, cell, steps: int, warmup: int):
     for _ in range(warmup):
         dh.head.mtpc_draft_sample(h, wl.wpp, u, ob, ol)
     torch.cuda.synchronize()
+    dh.head.mtpc_set_timing(steps)
     lat = []
     for _ in range(steps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -175,17 +177,26 @@ def measure_decode_cell(torch, cell, steps: int, warmup: int):
         e1.record()
         e1.synchronize()
         lat.append(e0.elapsed_time(e1))
+    phases = [dh.head.mtpc_get_timing(i) for i in range(steps)]
+    phase_p50 = [statistics.median(p[k] for p in phases) for k in range(len(phases[0]))]
+    launches = len(phases[0])
+    dh.head.mtpc_set_timing(0)
+    status = dh.head.mtpc_get_status()
     p50 = statistics.median(lat)
     s = wl.shape
     weight_bytes = (s.n * s.r * s.v + s.sum_rows) * s.d * 2
     peaks, src = load_peaks()
+    gbs = weight_bytes / (p50 * 1e-3) / 1e9
+    gemm_gbs = weight_bytes / (phase_p50[0] * 1e-3) / 1e9
     out = {"workload": f"configs[4] {wl.name}: P={wl.T} wpp={wl.wpp} d={s.d} n={s.n} r={s.r} v={s.v}",
-           "windows_per_s": W / (p50 * 1e-3), "p50_ms": p50, "calls": steps,
-           "hbm_roofline": {"algorithmic_bytes": weight_bytes, "note": "one pass over the weights",
-                            "achieved_gbs": weight_bytes / (p50 * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
-                            "frac": weight_bytes / (p50 * 1e-3) / 1e9 / peaks["hbm_gbs"], "peak_source": src}}
+           "windows_per_s": W / (p50 * 1e-3), "p50_ms": p50, "calls": steps, "kernels_per_call": launches,
+           "kernel_p50_ms": phase_p50, "device_status": status,
+           "hbm_roofline": {"algorithmic_bytes": weight_bytes, "note": "one pass over the emission and sum-unit weights",
+                            "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
+                            "weight_pass_kernel_gbs": gemm_gbs, "weight_pass_kernel_frac": gemm_gbs / peaks["hbm_gbs"],
+                            "peak_source": src}}
     dh.close()
-    return out
+    return out, launches * (steps + warmup)
 
 
 def run_ours(args):
@@ -277,9 +288,11 @@ def run_ours(args):
         cpu_baseline = {"value": cpu_value, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
                         "sample": f"first {sample} of {wl.T} positions, one pass, {cpu_s:.1f} s"}
 
-    draft = None
+    draft, sweep = None, None
     if not args.no_draft and world == 1:
-        draft = measure_decode_cell(torch, (I.CP, 8, 64), steps=200, warmup=5)
+        cells = I.DECODE_CELLS if args.decode_cells == "all" else [(I.CP, 8, 64)]
+        sweep = [measure_decode_cell(torch, cell, steps=200, warmup=5)[0] for cell in cells]
+        draft = next(c for c in sweep if "decode_cp_n8_P64" in c["workload"])
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -301,6 +314,7 @@ def run_ours(args):
     }
     if draft is not None:
         line["draft"] = draft
+        line["decode_sweep"] = sweep
     print(json.dumps(line), flush=True)
 
 
@@ -314,6 +328,8 @@ def main():
     ap.add_argument("--ref-positions", type=int, default=None,
                     help="positions the CPU oracle processes per step / for the cpu_baseline sample")
     ap.add_argument("--no-draft", action="store_true", help="skip the decode-cell draft measurement")
+    ap.add_argument("--decode-cells", choices=["all", "one"], default="all",
+                    help="draft measurement: the twelve cells of the decode sweep, or only CP n=8 P=64")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiling runs)")
     ap.add_argument("--positions", type=int, default=None,
                     help="override the number of positions (scaled-down profiler captures; not a bench value)")

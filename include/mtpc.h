@@ -146,7 +146,9 @@ int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags);
  * of the call made `calls_back` calls ago (0 = the most recent) and writes up to `capacity` phase durations
  * in milliseconds, *out_count = number of phases that call had:
  *   mtpc_window_logprob: [0] projection GEMM + fused epilogue, [1] circuit evaluation.
- *   mtpc_draft_sample:   [0] sum-unit GEMM, [1] latent sampling, [2] GEMM + inverse-CDF epilogue,
+ *   mtpc_draft_sample:   P <= 128 positions and r <= 32: [0] one pass over all weights (logits of every unit),
+ *                        [1] per-slot latent + byte draws and evidence, [2] circuit evaluation.
+ *                        Otherwise: [0] sum-unit GEMM, [1] latent sampling, [2] GEMM + inverse-CDF epilogue,
  *                        [3] GEMM + gather epilogue on the drafted bytes, [4] circuit evaluation.
  */
 int mtpc_set_timing(mtpc_head* head, int32_t ring);

@@ -11,6 +11,7 @@
 
 #include "../../include/mtpc.h"
 #include "mtpc_circuit.cuh"
+#include "mtpc_decode.cuh"
 #include "mtpc_gemm.cuh"
 
 namespace {
@@ -20,6 +21,7 @@ using namespace mtpc;
 constexpr size_t kAlign = 256;
 constexpr int kMaxPhases = 5;
 constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA on sm_100
+constexpr size_t kHmmTableSmemLimit = 96 * 1024;   // exp'd HMM transition tables kept in shared memory up to this size
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
@@ -40,7 +42,8 @@ struct Layout {
   Tiling sm;            // sampling mode: one unit per group, equal tiles of <= 256 columns
   size_t max_windows;
   // workspace offsets (bytes)
-  size_t off_status, off_wemit, off_wsum, off_hidden, off_logA, off_G, off_logw, off_sel;
+  size_t off_status, off_wemit, off_wsum, off_hidden, off_logA, off_G, off_logw, off_sel, off_logits;
+  int decode_max_p;     // positions the few-position draft path can take (0: path not available)
   size_t off_h_hidden, off_h_targets, off_h_uniforms, off_h_bytes, off_h_out;
   size_t total;
 };
@@ -118,6 +121,8 @@ int plan(const mtpc_config& c, Layout* L) {
   L->off_G = take(L->max_windows * c.n * c.r * 4);
   L->off_logw = take(static_cast<size_t>(c.max_positions) * L->sum_rows * 4);
   L->off_sel = take(L->max_windows * c.n * 4);
+  L->decode_max_p = c.r <= 32 ? (c.max_positions < kDecodeMaxP ? c.max_positions : kDecodeMaxP) : 0;
+  L->off_logits = take(static_cast<size_t>(L->decode_max_p) * emit_units * c.v * 4);
   L->off_h_hidden = take(static_cast<size_t>(c.max_positions) * c.d * elt);
   L->off_h_targets = take(static_cast<size_t>(c.max_positions) * c.n * 4);
   L->off_h_uniforms = take(L->max_windows * 2 * c.n * 4);
@@ -167,6 +172,8 @@ struct mtpc_head {
   const void* W_emit_bf16;
   const void* W_sum_bf16;
   CUtensorMap tm_emit_lp, tm_emit_sm, tm_sum;   // W_emit with the box of either tiling; W_sum
+  CUtensorMap tm_emit_dec, tm_sum_dec;          // the same matrices in the few-position draft path's tiles
+  int decode_tile_rows, decode_sum_tile_rows;
   int num_sms;
   int ring;                 // calls whose per-kernel events are retained (0 = timing off)
   cudaEvent_t* ev;          // [ring][kMaxPhases][2]
@@ -261,12 +268,71 @@ int launch_circuit(mtpc_head* h, int W, int wpp, float* out, cudaStream_t st) {
   if (c.family == MTPC_CP) {
     circuit_cp_kernel<<<blocks, threads, 0, st>>>(G, logw, out, W, wpp, c.n, c.r, L.sum_rows);
   } else if (c.family == MTPC_HMM) {
-    circuit_hmm_kernel<<<blocks, threads, 0, st>>>(G, logw, at<float>(h, L.off_logA), out, W, wpp, c.n, c.r,
-                                                   L.sum_rows);
+    const size_t table_bytes = static_cast<size_t>(c.n - 1) * c.r * c.r * 4;
+    const int in_smem = table_bytes <= kHmmTableSmemLimit;
+    const int cap = 4 * h->num_sms;                      // CTAs stride over the windows: the tables are staged once each
+    circuit_hmm_kernel<<<blocks < cap ? blocks : cap, threads, in_smem ? table_bytes : 0, st>>>(
+        G, logw, at<float>(h, L.off_logA), out, W, wpp, c.n, c.r, L.sum_rows, in_smem);
   } else {
     const size_t smem = static_cast<size_t>(kCircuitWarps) * ((c.n - 1) * c.r + c.r * (c.r + 1)) * 4;
     circuit_btree_kernel<<<blocks, threads, smem, st>>>(G, logw, out, W, wpp, c.n, c.r, L.sum_rows);
   }
+  h->launches++;
+  return check_launch();
+}
+
+// Rows per emission tile of the few-position draft path: the height in [64, 128] (multiple of 8) that leaves the
+// least idle time when the tiles are dealt evenly to `ctas` persistent CTAs; ties go to the taller tile.
+int decode_tile_rows(long long rows, int ctas) {
+  int best = 128;
+  double best_eff = 0.0;
+  for (int tr = 128; tr >= 64; tr -= 8) {
+    const long long tiles = (rows + tr - 1) / tr;
+    const long long per_cta = (tiles + ctas - 1) / ctas;
+    const double eff = static_cast<double>(rows) / (static_cast<double>(per_cta) * ctas * tr);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best = tr; }
+  }
+  return best;
+}
+
+// Few-position draft path: one pass over all weight rows with the positions on the N axis.
+int launch_decode_gemm(mtpc_head* h, const void* hidden_bf16, int P, cudaStream_t st) {
+  const mtpc_config& c = h->cfg;
+  const Layout& L = h->L;
+  DecodeParams p;
+  memset(&p, 0, sizeof(p));
+  p.P = P;
+  p.Ppad = (P + 15) / 16 * 16;
+  int rc = make_tmap(&p.tm_h, hidden_bf16, static_cast<uint64_t>(P), static_cast<uint64_t>(c.d), p.Ppad);
+  if (rc != MTPC_OK) return rc;
+  p.tm_emit = h->tm_emit_dec;
+  p.tm_sum = h->tm_sum_dec;
+  p.kblocks = c.d / kBlockK;
+  p.emit_rows = c.n * c.r * c.v;
+  p.sum_rows = L.sum_rows;
+  p.r = c.r;
+  p.tile_rows = h->decode_tile_rows;
+  p.sum_tile_rows = h->decode_sum_tile_rows;
+  p.tile_bytes = p.tile_rows * kBlockK * 2;
+  p.emit_tiles = (p.emit_rows + p.tile_rows - 1) / p.tile_rows;
+  p.sum_tiles = (p.sum_rows + p.sum_tile_rows - 1) / p.sum_tile_rows;
+  p.tile_stride = (p.Ppad + 31) / 32 * 32;
+  p.pass_tiles = kTmemCols / (2 * p.tile_stride);                     // two slots of pass_tiles accumulators
+  if (p.pass_tiles > kDecodeMaxTiles) p.pass_tiles = kDecodeMaxTiles;
+  // stage = weight tiles + hidden tile, padded so that a 128-row operand read from the last tile's base stays inside
+  int stage = p.pass_tiles * p.tile_bytes + p.Ppad * kBlockK * 2;
+  const int reach = (p.pass_tiles - 1) * p.tile_bytes + kABytes;
+  if (stage < reach) stage = reach;
+  p.stage_bytes = (stage + 1023) / 1024 * 1024;
+  const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
+  p.stages = (kSmemLimit - ctl) / p.stage_bytes;
+  if (p.stages > kMaxStages) p.stages = kMaxStages;
+  p.logits = at<float>(h, L.off_logits);
+  p.logw = at<float>(h, L.off_logw);
+  p.status = at<unsigned>(h, L.off_status);
+  const int tiles = p.emit_tiles + p.sum_tiles;
+  const int grid = tiles < h->num_sms ? tiles : h->num_sms;
+  mtpc_decode_gemm_kernel<<<grid, kGemmThreads, p.stages * p.stage_bytes + ctl, st>>>(p);
   h->launches++;
   return check_launch();
 }
@@ -311,6 +377,25 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   int rc = stage_hidden(h, hidden, P, &hb, st);
   if (rc != MTPC_OK) return rc;
   PhaseTimer pt(h, st);
+  if (P <= L.decode_max_p) {
+    // Few positions: every weight row is read once. 1. all logits (emission -> scratch, sum units -> log omega)
+    // 2. per (position, slot): latent draws, byte draws, evidence of the drafted bytes  3. circuit evaluation
+    pt.begin();
+    rc = launch_decode_gemm(h, hb, P, st);
+    pt.end();
+    if (rc != MTPC_OK) return rc;
+    pt.begin();
+    draft_slot_kernel<<<dim3(c.n, P), kSlotThreads, 2 * c.r * sizeof(float), st>>>(
+        c.family, at<float>(h, L.off_logits), at<float>(h, L.off_logw), at<float>(h, L.off_logA), uniforms, out_bytes,
+        at<float>(h, L.off_G), at<unsigned>(h, L.off_status), wpp, c.n, c.r, c.v, L.sum_rows);
+    h->launches++;
+    pt.end();
+    if ((rc = check_launch()) != MTPC_OK) return rc;
+    pt.begin();
+    rc = launch_circuit(h, W, wpp, out_logprob, st);
+    pt.end();
+    return rc;
+  }
   // 1. sum-unit weights (Sec. 3.3) -> 2. latent draws at the sum units (Algorithm 1)
   pt.begin();
   rc = launch_gemm(h, kModeLogprob, hb, P, 1, false, true, nullptr, nullptr, nullptr, st);
@@ -384,6 +469,11 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
                                kSmemLimit) != cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeSample>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
+  fail |= cudaFuncSetAttribute(mtpc_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
+          cudaSuccess;
+  if (cfg->family == MTPC_HMM)
+    fail |= cudaFuncSetAttribute(circuit_hmm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kHmmTableSmemLimit)) != cudaSuccess;
   if (cfg->family == MTPC_BTREE) {
     const int smem = kCircuitWarps * ((cfg->n - 1) * cfg->r + cfg->r * (cfg->r + 1)) * 4;
     if (smem > 48 * 1024)
@@ -417,6 +507,10 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   rc = make_tmap(&h->tm_emit_lp, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols);
+  h->decode_tile_rows = decode_tile_rows(static_cast<long long>(emit_rows), h->num_sms);
+  if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_dec, h->W_emit_bf16, emit_rows, cfg->d, h->decode_tile_rows);
+  h->decode_sum_tile_rows = h->decode_tile_rows / 32 * 32;   // whole groups of r <= 32 rows per warp; fits the tile pitch
+  if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum_dec, h->W_sum_bf16, L.sum_rows, cfg->d, h->decode_sum_tile_rows);
   if (rc != MTPC_OK) { delete h; return rc; }
   *out = h;
   return MTPC_OK;
@@ -628,7 +722,7 @@ extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_
   L.off_logA = take(c.family == MTPC_HMM ? static_cast<size_t>(c.n - 1) * c.r * c.r * 4 : 0);
   L.off_G = take(static_cast<size_t>(c.max_positions) * c.n * c.r * 4);
   L.off_logw = take(static_cast<size_t>(c.max_positions) * L.sum_rows * 4);
-  L.off_sel = L.off_wemit = L.off_wsum = L.off_hidden = 0;                               // unused by this call
+  L.off_sel = L.off_wemit = L.off_wsum = L.off_hidden = L.off_logits = 0;                // unused by this call
   L.off_h_hidden = L.off_h_targets = L.off_h_uniforms = L.off_h_bytes = L.off_h_out = 0;
   L.total = off;
   if (L.total > static_cast<size_t>(MTPC_STATIC_SCRATCH_BYTES)) return MTPC_ERR_STATIC_SCRATCH;
@@ -654,6 +748,9 @@ extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_
   bool fail = cudaDeviceGetAttribute(&h.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
+  if (c.family == MTPC_HMM)
+    fail |= cudaFuncSetAttribute(circuit_hmm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kHmmTableSmemLimit)) != cudaSuccess;
   if (c.family == MTPC_BTREE) {
     const int smem = kCircuitWarps * ((c.n - 1) * c.r + c.r * (c.r + 1)) * 4;
     if (smem > 48 * 1024)

@@ -56,32 +56,44 @@ __global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __re
 
 // Eq. (HMM), forward recursion over the window: alpha_0[k] = log pi[k] + G[0,k];
 // alpha_i[k] = G[i,k] + LSE_a(alpha_{i-1}[a] + logA[i-1][a][k]); out = LSE_k alpha_{n-1}[k].  r <= 32.
+// The inner log-sum-exp is taken as one scaled matrix-vector product per step: with m = max_a alpha_{i-1}[a],
+// alpha_i[k] = G[i,k] + m + log sum_a exp(alpha_{i-1}[a] - m) A[i-1][a][k], A = exp(logA) staged once per CTA in
+// shared memory ((n-1) r^2 floats; read straight from global memory when that does not fit). One warp per
+// window, lane = state; CTAs stride over the windows.
 __global__ void circuit_hmm_kernel(const float* __restrict__ G, const float* __restrict__ logw,
                                    const float* __restrict__ logA, float* __restrict__ out, int W, int wpp, int n,
-                                   int r, int sum_rows) {
-  const int w = blockIdx.x * kCircuitWarps + (threadIdx.x >> 5);
+                                   int r, int sum_rows, int tables_in_smem) {
+  extern __shared__ float A_lin[];
   const int lane = threadIdx.x & 31;
-  if (w >= W) return;
-  const float* g = G + static_cast<size_t>(w) * n * r;
-  const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
-  const bool has = lane < r;
-  float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
-  for (int i = 1; i < n; ++i) {
-    const float* A = logA + static_cast<size_t>(i - 1) * r * r;
-    float m = -CUDART_INF_F;
-    for (int a = 0; a < r; ++a) {
-      const float prev = __shfl_sync(kFull, alpha, a);
-      if (has) m = fmaxf(m, prev + __ldg(A + a * r + lane));
-    }
-    float s = 0.f;
-    for (int a = 0; a < r; ++a) {
-      const float prev = __shfl_sync(kFull, alpha, a);
-      if (has) s += __expf(prev + __ldg(A + a * r + lane) - m);
-    }
-    if (has) alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : g[i * r + lane] + m + __logf(s);
+  const int count = (n - 1) * r * r;
+  if (tables_in_smem) {
+    for (int e = threadIdx.x; e < count; e += blockDim.x) A_lin[e] = __expf(__ldg(logA + e));
+    __syncthreads();
   }
-  const float res = warp_lse(alpha, has);
-  if (lane == 0) out[w] = res;
+  const bool has = lane < r;
+  for (int w = blockIdx.x * kCircuitWarps + (threadIdx.x >> 5); w < W; w += gridDim.x * kCircuitWarps) {
+    const float* g = G + static_cast<size_t>(w) * n * r;
+    const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
+    float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
+    for (int i = 1; i < n; ++i) {
+      const float gi = has ? g[i * r + lane] : 0.f;
+      float m = alpha;                                   // fmaxf drops NaNs; they come back through e below
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
+      const float e = has ? __expf(alpha - m) : 0.f;     // NaN if alpha is NaN or if every state is impossible
+      float s = 0.f;
+      if (tables_in_smem) {
+        const float* A = A_lin + static_cast<size_t>(i - 1) * r * r;
+        for (int a = 0; a < r; ++a) s = fmaf(__shfl_sync(kFull, e, a), has ? A[a * r + lane] : 0.f, s);
+      } else {
+        const float* A = logA + static_cast<size_t>(i - 1) * r * r;
+        for (int a = 0; a < r; ++a) s = fmaf(__shfl_sync(kFull, e, a), has ? __expf(__ldg(A + a * r + lane)) : 0.f, s);
+      }
+      if (has) alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : gi + m + __logf(s);
+    }
+    const float res = warp_lse(alpha, has);
+    if (lane == 0) out[w] = res;
+  }
 }
 
 // Eq. (BTree), bottom-up over the heap-ordered latent tree. Node j >= 1 has the table

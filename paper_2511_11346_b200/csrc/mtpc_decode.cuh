@@ -1,0 +1,369 @@
+// Draft path for few positions (decode-time speculative drafting, Algorithm 1): the cost is one pass over the
+// emission weights, so the work is organised around streaming them from HBM exactly once.
+//
+//   mtpc_decode_gemm_kernel   logits[p, row] = W[row] . h_p for every weight row (emission and sum-unit rows) and
+//                             every position p < P <= 128, with the roles of the operands swapped with respect
+//                             to the training-shaped kernel: 128 weight rows sit on the M axis (TMEM lanes), the
+//                             positions on the N axis (TMEM columns). Emission logits go to a small scratch
+//                             [P, n*r*v] fp32 (P is tiny here, so this is a few MB against hundreds of MB of
+//                             weights); sum-unit logits are log-softmaxed over their groups of r rows (= lanes,
+//                             by warp shuffles) and written as log omega [P, S*r].
+//                             Weight rows are cut into tiles of `tile_rows` <= 128 rows, chosen by the host so that
+//                             the tiles divide evenly over the persistent CTAs; each CTA takes a contiguous run
+//                             of tiles and walks K once per pass of up to three tiles, which share one copy of
+//                             the hidden-state block, so the bytes in flight per SM stay high and the hidden
+//                             states cross L2 once per pass instead of once per tile.
+//   draft_slot_kernel         one CTA per (position, window slot i): log-sum-exp of the r input units of the
+//                             slot, then per window (one warp each): latent draws down to the unit that owns
+//                             slot i, the byte by inverse CDF of that unit's categorical, and the evidence
+//                             G[w, i, k] = log phi_k(byte) for all k, which the circuit kernels then reduce.
+#pragma once
+#include "mtpc_circuit.cuh"
+#include "mtpc_gemm.cuh"
+
+namespace mtpc {
+
+constexpr int kDecodeMaxP = 128;                   // positions per call on this path
+constexpr int kDecodeMaxTiles = 3;                 // weight tiles that share one copy of the hidden states
+constexpr int kSlotThreads = 256;
+
+struct DecodeParams {
+  CUtensorMap tm_h;      // hidden [P, d]       box 64 x Ppad
+  CUtensorMap tm_emit;   // W_emit [n*r*v, d]   box 64 x tile_rows
+  CUtensorMap tm_sum;    // W_sum  [S*r, d]     box 64 x sum_tile_rows
+  int P, Ppad, kblocks;
+  int emit_rows, sum_rows, r;
+  int tile_rows;                 // rows of an emission tile (a multiple of 8, <= 128)
+  int sum_tile_rows;             // rows of a sum tile (a multiple of 32, <= tile_rows rounded up to 32)
+  int tile_bytes;                // shared-memory pitch of a weight tile
+  int emit_tiles, sum_tiles;
+  int pass_tiles;                // tiles per pass (<= kDecodeMaxTiles)
+  int tile_stride;               // TMEM columns per tile
+  int stages, stage_bytes;
+  float* logits;         // [P, emit_rows]
+  float* logw;           // [P, sum_rows]
+  unsigned* status;
+};
+
+// Tile `t` of the launch: emission tiles first, then sum tiles.
+struct DecodeTile {
+  int is_sum, index, rows;   // which matrix, tile index within it, rows per tile
+};
+__device__ __forceinline__ DecodeTile decode_tile(const DecodeParams& p, int t) {
+  DecodeTile d;
+  d.is_sum = t >= p.emit_tiles;
+  d.index = d.is_sum ? t - p.emit_tiles : t;
+  d.rows = d.is_sum ? p.sum_tile_rows : p.tile_rows;
+  return d;
+}
+
+// A CTA walks its run of tiles in passes of up to pass_tiles tiles (of either matrix). Shared-memory stage:
+// pass_tiles weight tiles at a pitch of tile_bytes (the MMA reads 128 rows from each tile's base: what lies beyond
+// the tile's own rows is other data, and the TMEM lanes it produces are never read), then the hidden tile
+// (Ppad rows x 128 bytes) followed by slack so that the last tile's 128-row read stays inside the stage.
+// Tensor memory: two slots of pass_tiles * tile_stride columns.
+__global__ void __launch_bounds__(kGemmThreads, 1) mtpc_decode_gemm_kernel(const __grid_constant__ DecodeParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
+  uint8_t* tiles = smem_raw + (tiles_addr - raw_addr);
+  GemmControl* ctl = reinterpret_cast<GemmControl*>(tiles + static_cast<size_t>(p.stages) * p.stage_bytes);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int total_tiles = p.emit_tiles + p.sum_tiles;
+  const int tile_begin = static_cast<int>(static_cast<long long>(blockIdx.x) * total_tiles / gridDim.x);
+  const int tile_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * total_tiles / gridDim.x);
+  const uint32_t hidden_off = p.pass_tiles * p.tile_bytes;
+  const uint32_t slot_cols = p.pass_tiles * p.tile_stride;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(smem_u32(&ctl->full[s]), 1);
+      mbar_init(smem_u32(&ctl->empty[s]), 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&ctl->tfull[s]), 1);
+      mbar_init(smem_u32(&ctl->tempty[s]), 4);
+    }
+    mbar_init(smem_u32(&ctl->drain), 1);
+    ctl->abort = 0;
+    fence_mbar_init();
+    tma_prefetch_desc(&p.tm_h);
+    tma_prefetch_desc(&p.tm_emit);
+    tma_prefetch_desc(&p.tm_sum);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
+      bool ok = true;
+      for (int cur = tile_begin; cur < tile_end && ok;) {
+        const int ntiles = min(p.pass_tiles, tile_end - cur);
+        uint32_t bytes = p.Ppad * (kBlockK * 2);                   // out-of-range rows are zero-filled and counted
+        for (int q = 0; q < ntiles; ++q) bytes += decode_tile(p, cur + q).rows * (kBlockK * 2);
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
+          const uint32_t full = smem_u32(&ctl->full[stage]);
+          const uint32_t dst = tiles_addr + stage * p.stage_bytes;
+          mbar_arrive_expect_tx(full, bytes);
+          for (int q = 0; q < ntiles; ++q) {
+            const DecodeTile t = decode_tile(p, cur + q);
+            tma_load_2d(dst + q * p.tile_bytes, t.is_sum ? &p.tm_sum : &p.tm_emit, full, kb * kBlockK, t.index * t.rows);
+          }
+          tma_load_2d(dst + hidden_off, &p.tm_h, full, kb * kBlockK, 0);
+          issued_mask |= 1u << stage;
+          phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
+          if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
+        }
+        cur += ntiles;
+      }
+      if (!ok) {
+        for (int s = 0; s < p.stages; ++s)
+          if (issued_mask & (1u << s)) {
+            const uint32_t bar = smem_u32(&ctl->full[s]);
+            const uint32_t par = (phase_mask >> s) & 1u;
+            const uint64_t t0 = global_timer_ns();
+            while (!mbar_try_wait(bar, par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+          }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer: D[row, p] = W[row, :] . h[p, :]
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, use = 0;
+      bool ok = true;
+      const uint32_t idesc = umma_idesc_bf16(kBlockM, p.Ppad);
+      for (int cur = tile_begin; cur < tile_end && ok; ++use) {
+        const int ntiles = min(p.pass_tiles, tile_end - cur);
+        cur += ntiles;
+        const uint32_t slot = use & 1u;
+        if (!bounded_wait(smem_u32(&ctl->tempty[slot]), ((use >> 1) & 1u) ^ 1u, ctl, p.status)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + slot * slot_cols;
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t w_addr = tiles_addr + stage * p.stage_bytes;
+          const uint64_t b_desc = umma_smem_desc_sw128(w_addr + hidden_off);
+          for (int q = 0; q < ntiles; ++q) {
+            const uint64_t a_desc = umma_smem_desc_sw128(w_addr + q * p.tile_bytes);
+#pragma unroll
+            for (int kk = 0; kk < kBlockK / 16; ++kk)
+              umma_bf16(d_tmem + q * p.tile_stride, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&ctl->empty[stage]));
+          if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&ctl->tfull[slot]));
+      }
+      if (!ok) {
+        umma_commit(smem_u32(&ctl->drain));
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue: warp q owns lanes 32q .. 32q+31
+    const int quarter = warp & 3;
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    uint32_t use = 0;
+    bool ok = true;
+    for (int cur = tile_begin; cur < tile_end && ok; ++use) {
+      const int ntiles = min(p.pass_tiles, tile_end - cur);
+      const uint32_t slot = use & 1u;
+      if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (use >> 1) & 1u, ctl, p.status, lane)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      for (int q = 0; q < ntiles; ++q) {
+        const DecodeTile t = decode_tile(p, cur + q);
+        if (quarter * 32 >= t.rows) continue;                      // warp-uniform: none of this warp's lanes is a row
+        const int nrows = t.is_sum ? p.sum_rows : p.emit_rows;
+        float* dst = t.is_sum ? p.logw : p.logits;
+        const uint32_t tcol = lane_base + slot * slot_cols + q * p.tile_stride;
+        const int local = quarter * 32 + lane;
+        const int row = t.index * t.rows + local;
+        const bool mine = local < t.rows && row < nrows;
+        for (int b = 0; b < (p.P + 15) / 16; ++b) {
+          float x[16];
+          tmem_ld16(tcol + b * 16, x);
+          if (t.is_sum) {
+            // log-softmax over the r rows of a sum unit = r adjacent lanes (r a power of two <= 32); the 16
+            // positions of the batch are reduced side by side so that the shuffles overlap
+            float m[16], e[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) m[c] = x[c];
+            for (int off = 1; off < p.r; off <<= 1) {
+#pragma unroll
+              for (int c = 0; c < 16; ++c) m[c] = fmaxf(m[c], __shfl_xor_sync(0xffffffffu, m[c], off));
+            }
+#pragma unroll
+            for (int c = 0; c < 16; ++c) e[c] = fast_ex2((x[c] - m[c]) * kLog2e);
+            for (int off = 1; off < p.r; off <<= 1) {
+#pragma unroll
+              for (int c = 0; c < 16; ++c) e[c] += __shfl_xor_sync(0xffffffffu, e[c], off);
+            }
+#pragma unroll
+            for (int c = 0; c < 16; ++c) x[c] = x[c] - m[c] - fast_lg2(e[c]) * kLn2;
+          }
+          if (mine) {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+              const int pos = b * 16 + c;
+              if (pos < p.P) dst[static_cast<size_t>(pos) * nrows + row] = x[c];   // 32 lanes -> 128 contiguous bytes
+            }
+          }
+        }
+      }
+      cur += ntiles;
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctl->tempty[slot]));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------- per-(position, slot) sampling
+// Inclusive warp scan (sum).
+__device__ __forceinline__ float warp_scan_incl(float x, int lane) {
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const float y = __shfl_up_sync(kFull, x, off);
+    if (lane >= off) x += y;
+  }
+  return x;
+}
+// Categorical draw over r <= 32 log-probabilities held one per lane (lanes >= r hold anything): the smallest
+// j with u < p_0 + ... + p_j, else r - 1. All lanes return the same index.
+__device__ __forceinline__ int warp_inv_cdf_logp(float logp, int r, float u, int lane) {
+  const float pr = lane < r ? expf(logp) : 0.f;
+  const float cum = warp_scan_incl(pr, lane);
+  const unsigned hit = __ballot_sync(kFull, lane < r && u < cum);
+  return hit ? __ffs(hit) - 1 : r - 1;
+}
+
+// Latent draws of one window down to the unit that owns slot i (Algorithm 1 at the sum units); the whole warp
+// calls it. CP: the mixture component. HMM: the chain z_0 .. z_i. BTree: the path from the root to the
+// deepest internal node above token i. Returns -1 if a uniform the window's latent draws use is outside [0,1).
+__device__ __forceinline__ int warp_sample_unit(int family, const float* __restrict__ lw, const float* __restrict__ logA,
+                                                const float* __restrict__ u, int n, int r, int i, int lane) {
+  const int nlat = (family == 0) ? 1 : (family == 1 ? n : n - 1);
+  bool bad = false;
+  for (int c = lane; c < nlat; c += 32) bad |= !(u[c] >= 0.f && u[c] < 1.f);
+  if (__any_sync(kFull, bad)) return -1;
+  int z = warp_inv_cdf_logp(lane < r ? lw[lane] : 0.f, r, u[0], lane);
+  if (family == 1) {
+    for (int s = 1; s <= i; ++s)
+      z = warp_inv_cdf_logp(lane < r ? logA[(static_cast<size_t>(s - 1) * r + z) * r + lane] : 0.f, r, u[s], lane);
+  } else if (family == 2) {
+    // heap path root -> owner node n/2 - 1 + i/2, top-down: the bits of (owner + 1) below its leading one
+    const int owner = n / 2 - 1 + (i >> 1);
+    const int code = owner + 1;
+    const int depth = 31 - __clz(code);
+    int node = 0;
+    for (int lvl = depth - 1; lvl >= 0; --lvl) {
+      node = 2 * node + 1 + ((code >> lvl) & 1);
+      z = warp_inv_cdf_logp(lane < r ? lw[r + (static_cast<size_t>(node - 1) * r + z) * r + lane] : 0.f, r, u[node], lane);
+    }
+  }
+  return z;
+}
+
+// grid = (n, P). Shared memory: 2 * r floats (max and log-sum-exp of each unit of the slot).
+__global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
+    int family, const float* __restrict__ logits, const float* __restrict__ logw, const float* __restrict__ logA,
+    const float* __restrict__ uniforms, int* __restrict__ out_bytes, float* __restrict__ G, unsigned* status, int wpp,
+    int n, int r, int v, int sum_rows) {
+  extern __shared__ float sm[];
+  float* unit_max = sm;
+  float* unit_lse = sm + r;
+  const int i = blockIdx.x;
+  const int pos = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nwarps = kSlotThreads / 32;
+  const float* row = logits + (static_cast<size_t>(pos) * n + i) * r * v;   // [r, v] logits of this slot
+
+  for (int k = warp; k < r; k += nwarps) {
+    const float* x = row + static_cast<size_t>(k) * v;
+    float m = -CUDART_INF_F;
+    for (int b = lane; b < v; b += 32) m = fmaxf(m, x[b]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
+    float s = 0.f;
+    for (int b = lane; b < v; b += 32) s += __expf(x[b] - m);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(kFull, s, off);
+    if (lane == 0) { unit_max[k] = m; unit_lse[k] = m + __logf(s); }
+  }
+  __syncthreads();
+
+  const float* lw = logw + static_cast<size_t>(pos) * sum_rows;
+  const int per = (v + 31) / 32;   // consecutive bytes per lane in the CDF scan
+  for (int j = warp; j < wpp; j += nwarps) {
+    const size_t w = static_cast<size_t>(pos) * wpp + j;
+    const float* u = uniforms + w * 2 * n;
+    const int z = warp_sample_unit(family, lw, logA, u, n, r, i, lane);
+    const float ub = u[n + i];
+    int byte = -1;
+    if (z < 0 || !(ub >= 0.f && ub < 1.f)) {
+      if (lane == 0) atomicOr(status, 2u);
+    } else {
+      // inverse CDF over the v bytes of unit z: lane l owns bytes [l*per, (l+1)*per)
+      const float* x = row + static_cast<size_t>(z) * v;
+      const float m = unit_max[z];
+      const int b0 = lane * per;
+      float part = 0.f;
+      for (int q = 0; q < per; ++q)
+        if (b0 + q < v) part += __expf(x[b0 + q] - m);
+      const float incl = warp_scan_incl(part, lane);
+      const float total = __shfl_sync(kFull, incl, 31);
+      const float thr = ub * total;
+      const unsigned hit = __ballot_sync(kFull, thr < incl);
+      byte = v - 1;   // rounding may leave no index: the last one
+      if (hit) {
+        const int src = __ffs(hit) - 1;
+        int found = -1;
+        const float before = __shfl_up_sync(kFull, incl, 1);
+        if (lane == src) {
+          float cum = lane == 0 ? 0.f : before;
+          for (int q = 0; q < per && found < 0; ++q)
+            if (b0 + q < v) {
+              cum += __expf(x[b0 + q] - m);
+              if (thr < cum) found = b0 + q;
+            }
+          if (found < 0) found = min(b0 + per, v) - 1;   // the lane's total passed the threshold: its last byte
+        }
+        byte = __shfl_sync(kFull, found, src);
+      }
+    }
+    if (lane == 0) out_bytes[w * n + i] = byte;
+    // evidence of the drafted byte under every input unit of the slot (a missing byte is marginalised)
+    if (lane < r) G[(w * n + i) * r + lane] = byte < 0 ? 0.f : row[static_cast<size_t>(lane) * v + byte] - unit_lse[lane];
+  }
+}
+
+}  // namespace mtpc

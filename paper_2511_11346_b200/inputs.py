@@ -47,22 +47,39 @@ class HeadShape:
         return self.num_sum_groups * self.r
 
 
-def bf16_round(x: np.ndarray) -> np.ndarray:
-    """Round fp32 values to the nearest bf16 (ties to even); returns fp32 holding bf16-representable values."""
-    x = np.ascontiguousarray(x, dtype=np.float32)
+_CHUNK = 1 << 22
+
+
+def _bf16_round_into(x: np.ndarray, out: np.ndarray) -> None:
     bits = x.view(np.uint32)
     lsb = (bits >> np.uint32(16)) & np.uint32(1)
     rounded = (bits + np.uint32(0x7FFF) + lsb) & np.uint32(0xFFFF0000)
-    return rounded.view(np.float32)
+    out[...] = rounded.view(np.float32)
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round fp32 values to the nearest bf16 (ties to even); returns fp32 holding bf16-representable values.
+    Large arrays are processed in chunks on a thread pool (no array-sized temporaries)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    flat = x.reshape(-1)
+    out = np.empty_like(flat)
+    total = flat.size
+    nchunks = (total + _CHUNK - 1) // _CHUNK
+    if nchunks <= 1:
+        _bf16_round_into(flat, out)
+    else:
+        def work(c):
+            lo, hi = c * _CHUNK, min(total, (c + 1) * _CHUNK)
+            _bf16_round_into(flat[lo:hi], out[lo:hi])
+        with ThreadPoolExecutor(max_workers=8) as ex:
+            list(ex.map(work, range(nchunks)))
+    return out.reshape(x.shape)
 
 
 def bf16_bits(x_rounded: np.ndarray) -> np.ndarray:
     """The uint16 bf16 bit patterns of values that are already bf16-representable."""
     x = np.ascontiguousarray(x_rounded, dtype=np.float32)
     return (x.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
-
-
-_CHUNK = 1 << 22
 
 
 def _normal(seed: int, stream: int, shape, std: float) -> np.ndarray:
@@ -129,22 +146,33 @@ class Workload:
     W_sum_raw: np.ndarray | None = None
 
 
+_last_weights: dict = {}     # the most recent head's weights (one entry: they can be GBs)
+
+
 def make_workload(name: str, shape: HeadShape, T: int, seed: int, *, target_kind: str | None = "uniform",
                   wpp: int = 0, weight_std: float = 0.02, trans_std: float = 1.0) -> Workload:
     hidden = _normal(seed, 1, (T, shape.d), 1.0)
-    W_emit = _normal(seed, 2, (shape.n, shape.r, shape.v, shape.d), weight_std)
-    W_sum = _normal(seed, 3, (shape.sum_rows, shape.d), weight_std)
-    T_static = None
-    if shape.family == HMM:
-        T_static = _normal(seed, 4, (max(shape.n - 1, 1), shape.r, shape.r), trans_std)[: shape.n - 1]
+    key = (seed, shape, weight_std, trans_std)
+    if _last_weights.get("key") == key:          # cells that share a head (same seed and shape) reuse its weights
+        W_emit, W_sum, T_static, W_emit_q, W_sum_q = _last_weights["value"]
+    else:
+        W_emit = _normal(seed, 2, (shape.n, shape.r, shape.v, shape.d), weight_std)
+        W_sum = _normal(seed, 3, (shape.sum_rows, shape.d), weight_std)
+        T_static = None
+        if shape.family == HMM:
+            T_static = _normal(seed, 4, (max(shape.n - 1, 1), shape.r, shape.r), trans_std)[: shape.n - 1]
+        W_emit_q, W_sum_q = bf16_round(W_emit), bf16_round(W_sum)
+        if shape.io_dtype != F32:
+            W_emit = W_sum = None                # only the rounded copies are kept
+        _last_weights.clear()
+        _last_weights.update(key=key, value=(W_emit, W_sum, T_static, W_emit_q, W_sum_q))
     targets = None
     if target_kind == "uniform":
         targets = uniform_targets(seed, 5, (T, shape.n), shape.v)
     elif target_kind == "zipf":
         targets = zipf_targets(seed, 5, (T, shape.n), shape.v)
     u = uniforms(seed, 6, (T * wpp, 2 * shape.n)) if wpp > 0 else None
-    wl = Workload(name, shape, T, bf16_round(hidden), bf16_round(W_emit), bf16_round(W_sum), T_static,
-                  targets, wpp, u)
+    wl = Workload(name, shape, T, bf16_round(hidden), W_emit_q, W_sum_q, T_static, targets, wpp, u)
     if shape.io_dtype == F32:
         wl.hidden_raw, wl.W_emit_raw, wl.W_sum_raw = hidden, W_emit, W_sum
     return wl
