@@ -21,6 +21,9 @@ using namespace mtpc;
 constexpr size_t kAlign = 256;
 constexpr int kMaxPhases = 5;
 constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA on sm_100
+// Hidden states of one rasterisation block of the projection kernel: small enough to stay L2-resident next to the
+// weight tiles streaming past (data read by all SMs ends up in both halves of the 126 MB L2).
+constexpr size_t kHiddenBlockBytes = 36u << 20;
 constexpr size_t kHmmTableSmemLimit = 96 * 1024;   // exp'd HMM transition tables kept in shared memory up to this size
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -227,6 +230,12 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   p.T = rows;
   p.m_tiles = (rows + kBlockM - 1) / kBlockM;
   p.kblocks = c.d / kBlockK;
+  {
+    const size_t tile_bytes = static_cast<size_t>(kBlockM) * c.d * 2;
+    const int cap_tiles = kHiddenBlockBytes / tile_bytes > 0 ? static_cast<int>(kHiddenBlockBytes / tile_bytes) : 1;
+    const int nblocks = (p.m_tiles + cap_tiles - 1) / cap_tiles;
+    p.m_block = (p.m_tiles + nblocks - 1) / nblocks;
+  }
   p.n = c.n; p.r = c.r; p.v = c.v;
   p.emit_units = c.n * c.r;
   p.num_groups = with_emit ? tl.num_groups : 0;

@@ -43,6 +43,7 @@ struct GemmParams {
   CUtensorMap tm_emit;   // W_emit  [n*r*v, d]    box 64 x tile_cols
   CUtensorMap tm_sum;    // W_sum   [S*r, d]      box 64 x sum_cols
   int T, m_tiles, kblocks;
+  int m_block;                       // m-tiles per rasterisation block (see tile_coord)
   int n, r, v;
   int emit_units;                    // n * r
   int num_groups;                    // emission groups in this launch (0: sum tiles only)
@@ -112,11 +113,28 @@ __device__ __forceinline__ bool bounded_wait_warp(uint32_t bar, uint32_t parity,
 struct TileCoord {
   int mt, is_sum, ntiles, cols, brow0, unit0, nunits;
 };
-// Work items: m-tile fastest, so the CTAs that run at the same time share one group's weights through L2.
+// Work items. Emission items come first, in blocks of m_block m-tiles: inside a block the m-tile runs fastest and
+// the group next, so the CTAs that run at the same time share a few groups' weights through L2 while the block's
+// hidden states (m_block x 128 rows) stay L2-resident for every group; a block is finished before the next one
+// starts, so the weights are streamed from HBM once per block and the hidden states once. Sum items follow,
+// m-tile fastest.
 __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int item) {
   TileCoord c;
-  const int g = item / p.m_tiles;
-  c.mt = item % p.m_tiles;
+  const int emit_items = p.num_groups * p.m_tiles;
+  int g;
+  if (item < emit_items) {
+    const int per_block = p.m_block * p.num_groups;
+    const int blk = item / per_block;
+    const int rem = item - blk * per_block;
+    const int m0 = blk * p.m_block;
+    const int mcount = min(p.m_block, p.m_tiles - m0);   // only the last block can be short
+    g = rem / mcount;
+    c.mt = m0 + (rem - g * mcount);
+  } else {
+    const int rem = item - emit_items;
+    g = p.num_groups + rem / p.m_tiles;
+    c.mt = rem % p.m_tiles;
+  }
   c.is_sum = g >= p.num_groups;
   if (c.is_sum) {
     c.ntiles = 1;
