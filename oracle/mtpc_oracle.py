@@ -13,6 +13,9 @@ What follows which passage:
   btree_eval        Eq. (BTree), recursive halving with a latent per internal node
   draft_sample      App. B.2, Algorithm 1 (ancestral sampling), with inverse-CDF categorical draws
   circuit_counts    App. C, Table 3 (sizes of the circuits and of the linear head)
+  prefix_logprob    Algorithm 3, "compute marginals": q(x_1..x_i) for i = 1..n, by summing the later bytes out
+  next_byte_logprob the conditional q(X_{s+1} | x_1..x_s) as a ratio of two such marginals
+  speculative_accept Algorithm 3, acceptance loop and the last byte (residual or target distribution)
 
 Readings taken where the paper is silent or garbled (each is listed in the design notes too):
   * BTree: the left half is the first floor(n/2) tokens; a child latent depends on its parent's latent
@@ -28,8 +31,11 @@ Readings taken where the paper is silent or garbled (each is listed in the desig
 Pins (tests/test_oracle_*.py): brute-force normalisation over all v^n strings; CP with r=1 equals the
 product of marginals; CP/HMM/BTree equal literal enumeration over latent assignments; HMM with identity
 transitions equals CP; BTree with n=2 equals CP; masked targets equal brute-force marginals; closed-form
-softmax cases; sampled frequencies match the exact joint (chi-squared); Table 3 counts. No function here
-is left unpinned.
+softmax cases; sampled frequencies match the exact joint (chi-squared); Table 3 counts; prefix marginals equal
+brute-force sums over the later bytes; the conditional sums to one and chains back to the joint; the
+acceptance stage reproduces a hand-computed example, accepts everything when target and draft agree, and its
+output bytes follow the TARGET model's distribution (chi-squared) whatever the draft is. No function here is
+left unpinned.
 """
 from __future__ import annotations
 
@@ -241,3 +247,96 @@ def draft_sample(family: int, h, W_emit, W_sum, T_static, wpp: int, u: np.ndarra
     g = evidence(logphi, x, pos)
     logprob = circuit_eval(family, logw[pos], g, T_static)
     return dict(bytes=x, logprob=logprob, unit=unit, margin=margin)
+
+
+# ----------------------------------------------------------------------------------------------------
+# prefix marginals and speculative acceptance (Algorithm 3)
+# ----------------------------------------------------------------------------------------------------
+def prefix_logprob(family: int, logw: np.ndarray, logphi: np.ndarray, T_static, x: np.ndarray,
+                   pos: np.ndarray | None = None) -> np.ndarray:
+    """log q(x_1..x_i | context) for i = 1..n (Algorithm 3, "compute marginals"): the joint with the bytes
+    x_{i+1}..x_n summed out, which a smooth and decomposable circuit does by letting those input units output 1
+    (App. B.1). Written as that definition: one masked evaluation per prefix length.  -> [W, n]."""
+    x = np.asarray(x)
+    W, n = x.shape
+    lw = logw if pos is None else logw[pos]
+    out = np.zeros((W, n))
+    for i in range(n):
+        masked = x.copy()
+        masked[:, i + 1:] = -1
+        out[:, i] = circuit_eval(family, lw, evidence(logphi, masked, pos), T_static)
+    return out
+
+
+def window_prefix_logprob(family: int, h, W_emit, W_sum, T_static, targets) -> np.ndarray:
+    """Prefix log-marginals of the observed window at every position: [T, n]; column n-1 is the joint."""
+    r = np.asarray(W_emit).shape[1]
+    return prefix_logprob(family, sum_unit_logw(h, W_sum, r), emission_logphi(h, W_emit), T_static, targets)
+
+
+def next_byte_logprob(family: int, logw: np.ndarray, logphi: np.ndarray, T_static, x: np.ndarray, s: np.ndarray,
+                      pos: np.ndarray | None = None) -> np.ndarray:
+    """log q(X_{s+1} = b | x_1..x_s, context) for every byte b: [W, v]. s[w] in [0, n) is the number of bytes
+    already fixed in window w. By definition of the conditional: the marginal of (x_1..x_s, b) with everything
+    after summed out, divided by the marginal of (x_1..x_s)."""
+    x = np.asarray(x)
+    W, n = x.shape
+    v = logphi.shape[-1]
+    lw = logw if pos is None else logw[pos]
+    cols = np.arange(n)[None, :]
+    base = np.where(cols < s[:, None], x, -1)
+    denom = circuit_eval(family, lw, evidence(logphi, base, pos), T_static)
+    out = np.zeros((W, v))
+    for b in range(v):
+        ext = np.where(cols == s[:, None], b, base)
+        out[:, b] = circuit_eval(family, lw, evidence(logphi, ext, pos), T_static) - denom
+    return out
+
+
+def speculative_accept(prefix_lq: np.ndarray, x: np.ndarray, p: np.ndarray, u: np.ndarray, next_byte_fn):
+    """The acceptance stage of Algorithm 3 for a batch of drafted windows.
+      prefix_lq [W, n]   log q(x_1..x_i) of the draft, i = 1..n
+      x         [W, n]   the drafted bytes
+      p         [W, n+1, v]  target-model conditionals p(X_{t+i} | x_{<=t+i-1}) along the draft, i = 1..n+1
+      u         [W, n+1] uniforms: column i is the alpha of the test on byte i+1; column n draws the last byte
+      next_byte_fn(rows, s) -> [len(rows), v]  log q(X_{s+1} | x_1..x_s) for the given windows (needed only
+                         where a byte was rejected)
+    Steps, in the algorithm's order: s = 0; while s < n: the draft's conditional of byte s+1 is the ratio of
+    consecutive prefix marginals (the first prefix marginal itself for s = 0); stop if alpha > p / q; else
+    s += 1. Then one more byte: from the residual max(0, p - q) / Z if s < n, from p otherwise; both draws are
+    inverse-CDF with the row's last uniform.
+    Returns dict(accepted [W], next_byte [W], margin [W]): margin = how close any decision of the window was to
+    flipping (min over the tests of |alpha - ratio| and the final draw's distance to a CDF boundary)."""
+    x = np.asarray(x)
+    W, n = x.shape
+    v = p.shape[-1]
+    p = np.asarray(p, dtype=np.float64)
+    u = np.asarray(u, dtype=np.float64)
+    accepted = np.zeros(W, dtype=np.int64)
+    margin = np.full(W, np.inf)
+    for w in range(W):
+        s = 0
+        while s < n:
+            alpha = u[w, s]
+            lq = prefix_lq[w, s] - (prefix_lq[w, s - 1] if s > 0 else 0.0)
+            ratio = p[w, s, x[w, s]] / np.exp(lq)
+            margin[w] = min(margin[w], abs(alpha - ratio))
+            if alpha > ratio:
+                break
+            s += 1
+        accepted[w] = s
+    next_byte = np.zeros(W, dtype=np.int64)
+    rej = np.nonzero(accepted < n)[0]
+    if len(rej):
+        qn = np.exp(next_byte_fn(rej, accepted[rej]))
+        m = np.maximum(0.0, p[rej, accepted[rej], :] - qn)
+        resid = m / m.sum(axis=-1, keepdims=True)
+        idx, mg = inv_cdf(np.log(np.maximum(resid, 1e-300)), u[rej, n])
+        next_byte[rej] = idx
+        margin[rej] = np.minimum(margin[rej], mg)
+    full = np.nonzero(accepted == n)[0]
+    if len(full):
+        idx, mg = inv_cdf(np.log(np.maximum(p[full, n, :], 1e-300)), u[full, n])
+        next_byte[full] = idx
+        margin[full] = np.minimum(margin[full], mg)
+    return dict(accepted=accepted, next_byte=next_byte, margin=margin)

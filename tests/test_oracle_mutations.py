@@ -113,6 +113,56 @@ def masked_gap(orc):
     return float(np.abs(g[0, 0]).max() + np.abs(g[0, 1] - logphi[0, 1, :, 2]).max())
 
 
+def prefix_gap(orc):
+    """Prefix marginals against explicit sums of the joint over the later bytes (tiny HMM)."""
+    rng = np.random.default_rng(6)
+    n, r, v = 3, 2, 3
+    pi, A, phi = pins.rand_simplex(rng, r), pins.rand_simplex(rng, n - 1, r, r), pins.rand_simplex(rng, n, r, v)
+    table = np.zeros((v,) * n)
+    for x in itertools.product(range(v), repeat=n):
+        table[x] = pins.enum_hmm(pi, A, phi, x)
+    x = np.array([[2, 0, 1]])
+    with np.errstate(divide="ignore"):
+        got = orc.prefix_logprob(orc.HMM, np.log(pi)[None, None], np.log(phi)[None], np.log(A), x)
+    # np.log(A) are already log-probabilities: log_softmax leaves them unchanged
+    want = [table[2].sum(), table[2, 0].sum(), table[2, 0, 1]]
+    return float(np.abs(got[0] - np.log(want)).max())
+
+
+def conditional_gap(orc):
+    rng = np.random.default_rng(7)
+    n, r, v = 3, 2, 3
+    omega, phi = pins.rand_simplex(rng, r), pins.rand_simplex(rng, n, r, v)
+    table = np.zeros((v,) * n)
+    for x in itertools.product(range(v), repeat=n):
+        table[x] = pins.enum_cp(omega, phi, x)
+    x = np.array([[1, 2, 0]])
+    got = orc.next_byte_logprob(orc.CP, np.log(omega)[None, None], np.log(phi)[None], None, x, np.array([1]))
+    want = table[1].sum(axis=1) / table[1].sum()
+    return float(np.abs(np.exp(got[0]) - want).max())
+
+
+def accept_wrong(orc):
+    """The example worked by hand in test_oracle_speculative.py, plus a full acceptance."""
+    p = np.array([[[0.5, 0.3, 0.2], [0.1, 0.3, 0.6], [0.2, 0.2, 0.6]]])
+    q_first = np.log(np.array([[0.2, 0.7, 0.1]]))
+    q_second = np.log(np.array([[0.25, 0.25, 0.5]]))
+    bad = 0.0
+    out = orc.speculative_accept(np.log(np.array([[0.7, 0.35]])), np.array([[1, 2]]), p, np.array([[0.5, 0.0, 0.8]]),
+                                 lambda rows, s: q_first)
+    bad += out["accepted"].tolist() != [0] or out["next_byte"].tolist() != [2]
+    out = orc.speculative_accept(np.log(np.array([[0.7, 0.35]])), np.array([[1, 2]]), p, np.array([[0.4, 0.999, 0.15]]),
+                                 lambda rows, s: q_second)
+    bad += out["accepted"].tolist() != [2] or out["next_byte"].tolist() != [0]    # p(X_3 | 1, 2) = (0.2, 0.2, 0.6)
+    out = orc.speculative_accept(np.log(np.array([[0.7, 0.175]])), np.array([[1, 0]]), p, np.array([[0.1, 0.41, 0.3]]),
+                                 lambda rows, s: q_second)
+    bad += out["accepted"].tolist() != [1] or out["next_byte"].tolist() != [1]
+    out = orc.speculative_accept(np.log(np.array([[0.7, 0.175]])), np.array([[1, 0]]), p, np.array([[0.1, 0.39, 0.3]]),
+                                 lambda rows, s: q_second)
+    bad += out["accepted"].tolist() != [2] or out["next_byte"].tolist() != [1]
+    return float(bad)
+
+
 MUTANTS = [
     # (what is planted, old text, new text, pin that must notice)
     ("mixture weights dropped from Eq. CP", "logsumexp(logw + g.sum(axis=1), axis=-1)", "logsumexp(g.sum(axis=1), axis=-1)", cp_gap),
@@ -136,6 +186,25 @@ MUTANTS = [
     ("tree sampler gives tokens to the wrong node", "zs[:, n // 2 - 1 + i // 2]", "zs[:, n // 2 - 1 + (i + 1) // 2 % (n // 2)]",
      btree_sampler_wrong),
     ("marginalised byte not set to one", "return np.where((x < 0)[:, :, None], 0.0, g)", "return g", masked_gap),
+    ("prefix of length i keeps byte i+1", "masked[:, i + 1:] = -1", "masked[:, i + 2:] = -1", prefix_gap),
+    ("prefix of length i drops byte i", "masked[:, i + 1:] = -1", "masked[:, i:] = -1", prefix_gap),
+    ("conditional not divided by the prefix marginal", "evidence(logphi, ext, pos), T_static) - denom",
+     "evidence(logphi, ext, pos), T_static)", conditional_gap),
+    ("conditional places the byte one slot late", "ext = np.where(cols == s[:, None], b, base)",
+     "ext = np.where(cols == s[:, None] + 1, b, base)", conditional_gap),
+    ("acceptance uses the joint prefix instead of the conditional", "lq = prefix_lq[w, s] - (prefix_lq[w, s - 1] if s > 0 else 0.0)",
+     "lq = prefix_lq[w, s]", accept_wrong),
+    ("acceptance ratio inverted", "ratio = p[w, s, x[w, s]] / np.exp(lq)", "ratio = np.exp(lq) / p[w, s, x[w, s]]", accept_wrong),
+    ("acceptance test reversed", "if alpha > ratio:", "if alpha < ratio:", accept_wrong),
+    ("residual taken as q - p", "m = np.maximum(0.0, p[rej, accepted[rej], :] - qn)", "m = np.maximum(0.0, qn - p[rej, accepted[rej], :])",
+     accept_wrong),
+    ("residual not clipped at zero", "m = np.maximum(0.0, p[rej, accepted[rej], :] - qn)", "m = np.abs(p[rej, accepted[rej], :] - qn)",
+     accept_wrong),
+    ("residual uses the target row of the first byte", "m = np.maximum(0.0, p[rej, accepted[rej], :] - qn)",
+     "m = np.maximum(0.0, p[rej, 0, :] - qn)", accept_wrong),
+    ("byte after a full acceptance drawn from the wrong target row", "inv_cdf(np.log(np.maximum(p[full, n, :], 1e-300)), u[full, n])",
+     "inv_cdf(np.log(np.maximum(p[full, n - 1, :], 1e-300)), u[full, n])", accept_wrong),
+    ("acceptance test uses the last uniform", "alpha = u[w, s]", "alpha = u[w, n]", accept_wrong),
 ]
 
 
