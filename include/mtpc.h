@@ -48,7 +48,8 @@ enum {
   MTPC_ERR_WORKSPACE = -4,   /* workspace too small or misaligned                                     */
   MTPC_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed (includes: no device)               */
   MTPC_ERR_TIMEOUT = -6,     /* mtpc_get_status: a device-side bounded wait gave up                   */
-  MTPC_ERR_STATIC_SCRATCH = -7 /* mtpc_window_logprob_static: the call needs more than the built-in array */
+  MTPC_ERR_STATIC_SCRATCH = -7, /* mtpc_window_logprob_static: the call needs more than the built-in array */
+  MTPC_ERR_STATE = -8        /* mtpc_speculative_accept without a matching draft call before it         */
 };
 
 /* Bits of the device status word. */
@@ -122,6 +123,61 @@ int mtpc_draft_sample(mtpc_head* head, const void* hidden, int32_t P, int32_t wp
                       int32_t* out_bytes, float* out_logprob, void* stream);
 
 /*
+ * Prefix log-marginals (Algorithm 3, "compute marginals"; also the per-slot terms of Eq. 6):
+ *   out_prefix_logprob[t, i] = log q(x_{t,0..i} | h_t), the joint with the bytes after slot i summed out, which a
+ *   smooth and decomposable circuit gives in one pass (App. B.1). Column n-1 equals mtpc_window_logprob's output.
+ *   CP: log-sum-exp over the components of the first i+1 slots; HMM: log-sum-exp of the forward message alpha_i;
+ *   BTree: the subtrees right of token i evaluate to one, only the path from its owner to the root is re-evaluated.
+ * mtpc_window_prefix_logprob: arguments as mtpc_window_logprob, out_prefix_logprob dev [T, n] fp32.
+ * mtpc_draft_sample_prefix:   arguments as mtpc_draft_sample, out_prefix_logprob dev [P*wpp, n] fp32 for the
+ *                             drafted windows (what the acceptance stage consumes).
+ */
+int mtpc_window_prefix_logprob(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t T,
+                               float* out_prefix_logprob, void* stream);
+int mtpc_draft_sample_prefix(mtpc_head* head, const void* hidden, int32_t P, int32_t wpp, const float* uniforms,
+                             int32_t* out_bytes, float* out_prefix_logprob, void* stream);
+
+/*
+ * Acceptance stage of speculative sampling (Algorithm 3, from "determine the number of accepted tokens" to the
+ * last byte), for the P*wpp windows of the head's most recent draft. The target model's conditionals are an input:
+ * the LLM that produces them is outside this library.
+ *   draft_bytes     dev [W, n] int32, W = P*wpp: the drafted windows (as written by mtpc_draft_sample*).
+ *   prefix_logprob  dev [W, n] fp32: their prefix log-marginals (as written by mtpc_draft_sample_prefix).
+ *   target_probs    dev [W, n+1, v] fp32: row i is p(X_{t+i+1} | context, draft bytes 0..i-1), probabilities.
+ *   accept_uniforms dev [W, n+1] fp32 in [0,1): column i is the alpha of the test on byte i; column n draws the
+ *                   last byte.
+ *   out_accepted    dev [W] int32: s in [0, n], the number of accepted draft bytes: byte i is accepted while
+ *                   alpha_i <= p(x_i) / q(x_i | x_0..x_{i-1}), q being the ratio of consecutive prefix marginals.
+ *   out_next_byte   dev [W] int32: the byte that follows the accepted ones: drawn from target row n if s = n, else
+ *                   from the residual max(0, p - q(. | x_0..x_{s-1})) / Z with p = target row s. Inverse-CDF draws
+ *                   as in mtpc_draft_sample. (With zero residual mass, which exact arithmetic excludes after a
+ *                   rejection, the last byte v-1 is returned.)
+ * The conditional q(. | x_0..x_{s-1}) is a mixture of the r input units of slot s whose weights are the posterior of
+ * the latent that owns the slot; it is evaluated from the logits the draft call left in the workspace. Hence:
+ *   - the call must follow mtpc_draft_sample / mtpc_draft_sample_prefix on this head with the same P and hidden
+ *     states, with no other call on the head in between, else MTPC_ERR_STATE;
+ *   - only drafts of P <= 128 positions with r <= 32 keep that state (decode-time batches): otherwise
+ *     MTPC_ERR_UNSUPPORTED.
+ * A uniform outside [0,1) or a draft byte outside [0,v) sets the status bit and yields -1 / -1 for that window.
+ */
+int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32_t* draft_bytes,
+                            const float* prefix_logprob, const float* target_probs, const float* accept_uniforms,
+                            int32_t* out_accepted, int32_t* out_next_byte, void* stream);
+
+/*
+ * Training loss over overlapping windows (Eq. 6): num_sequences sequences of sequence_length positions each
+ * (T = num_sequences * sequence_length rows of hidden / targets, sequence-major).
+ *   out_slot_loss[j] = L_j = -(1/N) sum_i (1/V_ij) sum_t log q(x_{t,j} | h_t, x_{t,0..j-1}),
+ *   out_loss[0]      = sum_j gamma^j L_j   (j from 0; the paper's gamma^(j-1) with j from 1),
+ * where the conditional is the difference of consecutive prefix log-marginals, a negative target marks an invalid
+ * (masked, marginalised) byte and V_ij counts the valid targets of slot j in sequence i (a slot with none
+ * contributes 0). Forward value only. out_slot_loss dev [n] fp32, out_loss dev [1] fp32. The reduction order is
+ * fixed: the same inputs give the same bits.
+ */
+int mtpc_window_loss(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,
+                     int32_t sequence_length, float gamma, float* out_slot_loss, float* out_loss, void* stream);
+
+/*
  * Host-buffer variants: same results, but hidden / targets / uniforms are HOST pointers (pinned memory for
  * full copy speed) and the outputs are written to HOST buffers. The copies to and from the device go through
  * staging areas in the workspace on `stream`; the call returns after the stream has been synchronised, so
@@ -146,7 +202,9 @@ int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags);
  * of the call made `calls_back` calls ago (0 = the most recent) and writes up to `capacity` phase durations
  * in milliseconds, *out_count = number of phases that call had:
  *   mtpc_window_logprob: [0] projection GEMM + fused epilogue, [1] circuit evaluation.
- *   mtpc_draft_sample:   P <= 128 positions and r <= 32: [0] one pass over all weights (logits of every unit),
+ *   mtpc_window_prefix_logprob, mtpc_window_loss: as mtpc_window_logprob (the loss reduction is not timed).
+ *   mtpc_speculative_accept: [0] the acceptance kernel.
+ *   mtpc_draft_sample, mtpc_draft_sample_prefix:   P <= 128 positions and r <= 32: [0] one pass over all weights (logits of every unit),
  *                        [1] per-slot latent + byte draws and evidence, [2] circuit evaluation.
  *                        Otherwise: [0] sum-unit GEMM, [1] latent sampling, [2] GEMM + inverse-CDF epilogue,
  *                        [3] GEMM + gather epilogue on the drafted bytes, [4] circuit evaluation.

@@ -16,6 +16,7 @@ What follows which passage:
   prefix_logprob    Algorithm 3, "compute marginals": q(x_1..x_i) for i = 1..n, by summing the later bytes out
   next_byte_logprob the conditional q(X_{s+1} | x_1..x_s) as a ratio of two such marginals
   speculative_accept Algorithm 3, acceptance loop and the last byte (residual or target distribution)
+  composite_loss    Eq. (6): per-slot negative log-likelihood with valid-token normalisation and discount gamma
 
 Readings taken where the paper is silent or garbled (each is listed in the design notes too):
   * BTree: the left half is the first floor(n/2) tokens; a child latent depends on its parent's latent
@@ -34,8 +35,9 @@ transitions equals CP; BTree with n=2 equals CP; masked targets equal brute-forc
 softmax cases; sampled frequencies match the exact joint (chi-squared); Table 3 counts; prefix marginals equal
 brute-force sums over the later bytes; the conditional sums to one and chains back to the joint; the
 acceptance stage reproduces a hand-computed example, accepts everything when target and draft agree, and its
-output bytes follow the TARGET model's distribution (chi-squared) whatever the draft is. No function here is
-left unpinned.
+output bytes follow the TARGET model's distribution (chi-squared) whatever the draft is; the loss reproduces a
+hand-computed example and, with gamma = 1 and every byte valid, the mean joint negative log-likelihood. No
+function here is left unpinned.
 """
 from __future__ import annotations
 
@@ -306,37 +308,73 @@ def speculative_accept(prefix_lq: np.ndarray, x: np.ndarray, p: np.ndarray, u: n
     s += 1. Then one more byte: from the residual max(0, p - q) / Z if s < n, from p otherwise; both draws are
     inverse-CDF with the row's last uniform.
     Returns dict(accepted [W], next_byte [W], margin [W]): margin = how close any decision of the window was to
-    flipping (min over the tests of |alpha - ratio| and the final draw's distance to a CDF boundary)."""
+    flipping (min over the tests of |alpha - ratio| = margin_alpha, and the final draw's distance to a CDF
+    boundary of the normalised distribution = margin_final); resid_mass [W] = Z of the residual (1 where all n
+    bytes were accepted)."""
     x = np.asarray(x)
     W, n = x.shape
     v = p.shape[-1]
     p = np.asarray(p, dtype=np.float64)
     u = np.asarray(u, dtype=np.float64)
     accepted = np.zeros(W, dtype=np.int64)
-    margin = np.full(W, np.inf)
+    margin_alpha = np.full(W, np.inf)
     for w in range(W):
         s = 0
         while s < n:
             alpha = u[w, s]
             lq = prefix_lq[w, s] - (prefix_lq[w, s - 1] if s > 0 else 0.0)
             ratio = p[w, s, x[w, s]] / np.exp(lq)
-            margin[w] = min(margin[w], abs(alpha - ratio))
+            margin_alpha[w] = min(margin_alpha[w], abs(alpha - ratio))
             if alpha > ratio:
                 break
             s += 1
         accepted[w] = s
     next_byte = np.zeros(W, dtype=np.int64)
+    margin_final = np.full(W, np.inf)
+    resid_mass = np.ones(W)
     rej = np.nonzero(accepted < n)[0]
     if len(rej):
         qn = np.exp(next_byte_fn(rej, accepted[rej]))
         m = np.maximum(0.0, p[rej, accepted[rej], :] - qn)
+        resid_mass[rej] = m.sum(axis=-1)
         resid = m / m.sum(axis=-1, keepdims=True)
         idx, mg = inv_cdf(np.log(np.maximum(resid, 1e-300)), u[rej, n])
         next_byte[rej] = idx
-        margin[rej] = np.minimum(margin[rej], mg)
+        margin_final[rej] = mg
     full = np.nonzero(accepted == n)[0]
     if len(full):
         idx, mg = inv_cdf(np.log(np.maximum(p[full, n, :], 1e-300)), u[full, n])
         next_byte[full] = idx
-        margin[full] = np.minimum(margin[full], mg)
-    return dict(accepted=accepted, next_byte=next_byte, margin=margin)
+        margin_final[full] = mg
+    margin = np.minimum(margin_alpha, margin_final)
+    return dict(accepted=accepted, next_byte=next_byte, margin=margin, margin_alpha=margin_alpha,
+                margin_final=margin_final, resid_mass=resid_mass)
+
+
+# ----------------------------------------------------------------------------------------------------
+# training loss over overlapping windows (Eq. 6)
+# ----------------------------------------------------------------------------------------------------
+def composite_loss(prefix_lq: np.ndarray, targets: np.ndarray, num_sequences: int, gamma: float):
+    """Eq. (6): L_j = -(1/N) sum_i (1/V_ij) sum_t log p(x_{t+j} | x_{<t+j}) and L = sum_j gamma^(j-1) L_j.
+    prefix_lq [N*L, n] are the prefix log-marginals of every position's window (sequence-major rows); the
+    conditional of slot j given the context and the window's earlier bytes is prefix[:, j] - prefix[:, j-1].
+    A negative target is an invalid byte: it is left out of the sum and of the count V_ij (a slot of a sequence
+    with no valid byte contributes nothing). Returns (L_j for every slot [n], L)."""
+    pre = np.asarray(prefix_lq, dtype=np.float64)
+    tg = np.asarray(targets)
+    T, n = pre.shape
+    N = num_sequences
+    L = T // N
+    cond = pre - np.concatenate([np.zeros((T, 1)), pre[:, :-1]], axis=1)
+    slot = np.zeros(n)
+    for j in range(n):
+        acc = 0.0
+        for i in range(N):
+            rows = slice(i * L, (i + 1) * L)
+            valid = tg[rows, j] >= 0
+            V = int(valid.sum())
+            if V:
+                acc += cond[rows, j][valid].sum() / V
+        slot[j] = -acc / N
+    total = float(sum(gamma ** j * slot[j] for j in range(n)))
+    return slot, total

@@ -20,9 +20,11 @@ EXPORTS = [
     "mtpc_workspace_bytes", "mtpc_create_head", "mtpc_window_logprob", "mtpc_draft_sample",
     "mtpc_window_logprob_host", "mtpc_draft_sample_host", "mtpc_get_status", "mtpc_set_timing", "mtpc_get_timing",
     "mtpc_launch_count", "mtpc_destroy", "mtpc_status_string", "mtpc_window_logprob_static",
+    "mtpc_window_prefix_logprob", "mtpc_draft_sample_prefix", "mtpc_speculative_accept", "mtpc_window_loss",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 ERR_STATIC_SCRATCH = -7
+ERR_STATE = -8
 
 
 class MtpcConfig(ctypes.Structure):
@@ -62,6 +64,10 @@ def lib() -> ctypes.CDLL:
     L.mtpc_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
     L.mtpc_destroy.argtypes = [vp]
     L.mtpc_window_logprob_static.argtypes = [ctypes.POINTER(MtpcConfig), vp, vp, vp, vp, vp, i32, vp, vp, vp]
+    L.mtpc_window_prefix_logprob.argtypes = [vp, vp, vp, i32, vp, vp]
+    L.mtpc_draft_sample_prefix.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    L.mtpc_speculative_accept.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    L.mtpc_window_loss.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp, vp, vp]
     L.mtpc_status_string.argtypes = [ctypes.c_int]
     L.mtpc_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -136,6 +142,28 @@ class MtpcHead:
         P = hidden.shape[0]
         _check(lib().mtpc_draft_sample(self.handle, _ptr(hidden), P, wpp, _ptr(uniforms), _ptr(out_bytes),
                                        _ptr(out_logprob), _stream(stream)), "mtpc_draft_sample")
+
+    def mtpc_window_prefix_logprob(self, hidden, targets, out_prefix_logprob, stream=None) -> None:
+        T = hidden.shape[0]
+        _check(lib().mtpc_window_prefix_logprob(self.handle, _ptr(hidden), _ptr(targets), T, _ptr(out_prefix_logprob),
+                                                _stream(stream)), "mtpc_window_prefix_logprob")
+
+    def mtpc_draft_sample_prefix(self, hidden, wpp: int, uniforms, out_bytes, out_prefix_logprob, stream=None) -> None:
+        P = hidden.shape[0]
+        _check(lib().mtpc_draft_sample_prefix(self.handle, _ptr(hidden), P, wpp, _ptr(uniforms), _ptr(out_bytes),
+                                              _ptr(out_prefix_logprob), _stream(stream)), "mtpc_draft_sample_prefix")
+
+    def mtpc_speculative_accept(self, P: int, wpp: int, draft_bytes, prefix_logprob, target_probs, accept_uniforms,
+                                out_accepted, out_next_byte, stream=None) -> None:
+        _check(lib().mtpc_speculative_accept(self.handle, P, wpp, _ptr(draft_bytes), _ptr(prefix_logprob),
+                                             _ptr(target_probs), _ptr(accept_uniforms), _ptr(out_accepted),
+                                             _ptr(out_next_byte), _stream(stream)), "mtpc_speculative_accept")
+
+    def mtpc_window_loss(self, hidden, targets, num_sequences: int, sequence_length: int, gamma: float, out_slot_loss,
+                         out_loss, stream=None) -> None:
+        _check(lib().mtpc_window_loss(self.handle, _ptr(hidden), _ptr(targets), num_sequences, sequence_length,
+                                      ctypes.c_float(gamma), _ptr(out_slot_loss), _ptr(out_loss), _stream(stream)),
+               "mtpc_window_loss")
 
     # -- host-buffer calls (copies inside; outputs ready on return)
     def mtpc_window_logprob_host(self, hidden_host, targets_host, out_logprob_host, stream=None) -> None:

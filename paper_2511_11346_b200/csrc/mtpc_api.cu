@@ -45,7 +45,8 @@ struct Layout {
   Tiling sm;            // sampling mode: one unit per group, equal tiles of <= 256 columns
   size_t max_windows;
   // workspace offsets (bytes)
-  size_t off_status, off_wemit, off_wsum, off_hidden, off_logA, off_G, off_logw, off_sel, off_logits;
+  size_t off_status, off_wemit, off_wsum, off_hidden, off_logA, off_G, off_logw, off_sel, off_logits, off_unit_lse;
+  size_t off_prefix, off_partial;   // training loss: prefix log-marginals [max_positions, n], per-sequence terms
   int decode_max_p;     // positions the few-position draft path can take (0: path not available)
   size_t off_h_hidden, off_h_targets, off_h_uniforms, off_h_bytes, off_h_out;
   size_t total;
@@ -126,6 +127,9 @@ int plan(const mtpc_config& c, Layout* L) {
   L->off_sel = take(L->max_windows * c.n * 4);
   L->decode_max_p = c.r <= 32 ? (c.max_positions < kDecodeMaxP ? c.max_positions : kDecodeMaxP) : 0;
   L->off_logits = take(static_cast<size_t>(L->decode_max_p) * emit_units * c.v * 4);
+  L->off_unit_lse = take(static_cast<size_t>(L->decode_max_p) * emit_units * 4);
+  L->off_prefix = take(static_cast<size_t>(c.max_positions) * c.n * 4);
+  L->off_partial = take(static_cast<size_t>(c.max_positions) * c.n * 4);
   L->off_h_hidden = take(static_cast<size_t>(c.max_positions) * c.d * elt);
   L->off_h_targets = take(static_cast<size_t>(c.max_positions) * c.n * 4);
   L->off_h_uniforms = take(L->max_windows * 2 * c.n * 4);
@@ -178,6 +182,7 @@ struct mtpc_head {
   CUtensorMap tm_emit_dec, tm_sum_dec;          // the same matrices in the few-position draft path's tiles
   int decode_tile_rows, decode_sum_tile_rows;
   int num_sms;
+  int draft_P;              // positions whose logits the few-position draft path left in the workspace (0: none)
   int ring;                 // calls whose per-kernel events are retained (0 = timing off)
   cudaEvent_t* ev;          // [ring][kMaxPhases][2]
   int* ring_phases;         // [ring] phases recorded by the call in that slot
@@ -266,7 +271,16 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   return check_launch();
 }
 
-int launch_circuit(mtpc_head* h, int W, int wpp, float* out, cudaStream_t st) {
+// Shared memory of one CTA of the binary-tree circuit kernel (see circuit_btree_kernel).
+size_t btree_smem_bytes(int n, int r, bool with_prefix) {
+  const size_t per_warp = static_cast<size_t>(n - 1) * r + static_cast<size_t>(r) * (r + 1) +
+                          (with_prefix ? static_cast<size_t>(n - 1) * r + r : 0);
+  return kCircuitWarps * per_warp * sizeof(float);
+}
+
+// Circuit evaluation of W windows: out[w] = joint log-prob (may be NULL when prefix is given); prefix (may be NULL)
+// [W, n] = log-marginals of the prefixes x_0..x_i.
+int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cudaStream_t st) {
   if (W <= 0) return MTPC_OK;
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
@@ -275,19 +289,42 @@ int launch_circuit(mtpc_head* h, int W, int wpp, float* out, cudaStream_t st) {
   const int blocks = (W + kCircuitWarps - 1) / kCircuitWarps;
   const int threads = kCircuitWarps * 32;
   if (c.family == MTPC_CP) {
-    circuit_cp_kernel<<<blocks, threads, 0, st>>>(G, logw, out, W, wpp, c.n, c.r, L.sum_rows);
+    circuit_cp_kernel<<<blocks, threads, 0, st>>>(G, logw, out, prefix, W, wpp, c.n, c.r, L.sum_rows);
   } else if (c.family == MTPC_HMM) {
     const size_t table_bytes = static_cast<size_t>(c.n - 1) * c.r * c.r * 4;
     const int in_smem = table_bytes <= kHmmTableSmemLimit;
     const int cap = 4 * h->num_sms;                      // CTAs stride over the windows: the tables are staged once each
     circuit_hmm_kernel<<<blocks < cap ? blocks : cap, threads, in_smem ? table_bytes : 0, st>>>(
-        G, logw, at<float>(h, L.off_logA), out, W, wpp, c.n, c.r, L.sum_rows, in_smem);
+        G, logw, at<float>(h, L.off_logA), out, prefix, W, wpp, c.n, c.r, L.sum_rows, in_smem);
+  } else if (prefix != nullptr) {
+    circuit_btree_kernel<true><<<blocks, threads, btree_smem_bytes(c.n, c.r, true), st>>>(G, logw, out, prefix, W, wpp,
+                                                                                        c.n, c.r, L.sum_rows);
   } else {
-    const size_t smem = static_cast<size_t>(kCircuitWarps) * ((c.n - 1) * c.r + c.r * (c.r + 1)) * 4;
-    circuit_btree_kernel<<<blocks, threads, smem, st>>>(G, logw, out, W, wpp, c.n, c.r, L.sum_rows);
+    circuit_btree_kernel<false><<<blocks, threads, btree_smem_bytes(c.n, c.r, false), st>>>(G, logw, out, nullptr, W,
+                                                                                          wpp, c.n, c.r, L.sum_rows);
   }
   h->launches++;
   return check_launch();
+}
+
+// Kernel attributes that depend on the head's shape; they are per function, so every head (and the static entry
+// point) sets them to what it needs or more.
+bool set_circuit_attributes(const mtpc_config& c) {
+  bool fail = false;
+  if (c.family == MTPC_HMM)
+    fail |= cudaFuncSetAttribute(circuit_hmm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kHmmTableSmemLimit)) != cudaSuccess;
+  if (c.family == MTPC_BTREE) {
+    const int plain = static_cast<int>(btree_smem_bytes(c.n, c.r, false));
+    const int pre = static_cast<int>(btree_smem_bytes(c.n, c.r, true));
+    if (plain > 48 * 1024)
+      fail |= cudaFuncSetAttribute(circuit_btree_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, plain) !=
+              cudaSuccess;
+    if (pre > 48 * 1024)
+      fail |= cudaFuncSetAttribute(circuit_btree_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, pre) !=
+              cudaSuccess;
+  }
+  return !fail;
 }
 
 // Rows per emission tile of the few-position draft path: the height in [64, 128] (multiple of 8) that leaves the
@@ -361,9 +398,11 @@ int stage_hidden(mtpc_head* h, const void* hidden, int rows, const void** out_bf
   return MTPC_OK;
 }
 
-int window_logprob_impl(mtpc_head* h, const void* hidden, const int32_t* targets, int32_t T, float* out,
+// out [T] (joint) and / or prefix [T, n] (prefix log-marginals); either may be NULL, not both.
+int window_logprob_impl(mtpc_head* h, const void* hidden, const int32_t* targets, int32_t T, float* out, float* prefix,
                         cudaStream_t st) {
   const void* hb = nullptr;
+  h->draft_P = 0;   // log omega of the last draft is overwritten below
   int rc = stage_hidden(h, hidden, T, &hb, st);
   if (rc != MTPC_OK) return rc;
   PhaseTimer pt(h, st);
@@ -372,13 +411,14 @@ int window_logprob_impl(mtpc_head* h, const void* hidden, const int32_t* targets
   pt.end();
   if (rc != MTPC_OK) return rc;
   pt.begin();
-  rc = launch_circuit(h, T, 1, out, st);
+  rc = launch_circuit(h, T, 1, out, prefix, st);
   pt.end();
   return rc;
 }
 
+// out_logprob [W] (joint) and / or out_prefix [W, n] (prefix log-marginals of the draft); either may be NULL, not both.
 int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, const float* uniforms,
-                      int32_t* out_bytes, float* out_logprob, cudaStream_t st) {
+                      int32_t* out_bytes, float* out_logprob, float* out_prefix, cudaStream_t st) {
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
   const int W = P * wpp;
@@ -386,6 +426,7 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   int rc = stage_hidden(h, hidden, P, &hb, st);
   if (rc != MTPC_OK) return rc;
   PhaseTimer pt(h, st);
+  h->draft_P = 0;
   if (P <= L.decode_max_p) {
     // Few positions: every weight row is read once. 1. all logits (emission -> scratch, sum units -> log omega)
     // 2. per (position, slot): latent draws, byte draws, evidence of the drafted bytes  3. circuit evaluation
@@ -396,12 +437,14 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
     pt.begin();
     draft_slot_kernel<<<dim3(c.n, P), kSlotThreads, 2 * c.r * sizeof(float), st>>>(
         c.family, at<float>(h, L.off_logits), at<float>(h, L.off_logw), at<float>(h, L.off_logA), uniforms, out_bytes,
-        at<float>(h, L.off_G), at<unsigned>(h, L.off_status), wpp, c.n, c.r, c.v, L.sum_rows);
+        at<float>(h, L.off_G), at<float>(h, L.off_unit_lse), at<unsigned>(h, L.off_status), wpp, c.n, c.r, c.v,
+        L.sum_rows);
     h->launches++;
+    h->draft_P = P;
     pt.end();
     if ((rc = check_launch()) != MTPC_OK) return rc;
     pt.begin();
-    rc = launch_circuit(h, W, wpp, out_logprob, st);
+    rc = launch_circuit(h, W, wpp, out_logprob, out_prefix, st);
     pt.end();
     return rc;
   }
@@ -428,7 +471,7 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   pt.end();
   if (rc != MTPC_OK) return rc;
   pt.begin();
-  rc = launch_circuit(h, W, wpp, out_logprob, st);
+  rc = launch_circuit(h, W, wpp, out_logprob, out_prefix, st);
   pt.end();
   return rc;
 }
@@ -480,14 +523,12 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
                                kSmemLimit) != cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
           cudaSuccess;
-  if (cfg->family == MTPC_HMM)
-    fail |= cudaFuncSetAttribute(circuit_hmm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kHmmTableSmemLimit)) != cudaSuccess;
-  if (cfg->family == MTPC_BTREE) {
-    const int smem = kCircuitWarps * ((cfg->n - 1) * cfg->r + cfg->r * (cfg->r + 1)) * 4;
+  fail |= !set_circuit_attributes(*cfg);
+  {
+    const size_t smem = kAcceptWarps * accept_warp_floats(cfg->family, cfg->n, cfg->r, cfg->v) * sizeof(float);
     if (smem > 48 * 1024)
-      fail |= cudaFuncSetAttribute(circuit_btree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-              cudaSuccess;
+      fail |= cudaFuncSetAttribute(spec_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   static_cast<int>(smem)) != cudaSuccess;
   }
   fail |= cudaMemsetAsync(h->ws + L.off_status, 0, 256, st) != cudaSuccess;
   if (fail) { delete h; return MTPC_ERR_CUDA; }
@@ -531,7 +572,16 @@ int mtpc_window_logprob(mtpc_head* head, const void* hidden, const int32_t* targ
   if (rc != MTPC_OK) return rc;
   if (T == 0) return MTPC_OK;
   if (!hidden || !targets || !out_logprob) return MTPC_ERR_NULL;
-  return window_logprob_impl(head, hidden, targets, T, out_logprob, static_cast<cudaStream_t>(stream));
+  return window_logprob_impl(head, hidden, targets, T, out_logprob, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+int mtpc_window_prefix_logprob(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t T,
+                               float* out_prefix_logprob, void* stream) {
+  int rc = check_call(head, T);
+  if (rc != MTPC_OK) return rc;
+  if (T == 0) return MTPC_OK;
+  if (!hidden || !targets || !out_prefix_logprob) return MTPC_ERR_NULL;
+  return window_logprob_impl(head, hidden, targets, T, nullptr, out_prefix_logprob, static_cast<cudaStream_t>(stream));
 }
 
 int mtpc_draft_sample(mtpc_head* head, const void* hidden, int32_t P, int32_t wpp, const float* uniforms,
@@ -541,7 +591,66 @@ int mtpc_draft_sample(mtpc_head* head, const void* hidden, int32_t P, int32_t wp
   if (wpp < 1 || wpp > head->cfg.max_windows_per_pos) return MTPC_ERR_SHAPE;
   if (P == 0) return MTPC_OK;
   if (!hidden || !uniforms || !out_bytes || !out_logprob) return MTPC_ERR_NULL;
-  return draft_sample_impl(head, hidden, P, wpp, uniforms, out_bytes, out_logprob, static_cast<cudaStream_t>(stream));
+  return draft_sample_impl(head, hidden, P, wpp, uniforms, out_bytes, out_logprob, nullptr,
+                           static_cast<cudaStream_t>(stream));
+}
+
+int mtpc_draft_sample_prefix(mtpc_head* head, const void* hidden, int32_t P, int32_t wpp, const float* uniforms,
+                             int32_t* out_bytes, float* out_prefix_logprob, void* stream) {
+  int rc = check_call(head, P);
+  if (rc != MTPC_OK) return rc;
+  if (wpp < 1 || wpp > head->cfg.max_windows_per_pos) return MTPC_ERR_SHAPE;
+  if (P == 0) return MTPC_OK;
+  if (!hidden || !uniforms || !out_bytes || !out_prefix_logprob) return MTPC_ERR_NULL;
+  return draft_sample_impl(head, hidden, P, wpp, uniforms, out_bytes, nullptr, out_prefix_logprob,
+                           static_cast<cudaStream_t>(stream));
+}
+
+int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32_t* draft_bytes,
+                            const float* prefix_logprob, const float* target_probs, const float* accept_uniforms,
+                            int32_t* out_accepted, int32_t* out_next_byte, void* stream) {
+  int rc = check_call(head, P);
+  if (rc != MTPC_OK) return rc;
+  if (wpp < 1 || wpp > head->cfg.max_windows_per_pos) return MTPC_ERR_SHAPE;
+  if (P == 0) return MTPC_OK;
+  if (!draft_bytes || !prefix_logprob || !target_probs || !accept_uniforms || !out_accepted || !out_next_byte)
+    return MTPC_ERR_NULL;
+  if (P > head->L.decode_max_p) return MTPC_ERR_UNSUPPORTED;
+  if (head->draft_P != P) return MTPC_ERR_STATE;
+  const mtpc_config& c = head->cfg;
+  const Layout& L = head->L;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int W = P * wpp;
+  const size_t smem = kAcceptWarps * accept_warp_floats(c.family, c.n, c.r, c.v) * sizeof(float);
+  PhaseTimer pt(head, st);
+  pt.begin();
+  spec_accept_kernel<<<(W + kAcceptWarps - 1) / kAcceptWarps, kAcceptWarps * 32, smem, st>>>(
+      c.family, at<float>(head, L.off_logits), at<float>(head, L.off_unit_lse), at<float>(head, L.off_logw),
+      at<float>(head, L.off_logA), draft_bytes, prefix_logprob, target_probs, accept_uniforms, out_accepted,
+      out_next_byte, at<unsigned>(head, L.off_status), W, wpp, c.n, c.r, c.v, L.sum_rows);
+  head->launches++;
+  pt.end();
+  return check_launch();
+}
+
+int mtpc_window_loss(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,
+                     int32_t sequence_length, float gamma, float* out_slot_loss, float* out_loss, void* stream) {
+  if (!head) return MTPC_ERR_NULL;
+  if (num_sequences < 1 || sequence_length < 1) return MTPC_ERR_SHAPE;
+  const int64_t T64 = static_cast<int64_t>(num_sequences) * sequence_length;
+  if (T64 > head->cfg.max_positions) return MTPC_ERR_SHAPE;
+  if (!hidden || !targets || !out_slot_loss || !out_loss) return MTPC_ERR_NULL;
+  const int T = static_cast<int>(T64);
+  const Layout& L = head->L;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* prefix = at<float>(head, L.off_prefix);
+  float* partial = at<float>(head, L.off_partial);
+  int rc = window_logprob_impl(head, hidden, targets, T, nullptr, prefix, st);   // phases 0 and 1
+  if (rc != MTPC_OK) return rc;
+  loss_partial_kernel<<<num_sequences, kLossThreads, 0, st>>>(prefix, targets, partial, sequence_length, head->cfg.n);
+  loss_final_kernel<<<1, kLossThreads, 0, st>>>(partial, out_slot_loss, out_loss, num_sequences, head->cfg.n, gamma);
+  head->launches += 2;
+  return check_launch();
 }
 
 int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int32_t* targets_host, int32_t T,
@@ -561,7 +670,7 @@ int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int
   fail |= cudaMemcpyAsync(dt, targets_host, static_cast<size_t>(T) * head->cfg.n * 4, cudaMemcpyHostToDevice, st) !=
           cudaSuccess;
   if (fail) return MTPC_ERR_CUDA;
-  rc = window_logprob_impl(head, dh, dt, T, dout, st);
+  rc = window_logprob_impl(head, dh, dt, T, dout, nullptr, st);
   if (rc != MTPC_OK) return rc;
   fail = cudaMemcpyAsync(out_logprob_host, dout, static_cast<size_t>(T) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess;
   fail |= cudaStreamSynchronize(st) != cudaSuccess;
@@ -589,7 +698,7 @@ int mtpc_draft_sample_host(mtpc_head* head, const void* hidden_host, int32_t P, 
               cudaSuccess;
   fail |= cudaMemcpyAsync(du, uniforms_host, W * 2 * c.n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess;
   if (fail) return MTPC_ERR_CUDA;
-  rc = draft_sample_impl(head, dh, P, wpp, du, db, dout, st);
+  rc = draft_sample_impl(head, dh, P, wpp, du, db, dout, nullptr, st);
   if (rc != MTPC_OK) return rc;
   fail = cudaMemcpyAsync(out_bytes_host, db, W * c.n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess;
   fail |= cudaMemcpyAsync(out_logprob_host, dout, W * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess;
@@ -675,6 +784,8 @@ const char* mtpc_status_string(int code) {
     case MTPC_ERR_WORKSPACE: return "workspace too small or misaligned";
     case MTPC_ERR_CUDA: return "a CUDA call failed (no sm_100 device, launch error, or driver entry point missing)";
     case MTPC_ERR_TIMEOUT: return "a device-side bounded wait expired";
+    case MTPC_ERR_STATE:
+      return "the head holds no draft state for this call (mtpc_speculative_accept must follow a draft of the same positions)";
     case MTPC_ERR_STATIC_SCRATCH:
       return "the call needs more scratch than the library's built-in static array holds (mtpc_window_logprob_static)";
     default: return "unknown status code";
@@ -731,7 +842,8 @@ extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_
   L.off_logA = take(c.family == MTPC_HMM ? static_cast<size_t>(c.n - 1) * c.r * c.r * 4 : 0);
   L.off_G = take(static_cast<size_t>(c.max_positions) * c.n * c.r * 4);
   L.off_logw = take(static_cast<size_t>(c.max_positions) * L.sum_rows * 4);
-  L.off_sel = L.off_wemit = L.off_wsum = L.off_hidden = L.off_logits = 0;                // unused by this call
+  L.off_sel = L.off_wemit = L.off_wsum = L.off_hidden = L.off_logits = L.off_unit_lse = 0;   // unused by this call
+  L.off_prefix = L.off_partial = 0;
   L.off_h_hidden = L.off_h_targets = L.off_h_uniforms = L.off_h_bytes = L.off_h_out = 0;
   L.total = off;
   if (L.total > static_cast<size_t>(MTPC_STATIC_SCRATCH_BYTES)) return MTPC_ERR_STATIC_SCRATCH;
@@ -757,15 +869,7 @@ extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_
   bool fail = cudaDeviceGetAttribute(&h.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
-  if (c.family == MTPC_HMM)
-    fail |= cudaFuncSetAttribute(circuit_hmm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kHmmTableSmemLimit)) != cudaSuccess;
-  if (c.family == MTPC_BTREE) {
-    const int smem = kCircuitWarps * ((c.n - 1) * c.r + c.r * (c.r + 1)) * 4;
-    if (smem > 48 * 1024)
-      fail |= cudaFuncSetAttribute(circuit_btree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-              cudaSuccess;
-  }
+  fail |= !set_circuit_attributes(c);
   // The array keeps whatever the previous call left in it. Only the status word has to start at zero; G, log omega
   // and logA are fully rewritten for the rows this call reads.
   fail |= cudaMemsetAsync(scratch + L.off_status, 0, 256, st) != cudaSuccess;
@@ -778,7 +882,7 @@ extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_
   rc = make_tmap(&h.tm_emit_lp, W_emit, static_cast<uint64_t>(c.n) * c.r * c.v, c.d, L.lp.tile_cols);
   if (rc == MTPC_OK) rc = make_tmap(&h.tm_sum, W_sum, L.sum_rows, c.d, L.sum_cols);
   if (rc != MTPC_OK) return rc;
-  rc = window_logprob_impl(&h, hidden, targets, T, out_logprob, st);
+  rc = window_logprob_impl(&h, hidden, targets, T, out_logprob, nullptr, st);
   if (rc != MTPC_OK) return rc;
   if (out_status &&
       cudaMemcpyAsync(out_status, scratch + L.off_status, 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)

@@ -31,13 +31,44 @@ __device__ __forceinline__ float warp_lse(float val, bool has) {
 }
 
 // Eq. (CP): out[w] = LSE_k( log omega[p, k] + sum_i G[w, i, k] ),  p = w / wpp.
+// With `prefix` (may be NULL) the kernel also writes prefix[w, i] = log q(x_0..x_i), the joint with the later bytes
+// summed out (Algorithm 3's marginals): for a mixture that is the same log-sum-exp over the first i+1 slots only.
 __global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __restrict__ logw,
-                                  float* __restrict__ out, int W, int wpp, int n, int r, int sum_rows) {
+                                  float* __restrict__ out, float* __restrict__ prefix, int W, int wpp, int n, int r,
+                                  int sum_rows) {
   const int w = blockIdx.x * kCircuitWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (w >= W) return;
   const float* g = G + static_cast<size_t>(w) * n * r;
   const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
+  if (prefix != nullptr) {
+    // running sums of up to 4 units per lane (r <= 128); one warp log-sum-exp per slot
+    float a[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) a[q] = (lane + 32 * q < r) ? lw[lane + 32 * q] : 0.f;
+    float last = 0.f;
+    for (int i = 0; i < n; ++i) {
+      float m = -CUDART_INF_F, s = 0.f;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int k = lane + 32 * q;
+        if (k < r) {
+          a[q] += g[i * r + k];
+          if (a[q] != a[q]) { m = 0.f; s = a[q]; } else lse_merge(m, s, a[q], 1.f);
+        }
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        const float m2 = __shfl_xor_sync(kFull, m, off);
+        const float s2 = __shfl_xor_sync(kFull, s, off);
+        lse_merge(m, s, m2, s2);
+      }
+      last = m + __logf(s);
+      if (lane == 0) prefix[static_cast<size_t>(w) * n + i] = last;
+    }
+    if (lane == 0 && out != nullptr) out[w] = last;
+    return;
+  }
   float m = -CUDART_INF_F, s = 0.f;
   for (int k = lane; k < r; k += 32) {
     float a = lw[k];
@@ -59,10 +90,12 @@ __global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __re
 // The inner log-sum-exp is taken as one scaled matrix-vector product per step: with m = max_a alpha_{i-1}[a],
 // alpha_i[k] = G[i,k] + m + log sum_a exp(alpha_{i-1}[a] - m) A[i-1][a][k], A = exp(logA) staged once per CTA in
 // shared memory ((n-1) r^2 floats; read straight from global memory when that does not fit). One warp per
-// window, lane = state; CTAs stride over the windows.
+// window, lane = state; CTAs stride over the windows. With `prefix` (may be NULL) the kernel also writes
+// prefix[w, i] = log q(x_0..x_i) = LSE_k alpha_i[k].
 __global__ void circuit_hmm_kernel(const float* __restrict__ G, const float* __restrict__ logw,
-                                   const float* __restrict__ logA, float* __restrict__ out, int W, int wpp, int n,
-                                   int r, int sum_rows, int tables_in_smem) {
+                                   const float* __restrict__ logA, float* __restrict__ out,
+                                   float* __restrict__ prefix, int W, int wpp, int n, int r, int sum_rows,
+                                   int tables_in_smem) {
   extern __shared__ float A_lin[];
   const int lane = threadIdx.x & 31;
   const int count = (n - 1) * r * r;
@@ -76,6 +109,10 @@ __global__ void circuit_hmm_kernel(const float* __restrict__ G, const float* __r
     const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
     float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
     for (int i = 1; i < n; ++i) {
+      if (prefix != nullptr) {   // log q(x_0..x_{i-1}) = LSE_k alpha_{i-1}[k]: the later steps sum to one
+        const float pre = warp_lse(alpha, has);
+        if (lane == 0) prefix[static_cast<size_t>(w) * n + i - 1] = pre;
+      }
       const float gi = has ? g[i * r + lane] : 0.f;
       float m = alpha;                                   // fmaxf drops NaNs; they come back through e below
 #pragma unroll
@@ -92,22 +129,58 @@ __global__ void circuit_hmm_kernel(const float* __restrict__ G, const float* __r
       if (has) alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : gi + m + __logf(s);
     }
     const float res = warp_lse(alpha, has);
-    if (lane == 0) out[w] = res;
+    if (lane == 0) {
+      if (out != nullptr) out[w] = res;
+      if (prefix != nullptr) prefix[static_cast<size_t>(w) * n + n - 1] = res;
+    }
   }
 }
 
 // Eq. (BTree), bottom-up over the heap-ordered latent tree. Node j >= 1 has the table
 // logOmega_j[a][b] = logw[p, r + (j-1) r^2 + a r + b] (parent's value a, own value b); the deepest internal node
 // n/2-1+m multiplies the input units of tokens 2m and 2m+1. prod[j][z] is the product unit under z_j = z.
-// Shared memory per warp: (n-1) * r floats of prod + r * (r+1) floats of one staged table.  r <= 32.
+
+// One sum layer seen from the parent: returns, for lane = parent value z, LSE_b(logOmega_c[z][b] + pc[b]).
+// tab: the child's r x r table in global memory; pc: r floats in shared memory (written before the call; the
+// function synchronises the warp); table: r * (r+1) floats of per-warp shared scratch.
+__device__ __forceinline__ float btree_sum_layer(const float* __restrict__ tab, const float* pc, float* table,
+                                                 int lane, int r) {
+  const bool has = lane < r;
+  for (int a = 0; a < r; ++a)                      // coalesced rows -> padded shared tile
+    if (has) table[a * (r + 1) + lane] = tab[a * r + lane];
+  __syncwarp();
+  float res = 0.f;
+  if (has) {
+    const float* row = table + lane * (r + 1);     // row z = lane, over the child's values b
+    float m = -CUDART_INF_F;
+    for (int b = 0; b < r; ++b) m = fmaxf(m, row[b] + pc[b]);
+    float s = 0.f;
+    for (int b = 0; b < r; ++b) s += __expf(row[b] + pc[b] - m);
+    res = (m == -CUDART_INF_F) ? -CUDART_INF_F : m + __logf(s);
+    if (s != s) res = s;                           // NaN evidence must survive the max
+  }
+  __syncwarp();
+  return res;
+}
+
+// Shared memory per warp: (n-1) * r floats of prod + r * (r+1) floats of one staged table; with PREFIX another
+// (n-1) * r floats (the sum-layer outputs S[c][z], kept for the prefix passes) + r floats.  r <= 32.
+// PREFIX: also writes prefix[w, i] = log q(x_0..x_i). Summing the later bytes out sets their input units to one,
+// so every subtree right of token i evaluates to one, every subtree left of it keeps its value, and only the
+// nodes on the path from token i's owner to the root have to be re-evaluated.
+template <bool PREFIX>
 __global__ void circuit_btree_kernel(const float* __restrict__ G, const float* __restrict__ logw,
-                                     float* __restrict__ out, int W, int wpp, int n, int r, int sum_rows) {
+                                     float* __restrict__ out, float* __restrict__ prefix, int W, int wpp, int n, int r,
+                                     int sum_rows) {
   extern __shared__ float sm[];
   const int wib = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int w = blockIdx.x * kCircuitWarps + wib;
-  float* prod = sm + static_cast<size_t>(wib) * ((n - 1) * r + r * (r + 1));
+  const int per_warp = (n - 1) * r + r * (r + 1) + (PREFIX ? (n - 1) * r + r : 0);
+  float* prod = sm + static_cast<size_t>(wib) * per_warp;
   float* table = prod + (n - 1) * r;
+  float* S = table + r * (r + 1);                  // PREFIX only
+  float* cur = S + (n - 1) * r;                    // PREFIX only
   if (w >= W) return;
   const float* g = G + static_cast<size_t>(w) * n * r;
   const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
@@ -122,27 +195,39 @@ __global__ void circuit_btree_kernel(const float* __restrict__ G, const float* _
     float acc = 0.f;
     for (int side = 0; side < 2; ++side) {
       const int c = 2 * j + 1 + side;
-      const float* tab = lw + r + static_cast<size_t>(c - 1) * r * r;
-      for (int a = 0; a < r; ++a)                      // coalesced rows -> padded shared tile
-        if (has) table[a * (r + 1) + lane] = tab[a * r + lane];
-      __syncwarp();
-      if (has) {
-        const float* row = table + lane * (r + 1);     // row z_j = lane, over the child's values b
-        const float* pc = prod + c * r;
-        float m = -CUDART_INF_F;
-        for (int b = 0; b < r; ++b) m = fmaxf(m, row[b] + pc[b]);
-        float s = 0.f;
-        for (int b = 0; b < r; ++b) s += __expf(row[b] + pc[b] - m);
-        acc += (m == -CUDART_INF_F) ? -CUDART_INF_F : m + __logf(s);
-        if (s != s) acc = s;
-      }
-      __syncwarp();
+      const float sc = btree_sum_layer(lw + r + static_cast<size_t>(c - 1) * r * r, prod + c * r, table, lane, r);
+      if (PREFIX && has) S[c * r + lane] = sc;
+      acc += sc;
     }
     if (has) prod[j * r + lane] = acc;
     __syncwarp();
   }
   const float res = warp_lse(has ? lw[lane] + prod[lane] : 0.f, has);
-  if (lane == 0) out[w] = res;
+  if (lane == 0 && out != nullptr) out[w] = res;
+  if (PREFIX) {
+    if (lane == 0) prefix[static_cast<size_t>(w) * n + n - 1] = res;
+    for (int i = 0; i < n - 1; ++i) {
+      int c = first_leaf_node + (i >> 1);
+      bool full = (i & 1) != 0;                    // both tokens of the owner are inside the prefix
+      float val = has ? (full ? prod[c * r + lane] : g[i * r + lane]) : 0.f;
+      while (c > 0) {
+        const bool is_right = (c & 1) == 0;
+        float sc;
+        if (full) {
+          sc = has ? S[c * r + lane] : 0.f;
+        } else {
+          if (has) cur[lane] = val;
+          __syncwarp();
+          sc = btree_sum_layer(lw + r + static_cast<size_t>(c - 1) * r * r, cur, table, lane, r);
+        }
+        val = sc + ((is_right && has) ? S[(c - 1) * r + lane] : 0.f);   // left sibling: inside; right sibling: one
+        full = full && is_right;
+        c = (c - 1) >> 1;
+      }
+      const float pre = warp_lse(has ? lw[lane] + val : 0.f, has);
+      if (lane == 0) prefix[static_cast<size_t>(w) * n + i] = pre;
+    }
+  }
 }
 
 // ---------------------------------------------------------------- latent draws (Algorithm 1, sum units)
@@ -193,6 +278,69 @@ __global__ void latent_sample_kernel(int family, const float* __restrict__ logw,
     for (int j = 1; j < n - 1; ++j)
       zs[j] = inv_cdf_logp(lw + r + (static_cast<size_t>(j - 1) * r + zs[(j - 1) >> 1]) * r, r, u[j]);
     for (int i = 0; i < n; ++i) sel[i] = zs[n / 2 - 1 + (i >> 1)];
+  }
+}
+
+// ---------------------------------------------------------------- training loss (Eq. 6)
+// Eq. (6): L_j = -(1/N) sum_i (1/V_ij) sum_t log p(x_{t+j} | x_{<t+j}), L = sum_j gamma^(j-1) L_j, over N sequences of
+// L positions with overlapping windows. The conditional of slot j given the context and the window's earlier bytes
+// is the difference of consecutive prefix log-marginals; V_ij counts the valid (non-negative) targets of slot j in
+// sequence i. Two kernels, both with a fixed reduction order, so the result does not change from run to run.
+constexpr int kLossThreads = 256;
+
+// grid = N. partial[i, j] = (1/V_ij) sum_{t valid} (prefix[t, j] - prefix[t, j-1]), 0 if V_ij = 0.
+__global__ void __launch_bounds__(kLossThreads) loss_partial_kernel(const float* __restrict__ prefix,
+                                                                    const int* __restrict__ targets,
+                                                                    float* __restrict__ partial, int L, int n) {
+  __shared__ float ssum[kLossThreads / 32];
+  __shared__ int scnt[kLossThreads / 32];
+  const int i = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int j = 0; j < n; ++j) {
+    float sum = 0.f;
+    int cnt = 0;
+    for (int t = threadIdx.x; t < L; t += kLossThreads) {
+      const size_t row = (static_cast<size_t>(i) * L + t) * n;
+      if (targets[row + j] >= 0) {
+        sum += prefix[row + j] - (j > 0 ? prefix[row + j - 1] : 0.f);
+        cnt += 1;
+      }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      sum += __shfl_xor_sync(kFull, sum, off);
+      cnt += __shfl_xor_sync(kFull, cnt, off);
+    }
+    if (lane == 0) { ssum[warp] = sum; scnt[warp] = cnt; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float tot = 0.f;
+      int c = 0;
+      for (int q = 0; q < kLossThreads / 32; ++q) { tot += ssum[q]; c += scnt[q]; }
+      partial[static_cast<size_t>(i) * n + j] = c > 0 ? tot / static_cast<float>(c) : 0.f;
+    }
+    __syncthreads();
+  }
+}
+
+// One CTA; warp q reduces the slots q, q + warps, ...: slot_loss[j] = -(1/N) sum_i partial[i, j]; then
+// loss = sum_j gamma^j slot_loss[j] (j counted from 0).
+__global__ void __launch_bounds__(kLossThreads) loss_final_kernel(const float* __restrict__ partial,
+                                                                  float* __restrict__ slot_loss,
+                                                                  float* __restrict__ loss, int N, int n, float gamma) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int j = warp; j < n; j += kLossThreads / 32) {
+    float sum = 0.f;
+    for (int i = lane; i < N; i += 32) sum += partial[static_cast<size_t>(i) * n + j];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(kFull, sum, off);
+    if (lane == 0) slot_loss[j] = -sum / static_cast<float>(N);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f, wgt = 1.f;
+    for (int j = 0; j < n; ++j) { tot += wgt * slot_loss[j]; wgt *= gamma; }
+    *loss = tot;
   }
 }
 

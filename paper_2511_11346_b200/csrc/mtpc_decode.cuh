@@ -293,11 +293,12 @@ __device__ __forceinline__ int warp_sample_unit(int family, const float* __restr
   return z;
 }
 
-// grid = (n, P). Shared memory: 2 * r floats (max and log-sum-exp of each unit of the slot).
+// grid = (n, P). Shared memory: 2 * r floats (max and log-sum-exp of each unit of the slot). The log-sum-exps also
+// go to unit_lse_out [P, n, r], so that later calls can turn the retained logits into log phi.
 __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     int family, const float* __restrict__ logits, const float* __restrict__ logw, const float* __restrict__ logA,
-    const float* __restrict__ uniforms, int* __restrict__ out_bytes, float* __restrict__ G, unsigned* status, int wpp,
-    int n, int r, int v, int sum_rows) {
+    const float* __restrict__ uniforms, int* __restrict__ out_bytes, float* __restrict__ G,
+    float* __restrict__ unit_lse_out, unsigned* status, int wpp, int n, int r, int v, int sum_rows) {
   extern __shared__ float sm[];
   float* unit_max = sm;
   float* unit_lse = sm + r;
@@ -317,7 +318,11 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     for (int b = lane; b < v; b += 32) s += __expf(x[b] - m);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(kFull, s, off);
-    if (lane == 0) { unit_max[k] = m; unit_lse[k] = m + __logf(s); }
+    if (lane == 0) {
+      unit_max[k] = m;
+      unit_lse[k] = m + __logf(s);
+      unit_lse_out[(static_cast<size_t>(pos) * n + i) * r + k] = unit_lse[k];   // kept for the acceptance stage
+    }
   }
   __syncthreads();
 
@@ -364,6 +369,186 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     // evidence of the drafted byte under every input unit of the slot (a missing byte is marginalised)
     if (lane < r) G[(w * n + i) * r + lane] = byte < 0 ? 0.f : row[static_cast<size_t>(lane) * v + byte] - unit_lse[lane];
   }
+}
+
+// ---------------------------------------------------------------- acceptance stage (Algorithm 3)
+constexpr int kAcceptWarps = 4;
+
+// Per-warp shared memory of spec_accept_kernel, in floats: the residual weights of the v bytes, and for the binary
+// tree the product and sum-layer vectors of every node, one staged table and one vector.
+__host__ __device__ inline size_t accept_warp_floats(int family, int n, int r, int v) {
+  return static_cast<size_t>(v) + (family == 2 ? 2 * static_cast<size_t>(n - 1) * r + static_cast<size_t>(r) * (r + 1) + r : 0);
+}
+
+// One warp per drafted window w (position p = w / wpp). Inputs: the draft's bytes and prefix log-marginals, the
+// target model's conditionals along the draft, one uniform per test plus one for the last byte; the logits and
+// per-unit log-sum-exps the draft call left in the workspace.
+//   1. s = 0; while s < n: the draft's conditional of byte s is q_s = exp(prefix[s] - prefix[s-1]) (prefix[-1] = 0);
+//      stop if alpha_s > p(x_s) / q_s, tested as alpha_s * q_s > p(x_s); else s += 1.
+//   2. s == n: the extra byte is drawn from the target row n.
+//      s <  n: it is drawn from max(0, p(.) - q(. | x_0..x_{s-1})) / Z. The circuit's conditional of slot s is a
+//      mixture of the slot's r input units, q(b | ..) = sum_k c_k phi_{s,k}(b), with c the posterior of the latent that
+//      owns slot s given the accepted bytes: CP: omega_k prod_{i<s} phi_{i,k}(x_i); HMM: the one-step prediction
+//      from alpha_{s-1}; BTree: the upward pass with the bytes >= s summed out, then the downward pass along the
+//      path from the root to the node that owns token s.
+//   Both draws are inverse-CDF on unnormalised weights (u * total < running sum, index order, no division).
+__global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
+    int family, const float* __restrict__ logits, const float* __restrict__ unit_lse, const float* __restrict__ logw,
+    const float* __restrict__ logA, const int* __restrict__ bytes, const float* __restrict__ prefix,
+    const float* __restrict__ target, const float* __restrict__ uniforms, int* __restrict__ out_accepted,
+    int* __restrict__ out_next, unsigned* status, int W, int wpp, int n, int r, int v, int sum_rows) {
+  extern __shared__ float sm[];
+  const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int w = blockIdx.x * kAcceptWarps + wib;
+  if (w >= W) return;
+  float* mres = sm + static_cast<size_t>(wib) * accept_warp_floats(family, n, r, v);
+  const int pos = w / wpp;
+  const int* x = bytes + static_cast<size_t>(w) * n;
+  const float* pre = prefix + static_cast<size_t>(w) * n;
+  const float* u = uniforms + static_cast<size_t>(w) * (n + 1);
+  const float* tp = target + static_cast<size_t>(w) * (n + 1) * v;
+  const float* lw = logw + static_cast<size_t>(pos) * sum_rows;
+  const bool has = lane < r;
+
+  // ---- 1. acceptance tests (every lane takes the same decisions on the same values)
+  bool bad_u = false, bad_x = false;
+  for (int c = lane; c <= n; c += 32) bad_u |= !(u[c] >= 0.f && u[c] < 1.f);
+  for (int c = lane; c < n; c += 32) bad_x |= static_cast<unsigned>(x[c]) >= static_cast<unsigned>(v);
+  bad_u = __any_sync(kFull, bad_u);
+  bad_x = __any_sync(kFull, bad_x);
+  if (bad_u || bad_x) {
+    if (lane == 0) {
+      atomicOr(status, bad_u ? 2u : 1u);
+      out_accepted[w] = -1;
+      out_next[w] = -1;
+    }
+    return;
+  }
+  int s = 0;
+  while (s < n) {
+    const float q = __expf(pre[s] - (s > 0 ? pre[s - 1] : 0.f));
+    if (u[s] * q > tp[static_cast<size_t>(s) * v + x[s]]) break;
+    ++s;
+  }
+  if (lane == 0) out_accepted[w] = s;
+  const float* trow = tp + static_cast<size_t>(s) * v;
+
+  if (s == n) {
+    for (int b = lane; b < v; b += 32) mres[b] = trow[b];
+  } else {
+    // ---- 2. c[k]: log-weight of input unit k of slot s given the accepted bytes (lane = k)
+    auto g_of = [&](int i) -> float {   // log phi_{i,lane}(x_i)
+      const size_t unit = (static_cast<size_t>(pos) * n + i) * r + lane;
+      return logits[unit * v + x[i]] - unit_lse[unit];
+    };
+    float c = 0.f;
+    if (family == 0) {
+      c = has ? lw[lane] : 0.f;
+      for (int i = 0; i < s; ++i) c += has ? g_of(i) : 0.f;
+    } else if (family == 1) {
+      float alpha = has ? lw[lane] : -CUDART_INF_F;
+      for (int i = 0; i < s; ++i) {
+        // alpha_i = g_i + (i == 0 ? log pi : LSE_a(alpha_{i-1}[a] + logA[i-1][a][.])); then one more prediction step
+        if (has) alpha += g_of(i);
+        float m = alpha;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
+        const float e = has ? __expf(alpha - m) : 0.f;
+        const float* A = logA + static_cast<size_t>(i) * r * r;
+        float acc = 0.f;
+        for (int a = 0; a < r; ++a) acc = fmaf(__shfl_sync(kFull, e, a), has ? __expf(__ldg(A + a * r + lane)) : 0.f, acc);
+        alpha = has ? m + __logf(acc) : -CUDART_INF_F;
+      }
+      c = alpha;
+    } else {
+      float* prod = mres + v;
+      float* S = prod + (n - 1) * r;
+      float* table = S + (n - 1) * r;
+      float* cur = table + r * (r + 1);
+      const int first_leaf_node = n / 2 - 1;
+      for (int j = n - 2; j >= first_leaf_node; --j) {
+        const int t0 = 2 * (j - first_leaf_node);
+        if (has) prod[j * r + lane] = (t0 < s ? g_of(t0) : 0.f) + (t0 + 1 < s ? g_of(t0 + 1) : 0.f);
+      }
+      __syncwarp();
+      for (int j = first_leaf_node - 1; j >= 0; --j) {
+        float acc = 0.f;
+        for (int side = 0; side < 2; ++side) {
+          const int ch = 2 * j + 1 + side;
+          const float sc = btree_sum_layer(lw + r + static_cast<size_t>(ch - 1) * r * r, prod + ch * r, table, lane, r);
+          if (has) S[ch * r + lane] = sc;
+          acc += sc;
+        }
+        if (has) prod[j * r + lane] = acc;
+        __syncwarp();
+      }
+      // downward: up[z] = log-weight of the rest of the circuit seen from the current path node with latent z
+      const int owner = first_leaf_node + (s >> 1);
+      const int code = owner + 1;
+      const int depth = 31 - __clz(code);
+      int node = 0;
+      float up = has ? lw[lane] : -CUDART_INF_F;
+      for (int lvl = depth - 1; lvl >= 0; --lvl) {
+        const int child = 2 * node + 1 + ((code >> lvl) & 1);
+        const int sib = (child & 1) ? child + 1 : child - 1;
+        if (has) cur[lane] = up + S[sib * r + lane];
+        __syncwarp();
+        const float* tab = lw + r + static_cast<size_t>(child - 1) * r * r;   // [parent value z][own value b]
+        float m = -CUDART_INF_F;
+        for (int z = 0; z < r; ++z) m = fmaxf(m, has ? cur[z] + tab[z * r + lane] : -CUDART_INF_F);
+        float acc = 0.f;
+        for (int z = 0; z < r; ++z) acc += has ? __expf(cur[z] + tab[z * r + lane] - m) : 0.f;
+        up = has ? m + __logf(acc) : -CUDART_INF_F;
+        __syncwarp();
+        node = child;
+      }
+      const int other_leaf = s ^ 1;
+      c = up + ((has && other_leaf < s) ? g_of(other_leaf) : 0.f);
+    }
+    const float c_lse = warp_lse(c, has);             // every lane takes part in the shuffles
+    const float cprob = has ? __expf(c - c_lse) : 0.f;
+    const float ulse = has ? unit_lse[(static_cast<size_t>(pos) * n + s) * r + lane] : 0.f;
+    const float* lrow = logits + (static_cast<size_t>(pos) * n + s) * r * v;   // [r, v] logits of slot s
+    for (int b0 = 0; b0 < v; b0 += 32) {
+      const int b = b0 + lane;
+      float q = 0.f;
+      for (int k = 0; k < r; ++k) {
+        const float ck = __shfl_sync(kFull, cprob, k);
+        const float lk = __shfl_sync(kFull, ulse, k);
+        if (b < v) q = fmaf(ck, __expf(lrow[static_cast<size_t>(k) * v + b] - lk), q);
+      }
+      if (b < v) mres[b] = fmaxf(0.f, trow[b] - q);
+    }
+  }
+  __syncwarp();
+
+  // ---- 3. inverse CDF over the weights in mres: lane l owns bytes [l*per, (l+1)*per)
+  const int per = (v + 31) / 32;
+  const int b0 = lane * per;
+  float part = 0.f;
+  for (int q = 0; q < per; ++q)
+    if (b0 + q < v) part += mres[b0 + q];
+  const float incl = warp_scan_incl(part, lane);
+  const float total = __shfl_sync(kFull, incl, 31);
+  const float thr = u[n] * total;
+  const unsigned hit = __ballot_sync(kFull, thr < incl);
+  int byte = v - 1;   // rounding may leave no index: the last one
+  if (hit) {
+    const int src = __ffs(hit) - 1;
+    int found = -1;
+    const float before = __shfl_up_sync(kFull, incl, 1);
+    if (lane == src) {
+      float cum = lane == 0 ? 0.f : before;
+      for (int q = 0; q < per && found < 0; ++q)
+        if (b0 + q < v) {
+          cum += mres[b0 + q];
+          if (thr < cum) found = b0 + q;
+        }
+      if (found < 0) found = min(b0 + per, v) - 1;
+    }
+    byte = __shfl_sync(kFull, found, src);
+  }
+  if (lane == 0) out_next[w] = byte;
 }
 
 }  // namespace mtpc

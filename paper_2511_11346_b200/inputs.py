@@ -11,7 +11,8 @@ weights and data that are not available offline):
   2  HMM                T=8192 d=4096 n=8  r=32 v=320  bf16, static transitions ~N(0,1), Zipf(1.1) targets
   3  BTree              T=4096 d=3072 n=16 r=32 v=256  bf16, uniform targets, + draft wpp=1
   4  decode sweep cells P in {1,8,64}, d=4096, v=320, CP r=16 / HMM r=32, n in {8,16}, wpp=16
-Hidden states ~N(0,1); every weight ~N(0, std=0.02); uniforms in [0,1) as fp32.
+Hidden states ~N(0,1); every weight ~N(0, std=0.02); uniforms in [0,1) as fp32. For the acceptance stage the
+target model's conditionals are Dirichlet rows (target_rows) and its uniforms come from the same generator.
 """
 from __future__ import annotations
 
@@ -125,6 +126,14 @@ def uniforms(seed: int, stream: int, shape) -> np.ndarray:
     """fp32 uniforms in [0,1) on a 2^-24 grid (exactly representable, never 1.0)."""
     k = _gen(seed, stream).integers(0, 1 << 24, size=shape, dtype=np.int64)
     return (k.astype(np.float64) / float(1 << 24)).astype(np.float32)
+
+
+def target_rows(seed: int, stream: int, shape, concentration: float = 0.3) -> np.ndarray:
+    """Stand-in for a verifier LLM's next-byte distributions: fp32 rows on the simplex (last axis), drawn
+    Dirichlet(concentration): peaked like byte-level LM predictions and unrelated to the draft head, so some
+    drafted bytes get accepted and some rejected. No arithmetic of the method: gamma draws, normalised."""
+    g = _gen(seed, stream).gamma(concentration, size=shape) + 1e-6
+    return (g / g.sum(axis=-1, keepdims=True)).astype(np.float32)
 
 
 @dataclasses.dataclass

@@ -74,5 +74,42 @@ class DeviceHead:
         self.head.mtpc_draft_sample(h, wpp, u, out_bytes, out_lp)
         return out_bytes, out_lp
 
+    def window_prefix_logprob(self, hidden=None, targets=None):
+        import torch
+        h = self.hidden_device() if hidden is None else hidden
+        t = torch.from_numpy(self.wl.targets).to(self.device) if targets is None else targets
+        out = torch.empty((h.shape[0], self.wl.shape.n), dtype=torch.float32, device=self.device)
+        self.head.mtpc_window_prefix_logprob(h, t, out)
+        return out
+
+    def draft_sample_prefix(self, wpp=None, hidden=None, uniforms=None):
+        import torch
+        wpp = wpp or self.wl.wpp
+        h = self.hidden_device() if hidden is None else hidden
+        u = torch.from_numpy(self.wl.uniforms).to(self.device) if uniforms is None else uniforms
+        W = h.shape[0] * wpp
+        out_bytes = torch.empty((W, self.wl.shape.n), dtype=torch.int32, device=self.device)
+        out_prefix = torch.empty((W, self.wl.shape.n), dtype=torch.float32, device=self.device)
+        self.head.mtpc_draft_sample_prefix(h, wpp, u, out_bytes, out_prefix)
+        return out_bytes, out_prefix
+
+    def speculative_accept(self, P, wpp, draft_bytes, prefix_logprob, target_probs, accept_uniforms):
+        import torch
+        W = P * wpp
+        accepted = torch.empty(W, dtype=torch.int32, device=self.device)
+        next_byte = torch.empty(W, dtype=torch.int32, device=self.device)
+        self.head.mtpc_speculative_accept(P, wpp, draft_bytes, prefix_logprob, target_probs, accept_uniforms, accepted,
+                                          next_byte)
+        return accepted, next_byte
+
+    def window_loss(self, num_sequences, sequence_length, gamma, hidden=None, targets=None):
+        import torch
+        h = self.hidden_device() if hidden is None else hidden
+        t = torch.from_numpy(self.wl.targets).to(self.device) if targets is None else targets
+        slot = torch.empty(self.wl.shape.n, dtype=torch.float32, device=self.device)
+        loss = torch.empty(1, dtype=torch.float32, device=self.device)
+        self.head.mtpc_window_loss(h, t, num_sequences, sequence_length, gamma, slot, loss)
+        return slot, loss
+
     def close(self):
         self.head.mtpc_destroy()

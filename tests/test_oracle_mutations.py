@@ -163,6 +163,14 @@ def accept_wrong(orc):
     return float(bad)
 
 
+def loss_gap(orc):
+    ln = math.log
+    prefix = np.array([[ln(1 / 2), ln(1 / 8)], [ln(1 / 8), ln(1 / 8)], [ln(1 / 2), ln(1 / 4)], [0.0, 0.0]])
+    targets = np.array([[3, 1], [0, -1], [2, 2], [-1, -1]])
+    slot, total = orc.composite_loss(prefix, targets, 2, 0.8)
+    return float(np.abs(slot - 1.5 * ln(2)).max() + abs(total - 1.5 * ln(2) * 1.8))
+
+
 MUTANTS = [
     # (what is planted, old text, new text, pin that must notice)
     ("mixture weights dropped from Eq. CP", "logsumexp(logw + g.sum(axis=1), axis=-1)", "logsumexp(g.sum(axis=1), axis=-1)", cp_gap),
@@ -205,6 +213,14 @@ MUTANTS = [
     ("byte after a full acceptance drawn from the wrong target row", "inv_cdf(np.log(np.maximum(p[full, n, :], 1e-300)), u[full, n])",
      "inv_cdf(np.log(np.maximum(p[full, n - 1, :], 1e-300)), u[full, n])", accept_wrong),
     ("acceptance test uses the last uniform", "alpha = u[w, s]", "alpha = u[w, n]", accept_wrong),
+    ("loss normalised by the sequence length instead of the valid count", "acc += cond[rows, j][valid].sum() / V",
+     "acc += cond[rows, j][valid].sum() / L", loss_gap),
+    ("loss counts invalid bytes", "valid = tg[rows, j] >= 0", "valid = tg[rows, j] >= -1", loss_gap),
+    ("loss uses the prefix marginal instead of the conditional", "cond = pre - np.concatenate([np.zeros((T, 1)), pre[:, :-1]], axis=1)",
+     "cond = pre", loss_gap),
+    ("discount starts at gamma instead of one", "sum(gamma ** j * slot[j] for j in range(n))",
+     "sum(gamma ** (j + 1) * slot[j] for j in range(n))", loss_gap),
+    ("loss not averaged over the sequences", "slot[j] = -acc / N", "slot[j] = -acc", loss_gap),
 ]
 
 

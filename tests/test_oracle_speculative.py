@@ -200,3 +200,45 @@ def test_acceptance_uses_one_uniform_per_test_in_order():
     assert out["accepted"].tolist() == [1]
     # residual = max(0, (0.25, 0.75) - (0.5, 0.5)) = (0, 0.25) -> byte 1 whatever the uniform
     assert out["next_byte"].tolist() == [1]
+
+
+# ------------------------------------------------------------------ Eq. (6)
+def test_loss_example_worked_by_hand():
+    """N = 2 sequences of L = 2 positions, n = 2. Conditionals (probabilities) per position and slot:
+         seq 0: t0 (1/2, 1/4)  t1 (1/8, masked)      seq 1: t0 (1/2, 1/2)  t1 (masked, masked)
+    L_1 = -(1/2) [ (ln 1/2 + ln 1/8) / 2 + (ln 1/2) / 1 ] = (1/2)(2 ln 2 + ln 2) = 1.5 ln 2
+    L_2 = -(1/2) [ (ln 1/4) / 1 + (ln 1/2) / 1 ] = 1.5 ln 2;  L = L_1 + gamma L_2."""
+    ln = math.log
+    prefix = np.array([[ln(1 / 2), ln(1 / 8)], [ln(1 / 8), ln(1 / 8)], [ln(1 / 2), ln(1 / 4)], [0.0, 0.0]])
+    targets = np.array([[3, 1], [0, -1], [2, 2], [-1, -1]])
+    slot, total = orc.composite_loss(prefix, targets, 2, 0.8)
+    np.testing.assert_allclose(slot, [1.5 * ln(2), 1.5 * ln(2)], atol=1e-12)
+    assert abs(total - 1.5 * ln(2) * 1.8) < 1e-12
+    # a sequence whose slot has no valid byte adds nothing, but still counts in N
+    targets2 = targets.copy()
+    targets2[2, 1] = -1
+    slot2, _ = orc.composite_loss(prefix, targets2, 2, 0.8)
+    assert abs(slot2[1] - ln(4) / 2) < 1e-12
+
+
+@pytest.mark.parametrize("family", [CP, HMM, BTREE])
+def test_undiscounted_loss_with_all_bytes_valid_is_the_mean_joint_nll(family):
+    rng = np.random.default_rng(700 + family)
+    n, r, v, N, L = 4, 3, 5, 3, 6
+    W, R, Ts = _tiny_head(rng, family, n, r, v)
+    h = rng.normal(size=(N * L, 5))
+    x = rng.integers(0, v, size=(N * L, n))
+    prefix = orc.window_prefix_logprob(family, h, W, R, Ts, x)
+    slot, total = orc.composite_loss(prefix, x, N, 1.0)
+    joint = orc.window_logprob(family, h, W, R, Ts, x)
+    assert abs(total + joint.mean()) < 1e-12            # sum_j L_j = -(1/(N L)) sum_t log q(window)
+    # slot terms are per-slot means of conditionals; discounting weights them by gamma^j
+    _, disc = orc.composite_loss(prefix, x, N, 0.5)
+    assert abs(disc - sum(0.5 ** j * slot[j] for j in range(n))) < 1e-12
+    # masking the tail of a window leaves the earlier slots' terms unchanged
+    xm = x.copy()
+    xm[L - 1, 2:] = -1
+    pm = orc.window_prefix_logprob(family, h, W, R, Ts, xm)
+    slot_m, _ = orc.composite_loss(pm, xm, N, 1.0)
+    np.testing.assert_allclose(slot_m[:2], slot[:2], atol=1e-12)
+    assert abs(slot_m[2] - slot[2]) > 1e-6
