@@ -10,6 +10,7 @@ What follows which passage:
   evidence          Sec. 3.1 (input units) + App. B.1 (a marginalised input unit integrates to 1)
   cp_eval           Eq. (CP)
   hmm_eval          Eq. (HMM), evaluated layer by layer (one sum + one product layer per window step)
+  hmm_ctx_eval      the same with contextual transitions (App. H): tables produced from the hidden state
   btree_eval        Eq. (BTree), recursive halving with a latent per internal node
   draft_sample      App. B.2, Algorithm 1 (ancestral sampling), with inverse-CDF categorical draws
   circuit_counts    App. C, Table 3 (sizes of the circuits and of the linear head)
@@ -25,6 +26,8 @@ Readings taken where the paper is silent or garbled (each is listed in the desig
     Table 3's parameter counts fix the number of sum units at 1 + (n-2) r, each of fan-in r.
   * HMM: T_static[i-1, a, b] is the logit of z_i = b given z_{i-1} = a (softmax over b); only the initial
     distribution is contextual here (the paper's "non-contextual" transition variant).
+  * HMM_CTX (the paper's best configuration, App. H): transition logits = rows of R applied to the hidden state
+    plus a bias [n-1, r, r] (the "bias term" that allows the identity initialisation), softmax over the new state.
   * sampleCategorical is inverse-CDF: the smallest index j with u < p_0 + ... + p_j (last index if none).
   * The draft log-prob is the joint marginal log q(x_1..x_n) (latents summed out), as verification needs.
   * No bias and no temperature in either projection.
@@ -43,7 +46,7 @@ from __future__ import annotations
 
 import numpy as np
 
-CP, HMM, BTREE = 0, 1, 2
+CP, HMM, BTREE, HMM_CTX = 0, 1, 2, 3     # HMM_CTX: HMM whose transitions depend on the hidden state (App. H)
 
 
 # ----------------------------------------------------------------------------------------------------
@@ -64,6 +67,8 @@ def num_sum_units(family: int, n: int, r: int, contextual_transitions: bool = Fa
         return 1
     if family == HMM:
         return 1 + (n - 1) * r if contextual_transitions else 1
+    if family == HMM_CTX:
+        return 1 + (n - 1) * r
     if family == BTREE:
         return 1 + (n - 2) * r
     raise ValueError(family)
@@ -94,11 +99,16 @@ def emission_logphi(h: np.ndarray, W_emit: np.ndarray) -> np.ndarray:
     return log_softmax(logits, axis=-1)
 
 
-def sum_unit_logw(h: np.ndarray, W_sum: np.ndarray, r: int) -> np.ndarray:
-    """log omega[t, s, :] = log softmax(W_sum[s*r:(s+1)*r] @ h[t]);  -> [T, S, r]."""
+def sum_unit_logw(h: np.ndarray, W_sum: np.ndarray, r: int, bias: np.ndarray | None = None) -> np.ndarray:
+    """log omega[t, s, :] = log softmax(W_sum[s*r:(s+1)*r] @ h[t]);  -> [T, S, r].
+    `bias` (contextual HMM, App. H "adding a bias term"): [n-1, r, r] logits added to the sum units after the
+    first one, in row order, before the softmax; bias[i-1, a, :] belongs to the unit of z_i given z_{i-1} = a."""
     h = np.asarray(h, dtype=np.float64)
     R = np.asarray(W_sum, dtype=np.float64)
     logits = (h @ R.T).reshape(h.shape[0], R.shape[0] // r, r)
+    if bias is not None:
+        logits = logits.copy()
+        logits[:, 1:, :] += np.asarray(bias, dtype=np.float64).reshape(1, -1, r)
     return log_softmax(logits, axis=-1)
 
 
@@ -156,6 +166,17 @@ def btree_eval(logw: np.ndarray, g: np.ndarray) -> np.ndarray:
     return logsumexp(logw[:, 0, :] + _btree_product(0, 0, n, logw, g, r), axis=-1)
 
 
+def hmm_ctx_eval(logw: np.ndarray, g: np.ndarray) -> np.ndarray:
+    """Eq. (HMM) with contextual, inhomogeneous transitions (App. H): every position has its own tables.
+    logw [T, 1 + (n-1) r, r]: unit 0 = initial distribution; unit 1 + (i-1) r + a = log q(z_i = . | z_{i-1} = a)."""
+    T, n, r = g.shape
+    alpha = logw[:, 0, :] + g[:, 0, :]
+    for i in range(1, n):
+        logA = logw[:, 1 + (i - 1) * r:1 + i * r, :]                   # [T, a, b]
+        alpha = g[:, i, :] + logsumexp(alpha[:, :, None] + logA, axis=1)
+    return logsumexp(alpha, axis=-1)
+
+
 def static_log_transitions(T_static: np.ndarray) -> np.ndarray:
     return log_softmax(np.asarray(T_static, dtype=np.float64), axis=-1)
 
@@ -167,14 +188,21 @@ def circuit_eval(family: int, logw: np.ndarray, g: np.ndarray, T_static: np.ndar
         return hmm_eval(logw[:, 0, :], static_log_transitions(T_static), g)
     if family == BTREE:
         return btree_eval(logw, g)
+    if family == HMM_CTX:
+        return hmm_ctx_eval(logw, g)
     raise ValueError(family)
+
+
+def head_logw(family: int, h, W_sum, T_static, r: int) -> np.ndarray:
+    """Sum-unit log-weights of a head; for HMM_CTX the fourth argument is the transition bias (or None)."""
+    return sum_unit_logw(h, W_sum, r, bias=T_static if family == HMM_CTX else None)
 
 
 def window_logprob(family: int, h, W_emit, W_sum, T_static, targets) -> np.ndarray:
     """log q(x_{t+1..t+n} | context) in nats for every position: [T]."""
     r = np.asarray(W_emit).shape[1]
     logphi = emission_logphi(h, W_emit)
-    logw = sum_unit_logw(h, W_sum, r)
+    logw = head_logw(family, h, W_sum, T_static, r)
     return circuit_eval(family, logw, evidence(logphi, targets), T_static)
 
 
@@ -216,6 +244,13 @@ def sample_latents(family: int, logw: np.ndarray, T_static, wpp: int, u: np.ndar
             z, m = inv_cdf(logA[i - 1][z, :], u[:, i])
             unit[:, i] = z
             margin = np.minimum(margin, m)
+    elif family == HMM_CTX:
+        z, margin = inv_cdf(logw[pos, 0, :], u[:, 0])
+        unit[:, 0] = z
+        for i in range(1, n):
+            z, m = inv_cdf(logw[pos, 1 + (i - 1) * r + z, :], u[:, i])
+            unit[:, i] = z
+            margin = np.minimum(margin, m)
     elif family == BTREE:
         zs = np.zeros((W, n - 1), dtype=np.int64)
         zs[:, 0], margin = inv_cdf(logw[pos, 0, :], u[:, 0])
@@ -238,7 +273,7 @@ def draft_sample(family: int, h, W_emit, W_sum, T_static, wpp: int, u: np.ndarra
     W_emit = np.asarray(W_emit)
     n, r, v, d = W_emit.shape
     logphi = emission_logphi(h, W_emit)                     # [P, n, r, v]
-    logw = sum_unit_logw(h, W_sum, r)
+    logw = head_logw(family, h, W_sum, T_static, r)
     P = logphi.shape[0]
     pos = np.repeat(np.arange(P), wpp)
     unit, margin = sample_latents(family, logw, T_static, wpp, u, n)
@@ -273,7 +308,7 @@ def prefix_logprob(family: int, logw: np.ndarray, logphi: np.ndarray, T_static, 
 def window_prefix_logprob(family: int, h, W_emit, W_sum, T_static, targets) -> np.ndarray:
     """Prefix log-marginals of the observed window at every position: [T, n]; column n-1 is the joint."""
     r = np.asarray(W_emit).shape[1]
-    return prefix_logprob(family, sum_unit_logw(h, W_sum, r), emission_logphi(h, W_emit), T_static, targets)
+    return prefix_logprob(family, head_logw(family, h, W_sum, T_static, r), emission_logphi(h, W_emit), T_static, targets)
 
 
 def next_byte_logprob(family: int, logw: np.ndarray, logphi: np.ndarray, T_static, x: np.ndarray, s: np.ndarray,

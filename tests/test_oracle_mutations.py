@@ -163,6 +163,41 @@ def accept_wrong(orc):
     return float(bad)
 
 
+def hmm_ctx_gap(orc):
+    """Contextual HMM against path enumeration with each position's own tables (softmax taken here with scipy)."""
+    import scipy.special
+    rng = np.random.default_rng(8)
+    n, r, v, d, T = 3, 2, 3, 4, 2
+    h = rng.normal(size=(T, d))
+    R = rng.normal(size=((1 + (n - 1) * r) * r, d))
+    bias = rng.normal(size=(n - 1, r, r))
+    phi = pins.rand_simplex(rng, T, n, r, v)
+    logits = h @ R.T
+    gap = 0.0
+    for t in range(T):
+        pi = scipy.special.softmax(logits[t, :r])
+        A = scipy.special.softmax(logits[t, r:].reshape(n - 1, r, r) + bias, axis=-1)
+        for x in itertools.product(range(v), repeat=n):
+            g = orc.evidence(np.log(phi[t])[None], np.array([x]))
+            logw = orc.sum_unit_logw(h[t:t + 1], R, r, bias=bias)
+            got = orc.circuit_eval(orc.HMM_CTX, logw, g)[0]
+            gap = max(gap, abs(got - math.log(pins.enum_hmm(pi, A, phi[t], x))))
+    return gap
+
+
+def hmm_ctx_sampler_wrong(orc):
+    # deterministic chain through the bias (R = 0): 0 -> 1 -> 2 -> 0; a transposed table walks it backwards
+    r, n = 3, 4
+    bias = np.full((n - 1, r, r), -1e5)
+    for a in range(r):
+        bias[:, a, (a + 1) % r] = 0.0
+    R = np.zeros(((1 + (n - 1) * r) * r, 2))
+    R[0, 0] = 50.0                                      # initial state 0
+    logw = orc.sum_unit_logw(np.array([[1.0, 0.0]]), R, r, bias=bias)
+    unit, _ = orc.sample_latents(orc.HMM_CTX, logw, None, 1, np.full((1, 2 * n), 0.5), n)
+    return 0.0 if unit.tolist() == [[0, 1, 2, 0]] else 1.0
+
+
 def loss_gap(orc):
     ln = math.log
     prefix = np.array([[ln(1 / 2), ln(1 / 8)], [ln(1 / 8), ln(1 / 8)], [ln(1 / 2), ln(1 / 4)], [0.0, 0.0]])
@@ -213,6 +248,15 @@ MUTANTS = [
     ("byte after a full acceptance drawn from the wrong target row", "inv_cdf(np.log(np.maximum(p[full, n, :], 1e-300)), u[full, n])",
      "inv_cdf(np.log(np.maximum(p[full, n - 1, :], 1e-300)), u[full, n])", accept_wrong),
     ("acceptance test uses the last uniform", "alpha = u[w, s]", "alpha = u[w, n]", accept_wrong),
+    ("contextual table of the wrong step", "logA = logw[:, 1 + (i - 1) * r:1 + i * r, :]", "logA = logw[:, 1:1 + r, :]", hmm_ctx_gap),
+    ("contextual table transposed", "alpha = g[:, i, :] + logsumexp(alpha[:, :, None] + logA, axis=1)",
+     "alpha = g[:, i, :] + logsumexp(alpha[:, None, :] + logA, axis=2)", hmm_ctx_gap),
+    ("transition bias dropped", "logits[:, 1:, :] += np.asarray(bias, dtype=np.float64).reshape(1, -1, r)",
+     "logits[:, 1:, :] += 0.0", hmm_ctx_gap),
+    ("transition bias also added to the initial unit", "logits[:, 1:, :] += np.asarray(bias, dtype=np.float64).reshape(1, -1, r)",
+     "logits[:, :-1, :] += np.asarray(bias, dtype=np.float64).reshape(1, -1, r)", hmm_ctx_gap),
+    ("contextual sampler ignores the previous state", "inv_cdf(logw[pos, 1 + (i - 1) * r + z, :], u[:, i])",
+     "inv_cdf(logw[pos, 1 + (i - 1) * r, :], u[:, i])", hmm_ctx_sampler_wrong),
     ("loss normalised by the sequence length instead of the valid count", "acc += cond[rows, j][valid].sum() / V",
      "acc += cond[rows, j][valid].sum() / L", loss_gap),
     ("loss counts invalid bytes", "valid = tg[rows, j] >= 0", "valid = tg[rows, j] >= -1", loss_gap),
@@ -225,7 +269,7 @@ MUTANTS = [
 
 
 def test_every_pin_passes_on_the_real_oracle():
-    orc = mutant("CP, HMM, BTREE = 0, 1, 2", "CP, HMM, BTREE = 0, 1, 2")        # unmodified copy
+    orc = mutant("CP, HMM, BTREE, HMM_CTX = 0, 1, 2, 3", "CP, HMM, BTREE, HMM_CTX = 0, 1, 2, 3")   # unmodified copy
     for pin in {m[3] for m in MUTANTS}:
         assert pin(orc) < 1e-12, pin.__name__
 
