@@ -52,6 +52,11 @@ enum {
   MTPC_ERR_STATE = -8        /* mtpc_speculative_accept without a matching draft call before it         */
 };
 
+/* mtpc_config.flags */
+enum {
+  MTPC_FLAG_HMM_CONTEXTUAL = 1u /* MTPC_HMM only: the transitions depend on the hidden state (App. H), see below */
+};
+
 /* Bits of the device status word. */
 enum {
   MTPC_STATUS_BAD_TARGET = 1u,  /* a target >= v was seen; that window's log-prob is NaN               */
@@ -70,7 +75,7 @@ typedef struct {
   int32_t io_dtype;            /* MTPC_F32 | MTPC_BF16: dtype of hidden, W_emit and W_sum              */
   int32_t max_positions;       /* upper bound on T (log-prob) and P (draft) per call                   */
   int32_t max_windows_per_pos; /* upper bound on wpp (>= 1; <= 64)                                     */
-  uint32_t flags;              /* must be 0 (bit 0 is reserved for contextual HMM transitions)         */
+  uint32_t flags;              /* 0 or MTPC_FLAG_HMM_CONTEXTUAL                                        */
 } mtpc_config;
 
 /* Bytes of device workspace a head with this configuration needs (a multiple of 256). */
@@ -87,6 +92,11 @@ int mtpc_workspace_bytes(const mtpc_config* cfg, size_t* out_bytes);
  *            z_j = b given z_parent(j) = a (softmax over b).
  *   T_static dev [n-1, r, r] fp32, HMM only (else NULL): logit of z_i = b given z_{i-1} = a at
  *            [i-1, a, b], softmax over b (Eq. HMM with input-independent transitions, App. H).
+ *            With MTPC_FLAG_HMM_CONTEXTUAL (App. H, "contextual, inhomogeneous"; the paper's best HMM): the
+ *            transitions come from the hidden state. W_sum then has S = 1+(n-1)*r sum units: rows [0,r) the
+ *            initial-state logits, row r + ((i-1)*r + a)*r + b the logit of z_i = b given z_{i-1} = a, and
+ *            T_static is the bias added to those logits before the softmax (the term that allows the identity
+ *            initialisation), or NULL for no bias. The bias is copied into the workspace at creation.
  *   workspace dev, 256-byte aligned, >= mtpc_workspace_bytes(cfg); owned by the caller, used by every call
  *            on this head, and must outlive it. With MTPC_BF16 the head keeps the W_emit / W_sum pointers
  *            (they must outlive it too); with MTPC_F32 it keeps rounded copies in the workspace.
@@ -229,9 +239,9 @@ int mtpc_launch_count(mtpc_head* head, uint64_t* out_count);
  * holds those bytes until the process exits, whether or not this function is ever called. It calls no
  * cudaMalloc / cudaFree and no allocating library routine.
  *
- *   cfg        family, n, r, v, d as for mtpc_create_head; io_dtype must be MTPC_BF16 (MTPC_ERR_UNSUPPORTED
- *              otherwise: fp32 inputs would need a rounded copy of the weights); max_positions,
- *              max_windows_per_pos are ignored; flags must be 0.
+ *   cfg        family, n, r, v, d as for mtpc_create_head; io_dtype must be MTPC_BF16 and flags 0
+ *              (MTPC_ERR_UNSUPPORTED otherwise: fp32 inputs would need a rounded copy of the weights, contextual
+ *              transitions a copy of their bias); max_positions, max_windows_per_pos are ignored.
  *   W_emit, W_sum, T_static, hidden, targets, out_logprob: dev, exactly as for mtpc_create_head and
  *              mtpc_window_logprob; all caller-owned, read or written only by the work this call enqueues.
  *   out_status dev uint32 or NULL: receives this call's MTPC_STATUS_* bits (stream-ordered, like the outputs).

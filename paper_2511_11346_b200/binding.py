@@ -13,6 +13,7 @@ from . import build as _build
 
 MTPC_CP, MTPC_HMM, MTPC_BTREE = 0, 1, 2
 MTPC_F32, MTPC_BF16 = 0, 1
+MTPC_FLAG_HMM_CONTEXTUAL = 1
 MTPC_OK = 0
 STATUS_BAD_TARGET, STATUS_BAD_UNIFORM, STATUS_TIMEOUT = 1, 2, 4
 
@@ -120,9 +121,9 @@ class MtpcHead:
     """Owns the opaque head handle and keeps the tensors the head points into alive."""
 
     def __init__(self, family: int, n: int, r: int, v: int, d: int, io_dtype: int, max_positions: int,
-                 max_windows_per_pos: int, W_emit, W_sum, T_static=None, stream=None):
+                 max_windows_per_pos: int, W_emit, W_sum, T_static=None, stream=None, flags: int = 0):
         import torch
-        self.cfg = MtpcConfig(family, n, r, v, d, io_dtype, max_positions, max_windows_per_pos, 0)
+        self.cfg = MtpcConfig(family, n, r, v, d, io_dtype, max_positions, max_windows_per_pos, flags)
         nbytes = mtpc_workspace_bytes(self.cfg)
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=W_emit.device)
         self._keep = (W_emit, W_sum, T_static)

@@ -46,7 +46,7 @@ struct Layout {
   size_t max_windows;
   // workspace offsets (bytes)
   size_t off_status, off_wemit, off_wsum, off_hidden, off_logA, off_G, off_logw, off_sel, off_logits, off_unit_lse;
-  size_t off_prefix, off_partial;   // training loss: prefix log-marginals [max_positions, n], per-sequence terms
+  size_t off_prefix, off_partial, off_sum_bias;   // training loss: prefix log-marginals [max_positions, n], per-sequence terms
   int decode_max_p;     // positions the few-position draft path can take (0: path not available)
   size_t off_h_hidden, off_h_targets, off_h_uniforms, off_h_bytes, off_h_out;
   size_t total;
@@ -74,7 +74,9 @@ int plan(const mtpc_config& c, Layout* L) {
   if (c.io_dtype != MTPC_F32 && c.io_dtype != MTPC_BF16) return MTPC_ERR_SHAPE;
   if (c.n < 1 || c.r < 1 || c.v < 1 || c.d < 1 || c.max_positions < 1 || c.max_windows_per_pos < 1)
     return MTPC_ERR_SHAPE;
-  if (c.flags != 0) return MTPC_ERR_UNSUPPORTED;
+  if ((c.flags & ~MTPC_FLAG_HMM_CONTEXTUAL) != 0) return MTPC_ERR_UNSUPPORTED;
+  const bool ctx = (c.flags & MTPC_FLAG_HMM_CONTEXTUAL) != 0;
+  if (ctx && c.family != MTPC_HMM) return MTPC_ERR_UNSUPPORTED;
   if (c.n > 64 || c.max_windows_per_pos > 64) return MTPC_ERR_UNSUPPORTED;
   if (!is_pow2(c.r) || c.r > 128) return MTPC_ERR_UNSUPPORTED;
   if (c.family != MTPC_CP && c.r > 32) return MTPC_ERR_UNSUPPORTED;
@@ -83,7 +85,7 @@ int plan(const mtpc_config& c, Layout* L) {
   if (c.v % 16 != 0 || c.v > 512) return MTPC_ERR_UNSUPPORTED;
   if (static_cast<int64_t>(c.n) * c.r * c.v > (1ll << 30)) return MTPC_ERR_SHAPE;
 
-  L->S = (c.family == MTPC_BTREE) ? 1 + (c.n - 2) * c.r : 1;
+  L->S = (c.family == MTPC_BTREE) ? 1 + (c.n - 2) * c.r : (ctx ? 1 + (c.n - 1) * c.r : 1);
   L->sum_rows = L->S * c.r;
   // sum tile: a multiple of both r and 16, at most 256 columns
   const int unit = c.r > 16 ? c.r : 16;
@@ -121,7 +123,8 @@ int plan(const mtpc_config& c, Layout* L) {
   L->off_wemit = take(f32 ? static_cast<size_t>(c.n) * c.r * c.v * c.d * 2 : 0);
   L->off_wsum = take(f32 ? static_cast<size_t>(L->sum_rows) * c.d * 2 : 0);
   L->off_hidden = take(f32 ? static_cast<size_t>(c.max_positions) * c.d * 2 : 0);
-  L->off_logA = take(c.family == MTPC_HMM ? static_cast<size_t>(c.n - 1) * c.r * c.r * 4 : 0);
+  L->off_logA = take(c.family == MTPC_HMM && !ctx ? static_cast<size_t>(c.n - 1) * c.r * c.r * 4 : 0);
+  L->off_sum_bias = take(ctx ? static_cast<size_t>(L->sum_rows) * 4 : 0);
   L->off_G = take(L->max_windows * c.n * c.r * 4);
   L->off_logw = take(static_cast<size_t>(c.max_positions) * L->sum_rows * 4);
   L->off_sel = take(L->max_windows * c.n * 4);
@@ -195,6 +198,16 @@ namespace {
 template <typename T>
 T* at(mtpc_head* h, size_t off) { return reinterpret_cast<T*>(h->ws + off); }
 
+bool is_ctx(const mtpc_head* h) { return (h->cfg.flags & MTPC_FLAG_HMM_CONTEXTUAL) != 0; }
+// HMM transition log-probabilities as the kernels read them: position p's tables start at base + p * stride.
+// Static transitions: one set in the workspace, stride 0. Contextual (App. H): the sum units after the first one
+// in every position's row of log omega.
+const float* hmm_tables(mtpc_head* h) {
+  return is_ctx(h) ? at<float>(h, h->L.off_logw) + h->cfg.r : at<float>(h, h->L.off_logA);
+}
+int hmm_table_stride(const mtpc_head* h) { return is_ctx(h) ? h->L.sum_rows : 0; }
+const float* sum_bias(mtpc_head* h) { return is_ctx(h) ? at<float>(h, h->L.off_sum_bias) : nullptr; }
+
 struct PhaseTimer {
   mtpc_head* h;
   cudaStream_t st;
@@ -257,6 +270,7 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   p.targets = targets;
   p.G = at<float>(h, L.off_G);
   p.logw = at<float>(h, L.off_logw);
+  p.sum_bias = sum_bias(h);
   p.unit_sel = at<int>(h, L.off_sel);
   p.uniforms = uniforms;
   p.out_bytes = out_bytes;
@@ -292,10 +306,10 @@ int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cuda
     circuit_cp_kernel<<<blocks, threads, 0, st>>>(G, logw, out, prefix, W, wpp, c.n, c.r, L.sum_rows);
   } else if (c.family == MTPC_HMM) {
     const size_t table_bytes = static_cast<size_t>(c.n - 1) * c.r * c.r * 4;
-    const int in_smem = table_bytes <= kHmmTableSmemLimit;
+    const int in_smem = !is_ctx(h) && table_bytes <= kHmmTableSmemLimit;
     const int cap = 4 * h->num_sms;                      // CTAs stride over the windows: the tables are staged once each
     circuit_hmm_kernel<<<blocks < cap ? blocks : cap, threads, in_smem ? table_bytes : 0, st>>>(
-        G, logw, at<float>(h, L.off_logA), out, prefix, W, wpp, c.n, c.r, L.sum_rows, in_smem);
+        G, logw, hmm_tables(h), out, prefix, W, wpp, c.n, c.r, L.sum_rows, in_smem, hmm_table_stride(h));
   } else if (prefix != nullptr) {
     circuit_btree_kernel<true><<<blocks, threads, btree_smem_bytes(c.n, c.r, true), st>>>(G, logw, out, prefix, W, wpp,
                                                                                         c.n, c.r, L.sum_rows);
@@ -375,6 +389,7 @@ int launch_decode_gemm(mtpc_head* h, const void* hidden_bf16, int P, cudaStream_
   if (p.stages > kMaxStages) p.stages = kMaxStages;
   p.logits = at<float>(h, L.off_logits);
   p.logw = at<float>(h, L.off_logw);
+  p.sum_bias = sum_bias(h);
   p.status = at<unsigned>(h, L.off_status);
   const int tiles = p.emit_tiles + p.sum_tiles;
   const int grid = tiles < h->num_sms ? tiles : h->num_sms;
@@ -436,9 +451,9 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
     if (rc != MTPC_OK) return rc;
     pt.begin();
     draft_slot_kernel<<<dim3(c.n, P), kSlotThreads, 2 * c.r * sizeof(float), st>>>(
-        c.family, at<float>(h, L.off_logits), at<float>(h, L.off_logw), at<float>(h, L.off_logA), uniforms, out_bytes,
+        c.family, at<float>(h, L.off_logits), at<float>(h, L.off_logw), hmm_tables(h), uniforms, out_bytes,
         at<float>(h, L.off_G), at<float>(h, L.off_unit_lse), at<unsigned>(h, L.off_status), wpp, c.n, c.r, c.v,
-        L.sum_rows);
+        L.sum_rows, hmm_table_stride(h));
     h->launches++;
     h->draft_P = P;
     pt.end();
@@ -454,9 +469,10 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   pt.end();
   if (rc != MTPC_OK) return rc;
   pt.begin();
-  latent_sample_kernel<<<(W + 127) / 128, 128, 0, st>>>(c.family, at<float>(h, L.off_logw), at<float>(h, L.off_logA),
-                                                        uniforms, at<int>(h, L.off_sel), out_bytes,
-                                                        at<unsigned>(h, L.off_status), W, wpp, c.n, c.r, L.sum_rows);
+  latent_sample_kernel<<<(W + 127) / 128, 128, 0, st>>>(c.family, at<float>(h, L.off_logw), hmm_tables(h), uniforms,
+                                                        at<int>(h, L.off_sel), out_bytes,
+                                                        at<unsigned>(h, L.off_status), W, wpp, c.n, c.r, L.sum_rows,
+                                                        hmm_table_stride(h));
   h->launches++;
   pt.end();
   if ((rc = check_launch()) != MTPC_OK) return rc;
@@ -502,7 +518,8 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   Layout L;
   int rc = plan(*cfg, &L);
   if (rc != MTPC_OK) return rc;
-  if (cfg->family == MTPC_HMM && cfg->n > 1 && !T_static) return MTPC_ERR_NULL;
+  const bool ctx = (cfg->flags & MTPC_FLAG_HMM_CONTEXTUAL) != 0;
+  if (cfg->family == MTPC_HMM && cfg->n > 1 && !ctx && !T_static) return MTPC_ERR_NULL;
   if (workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0) return MTPC_ERR_WORKSPACE;
   int dev = 0, cc_major = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return MTPC_ERR_CUDA;
@@ -547,7 +564,15 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
     h->W_emit_bf16 = W_emit;
     h->W_sum_bf16 = W_sum;
   }
-  if (cfg->family == MTPC_HMM && cfg->n > 1) {
+  if (ctx) {
+    // bias of the contextual transition logits, laid out like the sum-unit rows: zeros for the initial unit
+    bool bad = cudaMemsetAsync(h->ws + L.off_sum_bias, 0, static_cast<size_t>(L.sum_rows) * 4, st) != cudaSuccess;
+    if (T_static && cfg->n > 1)
+      bad |= cudaMemcpyAsync(h->ws + L.off_sum_bias + static_cast<size_t>(cfg->r) * 4, T_static,
+                             static_cast<size_t>(cfg->n - 1) * cfg->r * cfg->r * 4, cudaMemcpyDeviceToDevice,
+                             st) != cudaSuccess;
+    if (bad) { delete h; return MTPC_ERR_CUDA; }
+  } else if (cfg->family == MTPC_HMM && cfg->n > 1) {
     const int rows = (cfg->n - 1) * cfg->r;
     log_softmax_rows_kernel<<<(rows + 127) / 128, 128, 0, st>>>(T_static, at<float>(h, L.off_logA), rows, cfg->r);
     h->launches++;
@@ -626,8 +651,8 @@ int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32
   pt.begin();
   spec_accept_kernel<<<(W + kAcceptWarps - 1) / kAcceptWarps, kAcceptWarps * 32, smem, st>>>(
       c.family, at<float>(head, L.off_logits), at<float>(head, L.off_unit_lse), at<float>(head, L.off_logw),
-      at<float>(head, L.off_logA), draft_bytes, prefix_logprob, target_probs, accept_uniforms, out_accepted,
-      out_next_byte, at<unsigned>(head, L.off_status), W, wpp, c.n, c.r, c.v, L.sum_rows);
+      hmm_tables(head), draft_bytes, prefix_logprob, target_probs, accept_uniforms, out_accepted,
+      out_next_byte, at<unsigned>(head, L.off_status), W, wpp, c.n, c.r, c.v, L.sum_rows, hmm_table_stride(head));
   head->launches++;
   pt.end();
   return check_launch();
@@ -828,6 +853,7 @@ extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_
                                           int32_t T, float* out_logprob, uint32_t* out_status, void* stream) {
   if (!cfg) return MTPC_ERR_NULL;
   if (cfg->io_dtype != MTPC_BF16) return MTPC_ERR_UNSUPPORTED;   // fp32 inputs would need rounded copies of the weights
+  if (cfg->flags != 0) return MTPC_ERR_UNSUPPORTED;
   if (T < 0) return MTPC_ERR_SHAPE;
   mtpc_config c = *cfg;
   c.max_positions = T > 0 ? T : 1;
@@ -843,7 +869,7 @@ extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_
   L.off_G = take(static_cast<size_t>(c.max_positions) * c.n * c.r * 4);
   L.off_logw = take(static_cast<size_t>(c.max_positions) * L.sum_rows * 4);
   L.off_sel = L.off_wemit = L.off_wsum = L.off_hidden = L.off_logits = L.off_unit_lse = 0;   // unused by this call
-  L.off_prefix = L.off_partial = 0;
+  L.off_prefix = L.off_partial = L.off_sum_bias = 0;
   L.off_h_hidden = L.off_h_targets = L.off_h_uniforms = L.off_h_bytes = L.off_h_out = 0;
   L.total = off;
   if (L.total > static_cast<size_t>(MTPC_STATIC_SCRATCH_BYTES)) return MTPC_ERR_STATIC_SCRATCH;

@@ -91,11 +91,12 @@ __global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __re
 // alpha_i[k] = G[i,k] + m + log sum_a exp(alpha_{i-1}[a] - m) A[i-1][a][k], A = exp(logA) staged once per CTA in
 // shared memory ((n-1) r^2 floats; read straight from global memory when that does not fit). One warp per
 // window, lane = state; CTAs stride over the windows. With `prefix` (may be NULL) the kernel also writes
-// prefix[w, i] = log q(x_0..x_i) = LSE_k alpha_i[k].
+// prefix[w, i] = log q(x_0..x_i) = LSE_k alpha_i[k]. Contextual transitions (App. H): logA = log omega + r and
+// logA_stride = sum_rows, so that position p reads its own tables (never staged: tables_in_smem = 0).
 __global__ void circuit_hmm_kernel(const float* __restrict__ G, const float* __restrict__ logw,
                                    const float* __restrict__ logA, float* __restrict__ out,
                                    float* __restrict__ prefix, int W, int wpp, int n, int r, int sum_rows,
-                                   int tables_in_smem) {
+                                   int tables_in_smem, int logA_stride) {
   extern __shared__ float A_lin[];
   const int lane = threadIdx.x & 31;
   const int count = (n - 1) * r * r;
@@ -123,7 +124,7 @@ __global__ void circuit_hmm_kernel(const float* __restrict__ G, const float* __r
         const float* A = A_lin + static_cast<size_t>(i - 1) * r * r;
         for (int a = 0; a < r; ++a) s = fmaf(__shfl_sync(kFull, e, a), has ? A[a * r + lane] : 0.f, s);
       } else {
-        const float* A = logA + static_cast<size_t>(i - 1) * r * r;
+        const float* A = logA + static_cast<size_t>(w / wpp) * logA_stride + static_cast<size_t>(i - 1) * r * r;
         for (int a = 0; a < r; ++a) s = fmaf(__shfl_sync(kFull, e, a), has ? __expf(__ldg(A + a * r + lane)) : 0.f, s);
       }
       if (has) alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : gi + m + __logf(s);
@@ -247,7 +248,7 @@ __device__ __forceinline__ int inv_cdf_logp(const float* __restrict__ logp, int 
 __global__ void latent_sample_kernel(int family, const float* __restrict__ logw, const float* __restrict__ logA,
                                      const float* __restrict__ uniforms, int* __restrict__ unit_sel,
                                      int* __restrict__ out_bytes, unsigned* status, int W, int wpp, int n, int r,
-                                     int sum_rows) {
+                                     int sum_rows, int logA_stride) {
   const int w = blockIdx.x * blockDim.x + threadIdx.x;
   if (w >= W) return;
   const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
@@ -269,7 +270,7 @@ __global__ void latent_sample_kernel(int family, const float* __restrict__ logw,
     int z = inv_cdf_logp(lw, r, u[0]);
     sel[0] = z;
     for (int i = 1; i < n; ++i) {
-      z = inv_cdf_logp(logA + (static_cast<size_t>(i - 1) * r + z) * r, r, u[i]);
+      z = inv_cdf_logp(logA + static_cast<size_t>(w / wpp) * logA_stride + (static_cast<size_t>(i - 1) * r + z) * r, r, u[i]);
       sel[i] = z;
     }
   } else {

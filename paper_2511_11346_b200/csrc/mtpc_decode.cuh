@@ -42,6 +42,7 @@ struct DecodeParams {
   int stages, stage_bytes;
   float* logits;         // [P, emit_rows]
   float* logw;           // [P, sum_rows]
+  const float* sum_bias; // [sum_rows] or NULL: added to the sum-unit logits before their softmax
   unsigned* status;
 };
 
@@ -201,10 +202,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_decode_gemm_kernel(const
         const int local = quarter * 32 + lane;
         const int row = t.index * t.rows + local;
         const bool mine = local < t.rows && row < nrows;
+        const float bias = (t.is_sum && p.sum_bias != nullptr && mine) ? p.sum_bias[row] : 0.f;
         for (int b = 0; b < (p.P + 15) / 16; ++b) {
           float x[16];
           tmem_ld16(tcol + b * 16, x);
           if (t.is_sum) {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) x[c] += bias;
             // log-softmax over the r rows of a sum unit = r adjacent lanes (r a power of two <= 32); the 16
             // positions of the batch are reduced side by side so that the shuffles overlap
             float m[16], e[16];
@@ -293,12 +297,14 @@ __device__ __forceinline__ int warp_sample_unit(int family, const float* __restr
   return z;
 }
 
+// logA: HMM transition log-probabilities [n-1, r, r]; position p reads them at logA + p * logA_stride (stride 0:
+// one static set for all positions; stride sum_rows with logA = log omega + r: contextual tables, App. H).
 // grid = (n, P). Shared memory: 2 * r floats (max and log-sum-exp of each unit of the slot). The log-sum-exps also
 // go to unit_lse_out [P, n, r], so that later calls can turn the retained logits into log phi.
 __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     int family, const float* __restrict__ logits, const float* __restrict__ logw, const float* __restrict__ logA,
     const float* __restrict__ uniforms, int* __restrict__ out_bytes, float* __restrict__ G,
-    float* __restrict__ unit_lse_out, unsigned* status, int wpp, int n, int r, int v, int sum_rows) {
+    float* __restrict__ unit_lse_out, unsigned* status, int wpp, int n, int r, int v, int sum_rows, int logA_stride) {
   extern __shared__ float sm[];
   float* unit_max = sm;
   float* unit_lse = sm + r;
@@ -331,7 +337,7 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
   for (int j = warp; j < wpp; j += nwarps) {
     const size_t w = static_cast<size_t>(pos) * wpp + j;
     const float* u = uniforms + w * 2 * n;
-    const int z = warp_sample_unit(family, lw, logA, u, n, r, i, lane);
+    const int z = warp_sample_unit(family, lw, logA + static_cast<size_t>(pos) * logA_stride, u, n, r, i, lane);
     const float ub = u[n + i];
     int byte = -1;
     if (z < 0 || !(ub >= 0.f && ub < 1.f)) {
@@ -396,7 +402,7 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
     int family, const float* __restrict__ logits, const float* __restrict__ unit_lse, const float* __restrict__ logw,
     const float* __restrict__ logA, const int* __restrict__ bytes, const float* __restrict__ prefix,
     const float* __restrict__ target, const float* __restrict__ uniforms, int* __restrict__ out_accepted,
-    int* __restrict__ out_next, unsigned* status, int W, int wpp, int n, int r, int v, int sum_rows) {
+    int* __restrict__ out_next, unsigned* status, int W, int wpp, int n, int r, int v, int sum_rows, int logA_stride) {
   extern __shared__ float sm[];
   const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int w = blockIdx.x * kAcceptWarps + wib;
@@ -454,7 +460,7 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
         const float e = has ? __expf(alpha - m) : 0.f;
-        const float* A = logA + static_cast<size_t>(i) * r * r;
+        const float* A = logA + static_cast<size_t>(pos) * logA_stride + static_cast<size_t>(i) * r * r;
         float acc = 0.f;
         for (int a = 0; a < r; ++a) acc = fmaf(__shfl_sync(kFull, e, a), has ? __expf(__ldg(A + a * r + lane)) : 0.f, acc);
         alpha = has ? m + __logf(acc) : -CUDART_INF_F;

@@ -57,6 +57,7 @@ struct GemmParams {
   const int* targets;                // [T*wpp, n]
   float* G;                          // [T*wpp, n, r]   log phi at the target
   float* logw;                       // [T, S*r]        log-softmaxed sum-unit weights
+  const float* sum_bias;             // [S*r] or NULL   added to the sum-unit logits before their softmax
   const int* unit_sel;               // [T*wpp, n]      selected input unit per token (sample mode)
   const float* uniforms;             // [T*wpp, 2n]
   int* out_bytes;                    // [T*wpp, n]
@@ -310,6 +311,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
             tmem_ld16(tcol + b * 16, x);
             if (valid) {
               const int col0 = col_base + b * 16;
+              if (p.sum_bias != nullptr) {
+#pragma unroll
+                for (int q = 0; q < 16; ++q)
+                  if (col0 + q < p.sum_rows) x[q] += p.sum_bias[col0 + q];
+              }
               switch (p.r) {
                 case 1: sum_groups_in_batch<1>(x, dst, col0, p.sum_rows); break;
                 case 2: sum_groups_in_batch<2>(x, dst, col0, p.sum_rows); break;
@@ -323,9 +329,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
           const int bpg = p.r / 16;   // batches per group
           for (int g = 0; g < tc.cols / p.r; ++g) {
             float m = -CUDART_INF_F, s = 0.f;
+            const int gcol = col_base + g * p.r;
+            const bool biased = p.sum_bias != nullptr && gcol < p.sum_rows;
             for (int b = 0; b < bpg; ++b) {
               float x[16];
               tmem_ld16(tcol + (g * bpg + b) * 16, x);
+              if (biased) {
+#pragma unroll
+                for (int q = 0; q < 16; ++q) x[q] += p.sum_bias[gcol + b * 16 + q];
+              }
               float bm = x[0];
 #pragma unroll
               for (int q = 1; q < 16; ++q) bm = fmaxf(bm, x[q]);
@@ -336,10 +348,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
               m = mn;
             }
             const float lse = m + fast_lg2(s) * kLn2;
-            const int gcol = col_base + g * p.r;
             for (int b = 0; b < bpg; ++b) {
               float x[16];
               tmem_ld16(tcol + (g * bpg + b) * 16, x);
+              if (biased) {
+#pragma unroll
+                for (int q = 0; q < 16; ++q) x[q] += p.sum_bias[gcol + b * 16 + q];
+              }
               if (valid && gcol < p.sum_rows) {
                 float4* d4 = reinterpret_cast<float4*>(dst + gcol + b * 16);
 #pragma unroll

@@ -11,6 +11,7 @@ weights and data that are not available offline):
   2  HMM                T=8192 d=4096 n=8  r=32 v=320  bf16, static transitions ~N(0,1), Zipf(1.1) targets
   3  BTree              T=4096 d=3072 n=16 r=32 v=256  bf16, uniform targets, + draft wpp=1
   4  decode sweep cells P in {1,8,64}, d=4096, v=320, CP r=16 / HMM r=32, n in {8,16}, wpp=16
+  5  HMM with contextual transitions: as 2, plus (n-1) r r = 7168 transition rows in W_sum and a bias ~N(0,1) + 4 I
 Hidden states ~N(0,1); every weight ~N(0, std=0.02); uniforms in [0,1) as fp32. For the acceptance stage the
 target model's conditionals are Dirichlet rows (target_rows) and its uniforms come from the same generator.
 """
@@ -22,8 +23,9 @@ from concurrent.futures import ThreadPoolExecutor
 import numpy as np
 
 CP, HMM, BTREE = 0, 1, 2
+HMM_CTX = 3          # HMM with contextual transitions (C ABI: MTPC_HMM with MTPC_FLAG_HMM_CONTEXTUAL)
 F32, BF16 = 0, 1
-FAMILY_NAMES = {CP: "cp", HMM: "hmm", BTREE: "btree"}
+FAMILY_NAMES = {CP: "cp", HMM: "hmm", BTREE: "btree", HMM_CTX: "hmmctx"}
 BASE_SEED = 2511113460
 
 
@@ -41,6 +43,8 @@ class HeadShape:
         """Number of contextual sum units S (each has r weights produced from the hidden state)."""
         if self.family == BTREE:
             return 1 + (self.n - 2) * self.r
+        if self.family == HMM_CTX:
+            return 1 + (self.n - 1) * self.r
         return 1
 
     @property
@@ -170,6 +174,10 @@ def make_workload(name: str, shape: HeadShape, T: int, seed: int, *, target_kind
         T_static = None
         if shape.family == HMM:
             T_static = _normal(seed, 4, (max(shape.n - 1, 1), shape.r, shape.r), trans_std)[: shape.n - 1]
+        elif shape.family == HMM_CTX:
+            # transition bias: a noisy multiple of the identity, as after training from the identity initialisation
+            T_static = _normal(seed, 4, (max(shape.n - 1, 1), shape.r, shape.r), trans_std)[: shape.n - 1]
+            T_static = T_static + np.float32(4.0) * np.eye(shape.r, dtype=np.float32)[None]
         W_emit_q, W_sum_q = bf16_round(W_emit), bf16_round(W_sum)
         if shape.io_dtype != F32:
             W_emit = W_sum = None                # only the rounded copies are kept
@@ -204,9 +212,11 @@ def config_workload(idx: int, *, cell: tuple[int, int, int] | None = None, T: in
     if idx == 3:
         return make_workload("btree_train", HeadShape(BTREE, 16, 32, 256, 3072), T or 4096, seed,
                              target_kind="uniform", wpp=1)
+    if idx == 5:
+        return make_workload("hmmctx_train", HeadShape(HMM_CTX, 8, 32, 320, 4096), T or 8192, seed, target_kind="zipf")
     if idx == 4:
         fam, n, P = cell or (CP, 8, 8)
-        r = 16 if fam == CP else 32
+        r = 16 if fam == CP else 32          # HMM and HMM_CTX
         cseed = seed + 1000 * (fam * 2 + (n // 8 - 1))   # weights shared by the three P of a (family, n)
         return make_workload(f"decode_{FAMILY_NAMES[fam]}_n{n}_P{P}", HeadShape(fam, n, r, 320, 4096), T or P,
                              cseed, target_kind=None, wpp=16)

@@ -51,7 +51,7 @@ def check_draft(dh, wl, rows, wpp=None):
     # joint log-prob of what the GPU actually drafted, all windows
     pos = np.repeat(np.arange(len(rows)), wpp)
     logphi = orc.emission_logphi(wl.hidden_q[rows], wl.W_emit_q)
-    logw = orc.sum_unit_logw(wl.hidden_q[rows], wl.W_sum_q, wl.shape.r)
+    logw = orc.head_logw(wl.shape.family, wl.hidden_q[rows], wl.W_sum_q, wl.T_static, wl.shape.r)
     want = orc.circuit_eval(wl.shape.family, logw[pos], orc.evidence(logphi, gb[wsel], pos), wl.T_static)
     err = np.abs(gl[wsel] - want).max()
     assert err <= LOGPROB_TOL, f"{wl.name}: draft log-prob error {err}"
@@ -68,7 +68,7 @@ def test_config0_cp_tiny_whole():
     dh.close()
 
 
-@pytest.mark.parametrize("idx,nsample", [(1, 256), (2, 256), (3, 128)])
+@pytest.mark.parametrize("idx,nsample", [(1, 256), (2, 256), (3, 128), (5, 128)])
 def test_full_size_configs_on_sampled_positions(idx, nsample):
     """Full-size launch (the configuration the benchmark times); the oracle checks a seeded sample of
     positions, always including the first and last rows of the first and last 128-row tiles."""
@@ -105,6 +105,11 @@ SMALL = [
     (I.HMM, 6, 8, 64, 128, 257, 1),
     (I.HMM, 4, 32, 320, 64, 64, 16),
     (I.HMM, 3, 1, 16, 64, 3, 1),
+    (I.HMM_CTX, 1, 4, 32, 64, 7, 2),
+    (I.HMM_CTX, 6, 8, 64, 128, 257, 1),
+    (I.HMM_CTX, 4, 32, 320, 64, 64, 16),
+    (I.HMM_CTX, 3, 1, 16, 64, 3, 1),
+    (I.HMM_CTX, 5, 16, 48, 64, 140, 3),
     (I.BTREE, 2, 4, 32, 64, 9, 2),
     (I.BTREE, 4, 16, 256, 128, 130, 1),
     (I.BTREE, 8, 32, 48, 64, 33, 4),

@@ -27,7 +27,7 @@ FULL_BAND = 1e-5           # the same for a draw from a target row (both sides r
 
 def oracle_params(wl, rows):
     logphi = orc.emission_logphi(wl.hidden_q[rows], wl.W_emit_q)
-    logw = orc.sum_unit_logw(wl.hidden_q[rows], wl.W_sum_q, wl.shape.r)
+    logw = orc.head_logw(wl.shape.family, wl.hidden_q[rows], wl.W_sum_q, wl.T_static, wl.shape.r)
     return logphi, logw
 
 
@@ -40,6 +40,8 @@ SMALL = [
     (I.HMM, 1, 4, 32, 64, 7),
     (I.HMM, 6, 8, 64, 128, 257),
     (I.HMM, 4, 32, 320, 64, 64),
+    (I.HMM_CTX, 6, 8, 64, 128, 257),
+    (I.HMM_CTX, 4, 32, 320, 64, 64),
     (I.BTREE, 2, 4, 32, 64, 9),
     (I.BTREE, 4, 16, 256, 128, 130),
     (I.BTREE, 8, 32, 48, 64, 33),
@@ -159,6 +161,8 @@ ACCEPT_SMALL = [
     (I.HMM, 1, 4, 32, 64, 2, 8),
     (I.HMM, 6, 8, 64, 128, 9, 8),
     (I.HMM, 4, 32, 512, 64, 3, 16),
+    (I.HMM_CTX, 6, 8, 64, 128, 9, 8),
+    (I.HMM_CTX, 4, 32, 512, 64, 3, 16),
     (I.BTREE, 2, 4, 32, 64, 9, 4),
     (I.BTREE, 4, 16, 256, 128, 6, 8),
     (I.BTREE, 8, 32, 48, 64, 5, 16),
@@ -223,7 +227,8 @@ def test_accept_needs_the_draft_state_and_flags_bad_inputs():
 
 # --------------------------------------------------------------------------- Eq. 6
 @pytest.mark.parametrize("family,n,r,v,d,N,L", [(I.CP, 4, 8, 320, 128, 3, 50), (I.HMM, 8, 16, 64, 64, 5, 33),
-                                                 (I.BTREE, 8, 8, 32, 64, 2, 140), (I.CP, 2, 2, 16, 64, 300, 1)])
+                                                 (I.BTREE, 8, 8, 32, 64, 2, 140), (I.CP, 2, 2, 16, 64, 300, 1),
+                                                 (I.HMM_CTX, 4, 8, 64, 64, 4, 40)])
 def test_window_loss_matches_oracle(family, n, r, v, d, N, L):
     wl = I.make_workload(f"loss_{family}", I.HeadShape(family, n, r, v, d), N * L, seed=4000 + n + N, weight_std=0.25)
     t = wl.targets.copy().reshape(N, L, n)
