@@ -2,7 +2,7 @@
 """Benchmark of the MtPC head on B200: window log-likelihood positions/s on the training-shaped CP workload
 (8192 positions, d=4096, n=8, r=16, v=320), plus draft windows/s on one decode cell.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|5] [--impl reference]
 
 One step = one mtpc_window_logprob call over the whole batch (projection GEMM with fused softmax/gather
 epilogue + circuit evaluation). Prints ONE JSON line on rank 0. With N > 1 (launched by torchrun, one process
@@ -34,7 +34,7 @@ UNIT = "positions/s"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one projection-kernel launch, from the ncu capture
 # summarised in profiles/ (captured at a quarter of the positions and scaled). None = not captured.
-NCU_TRAFFIC_BYTES = {1: None, 2: None, 3: None}
+NCU_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 5: None}
 
 
 def workload_name(idx: int, wl) -> str:
@@ -154,6 +154,12 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def circuit_bytes(wl) -> int:
+    """Algorithmic bytes of one circuit-evaluation launch: it reads G [T, n, r] and log omega [T, S r] and writes [T]."""
+    s = wl.shape
+    return 4 * wl.T * (s.n * s.r + s.sum_rows + 1)
+
+
 def measure_decode_cell(torch, cell, steps: int, warmup: int):
     """Draft windows/s and p50 latency on one decode cell (family, n, P) with 16 windows per position. Every call
     is timed on its own (CUDA events on the launching stream); the library's event ring gives the per-kernel split."""
@@ -181,9 +187,26 @@ def measure_decode_cell(torch, cell, steps: int, warmup: int):
     phase_p50 = [statistics.median(p[k] for p in phases) for k in range(len(phases[0]))]
     launches = len(phases[0])
     dh.head.mtpc_set_timing(0)
+    # draft with prefix marginals + acceptance stage (Algorithm 3) against synthetic target-model rows
+    s = wl.shape
+    tp = torch.from_numpy(I.target_rows(I.BASE_SEED + 77, 9, (W, s.n + 1, s.v))).cuda()
+    ua = torch.from_numpy(I.uniforms(I.BASE_SEED + 78, 10, (W, s.n + 1))).cuda()
+    opre = torch.empty((W, s.n), dtype=torch.float32, device="cuda")
+    oacc = torch.empty(W, dtype=torch.int32, device="cuda")
+    onxt = torch.empty(W, dtype=torch.int32, device="cuda")
+    cyc = []
+    for it in range(warmup + steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        dh.head.mtpc_draft_sample_prefix(h, wl.wpp, u, ob, opre)
+        dh.head.mtpc_speculative_accept(wl.T, wl.wpp, ob, opre, tp, ua, oacc, onxt)
+        e1.record()
+        e1.synchronize()
+        if it >= warmup:
+            cyc.append(e0.elapsed_time(e1))
+    mean_accepted = float(oacc.float().mean().cpu())
     status = dh.head.mtpc_get_status()
     p50 = statistics.median(lat)
-    s = wl.shape
     weight_bytes = (s.n * s.r * s.v + s.sum_rows) * s.d * 2
     peaks, src = load_peaks()
     gbs = weight_bytes / (p50 * 1e-3) / 1e9
@@ -191,12 +214,15 @@ def measure_decode_cell(torch, cell, steps: int, warmup: int):
     out = {"workload": f"configs[4] {wl.name}: P={wl.T} wpp={wl.wpp} d={s.d} n={s.n} r={s.r} v={s.v}",
            "windows_per_s": W / (p50 * 1e-3), "p50_ms": p50, "calls": steps, "kernels_per_call": launches,
            "kernel_p50_ms": phase_p50, "device_status": status,
+           "draft_plus_accept": {"p50_ms": statistics.median(cyc), "kernels_per_call": launches + 1,
+                                 "mean_accepted_bytes_vs_synthetic_target": mean_accepted,
+                                 "calls": "mtpc_draft_sample_prefix + mtpc_speculative_accept"},
            "hbm_roofline": {"algorithmic_bytes": weight_bytes, "note": "one pass over the emission and sum-unit weights",
                             "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
                             "weight_pass_kernel_gbs": gemm_gbs, "weight_pass_kernel_frac": gemm_gbs / peaks["hbm_gbs"],
                             "peak_source": src}}
     dh.close()
-    return out, launches * (steps + warmup)
+    return out, launches * (steps + warmup) + (launches + 1) * (steps + warmup)
 
 
 def run_ours(args):
@@ -279,6 +305,16 @@ def run_ours(args):
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "burst_peak": peaks["bf16_tflops"],
                 "flops_per_launch": flops, "avg_launch_ms": gemm_ms, "circuit_kernel_avg_ms": circuit_ms,
                 "timed_launches": kept}
+    cbytes = circuit_bytes(wl)
+    cgbs = cbytes / (circuit_ms * 1e-3) / 1e9
+    kernels = [
+        {"kernel": "mtpc_gemm_kernel<logprob>", "avg_ms": gemm_ms, "bound": "tensor", "achieved_tflops": achieved,
+         "frac_of_sustained_peak": achieved / peak, "share_of_step": gemm_ms / (gemm_ms + circuit_ms)},
+        {"kernel": {I.CP: "circuit_cp_kernel", I.HMM: "circuit_hmm_kernel", I.BTREE: "circuit_btree_kernel",
+                    I.HMM_CTX: "circuit_hmm_kernel (per-position tables)"}[s.family], "avg_ms": circuit_ms, "bound": "hbm",
+         "algorithmic_bytes": cbytes, "achieved_gbs": cgbs, "peak_gbs": peaks["hbm_gbs"],
+         "frac": cgbs / peaks["hbm_gbs"], "share_of_step": circuit_ms / (gemm_ms + circuit_ms)},
+    ]
 
     # CPU baseline: the oracle as it stands on a bounded sample of the same workload
     cpu_baseline = None
@@ -309,6 +345,7 @@ def run_ours(args):
                 "call": "mtpc_window_logprob_host (pinned host buffers, copies inside the call)"},
         "gpu_launches": int(launches),
         "roofline": roofline,
+        "kernels": kernels,
         "cpu_baseline": cpu_baseline,
         "device_status": status,
     }
@@ -324,7 +361,8 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3])
+    ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3, 5],
+                    help="1 CP (the metric's configuration), 2 HMM, 3 binary tree, 5 HMM with contextual transitions")
     ap.add_argument("--ref-positions", type=int, default=None,
                     help="positions the CPU oracle processes per step / for the cpu_baseline sample")
     ap.add_argument("--no-draft", action="store_true", help="skip the decode-cell draft measurement")

@@ -20,6 +20,7 @@ using namespace mtpc;
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxPhases = 5;
+constexpr int kWorkCounterWord = 16;   // word of the 256-byte status area used as the circuit kernels' work counter
 constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA on sm_100
 // Hidden states of one rasterisation block of the projection kernel: small enough to stay L2-resident next to the
 // weight tiles streaming past (data read by all SMs ends up in both halves of the 126 MB L2).
@@ -286,10 +287,9 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
 }
 
 // Shared memory of one CTA of the binary-tree circuit kernel (see circuit_btree_kernel).
+size_t hmm_ctx_smem_bytes(int r) { return static_cast<size_t>(kCircuitWarps) * (2 * r * r + 32) * sizeof(float); }
 size_t btree_smem_bytes(int n, int r, bool with_prefix) {
-  const size_t per_warp = static_cast<size_t>(n - 1) * r + static_cast<size_t>(r) * (r + 1) +
-                          (with_prefix ? static_cast<size_t>(n - 1) * r + r : 0);
-  return kCircuitWarps * per_warp * sizeof(float);
+  return static_cast<size_t>(kCircuitWarps) * btree_warp_floats(n, r, with_prefix) * sizeof(float);
 }
 
 // Circuit evaluation of W windows: out[w] = joint log-prob (may be NULL when prefix is given); prefix (may be NULL)
@@ -302,20 +302,29 @@ int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cuda
   const float* logw = at<float>(h, L.off_logw);
   const int blocks = (W + kCircuitWarps - 1) / kCircuitWarps;
   const int threads = kCircuitWarps * 32;
+  // kernels that stream per-position tables hand out windows through a counter next to the status word
+  unsigned* counter = at<unsigned>(h, L.off_status) + kWorkCounterWord;
+  const int resident = blocks < 8 * h->num_sms ? blocks : 8 * h->num_sms;   // more CTAs than an SM can hold do no harm
+  if (c.family == MTPC_BTREE || is_ctx(h)) {
+    if (cudaMemsetAsync(counter, 0, sizeof(unsigned), st) != cudaSuccess) return MTPC_ERR_CUDA;
+  }
   if (c.family == MTPC_CP) {
     circuit_cp_kernel<<<blocks, threads, 0, st>>>(G, logw, out, prefix, W, wpp, c.n, c.r, L.sum_rows);
+  } else if (c.family == MTPC_HMM && is_ctx(h)) {
+    circuit_hmm_ctx_kernel<<<resident, threads, hmm_ctx_smem_bytes(c.r), st>>>(G, logw, out, prefix, counter, W, wpp,
+                                                                              c.n, c.r, L.sum_rows);
   } else if (c.family == MTPC_HMM) {
     const size_t table_bytes = static_cast<size_t>(c.n - 1) * c.r * c.r * 4;
-    const int in_smem = !is_ctx(h) && table_bytes <= kHmmTableSmemLimit;
+    const int in_smem = table_bytes <= kHmmTableSmemLimit;
     const int cap = 4 * h->num_sms;                      // CTAs stride over the windows: the tables are staged once each
     circuit_hmm_kernel<<<blocks < cap ? blocks : cap, threads, in_smem ? table_bytes : 0, st>>>(
         G, logw, hmm_tables(h), out, prefix, W, wpp, c.n, c.r, L.sum_rows, in_smem, hmm_table_stride(h));
   } else if (prefix != nullptr) {
-    circuit_btree_kernel<true><<<blocks, threads, btree_smem_bytes(c.n, c.r, true), st>>>(G, logw, out, prefix, W, wpp,
-                                                                                        c.n, c.r, L.sum_rows);
+    circuit_btree_kernel<true><<<resident, threads, btree_smem_bytes(c.n, c.r, true), st>>>(
+        G, logw, out, prefix, counter, W, wpp, c.n, c.r, L.sum_rows);
   } else {
-    circuit_btree_kernel<false><<<blocks, threads, btree_smem_bytes(c.n, c.r, false), st>>>(G, logw, out, nullptr, W,
-                                                                                          wpp, c.n, c.r, L.sum_rows);
+    circuit_btree_kernel<false><<<resident, threads, btree_smem_bytes(c.n, c.r, false), st>>>(
+        G, logw, out, nullptr, counter, W, wpp, c.n, c.r, L.sum_rows);
   }
   h->launches++;
   return check_launch();
@@ -328,6 +337,9 @@ bool set_circuit_attributes(const mtpc_config& c) {
   if (c.family == MTPC_HMM)
     fail |= cudaFuncSetAttribute(circuit_hmm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(kHmmTableSmemLimit)) != cudaSuccess;
+  if (c.family == MTPC_HMM && hmm_ctx_smem_bytes(c.r) > 48 * 1024)
+    fail |= cudaFuncSetAttribute(circuit_hmm_ctx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(hmm_ctx_smem_bytes(c.r))) != cudaSuccess;
   if (c.family == MTPC_BTREE) {
     const int plain = static_cast<int>(btree_smem_bytes(c.n, c.r, false));
     const int pre = static_cast<int>(btree_smem_bytes(c.n, c.r, true));

@@ -164,44 +164,144 @@ __device__ __forceinline__ float btree_sum_layer(const float* __restrict__ tab, 
   return res;
 }
 
-// Shared memory per warp: (n-1) * r floats of prod + r * (r+1) floats of one staged table; with PREFIX another
+// Dynamic work distribution for the kernels whose cost per window is large: every warp takes the next window index
+// from a counter the host zeroes before the launch, so that all SMs stay busy until the last window.
+__device__ __forceinline__ int next_window(unsigned* counter, int lane) {
+  unsigned w = 0;
+  if (lane == 0) w = atomicAdd(counter, 1u);
+  return static_cast<int>(__shfl_sync(kFull, w, 0));
+}
+
+// ---- asynchronous staging of an r x r table (global -> shared) by one warp, for kernels that stream one set of
+// tables per position from HBM: the copy of the next table is in flight while the current one is reduced.
+__device__ __forceinline__ void cp_async_16(float* dst, const float* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(dst))),
+               "l"(src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_4(float* dst, const float* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(dst))),
+               "l"(src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// Copies `count` floats; 16 bytes per request when both addresses allow it (count, src and dst multiples of 4 floats).
+__device__ __forceinline__ void warp_table_load_async(float* dst, const float* __restrict__ src, int count, int lane) {
+  const bool vec = (count & 3) == 0 && ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u) == 0;
+  if (vec) {
+    for (int e = lane * 4; e < count; e += 128) cp_async_16(dst + e, src + e);
+  } else {
+    for (int e = lane; e < count; e += 32) cp_async_4(dst + e, src + e);
+  }
+  cp_async_commit();
+}
+// The same sum layer as btree_sum_layer on a table already in shared memory, unpadded [z][b]; lane z walks its row
+// starting at column z, so that the 32 lanes hit 32 different banks. R a multiple of 4 (both arrays 16-byte aligned):
+// the row and the child's vector are read as float4, rotated by the lane so that a quarter-warp's requests fall in
+// different bank groups, and reduced in registers (max, then sum of exponentials).
+template <int R>
+__device__ __forceinline__ float sum_layer_staged_vec(const float* tab, const float* pc, int lane) {
+  if (lane >= R) return 0.f;
+  constexpr int Q = R / 4;
+  const float4* row4 = reinterpret_cast<const float4*>(tab + lane * R);
+  const float4* pc4 = reinterpret_cast<const float4*>(pc);
+  float v[R];
+#pragma unroll
+  for (int q = 0; q < Q; ++q) {
+    const int j = (q + lane) & (Q - 1);
+    const float4 a = row4[j];
+    const float4 b = pc4[j];
+    v[4 * q] = a.x + b.x;
+    v[4 * q + 1] = a.y + b.y;
+    v[4 * q + 2] = a.z + b.z;
+    v[4 * q + 3] = a.w + b.w;
+  }
+  float m = v[0];
+#pragma unroll
+  for (int q = 1; q < R; ++q) m = fmaxf(m, v[q]);
+  float s = 0.f;
+#pragma unroll
+  for (int q = 0; q < R; ++q) s += __expf(v[q] - m);
+  float res = (m == -CUDART_INF_F) ? -CUDART_INF_F : m + __logf(s);
+  if (s != s) res = s;                             // NaN evidence must survive the max
+  return res;
+}
+__device__ __forceinline__ float sum_layer_staged(const float* tab, const float* pc, int lane, int r) {
+  switch (r) {
+    case 32: return sum_layer_staged_vec<32>(tab, pc, lane);
+    case 16: return sum_layer_staged_vec<16>(tab, pc, lane);
+    case 8: return sum_layer_staged_vec<8>(tab, pc, lane);
+    case 4: return sum_layer_staged_vec<4>(tab, pc, lane);
+    default: break;
+  }
+  if (lane >= r) return 0.f;
+  const float* row = tab + lane * r;
+  float m = -CUDART_INF_F;
+  for (int b = 0; b < r; ++b) m = fmaxf(m, row[b] + pc[b]);
+  float s = 0.f;
+  for (int b = 0; b < r; ++b) s += __expf(row[b] + pc[b] - m);
+  float res = (m == -CUDART_INF_F) ? -CUDART_INF_F : m + __logf(s);
+  if (s != s) res = s;
+  return res;
+}
+
+// Shared memory per warp: (n-1) * r floats of prod + 2 * r * r floats (two staged tables); with PREFIX another
 // (n-1) * r floats (the sum-layer outputs S[c][z], kept for the prefix passes) + r floats.  r <= 32.
+// The n-2 tables of a position (57 KB at n = 16, r = 32) are read exactly once, in the order the bottom-up pass
+// needs them, through a two-deep cp.async pipeline: this kernel is bound by that stream from HBM.
 // PREFIX: also writes prefix[w, i] = log q(x_0..x_i). Summing the later bytes out sets their input units to one,
 // so every subtree right of token i evaluates to one, every subtree left of it keeps its value, and only the
 // nodes on the path from token i's owner to the root have to be re-evaluated.
+__host__ __device__ inline int btree_warp_floats(int n, int r, bool with_prefix) {
+  return (n - 1) * r + 2 * r * r + (with_prefix ? (n - 1) * r + r : 0);
+}
+
 template <bool PREFIX>
 __global__ void circuit_btree_kernel(const float* __restrict__ G, const float* __restrict__ logw,
-                                     float* __restrict__ out, float* __restrict__ prefix, int W, int wpp, int n, int r,
-                                     int sum_rows) {
-  extern __shared__ float sm[];
+                                     float* __restrict__ out, float* __restrict__ prefix, unsigned* work_counter,
+                                     int W, int wpp, int n, int r, int sum_rows) {
+  extern __shared__ __align__(16) float sm[];
   const int wib = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int w = blockIdx.x * kCircuitWarps + wib;
-  const int per_warp = (n - 1) * r + r * (r + 1) + (PREFIX ? (n - 1) * r + r : 0);
-  float* prod = sm + static_cast<size_t>(wib) * per_warp;
-  float* table = prod + (n - 1) * r;
-  float* S = table + r * (r + 1);                  // PREFIX only
+  float* prod = sm + static_cast<size_t>(wib) * btree_warp_floats(n, r, PREFIX);
+  float* tabs = prod + (n - 1) * r;                // two tables; the prefix passes reuse the space as one padded table
+  float* table = tabs;
+  float* S = tabs + 2 * r * r;                     // PREFIX only
   float* cur = S + (n - 1) * r;                    // PREFIX only
-  if (w >= W) return;
-  const float* g = G + static_cast<size_t>(w) * n * r;
-  const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
   const bool has = lane < r;
   const int first_leaf_node = n / 2 - 1;
+  const int rr = r * r;
+  const int ntab = n - 2;                          // table t belongs to child c(t) of node j(t), deepest parents first
+  auto child_of = [&](int t) { return 2 * (first_leaf_node - 1 - (t >> 1)) + 1 + (t & 1); };
+  for (int w = next_window(work_counter, lane); w < W; w = next_window(work_counter, lane)) {
+  const float* g = G + static_cast<size_t>(w) * n * r;
+  const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
+  if (ntab > 0) warp_table_load_async(tabs, lw + r + static_cast<size_t>(child_of(0) - 1) * rr, rr, lane);
   for (int j = n - 2; j >= first_leaf_node; --j) {
     const int m = j - first_leaf_node;
     if (has) prod[j * r + lane] = g[(2 * m) * r + lane] + g[(2 * m + 1) * r + lane];
   }
   __syncwarp();
-  for (int j = first_leaf_node - 1; j >= 0; --j) {
-    float acc = 0.f;
-    for (int side = 0; side < 2; ++side) {
-      const int c = 2 * j + 1 + side;
-      const float sc = btree_sum_layer(lw + r + static_cast<size_t>(c - 1) * r * r, prod + c * r, table, lane, r);
-      if (PREFIX && has) S[c * r + lane] = sc;
-      acc += sc;
+  float acc = 0.f;
+  for (int t = 0; t < ntab; ++t) {
+    const int c = child_of(t);
+    if (t + 1 < ntab) {
+      warp_table_load_async(tabs + ((t + 1) & 1) * rr, lw + r + static_cast<size_t>(child_of(t + 1) - 1) * rr, rr, lane);
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
     }
-    if (has) prod[j * r + lane] = acc;
-    __syncwarp();
+    __syncwarp();                                  // table t is in shared memory for every lane
+    const float sc = sum_layer_staged(tabs + (t & 1) * rr, prod + c * r, lane, r);
+    if (PREFIX && has) S[c * r + lane] = sc;
+    acc += sc;
+    if (t & 1) {                                   // both children of node j done
+      if (has) prod[((c - 2) >> 1) * r + lane] = acc;
+      acc = 0.f;
+    }
+    __syncwarp();                                  // the buffer may be overwritten, prod[j] may be read
   }
   const float res = warp_lse(has ? lw[lane] + prod[lane] : 0.f, has);
   if (lane == 0 && out != nullptr) out[w] = res;
@@ -227,6 +327,75 @@ __global__ void circuit_btree_kernel(const float* __restrict__ G, const float* _
       }
       const float pre = warp_lse(has ? lw[lane] + val : 0.f, has);
       if (lane == 0) prefix[static_cast<size_t>(w) * n + i] = pre;
+    }
+  }
+  __syncwarp();                                    // the next window reuses the warp's shared memory
+  }
+}
+
+// Eq. (HMM) with contextual transitions (App. H): position p = w / wpp has its own tables
+// logA_i[a][k] = logw[p, r + (i-1) r^2 + a r + k], 28 KB per position at n = 8, r = 32, read exactly once: the kernel is
+// bound by that stream from HBM. One warp per window, lane = state; table i+1 is copied into shared memory by
+// cp.async while table i is reduced. Same recursion and same scaled matrix-vector form as circuit_hmm_kernel.
+// Shared memory per warp: 2 * r * r + 32 floats. With `prefix` (may be NULL) also writes prefix[w, i] = LSE_k alpha_i[k].
+__global__ void circuit_hmm_ctx_kernel(const float* __restrict__ G, const float* __restrict__ logw,
+                                       float* __restrict__ out, float* __restrict__ prefix, unsigned* work_counter,
+                                       int W, int wpp, int n, int r, int sum_rows) {
+  extern __shared__ __align__(16) float sm[];
+  const int lane = threadIdx.x & 31;
+  const int rr = r * r;
+  float* tabs = sm + static_cast<size_t>(threadIdx.x >> 5) * (2 * rr + 32);
+  float* evec = tabs + 2 * rr;
+  const bool has = lane < r;
+  for (int w = next_window(work_counter, lane); w < W; w = next_window(work_counter, lane)) {
+    const float* g = G + static_cast<size_t>(w) * n * r;
+    const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
+    if (n > 1) warp_table_load_async(tabs, lw + r, rr, lane);
+    float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
+    for (int i = 1; i < n; ++i) {
+      if (i + 1 < n) {
+        warp_table_load_async(tabs + (i & 1) * rr, lw + r + static_cast<size_t>(i) * rr, rr, lane);
+        cp_async_wait<1>();
+      } else {
+        cp_async_wait<0>();
+      }
+      __syncwarp();                                      // table i is in shared memory for every lane
+      if (prefix != nullptr) {
+        const float pre = warp_lse(alpha, has);
+        if (lane == 0) prefix[static_cast<size_t>(w) * n + i - 1] = pre;
+      }
+      const float* A = tabs + ((i - 1) & 1) * rr;
+      const float gi = has ? g[i * r + lane] : 0.f;
+      float m = alpha;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
+      // e[a] = exp(alpha[a] - m) goes through shared memory: every lane then reads four of them per request
+      // (a broadcast) instead of one shuffle each
+      evec[lane] = has ? __expf(alpha - m) : 0.f;
+      __syncwarp();
+      float s = 0.f;
+      if (has) {
+        if ((r & 3) == 0) {
+          const float4* e4 = reinterpret_cast<const float4*>(evec);
+#pragma unroll 2
+          for (int a = 0; a < r; a += 4) {
+            const float4 ev = e4[a >> 2];
+            s = fmaf(ev.x, __expf(A[a * r + lane]), s);
+            s = fmaf(ev.y, __expf(A[(a + 1) * r + lane]), s);
+            s = fmaf(ev.z, __expf(A[(a + 2) * r + lane]), s);
+            s = fmaf(ev.w, __expf(A[(a + 3) * r + lane]), s);
+          }
+        } else {
+          for (int a = 0; a < r; ++a) s = fmaf(evec[a], __expf(A[a * r + lane]), s);
+        }
+        alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : gi + m + __logf(s);
+      }
+      __syncwarp();                                      // the buffers may be overwritten
+    }
+    const float res = warp_lse(alpha, has);
+    if (lane == 0) {
+      if (out != nullptr) out[w] = res;
+      if (prefix != nullptr) prefix[static_cast<size_t>(w) * n + n - 1] = res;
     }
   }
 }
