@@ -20,12 +20,12 @@ using namespace mtpc;
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxPhases = 5;
+constexpr size_t kSlotSmemLimit = 160 * 1024;   // latent-draw tables of the draft slot kernel kept in shared memory up to this
 constexpr int kWorkCounterWord = 16;   // word of the 256-byte status area used as the circuit kernels' work counter
 constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA on sm_100
 // Hidden states of one rasterisation block of the projection kernel: small enough to stay L2-resident next to the
 // weight tiles streaming past (data read by all SMs ends up in both halves of the 126 MB L2).
 constexpr size_t kHiddenBlockBytes = 36u << 20;
-constexpr size_t kHmmTableSmemLimit = 96 * 1024;   // exp'd HMM transition tables kept in shared memory up to this size
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
@@ -305,20 +305,14 @@ int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cuda
   // kernels that stream per-position tables hand out windows through a counter next to the status word
   unsigned* counter = at<unsigned>(h, L.off_status) + kWorkCounterWord;
   const int resident = blocks < 8 * h->num_sms ? blocks : 8 * h->num_sms;   // more CTAs than an SM can hold do no harm
-  if (c.family == MTPC_BTREE || is_ctx(h)) {
+  if (c.family == MTPC_BTREE || c.family == MTPC_HMM) {
     if (cudaMemsetAsync(counter, 0, sizeof(unsigned), st) != cudaSuccess) return MTPC_ERR_CUDA;
   }
   if (c.family == MTPC_CP) {
     circuit_cp_kernel<<<blocks, threads, 0, st>>>(G, logw, out, prefix, W, wpp, c.n, c.r, L.sum_rows);
-  } else if (c.family == MTPC_HMM && is_ctx(h)) {
-    circuit_hmm_ctx_kernel<<<resident, threads, hmm_ctx_smem_bytes(c.r), st>>>(G, logw, out, prefix, counter, W, wpp,
-                                                                              c.n, c.r, L.sum_rows);
   } else if (c.family == MTPC_HMM) {
-    const size_t table_bytes = static_cast<size_t>(c.n - 1) * c.r * c.r * 4;
-    const int in_smem = table_bytes <= kHmmTableSmemLimit;
-    const int cap = 4 * h->num_sms;                      // CTAs stride over the windows: the tables are staged once each
-    circuit_hmm_kernel<<<blocks < cap ? blocks : cap, threads, in_smem ? table_bytes : 0, st>>>(
-        G, logw, hmm_tables(h), out, prefix, W, wpp, c.n, c.r, L.sum_rows, in_smem, hmm_table_stride(h));
+    circuit_hmm_stream_kernel<<<resident, threads, hmm_ctx_smem_bytes(c.r), st>>>(
+        G, logw, hmm_tables(h), hmm_table_stride(h), out, prefix, counter, W, wpp, c.n, c.r, L.sum_rows);
   } else if (prefix != nullptr) {
     circuit_btree_kernel<true><<<resident, threads, btree_smem_bytes(c.n, c.r, true), st>>>(
         G, logw, out, prefix, counter, W, wpp, c.n, c.r, L.sum_rows);
@@ -334,11 +328,8 @@ int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cuda
 // point) sets them to what it needs or more.
 bool set_circuit_attributes(const mtpc_config& c) {
   bool fail = false;
-  if (c.family == MTPC_HMM)
-    fail |= cudaFuncSetAttribute(circuit_hmm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kHmmTableSmemLimit)) != cudaSuccess;
   if (c.family == MTPC_HMM && hmm_ctx_smem_bytes(c.r) > 48 * 1024)
-    fail |= cudaFuncSetAttribute(circuit_hmm_ctx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    fail |= cudaFuncSetAttribute(circuit_hmm_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(hmm_ctx_smem_bytes(c.r))) != cudaSuccess;
   if (c.family == MTPC_BTREE) {
     const int plain = static_cast<int>(btree_smem_bytes(c.n, c.r, false));
@@ -462,10 +453,18 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
     pt.end();
     if (rc != MTPC_OK) return rc;
     pt.begin();
-    draft_slot_kernel<<<dim3(c.n, P), kSlotThreads, 2 * c.r * sizeof(float), st>>>(
-        c.family, at<float>(h, L.off_logits), at<float>(h, L.off_logw), hmm_tables(h), uniforms, out_bytes,
-        at<float>(h, L.off_G), at<float>(h, L.off_unit_lse), at<unsigned>(h, L.off_status), wpp, c.n, c.r, c.v,
-        L.sum_rows, hmm_table_stride(h));
+    {
+      int chain = 0;                                       // longest chain of latent-draw tables of any slot
+      if (c.family == MTPC_HMM) chain = c.n - 1;
+      if (c.family == MTPC_BTREE) { for (int m = c.n; m > 2; m >>= 1) ++chain; }
+      const size_t base = static_cast<size_t>((2 * c.r + 3) & ~3) * sizeof(float);
+      const size_t with_tables = base + static_cast<size_t>(chain) * c.r * c.r * sizeof(float);
+      const int in_smem = chain > 0 && with_tables <= kSlotSmemLimit;
+      draft_slot_kernel<<<dim3(c.n, P), kSlotThreads, in_smem ? with_tables : base, st>>>(
+          c.family, at<float>(h, L.off_logits), at<float>(h, L.off_logw), hmm_tables(h), uniforms, out_bytes,
+          at<float>(h, L.off_G), at<float>(h, L.off_unit_lse), at<unsigned>(h, L.off_status), wpp, c.n, c.r, c.v,
+          L.sum_rows, hmm_table_stride(h), in_smem);
+    }
     h->launches++;
     h->draft_P = P;
     pt.end();
@@ -552,6 +551,8 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
                                kSmemLimit) != cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
           cudaSuccess;
+  fail |= cudaFuncSetAttribute(draft_slot_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               static_cast<int>(kSlotSmemLimit)) != cudaSuccess;
   fail |= !set_circuit_attributes(*cfg);
   {
     const size_t smem = kAcceptWarps * accept_warp_floats(cfg->family, cfg->n, cfg->r, cfg->v) * sizeof(float);

@@ -85,58 +85,6 @@ __global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __re
   if (lane == 0) out[w] = m + __logf(s);
 }
 
-// Eq. (HMM), forward recursion over the window: alpha_0[k] = log pi[k] + G[0,k];
-// alpha_i[k] = G[i,k] + LSE_a(alpha_{i-1}[a] + logA[i-1][a][k]); out = LSE_k alpha_{n-1}[k].  r <= 32.
-// The inner log-sum-exp is taken as one scaled matrix-vector product per step: with m = max_a alpha_{i-1}[a],
-// alpha_i[k] = G[i,k] + m + log sum_a exp(alpha_{i-1}[a] - m) A[i-1][a][k], A = exp(logA) staged once per CTA in
-// shared memory ((n-1) r^2 floats; read straight from global memory when that does not fit). One warp per
-// window, lane = state; CTAs stride over the windows. With `prefix` (may be NULL) the kernel also writes
-// prefix[w, i] = log q(x_0..x_i) = LSE_k alpha_i[k]. Contextual transitions (App. H): logA = log omega + r and
-// logA_stride = sum_rows, so that position p reads its own tables (never staged: tables_in_smem = 0).
-__global__ void circuit_hmm_kernel(const float* __restrict__ G, const float* __restrict__ logw,
-                                   const float* __restrict__ logA, float* __restrict__ out,
-                                   float* __restrict__ prefix, int W, int wpp, int n, int r, int sum_rows,
-                                   int tables_in_smem, int logA_stride) {
-  extern __shared__ float A_lin[];
-  const int lane = threadIdx.x & 31;
-  const int count = (n - 1) * r * r;
-  if (tables_in_smem) {
-    for (int e = threadIdx.x; e < count; e += blockDim.x) A_lin[e] = __expf(__ldg(logA + e));
-    __syncthreads();
-  }
-  const bool has = lane < r;
-  for (int w = blockIdx.x * kCircuitWarps + (threadIdx.x >> 5); w < W; w += gridDim.x * kCircuitWarps) {
-    const float* g = G + static_cast<size_t>(w) * n * r;
-    const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
-    float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
-    for (int i = 1; i < n; ++i) {
-      if (prefix != nullptr) {   // log q(x_0..x_{i-1}) = LSE_k alpha_{i-1}[k]: the later steps sum to one
-        const float pre = warp_lse(alpha, has);
-        if (lane == 0) prefix[static_cast<size_t>(w) * n + i - 1] = pre;
-      }
-      const float gi = has ? g[i * r + lane] : 0.f;
-      float m = alpha;                                   // fmaxf drops NaNs; they come back through e below
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
-      const float e = has ? __expf(alpha - m) : 0.f;     // NaN if alpha is NaN or if every state is impossible
-      float s = 0.f;
-      if (tables_in_smem) {
-        const float* A = A_lin + static_cast<size_t>(i - 1) * r * r;
-        for (int a = 0; a < r; ++a) s = fmaf(__shfl_sync(kFull, e, a), has ? A[a * r + lane] : 0.f, s);
-      } else {
-        const float* A = logA + static_cast<size_t>(w / wpp) * logA_stride + static_cast<size_t>(i - 1) * r * r;
-        for (int a = 0; a < r; ++a) s = fmaf(__shfl_sync(kFull, e, a), has ? __expf(__ldg(A + a * r + lane)) : 0.f, s);
-      }
-      if (has) alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : gi + m + __logf(s);
-    }
-    const float res = warp_lse(alpha, has);
-    if (lane == 0) {
-      if (out != nullptr) out[w] = res;
-      if (prefix != nullptr) prefix[static_cast<size_t>(w) * n + n - 1] = res;
-    }
-  }
-}
-
 // Eq. (BTree), bottom-up over the heap-ordered latent tree. Node j >= 1 has the table
 // logOmega_j[a][b] = logw[p, r + (j-1) r^2 + a r + b] (parent's value a, own value b); the deepest internal node
 // n/2-1+m multiplies the input units of tokens 2m and 2m+1. prod[j][z] is the product unit under z_j = z.
@@ -333,14 +281,20 @@ __global__ void circuit_btree_kernel(const float* __restrict__ G, const float* _
   }
 }
 
-// Eq. (HMM) with contextual transitions (App. H): position p = w / wpp has its own tables
-// logA_i[a][k] = logw[p, r + (i-1) r^2 + a r + k], 28 KB per position at n = 8, r = 32, read exactly once: the kernel is
-// bound by that stream from HBM. One warp per window, lane = state; table i+1 is copied into shared memory by
-// cp.async while table i is reduced. Same recursion and same scaled matrix-vector form as circuit_hmm_kernel.
+// Eq. (HMM), forward recursion over the window: alpha_0[k] = log pi[k] + G[0,k];
+// alpha_i[k] = G[i,k] + LSE_a(alpha_{i-1}[a] + logA_i[a][k]); out = LSE_k alpha_{n-1}[k].  r <= 32.
+// The inner log-sum-exp is taken as one scaled matrix-vector product per step: with m = max_a alpha_{i-1}[a],
+// alpha_i[k] = G[i,k] + m + log sum_a exp(alpha_{i-1}[a] - m) exp(logA_i[a][k]).
+// The transition tables are streamed per window: position p = w / wpp reads logA_i[a][k] at
+// tables[p * table_stride + (i-1) r^2 + a r + k]. Contextual transitions (App. H): tables = log omega + r and
+// table_stride = sum_rows, 28 KB per position at n = 8, r = 32, read exactly once from HBM, which bounds the kernel.
+// Static transitions: table_stride = 0, the one set of tables stays in L2. One warp per window, lane = state; table
+// i+1 is copied into shared memory by cp.async while table i is reduced.
 // Shared memory per warp: 2 * r * r + 32 floats. With `prefix` (may be NULL) also writes prefix[w, i] = LSE_k alpha_i[k].
-__global__ void circuit_hmm_ctx_kernel(const float* __restrict__ G, const float* __restrict__ logw,
-                                       float* __restrict__ out, float* __restrict__ prefix, unsigned* work_counter,
-                                       int W, int wpp, int n, int r, int sum_rows) {
+__global__ void circuit_hmm_stream_kernel(const float* __restrict__ G, const float* __restrict__ logw,
+                                          const float* __restrict__ tables, int table_stride,
+                                          float* __restrict__ out, float* __restrict__ prefix, unsigned* work_counter,
+                                          int W, int wpp, int n, int r, int sum_rows) {
   extern __shared__ __align__(16) float sm[];
   const int lane = threadIdx.x & 31;
   const int rr = r * r;
@@ -350,11 +304,12 @@ __global__ void circuit_hmm_ctx_kernel(const float* __restrict__ G, const float*
   for (int w = next_window(work_counter, lane); w < W; w = next_window(work_counter, lane)) {
     const float* g = G + static_cast<size_t>(w) * n * r;
     const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
-    if (n > 1) warp_table_load_async(tabs, lw + r, rr, lane);
+    const float* tb = tables + static_cast<size_t>(w / wpp) * table_stride;   // logA_1 .. logA_{n-1} of this position
+    if (n > 1) warp_table_load_async(tabs, tb, rr, lane);
     float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
     for (int i = 1; i < n; ++i) {
       if (i + 1 < n) {
-        warp_table_load_async(tabs + (i & 1) * rr, lw + r + static_cast<size_t>(i) * rr, rr, lane);
+        warp_table_load_async(tabs + (i & 1) * rr, tb + static_cast<size_t>(i) * rr, rr, lane);
         cp_async_wait<1>();
       } else {
         cp_async_wait<0>();

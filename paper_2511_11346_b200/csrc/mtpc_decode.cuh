@@ -25,7 +25,7 @@ namespace mtpc {
 
 constexpr int kDecodeMaxP = 128;                   // positions per call on this path
 constexpr int kDecodeMaxTiles = 3;                 // weight tiles that share one copy of the hidden states
-constexpr int kSlotThreads = 256;
+constexpr int kSlotThreads = 512;
 
 struct DecodeParams {
   CUtensorMap tm_h;      // hidden [P, d]       box 64 x Ppad
@@ -270,58 +270,82 @@ __device__ __forceinline__ int warp_inv_cdf_logp(float logp, int r, float u, int
   return hit ? __ffs(hit) - 1 : r - 1;
 }
 
-// Latent draws of one window down to the unit that owns slot i (Algorithm 1 at the sum units); the whole warp
-// calls it. CP: the mixture component. HMM: the chain z_0 .. z_i. BTree: the path from the root to the
-// deepest internal node above token i. Returns -1 if a uniform the window's latent draws use is outside [0,1).
-__device__ __forceinline__ int warp_sample_unit(int family, const float* __restrict__ lw, const float* __restrict__ logA,
-                                                const float* __restrict__ u, int n, int r, int i, int lane) {
-  const int nlat = (family == 0) ? 1 : (family == 1 ? n : n - 1);
-  bool bad = false;
-  for (int c = lane; c < nlat; c += 32) bad |= !(u[c] >= 0.f && u[c] < 1.f);
-  if (__any_sync(kFull, bad)) return -1;
-  int z = warp_inv_cdf_logp(lane < r ? lw[lane] : 0.f, r, u[0], lane);
-  if (family == 1) {
-    for (int s = 1; s <= i; ++s)
-      z = warp_inv_cdf_logp(lane < r ? logA[(static_cast<size_t>(s - 1) * r + z) * r + lane] : 0.f, r, u[s], lane);
-  } else if (family == 2) {
-    // heap path root -> owner node n/2 - 1 + i/2, top-down: the bits of (owner + 1) below its leading one
-    const int owner = n / 2 - 1 + (i >> 1);
-    const int code = owner + 1;
-    const int depth = 31 - __clz(code);
-    int node = 0;
-    for (int lvl = depth - 1; lvl >= 0; --lvl) {
-      node = 2 * node + 1 + ((code >> lvl) & 1);
-      z = warp_inv_cdf_logp(lane < r ? lw[r + (static_cast<size_t>(node - 1) * r + z) * r + lane] : 0.f, r, u[node], lane);
-    }
-  }
-  return z;
+// Tables the latent draws of slot i walk through (Algorithm 1 at the sum units), in the order they are used.
+// CP: none. HMM: the transitions into steps 1..i. BTree: the nodes on the path from the root (exclusive) down to
+// the deepest internal node above token i.
+__device__ __forceinline__ int slot_chain_length(int family, int n, int i) {
+  if (family == 1) return i;
+  if (family == 2) return 31 - __clz(n / 2 + (i >> 1));   // depth of the owner node n/2 - 1 + i/2 in heap order
+  return 0;
+}
+// Global address of table `step` (0-based) of the chain. lw: this position's log omega; hmm: this position's
+// (or the static) transition tables [n-1, r, r].
+__device__ __forceinline__ const float* slot_chain_table(int family, const float* lw, const float* hmm, int n, int r,
+                                                         int i, int step) {
+  if (family == 1) return hmm + static_cast<size_t>(step) * r * r;
+  const int code = n / 2 + (i >> 1);                       // owner + 1
+  const int depth = 31 - __clz(code);
+  const int node = (code >> (depth - 1 - step)) - 1;       // path node at level step + 1
+  return lw + r + static_cast<size_t>(node - 1) * r * r;
 }
 
 // logA: HMM transition log-probabilities [n-1, r, r]; position p reads them at logA + p * logA_stride (stride 0:
 // one static set for all positions; stride sum_rows with logA = log omega + r: contextual tables, App. H).
-// grid = (n, P). Shared memory: 2 * r floats (max and log-sum-exp of each unit of the slot). The log-sum-exps also
-// go to unit_lse_out [P, n, r], so that later calls can turn the retained logits into log phi.
+// grid = (n, P), 16 warps. Shared memory: 2 * r floats (max and log-sum-exp of each unit of the slot), then, when
+// tables_in_smem, the chain's tables (slot_chain_length * r * r floats), fetched by cp.async while the log-sum-exps
+// are computed, so that the data-dependent row reads of the latent draws do not each cost a trip to L2.
+// The log-sum-exps also go to unit_lse_out [P, n, r], so that later calls can turn the retained logits into log phi.
+constexpr int kSlotMaxPerLane = 16;   // v <= 512
 __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     int family, const float* __restrict__ logits, const float* __restrict__ logw, const float* __restrict__ logA,
     const float* __restrict__ uniforms, int* __restrict__ out_bytes, float* __restrict__ G,
-    float* __restrict__ unit_lse_out, unsigned* status, int wpp, int n, int r, int v, int sum_rows, int logA_stride) {
-  extern __shared__ float sm[];
+    float* __restrict__ unit_lse_out, unsigned* status, int wpp, int n, int r, int v, int sum_rows, int logA_stride,
+    int tables_in_smem) {
+  extern __shared__ __align__(16) float sm[];
   float* unit_max = sm;
   float* unit_lse = sm + r;
+  float* tabs = sm + ((2 * r + 3) & ~3);
   const int i = blockIdx.x;
   const int pos = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nwarps = kSlotThreads / 32;
+  const int rr = r * r;
   const float* row = logits + (static_cast<size_t>(pos) * n + i) * r * v;   // [r, v] logits of this slot
+  const float* lw = logw + static_cast<size_t>(pos) * sum_rows;
+  const float* hmm = logA + static_cast<size_t>(pos) * logA_stride;
+  const int chain = slot_chain_length(family, n, i);
 
+  if (tables_in_smem) {
+    for (int step = 0; step < chain; ++step) {
+      const float* src = slot_chain_table(family, lw, hmm, n, r, i, step);
+      float* dst = tabs + step * rr;
+      const bool vec = (rr & 3) == 0 && ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u) == 0;
+      if (vec) {
+        for (int e = threadIdx.x * 4; e < rr; e += kSlotThreads * 4) cp_async_16(dst + e, src + e);
+      } else {
+        for (int e = threadIdx.x; e < rr; e += kSlotThreads) cp_async_4(dst + e, src + e);
+      }
+    }
+    cp_async_commit();
+  }
+
+  // ---- log-sum-exp of every input unit of the slot: a lane's logits are fetched in one batch of independent loads
   for (int k = warp; k < r; k += nwarps) {
     const float* x = row + static_cast<size_t>(k) * v;
-    float m = -CUDART_INF_F;
-    for (int b = lane; b < v; b += 32) m = fmaxf(m, x[b]);
+    float xv[kSlotMaxPerLane];
+#pragma unroll
+    for (int q = 0; q < kSlotMaxPerLane; ++q) {
+      const int b = lane + 32 * q;
+      xv[q] = b < v ? x[b] : -CUDART_INF_F;
+    }
+    float m = xv[0];
+#pragma unroll
+    for (int q = 1; q < kSlotMaxPerLane; ++q) m = fmaxf(m, xv[q]);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
     float s = 0.f;
-    for (int b = lane; b < v; b += 32) s += __expf(x[b] - m);
+#pragma unroll
+    for (int q = 0; q < kSlotMaxPerLane; ++q) s += __expf(xv[q] - m);   // padding: exp(-inf) = 0
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(kFull, s, off);
     if (lane == 0) {
@@ -330,26 +354,50 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
       unit_lse_out[(static_cast<size_t>(pos) * n + i) * r + k] = unit_lse[k];   // kept for the acceptance stage
     }
   }
+  if (tables_in_smem) cp_async_wait<0>();
   __syncthreads();
 
-  const float* lw = logw + static_cast<size_t>(pos) * sum_rows;
-  const int per = (v + 31) / 32;   // consecutive bytes per lane in the CDF scan
+  const int per = (v + 31) / 32;   // consecutive bytes per lane in the CDF scan (<= kSlotMaxPerLane)
+  const int nlat = (family == 0) ? 1 : (family == 1 ? n : n - 1);
   for (int j = warp; j < wpp; j += nwarps) {
     const size_t w = static_cast<size_t>(pos) * wpp + j;
     const float* u = uniforms + w * 2 * n;
-    const int z = warp_sample_unit(family, lw, logA + static_cast<size_t>(pos) * logA_stride, u, n, r, i, lane);
     const float ub = u[n + i];
+    // ---- latent draws down to the unit that owns slot i; every uniform the window's latent draws use is checked
+    bool bad = false;
+    for (int c = lane; c < nlat; c += 32) bad |= !(u[c] >= 0.f && u[c] < 1.f);
+    bad = __any_sync(kFull, bad) || !(ub >= 0.f && ub < 1.f);
     int byte = -1;
-    if (z < 0 || !(ub >= 0.f && ub < 1.f)) {
+    if (bad) {
       if (lane == 0) atomicOr(status, 2u);
     } else {
-      // inverse CDF over the v bytes of unit z: lane l owns bytes [l*per, (l+1)*per)
+      int z = warp_inv_cdf_logp(lane < r ? lw[lane] : 0.f, r, u[0], lane);
+      if (family == 1) {
+        for (int st = 0; st < chain; ++st) {
+          const float* tab = tables_in_smem ? tabs + st * rr : hmm + static_cast<size_t>(st) * rr;
+          z = warp_inv_cdf_logp(lane < r ? tab[z * r + lane] : 0.f, r, u[st + 1], lane);
+        }
+      } else if (family == 2) {
+        const int code = n / 2 + (i >> 1);
+        for (int st = 0; st < chain; ++st) {
+          const int node = (code >> (chain - 1 - st)) - 1;
+          const float* tab = tables_in_smem ? tabs + st * rr : lw + r + static_cast<size_t>(node - 1) * rr;
+          z = warp_inv_cdf_logp(lane < r ? tab[z * r + lane] : 0.f, r, u[node], lane);
+        }
+      }
+      // ---- inverse CDF over the v bytes of unit z: lane l owns bytes [l*per, (l+1)*per)
       const float* x = row + static_cast<size_t>(z) * v;
       const float m = unit_max[z];
       const int b0 = lane * per;
+      float ev[kSlotMaxPerLane];
+#pragma unroll
+      for (int q = 0; q < kSlotMaxPerLane; ++q) ev[q] = (q < per && b0 + q < v) ? x[b0 + q] : -CUDART_INF_F;
       float part = 0.f;
-      for (int q = 0; q < per; ++q)
-        if (b0 + q < v) part += __expf(x[b0 + q] - m);
+#pragma unroll
+      for (int q = 0; q < kSlotMaxPerLane; ++q) {
+        ev[q] = __expf(ev[q] - m);
+        part += ev[q];
+      }
       const float incl = warp_scan_incl(part, lane);
       const float total = __shfl_sync(kFull, incl, 31);
       const float thr = ub * total;
@@ -361,9 +409,10 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
         const float before = __shfl_up_sync(kFull, incl, 1);
         if (lane == src) {
           float cum = lane == 0 ? 0.f : before;
-          for (int q = 0; q < per && found < 0; ++q)
-            if (b0 + q < v) {
-              cum += __expf(x[b0 + q] - m);
+#pragma unroll
+          for (int q = 0; q < kSlotMaxPerLane; ++q)
+            if (found < 0 && q < per && b0 + q < v) {
+              cum += ev[q];
               if (thr < cum) found = b0 + q;
             }
           if (found < 0) found = min(b0 + per, v) - 1;   // the lane's total passed the threshold: its last byte
