@@ -33,8 +33,8 @@ METRIC = "window_loglik_positions_per_s"
 UNIT = "positions/s"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one projection-kernel launch, from the ncu capture
-# summarised in profiles/ (captured at a quarter of the positions and scaled). None = not captured.
-NCU_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 5: None}
+# summarised in profiles/ (captured on the full configuration). None = not captured.
+NCU_TRAFFIC_BYTES = {1: 922_700_000, 2: None, 3: None, 5: None}   # configs[1]: mean of 925.1 and 920.3 MB (profiles/)
 
 
 def workload_name(idx: int, wl) -> str:

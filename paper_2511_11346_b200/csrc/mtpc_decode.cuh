@@ -465,7 +465,7 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
   const float* lw = logw + static_cast<size_t>(pos) * sum_rows;
   const bool has = lane < r;
 
-  // ---- 1. acceptance tests (every lane takes the same decisions on the same values)
+  // ---- 1. acceptance tests
   bool bad_u = false, bad_x = false;
   for (int c = lane; c <= n; c += 32) bad_u |= !(u[c] >= 0.f && u[c] < 1.f);
   for (int c = lane; c < n; c += 32) bad_x |= static_cast<unsigned>(x[c]) >= static_cast<unsigned>(v);
@@ -479,11 +479,17 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
     }
     return;
   }
-  int s = 0;
-  while (s < n) {
-    const float q = __expf(pre[s] - (s > 0 ? pre[s - 1] : 0.f));
-    if (u[s] * q > tp[static_cast<size_t>(s) * v + x[s]]) break;
-    ++s;
+  // lane i runs the test of byte i (all loads in flight at once); the first rejecting lane ends the accepted run
+  int s = n;
+  for (int base = 0; base < n && s == n; base += 32) {
+    const int i = base + lane;
+    bool rej = false;
+    if (i < n) {
+      const float q = __expf(pre[i] - (i > 0 ? pre[i - 1] : 0.f));
+      rej = u[i] * q > tp[static_cast<size_t>(i) * v + x[i]];
+    }
+    const unsigned m = __ballot_sync(kFull, rej);
+    if (m) s = base + __ffs(m) - 1;
   }
   if (lane == 0) out_accepted[w] = s;
   const float* trow = tp + static_cast<size_t>(s) * v;
