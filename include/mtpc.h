@@ -188,6 +188,32 @@ int mtpc_window_loss(mtpc_head* head, const void* hidden, const int32_t* targets
                      int32_t sequence_length, float gamma, float* out_slot_loss, float* out_loss, void* stream);
 
 /*
+ * Backward pass of the window log-likelihood (training, Sec. 4.1): gradients of
+ *     L = sum_t weight[t] * log q(x_{t,0..n-1} | h_t)
+ * through the circuit (Eq. CP / Eq. HMM / Eq. BTree), the softmaxes of Sec. 3.3 and the two projections.
+ * (weight[t] = -1/T gives the mean negative log-likelihood; a zero weight masks a position.)
+ *   hidden, targets, T   as for mtpc_window_logprob (a negative target is a marginalised byte: no gradient).
+ *   weight        dev [T] fp32.
+ *   bwd_workspace dev, 256-byte aligned, >= mtpc_backward_workspace_bytes(cfg, T): holds the units' log-sum-exps and
+ *                 posteriors, the bf16 gradient of the logits in both orientations (2 * T * n*r*v * 2 bytes: the one
+ *                 large buffer; the fp32 logits themselves are recomputed on chip and never stored) and transposed bf16
+ *                 copies of W_emit, W_sum and hidden. Caller-owned, used only during the call's work.
+ *   out_logprob   dev [T] fp32 or NULL: the forward value.
+ *   d_hidden      dev [T, d] fp32;  dW_emit dev [n, r, v, d] fp32;  dW_sum dev [S*r, d] fp32: overwritten, not
+ *                 accumulated.
+ *   dT_static     dev [n-1, r, r] fp32: gradient of the static transition logits (MTPC_HMM without the contextual
+ *                 flag; required there, ignored otherwise). With MTPC_FLAG_HMM_CONTEXTUAL the gradient of the bias is the
+ *                 column sum of the transition-logit gradients and is not returned separately.
+ * Arithmetic: posteriors in fp32; the logit gradients are rounded to bf16 (the operand type of the tensor cores) before
+ * the three weight-sized GEMMs, fp32 accumulation. dT_static is accumulated with atomic adds (order not fixed).
+ */
+int mtpc_backward_workspace_bytes(const mtpc_config* cfg, int32_t T, size_t* out_bytes);
+int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t T,
+                                 const float* weight, void* bwd_workspace, size_t bwd_workspace_bytes,
+                                 float* out_logprob, float* d_hidden, float* dW_emit, float* dW_sum, float* dT_static,
+                                 void* stream);
+
+/*
  * Host-buffer variants: same results, but hidden / targets / uniforms are HOST pointers (pinned memory for
  * full copy speed) and the outputs are written to HOST buffers. The copies to and from the device go through
  * staging areas in the workspace on `stream`; the call returns after the stream has been synchronised, so
@@ -214,6 +240,8 @@ int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags);
  *   mtpc_window_logprob: [0] projection GEMM + fused epilogue, [1] circuit evaluation.
  *   mtpc_window_prefix_logprob, mtpc_window_loss: as mtpc_window_logprob (the loss reduction is not timed).
  *   mtpc_speculative_accept: [0] the acceptance kernel.
+ *   mtpc_window_logprob_backward: [0] forward projection, [1] circuit backward, [2] projection in gradient mode,
+ *                        [3] transposes and the plain GEMMs.
  *   mtpc_draft_sample, mtpc_draft_sample_prefix:   P <= 128 positions and r <= 32: [0] one pass over all weights (logits of every unit),
  *                        [1] per-slot latent + byte draws and evidence, [2] circuit evaluation.
  *                        Otherwise: [0] sum-unit GEMM, [1] latent sampling, [2] GEMM + inverse-CDF epilogue,

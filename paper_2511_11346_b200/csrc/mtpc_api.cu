@@ -10,6 +10,7 @@
 #include <new>
 
 #include "../../include/mtpc.h"
+#include "mtpc_backward.cuh"
 #include "mtpc_circuit.cuh"
 #include "mtpc_decode.cuh"
 #include "mtpc_gemm.cuh"
@@ -159,13 +160,16 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 matrix [rows, cols] row-major -> tiles of box_rows x 64 elements, 128-byte swizzle, zero fill outside.
-int make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+// bf16 matrix [rows, cols] row-major (row pitch `pitch` elements, 0 = cols) -> tiles of box_rows x 64 elements,
+// 128-byte swizzle, zero fill outside.
+int make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint64_t pitch = 0) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return MTPC_ERR_CUDA;
   if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0) return MTPC_ERR_WORKSPACE;
+  if (pitch == 0) pitch = cols;
+  if ((pitch * 2) % 16 != 0) return MTPC_ERR_WORKSPACE;
   cuuint64_t gdim[2] = {cols, rows};
-  cuuint64_t gstride[1] = {cols * 2};
+  cuuint64_t gstride[1] = {pitch * 2};
   cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
@@ -234,14 +238,32 @@ struct PhaseTimer {
 int check_launch() { return cudaGetLastError() == cudaSuccess ? MTPC_OK : MTPC_ERR_CUDA; }
 
 // Launch the projection kernel for `rows` positions over the emission groups (with_emit) and / or the sum tiles.
+struct GradArgs {            // what the projection kernel needs beyond the forward arguments (backward pass only)
+  float* lse_out = nullptr;                  // forward for training: keep the units' log-sum-exps
+  const float* lse_in = nullptr;             // gradient mode
+  const float* post = nullptr;
+  __nv_bfloat16* dlogit = nullptr;
+  __nv_bfloat16* dlogit_t = nullptr;
+  size_t t_pitch = 0;
+};
+
 int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int wpp, bool with_emit, bool with_sum,
-                const int* targets, const float* uniforms, int* out_bytes, cudaStream_t st) {
+                const int* targets, const float* uniforms, int* out_bytes, cudaStream_t st,
+                const GradArgs* ga = nullptr) {
   if (rows <= 0 || (!with_emit && !with_sum)) return MTPC_OK;
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
   const Tiling& tl = mode == kModeSample ? L.sm : L.lp;
   GemmParams p;
   memset(&p, 0, sizeof(p));
+  if (ga) {
+    p.lse_out = ga->lse_out;
+    p.lse_in = ga->lse_in;
+    p.post = ga->post;
+    p.dlogit = ga->dlogit;
+    p.dlogit_t = ga->dlogit_t;
+    p.t_pitch = ga->t_pitch;
+  }
   int rc = make_tmap(&p.tm_a, hidden_bf16, static_cast<uint64_t>(rows), static_cast<uint64_t>(c.d), kBlockM);
   if (rc != MTPC_OK) return rc;
   p.tm_emit = mode == kModeSample ? h->tm_emit_sm : h->tm_emit_lp;
@@ -280,6 +302,8 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
   if (mode == kModeLogprob)
     mtpc_gemm_kernel<kModeLogprob><<<grid, kGemmThreads, tl.smem, st>>>(p);
+  else if (mode == kModeGrad)
+    mtpc_gemm_kernel<kModeGrad><<<grid, kGemmThreads, tl.smem, st>>>(p);
   else
     mtpc_gemm_kernel<kModeSample><<<grid, kGemmThreads, tl.smem, st>>>(p);
   h->launches++;
@@ -503,6 +527,98 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   return rc;
 }
 
+// ---------------------------------------------------------------- backward pass (host side)
+size_t round64(size_t x) { return (x + 63) / 64 * 64; }
+
+// Carving of the backward workspace for T positions (all buffers 256-byte aligned).
+struct BackwardLayout {
+  size_t Nc, Spad, Tpad;
+  size_t off_lse, off_post, off_dsum, off_dsum_t, off_dlogit, off_dlogit_t, off_wt, off_rt, off_ht, total;
+};
+void plan_backward(const mtpc_config& c, const Layout& L, int T, BackwardLayout* B) {
+  B->Nc = static_cast<size_t>(c.n) * c.r * c.v;
+  B->Spad = round64(L.sum_rows);
+  B->Tpad = round64(T);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  B->off_lse = take(static_cast<size_t>(T) * c.n * c.r * 4);
+  B->off_post = take(static_cast<size_t>(T) * c.n * c.r * 4);
+  B->off_dsum = take(static_cast<size_t>(T) * B->Spad * 2);          // [T, Spad] bf16
+  B->off_dsum_t = take(static_cast<size_t>(L.sum_rows) * B->Tpad * 2);  // [S r, Tpad]
+  B->off_dlogit = take(static_cast<size_t>(T) * B->Nc * 2);          // [T, Nc]
+  B->off_dlogit_t = take(B->Nc * B->Tpad * 2);                       // [Nc, Tpad]
+  B->off_wt = take(static_cast<size_t>(c.d) * B->Nc * 2);            // W_emit^T [d, Nc]
+  B->off_rt = take(static_cast<size_t>(c.d) * B->Spad * 2);          // W_sum^T  [d, Spad]
+  B->off_ht = take(static_cast<size_t>(c.d) * B->Tpad * 2);          // hidden^T [d, Tpad]
+  B->total = off;
+}
+
+int launch_transpose(mtpc_head* h, const void* src, void* dst, int rows, int cols, size_t src_pitch, size_t dst_pitch,
+                     cudaStream_t st) {
+  if (rows <= 0 || cols <= 0) return MTPC_OK;
+  dim3 grid((cols + 63) / 64, (rows + 63) / 64);
+  transpose_bf16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), static_cast<__nv_bfloat16*>(dst),
+                                              rows, cols, src_pitch, dst_pitch);
+  h->launches++;
+  return check_launch();
+}
+
+// C[M, N] fp32 (pitch ldc) = A[M, K] B[N, K]^T (+ C): A, B bf16 with K contiguous and row pitches lda, ldb (elements).
+int launch_plain_gemm(mtpc_head* h, const void* A, size_t lda, const void* Bm, size_t ldb, float* C, size_t ldc, int M,
+                      int N, int K, bool accumulate, cudaStream_t st) {
+  if (M <= 0 || N <= 0 || K <= 0) return MTPC_OK;
+  PlainGemmParams p;
+  memset(&p, 0, sizeof(p));
+  int rc = make_tmap(&p.tm_a, A, M, K, kBlockM, lda);
+  if (rc == MTPC_OK) rc = make_tmap(&p.tm_b, Bm, N, K, kPlainTileN, ldb);
+  if (rc != MTPC_OK) return rc;
+  p.M = M; p.N = N;
+  p.kblocks = (K + kBlockK - 1) / kBlockK;
+  p.m_tiles = (M + kBlockM - 1) / kBlockM;
+  p.n_tiles = (N + kPlainTileN - 1) / kPlainTileN;
+  p.stage_bytes = kABytes + kPlainTileN * kBlockK * 2;
+  const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
+  p.stages = (kSmemLimit - ctl) / p.stage_bytes;
+  if (p.stages > kMaxStages) p.stages = kMaxStages;
+  p.accumulate = accumulate ? 1 : 0;
+  p.C = C;
+  p.ldc = ldc;
+  p.status = at<unsigned>(h, h->L.off_status);
+  const long long items = static_cast<long long>(p.m_tiles) * p.n_tiles;
+  const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
+  plain_gemm_kernel<<<grid, kGemmThreads, p.stages * p.stage_bytes + ctl, st>>>(p);
+  h->launches++;
+  return check_launch();
+}
+
+int launch_circuit_backward(mtpc_head* h, int T, const int32_t* targets, const float* weight, float* out, float* post,
+                            __nv_bfloat16* dsum, int dsum_pitch, float* dT, cudaStream_t st) {
+  const mtpc_config& c = h->cfg;
+  const Layout& L = h->L;
+  const float* G = at<float>(h, L.off_G);
+  const float* logw = at<float>(h, L.off_logw);
+  unsigned* counter = at<unsigned>(h, L.off_status) + kWorkCounterWord;
+  const int blocks = (T + kCircuitWarps - 1) / kCircuitWarps;
+  const int threads = kCircuitWarps * 32;
+  const int resident = blocks < 8 * h->num_sms ? blocks : 8 * h->num_sms;
+  if (c.family != MTPC_CP && cudaMemsetAsync(counter, 0, sizeof(unsigned), st) != cudaSuccess) return MTPC_ERR_CUDA;
+  if (c.family == MTPC_CP) {
+    circuit_cp_backward_kernel<<<blocks, threads, 0, st>>>(G, logw, targets, weight, out, post, dsum, dsum_pitch, T, c.n,
+                                                          c.r, L.sum_rows);
+  } else if (c.family == MTPC_HMM) {
+    const size_t smem = hmm_backward_smem_floats(c.n, c.r, !is_ctx(h), kCircuitWarps) * sizeof(float);
+    circuit_hmm_backward_kernel<<<resident, threads, smem, st>>>(G, logw, hmm_tables(h), hmm_table_stride(h), targets,
+                                                                weight, out, post, dsum, dsum_pitch, dT, counter, T,
+                                                                c.n, c.r, L.sum_rows);
+  } else {
+    const size_t smem = kCircuitWarps * btree_backward_warp_floats(c.n, c.r) * sizeof(float);
+    circuit_btree_backward_kernel<<<resident, threads, smem, st>>>(G, logw, targets, weight, out, post, dsum, dsum_pitch,
+                                                                  counter, T, c.n, c.r, L.sum_rows);
+  }
+  h->launches++;
+  return check_launch();
+}
+
 int check_call(mtpc_head* h, int32_t rows) {
   if (!h) return MTPC_ERR_NULL;
   if (rows < 0 || rows > h->cfg.max_positions) return MTPC_ERR_SHAPE;
@@ -549,6 +665,10 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
                                kSmemLimit) != cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeSample>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
+  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeGrad>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               kSmemLimit) != cudaSuccess;
+  fail |= cudaFuncSetAttribute(plain_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
+          cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
           cudaSuccess;
   fail |= cudaFuncSetAttribute(draft_slot_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -689,6 +809,112 @@ int mtpc_window_loss(mtpc_head* head, const void* hidden, const int32_t* targets
   loss_final_kernel<<<1, kLossThreads, 0, st>>>(partial, out_slot_loss, out_loss, num_sequences, head->cfg.n, gamma);
   head->launches += 2;
   return check_launch();
+}
+
+int mtpc_backward_workspace_bytes(const mtpc_config* cfg, int32_t T, size_t* out_bytes) {
+  if (!cfg || !out_bytes) return MTPC_ERR_NULL;
+  if (T < 1) return MTPC_ERR_SHAPE;
+  Layout L;
+  int rc = plan(*cfg, &L);
+  if (rc != MTPC_OK) return rc;
+  BackwardLayout B;
+  plan_backward(*cfg, L, T, &B);
+  *out_bytes = B.total;
+  return MTPC_OK;
+}
+
+int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t T,
+                                 const float* weight, void* bwd_workspace, size_t bwd_workspace_bytes,
+                                 float* out_logprob, float* d_hidden, float* dW_emit, float* dW_sum, float* dT_static,
+                                 void* stream) {
+  int rc = check_call(head, T);
+  if (rc != MTPC_OK) return rc;
+  if (T == 0) return MTPC_OK;
+  if (!hidden || !targets || !weight || !bwd_workspace || !d_hidden || !dW_emit || !dW_sum) return MTPC_ERR_NULL;
+  const mtpc_config& c = head->cfg;
+  const Layout& L = head->L;
+  const bool static_hmm = c.family == MTPC_HMM && !is_ctx(head) && c.n > 1;
+  if (static_hmm && !dT_static) return MTPC_ERR_NULL;
+  BackwardLayout B;
+  plan_backward(c, L, T, &B);
+  if (bwd_workspace_bytes < B.total || (reinterpret_cast<uintptr_t>(bwd_workspace) % kAlign) != 0)
+    return MTPC_ERR_WORKSPACE;
+  // shared-memory sizes of the circuit backward kernels (per function, set to what this head needs)
+  {
+    bool fail = false;
+    if (c.family == MTPC_HMM) {
+      const size_t smem = hmm_backward_smem_floats(c.n, c.r, !is_ctx(head), kCircuitWarps) * sizeof(float);
+      if (smem > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;
+      if (smem > 48 * 1024)
+        fail |= cudaFuncSetAttribute(circuit_hmm_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(smem)) != cudaSuccess;
+    } else if (c.family == MTPC_BTREE) {
+      const size_t smem = kCircuitWarps * btree_backward_warp_floats(c.n, c.r) * sizeof(float);
+      if (smem > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;
+      if (smem > 48 * 1024)
+        fail |= cudaFuncSetAttribute(circuit_btree_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(smem)) != cudaSuccess;
+    }
+    if (fail) return MTPC_ERR_CUDA;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* bw = static_cast<uint8_t*>(bwd_workspace);
+  float* lse = reinterpret_cast<float*>(bw + B.off_lse);
+  float* post = reinterpret_cast<float*>(bw + B.off_post);
+  __nv_bfloat16* dsum = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dsum);
+  __nv_bfloat16* dsum_t = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dsum_t);
+  __nv_bfloat16* dlogit = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit);
+  __nv_bfloat16* dlogit_t = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit_t);
+  void* wt = bw + B.off_wt;
+  void* rt = bw + B.off_rt;
+  void* ht = bw + B.off_ht;
+  const int Nc = static_cast<int>(B.Nc);
+
+  const void* hb = nullptr;
+  head->draft_P = 0;
+  rc = stage_hidden(head, hidden, T, &hb, st);
+  if (rc != MTPC_OK) return rc;
+  PhaseTimer pt(head, st);
+  // 1. forward projection, keeping the units' log-sum-exps
+  pt.begin();
+  GradArgs fwd;
+  fwd.lse_out = lse;
+  rc = launch_gemm(head, kModeLogprob, hb, T, 1, true, true, targets, nullptr, nullptr, st, &fwd);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  // 2. circuit backward: posteriors of the input units and of the sum units
+  pt.begin();
+  bool bad = false;
+  if (static_hmm) bad |= cudaMemsetAsync(dT_static, 0, static_cast<size_t>(c.n - 1) * c.r * c.r * 4, st) != cudaSuccess;
+  if (bad) return MTPC_ERR_CUDA;
+  rc = launch_circuit_backward(head, T, targets, weight, out_logprob, post, dsum, static_cast<int>(B.Spad), dT_static, st);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  // 3. logits recomputed, turned into their gradient (bf16, both orientations)
+  pt.begin();
+  GradArgs ga;
+  ga.lse_in = lse;
+  ga.post = post;
+  ga.dlogit = dlogit;
+  ga.dlogit_t = dlogit_t;
+  ga.t_pitch = B.Tpad;
+  rc = launch_gemm(head, kModeGrad, hb, T, 1, true, false, targets, nullptr, nullptr, st, &ga);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  // 4. transposed operands, then the plain GEMMs
+  pt.begin();
+  rc = launch_transpose(head, head->W_emit_bf16, wt, Nc, c.d, c.d, B.Nc, st);
+  if (rc == MTPC_OK) rc = launch_transpose(head, head->W_sum_bf16, rt, L.sum_rows, c.d, c.d, B.Spad, st);
+  if (rc == MTPC_OK) rc = launch_transpose(head, hb, ht, T, c.d, c.d, B.Tpad, st);
+  if (rc == MTPC_OK) rc = launch_transpose(head, dsum, dsum_t, T, L.sum_rows, B.Spad, B.Tpad, st);
+  // d hidden [T, d] = dlogit [T, Nc] W_emit [Nc, d] + dsum [T, S r] W_sum [S r, d]
+  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dlogit, B.Nc, wt, B.Nc, d_hidden, c.d, T, c.d, Nc, false, st);
+  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dsum, B.Spad, rt, B.Spad, d_hidden, c.d, T, c.d, L.sum_rows, true, st);
+  // dW_emit [Nc, d] = dlogit^T [Nc, T] hidden [T, d];  dW_sum [S r, d] = dsum^T [S r, T] hidden [T, d]
+  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dlogit_t, B.Tpad, ht, B.Tpad, dW_emit, c.d, Nc, c.d, T, false, st);
+  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dsum_t, B.Tpad, ht, B.Tpad, dW_sum, c.d, L.sum_rows, c.d, T, false, st);
+  pt.end();
+  return rc;
 }
 
 int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int32_t* targets_host, int32_t T,

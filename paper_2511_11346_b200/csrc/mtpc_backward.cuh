@@ -1,0 +1,483 @@
+// Backward pass of the window log-likelihood (training, Sec. 4.1 / Eq. 6): gradient of
+//     L = sum_t weight[t] * log q(x_t | h_t)
+// with respect to the hidden states, the emission weights, the sum-unit weights and the static transition logits.
+//
+// Stages (host side in mtpc_api.cu):
+//   1. forward projection kernel, also saving the log-sum-exp of every input unit (lse [T, n, r]);
+//   2. circuit backward (this file): one warp per window runs the upward and the downward pass of the circuit and
+//      writes post[w, i, k] = weight * d log q / d G[w, i, k] (the posterior of "token i is emitted by unit k") and
+//      dsum[w, :] = weight * d log q / d (sum-unit logits), i.e. posterior minus prior of every sum unit, in bf16;
+//   3. the projection kernel once more in gradient mode: logits are recomputed tile by tile in tensor memory and turned
+//      into dlogit = post * (onehot(target) - softmax) in the epilogue, written as bf16 in both orientations;
+//   4. plain bf16 GEMMs (plain_gemm_kernel, this file) on those: d hidden = dlogit W + dsum R, dW = dlogit^T h,
+//      dR = dsum^T h. The [T, n, r, v] fp32 logit tensor still never exists; its bf16 gradient does, as the operand of
+//      the two weight-sized GEMMs.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "mtpc_circuit.cuh"
+#include "mtpc_gemm.cuh"
+
+namespace mtpc {
+
+// ---------------------------------------------------------------- circuit backward: mixture (Eq. CP)
+// log q = LSE_k a_k, a_k = log omega_k + sum_i G[i, k]:  d log q / d a_k = rho_k = softmax(a)_k for every slot and for
+// the mixture weight; through the softmax of the mixture logits: rho_k - omega_k.
+__global__ void circuit_cp_backward_kernel(const float* __restrict__ G, const float* __restrict__ logw,
+                                           const int* __restrict__ targets, const float* __restrict__ weight,
+                                           float* __restrict__ out, float* __restrict__ post,
+                                           __nv_bfloat16* __restrict__ dsum, int dsum_pitch, int W, int n, int r,
+                                           int sum_rows) {
+  const int w = blockIdx.x * kCircuitWarps + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (w >= W) return;
+  const float* g = G + static_cast<size_t>(w) * n * r;
+  const float* lw = logw + static_cast<size_t>(w) * sum_rows;
+  const float wt = weight[w];
+  float a[4];
+  float m = -CUDART_INF_F, s = 0.f;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int k = lane + 32 * q;
+    a[q] = -CUDART_INF_F;
+    if (k < r) {
+      a[q] = lw[k];
+      for (int i = 0; i < n; ++i) a[q] += g[i * r + k];
+      lse_merge(m, s, a[q], 1.f);
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float m2 = __shfl_xor_sync(kFull, m, off);
+    const float s2 = __shfl_xor_sync(kFull, s, off);
+    lse_merge(m, s, m2, s2);
+  }
+  const float logq = m + __logf(s);
+  if (lane == 0 && out != nullptr) out[w] = logq;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int k = lane + 32 * q;
+    if (k < r) {
+      const float rho = __expf(a[q] - logq);
+      for (int i = 0; i < n; ++i)
+        post[(static_cast<size_t>(w) * n + i) * r + k] = targets[static_cast<size_t>(w) * n + i] >= 0 ? wt * rho : 0.f;
+      dsum[static_cast<size_t>(w) * dsum_pitch + k] = __float2bfloat16_rn(wt * (rho - __expf(lw[k])));
+    }
+  }
+}
+
+// ---------------------------------------------------------------- circuit backward: HMM (Eq. HMM), forward-backward
+// Forward messages alpha_i (kept for all steps in shared memory), backward messages
+// beta_{i-1}[a] = LSE_b(logA_i[a][b] + G[i][b] + beta_i[b]). Posterior of the state: gamma_i = exp(alpha_i + beta_i - log q)
+// = d log q / d G[i, .]; pairwise posterior xi_i[a][b] = exp(alpha_{i-1}[a] + logA_i[a][b] + G[i][b] + beta_i[b] - log q)
+// = d log q / d logA_i[a][b]; through the row softmax of the transition logits: xi_i[a][b] - A_i[a][b] gamma_{i-1}[a].
+// Tables as in circuit_hmm_stream_kernel (static: stride 0; contextual: one set per position inside log omega).
+// Contextual: the transition-logit gradients go to dsum (bf16, one row per position). Static: they are summed over
+// the windows into dT [n-1, r, r] (fp32): per CTA in shared memory first, then one atomicAdd per entry and CTA.
+// Shared memory: per warp n*r (alpha) + 2*r*r (tables) + 32 floats; static: + (n-1)*r*r floats per CTA.  r <= 32.
+__host__ __device__ inline size_t hmm_backward_smem_floats(int n, int r, bool is_static, int warps) {
+  return static_cast<size_t>(warps) * (static_cast<size_t>(n) * r + 2 * r * r + 32) +
+         (is_static ? static_cast<size_t>(n - 1) * r * r : 0);
+}
+
+__global__ void circuit_hmm_backward_kernel(const float* __restrict__ G, const float* __restrict__ logw,
+                                            const float* __restrict__ tables, int table_stride,
+                                            const int* __restrict__ targets, const float* __restrict__ weight,
+                                            float* __restrict__ out, float* __restrict__ post,
+                                            __nv_bfloat16* __restrict__ dsum, int dsum_pitch, float* __restrict__ dT,
+                                            unsigned* work_counter, int W, int n, int r, int sum_rows) {
+  extern __shared__ __align__(16) float sm[];
+  const int lane = threadIdx.x & 31;
+  const int wib = threadIdx.x >> 5;
+  const int rr = r * r;
+  const bool is_static = table_stride == 0;
+  float* acc = sm;                                                       // static only: [n-1, r, r]
+  float* mine = sm + (is_static ? (n - 1) * rr : 0) + static_cast<size_t>(wib) * (n * r + 2 * rr + 32);
+  float* alphas = mine;                                                  // [n, r]
+  float* tabs = alphas + n * r;
+  float* cvec = tabs + 2 * rr;
+  const bool has = lane < r;
+  if (is_static) {
+    for (int e = threadIdx.x; e < (n - 1) * rr; e += blockDim.x) acc[e] = 0.f;
+    __syncthreads();
+  }
+  for (int w = next_window(work_counter, lane); w < W; w = next_window(work_counter, lane)) {
+    const float* g = G + static_cast<size_t>(w) * n * r;
+    const float* lw = logw + static_cast<size_t>(w) * sum_rows;
+    const float* tb = tables + static_cast<size_t>(w) * table_stride;
+    const float wt = weight[w];
+    // ---- forward, keeping every alpha_i
+    if (n > 1) warp_table_load_async(tabs, tb, rr, lane);
+    float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
+    if (has) alphas[lane] = alpha;
+    for (int i = 1; i < n; ++i) {
+      if (i + 1 < n) {
+        warp_table_load_async(tabs + (i & 1) * rr, tb + static_cast<size_t>(i) * rr, rr, lane);
+        cp_async_wait<1>();
+      } else {
+        cp_async_wait<0>();
+      }
+      __syncwarp();
+      const float* A = tabs + ((i - 1) & 1) * rr;
+      float m = alpha;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
+      cvec[lane] = has ? __expf(alpha - m) : 0.f;
+      __syncwarp();
+      if (has) {
+        float s = 0.f;
+        for (int a = 0; a < r; ++a) s = fmaf(cvec[a], __expf(A[a * r + lane]), s);
+        alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : g[i * r + lane] + m + __logf(s);
+        alphas[i * r + lane] = alpha;
+      }
+      __syncwarp();
+    }
+    const float logq = warp_lse(alpha, has);
+    if (lane == 0 && out != nullptr) out[w] = logq;
+    // ---- backward: tables in reverse order; table n-1 is still in its buffer
+    float beta = 0.f;                                                    // beta_{n-1}
+    for (int i = n - 1; i >= 1; --i) {
+      // table i (index i-1) sits in buffer (i-1)&1 if it was the last one loaded or was prefetched below
+      if (i < n - 1) {
+        cp_async_wait<0>();
+        __syncwarp();
+      }
+      if (i - 1 >= 1) warp_table_load_async(tabs + (i & 1) * rr, tb + static_cast<size_t>(i - 2) * rr, rr, lane);
+      const float* A = tabs + ((i - 1) & 1) * rr;
+      const bool valid = targets[static_cast<size_t>(w) * n + i] >= 0;
+      if (has) {
+        const float gamma = __expf(alphas[i * r + lane] + beta - logq);
+        post[(static_cast<size_t>(w) * n + i) * r + lane] = valid ? wt * gamma : 0.f;
+        cvec[lane] = g[i * r + lane] + beta;
+      }
+      __syncwarp();
+      const float beta_prev = sum_layer_staged(A, cvec, lane, r);        // lane a: LSE_b(logA[a][b] + c[b])
+      if (has) {
+        const float al = alphas[(i - 1) * r + lane];
+        const float gam_prev = __expf(al + beta_prev - logq);
+        const float* row = A + lane * r;
+        // the row is walked starting at column `lane` (r is a power of two): 32 lanes, 32 different banks
+        if (is_static) {
+          float* dst = acc + static_cast<size_t>(i - 1) * rr + lane * r;
+          for (int q = 0; q < r; ++q) {
+            const int b = (q + lane) & (r - 1);
+            const float la = row[b];
+            atomicAdd(dst + b, wt * (__expf(al + la + cvec[b] - logq) - __expf(la) * gam_prev));
+          }
+        } else {
+          __nv_bfloat16* dst = dsum + static_cast<size_t>(w) * dsum_pitch + r + static_cast<size_t>(i - 1) * rr + lane * r;
+          for (int q = 0; q < r; ++q) {
+            const int b = (q + lane) & (r - 1);
+            const float la = row[b];
+            dst[b] = __float2bfloat16_rn(wt * (__expf(al + la + cvec[b] - logq) - __expf(la) * gam_prev));
+          }
+        }
+      }
+      beta = beta_prev;
+      __syncwarp();                                                      // cvec and the table buffer are free again
+    }
+    if (has) {
+      const float gamma0 = __expf(alphas[lane] + beta - logq);
+      post[static_cast<size_t>(w) * n * r + lane] = targets[static_cast<size_t>(w) * n] >= 0 ? wt * gamma0 : 0.f;
+      dsum[static_cast<size_t>(w) * dsum_pitch + lane] = __float2bfloat16_rn(wt * (gamma0 - __expf(lw[lane])));
+    }
+    __syncwarp();
+  }
+  if (is_static) {
+    __syncthreads();
+    for (int e = threadIdx.x; e < (n - 1) * rr; e += blockDim.x) {
+      const float v = acc[e];
+      if (v != 0.f) atomicAdd(dT + e, v);
+    }
+  }
+}
+
+// ---------------------------------------------------------------- circuit backward: binary tree (Eq. BTree)
+// Upward pass as in circuit_btree_kernel (prod[j][z], S[c][z]); downward pass with U[j][z] = log-weight of everything
+// outside node j's subtree given z_j = z: U[0] = log omega_root, U[c][b] = LSE_z(U[j][z] + S[sibling][z] + logOmega_c[z][b]).
+// Posterior of a latent: gamma_j = exp(U[j] + prod[j] - log q); a token's evidence gradient is its owner's gamma.
+// Pairwise posterior xi_c[z][b] = exp(U[j][z] + S[sib][z] + logOmega_c[z][b] + prod[c][b] - log q); through the row
+// softmax: xi_c[z][b] - Omega_c[z][b] gamma_j[z]. The tables are streamed twice (up: deepest parents first; down: in
+// address order). Shared memory per warp: 3*(n-1)*r + 2*r*r + 32 floats.  r <= 32.
+__host__ __device__ inline size_t btree_backward_warp_floats(int n, int r) {
+  return 3 * static_cast<size_t>(n - 1) * r + 2 * static_cast<size_t>(r) * r + 32;
+}
+
+__global__ void circuit_btree_backward_kernel(const float* __restrict__ G, const float* __restrict__ logw,
+                                              const int* __restrict__ targets, const float* __restrict__ weight,
+                                              float* __restrict__ out, float* __restrict__ post,
+                                              __nv_bfloat16* __restrict__ dsum, int dsum_pitch, unsigned* work_counter,
+                                              int W, int n, int r, int sum_rows) {
+  extern __shared__ __align__(16) float sm[];
+  const int wib = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  float* prod = sm + static_cast<size_t>(wib) * btree_backward_warp_floats(n, r);
+  float* S = prod + (n - 1) * r;
+  float* U = S + (n - 1) * r;
+  float* tabs = U + (n - 1) * r;
+  float* cur = tabs + 2 * r * r;
+  const bool has = lane < r;
+  const int first_leaf_node = n / 2 - 1;
+  const int rr = r * r;
+  const int ntab = n - 2;
+  auto child_of = [&](int t) { return 2 * (first_leaf_node - 1 - (t >> 1)) + 1 + (t & 1); };
+  for (int w = next_window(work_counter, lane); w < W; w = next_window(work_counter, lane)) {
+    const float* g = G + static_cast<size_t>(w) * n * r;
+    const float* lw = logw + static_cast<size_t>(w) * sum_rows;
+    const float wt = weight[w];
+    __nv_bfloat16* ds = dsum + static_cast<size_t>(w) * dsum_pitch;
+    // ---- upward
+    if (ntab > 0) warp_table_load_async(tabs, lw + r + static_cast<size_t>(child_of(0) - 1) * rr, rr, lane);
+    for (int j = n - 2; j >= first_leaf_node; --j) {
+      const int m = j - first_leaf_node;
+      if (has) prod[j * r + lane] = g[(2 * m) * r + lane] + g[(2 * m + 1) * r + lane];
+    }
+    __syncwarp();
+    float acc = 0.f;
+    for (int t = 0; t < ntab; ++t) {
+      const int c = child_of(t);
+      if (t + 1 < ntab) {
+        warp_table_load_async(tabs + ((t + 1) & 1) * rr, lw + r + static_cast<size_t>(child_of(t + 1) - 1) * rr, rr, lane);
+        cp_async_wait<1>();
+      } else {
+        cp_async_wait<0>();
+      }
+      __syncwarp();
+      const float sc = sum_layer_staged(tabs + (t & 1) * rr, prod + c * r, lane, r);
+      if (has) S[c * r + lane] = sc;
+      acc += sc;
+      if (t & 1) {
+        if (has) prod[((c - 2) >> 1) * r + lane] = acc;
+        acc = 0.f;
+      }
+      __syncwarp();
+    }
+    const float logq = warp_lse(has ? lw[lane] + prod[lane] : 0.f, has);
+    if (lane == 0 && out != nullptr) out[w] = logq;
+    // ---- downward, children c = 1 .. n-2 in address order
+    if (has) {
+      U[lane] = lw[lane];
+      ds[lane] = __float2bfloat16_rn(wt * (__expf(lw[lane] + prod[lane] - logq) - __expf(lw[lane])));
+    }
+    if (ntab > 0) warp_table_load_async(tabs, lw + r, rr, lane);
+    __syncwarp();
+    for (int c = 1; c <= ntab; ++c) {
+      const int j = (c - 1) >> 1;
+      const int sib = (c & 1) ? c + 1 : c - 1;
+      if (c < ntab) {
+        warp_table_load_async(tabs + (c & 1) * rr, lw + r + static_cast<size_t>(c) * rr, rr, lane);
+        cp_async_wait<1>();
+      } else {
+        cp_async_wait<0>();
+      }
+      if (has) cur[lane] = U[j * r + lane] + S[sib * r + lane];          // in[z]
+      __syncwarp();
+      const float* tab = tabs + ((c - 1) & 1) * rr;
+      if (has) {
+        // message to the child: lane b, over the parent's values z (column of the table)
+        float m = -CUDART_INF_F;
+        for (int z = 0; z < r; ++z) m = fmaxf(m, cur[z] + tab[z * r + lane]);
+        float s = 0.f;
+        for (int z = 0; z < r; ++z) s += __expf(cur[z] + tab[z * r + lane] - m);
+        U[c * r + lane] = (m == -CUDART_INF_F) ? -CUDART_INF_F : m + __logf(s);
+        // gradient of the child's table: lane z (row), over the child's values b
+        const float in_z = cur[lane];
+        const float gam_parent = __expf(U[j * r + lane] + prod[j * r + lane] - logq);
+        const float* row = tab + lane * r;
+        const float* pc = prod + c * r;
+        __nv_bfloat16* dst = ds + r + static_cast<size_t>(c - 1) * rr + lane * r;
+        for (int q = 0; q < r; ++q) {                     // start at column `lane`: conflict-free (r a power of two)
+          const int b = (q + lane) & (r - 1);
+          const float lo = row[b];
+          dst[b] = __float2bfloat16_rn(wt * (__expf(in_z + lo + pc[b] - logq) - __expf(lo) * gam_parent));
+        }
+      }
+      __syncwarp();
+    }
+    // ---- evidence gradients: token i under its owner's posterior
+    for (int i = 0; i < n; ++i) {
+      const int o = first_leaf_node + (i >> 1);
+      const bool valid = targets[static_cast<size_t>(w) * n + i] >= 0;
+      if (has)
+        post[(static_cast<size_t>(w) * n + i) * r + lane] = valid ? wt * __expf(U[o * r + lane] + prod[o * r + lane] - logq) : 0.f;
+    }
+    __syncwarp();
+  }
+}
+
+// ---------------------------------------------------------------- bf16 transpose with a padded pitch
+// dst[c, r] = src[r, c] for r < rows, c < cols; dst rows have `dst_pitch` elements (>= rows; the padding is not written).
+__global__ void transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int rows,
+                                      int cols, size_t src_pitch, size_t dst_pitch) {
+  __shared__ __nv_bfloat16 tile[64][66];
+  const int c0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
+  for (int e = threadIdx.x; e < 64 * 64; e += blockDim.x) {
+    const int rr_ = e / 64, cc = e % 64;
+    if (r0 + rr_ < rows && c0 + cc < cols) tile[rr_][cc] = src[static_cast<size_t>(r0 + rr_) * src_pitch + c0 + cc];
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < 64 * 64; e += blockDim.x) {
+    const int cc = e / 64, rr_ = e % 64;
+    if (r0 + rr_ < rows && c0 + cc < cols) dst[static_cast<size_t>(c0 + cc) * dst_pitch + r0 + rr_] = tile[rr_][cc];
+  }
+}
+
+// ---------------------------------------------------------------- plain bf16 GEMM on the tcgen05 tensor cores
+// C[M, N] (fp32, row-major, pitch ldc) = A[M, K] B[N, K]^T (+ C if accumulate); A and B bf16, K contiguous (K-major), read
+// through TMA descriptors with 64-element boxes (out-of-range rows and K columns read as zero). Same pipeline as the
+// projection kernel: one persistent CTA per SM, warp 0 TMA producer, warp 1 MMA issuer (M=128, N=256 tiles, two TMEM
+// slots), warps 2..5 epilogue (one thread per row, 16 fp32 columns per step).
+struct PlainGemmParams {
+  CUtensorMap tm_a;      // A [M, K]  box 64 x 128
+  CUtensorMap tm_b;      // B [N, K]  box 64 x 256
+  int M, N, kblocks;
+  int m_tiles, n_tiles;
+  int stages, stage_bytes;
+  int accumulate;
+  float* C;
+  size_t ldc;
+  unsigned* status;
+};
+constexpr int kPlainTileN = 256;
+
+__global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __grid_constant__ PlainGemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
+  uint8_t* tiles = smem_raw + (tiles_addr - raw_addr);
+  GemmControl* ctl = reinterpret_cast<GemmControl*>(tiles + static_cast<size_t>(p.stages) * p.stage_bytes);
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int num_items = p.m_tiles * p.n_tiles;      // m-tile fastest: CTAs running together share a B tile through L2
+  constexpr uint32_t kSlots = 2;
+  constexpr uint32_t kBBytes = kPlainTileN * kBlockK * 2;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(smem_u32(&ctl->full[s]), 1);
+      mbar_init(smem_u32(&ctl->empty[s]), 1);
+    }
+    for (uint32_t s = 0; s < kSlots; ++s) {
+      mbar_init(smem_u32(&ctl->tfull[s]), 1);
+      mbar_init(smem_u32(&ctl->tempty[s]), 4);
+    }
+    mbar_init(smem_u32(&ctl->drain), 1);
+    ctl->abort = 0;
+    fence_mbar_init();
+    tma_prefetch_desc(&p.tm_a);
+    tma_prefetch_desc(&p.tm_b);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+        const int mt = item % p.m_tiles, nt = item / p.m_tiles;
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
+          const uint32_t full = smem_u32(&ctl->full[stage]);
+          const uint32_t a_dst = tiles_addr + stage * p.stage_bytes;
+          mbar_arrive_expect_tx(full, kABytes + kBBytes);
+          tma_load_2d(a_dst, &p.tm_a, full, kb * kBlockK, mt * kBlockM);
+          tma_load_2d(a_dst + kABytes, &p.tm_b, full, kb * kBlockK, nt * kPlainTileN);
+          issued_mask |= 1u << stage;
+          phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
+          if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        for (int s = 0; s < p.stages; ++s)
+          if (issued_mask & (1u << s)) {
+            const uint32_t bar = smem_u32(&ctl->full[s]);
+            const uint32_t par = (phase_mask >> s) & 1u;
+            const uint64_t t0 = global_timer_ns();
+            while (!mbar_try_wait(bar, par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+          }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, use = 0;
+      bool ok = true;
+      const uint32_t idesc = umma_idesc_bf16(kBlockM, kPlainTileN);
+      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++use) {
+        const uint32_t slot = use % kSlots;
+        if (!bounded_wait(smem_u32(&ctl->tempty[slot]), ((use / kSlots) & 1u) ^ 1u, ctl, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + slot * kPlainTileN;
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = tiles_addr + stage * p.stage_bytes;
+          const uint64_t a_desc = umma_smem_desc_sw128(a_addr);
+          const uint64_t b_desc = umma_smem_desc_sw128(a_addr + kABytes);
+#pragma unroll
+          for (int kk = 0; kk < kBlockK / 16; ++kk)
+            umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+          umma_commit(smem_u32(&ctl->empty[stage]));
+          if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&ctl->tfull[slot]));
+      }
+      if (!ok) {
+        umma_commit(smem_u32(&ctl->drain));
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+    __syncwarp();
+  } else {
+    const int quarter = warp & 3;
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    uint32_t use = 0;
+    for (int item = blockIdx.x; item < num_items; item += gridDim.x, ++use) {
+      const int mt = item % p.m_tiles, nt = item / p.m_tiles;
+      const uint32_t slot = use % kSlots;
+      if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (use / kSlots) & 1u, ctl, p.status, lane)) break;
+      tc_fence_after();
+      const int row = mt * kBlockM + quarter * 32 + lane;
+      const uint32_t tcol = lane_base + slot * kPlainTileN;
+      float* crow = p.C + static_cast<size_t>(row < p.M ? row : 0) * p.ldc;
+      for (int b = 0; b < kPlainTileN / 16; ++b) {
+        float x[16];
+        tmem_ld16(tcol + b * 16, x);
+        const int col0 = nt * kPlainTileN + b * 16;
+        if (row < p.M && col0 < p.N) {                 // N is a multiple of 16
+          float4* c4 = reinterpret_cast<float4*>(crow + col0);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            float4 v = make_float4(x[4 * q], x[4 * q + 1], x[4 * q + 2], x[4 * q + 3]);
+            if (p.accumulate) {
+              const float4 o = c4[q];
+              v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+            }
+            c4[q] = v;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctl->tempty[slot]));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace mtpc

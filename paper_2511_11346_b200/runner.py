@@ -113,5 +113,20 @@ class DeviceHead:
         self.head.mtpc_window_loss(h, t, num_sequences, sequence_length, gamma, slot, loss)
         return slot, loss
 
+    def window_logprob_backward(self, weight, hidden=None, targets=None):
+        """-> dict(logprob [T], dh [T, d], dW_emit, dW_sum, dT_static or None) as fp32 device tensors."""
+        import torch
+        s = self.wl.shape
+        h = self.hidden_device() if hidden is None else hidden
+        t = torch.from_numpy(self.wl.targets).to(self.device) if targets is None else targets
+        T = h.shape[0]
+        f32 = dict(dtype=torch.float32, device=self.device)
+        out = dict(logprob=torch.empty(T, **f32), dh=torch.empty((T, s.d), **f32),
+                   dW_emit=torch.empty((s.n, s.r, s.v, s.d), **f32), dW_sum=torch.empty((s.sum_rows, s.d), **f32),
+                   dT_static=torch.empty((max(s.n - 1, 1), s.r, s.r), **f32) if s.family == I.HMM else None)
+        self.head.mtpc_window_logprob_backward(h, t, weight, out["logprob"], out["dh"], out["dW_emit"], out["dW_sum"],
+                                               out["dT_static"])
+        return out
+
     def close(self):
         self.head.mtpc_destroy()
