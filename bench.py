@@ -225,6 +225,39 @@ def measure_decode_cell(torch, cell, steps: int, warmup: int):
     return out, launches * (steps + warmup) + (launches + 1) * (steps + warmup)
 
 
+def measure_backward(torch, dh, wl, hidden, targets, steps: int, peaks):
+    """One training step of the head = mtpc_window_logprob_backward (forward value + all gradients): ms per call,
+    the per-phase split from the library's event ring, and the tensor throughput over the four weight-sized
+    contractions it runs (forward, recompute, d hidden, dW): 4 x the forward's algorithmic FLOPs."""
+    s = wl.shape
+    f32 = dict(dtype=torch.float32, device="cuda")
+    weight = torch.full((wl.T,), -1.0 / wl.T, **f32)
+    out = (torch.empty(wl.T, **f32), torch.empty((wl.T, s.d), **f32), torch.empty((s.n, s.r, s.v, s.d), **f32),
+           torch.empty((s.sum_rows, s.d), **f32), torch.empty((max(s.n - 1, 1), s.r, s.r), **f32) if s.family == I.HMM else None)
+    call = lambda: dh.head.mtpc_window_logprob_backward(hidden, targets, weight, *out)
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    dh.head.mtpc_set_timing(steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    phases = [dh.head.mtpc_get_timing(i) for i in range(steps)]
+    phase_ms = [statistics.mean(p[k] for p in phases) for k in range(len(phases[0]))]
+    dh.head.mtpc_set_timing(0)
+    flops = 4.0 * algorithmic_flops(wl)
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"call": "mtpc_window_logprob_backward", "ms_per_call": ms, "positions_per_s": wl.T / (ms * 1e-3),
+            "phase_ms": {"forward_projection": phase_ms[0], "circuit_backward": phase_ms[1],
+                         "projection_gradient_mode": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]},
+            "flops_per_call": flops, "achieved_tflops": tf, "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
+            "device_status": dh.head.mtpc_get_status()}
+
+
 def run_ours(args):
     import torch
     from paper_2511_11346_b200.runner import DeviceHead
@@ -324,6 +357,10 @@ def run_ours(args):
         cpu_baseline = {"value": cpu_value, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
                         "sample": f"first {sample} of {wl.T} positions, one pass, {cpu_s:.1f} s"}
 
+    backward = None
+    if args.backward and world == 1:
+        backward = measure_backward(torch, dh, wl, hidden, targets, steps=max(5, min(args.steps, 30)), peaks=peaks)
+
     draft, sweep = None, None
     if not args.no_draft and world == 1:
         cells = I.DECODE_CELLS if args.decode_cells == "all" else [(I.CP, 8, 64)]
@@ -349,6 +386,8 @@ def run_ours(args):
         "cpu_baseline": cpu_baseline,
         "device_status": status,
     }
+    if backward is not None:
+        line["backward"] = backward
     if draft is not None:
         line["draft"] = draft
         line["decode_sweep"] = sweep
@@ -369,6 +408,7 @@ def main():
     ap.add_argument("--decode-cells", choices=["all", "one"], default="all",
                     help="draft measurement: the twelve cells of the decode sweep, or only CP n=8 P=64")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiling runs)")
+    ap.add_argument("--backward", action="store_true", help="also time mtpc_window_logprob_backward on the workload")
     ap.add_argument("--positions", type=int, default=None,
                     help="override the number of positions (scaled-down profiler captures; not a bench value)")
     args = ap.parse_args()

@@ -348,7 +348,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
   GemmControl* ctl = reinterpret_cast<GemmControl*>(tiles + static_cast<size_t>(p.stages) * p.stage_bytes);
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int num_items = p.m_tiles * p.n_tiles;      // m-tile fastest: CTAs running together share a B tile through L2
+  // n-tile fastest: the CTAs running together cover a few m-tiles x all n-tiles, so the (larger) A operand is
+  // streamed from HBM once and the B operand once per wave of m-tiles
+  const int num_items = p.m_tiles * p.n_tiles;
   constexpr uint32_t kSlots = 2;
   constexpr uint32_t kBBytes = kPlainTileN * kBlockK * 2;
 
@@ -381,7 +383,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
       uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
-        const int mt = item % p.m_tiles, nt = item / p.m_tiles;
+        const int nt = item % p.n_tiles, mt = item / p.n_tiles;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
           const uint32_t full = smem_u32(&ctl->full[stage]);
@@ -442,7 +444,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     uint32_t use = 0;
     for (int item = blockIdx.x; item < num_items; item += gridDim.x, ++use) {
-      const int mt = item % p.m_tiles, nt = item / p.m_tiles;
+      const int nt = item % p.n_tiles, mt = item / p.n_tiles;
       const uint32_t slot = use % kSlots;
       if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (use / kSlots) & 1u, ctl, p.status, lane)) break;
       tc_fence_after();

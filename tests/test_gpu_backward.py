@@ -74,3 +74,44 @@ def test_backward_small_shapes(family, n, r, v, d, T):
     fwd = dh.window_logprob(targets=torch.from_numpy(t).cuda())
     assert torch.equal(fwd, out["logprob"])
     dh.close()
+
+
+@pytest.mark.parametrize("idx,nsample", [(1, 48), (3, 24)])
+def test_backward_full_size_configs_on_sampled_positions(idx, nsample):
+    """Full-size launch (the configuration the benchmark times). The loss weights are non-zero on a seeded sample of
+    positions only, so the weight gradients are sums over exactly those positions, which the oracle can afford; the
+    gradient of the hidden states must vanish everywhere else. Properties that hold at any size are checked on a
+    second launch with every weight non-zero: the logit gradients of an input unit sum to zero over the bytes, so
+    dW_emit summed over the bytes of a unit is zero, and likewise dW_sum summed over the inputs of a sum unit."""
+    wl = I.config_workload(idx)
+    s = wl.shape
+    rng = np.random.default_rng(60 + idx)
+    rows = np.unique(np.concatenate([[0, 127, 128, wl.T - 129, wl.T - 128, wl.T - 1],
+                                     rng.choice(wl.T, nsample, replace=False)]))
+    weight = np.zeros(wl.T, dtype=np.float32)
+    weight[rows] = rng.normal(size=len(rows)).astype(np.float32)
+    dh = DeviceHead(wl)
+    out = dh.window_logprob_backward(torch.from_numpy(weight).cuda())
+    assert dh.head.mtpc_get_status() == 0
+    ref = og.window_logprob_grad(s.family, wl.hidden_q[rows], wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets[rows],
+                                 weight[rows])
+    floor = 2e-5 * float(np.abs(weight).max()) * len(rows) ** 0.5
+    got_dh = out["dh"].cpu().numpy()
+    assert np.abs(out["logprob"].cpu().numpy()[rows] - ref["logprob"]).max() <= 2e-3
+    check("d_hidden", torch.from_numpy(got_dh[rows]), ref["dh"], floor)
+    others = np.setdiff1d(np.arange(wl.T), rows)
+    assert np.abs(got_dh[others]).max() == 0.0
+    check("dW_emit", out["dW_emit"], ref["dW_emit"], floor)
+    check("dW_sum", out["dW_sum"], ref["dW_sum"], floor)
+    del ref
+    # every position weighted: sums over the bytes of a unit / the inputs of a sum unit vanish
+    weight_all = torch.full((wl.T,), -1.0 / wl.T, device="cuda")
+    out = dh.window_logprob_backward(weight_all)
+    assert dh.head.mtpc_get_status() == 0
+    dW = out["dW_emit"]
+    scale = float(dW.abs().max())
+    assert scale > 0 and float(dW.sum(dim=2).abs().max()) <= 2e-2 * scale
+    dR = out["dW_sum"].reshape(-1, s.r, s.d)
+    assert float(dR.sum(dim=1).abs().max()) <= 2e-2 * float(dR.abs().max()) + 1e-9
+    assert torch.isfinite(out["dh"]).all() and float(out["dh"].abs().max()) > 0
+    dh.close()
