@@ -245,6 +245,7 @@ struct GradArgs {            // what the projection kernel needs beyond the forw
   __nv_bfloat16* dlogit = nullptr;
   __nv_bfloat16* dlogit_t = nullptr;
   size_t t_pitch = 0;
+  size_t dlogit_pitch = 0;
 };
 
 int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int wpp, bool with_emit, bool with_sum,
@@ -263,6 +264,7 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
     p.dlogit = ga->dlogit;
     p.dlogit_t = ga->dlogit_t;
     p.t_pitch = ga->t_pitch;
+    p.dlogit_pitch = ga->dlogit_pitch;
   }
   int rc = make_tmap(&p.tm_a, hidden_bf16, static_cast<uint64_t>(rows), static_cast<uint64_t>(c.d), kBlockM);
   if (rc != MTPC_OK) return rc;
@@ -531,24 +533,25 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
 size_t round64(size_t x) { return (x + 63) / 64 * 64; }
 
 // Carving of the backward workspace for T positions (all buffers 256-byte aligned).
+// The sum-unit logit gradients sit to the right of the emission logit gradients in one matrix [T, Kd], Kd = Nc + Spad,
+// and W_sum^T to the right of W_emit^T in [d, Kd], so that d hidden is a single GEMM over K = Nc + S r.
 struct BackwardLayout {
-  size_t Nc, Spad, Tpad;
-  size_t off_lse, off_post, off_dsum, off_dsum_t, off_dlogit, off_dlogit_t, off_wt, off_rt, off_ht, total;
+  size_t Nc, Spad, Tpad, Kd;
+  size_t off_lse, off_post, off_dsum_t, off_dlogit, off_dlogit_t, off_wt, off_ht, total;
 };
 void plan_backward(const mtpc_config& c, const Layout& L, int T, BackwardLayout* B) {
   B->Nc = static_cast<size_t>(c.n) * c.r * c.v;
   B->Spad = round64(L.sum_rows);
   B->Tpad = round64(T);
+  B->Kd = B->Nc + B->Spad;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
   B->off_lse = take(static_cast<size_t>(T) * c.n * c.r * 4);
   B->off_post = take(static_cast<size_t>(T) * c.n * c.r * 4);
-  B->off_dsum = take(static_cast<size_t>(T) * B->Spad * 2);          // [T, Spad] bf16
-  B->off_dsum_t = take(static_cast<size_t>(L.sum_rows) * B->Tpad * 2);  // [S r, Tpad]
-  B->off_dlogit = take(static_cast<size_t>(T) * B->Nc * 2);          // [T, Nc]
+  B->off_dsum_t = take(static_cast<size_t>(L.sum_rows) * B->Tpad * 2);  // [S r, Tpad] bf16
+  B->off_dlogit = take(static_cast<size_t>(T) * B->Kd * 2);          // [T, Nc | Spad]
   B->off_dlogit_t = take(B->Nc * B->Tpad * 2);                       // [Nc, Tpad]
-  B->off_wt = take(static_cast<size_t>(c.d) * B->Nc * 2);            // W_emit^T [d, Nc]
-  B->off_rt = take(static_cast<size_t>(c.d) * B->Spad * 2);          // W_sum^T  [d, Spad]
+  B->off_wt = take(static_cast<size_t>(c.d) * B->Kd * 2);            // [d, Nc | Spad]: W_emit^T | W_sum^T
   B->off_ht = take(static_cast<size_t>(c.d) * B->Tpad * 2);          // hidden^T [d, Tpad]
   B->total = off;
 }
@@ -557,8 +560,10 @@ int launch_transpose(mtpc_head* h, const void* src, void* dst, int rows, int col
                      cudaStream_t st) {
   if (rows <= 0 || cols <= 0) return MTPC_OK;
   dim3 grid((cols + 63) / 64, (rows + 63) / 64);
+  const int vec_ok = src_pitch % 8 == 0 && dst_pitch % 8 == 0 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0 &&
+                     (reinterpret_cast<uintptr_t>(dst) & 15u) == 0;
   transpose_bf16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), static_cast<__nv_bfloat16*>(dst),
-                                              rows, cols, src_pitch, dst_pitch);
+                                              rows, cols, src_pitch, dst_pitch, vec_ok);
   h->launches++;
   return check_launch();
 }
@@ -861,12 +866,11 @@ int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int3
   uint8_t* bw = static_cast<uint8_t*>(bwd_workspace);
   float* lse = reinterpret_cast<float*>(bw + B.off_lse);
   float* post = reinterpret_cast<float*>(bw + B.off_post);
-  __nv_bfloat16* dsum = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dsum);
   __nv_bfloat16* dsum_t = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dsum_t);
   __nv_bfloat16* dlogit = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit);
+  __nv_bfloat16* dsum = dlogit + B.Nc;                       // columns [Nc, Nc + S r) of the same rows
   __nv_bfloat16* dlogit_t = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit_t);
-  void* wt = bw + B.off_wt;
-  void* rt = bw + B.off_rt;
+  __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(bw + B.off_wt);
   void* ht = bw + B.off_ht;
   const int Nc = static_cast<int>(B.Nc);
 
@@ -887,7 +891,7 @@ int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int3
   bool bad = false;
   if (static_hmm) bad |= cudaMemsetAsync(dT_static, 0, static_cast<size_t>(c.n - 1) * c.r * c.r * 4, st) != cudaSuccess;
   if (bad) return MTPC_ERR_CUDA;
-  rc = launch_circuit_backward(head, T, targets, weight, out_logprob, post, dsum, static_cast<int>(B.Spad), dT_static, st);
+  rc = launch_circuit_backward(head, T, targets, weight, out_logprob, post, dsum, static_cast<int>(B.Kd), dT_static, st);
   pt.end();
   if (rc != MTPC_OK) return rc;
   // 3. logits recomputed, turned into their gradient (bf16, both orientations)
@@ -898,18 +902,19 @@ int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int3
   ga.dlogit = dlogit;
   ga.dlogit_t = dlogit_t;
   ga.t_pitch = B.Tpad;
+  ga.dlogit_pitch = B.Kd;
   rc = launch_gemm(head, kModeGrad, hb, T, 1, true, false, targets, nullptr, nullptr, st, &ga);
   pt.end();
   if (rc != MTPC_OK) return rc;
   // 4. transposed operands, then the plain GEMMs
   pt.begin();
-  rc = launch_transpose(head, head->W_emit_bf16, wt, Nc, c.d, c.d, B.Nc, st);
-  if (rc == MTPC_OK) rc = launch_transpose(head, head->W_sum_bf16, rt, L.sum_rows, c.d, c.d, B.Spad, st);
+  rc = launch_transpose(head, head->W_emit_bf16, wt, Nc, c.d, c.d, B.Kd, st);
+  if (rc == MTPC_OK) rc = launch_transpose(head, head->W_sum_bf16, wt + B.Nc, L.sum_rows, c.d, c.d, B.Kd, st);
   if (rc == MTPC_OK) rc = launch_transpose(head, hb, ht, T, c.d, c.d, B.Tpad, st);
-  if (rc == MTPC_OK) rc = launch_transpose(head, dsum, dsum_t, T, L.sum_rows, B.Spad, B.Tpad, st);
-  // d hidden [T, d] = dlogit [T, Nc] W_emit [Nc, d] + dsum [T, S r] W_sum [S r, d]
-  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dlogit, B.Nc, wt, B.Nc, d_hidden, c.d, T, c.d, Nc, false, st);
-  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dsum, B.Spad, rt, B.Spad, d_hidden, c.d, T, c.d, L.sum_rows, true, st);
+  if (rc == MTPC_OK) rc = launch_transpose(head, dsum, dsum_t, T, L.sum_rows, B.Kd, B.Tpad, st);
+  // d hidden [T, d] = [dlogit | dsum] [T, Nc + S r] [W_emit ; W_sum] [Nc + S r, d]
+  if (rc == MTPC_OK)
+    rc = launch_plain_gemm(head, dlogit, B.Kd, wt, B.Kd, d_hidden, c.d, T, c.d, Nc + L.sum_rows, false, st);
   // dW_emit [Nc, d] = dlogit^T [Nc, T] hidden [T, d];  dW_sum [S r, d] = dsum^T [S r, T] hidden [T, d]
   if (rc == MTPC_OK) rc = launch_plain_gemm(head, dlogit_t, B.Tpad, ht, B.Tpad, dW_emit, c.d, Nc, c.d, T, false, st);
   if (rc == MTPC_OK) rc = launch_plain_gemm(head, dsum_t, B.Tpad, ht, B.Tpad, dW_sum, c.d, L.sum_rows, c.d, T, false, st);

@@ -307,16 +307,37 @@ __global__ void circuit_btree_backward_kernel(const float* __restrict__ G, const
 
 // ---------------------------------------------------------------- bf16 transpose with a padded pitch
 // dst[c, r] = src[r, c] for r < rows, c < cols; dst rows have `dst_pitch` elements (>= rows; the padding is not written).
-__global__ void transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int rows,
-                                      int cols, size_t src_pitch, size_t dst_pitch) {
-  __shared__ __nv_bfloat16 tile[64][66];
+// 64 x 64 tiles through shared memory, 256 threads. Inner tiles move 16 bytes per thread and request on both sides
+// (pitches and base addresses allow it: multiples of 8 elements); edge tiles fall back to element-wise copies.
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src,
+                                                             __nv_bfloat16* __restrict__ dst, int rows, int cols,
+                                                             size_t src_pitch, size_t dst_pitch, int vec_ok) {
+  __shared__ __align__(16) __nv_bfloat16 tile[64][72];
   const int c0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
-  for (int e = threadIdx.x; e < 64 * 64; e += blockDim.x) {
+  const bool inner = vec_ok && r0 + 64 <= rows && c0 + 64 <= cols;
+  if (inner) {
+    for (int e = threadIdx.x; e < 64 * 8; e += 256) {
+      const int rr_ = e >> 3, ch = e & 7;
+      *reinterpret_cast<uint4*>(&tile[rr_][ch * 8]) =
+          *reinterpret_cast<const uint4*>(src + static_cast<size_t>(r0 + rr_) * src_pitch + c0 + ch * 8);
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < 64 * 8; e += 256) {
+      const int cc = e & 63, ch = e >> 6;              // consecutive threads: consecutive columns of the tile
+      __align__(16) __nv_bfloat16 v[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) v[q] = tile[ch * 8 + q][cc];
+      *reinterpret_cast<uint4*>(dst + static_cast<size_t>(c0 + cc) * dst_pitch + r0 + ch * 8) =
+          *reinterpret_cast<const uint4*>(v);
+    }
+    return;
+  }
+  for (int e = threadIdx.x; e < 64 * 64; e += 256) {
     const int rr_ = e / 64, cc = e % 64;
     if (r0 + rr_ < rows && c0 + cc < cols) tile[rr_][cc] = src[static_cast<size_t>(r0 + rr_) * src_pitch + c0 + cc];
   }
   __syncthreads();
-  for (int e = threadIdx.x; e < 64 * 64; e += blockDim.x) {
+  for (int e = threadIdx.x; e < 64 * 64; e += 256) {
     const int cc = e / 64, rr_ = e % 64;
     if (r0 + rr_ < rows && c0 + cc < cols) dst[static_cast<size_t>(c0 + cc) * dst_pitch + r0 + rr_] = tile[rr_][cc];
   }

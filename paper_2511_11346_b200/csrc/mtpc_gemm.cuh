@@ -63,7 +63,8 @@ struct GemmParams {
   // gradient mode: dlogit[t, col] = post[t, i, k] * (onehot(target) - exp(logit - lse[t, i, k])), bf16, both orientations
   const float* lse_in;               // [T, n, r]
   const float* post;                 // [T, n, r]   weight * d log q / d G
-  __nv_bfloat16* dlogit;             // [T, n*r*v]
+  __nv_bfloat16* dlogit;             // [T, n*r*v] with row pitch dlogit_pitch
+  size_t dlogit_pitch;
   __nv_bfloat16* dlogit_t;           // [n*r*v, t_pitch]
   size_t t_pitch;
   const int* unit_sel;               // [T*wpp, n]      selected input unit per token (sample mode)
@@ -499,7 +500,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
               o[q] = __float2bfloat16_rn(pst * ((rel == q ? 1.f : 0.f) - sm_));
             }
             if (valid) {
-              uint4* d4 = reinterpret_cast<uint4*>(p.dlogit + trow * (static_cast<size_t>(p.emit_units) * p.v) + col0);
+              uint4* d4 = reinterpret_cast<uint4*>(p.dlogit + trow * p.dlogit_pitch + col0);
               d4[0] = *reinterpret_cast<const uint4*>(&o[0]);
               d4[1] = *reinterpret_cast<const uint4*>(&o[8]);
 #pragma unroll
