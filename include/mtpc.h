@@ -69,8 +69,10 @@ typedef struct {
   int32_t n;                   /* window length. BTREE: a power of two >= 2                            */
   int32_t r;                   /* units per layer (mixture components / hidden states): a power of two,
                                   <= 128 for CP, <= 32 for HMM and BTREE                               */
-  int32_t v;                   /* vocabulary: a multiple of 16, <= 512, splittable into equal chunks of
-                                  <= 256 columns that are multiples of 16 (256 and 320 are)            */
+  int32_t v;                   /* vocabulary: a multiple of 16. Up to 512 (splittable into equal chunks of
+                                  <= 256 columns that are multiples of 16: 256 and 320 are) everything
+                                  works; larger vocabularies evaluate and train (the softmax runs online
+                                  across accumulator tiles) but the draft calls return UNSUPPORTED        */
   int32_t d;                   /* hidden size: a multiple of 64                                        */
   int32_t io_dtype;            /* MTPC_F32 | MTPC_BF16: dtype of hidden, W_emit and W_sum              */
   int32_t max_positions;       /* upper bound on T (log-prob) and P (draft) per call                   */

@@ -22,6 +22,7 @@ using namespace mtpc;
 constexpr size_t kAlign = 256;
 constexpr int kMaxPhases = 5;
 constexpr size_t kSlotSmemLimit = 160 * 1024;   // latent-draw tables of the draft slot kernel kept in shared memory up to this
+constexpr int kMaxDraftVocab = 512;     // draft sampling: the v logits of a unit live in 512 TMEM columns / 16 per lane
 constexpr int kWorkCounterWord = 16;   // word of the 256-byte status area used as the circuit kernels' work counter
 constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA on sm_100
 // Hidden states of one rasterisation block of the projection kernel: small enough to stay L2-resident next to the
@@ -50,6 +51,7 @@ struct Layout {
   size_t off_status, off_wemit, off_wsum, off_hidden, off_logA, off_G, off_logw, off_sel, off_logits, off_unit_lse;
   size_t off_prefix, off_partial, off_sum_bias;   // training loss: prefix log-marginals [max_positions, n], per-sequence terms
   int decode_max_p;     // positions the few-position draft path can take (0: path not available)
+  bool can_draft;       // v <= 512: the sampling kernels hold a whole input unit on chip
   size_t off_h_hidden, off_h_targets, off_h_uniforms, off_h_bytes, off_h_out;
   size_t total;
 };
@@ -84,7 +86,7 @@ int plan(const mtpc_config& c, Layout* L) {
   if (c.family != MTPC_CP && c.r > 32) return MTPC_ERR_UNSUPPORTED;
   if (c.family == MTPC_BTREE && (c.n < 2 || !is_pow2(c.n))) return MTPC_ERR_UNSUPPORTED;
   if (c.d % kBlockK != 0) return MTPC_ERR_UNSUPPORTED;
-  if (c.v % 16 != 0 || c.v > 512) return MTPC_ERR_UNSUPPORTED;
+  if (c.v % 16 != 0) return MTPC_ERR_UNSUPPORTED;
   if (static_cast<int64_t>(c.n) * c.r * c.v > (1ll << 30)) return MTPC_ERR_SHAPE;
 
   L->S = (c.family == MTPC_BTREE) ? 1 + (c.n - 2) * c.r : (ctx ? 1 + (c.n - 1) * c.r : 1);
@@ -97,13 +99,19 @@ int plan(const mtpc_config& c, Layout* L) {
   L->sum_tiles = (L->sum_rows + sum_cols - 1) / sum_cols;
   const int emit_units = c.n * c.r;
   // sampling: emission unit -> equal tiles of <= 256 columns, each a multiple of 16, all in TMEM at once
-  int chunks = (c.v + 255) / 256;
-  while (c.v % chunks != 0 || (c.v / chunks) % 16 != 0) ++chunks;
-  L->sm.tile_cols = c.v / chunks;
-  L->sm.group_units = 1;
-  L->sm.group_tiles = chunks;
-  L->sm.num_groups = emit_units;
-  if (!fit_tiling(&L->sm, sum_cols) || L->sm.num_slots < chunks) return MTPC_ERR_UNSUPPORTED;
+  // (a unit of more than 512 bytes does not fit tensor memory: such heads evaluate and train, but do not draft)
+  L->can_draft = c.v <= kMaxDraftVocab;
+  if (L->can_draft) {
+    int chunks = (c.v + 255) / 256;
+    while (c.v % chunks != 0 || (c.v / chunks) % 16 != 0) ++chunks;
+    L->sm.tile_cols = c.v / chunks;
+    L->sm.group_units = 1;
+    L->sm.group_tiles = chunks;
+    L->sm.num_groups = emit_units;
+    if (!fit_tiling(&L->sm, sum_cols) || L->sm.num_slots < chunks) return MTPC_ERR_UNSUPPORTED;
+  } else {
+    memset(&L->sm, 0, sizeof(L->sm));
+  }
   // log-likelihood: 256-column tiles; a group is the shortest run of whole units that is a whole number of tiles
   const int lcm = c.v / gcd_int(c.v, 256) * 256;
   L->lp.tile_cols = 256;
@@ -130,7 +138,7 @@ int plan(const mtpc_config& c, Layout* L) {
   L->off_G = take(L->max_windows * c.n * c.r * 4);
   L->off_logw = take(static_cast<size_t>(c.max_positions) * L->sum_rows * 4);
   L->off_sel = take(L->max_windows * c.n * 4);
-  L->decode_max_p = c.r <= 32 ? (c.max_positions < kDecodeMaxP ? c.max_positions : kDecodeMaxP) : 0;
+  L->decode_max_p = (c.r <= 32 && L->can_draft) ? (c.max_positions < kDecodeMaxP ? c.max_positions : kDecodeMaxP) : 0;
   L->off_logits = take(static_cast<size_t>(L->decode_max_p) * emit_units * c.v * 4);
   L->off_unit_lse = take(static_cast<size_t>(L->decode_max_p) * emit_units * 4);
   L->off_prefix = take(static_cast<size_t>(c.max_positions) * c.n * 4);
@@ -466,6 +474,7 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
   const int W = P * wpp;
+  if (!L.can_draft) return MTPC_ERR_UNSUPPORTED;
   const void* hb = nullptr;
   int rc = stage_hidden(h, hidden, P, &hb, st);
   if (rc != MTPC_OK) return rc;
@@ -681,7 +690,7 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   fail |= !set_circuit_attributes(*cfg);
   {
     const size_t smem = kAcceptWarps * accept_warp_floats(cfg->family, cfg->n, cfg->r, cfg->v) * sizeof(float);
-    if (smem > 48 * 1024)
+    if (L.can_draft && smem > 48 * 1024)
       fail |= cudaFuncSetAttribute(spec_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    static_cast<int>(smem)) != cudaSuccess;
   }
@@ -718,7 +727,7 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   if (check_launch() != MTPC_OK) { delete h; return MTPC_ERR_CUDA; }
   const uint64_t emit_rows = static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v;
   rc = make_tmap(&h->tm_emit_lp, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols);
-  if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
+  if (rc == MTPC_OK && L.can_draft) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols);
   h->decode_tile_rows = decode_tile_rows(static_cast<long long>(emit_rows), h->num_sms);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_dec, h->W_emit_bf16, emit_rows, cfg->d, h->decode_tile_rows);

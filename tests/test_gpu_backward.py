@@ -115,3 +115,31 @@ def test_backward_full_size_configs_on_sampled_positions(idx, nsample):
     assert float(dR.sum(dim=1).abs().max()) <= 2e-2 * float(dR.abs().max()) + 1e-9
     assert torch.isfinite(out["dh"]).all() and float(out["dh"].abs().max()) > 0
     dh.close()
+
+
+@pytest.mark.parametrize("family,n,r,v,d,T", [(I.CP, 2, 2, 1024, 64, 130), (I.HMM, 2, 4, 2048, 64, 70),
+                                               (I.BTREE, 4, 4, 4112, 64, 33), (I.CP, 1, 1, 32768, 64, 5)])
+def test_large_vocabulary_heads_evaluate_and_train_but_do_not_draft(family, n, r, v, d, T):
+    """More than 512 symbols: a unit's logits no longer fit tensor memory at once; the softmax runs online across the
+    accumulator tiles (log-likelihood, prefix marginals, backward). Drafting is refused."""
+    from oracle import mtpc_oracle as orc
+    from paper_2511_11346_b200 import binding as B
+    wl = I.make_workload(f"bigv_{family}_{v}", I.HeadShape(family, n, r, v, d), T, seed=7000 + v + T, wpp=1, weight_std=0.25)
+    dh = DeviceHead(wl)
+    got = dh.window_logprob().cpu().numpy()
+    ref = orc.window_logprob(family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets)
+    assert np.abs(got - ref).max() <= 2e-3
+    pre = dh.window_prefix_logprob().cpu().numpy()
+    assert np.abs(pre - orc.window_prefix_logprob(family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets)).max() <= 2e-3
+    weight = np.random.default_rng(v).normal(size=T).astype(np.float32)
+    out = dh.window_logprob_backward(torch.from_numpy(weight).cuda())
+    assert dh.head.mtpc_get_status() == 0
+    g = og.window_logprob_grad(family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets, weight)
+    floor = 2e-5 * float(np.abs(weight).max()) * T ** 0.5
+    check("d_hidden", out["dh"], g["dh"], floor)
+    check("dW_emit", out["dW_emit"], g["dW_emit"], floor)
+    check("dW_sum", out["dW_sum"], g["dW_sum"], floor)
+    with pytest.raises(B.MtpcError) as e:
+        dh.draft_sample(1)
+    assert e.value.code == -3
+    dh.close()
