@@ -23,6 +23,7 @@ constexpr size_t kAlign = 256;
 constexpr int kMaxPhases = 5;
 constexpr size_t kSlotSmemLimit = 160 * 1024;   // latent-draw tables of the draft slot kernel kept in shared memory up to this
 constexpr int kMaxDraftVocab = 512;     // draft sampling: the v logits of a unit live in 512 TMEM columns / 16 per lane
+constexpr int kHostChunkPositions = 2048;   // host-buffer calls upload and process this many positions at a time
 constexpr int kWorkCounterWord = 16;   // word of the 256-byte status area used as the circuit kernels' work counter
 constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA on sm_100
 // Hidden states of one rasterisation block of the projection kernel: small enough to stay L2-resident next to the
@@ -198,6 +199,9 @@ struct mtpc_head {
   CUtensorMap tm_emit_dec, tm_sum_dec;          // the same matrices in the few-position draft path's tiles
   int decode_tile_rows, decode_sum_tile_rows;
   int num_sms;
+  cudaStream_t copy_stream; // host-buffer calls: uploads run here, ahead of the kernels (created on first use)
+  cudaEvent_t* copy_events; // [copy_event_count]: "chunk c is on the device"; [0] doubles as "the call may start"
+  int copy_event_count;
   int draft_P;              // positions whose logits the few-position draft path left in the workspace (0: none)
   int ring;                 // calls whose per-kernel events are retained (0 = timing off)
   cudaEvent_t* ev;          // [ring][kMaxPhases][2]
@@ -931,6 +935,24 @@ int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int3
   return rc;
 }
 
+// Streams and events of the chunked host-buffer path; no device memory is allocated.
+static int ensure_copy_pipeline(mtpc_head* head, int chunks) {
+  if (!head->copy_stream && cudaStreamCreateWithFlags(&head->copy_stream, cudaStreamNonBlocking) != cudaSuccess)
+    return MTPC_ERR_CUDA;
+  if (head->copy_event_count < chunks + 1) {
+    cudaEvent_t* ev = static_cast<cudaEvent_t*>(calloc(chunks + 1, sizeof(cudaEvent_t)));
+    if (!ev) return MTPC_ERR_CUDA;
+    for (int i = 0; i < chunks + 1; ++i) {
+      if (i < head->copy_event_count) ev[i] = head->copy_events[i];
+      else if (cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming) != cudaSuccess) { free(ev); return MTPC_ERR_CUDA; }
+    }
+    free(head->copy_events);
+    head->copy_events = ev;
+    head->copy_event_count = chunks + 1;
+  }
+  return MTPC_OK;
+}
+
 int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int32_t* targets_host, int32_t T,
                              float* out_logprob_host, void* stream) {
   int rc = check_call(head, T);
@@ -939,17 +961,34 @@ int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int
   if (!hidden_host || !targets_host || !out_logprob_host) return MTPC_ERR_NULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Layout& L = head->L;
-  const size_t elt = head->cfg.io_dtype == MTPC_F32 ? 4 : 2;
-  void* dh = head->ws + L.off_h_hidden;
+  const mtpc_config& c = head->cfg;
+  const size_t elt = c.io_dtype == MTPC_F32 ? 4 : 2;
+  uint8_t* dh = head->ws + L.off_h_hidden;
   int32_t* dt = at<int32_t>(head, L.off_h_targets);
   float* dout = at<float>(head, L.off_h_out);
-  bool fail = cudaMemcpyAsync(dh, hidden_host, static_cast<size_t>(T) * head->cfg.d * elt, cudaMemcpyHostToDevice, st) !=
-              cudaSuccess;
-  fail |= cudaMemcpyAsync(dt, targets_host, static_cast<size_t>(T) * head->cfg.n * 4, cudaMemcpyHostToDevice, st) !=
-          cudaSuccess;
+  // The positions are uploaded in chunks on a second stream while the kernels of the chunks before run on `stream`:
+  // only the first chunk's upload is not hidden behind compute.
+  const int chunks = (T + kHostChunkPositions - 1) / kHostChunkPositions;
+  if ((rc = ensure_copy_pipeline(head, chunks)) != MTPC_OK) return rc;
+  cudaStream_t cs = head->copy_stream;
+  bool fail = cudaEventRecord(head->copy_events[chunks], st) != cudaSuccess;     // uploads wait for earlier work on `stream`
+  fail |= cudaStreamWaitEvent(cs, head->copy_events[chunks], 0) != cudaSuccess;
+  for (int k = 0; k < chunks && !fail; ++k) {
+    const size_t t0 = static_cast<size_t>(k) * kHostChunkPositions;
+    const size_t tc = (T - t0) < static_cast<size_t>(kHostChunkPositions) ? (T - t0) : kHostChunkPositions;
+    fail |= cudaMemcpyAsync(dh + t0 * c.d * elt, static_cast<const uint8_t*>(hidden_host) + t0 * c.d * elt, tc * c.d * elt,
+                            cudaMemcpyHostToDevice, cs) != cudaSuccess;
+    fail |= cudaMemcpyAsync(dt + t0 * c.n, targets_host + t0 * c.n, tc * c.n * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess;
+    fail |= cudaEventRecord(head->copy_events[k], cs) != cudaSuccess;
+  }
   if (fail) return MTPC_ERR_CUDA;
-  rc = window_logprob_impl(head, dh, dt, T, dout, nullptr, st);
-  if (rc != MTPC_OK) return rc;
+  for (int k = 0; k < chunks; ++k) {
+    const size_t t0 = static_cast<size_t>(k) * kHostChunkPositions;
+    const int tc = static_cast<int>((T - t0) < static_cast<size_t>(kHostChunkPositions) ? (T - t0) : kHostChunkPositions);
+    if (cudaStreamWaitEvent(st, head->copy_events[k], 0) != cudaSuccess) return MTPC_ERR_CUDA;
+    rc = window_logprob_impl(head, dh + t0 * c.d * elt, dt + t0 * c.n, tc, dout + t0, nullptr, st);
+    if (rc != MTPC_OK) { cudaStreamSynchronize(cs); return rc; }
+  }
   fail = cudaMemcpyAsync(out_logprob_host, dout, static_cast<size_t>(T) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess;
   fail |= cudaStreamSynchronize(st) != cudaSuccess;
   return fail ? MTPC_ERR_CUDA : MTPC_OK;
@@ -1049,6 +1088,9 @@ int mtpc_launch_count(mtpc_head* head, uint64_t* out_count) {
 int mtpc_destroy(mtpc_head* head) {
   if (!head) return MTPC_ERR_NULL;
   free_timing(head);
+  for (int i = 0; i < head->copy_event_count; ++i) cudaEventDestroy(head->copy_events[i]);
+  free(head->copy_events);
+  if (head->copy_stream) cudaStreamDestroy(head->copy_stream);
   delete head;
   return MTPC_OK;
 }

@@ -233,3 +233,19 @@ def test_max_windows_per_position():
     dh = DeviceHead(wl)
     check_draft(dh, wl, np.arange(3))
     dh.close()
+
+
+def test_chunked_host_call_equals_device_call():
+    """The host-buffer entry point uploads and processes 2048 positions at a time; the results are those of one
+    device-buffer call (same arithmetic per position), ragged last chunk included, twice in a row."""
+    wl = I.make_workload("host_chunks", I.HeadShape(I.HMM, 4, 8, 320, 128), 5000, seed=91, weight_std=0.2)
+    dh = DeviceHead(wl)
+    dev = dh.window_logprob().cpu()
+    hh = dh.hidden_host()
+    th = torch.from_numpy(wl.targets).pin_memory()
+    for _ in range(2):
+        oh = torch.full((wl.T,), 7.0).pin_memory()
+        dh.head.mtpc_window_logprob_host(hh, th, oh)
+        assert torch.equal(oh, dev)
+    assert dh.head.mtpc_get_status() == 0
+    dh.close()
