@@ -249,6 +249,25 @@ struct PhaseTimer {
 
 int check_launch() { return cudaGetLastError() == cudaSuccess ? MTPC_OK : MTPC_ERR_CUDA; }
 
+// Launch `kernel`, optionally allowed to start before the kernel ahead of it in the stream has finished (programmatic
+// dependent launch): such a kernel calls grid_dependency_wait() before it touches the earlier kernel's results.
+template <typename... Params, typename... Args>
+void launch_kernel(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool dependent,
+                   Args&&... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 // Launch the projection kernel for `rows` positions over the emission groups (with_emit) and / or the sum tiles.
 struct GradArgs {            // what the projection kernel needs beyond the forward arguments (backward pass only)
   float* lse_out = nullptr;                  // forward for training: keep the units' log-sum-exps
@@ -325,14 +344,15 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
 }
 
 // Shared memory of one CTA of the binary-tree circuit kernel (see circuit_btree_kernel).
-size_t hmm_ctx_smem_bytes(int r) { return static_cast<size_t>(kCircuitWarps) * (2 * r * r + 32) * sizeof(float); }
+size_t hmm_stream_smem_bytes(int r) { return static_cast<size_t>(kCircuitWarps) * (kHmmDepth * r * r + 32) * sizeof(float); }
 size_t btree_smem_bytes(int n, int r, bool with_prefix) {
   return static_cast<size_t>(kCircuitWarps) * btree_warp_floats(n, r, with_prefix) * sizeof(float);
 }
 
 // Circuit evaluation of W windows: out[w] = joint log-prob (may be NULL when prefix is given); prefix (may be NULL)
 // [W, n] = log-marginals of the prefixes x_0..x_i.
-int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cudaStream_t st) {
+// dependent: the launch directly follows draft_slot_kernel, which has zeroed the work counter, and may overlap its tail.
+int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cudaStream_t st, bool dependent = false) {
   if (W <= 0) return MTPC_OK;
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
@@ -343,20 +363,20 @@ int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cuda
   // kernels that stream per-position tables hand out windows through a counter next to the status word
   unsigned* counter = at<unsigned>(h, L.off_status) + kWorkCounterWord;
   const int resident = blocks < 8 * h->num_sms ? blocks : 8 * h->num_sms;   // more CTAs than an SM can hold do no harm
-  if (c.family == MTPC_BTREE || c.family == MTPC_HMM) {
+  if (!dependent && (c.family == MTPC_BTREE || c.family == MTPC_HMM)) {
     if (cudaMemsetAsync(counter, 0, sizeof(unsigned), st) != cudaSuccess) return MTPC_ERR_CUDA;
   }
   if (c.family == MTPC_CP) {
-    circuit_cp_kernel<<<blocks, threads, 0, st>>>(G, logw, out, prefix, W, wpp, c.n, c.r, L.sum_rows);
+    launch_kernel(circuit_cp_kernel, blocks, threads, 0, st, dependent, G, logw, out, prefix, W, wpp, c.n, c.r, L.sum_rows);
   } else if (c.family == MTPC_HMM) {
-    circuit_hmm_stream_kernel<<<resident, threads, hmm_ctx_smem_bytes(c.r), st>>>(
-        G, logw, hmm_tables(h), hmm_table_stride(h), out, prefix, counter, W, wpp, c.n, c.r, L.sum_rows);
+    launch_kernel(circuit_hmm_stream_kernel, resident, threads, hmm_stream_smem_bytes(c.r), st, dependent, G, logw,
+                  hmm_tables(h), hmm_table_stride(h), out, prefix, counter, W, wpp, c.n, c.r, L.sum_rows);
   } else if (prefix != nullptr) {
-    circuit_btree_kernel<true><<<resident, threads, btree_smem_bytes(c.n, c.r, true), st>>>(
-        G, logw, out, prefix, counter, W, wpp, c.n, c.r, L.sum_rows);
+    launch_kernel(circuit_btree_kernel<true>, resident, threads, btree_smem_bytes(c.n, c.r, true), st, dependent, G, logw,
+                  out, prefix, counter, W, wpp, c.n, c.r, L.sum_rows);
   } else {
-    circuit_btree_kernel<false><<<resident, threads, btree_smem_bytes(c.n, c.r, false), st>>>(
-        G, logw, out, nullptr, counter, W, wpp, c.n, c.r, L.sum_rows);
+    launch_kernel(circuit_btree_kernel<false>, resident, threads, btree_smem_bytes(c.n, c.r, false), st, dependent, G,
+                  logw, out, static_cast<float*>(nullptr), counter, W, wpp, c.n, c.r, L.sum_rows);
   }
   h->launches++;
   return check_launch();
@@ -366,9 +386,9 @@ int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cuda
 // point) sets them to what it needs or more.
 bool set_circuit_attributes(const mtpc_config& c) {
   bool fail = false;
-  if (c.family == MTPC_HMM && hmm_ctx_smem_bytes(c.r) > 48 * 1024)
+  if (c.family == MTPC_HMM && hmm_stream_smem_bytes(c.r) > 48 * 1024)
     fail |= cudaFuncSetAttribute(circuit_hmm_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(hmm_ctx_smem_bytes(c.r))) != cudaSuccess;
+                                 static_cast<int>(hmm_stream_smem_bytes(c.r))) != cudaSuccess;
   if (c.family == MTPC_BTREE) {
     const int plain = static_cast<int>(btree_smem_bytes(c.n, c.r, false));
     const int pre = static_cast<int>(btree_smem_bytes(c.n, c.r, true));
@@ -499,17 +519,18 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
       const size_t base = static_cast<size_t>((2 * c.r + 3) & ~3) * sizeof(float);
       const size_t with_tables = base + static_cast<size_t>(chain) * c.r * c.r * sizeof(float);
       const int in_smem = chain > 0 && with_tables <= kSlotSmemLimit;
-      draft_slot_kernel<<<dim3(c.n, P), kSlotThreads, in_smem ? with_tables : base, st>>>(
-          c.family, at<float>(h, L.off_logits), at<float>(h, L.off_logw), hmm_tables(h), uniforms, out_bytes,
-          at<float>(h, L.off_G), at<float>(h, L.off_unit_lse), at<unsigned>(h, L.off_status), wpp, c.n, c.r, c.v,
-          L.sum_rows, hmm_table_stride(h), in_smem);
+      launch_kernel(draft_slot_kernel, dim3(c.n, P), kSlotThreads, in_smem ? with_tables : base, st, h->ring == 0, c.family,
+                    at<float>(h, L.off_logits), at<float>(h, L.off_logw), hmm_tables(h), uniforms, out_bytes,
+                    at<float>(h, L.off_G), at<float>(h, L.off_unit_lse), at<unsigned>(h, L.off_status),
+                    at<unsigned>(h, L.off_status) + kWorkCounterWord, wpp, c.n, c.r, c.v, L.sum_rows,
+                    hmm_table_stride(h), in_smem);
     }
     h->launches++;
     h->draft_P = P;
     pt.end();
     if ((rc = check_launch()) != MTPC_OK) return rc;
     pt.begin();
-    rc = launch_circuit(h, W, wpp, out_logprob, out_prefix, st);
+    rc = launch_circuit(h, W, wpp, out_logprob, out_prefix, st, /*dependent=*/h->ring == 0);
     pt.end();
     return rc;
   }

@@ -5,6 +5,8 @@
 #include <math_constants.h>
 #include <stdint.h>
 
+#include "mtpc_ptx.cuh"
+
 namespace mtpc {
 
 constexpr int kCircuitWarps = 8;
@@ -36,6 +38,7 @@ __device__ __forceinline__ float warp_lse(float val, bool has) {
 __global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __restrict__ logw,
                                   float* __restrict__ out, float* __restrict__ prefix, int W, int wpp, int n, int r,
                                   int sum_rows) {
+  grid_dependency_wait();   // G and log omega come from the kernel before this one
   const int w = blockIdx.x * kCircuitWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (w >= W) return;
@@ -211,6 +214,7 @@ __global__ void circuit_btree_kernel(const float* __restrict__ G, const float* _
                                      float* __restrict__ out, float* __restrict__ prefix, unsigned* work_counter,
                                      int W, int wpp, int n, int r, int sum_rows) {
   extern __shared__ __align__(16) float sm[];
+  grid_dependency_wait();   // G, log omega and the zeroed work counter come from the kernels before this one
   const int wib = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   float* prod = sm + static_cast<size_t>(wib) * btree_warp_floats(n, r, PREFIX);
@@ -289,37 +293,43 @@ __global__ void circuit_btree_kernel(const float* __restrict__ G, const float* _
 // tables[p * table_stride + (i-1) r^2 + a r + k]. Contextual transitions (App. H): tables = log omega + r and
 // table_stride = sum_rows, 28 KB per position at n = 8, r = 32, read exactly once from HBM, which bounds the kernel.
 // Static transitions: table_stride = 0, the one set of tables stays in L2. One warp per window, lane = state; table
-// i+1 is copied into shared memory by cp.async while table i is reduced.
-// Shared memory per warp: 2 * r * r + 32 floats. With `prefix` (may be NULL) also writes prefix[w, i] = LSE_k alpha_i[k].
+// i+1 is copied into shared memory by cp.async while table i is reduced (kHmmDepth buffers per warp).
+// Shared memory per warp: kHmmDepth * r * r + 32 floats. With `prefix` (may be NULL) also writes prefix[w, i] = LSE_k alpha_i[k].
+constexpr int kHmmDepth = 2;   // table buffers per warp (deeper pipelines were measured and bought nothing)
 __global__ void circuit_hmm_stream_kernel(const float* __restrict__ G, const float* __restrict__ logw,
                                           const float* __restrict__ tables, int table_stride,
                                           float* __restrict__ out, float* __restrict__ prefix, unsigned* work_counter,
                                           int W, int wpp, int n, int r, int sum_rows) {
   extern __shared__ __align__(16) float sm[];
+  grid_dependency_wait();   // G, log omega and the zeroed work counter come from the kernels before this one
   const int lane = threadIdx.x & 31;
   const int rr = r * r;
-  float* tabs = sm + static_cast<size_t>(threadIdx.x >> 5) * (2 * rr + 32);
-  float* evec = tabs + 2 * rr;
+  float* tabs = sm + static_cast<size_t>(threadIdx.x >> 5) * (kHmmDepth * rr + 32);
+  float* evec = tabs + kHmmDepth * rr;
   const bool has = lane < r;
   for (int w = next_window(work_counter, lane); w < W; w = next_window(work_counter, lane)) {
     const float* g = G + static_cast<size_t>(w) * n * r;
     const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
     const float* tb = tables + static_cast<size_t>(w / wpp) * table_stride;   // logA_1 .. logA_{n-1} of this position
-    if (n > 1) warp_table_load_async(tabs, tb, rr, lane);
+    // kHmmDepth - 1 tables are in flight ahead of the one being reduced; every step commits exactly one copy group (an
+    // empty one once the tables run out), so "all but the newest kHmmDepth - 1 groups" always means "table i has landed"
+#pragma unroll
+    for (int s = 0; s < kHmmDepth - 1; ++s) {
+      if (s < n - 1) warp_table_load_async(tabs + s * rr, tb + static_cast<size_t>(s) * rr, rr, lane);
+      else cp_async_commit();
+    }
     float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
     for (int i = 1; i < n; ++i) {
-      if (i + 1 < n) {
-        warp_table_load_async(tabs + (i & 1) * rr, tb + static_cast<size_t>(i) * rr, rr, lane);
-        cp_async_wait<1>();
-      } else {
-        cp_async_wait<0>();
-      }
+      const int nxt = i - 1 + kHmmDepth - 1;                 // index of the table to fetch now
+      if (nxt < n - 1) warp_table_load_async(tabs + (nxt % kHmmDepth) * rr, tb + static_cast<size_t>(nxt) * rr, rr, lane);
+      else cp_async_commit();
+      cp_async_wait<kHmmDepth - 1>();
       __syncwarp();                                      // table i is in shared memory for every lane
       if (prefix != nullptr) {
         const float pre = warp_lse(alpha, has);
         if (lane == 0) prefix[static_cast<size_t>(w) * n + i - 1] = pre;
       }
-      const float* A = tabs + ((i - 1) & 1) * rr;
+      const float* A = tabs + ((i - 1) % kHmmDepth) * rr;
       const float gi = has ? g[i * r + lane] : 0.f;
       float m = alpha;
 #pragma unroll
@@ -332,14 +342,16 @@ __global__ void circuit_hmm_stream_kernel(const float* __restrict__ G, const flo
       if (has) {
         if ((r & 3) == 0) {
           const float4* e4 = reinterpret_cast<const float4*>(evec);
-#pragma unroll 2
+          float s1 = 0.f, s2 = 0.f, s3 = 0.f;              // four independent accumulation chains
+#pragma unroll 4
           for (int a = 0; a < r; a += 4) {
             const float4 ev = e4[a >> 2];
             s = fmaf(ev.x, __expf(A[a * r + lane]), s);
-            s = fmaf(ev.y, __expf(A[(a + 1) * r + lane]), s);
-            s = fmaf(ev.z, __expf(A[(a + 2) * r + lane]), s);
-            s = fmaf(ev.w, __expf(A[(a + 3) * r + lane]), s);
+            s1 = fmaf(ev.y, __expf(A[(a + 1) * r + lane]), s1);
+            s2 = fmaf(ev.z, __expf(A[(a + 2) * r + lane]), s2);
+            s3 = fmaf(ev.w, __expf(A[(a + 3) * r + lane]), s3);
           }
+          s = (s + s1) + (s2 + s3);
         } else {
           for (int a = 0; a < r; ++a) s = fmaf(evec[a], __expf(A[a * r + lane]), s);
         }

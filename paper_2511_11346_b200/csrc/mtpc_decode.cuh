@@ -102,6 +102,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_decode_gemm_kernel(const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+  grid_launch_dependents();   // the per-slot kernel may be scheduled as SMs free up; it waits for this grid's results
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -299,9 +300,13 @@ constexpr int kSlotMaxPerLane = 16;   // v <= 512
 __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     int family, const float* __restrict__ logits, const float* __restrict__ logw, const float* __restrict__ logA,
     const float* __restrict__ uniforms, int* __restrict__ out_bytes, float* __restrict__ G,
-    float* __restrict__ unit_lse_out, unsigned* status, int wpp, int n, int r, int v, int sum_rows, int logA_stride,
-    int tables_in_smem) {
+    float* __restrict__ unit_lse_out, unsigned* status, unsigned* work_counter, int wpp, int n, int r, int v,
+    int sum_rows, int logA_stride, int tables_in_smem) {
   extern __shared__ __align__(16) float sm[];
+  grid_launch_dependents();
+  grid_dependency_wait();     // the logits and log omega come from the kernel before this one
+  if (work_counter != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0)
+    *work_counter = 0;        // the circuit kernel that follows hands out its windows through this counter
   float* unit_max = sm;
   float* unit_lse = sm + r;
   float* tabs = sm + ((2 * r + 3) & ~3);
