@@ -143,3 +143,37 @@ def test_large_vocabulary_heads_evaluate_and_train_but_do_not_draft(family, n, r
         dh.draft_sample(1)
     assert e.value.code == -3
     dh.close()
+
+
+def test_backward_argument_checks():
+    import ctypes
+    from paper_2511_11346_b200 import binding as B
+    wl = I.make_workload("bwd_args", I.HeadShape(I.HMM, 3, 4, 32, 64), 10, seed=12, weight_std=0.3)
+    dh = DeviceHead(wl)
+    lib = B.lib()
+    need = ctypes.c_size_t(0)
+    assert lib.mtpc_backward_workspace_bytes(ctypes.byref(dh.head.cfg), 10, ctypes.byref(need)) == 0 and need.value % 256 == 0
+    assert lib.mtpc_backward_workspace_bytes(ctypes.byref(dh.head.cfg), 0, ctypes.byref(need)) == -2
+    assert lib.mtpc_backward_workspace_bytes(None, 10, ctypes.byref(need)) == -1
+    lib.mtpc_backward_workspace_bytes(ctypes.byref(dh.head.cfg), 10, ctypes.byref(need))
+    s = wl.shape
+    f32 = dict(dtype=torch.float32, device="cuda")
+    h, t = dh.hidden_device(), torch.from_numpy(wl.targets).cuda()
+    w = torch.ones(10, **f32)
+    ws = torch.empty(need.value, dtype=torch.uint8, device="cuda")
+    lp, dhid = torch.empty(10, **f32), torch.empty((10, s.d), **f32)
+    dW, dR, dT = torch.empty((s.n, s.r, s.v, s.d), **f32), torch.empty((s.sum_rows, s.d), **f32), torch.empty((2, 4, 4), **f32)
+    st = torch.cuda.current_stream().cuda_stream
+    call = lambda **kw: lib.mtpc_window_logprob_backward(
+        dh.head.handle, kw.get("h", h.data_ptr()), t.data_ptr(), kw.get("T", 10), w.data_ptr(), kw.get("ws", ws.data_ptr()),
+        kw.get("wsb", need.value), lp.data_ptr(), dhid.data_ptr(), dW.data_ptr(), dR.data_ptr(), kw.get("dT", dT.data_ptr()), st)
+    assert call() == 0
+    assert call(T=0) == 0
+    assert call(T=11) == -2                     # more positions than the head was created for
+    assert call(h=None) == -1
+    assert call(dT=None) == -1                  # a static HMM needs room for the transition gradients
+    assert call(wsb=need.value - 256) == -4     # workspace too small
+    assert call(ws=ws.data_ptr() + 8) == -4     # misaligned
+    torch.cuda.synchronize()
+    assert dh.head.mtpc_get_status() == 0
+    dh.close()
