@@ -66,6 +66,60 @@ __global__ void circuit_cp_backward_kernel(const float* __restrict__ G, const fl
   }
 }
 
+// ---------------------------------------------------------------- gradient of one row of a transition table
+// Lane = row (the conditioning value). For every column b: out[b] = wt * (exp(base + row[b] + pc[b]) - exp(row[b]) * gam),
+// i.e. pairwise posterior minus conditional probability times the posterior of the conditioning value (the gradient
+// with respect to the row's logits). `row` and `pc` are in shared memory; the results go either to a bf16 row in global
+// memory (contextual tables: one set per position) or, by atomic adds, to an fp32 row in shared memory (static tables,
+// summed over the windows). R a multiple of 4: float4 reads rotated by the lane (conflict-free), 8-byte stores.
+template <int R>
+__device__ __forceinline__ void row_grad_vec(const float* row, const float* pc, float base, float gam, float wt, int lane,
+                                             __nv_bfloat16* dst, float* acc_row) {
+  constexpr int Q = R / 4;
+  const float4* row4 = reinterpret_cast<const float4*>(row);
+  const float4* pc4 = reinterpret_cast<const float4*>(pc);
+#pragma unroll
+  for (int q = 0; q < Q; ++q) {
+    const int j = (q + lane) & (Q - 1);
+    const float4 a = row4[j];
+    const float4 p = pc4[j];
+    const float ox = wt * (__expf(base + a.x + p.x) - __expf(a.x) * gam);
+    const float oy = wt * (__expf(base + a.y + p.y) - __expf(a.y) * gam);
+    const float oz = wt * (__expf(base + a.z + p.z) - __expf(a.z) * gam);
+    const float ow = wt * (__expf(base + a.w + p.w) - __expf(a.w) * gam);
+    if (acc_row != nullptr) {
+      atomicAdd(acc_row + 4 * j, ox);
+      atomicAdd(acc_row + 4 * j + 1, oy);
+      atomicAdd(acc_row + 4 * j + 2, oz);
+      atomicAdd(acc_row + 4 * j + 3, ow);
+    } else {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(ox, oy);
+      __nv_bfloat162 hi = __floats2bfloat162_rn(oz, ow);
+      uint2 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(dst + 4 * j) = pk;
+    }
+  }
+}
+__device__ __forceinline__ void row_grad(const float* row, const float* pc, float base, float gam, float wt, int lane, int r,
+                                         __nv_bfloat16* dst, float* acc_row) {
+  switch (r) {
+    case 32: row_grad_vec<32>(row, pc, base, gam, wt, lane, dst, acc_row); return;
+    case 16: row_grad_vec<16>(row, pc, base, gam, wt, lane, dst, acc_row); return;
+    case 8: row_grad_vec<8>(row, pc, base, gam, wt, lane, dst, acc_row); return;
+    case 4: row_grad_vec<4>(row, pc, base, gam, wt, lane, dst, acc_row); return;
+    default: break;
+  }
+  for (int q = 0; q < r; ++q) {                       // start at column `lane` (r a power of two): conflict-free
+    const int b = (q + lane) & (r - 1);
+    const float la = row[b];
+    const float o = wt * (__expf(base + la + pc[b]) - __expf(la) * gam);
+    if (acc_row != nullptr) atomicAdd(acc_row + b, o);
+    else dst[b] = __float2bfloat16_rn(o);
+  }
+}
+
 // ---------------------------------------------------------------- circuit backward: HMM (Eq. HMM), forward-backward
 // Forward messages alpha_i (kept for all steps in shared memory), backward messages
 // beta_{i-1}[a] = LSE_b(logA_i[a][b] + G[i][b] + beta_i[b]). Posterior of the state: gamma_i = exp(alpha_i + beta_i - log q)
@@ -125,8 +179,7 @@ __global__ void circuit_hmm_backward_kernel(const float* __restrict__ G, const f
       cvec[lane] = has ? __expf(alpha - m) : 0.f;
       __syncwarp();
       if (has) {
-        float s = 0.f;
-        for (int a = 0; a < r; ++a) s = fmaf(cvec[a], __expf(A[a * r + lane]), s);
+        const float s = hmm_matvec(cvec, A, lane, r);
         alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : g[i * r + lane] + m + __logf(s);
         alphas[i * r + lane] = alpha;
       }
@@ -156,22 +209,9 @@ __global__ void circuit_hmm_backward_kernel(const float* __restrict__ G, const f
         const float al = alphas[(i - 1) * r + lane];
         const float gam_prev = __expf(al + beta_prev - logq);
         const float* row = A + lane * r;
-        // the row is walked starting at column `lane` (r is a power of two): 32 lanes, 32 different banks
-        if (is_static) {
-          float* dst = acc + static_cast<size_t>(i - 1) * rr + lane * r;
-          for (int q = 0; q < r; ++q) {
-            const int b = (q + lane) & (r - 1);
-            const float la = row[b];
-            atomicAdd(dst + b, wt * (__expf(al + la + cvec[b] - logq) - __expf(la) * gam_prev));
-          }
-        } else {
-          __nv_bfloat16* dst = dsum + static_cast<size_t>(w) * dsum_pitch + r + static_cast<size_t>(i - 1) * rr + lane * r;
-          for (int q = 0; q < r; ++q) {
-            const int b = (q + lane) & (r - 1);
-            const float la = row[b];
-            dst[b] = __float2bfloat16_rn(wt * (__expf(al + la + cvec[b] - logq) - __expf(la) * gam_prev));
-          }
-        }
+        row_grad(row, cvec, al - logq, gam_prev, wt, lane, r,
+                 is_static ? nullptr : dsum + static_cast<size_t>(w) * dsum_pitch + r + static_cast<size_t>(i - 1) * rr + lane * r,
+                 is_static ? acc + static_cast<size_t>(i - 1) * rr + lane * r : nullptr);
       }
       beta = beta_prev;
       __syncwarp();                                                      // cvec and the table buffer are free again
@@ -283,14 +323,8 @@ __global__ void circuit_btree_backward_kernel(const float* __restrict__ G, const
         // gradient of the child's table: lane z (row), over the child's values b
         const float in_z = cur[lane];
         const float gam_parent = __expf(U[j * r + lane] + prod[j * r + lane] - logq);
-        const float* row = tab + lane * r;
-        const float* pc = prod + c * r;
-        __nv_bfloat16* dst = ds + r + static_cast<size_t>(c - 1) * rr + lane * r;
-        for (int q = 0; q < r; ++q) {                     // start at column `lane`: conflict-free (r a power of two)
-          const int b = (q + lane) & (r - 1);
-          const float lo = row[b];
-          dst[b] = __float2bfloat16_rn(wt * (__expf(in_z + lo + pc[b] - logq) - __expf(lo) * gam_parent));
-        }
+        row_grad(tab + lane * r, prod + c * r, in_z - logq, gam_parent, wt, lane, r,
+                 ds + r + static_cast<size_t>(c - 1) * rr + lane * r, nullptr);
       }
       __syncwarp();
     }

@@ -285,6 +285,28 @@ __global__ void circuit_btree_kernel(const float* __restrict__ G, const float* _
   }
 }
 
+// sum_a e[a] * exp(A[a][lane]) for lane < r: e (r floats) and the table A [r, r] are in shared memory. Every lane reads
+// four e's per request (a broadcast) and keeps four independent accumulation chains.
+__device__ __forceinline__ float hmm_matvec(const float* evec, const float* A, int lane, int r) {
+  float s = 0.f;
+  if ((r & 3) == 0) {
+    const float4* e4 = reinterpret_cast<const float4*>(evec);
+    float s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll 4
+    for (int a = 0; a < r; a += 4) {
+      const float4 ev = e4[a >> 2];
+      s = fmaf(ev.x, __expf(A[a * r + lane]), s);
+      s1 = fmaf(ev.y, __expf(A[(a + 1) * r + lane]), s1);
+      s2 = fmaf(ev.z, __expf(A[(a + 2) * r + lane]), s2);
+      s3 = fmaf(ev.w, __expf(A[(a + 3) * r + lane]), s3);
+    }
+    s = (s + s1) + (s2 + s3);
+  } else {
+    for (int a = 0; a < r; ++a) s = fmaf(evec[a], __expf(A[a * r + lane]), s);
+  }
+  return s;
+}
+
 // Eq. (HMM), forward recursion over the window: alpha_0[k] = log pi[k] + G[0,k];
 // alpha_i[k] = G[i,k] + LSE_a(alpha_{i-1}[a] + logA_i[a][k]); out = LSE_k alpha_{n-1}[k].  r <= 32.
 // The inner log-sum-exp is taken as one scaled matrix-vector product per step: with m = max_a alpha_{i-1}[a],
@@ -338,23 +360,8 @@ __global__ void circuit_hmm_stream_kernel(const float* __restrict__ G, const flo
       // (a broadcast) instead of one shuffle each
       evec[lane] = has ? __expf(alpha - m) : 0.f;
       __syncwarp();
-      float s = 0.f;
       if (has) {
-        if ((r & 3) == 0) {
-          const float4* e4 = reinterpret_cast<const float4*>(evec);
-          float s1 = 0.f, s2 = 0.f, s3 = 0.f;              // four independent accumulation chains
-#pragma unroll 4
-          for (int a = 0; a < r; a += 4) {
-            const float4 ev = e4[a >> 2];
-            s = fmaf(ev.x, __expf(A[a * r + lane]), s);
-            s1 = fmaf(ev.y, __expf(A[(a + 1) * r + lane]), s1);
-            s2 = fmaf(ev.z, __expf(A[(a + 2) * r + lane]), s2);
-            s3 = fmaf(ev.w, __expf(A[(a + 3) * r + lane]), s3);
-          }
-          s = (s + s1) + (s2 + s3);
-        } else {
-          for (int a = 0; a < r; ++a) s = fmaf(evec[a], __expf(A[a * r + lane]), s);
-        }
+        const float s = hmm_matvec(evec, A, lane, r);
         alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : gi + m + __logf(s);
       }
       __syncwarp();                                      // the buffers may be overwritten
