@@ -2,7 +2,7 @@
 """Benchmark of the MtPC head on B200: window log-likelihood positions/s on the training-shaped CP workload
 (8192 positions, d=4096, n=8, r=16, v=320), plus draft windows/s on one decode cell.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|5] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1|2|3|5|6] [--impl reference]
 
 One step = one mtpc_window_logprob call over the whole batch (projection GEMM with fused softmax/gather
 epilogue + circuit evaluation). Prints ONE JSON line on rank 0. With N > 1 (launched by torchrun, one process
@@ -34,7 +34,7 @@ UNIT = "positions/s"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one projection-kernel launch, from the ncu capture
 # summarised in profiles/ (captured on the full configuration). None = not captured.
-NCU_TRAFFIC_BYTES = {1: 922_700_000, 2: None, 3: None, 5: None}   # configs[1]: mean of 925.1 and 920.3 MB (profiles/)
+NCU_TRAFFIC_BYTES = {1: 922_700_000, 2: None, 3: None, 5: None, 6: None}   # configs[1]: mean of 925.1 and 920.3 MB (profiles/)
 
 
 def workload_name(idx: int, wl) -> str:
@@ -46,7 +46,7 @@ def workload_name(idx: int, wl) -> str:
 def algorithmic_flops(wl) -> float:
     """2 d (n r v + S r) per position: the method's own projection work (Table 3's 'MTP head linear')."""
     s = wl.shape
-    return 2.0 * s.d * (s.n * s.r * s.v + s.sum_rows) * wl.T
+    return 2.0 * s.d * (s.n * s.r * s.symbols + s.sum_rows) * wl.T      # padding symbols earn no credit
 
 
 def load_peaks():
@@ -411,8 +411,9 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3, 5],
-                    help="1 CP (the metric's configuration), 2 HMM, 3 binary tree, 5 HMM with contextual transitions")
+    ap.add_argument("--workload", type=int, default=1, choices=[1, 2, 3, 5, 6],
+                    help="1 CP (the metric's configuration), 2 HMM, 3 binary tree, 5 HMM with contextual transitions, "
+                         "6 CP with the byte-level Llama shape (d=3072, 268 symbols padded to 272)")
     ap.add_argument("--ref-positions", type=int, default=None,
                     help="positions the CPU oracle processes per step / for the cpu_baseline sample")
     ap.add_argument("--no-draft", action="store_true", help="skip the decode-cell draft measurement")

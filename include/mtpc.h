@@ -78,6 +78,11 @@ typedef struct {
   int32_t max_positions;       /* upper bound on T (log-prob) and P (draft) per call                   */
   int32_t max_windows_per_pos; /* upper bound on wpp (>= 1; <= 64)                                     */
   uint32_t flags;              /* 0 or MTPC_FLAG_HMM_CONTEXTUAL                                        */
+  int32_t v_valid;             /* 0, or the number of symbols that exist when the vocabulary is not a
+                                  multiple of 16 (v - 16 < v_valid <= v; a byte-level Llama has 268: v = 272):
+                                  every unit of W_emit keeps v rows, the last v - v_valid of them are padding
+                                  whose values are ignored (logit -inf: no mass, never sampled, no gradient);
+                                  targets and bytes are < v_valid; target_probs rows keep v entries          */
 } mtpc_config;
 
 /* Bytes of device workspace a head with this configuration needs (a multiple of 256). */

@@ -32,7 +32,7 @@ ERR_STATE = -8
 class MtpcConfig(ctypes.Structure):
     _fields_ = [("family", ctypes.c_int32), ("n", ctypes.c_int32), ("r", ctypes.c_int32), ("v", ctypes.c_int32),
                 ("d", ctypes.c_int32), ("io_dtype", ctypes.c_int32), ("max_positions", ctypes.c_int32),
-                ("max_windows_per_pos", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+                ("max_windows_per_pos", ctypes.c_int32), ("flags", ctypes.c_uint32), ("v_valid", ctypes.c_int32)]
 
 
 class MtpcError(RuntimeError):
@@ -124,9 +124,9 @@ class MtpcHead:
     """Owns the opaque head handle and keeps the tensors the head points into alive."""
 
     def __init__(self, family: int, n: int, r: int, v: int, d: int, io_dtype: int, max_positions: int,
-                 max_windows_per_pos: int, W_emit, W_sum, T_static=None, stream=None, flags: int = 0):
+                 max_windows_per_pos: int, W_emit, W_sum, T_static=None, stream=None, flags: int = 0, v_valid: int = 0):
         import torch
-        self.cfg = MtpcConfig(family, n, r, v, d, io_dtype, max_positions, max_windows_per_pos, flags)
+        self.cfg = MtpcConfig(family, n, r, v, d, io_dtype, max_positions, max_windows_per_pos, flags, v_valid)
         nbytes = mtpc_workspace_bytes(self.cfg)
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=W_emit.device)
         self._keep = (W_emit, W_sum, T_static)

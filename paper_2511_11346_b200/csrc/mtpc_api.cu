@@ -53,6 +53,7 @@ struct Layout {
   size_t off_prefix, off_partial, off_sum_bias;   // training loss: prefix log-marginals [max_positions, n], per-sequence terms
   int decode_max_p;     // positions the few-position draft path can take (0: path not available)
   bool can_draft;       // v <= 512: the sampling kernels hold a whole input unit on chip
+  bool can_draft_many;  // the sampling epilogue of the projection kernel can tile a unit (draft of more than 128 positions)
   size_t off_h_hidden, off_h_targets, off_h_uniforms, off_h_bytes, off_h_out;
   size_t total;
 };
@@ -88,6 +89,7 @@ int plan(const mtpc_config& c, Layout* L) {
   if (c.family == MTPC_BTREE && (c.n < 2 || !is_pow2(c.n))) return MTPC_ERR_UNSUPPORTED;
   if (c.d % kBlockK != 0) return MTPC_ERR_UNSUPPORTED;
   if (c.v % 16 != 0) return MTPC_ERR_UNSUPPORTED;
+  if (c.v_valid != 0 && (c.v_valid > c.v || c.v_valid <= c.v - 16)) return MTPC_ERR_SHAPE;
   if (static_cast<int64_t>(c.n) * c.r * c.v > (1ll << 30)) return MTPC_ERR_SHAPE;
 
   L->S = (c.family == MTPC_BTREE) ? 1 + (c.n - 2) * c.r : (ctx ? 1 + (c.n - 1) * c.r : 1);
@@ -109,10 +111,12 @@ int plan(const mtpc_config& c, Layout* L) {
     L->sm.group_units = 1;
     L->sm.group_tiles = chunks;
     L->sm.num_groups = emit_units;
-    if (!fit_tiling(&L->sm, sum_cols) || L->sm.num_slots < chunks) return MTPC_ERR_UNSUPPORTED;
+    // (no such split, e.g. v = 272 = 17 x 16: only the few-position draft path, which needs none, is available)
+    L->can_draft_many = fit_tiling(&L->sm, sum_cols) && L->sm.num_slots >= chunks;
   } else {
-    memset(&L->sm, 0, sizeof(L->sm));
+    L->can_draft_many = false;
   }
+  if (!L->can_draft_many) memset(&L->sm, 0, sizeof(L->sm));
   // log-likelihood: 256-column tiles; a group is the shortest run of whole units that is a whole number of tiles
   const int lcm = c.v / gcd_int(c.v, 256) * 256;
   L->lp.tile_cols = 256;
@@ -215,6 +219,7 @@ namespace {
 template <typename T>
 T* at(mtpc_head* h, size_t off) { return reinterpret_cast<T*>(h->ws + off); }
 
+int valid_symbols(const mtpc_config& c) { return c.v_valid > 0 ? c.v_valid : c.v; }
 bool is_ctx(const mtpc_head* h) { return (h->cfg.flags & MTPC_FLAG_HMM_CONTEXTUAL) != 0; }
 // HMM transition log-probabilities as the kernels read them: position p's tables start at base + p * stride.
 // Static transitions: one set in the workspace, stride 0. Contextual (App. H): the sum units after the first one
@@ -311,6 +316,7 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
     p.m_block = (p.m_tiles + nblocks - 1) / nblocks;
   }
   p.n = c.n; p.r = c.r; p.v = c.v;
+  p.vv = valid_symbols(c);
   p.emit_units = c.n * c.r;
   p.num_groups = with_emit ? tl.num_groups : 0;
   p.group_units = tl.group_units;
@@ -522,7 +528,7 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
       launch_kernel(draft_slot_kernel, dim3(c.n, P), kSlotThreads, in_smem ? with_tables : base, st, h->ring == 0, c.family,
                     at<float>(h, L.off_logits), at<float>(h, L.off_logw), hmm_tables(h), uniforms, out_bytes,
                     at<float>(h, L.off_G), at<float>(h, L.off_unit_lse), at<unsigned>(h, L.off_status),
-                    at<unsigned>(h, L.off_status) + kWorkCounterWord, wpp, c.n, c.r, c.v, L.sum_rows,
+                    at<unsigned>(h, L.off_status) + kWorkCounterWord, wpp, c.n, c.r, c.v, valid_symbols(c), L.sum_rows,
                     hmm_table_stride(h), in_smem);
     }
     h->launches++;
@@ -534,6 +540,7 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
     pt.end();
     return rc;
   }
+  if (!L.can_draft_many) return MTPC_ERR_UNSUPPORTED;
   // 1. sum-unit weights (Sec. 3.3) -> 2. latent draws at the sum units (Algorithm 1)
   pt.begin();
   rc = launch_gemm(h, kModeLogprob, hb, P, 1, false, true, nullptr, nullptr, nullptr, st);
@@ -752,7 +759,7 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   if (check_launch() != MTPC_OK) { delete h; return MTPC_ERR_CUDA; }
   const uint64_t emit_rows = static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v;
   rc = make_tmap(&h->tm_emit_lp, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols);
-  if (rc == MTPC_OK && L.can_draft) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
+  if (rc == MTPC_OK && L.can_draft_many) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols);
   h->decode_tile_rows = decode_tile_rows(static_cast<long long>(emit_rows), h->num_sms);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_dec, h->W_emit_bf16, emit_rows, cfg->d, h->decode_tile_rows);
@@ -824,7 +831,8 @@ int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32
   spec_accept_kernel<<<(W + kAcceptWarps - 1) / kAcceptWarps, kAcceptWarps * 32, smem, st>>>(
       c.family, at<float>(head, L.off_logits), at<float>(head, L.off_unit_lse), at<float>(head, L.off_logw),
       hmm_tables(head), draft_bytes, prefix_logprob, target_probs, accept_uniforms, out_accepted,
-      out_next_byte, at<unsigned>(head, L.off_status), W, wpp, c.n, c.r, c.v, L.sum_rows, hmm_table_stride(head));
+      out_next_byte, at<unsigned>(head, L.off_status), W, wpp, c.n, c.r, c.v, valid_symbols(c), L.sum_rows,
+      hmm_table_stride(head));
   head->launches++;
   pt.end();
   return check_launch();

@@ -300,7 +300,7 @@ constexpr int kSlotMaxPerLane = 16;   // v <= 512
 __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     int family, const float* __restrict__ logits, const float* __restrict__ logw, const float* __restrict__ logA,
     const float* __restrict__ uniforms, int* __restrict__ out_bytes, float* __restrict__ G,
-    float* __restrict__ unit_lse_out, unsigned* status, unsigned* work_counter, int wpp, int n, int r, int v,
+    float* __restrict__ unit_lse_out, unsigned* status, unsigned* work_counter, int wpp, int n, int r, int v, int vv,
     int sum_rows, int logA_stride, int tables_in_smem) {
   extern __shared__ __align__(16) float sm[];
   grid_launch_dependents();
@@ -341,7 +341,7 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
 #pragma unroll
     for (int q = 0; q < kSlotMaxPerLane; ++q) {
       const int b = lane + 32 * q;
-      xv[q] = b < v ? x[b] : -CUDART_INF_F;
+      xv[q] = b < vv ? x[b] : -CUDART_INF_F;   // [vv, v): padding symbols
     }
     float m = xv[0];
 #pragma unroll
@@ -396,7 +396,7 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
       const int b0 = lane * per;
       float ev[kSlotMaxPerLane];
 #pragma unroll
-      for (int q = 0; q < kSlotMaxPerLane; ++q) ev[q] = (q < per && b0 + q < v) ? x[b0 + q] : -CUDART_INF_F;
+      for (int q = 0; q < kSlotMaxPerLane; ++q) ev[q] = (q < per && b0 + q < vv) ? x[b0 + q] : -CUDART_INF_F;
       float part = 0.f;
 #pragma unroll
       for (int q = 0; q < kSlotMaxPerLane; ++q) {
@@ -407,7 +407,7 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
       const float total = __shfl_sync(kFull, incl, 31);
       const float thr = ub * total;
       const unsigned hit = __ballot_sync(kFull, thr < incl);
-      byte = v - 1;   // rounding may leave no index: the last one
+      byte = vv - 1;   // rounding may leave no index: the last one
       if (hit) {
         const int src = __ffs(hit) - 1;
         int found = -1;
@@ -416,11 +416,11 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
           float cum = lane == 0 ? 0.f : before;
 #pragma unroll
           for (int q = 0; q < kSlotMaxPerLane; ++q)
-            if (found < 0 && q < per && b0 + q < v) {
+            if (found < 0 && q < per && b0 + q < vv) {
               cum += ev[q];
               if (thr < cum) found = b0 + q;
             }
-          if (found < 0) found = min(b0 + per, v) - 1;   // the lane's total passed the threshold: its last byte
+          if (found < 0) found = min(b0 + per, vv) - 1;   // the lane's total passed the threshold: its last byte
         }
         byte = __shfl_sync(kFull, found, src);
       }
@@ -456,7 +456,8 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
     int family, const float* __restrict__ logits, const float* __restrict__ unit_lse, const float* __restrict__ logw,
     const float* __restrict__ logA, const int* __restrict__ bytes, const float* __restrict__ prefix,
     const float* __restrict__ target, const float* __restrict__ uniforms, int* __restrict__ out_accepted,
-    int* __restrict__ out_next, unsigned* status, int W, int wpp, int n, int r, int v, int sum_rows, int logA_stride) {
+    int* __restrict__ out_next, unsigned* status, int W, int wpp, int n, int r, int v, int vv, int sum_rows,
+    int logA_stride) {
   extern __shared__ float sm[];
   const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int w = blockIdx.x * kAcceptWarps + wib;
@@ -473,7 +474,7 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
   // ---- 1. acceptance tests
   bool bad_u = false, bad_x = false;
   for (int c = lane; c <= n; c += 32) bad_u |= !(u[c] >= 0.f && u[c] < 1.f);
-  for (int c = lane; c < n; c += 32) bad_x |= static_cast<unsigned>(x[c]) >= static_cast<unsigned>(v);
+  for (int c = lane; c < n; c += 32) bad_x |= static_cast<unsigned>(x[c]) >= static_cast<unsigned>(vv);
   bad_u = __any_sync(kFull, bad_u);
   bad_x = __any_sync(kFull, bad_x);
   if (bad_u || bad_x) {
@@ -500,7 +501,7 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
   const float* trow = tp + static_cast<size_t>(s) * v;
 
   if (s == n) {
-    for (int b = lane; b < v; b += 32) mres[b] = trow[b];
+    for (int b = lane; b < v; b += 32) mres[b] = b < vv ? trow[b] : 0.f;
   } else {
     // ---- 2. c[k]: log-weight of input unit k of slot s given the accepted bytes (lane = k)
     auto g_of = [&](int i) -> float {   // log phi_{i,lane}(x_i)
@@ -581,9 +582,9 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
       for (int k = 0; k < r; ++k) {
         const float ck = __shfl_sync(kFull, cprob, k);
         const float lk = __shfl_sync(kFull, ulse, k);
-        if (b < v) q = fmaf(ck, __expf(lrow[static_cast<size_t>(k) * v + b] - lk), q);
+        if (b < vv) q = fmaf(ck, __expf(lrow[static_cast<size_t>(k) * v + b] - lk), q);
       }
-      if (b < v) mres[b] = fmaxf(0.f, trow[b] - q);
+      if (b < v) mres[b] = b < vv ? fmaxf(0.f, trow[b] - q) : 0.f;   // padding symbols carry no mass
     }
   }
   __syncwarp();
@@ -598,7 +599,7 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
   const float total = __shfl_sync(kFull, incl, 31);
   const float thr = u[n] * total;
   const unsigned hit = __ballot_sync(kFull, thr < incl);
-  int byte = v - 1;   // rounding may leave no index: the last one
+  int byte = vv - 1;   // rounding may leave no index: the last one
   if (hit) {
     const int src = __ffs(hit) - 1;
     int found = -1;
@@ -606,11 +607,11 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
     if (lane == src) {
       float cum = lane == 0 ? 0.f : before;
       for (int q = 0; q < per && found < 0; ++q)
-        if (b0 + q < v) {
+        if (b0 + q < vv) {
           cum += mres[b0 + q];
           if (thr < cum) found = b0 + q;
         }
-      if (found < 0) found = min(b0 + per, v) - 1;
+      if (found < 0) found = min(b0 + per, vv) - 1;
     }
     byte = __shfl_sync(kFull, found, src);
   }

@@ -46,6 +46,7 @@ struct GemmParams {
   int T, m_tiles, kblocks;
   int m_block;                       // m-tiles per rasterisation block (see tile_coord)
   int n, r, v;
+  int vv;                            // symbols that exist (<= v, > v - 16): the columns [vv, v) of every unit are padding
   int emit_units;                    // n * r
   int num_groups;                    // emission groups in this launch (0: sum tiles only)
   int group_units;                   // emission units per full group (the last group may hold fewer)
@@ -160,6 +161,15 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int item) {
     c.ntiles = (c.nunits * p.v + p.tile_cols - 1) / p.tile_cols;
   }
   return c;
+}
+
+// Padding columns of a unit (vocabulary not a multiple of 16) count as logit = -inf: never the maximum, no mass.
+__device__ __forceinline__ void mask_padding(float (&x)[16], int col_in_unit, int vv) {
+  if (col_in_unit + 16 > vv) {
+#pragma unroll
+    for (int q = 0; q < 16; ++q)
+      if (col_in_unit + q >= vv) x[q] = -CUDART_INF_F;
+  }
 }
 
 // log-softmax over groups of R adjacent columns inside one 16-column batch (R in {1,2,4,8,16}).
@@ -401,6 +411,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
           for (int b = 0; b < nbatch && unit < units_end; ++b) {
             float x[16];
             tmem_ld16(tcol + b * 16, x);
+            mask_padding(x, col_in_unit, p.vv);
             float bm = x[0];
 #pragma unroll
             for (int q = 1; q < 16; ++q) bm = fmaxf(bm, x[q]);
@@ -441,7 +452,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
                   float* g = p.G + ((wrow0 + j) * p.n + slot_i) * p.r + k;
                   if (tj < 0) {
                     *g = 0.f;                                  // marginalised byte: the input unit sums to 1
-                  } else if (tj >= p.v) {
+                  } else if (tj >= p.vv) {
                     *g = CUDART_NAN_F;
                     atomicOr(p.status, kStatusBadTarget);
                   } else {
@@ -491,6 +502,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
           for (int b = 0; b < nbatch && unit < units_end; ++b) {
             float x[16];
             tmem_ld16(tcol + b * 16, x);
+            mask_padding(x, col_in_unit, p.vv);                         // padding columns: softmax 0, gradient 0
             const int col0 = tc.brow0 + t * tc.cols + b * 16;           // row of W_emit = column of the logit matrix
             const int rel = tgt - col_in_unit;
             __align__(16) __nv_bfloat16 o[16];
@@ -547,6 +559,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
             for (int b = 0; b < nbatch; ++b) {
               float x[16];
               tmem_ld16(tcol + b * 16, x);
+              mask_padding(x, c * tc.cols + b * 16, p.vv);
 #pragma unroll
               for (int q = 0; q < 16; ++q) m = fmaxf(m, x[q]);
             }
@@ -558,6 +571,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
             for (int b = 0; b < nbatch; ++b) {
               float x[16];
               tmem_ld16(tcol + b * 16, x);
+              mask_padding(x, c * tc.cols + b * 16, p.vv);
 #pragma unroll
               for (int q = 0; q < 16; ++q) total += fast_ex2(fmaf(x[q], kLog2e, -m2));
             }
@@ -568,7 +582,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
             if (j >= 0) uval = p.uniforms[(wrow0 + j) * (2 * p.n) + p.n + slot_i];
             const float thr = uval * total;
             float cum = 0.f;
-            int found = p.v - 1;   // rounding may leave no index: the last one
+            int found = p.vv - 1;   // rounding may leave no index: the last one
             bool hit = false;
             for (int c = 0; c < tc.ntiles; ++c) {
               const uint32_t tcol = lane_base + ((use + c) % p.num_slots) * p.slot_stride;
@@ -576,6 +590,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
                 float x[16];
                 tmem_ld16(tcol + b * 16, x);
                 const int col0 = c * tc.cols + b * 16;
+                mask_padding(x, col0, p.vv);
 #pragma unroll
                 for (int q = 0; q < 16; ++q) {
                   cum += fast_ex2(fmaf(x[q], kLog2e, -m2));

@@ -12,6 +12,7 @@ weights and data that are not available offline):
   3  BTree              T=4096 d=3072 n=16 r=32 v=256  bf16, uniform targets, + draft wpp=1
   4  decode sweep cells P in {1,8,64}, d=4096, v=320, CP r=16 / HMM r=32, n in {8,16}, wpp=16
   5  HMM with contextual transitions: as 2, plus (n-1) r r = 7168 transition rows in W_sum and a bias ~N(0,1) + 4 I
+  6  CP head shaped like the paper's byte-level Llama-3.2-3B (Table 4): d=3072, 268 symbols stored as v=272, n=8, r=16
 Hidden states ~N(0,1); every weight ~N(0, std=0.02); uniforms in [0,1) as fp32. For the acceptance stage the
 target model's conditionals are Dirichlet rows (target_rows) and its uniforms come from the same generator.
 """
@@ -37,6 +38,11 @@ class HeadShape:
     v: int
     d: int
     io_dtype: int = BF16
+    v_valid: int = 0          # symbols that exist when v is padded to a multiple of 16 (0: all v)
+
+    @property
+    def symbols(self) -> int:
+        return self.v_valid or self.v
 
     @property
     def num_sum_groups(self) -> int:
@@ -157,6 +163,8 @@ class Workload:
     hidden_raw: np.ndarray | None = None
     W_emit_raw: np.ndarray | None = None
     W_sum_raw: np.ndarray | None = None
+    W_emit_dev_q: np.ndarray | None = None   # padded vocabulary: what the device gets ([n, r, v, d], padding rows filled
+                                             # with noise); W_emit_q then holds the rows of the existing symbols only
 
 
 _last_weights: dict = {}     # the most recent head's weights (one entry: they can be GBs)
@@ -185,13 +193,16 @@ def make_workload(name: str, shape: HeadShape, T: int, seed: int, *, target_kind
         _last_weights.update(key=key, value=(W_emit, W_sum, T_static, W_emit_q, W_sum_q))
     targets = None
     if target_kind == "uniform":
-        targets = uniform_targets(seed, 5, (T, shape.n), shape.v)
+        targets = uniform_targets(seed, 5, (T, shape.n), shape.symbols)
     elif target_kind == "zipf":
-        targets = zipf_targets(seed, 5, (T, shape.n), shape.v)
+        targets = zipf_targets(seed, 5, (T, shape.n), shape.symbols)
     u = uniforms(seed, 6, (T * wpp, 2 * shape.n)) if wpp > 0 else None
     wl = Workload(name, shape, T, bf16_round(hidden), W_emit_q, W_sum_q, T_static, targets, wpp, u)
     if shape.io_dtype == F32:
         wl.hidden_raw, wl.W_emit_raw, wl.W_sum_raw = hidden, W_emit, W_sum
+    if shape.v_valid:
+        wl.W_emit_dev_q = W_emit_q
+        wl.W_emit_q = np.ascontiguousarray(W_emit_q[:, :, :shape.v_valid, :])
     return wl
 
 
@@ -212,6 +223,8 @@ def config_workload(idx: int, *, cell: tuple[int, int, int] | None = None, T: in
     if idx == 3:
         return make_workload("btree_train", HeadShape(BTREE, 16, 32, 256, 3072), T or 4096, seed,
                              target_kind="uniform", wpp=1)
+    if idx == 6:
+        return make_workload("cp_llama_byte", HeadShape(CP, 8, 16, 272, 3072, v_valid=268), T or 8192, seed, target_kind="zipf")
     if idx == 5:
         return make_workload("hmmctx_train", HeadShape(HMM_CTX, 8, 32, 320, 4096), T or 8192, seed, target_kind="zipf")
     if idx == 4:

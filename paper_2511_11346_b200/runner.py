@@ -32,13 +32,13 @@ class DeviceHead:
             self.W_emit = torch.from_numpy(wl.W_emit_raw).to(device)
             self.W_sum = torch.from_numpy(wl.W_sum_raw).to(device)
         else:
-            self.W_emit = to_device_bf16(wl.W_emit_q, device)
+            self.W_emit = to_device_bf16(wl.W_emit_q if wl.W_emit_dev_q is None else wl.W_emit_dev_q, device)
             self.W_sum = to_device_bf16(wl.W_sum_q, device)
         self.T_static = torch.from_numpy(np.ascontiguousarray(wl.T_static)).to(device) if wl.T_static is not None else None
         ctx = s.family == I.HMM_CTX
         self.head = B.MtpcHead(B.MTPC_HMM if ctx else s.family, s.n, s.r, s.v, s.d, s.io_dtype,
                                max_positions or max(wl.T, 1), max_wpp or max(wl.wpp, 1), self.W_emit, self.W_sum,
-                               self.T_static, flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0)
+                               self.T_static, flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0, v_valid=s.v_valid)
 
     def hidden_device(self, rows=None):
         import torch

@@ -28,7 +28,7 @@ def test_library_exports_every_declared_symbol():
 
 def cfg(**kw):
     base = dict(family=B.MTPC_CP, n=8, r=16, v=320, d=4096, io_dtype=B.MTPC_BF16, max_positions=8192,
-                max_windows_per_pos=1, flags=0)
+                max_windows_per_pos=1, flags=0, v_valid=0)
     base.update(kw)
     return B.MtpcConfig(*[base[f] for f, _ in B.MtpcConfig._fields_])
 
@@ -47,6 +47,8 @@ def test_workspace_bytes_for_the_named_configs():
     assert code == 0 and nb3 >= 4096 * (1 + 14 * 32) * 32 * 4
     code, nb5 = ws(cfg(family=B.MTPC_HMM, r=32, flags=B.MTPC_FLAG_HMM_CONTEXTUAL))
     assert code == 0 and nb5 >= 8192 * (1 + 7 * 32) * 32 * 4   # contextual transitions: a table set per position
+    code, nbp = ws(cfg(v=272, v_valid=268, d=3072))                   # byte-level Llama head: 268 symbols padded to 272
+    assert code == 0 and nbp > 0
     code, nbv = ws(cfg(v=32768, r=2, n=2, max_positions=1024))        # large vocabularies plan (evaluation / training only)
     assert code == 0 and nbv > 0
     code, nb0 = ws(cfg(n=4, r=8, v=256, d=256, io_dtype=B.MTPC_F32, max_positions=256))
@@ -55,9 +57,10 @@ def test_workspace_bytes_for_the_named_configs():
 
 @pytest.mark.parametrize("kw,code", [
     (dict(family=3), -2), (dict(n=0), -2), (dict(io_dtype=2), -2), (dict(max_positions=0), -2),
+    (dict(v=272, v_valid=256), -2), (dict(v=272, v_valid=273), -2), (dict(v_valid=-3), -2),
     (dict(flags=1), -3), (dict(flags=2), -3), (dict(family=B.MTPC_BTREE, n=8, r=8, flags=1), -3), (dict(r=3), -3), (dict(r=256), -3), (dict(family=B.MTPC_HMM, r=64), -3),
     (dict(family=B.MTPC_BTREE, n=6, r=8), -3), (dict(family=B.MTPC_BTREE, n=1, r=8), -3), (dict(d=100), -3),
-    (dict(v=100), -3), (dict(v=272), -3), (dict(n=65), -3), (dict(max_windows_per_pos=65), -3),
+    (dict(v=100), -3), (dict(n=65), -3), (dict(max_windows_per_pos=65), -3),
 ])
 def test_bad_configurations_are_refused(kw, code):
     got, _ = ws(cfg(**kw))

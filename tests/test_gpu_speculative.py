@@ -247,3 +247,63 @@ def test_window_loss_matches_oracle(family, n, r, v, d, N, L):
     assert np.abs(slot.cpu().numpy() - ref_slot).max() <= LOGPROB_TOL
     assert abs(float(loss.cpu()[0]) - ref_loss) <= LOGPROB_TOL * n
     dh.close()
+
+
+# --------------------------------------------------------------------------- vocabulary not a multiple of 16
+@pytest.mark.parametrize("family,n,r,v,vv,d,P,wpp", [(I.CP, 3, 4, 272, 268, 128, 6, 8), (I.HMM, 4, 8, 32, 17, 64, 5, 16),
+                                                      (I.BTREE, 4, 4, 320, 305, 64, 4, 8), (I.HMM_CTX, 3, 4, 16, 1, 64, 3, 4)])
+def test_padded_vocabulary_every_entry_point(family, n, r, v, vv, d, P, wpp):
+    """v symbols per unit in memory, only the first vv exist (a byte-level Llama head has 268, stored as 272). The device
+    gets weights whose padding rows hold noise; the oracle never sees them. Log-likelihood, prefix marginals, draft,
+    acceptance and gradients must all ignore the padding."""
+    from oracle import mtpc_oracle_grad as og
+    shape = I.HeadShape(family, n, r, v, d, v_valid=vv)
+    wl = I.make_workload(f"pad_{family}_{v}_{vv}", shape, P, seed=8000 + v + vv, wpp=wpp, weight_std=0.3)
+    assert wl.W_emit_q.shape[2] == vv and wl.W_emit_dev_q.shape[2] == v and wl.targets.max() < vv
+    dh = DeviceHead(wl)
+    rows = np.arange(P)
+    logphi, logw = oracle_params(wl, rows)
+    assert logphi.shape[-1] == vv
+    # log-likelihood and prefix marginals
+    got = dh.window_logprob().cpu().numpy()
+    assert np.abs(got - orc.window_logprob(family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets)).max() <= LOGPROB_TOL
+    pre = dh.window_prefix_logprob().cpu().numpy()
+    assert np.abs(pre - orc.prefix_logprob(family, logw, logphi, wl.T_static, wl.targets)).max() <= LOGPROB_TOL
+    # draft: never a padding symbol, bytes as the oracle's
+    bytes_g, prefix_g = dh.draft_sample_prefix(wpp)
+    assert dh.head.mtpc_get_status() == 0
+    gb = bytes_g.cpu().numpy()
+    assert gb.min() >= 0 and gb.max() < vv
+    dsm = orc.draft_sample(family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wpp, wl.uniforms)
+    differ = (gb != dsm["bytes"]).any(axis=1)
+    assert not (differ & (dsm["margin"] >= BOUNDARY_BAND)).any()
+    pos = np.repeat(rows, wpp)
+    assert np.abs(prefix_g.cpu().numpy() - orc.prefix_logprob(family, logw, logphi, wl.T_static, gb, pos)).max() <= LOGPROB_TOL
+    # acceptance: target rows keep v entries on the device, the padding entries are ignored (filled with junk here)
+    W = P * wpp
+    p_valid = I.target_rows(99, 3, (W, n + 1, vv))
+    p_dev = np.full((W, n + 1, v), 0.37, dtype=np.float32)
+    p_dev[:, :, :vv] = p_valid
+    ua = I.uniforms(99, 4, (W, n + 1))
+    acc_g, next_g = dh.speculative_accept(P, wpp, bytes_g, prefix_g, torch.from_numpy(p_dev).cuda(), torch.from_numpy(ua).cuda())
+    assert dh.head.mtpc_get_status() == 0
+    bytes_o = dsm["bytes"]
+    prefix_o = orc.prefix_logprob(family, logw, logphi, wl.T_static, bytes_o, pos)
+    ref = orc.speculative_accept(prefix_o, bytes_o, p_valid.astype(np.float64), ua,
+                                 lambda r_, s_: orc.next_byte_logprob(family, logw, logphi, wl.T_static, bytes_o[r_], s_, pos[r_]))
+    near_final = np.where(ref["accepted"] == n, ref["margin_final"] < FULL_BAND, ref["margin_final"] * ref["resid_mass"] < FINAL_BAND)
+    ok = ~differ & ~((ref["margin_alpha"] < ALPHA_BAND) | near_final)
+    acc_g, next_g = acc_g.cpu().numpy(), next_g.cpu().numpy()
+    assert next_g.max() < vv
+    assert not (ok & ((acc_g != ref["accepted"]) | (next_g != ref["next_byte"]))).any()
+    # gradients: nothing flows into the padding rows
+    weight = np.random.default_rng(vv).normal(size=P).astype(np.float32)
+    out = dh.window_logprob_backward(torch.from_numpy(weight).cuda())
+    g = og.window_logprob_grad(family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets, weight)
+    dW = out["dW_emit"].cpu().numpy()
+    assert np.abs(dW[:, :, vv:, :]).max() == 0.0 if v > vv else True
+    for name, got_t, want in (("dh", out["dh"].cpu().numpy(), g["dh"]), ("dW_emit", dW[:, :, :vv, :], g["dW_emit"]),
+                              ("dW_sum", out["dW_sum"].cpu().numpy(), g["dW_sum"])):
+        scale = np.abs(want).max()
+        assert np.abs(got_t - want).max() <= 1e-2 * scale + 1e-4, name
+    dh.close()
