@@ -9,10 +9,15 @@ float64 (matmul, log_softmax, gather, logsumexp - the same steps, in the same or
 lets reverse-mode differentiation of exactly those steps produce it. It shares no code with the CUDA library and is
 only called by the tests, the smoke check and the benchmark's CPU legs.
 
+composite_loss_grad does the same for the training loss itself (Eq. 6: per-slot conditionals, valid-token normalisation,
+discount gamma).
+
 Pins (tests/test_oracle_grad.py): the torch forward equals the numpy oracle's forward to 1e-12; every gradient
 equals central finite differences of the NUMPY oracle's log-likelihood (an independent route: no autograd, no torch);
 closed forms (CP with r = 1: d/dlogit = weight * (onehot - softmax); a masked byte has zero gradient; gradients of
-a normalised circuit's weights sum to zero within each sum unit). No function here is left unpinned.
+a normalised circuit's weights sum to zero within each sum unit); the Eq. 6 loss equals the numpy oracle's
+composite_loss and its gradient equals central finite differences of that; with gamma = 1 and every byte valid it is
+the gradient of the mean joint negative log-likelihood. No function here is left unpinned.
 """
 from __future__ import annotations
 
@@ -95,3 +100,44 @@ def window_logprob_grad(family: int, h, W_emit, W_sum, T_static, targets, weight
     zero = lambda t: np.zeros(tuple(t.shape)) if t.grad is None else t.grad.numpy()
     return dict(logprob=lp.detach().numpy(), dh=zero(th), dW_emit=zero(tW), dW_sum=zero(tR),
                 dT_static=None if tT is None else zero(tT))
+
+
+def composite_loss_grad(family: int, h, W_emit, W_sum, T_static, targets, num_sequences: int, gamma: float):
+    """Eq. (6) and its gradient: L = sum_j gamma^(j-1) L_j with L_j = -(1/N) sum_i (1/V_ij) sum_t log p(x_{t+j} | x_{<t+j}),
+    the conditional of slot j being the ratio of consecutive prefix marginals of the window's circuit. Written as
+    that definition (one masked evaluation of the circuit per prefix length, then the sums of Eq. 6 with explicit
+    loops over slots and sequences) and differentiated by reverse mode.
+    Returns dict(slot_loss [n], loss, dh, dW_emit, dW_sum, dT_static)."""
+    th = torch.tensor(np.asarray(h, dtype=np.float64), requires_grad=True)
+    tW = torch.tensor(np.asarray(W_emit, dtype=np.float64), requires_grad=True)
+    tR = torch.tensor(np.asarray(W_sum, dtype=np.float64), requires_grad=True)
+    tT = None
+    if T_static is not None and family in (HMM, HMM_CTX):
+        tT = torch.tensor(np.asarray(T_static, dtype=np.float64), requires_grad=True)
+    tx = torch.tensor(np.asarray(targets, dtype=np.int64))
+    T, n = tx.shape
+    N = num_sequences
+    L = T // N
+    prefix = []
+    for j in range(n):
+        masked = tx.clone()
+        masked[:, j + 1:] = -1
+        prefix.append(forward(family, th, tW, tR, tT, masked))
+    slot = []
+    total = 0.0
+    for j in range(n):
+        cond = prefix[j] - (prefix[j - 1] if j > 0 else 0.0)
+        acc = 0.0
+        for i in range(N):
+            rows = slice(i * L, (i + 1) * L)
+            valid = tx[rows, j] >= 0
+            V = int(valid.sum())
+            if V:
+                acc = acc + cond[rows][valid].sum() / V
+        Lj = -acc / N
+        slot.append(Lj)
+        total = total + gamma ** j * Lj
+    total.backward()
+    zero = lambda t: np.zeros(tuple(t.shape)) if t.grad is None else t.grad.numpy()
+    return dict(slot_loss=np.array([float(s) for s in slot]), loss=float(total), dh=zero(th), dW_emit=zero(tW),
+                dW_sum=zero(tR), dT_static=None if tT is None else zero(tT))

@@ -110,3 +110,42 @@ def test_sum_unit_logit_gradients_sum_to_zero_per_unit(family, n, r, v):
     dlogit = g["dh"][:, :S * r].reshape(2, S, r)               # = d loss / d (sum-unit logits)
     assert np.abs(dlogit).max() > 1e-3
     assert np.abs(dlogit.sum(axis=-1)).max() < 1e-12
+
+
+# ------------------------------------------------------------------ Eq. (6) and its gradient
+def loss6_numpy(family, h, W, R, Ts, x, N, gamma):
+    pre = orc.window_prefix_logprob(family, h, W, R, Ts, x)
+    return orc.composite_loss(pre, x, N, gamma)
+
+
+@pytest.mark.parametrize("family,n,r,v", [(CP, 3, 3, 4), (HMM, 3, 2, 3), (HMM_CTX, 3, 2, 3), (BTREE, 4, 2, 3)])
+def test_eq6_loss_and_gradient_against_the_numpy_oracle(family, n, r, v):
+    rng = np.random.default_rng(950 + family)
+    N, L = 2, 4
+    h, W, R, Ts, x, _ = tiny(rng, family, n, r, v, T=N * L)
+    for j in range(1, n):                                     # windows running past the end of their sequence
+        x.reshape(N, L, n)[:, L - j:, j] = -1
+    x[0, 0] = -1                                              # and a hole at the front of one window
+    gamma = 0.8
+    g = og.composite_loss_grad(family, h, W, R, Ts, x, N, gamma)
+    slot, total = loss6_numpy(family, h, W, R, Ts, x, N, gamma)
+    np.testing.assert_allclose(g["slot_loss"], slot, atol=1e-12)
+    assert abs(g["loss"] - total) < 1e-12
+    fn = lambda: loss6_numpy(family, h, W, R, Ts, x, N, gamma)[1]
+    for name, arr in (("dh", h), ("dW_emit", W), ("dW_sum", R), ("dT_static", Ts)):
+        if arr is None:
+            continue
+        idx, fd = finite_difference(fn, arr, sample=40, rng=rng)
+        np.testing.assert_allclose(g[name].reshape(-1)[idx], fd, atol=2e-7, err_msg=name)
+        assert np.abs(fd).max() > 1e-4
+
+
+@pytest.mark.parametrize("family", [CP, HMM, BTREE])
+def test_undiscounted_eq6_gradient_is_the_mean_nll_gradient(family):
+    rng = np.random.default_rng(960 + family)
+    n, r, v, N, L = 4, 2, 3, 2, 3
+    h, W, R, Ts, x, _ = tiny(rng, family, n, r, v, T=N * L)
+    g6 = og.composite_loss_grad(family, h, W, R, Ts, x, N, 1.0)
+    gj = og.window_logprob_grad(family, h, W, R, Ts, x, np.full(N * L, -1.0 / (N * L)))
+    for name in ("dh", "dW_emit", "dW_sum"):
+        np.testing.assert_allclose(g6[name], gj[name], atol=1e-12)
