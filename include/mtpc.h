@@ -214,11 +214,24 @@ int mtpc_window_loss(mtpc_head* head, const void* hidden, const int32_t* targets
  * Arithmetic: posteriors in fp32; the logit gradients are rounded to bf16 (the operand type of the tensor cores) before
  * the three weight-sized GEMMs, fp32 accumulation. dT_static is accumulated with atomic adds (order not fixed).
  */
+/*
+ * mtpc_window_loss_backward: the training loss of Eq. 6 (as mtpc_window_loss: per-slot conditionals, valid-token
+ * normalisation V_ij, discount gamma^j) AND its gradients, for num_sequences sequences of sequence_length positions.
+ * Eq. 6 is linear in the prefix log-marginals, L = sum_t sum_j coeff[t, j] log q(x_{t,0..j}), with
+ * coeff[t, j] = c[t, j] - c[t, j+1], c[t, j] = -gamma^j / (N V_ij) for a valid target and 0 otherwise; the call runs one
+ * circuit backward pass per prefix length j+1 (later bytes summed out), accumulates the posteriors in fp32, and then
+ * shares the projection-sized work (logit gradients, the three GEMMs) with mtpc_window_logprob_backward. Same workspace
+ * (mtpc_backward_workspace_bytes with T = num_sequences * sequence_length), same outputs, same arithmetic notes.
+ */
 int mtpc_backward_workspace_bytes(const mtpc_config* cfg, int32_t T, size_t* out_bytes);
 int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t T,
                                  const float* weight, void* bwd_workspace, size_t bwd_workspace_bytes,
                                  float* out_logprob, float* d_hidden, float* dW_emit, float* dW_sum, float* dT_static,
                                  void* stream);
+int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,
+                              int32_t sequence_length, float gamma, void* bwd_workspace, size_t bwd_workspace_bytes,
+                              float* out_slot_loss, float* out_loss, float* d_hidden, float* dW_emit, float* dW_sum,
+                              float* dT_static, void* stream);
 
 /*
  * Host-buffer variants: same results, but hidden / targets / uniforms are HOST pointers (pinned memory for
@@ -251,6 +264,8 @@ int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags);
  *   mtpc_speculative_accept: [0] the acceptance kernel.
  *   mtpc_window_logprob_backward: [0] forward projection, [1] circuit backward, [2] projection in gradient mode,
  *                        [3] transposes and the plain GEMMs.
+ *   mtpc_window_loss_backward: [0] forward projection + prefix marginals + loss, [1] the n circuit backward passes,
+ *                        [2] and [3] as above.
  *   mtpc_draft_sample, mtpc_draft_sample_prefix:   P <= 128 positions and r <= 32: [0] one pass over all weights (logits of every unit),
  *                        [1] per-slot latent + byte draws and evidence, [2] circuit evaluation.
  *                        Otherwise: [0] sum-unit GEMM, [1] latent sampling, [2] GEMM + inverse-CDF epilogue,

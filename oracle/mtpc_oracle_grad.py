@@ -139,5 +139,5 @@ def composite_loss_grad(family: int, h, W_emit, W_sum, T_static, targets, num_se
         total = total + gamma ** j * Lj
     total.backward()
     zero = lambda t: np.zeros(tuple(t.shape)) if t.grad is None else t.grad.numpy()
-    return dict(slot_loss=np.array([float(s) for s in slot]), loss=float(total), dh=zero(th), dW_emit=zero(tW),
+    return dict(slot_loss=np.array([float(s.detach()) for s in slot]), loss=float(total.detach()), dh=zero(th), dW_emit=zero(tW),
                 dW_sum=zero(tR), dT_static=None if tT is None else zero(tT))

@@ -22,7 +22,7 @@ EXPORTS = [
     "mtpc_window_logprob_host", "mtpc_draft_sample_host", "mtpc_get_status", "mtpc_set_timing", "mtpc_get_timing",
     "mtpc_launch_count", "mtpc_destroy", "mtpc_status_string", "mtpc_window_logprob_static",
     "mtpc_window_prefix_logprob", "mtpc_draft_sample_prefix", "mtpc_speculative_accept", "mtpc_window_loss",
-    "mtpc_backward_workspace_bytes", "mtpc_window_logprob_backward",
+    "mtpc_backward_workspace_bytes", "mtpc_window_logprob_backward", "mtpc_window_loss_backward",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 ERR_STATIC_SCRATCH = -7
@@ -72,6 +72,7 @@ def lib() -> ctypes.CDLL:
     L.mtpc_window_loss.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp, vp, vp]
     L.mtpc_backward_workspace_bytes.argtypes = [ctypes.POINTER(MtpcConfig), i32, ctypes.POINTER(sz)]
     L.mtpc_window_logprob_backward.argtypes = [vp, vp, vp, i32, vp, vp, sz, vp, vp, vp, vp, vp, vp]
+    L.mtpc_window_loss_backward.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp, sz, vp, vp, vp, vp, vp, vp, vp]
     L.mtpc_status_string.argtypes = [ctypes.c_int]
     L.mtpc_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -169,17 +170,30 @@ class MtpcHead:
                                       ctypes.c_float(gamma), _ptr(out_slot_loss), _ptr(out_loss), _stream(stream)),
                "mtpc_window_loss")
 
-    def mtpc_window_logprob_backward(self, hidden, targets, weight, out_logprob, d_hidden, dW_emit, dW_sum, dT_static=None,
-                                     stream=None) -> None:
-        """Gradients of sum_t weight[t] log q_t; the backward workspace is allocated here (torch) and kept for reuse."""
+    def _backward_workspace(self, T: int, device):
         import torch
-        T = hidden.shape[0]
         need = ctypes.c_size_t(0)
         _check(lib().mtpc_backward_workspace_bytes(ctypes.byref(self.cfg), T, ctypes.byref(need)),
                "mtpc_backward_workspace_bytes")
         ws = getattr(self, "_bwd_ws", None)
         if ws is None or ws.numel() < need.value:
-            ws = self._bwd_ws = torch.empty(need.value, dtype=torch.uint8, device=hidden.device)
+            ws = self._bwd_ws = torch.empty(need.value, dtype=torch.uint8, device=device)
+        return ws
+
+    def mtpc_window_loss_backward(self, hidden, targets, num_sequences: int, sequence_length: int, gamma: float,
+                                  out_slot_loss, out_loss, d_hidden, dW_emit, dW_sum, dT_static=None, stream=None) -> None:
+        """Eq. 6 loss and its gradients; the backward workspace is allocated here (torch) and kept for reuse."""
+        ws = self._backward_workspace(hidden.shape[0], hidden.device)
+        _check(lib().mtpc_window_loss_backward(self.handle, _ptr(hidden), _ptr(targets), num_sequences, sequence_length,
+                                               ctypes.c_float(gamma), ws.data_ptr(), ws.numel(), _ptr(out_slot_loss),
+                                               _ptr(out_loss), _ptr(d_hidden), _ptr(dW_emit), _ptr(dW_sum), _ptr(dT_static),
+                                               _stream(stream)), "mtpc_window_loss_backward")
+
+    def mtpc_window_logprob_backward(self, hidden, targets, weight, out_logprob, d_hidden, dW_emit, dW_sum, dT_static=None,
+                                     stream=None) -> None:
+        """Gradients of sum_t weight[t] log q_t; the backward workspace is allocated here (torch) and kept for reuse."""
+        T = hidden.shape[0]
+        ws = self._backward_workspace(T, hidden.device)
         _check(lib().mtpc_window_logprob_backward(self.handle, _ptr(hidden), _ptr(targets), T, _ptr(weight), ws.data_ptr(),
                                                   ws.numel(), _ptr(out_logprob), _ptr(d_hidden), _ptr(dW_emit), _ptr(dW_sum),
                                                   _ptr(dT_static), _stream(stream)), "mtpc_window_logprob_backward")

@@ -578,7 +578,7 @@ size_t round64(size_t x) { return (x + 63) / 64 * 64; }
 // and W_sum^T to the right of W_emit^T in [d, Kd], so that d hidden is a single GEMM over K = Nc + S r.
 struct BackwardLayout {
   size_t Nc, Spad, Tpad, Kd;
-  size_t off_lse, off_post, off_dsum_t, off_dlogit, off_dlogit_t, off_wt, off_ht, total;
+  size_t off_lse, off_post, off_dsum_t, off_dlogit, off_dlogit_t, off_wt, off_ht, off_dsum_f32, off_coeff, total;
 };
 void plan_backward(const mtpc_config& c, const Layout& L, int T, BackwardLayout* B) {
   B->Nc = static_cast<size_t>(c.n) * c.r * c.v;
@@ -594,6 +594,8 @@ void plan_backward(const mtpc_config& c, const Layout& L, int T, BackwardLayout*
   B->off_dlogit_t = take(B->Nc * B->Tpad * 2);                       // [Nc, Tpad]
   B->off_wt = take(static_cast<size_t>(c.d) * B->Kd * 2);            // [d, Nc | Spad]: W_emit^T | W_sum^T
   B->off_ht = take(static_cast<size_t>(c.d) * B->Tpad * 2);          // hidden^T [d, Tpad]
+  B->off_dsum_f32 = take(static_cast<size_t>(T) * L.sum_rows * 4);   // Eq. 6: sum-unit logit gradients accumulated over the passes
+  B->off_coeff = take(static_cast<size_t>(T) * c.n * 4);             // Eq. 6: weights of the prefix marginals
   B->total = off;
 }
 
@@ -637,32 +639,89 @@ int launch_plain_gemm(mtpc_head* h, const void* A, size_t lda, const void* Bm, s
   return check_launch();
 }
 
-int launch_circuit_backward(mtpc_head* h, int T, const int32_t* targets, const float* weight, float* out, float* post,
-                            __nv_bfloat16* dsum, int dsum_pitch, float* dT, cudaStream_t st) {
+int launch_circuit_backward(mtpc_head* h, CircuitBackwardArgs a, float* dT, cudaStream_t st) {
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
-  const float* G = at<float>(h, L.off_G);
-  const float* logw = at<float>(h, L.off_logw);
+  a.G = at<float>(h, L.off_G);
+  a.logw = at<float>(h, L.off_logw);
+  a.n = c.n;
+  a.r = c.r;
+  a.sum_rows = L.sum_rows;
   unsigned* counter = at<unsigned>(h, L.off_status) + kWorkCounterWord;
-  const int blocks = (T + kCircuitWarps - 1) / kCircuitWarps;
+  const int blocks = (a.W + kCircuitWarps - 1) / kCircuitWarps;
   const int threads = kCircuitWarps * 32;
   const int resident = blocks < 8 * h->num_sms ? blocks : 8 * h->num_sms;
   if (c.family != MTPC_CP && cudaMemsetAsync(counter, 0, sizeof(unsigned), st) != cudaSuccess) return MTPC_ERR_CUDA;
   if (c.family == MTPC_CP) {
-    circuit_cp_backward_kernel<<<blocks, threads, 0, st>>>(G, logw, targets, weight, out, post, dsum, dsum_pitch, T, c.n,
-                                                          c.r, L.sum_rows);
+    circuit_cp_backward_kernel<<<blocks, threads, 0, st>>>(a);
   } else if (c.family == MTPC_HMM) {
     const size_t smem = hmm_backward_smem_floats(c.n, c.r, !is_ctx(h), kCircuitWarps) * sizeof(float);
-    circuit_hmm_backward_kernel<<<resident, threads, smem, st>>>(G, logw, hmm_tables(h), hmm_table_stride(h), targets,
-                                                                weight, out, post, dsum, dsum_pitch, dT, counter, T,
-                                                                c.n, c.r, L.sum_rows);
+    circuit_hmm_backward_kernel<<<resident, threads, smem, st>>>(a, hmm_tables(h), hmm_table_stride(h), dT, counter);
   } else {
     const size_t smem = kCircuitWarps * btree_backward_warp_floats(c.n, c.r) * sizeof(float);
-    circuit_btree_backward_kernel<<<resident, threads, smem, st>>>(G, logw, targets, weight, out, post, dsum, dsum_pitch,
-                                                                  counter, T, c.n, c.r, L.sum_rows);
+    circuit_btree_backward_kernel<<<resident, threads, smem, st>>>(a, counter);
   }
   h->launches++;
   return check_launch();
+}
+
+// Shared-memory attributes of the circuit backward kernels (per function, set to what this head needs).
+int set_backward_attributes(const mtpc_head* head) {
+  const mtpc_config& c = head->cfg;
+  bool fail = false;
+  if (c.family == MTPC_HMM) {
+    const size_t smem = hmm_backward_smem_floats(c.n, c.r, !is_ctx(head), kCircuitWarps) * sizeof(float);
+    if (smem > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;
+    if (smem > 48 * 1024)
+      fail |= cudaFuncSetAttribute(circuit_hmm_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   static_cast<int>(smem)) != cudaSuccess;
+  } else if (c.family == MTPC_BTREE) {
+    const size_t smem = kCircuitWarps * btree_backward_warp_floats(c.n, c.r) * sizeof(float);
+    if (smem > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;
+    if (smem > 48 * 1024)
+      fail |= cudaFuncSetAttribute(circuit_btree_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   static_cast<int>(smem)) != cudaSuccess;
+  }
+  return fail ? MTPC_ERR_CUDA : MTPC_OK;
+}
+
+// Phases 3 and 4 of a backward call: the projection kernel in gradient mode (post, lse -> bf16 logit gradients), the
+// transposes and the plain GEMMs. The sum-unit logit gradients are already in place to the right of dlogit.
+int backward_tail(mtpc_head* head, const BackwardLayout& B, uint8_t* bw, const void* hb, const int32_t* targets, int T,
+                  float* d_hidden, float* dW_emit, float* dW_sum, PhaseTimer& pt, cudaStream_t st) {
+  const mtpc_config& c = head->cfg;
+  const Layout& L = head->L;
+  __nv_bfloat16* dsum_t = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dsum_t);
+  __nv_bfloat16* dlogit = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit);
+  __nv_bfloat16* dsum = dlogit + B.Nc;
+  __nv_bfloat16* dlogit_t = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit_t);
+  __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(bw + B.off_wt);
+  void* ht = bw + B.off_ht;
+  const int Nc = static_cast<int>(B.Nc);
+  pt.begin();
+  GradArgs ga;
+  ga.lse_in = reinterpret_cast<float*>(bw + B.off_lse);
+  ga.post = reinterpret_cast<float*>(bw + B.off_post);
+  ga.dlogit = dlogit;
+  ga.dlogit_t = dlogit_t;
+  ga.t_pitch = B.Tpad;
+  ga.dlogit_pitch = B.Kd;
+  int rc = launch_gemm(head, kModeGrad, hb, T, 1, true, false, targets, nullptr, nullptr, st, &ga);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  pt.begin();
+  rc = launch_transpose(head, head->W_emit_bf16, wt, Nc, c.d, c.d, B.Kd, st);
+  if (rc == MTPC_OK) rc = launch_transpose(head, head->W_sum_bf16, wt + B.Nc, L.sum_rows, c.d, c.d, B.Kd, st);
+  if (rc == MTPC_OK) rc = launch_transpose(head, hb, ht, T, c.d, c.d, B.Tpad, st);
+  if (rc == MTPC_OK) rc = launch_transpose(head, dsum, dsum_t, T, L.sum_rows, B.Kd, B.Tpad, st);
+  // d hidden [T, d] = [dlogit | dsum] [T, Nc + S r] [W_emit ; W_sum] [Nc + S r, d]
+  if (rc == MTPC_OK)
+    rc = launch_plain_gemm(head, dlogit, B.Kd, wt, B.Kd, d_hidden, c.d, T, c.d, Nc + L.sum_rows, false, st);
+  // dW_emit [Nc, d] = dlogit^T [Nc, T] hidden [T, d];  dW_sum [S r, d] = dsum^T [S r, T] hidden [T, d]
+  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dlogit_t, B.Tpad, ht, B.Tpad, dW_emit, c.d, Nc, c.d, T, false, st);
+  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dsum_t, B.Tpad, ht, B.Tpad, dW_sum, c.d, L.sum_rows, c.d, T, false, st);
+  pt.end();
+  return rc;
 }
 
 int check_call(mtpc_head* h, int32_t rows) {
@@ -879,43 +938,15 @@ int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int3
   if (T == 0) return MTPC_OK;
   if (!hidden || !targets || !weight || !bwd_workspace || !d_hidden || !dW_emit || !dW_sum) return MTPC_ERR_NULL;
   const mtpc_config& c = head->cfg;
-  const Layout& L = head->L;
   const bool static_hmm = c.family == MTPC_HMM && !is_ctx(head) && c.n > 1;
   if (static_hmm && !dT_static) return MTPC_ERR_NULL;
   BackwardLayout B;
-  plan_backward(c, L, T, &B);
+  plan_backward(c, head->L, T, &B);
   if (bwd_workspace_bytes < B.total || (reinterpret_cast<uintptr_t>(bwd_workspace) % kAlign) != 0)
     return MTPC_ERR_WORKSPACE;
-  // shared-memory sizes of the circuit backward kernels (per function, set to what this head needs)
-  {
-    bool fail = false;
-    if (c.family == MTPC_HMM) {
-      const size_t smem = hmm_backward_smem_floats(c.n, c.r, !is_ctx(head), kCircuitWarps) * sizeof(float);
-      if (smem > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;
-      if (smem > 48 * 1024)
-        fail |= cudaFuncSetAttribute(circuit_hmm_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(smem)) != cudaSuccess;
-    } else if (c.family == MTPC_BTREE) {
-      const size_t smem = kCircuitWarps * btree_backward_warp_floats(c.n, c.r) * sizeof(float);
-      if (smem > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;
-      if (smem > 48 * 1024)
-        fail |= cudaFuncSetAttribute(circuit_btree_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(smem)) != cudaSuccess;
-    }
-    if (fail) return MTPC_ERR_CUDA;
-  }
+  if ((rc = set_backward_attributes(head)) != MTPC_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* bw = static_cast<uint8_t*>(bwd_workspace);
-  float* lse = reinterpret_cast<float*>(bw + B.off_lse);
-  float* post = reinterpret_cast<float*>(bw + B.off_post);
-  __nv_bfloat16* dsum_t = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dsum_t);
-  __nv_bfloat16* dlogit = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit);
-  __nv_bfloat16* dsum = dlogit + B.Nc;                       // columns [Nc, Nc + S r) of the same rows
-  __nv_bfloat16* dlogit_t = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit_t);
-  __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(bw + B.off_wt);
-  void* ht = bw + B.off_ht;
-  const int Nc = static_cast<int>(B.Nc);
-
   const void* hb = nullptr;
   head->draft_P = 0;
   rc = stage_hidden(head, hidden, T, &hb, st);
@@ -924,44 +955,108 @@ int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int3
   // 1. forward projection, keeping the units' log-sum-exps
   pt.begin();
   GradArgs fwd;
-  fwd.lse_out = lse;
+  fwd.lse_out = reinterpret_cast<float*>(bw + B.off_lse);
   rc = launch_gemm(head, kModeLogprob, hb, T, 1, true, true, targets, nullptr, nullptr, st, &fwd);
   pt.end();
   if (rc != MTPC_OK) return rc;
   // 2. circuit backward: posteriors of the input units and of the sum units
   pt.begin();
-  bool bad = false;
+  if (static_hmm && cudaMemsetAsync(dT_static, 0, static_cast<size_t>(c.n - 1) * c.r * c.r * 4, st) != cudaSuccess)
+    return MTPC_ERR_CUDA;
+  CircuitBackwardArgs a;
+  memset(&a, 0, sizeof(a));
+  a.targets = targets;
+  a.weight = weight;
+  a.weight_stride = 1;
+  a.out = out_logprob;
+  a.post = reinterpret_cast<float*>(bw + B.off_post);
+  a.dsum = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit) + B.Nc;      // columns [Nc, Nc + S r) of the dlogit rows
+  a.dsum_pitch = static_cast<int>(B.Kd);
+  a.len = c.n;
+  a.W = T;
+  rc = launch_circuit_backward(head, a, dT_static, st);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  // 3., 4. logit gradients from the recomputed logits, then the plain GEMMs
+  return backward_tail(head, B, bw, hb, targets, T, d_hidden, dW_emit, dW_sum, pt, st);
+}
+
+int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,
+                              int32_t sequence_length, float gamma, void* bwd_workspace, size_t bwd_workspace_bytes,
+                              float* out_slot_loss, float* out_loss, float* d_hidden, float* dW_emit, float* dW_sum,
+                              float* dT_static, void* stream) {
+  if (!head) return MTPC_ERR_NULL;
+  if (num_sequences < 1 || sequence_length < 1) return MTPC_ERR_SHAPE;
+  const int64_t T64 = static_cast<int64_t>(num_sequences) * sequence_length;
+  if (T64 > head->cfg.max_positions) return MTPC_ERR_SHAPE;
+  if (!hidden || !targets || !bwd_workspace || !out_slot_loss || !out_loss || !d_hidden || !dW_emit || !dW_sum)
+    return MTPC_ERR_NULL;
+  const int T = static_cast<int>(T64);
+  const mtpc_config& c = head->cfg;
+  const Layout& L = head->L;
+  const bool static_hmm = c.family == MTPC_HMM && !is_ctx(head) && c.n > 1;
+  if (static_hmm && !dT_static) return MTPC_ERR_NULL;
+  BackwardLayout B;
+  plan_backward(c, L, T, &B);
+  if (bwd_workspace_bytes < B.total || (reinterpret_cast<uintptr_t>(bwd_workspace) % kAlign) != 0)
+    return MTPC_ERR_WORKSPACE;
+  int rc = set_backward_attributes(head);
+  if (rc != MTPC_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* bw = static_cast<uint8_t*>(bwd_workspace);
+  float* post = reinterpret_cast<float*>(bw + B.off_post);
+  float* dsum_f32 = reinterpret_cast<float*>(bw + B.off_dsum_f32);
+  float* coeff = reinterpret_cast<float*>(bw + B.off_coeff);
+  float* prefix = at<float>(head, L.off_prefix);
+  float* partial = at<float>(head, L.off_partial);
+  const void* hb = nullptr;
+  head->draft_P = 0;
+  rc = stage_hidden(head, hidden, T, &hb, st);
+  if (rc != MTPC_OK) return rc;
+  PhaseTimer pt(head, st);
+  // 1. forward projection (keeping the log-sum-exps), prefix marginals, the loss of Eq. 6 and the weight of every prefix
+  pt.begin();
+  GradArgs fwd;
+  fwd.lse_out = reinterpret_cast<float*>(bw + B.off_lse);
+  rc = launch_gemm(head, kModeLogprob, hb, T, 1, true, true, targets, nullptr, nullptr, st, &fwd);
+  if (rc == MTPC_OK) rc = launch_circuit(head, T, 1, nullptr, prefix, st);
+  if (rc != MTPC_OK) return rc;
+  loss_partial_kernel<<<num_sequences, kLossThreads, 0, st>>>(prefix, targets, partial, sequence_length, c.n);
+  loss_final_kernel<<<1, kLossThreads, 0, st>>>(partial, out_slot_loss, out_loss, num_sequences, c.n, gamma);
+  loss_coeff_kernel<<<num_sequences, kLossThreads, 0, st>>>(targets, coeff, sequence_length, c.n, num_sequences, gamma);
+  head->launches += 3;
+  pt.end();
+  if ((rc = check_launch()) != MTPC_OK) return rc;
+  // 2. one circuit backward pass per prefix length, accumulating
+  pt.begin();
+  bool bad = cudaMemsetAsync(post, 0, static_cast<size_t>(T) * c.n * c.r * 4, st) != cudaSuccess;
+  bad |= cudaMemsetAsync(dsum_f32, 0, static_cast<size_t>(T) * L.sum_rows * 4, st) != cudaSuccess;
   if (static_hmm) bad |= cudaMemsetAsync(dT_static, 0, static_cast<size_t>(c.n - 1) * c.r * c.r * 4, st) != cudaSuccess;
   if (bad) return MTPC_ERR_CUDA;
-  rc = launch_circuit_backward(head, T, targets, weight, out_logprob, post, dsum, static_cast<int>(B.Kd), dT_static, st);
+  for (int j = 0; j < c.n; ++j) {
+    CircuitBackwardArgs a;
+    memset(&a, 0, sizeof(a));
+    a.targets = targets;
+    a.weight = coeff + j;
+    a.weight_stride = c.n;
+    a.post = post;
+    a.dsum_f32 = dsum_f32;
+    a.dsum_pitch = L.sum_rows;
+    a.len = j + 1;
+    a.accumulate = 1;
+    a.W = T;
+    if ((rc = launch_circuit_backward(head, a, dT_static, st)) != MTPC_OK) return rc;
+  }
+  {
+    const size_t total = static_cast<size_t>(T) * L.sum_rows;
+    const int blocks = static_cast<int>((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
+    f32_rows_to_bf16_kernel<<<blocks, 256, 0, st>>>(dsum_f32, reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit) + B.Nc, T,
+                                                    L.sum_rows, L.sum_rows, B.Kd);
+    head->launches++;
+  }
   pt.end();
-  if (rc != MTPC_OK) return rc;
-  // 3. logits recomputed, turned into their gradient (bf16, both orientations)
-  pt.begin();
-  GradArgs ga;
-  ga.lse_in = lse;
-  ga.post = post;
-  ga.dlogit = dlogit;
-  ga.dlogit_t = dlogit_t;
-  ga.t_pitch = B.Tpad;
-  ga.dlogit_pitch = B.Kd;
-  rc = launch_gemm(head, kModeGrad, hb, T, 1, true, false, targets, nullptr, nullptr, st, &ga);
-  pt.end();
-  if (rc != MTPC_OK) return rc;
-  // 4. transposed operands, then the plain GEMMs
-  pt.begin();
-  rc = launch_transpose(head, head->W_emit_bf16, wt, Nc, c.d, c.d, B.Kd, st);
-  if (rc == MTPC_OK) rc = launch_transpose(head, head->W_sum_bf16, wt + B.Nc, L.sum_rows, c.d, c.d, B.Kd, st);
-  if (rc == MTPC_OK) rc = launch_transpose(head, hb, ht, T, c.d, c.d, B.Tpad, st);
-  if (rc == MTPC_OK) rc = launch_transpose(head, dsum, dsum_t, T, L.sum_rows, B.Kd, B.Tpad, st);
-  // d hidden [T, d] = [dlogit | dsum] [T, Nc + S r] [W_emit ; W_sum] [Nc + S r, d]
-  if (rc == MTPC_OK)
-    rc = launch_plain_gemm(head, dlogit, B.Kd, wt, B.Kd, d_hidden, c.d, T, c.d, Nc + L.sum_rows, false, st);
-  // dW_emit [Nc, d] = dlogit^T [Nc, T] hidden [T, d];  dW_sum [S r, d] = dsum^T [S r, T] hidden [T, d]
-  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dlogit_t, B.Tpad, ht, B.Tpad, dW_emit, c.d, Nc, c.d, T, false, st);
-  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dsum_t, B.Tpad, ht, B.Tpad, dW_sum, c.d, L.sum_rows, c.d, T, false, st);
-  pt.end();
-  return rc;
+  if ((rc = check_launch()) != MTPC_OK) return rc;
+  return backward_tail(head, B, bw, hb, targets, T, d_hidden, dW_emit, dW_sum, pt, st);
 }
 
 // Streams and events of the chunked host-buffer path; no device memory is allocated.

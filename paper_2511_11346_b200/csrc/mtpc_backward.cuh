@@ -20,20 +20,48 @@
 
 namespace mtpc {
 
+// Arguments the three circuit backward kernels share beyond the forward ones:
+//   weight, weight_stride   window w is weighted by weight[w * weight_stride]
+//   len                     only the first `len` slots carry evidence, the later bytes are summed out: the kernels then
+//                           differentiate the prefix marginal log q(x_0..x_{len-1}) (len = n: the joint)
+//   accumulate              0: post and dsum are overwritten (dsum as bf16). 1: results are ADDED to post and to the fp32
+//                           buffer dsum_f32 (several passes with different len and weights, Eq. 6); only slots < len are
+//                           touched, the buffers must have been zeroed before the first pass.
+//   dsum_pitch              row pitch, in elements, of whichever of dsum / dsum_f32 is written
+struct CircuitBackwardArgs {
+  const float* G;
+  const float* logw;
+  const int* targets;
+  const float* weight;
+  int weight_stride;
+  float* out;                 // [W] log q of the (prefix) window, or NULL
+  float* post;                // [W, n, r]
+  __nv_bfloat16* dsum;        // [W, dsum_pitch] (accumulate == 0)
+  float* dsum_f32;            // [W, dsum_pitch] (accumulate == 1)
+  int dsum_pitch;
+  int len, accumulate;
+  int W, n, r, sum_rows;
+};
+__device__ __forceinline__ void put_post(const CircuitBackwardArgs& a, size_t idx, float v) {
+  if (a.accumulate) a.post[idx] += v;
+  else a.post[idx] = v;
+}
+__device__ __forceinline__ void put_dsum(const CircuitBackwardArgs& a, size_t idx, float v) {
+  if (a.accumulate) a.dsum_f32[idx] += v;
+  else a.dsum[idx] = __float2bfloat16_rn(v);
+}
+
 // ---------------------------------------------------------------- circuit backward: mixture (Eq. CP)
 // log q = LSE_k a_k, a_k = log omega_k + sum_i G[i, k]:  d log q / d a_k = rho_k = softmax(a)_k for every slot and for
 // the mixture weight; through the softmax of the mixture logits: rho_k - omega_k.
-__global__ void circuit_cp_backward_kernel(const float* __restrict__ G, const float* __restrict__ logw,
-                                           const int* __restrict__ targets, const float* __restrict__ weight,
-                                           float* __restrict__ out, float* __restrict__ post,
-                                           __nv_bfloat16* __restrict__ dsum, int dsum_pitch, int W, int n, int r,
-                                           int sum_rows) {
+__global__ void circuit_cp_backward_kernel(const CircuitBackwardArgs a_) {
   const int w = blockIdx.x * kCircuitWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  if (w >= W) return;
-  const float* g = G + static_cast<size_t>(w) * n * r;
-  const float* lw = logw + static_cast<size_t>(w) * sum_rows;
-  const float wt = weight[w];
+  if (w >= a_.W) return;
+  const int n = a_.n, r = a_.r, len = a_.len;
+  const float* g = a_.G + static_cast<size_t>(w) * n * r;
+  const float* lw = a_.logw + static_cast<size_t>(w) * a_.sum_rows;
+  const float wt = a_.weight[static_cast<size_t>(w) * a_.weight_stride];
   float a[4];
   float m = -CUDART_INF_F, s = 0.f;
 #pragma unroll
@@ -42,7 +70,7 @@ __global__ void circuit_cp_backward_kernel(const float* __restrict__ G, const fl
     a[q] = -CUDART_INF_F;
     if (k < r) {
       a[q] = lw[k];
-      for (int i = 0; i < n; ++i) a[q] += g[i * r + k];
+      for (int i = 0; i < len; ++i) a[q] += g[i * r + k];
       lse_merge(m, s, a[q], 1.f);
     }
   }
@@ -53,15 +81,16 @@ __global__ void circuit_cp_backward_kernel(const float* __restrict__ G, const fl
     lse_merge(m, s, m2, s2);
   }
   const float logq = m + __logf(s);
-  if (lane == 0 && out != nullptr) out[w] = logq;
+  if (lane == 0 && a_.out != nullptr) a_.out[w] = logq;
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int k = lane + 32 * q;
     if (k < r) {
       const float rho = __expf(a[q] - logq);
-      for (int i = 0; i < n; ++i)
-        post[(static_cast<size_t>(w) * n + i) * r + k] = targets[static_cast<size_t>(w) * n + i] >= 0 ? wt * rho : 0.f;
-      dsum[static_cast<size_t>(w) * dsum_pitch + k] = __float2bfloat16_rn(wt * (rho - __expf(lw[k])));
+      for (int i = 0; i < len; ++i)
+        put_post(a_, (static_cast<size_t>(w) * n + i) * r + k, a_.targets[static_cast<size_t>(w) * n + i] >= 0 ? wt * rho : 0.f);
+      for (int i = len; i < n && !a_.accumulate; ++i) a_.post[(static_cast<size_t>(w) * n + i) * r + k] = 0.f;
+      put_dsum(a_, static_cast<size_t>(w) * a_.dsum_pitch + k, wt * (rho - __expf(lw[k])));
     }
   }
 }
@@ -70,11 +99,11 @@ __global__ void circuit_cp_backward_kernel(const float* __restrict__ G, const fl
 // Lane = row (the conditioning value). For every column b: out[b] = wt * (exp(base + row[b] + pc[b]) - exp(row[b]) * gam),
 // i.e. pairwise posterior minus conditional probability times the posterior of the conditioning value (the gradient
 // with respect to the row's logits). `row` and `pc` are in shared memory; the results go either to a bf16 row in global
-// memory (contextual tables: one set per position) or, by atomic adds, to an fp32 row in shared memory (static tables,
-// summed over the windows). R a multiple of 4: float4 reads rotated by the lane (conflict-free), 8-byte stores.
+// memory (contextual tables: one set per position), or by atomic adds to an fp32 row in shared memory (static tables,
+// summed over the windows), or added to an fp32 row in global memory (several passes accumulating, Eq. 6). R a multiple of 4: float4 reads rotated by the lane (conflict-free), 8-byte stores.
 template <int R>
 __device__ __forceinline__ void row_grad_vec(const float* row, const float* pc, float base, float gam, float wt, int lane,
-                                             __nv_bfloat16* dst, float* acc_row) {
+                                             __nv_bfloat16* dst, float* acc_row, float* f32_row) {
   constexpr int Q = R / 4;
   const float4* row4 = reinterpret_cast<const float4*>(row);
   const float4* pc4 = reinterpret_cast<const float4*>(pc);
@@ -92,6 +121,11 @@ __device__ __forceinline__ void row_grad_vec(const float* row, const float* pc, 
       atomicAdd(acc_row + 4 * j + 1, oy);
       atomicAdd(acc_row + 4 * j + 2, oz);
       atomicAdd(acc_row + 4 * j + 3, ow);
+    } else if (f32_row != nullptr) {                  // this lane owns the row: plain read-add-write
+      float4* d4 = reinterpret_cast<float4*>(f32_row + 4 * j);
+      float4 o = *d4;
+      o.x += ox; o.y += oy; o.z += oz; o.w += ow;
+      *d4 = o;
     } else {
       __nv_bfloat162 lo = __floats2bfloat162_rn(ox, oy);
       __nv_bfloat162 hi = __floats2bfloat162_rn(oz, ow);
@@ -103,12 +137,12 @@ __device__ __forceinline__ void row_grad_vec(const float* row, const float* pc, 
   }
 }
 __device__ __forceinline__ void row_grad(const float* row, const float* pc, float base, float gam, float wt, int lane, int r,
-                                         __nv_bfloat16* dst, float* acc_row) {
+                                         __nv_bfloat16* dst, float* acc_row, float* f32_row) {
   switch (r) {
-    case 32: row_grad_vec<32>(row, pc, base, gam, wt, lane, dst, acc_row); return;
-    case 16: row_grad_vec<16>(row, pc, base, gam, wt, lane, dst, acc_row); return;
-    case 8: row_grad_vec<8>(row, pc, base, gam, wt, lane, dst, acc_row); return;
-    case 4: row_grad_vec<4>(row, pc, base, gam, wt, lane, dst, acc_row); return;
+    case 32: row_grad_vec<32>(row, pc, base, gam, wt, lane, dst, acc_row, f32_row); return;
+    case 16: row_grad_vec<16>(row, pc, base, gam, wt, lane, dst, acc_row, f32_row); return;
+    case 8: row_grad_vec<8>(row, pc, base, gam, wt, lane, dst, acc_row, f32_row); return;
+    case 4: row_grad_vec<4>(row, pc, base, gam, wt, lane, dst, acc_row, f32_row); return;
     default: break;
   }
   for (int q = 0; q < r; ++q) {                       // start at column `lane` (r a power of two): conflict-free
@@ -116,6 +150,7 @@ __device__ __forceinline__ void row_grad(const float* row, const float* pc, floa
     const float la = row[b];
     const float o = wt * (__expf(base + la + pc[b]) - __expf(la) * gam);
     if (acc_row != nullptr) atomicAdd(acc_row + b, o);
+    else if (f32_row != nullptr) f32_row[b] += o;
     else dst[b] = __float2bfloat16_rn(o);
   }
 }
@@ -134,15 +169,12 @@ __host__ __device__ inline size_t hmm_backward_smem_floats(int n, int r, bool is
          (is_static ? static_cast<size_t>(n - 1) * r * r : 0);
 }
 
-__global__ void circuit_hmm_backward_kernel(const float* __restrict__ G, const float* __restrict__ logw,
-                                            const float* __restrict__ tables, int table_stride,
-                                            const int* __restrict__ targets, const float* __restrict__ weight,
-                                            float* __restrict__ out, float* __restrict__ post,
-                                            __nv_bfloat16* __restrict__ dsum, int dsum_pitch, float* __restrict__ dT,
-                                            unsigned* work_counter, int W, int n, int r, int sum_rows) {
+__global__ void circuit_hmm_backward_kernel(const CircuitBackwardArgs a_, const float* __restrict__ tables,
+                                            int table_stride, float* __restrict__ dT, unsigned* work_counter) {
   extern __shared__ __align__(16) float sm[];
   const int lane = threadIdx.x & 31;
   const int wib = threadIdx.x >> 5;
+  const int n = a_.n, r = a_.r, len = a_.len;
   const int rr = r * r;
   const bool is_static = table_stride == 0;
   float* acc = sm;                                                       // static only: [n-1, r, r]
@@ -155,17 +187,20 @@ __global__ void circuit_hmm_backward_kernel(const float* __restrict__ G, const f
     for (int e = threadIdx.x; e < (n - 1) * rr; e += blockDim.x) acc[e] = 0.f;
     __syncthreads();
   }
-  for (int w = next_window(work_counter, lane); w < W; w = next_window(work_counter, lane)) {
-    const float* g = G + static_cast<size_t>(w) * n * r;
-    const float* lw = logw + static_cast<size_t>(w) * sum_rows;
+  // The steps after `len` carry no evidence and the transitions are normalised: the recursion stops at step len - 1.
+  for (int w = next_window(work_counter, lane); w < a_.W; w = next_window(work_counter, lane)) {
+    const float* g = a_.G + static_cast<size_t>(w) * n * r;
+    const float* lw = a_.logw + static_cast<size_t>(w) * a_.sum_rows;
     const float* tb = tables + static_cast<size_t>(w) * table_stride;
-    const float wt = weight[w];
+    const float wt = a_.weight[static_cast<size_t>(w) * a_.weight_stride];
+    const size_t prow = static_cast<size_t>(w) * n * r;
+    const size_t drow = static_cast<size_t>(w) * a_.dsum_pitch;
     // ---- forward, keeping every alpha_i
-    if (n > 1) warp_table_load_async(tabs, tb, rr, lane);
+    if (len > 1) warp_table_load_async(tabs, tb, rr, lane);
     float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
     if (has) alphas[lane] = alpha;
-    for (int i = 1; i < n; ++i) {
-      if (i + 1 < n) {
+    for (int i = 1; i < len; ++i) {
+      if (i + 1 < len) {
         warp_table_load_async(tabs + (i & 1) * rr, tb + static_cast<size_t>(i) * rr, rr, lane);
         cp_async_wait<1>();
       } else {
@@ -186,21 +221,20 @@ __global__ void circuit_hmm_backward_kernel(const float* __restrict__ G, const f
       __syncwarp();
     }
     const float logq = warp_lse(alpha, has);
-    if (lane == 0 && out != nullptr) out[w] = logq;
-    // ---- backward: tables in reverse order; table n-1 is still in its buffer
-    float beta = 0.f;                                                    // beta_{n-1}
-    for (int i = n - 1; i >= 1; --i) {
-      // table i (index i-1) sits in buffer (i-1)&1 if it was the last one loaded or was prefetched below
-      if (i < n - 1) {
+    if (lane == 0 && a_.out != nullptr) a_.out[w] = logq;
+    // ---- backward: tables in reverse order; the table of step len - 1 is still in its buffer
+    float beta = 0.f;                                                    // beta_{len-1}
+    for (int i = len - 1; i >= 1; --i) {
+      if (i < len - 1) {
         cp_async_wait<0>();
         __syncwarp();
       }
       if (i - 1 >= 1) warp_table_load_async(tabs + (i & 1) * rr, tb + static_cast<size_t>(i - 2) * rr, rr, lane);
       const float* A = tabs + ((i - 1) & 1) * rr;
-      const bool valid = targets[static_cast<size_t>(w) * n + i] >= 0;
+      const bool valid = a_.targets[static_cast<size_t>(w) * n + i] >= 0;
       if (has) {
         const float gamma = __expf(alphas[i * r + lane] + beta - logq);
-        post[(static_cast<size_t>(w) * n + i) * r + lane] = valid ? wt * gamma : 0.f;
+        put_post(a_, prow + static_cast<size_t>(i) * r + lane, valid ? wt * gamma : 0.f);
         cvec[lane] = g[i * r + lane] + beta;
       }
       __syncwarp();
@@ -208,18 +242,24 @@ __global__ void circuit_hmm_backward_kernel(const float* __restrict__ G, const f
       if (has) {
         const float al = alphas[(i - 1) * r + lane];
         const float gam_prev = __expf(al + beta_prev - logq);
-        const float* row = A + lane * r;
-        row_grad(row, cvec, al - logq, gam_prev, wt, lane, r,
-                 is_static ? nullptr : dsum + static_cast<size_t>(w) * dsum_pitch + r + static_cast<size_t>(i - 1) * rr + lane * r,
-                 is_static ? acc + static_cast<size_t>(i - 1) * rr + lane * r : nullptr);
+        const size_t off = static_cast<size_t>(r) + static_cast<size_t>(i - 1) * rr + lane * r;
+        row_grad(A + lane * r, cvec, al - logq, gam_prev, wt, lane, r,
+                 (is_static || a_.accumulate) ? nullptr : a_.dsum + drow + off,
+                 is_static ? acc + static_cast<size_t>(i - 1) * rr + lane * r : nullptr,
+                 (!is_static && a_.accumulate) ? a_.dsum_f32 + drow + off : nullptr);
       }
       beta = beta_prev;
       __syncwarp();                                                      // cvec and the table buffer are free again
     }
     if (has) {
       const float gamma0 = __expf(alphas[lane] + beta - logq);
-      post[static_cast<size_t>(w) * n * r + lane] = targets[static_cast<size_t>(w) * n] >= 0 ? wt * gamma0 : 0.f;
-      dsum[static_cast<size_t>(w) * dsum_pitch + lane] = __float2bfloat16_rn(wt * (gamma0 - __expf(lw[lane])));
+      put_post(a_, prow + lane, a_.targets[static_cast<size_t>(w) * n] >= 0 ? wt * gamma0 : 0.f);
+      put_dsum(a_, drow + lane, wt * (gamma0 - __expf(lw[lane])));
+      if (!a_.accumulate) {                                              // slots and tables past the prefix: no gradient
+        for (int i = len; i < n; ++i) a_.post[prow + static_cast<size_t>(i) * r + lane] = 0.f;
+        if (!is_static)
+          for (int e = (len - 1) * rr + lane; e < (n - 1) * rr; e += r) a_.dsum[drow + r + e] = __float2bfloat16_rn(0.f);
+      }
     }
     __syncwarp();
   }
@@ -243,14 +283,11 @@ __host__ __device__ inline size_t btree_backward_warp_floats(int n, int r) {
   return 3 * static_cast<size_t>(n - 1) * r + 2 * static_cast<size_t>(r) * r + 32;
 }
 
-__global__ void circuit_btree_backward_kernel(const float* __restrict__ G, const float* __restrict__ logw,
-                                              const int* __restrict__ targets, const float* __restrict__ weight,
-                                              float* __restrict__ out, float* __restrict__ post,
-                                              __nv_bfloat16* __restrict__ dsum, int dsum_pitch, unsigned* work_counter,
-                                              int W, int n, int r, int sum_rows) {
+__global__ void circuit_btree_backward_kernel(const CircuitBackwardArgs a_, unsigned* work_counter) {
   extern __shared__ __align__(16) float sm[];
   const int wib = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const int n = a_.n, r = a_.r, len = a_.len;
   float* prod = sm + static_cast<size_t>(wib) * btree_backward_warp_floats(n, r);
   float* S = prod + (n - 1) * r;
   float* U = S + (n - 1) * r;
@@ -261,16 +298,16 @@ __global__ void circuit_btree_backward_kernel(const float* __restrict__ G, const
   const int rr = r * r;
   const int ntab = n - 2;
   auto child_of = [&](int t) { return 2 * (first_leaf_node - 1 - (t >> 1)) + 1 + (t & 1); };
-  for (int w = next_window(work_counter, lane); w < W; w = next_window(work_counter, lane)) {
-    const float* g = G + static_cast<size_t>(w) * n * r;
-    const float* lw = logw + static_cast<size_t>(w) * sum_rows;
-    const float wt = weight[w];
-    __nv_bfloat16* ds = dsum + static_cast<size_t>(w) * dsum_pitch;
-    // ---- upward
+  for (int w = next_window(work_counter, lane); w < a_.W; w = next_window(work_counter, lane)) {
+    const float* g = a_.G + static_cast<size_t>(w) * n * r;
+    const float* lw = a_.logw + static_cast<size_t>(w) * a_.sum_rows;
+    const float wt = a_.weight[static_cast<size_t>(w) * a_.weight_stride];
+    const size_t drow = static_cast<size_t>(w) * a_.dsum_pitch;
+    // ---- upward (tokens >= len are summed out: their input units output one)
     if (ntab > 0) warp_table_load_async(tabs, lw + r + static_cast<size_t>(child_of(0) - 1) * rr, rr, lane);
     for (int j = n - 2; j >= first_leaf_node; --j) {
-      const int m = j - first_leaf_node;
-      if (has) prod[j * r + lane] = g[(2 * m) * r + lane] + g[(2 * m + 1) * r + lane];
+      const int t0 = 2 * (j - first_leaf_node);
+      if (has) prod[j * r + lane] = (t0 < len ? g[t0 * r + lane] : 0.f) + (t0 + 1 < len ? g[(t0 + 1) * r + lane] : 0.f);
     }
     __syncwarp();
     float acc = 0.f;
@@ -293,11 +330,11 @@ __global__ void circuit_btree_backward_kernel(const float* __restrict__ G, const
       __syncwarp();
     }
     const float logq = warp_lse(has ? lw[lane] + prod[lane] : 0.f, has);
-    if (lane == 0 && out != nullptr) out[w] = logq;
+    if (lane == 0 && a_.out != nullptr) a_.out[w] = logq;
     // ---- downward, children c = 1 .. n-2 in address order
     if (has) {
       U[lane] = lw[lane];
-      ds[lane] = __float2bfloat16_rn(wt * (__expf(lw[lane] + prod[lane] - logq) - __expf(lw[lane])));
+      put_dsum(a_, drow + lane, wt * (__expf(lw[lane] + prod[lane] - logq) - __expf(lw[lane])));
     }
     if (ntab > 0) warp_table_load_async(tabs, lw + r, rr, lane);
     __syncwarp();
@@ -323,19 +360,35 @@ __global__ void circuit_btree_backward_kernel(const float* __restrict__ G, const
         // gradient of the child's table: lane z (row), over the child's values b
         const float in_z = cur[lane];
         const float gam_parent = __expf(U[j * r + lane] + prod[j * r + lane] - logq);
+        const size_t off = static_cast<size_t>(r) + static_cast<size_t>(c - 1) * rr + lane * r;
         row_grad(tab + lane * r, prod + c * r, in_z - logq, gam_parent, wt, lane, r,
-                 ds + r + static_cast<size_t>(c - 1) * rr + lane * r, nullptr);
+                 a_.accumulate ? nullptr : a_.dsum + drow + off, nullptr, a_.accumulate ? a_.dsum_f32 + drow + off : nullptr);
       }
       __syncwarp();
     }
     // ---- evidence gradients: token i under its owner's posterior
     for (int i = 0; i < n; ++i) {
       const int o = first_leaf_node + (i >> 1);
-      const bool valid = targets[static_cast<size_t>(w) * n + i] >= 0;
-      if (has)
-        post[(static_cast<size_t>(w) * n + i) * r + lane] = valid ? wt * __expf(U[o * r + lane] + prod[o * r + lane] - logq) : 0.f;
+      const bool valid = a_.targets[static_cast<size_t>(w) * n + i] >= 0;
+      if (has) {
+        const size_t idx = (static_cast<size_t>(w) * n + i) * r + lane;
+        if (i < len) put_post(a_, idx, valid ? wt * __expf(U[o * r + lane] + prod[o * r + lane] - logq) : 0.f);
+        else if (!a_.accumulate) a_.post[idx] = 0.f;
+      }
     }
     __syncwarp();
+  }
+}
+
+// fp32 [rows, cols] (pitch src_pitch) -> bf16 (pitch dst_pitch): the accumulated sum-unit logit gradients become the
+// tensor cores' operand.
+__global__ void f32_rows_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int rows, int cols,
+                                        size_t src_pitch, size_t dst_pitch) {
+  const size_t total = static_cast<size_t>(rows) * cols;
+  for (size_t e = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; e < total;
+       e += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const size_t rw = e / cols, c = e - rw * cols;
+    dst[rw * dst_pitch + c] = __float2bfloat16_rn(src[rw * src_pitch + c]);
   }
 }
 

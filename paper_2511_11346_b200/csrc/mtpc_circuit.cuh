@@ -488,6 +488,42 @@ __global__ void __launch_bounds__(kLossThreads) loss_final_kernel(const float* _
   }
 }
 
+// Coefficients of the prefix log-marginals in Eq. (6). With c[t, j] = -gamma^j / (N V_ij) for a valid target (i the
+// sequence of position t) and 0 otherwise, L = sum_t sum_j c[t, j] (P[t, j] - P[t, j-1]) = sum_t sum_j coeff[t, j] P[t, j]
+// with coeff[t, j] = c[t, j] - c[t, j+1] (c[t, n] = 0): the weights of the n backward passes. grid = N, n <= 64.
+__global__ void __launch_bounds__(kLossThreads) loss_coeff_kernel(const int* __restrict__ targets,
+                                                                  float* __restrict__ coeff, int L, int n, int N,
+                                                                  float gamma) {
+  __shared__ int scnt[kLossThreads / 32];
+  __shared__ float cj[64];
+  const int i = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float wgt = 1.f;
+  for (int j = 0; j < n; ++j) {
+    int cnt = 0;
+    for (int t = threadIdx.x; t < L; t += kLossThreads) cnt += targets[(static_cast<size_t>(i) * L + t) * n + j] >= 0;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(kFull, cnt, off);
+    if (lane == 0) scnt[warp] = cnt;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int c = 0;
+      for (int q = 0; q < kLossThreads / 32; ++q) c += scnt[q];
+      cj[j] = c > 0 ? -wgt / (static_cast<float>(N) * static_cast<float>(c)) : 0.f;
+    }
+    wgt *= gamma;
+    __syncthreads();
+  }
+  for (int t = threadIdx.x; t < L; t += kLossThreads) {
+    const size_t row = (static_cast<size_t>(i) * L + t) * n;
+    for (int j = 0; j < n; ++j) {
+      const float here = targets[row + j] >= 0 ? cj[j] : 0.f;
+      const float next = (j + 1 < n && targets[row + j + 1] >= 0) ? cj[j + 1] : 0.f;
+      coeff[row + j] = here - next;
+    }
+  }
+}
+
 // ---------------------------------------------------------------- preparation
 __global__ void f32_to_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t count) {
   size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;

@@ -128,5 +128,20 @@ class DeviceHead:
                                                out["dT_static"])
         return out
 
+    def window_loss_backward(self, num_sequences, sequence_length, gamma, hidden=None, targets=None):
+        """-> dict(slot_loss [n], loss [1], dh, dW_emit, dW_sum, dT_static or None) as fp32 device tensors."""
+        import torch
+        s = self.wl.shape
+        h = self.hidden_device() if hidden is None else hidden
+        t = torch.from_numpy(self.wl.targets).to(self.device) if targets is None else targets
+        T = h.shape[0]
+        f32 = dict(dtype=torch.float32, device=self.device)
+        out = dict(slot_loss=torch.empty(s.n, **f32), loss=torch.empty(1, **f32), dh=torch.empty((T, s.d), **f32),
+                   dW_emit=torch.empty((s.n, s.r, s.v, s.d), **f32), dW_sum=torch.empty((s.sum_rows, s.d), **f32),
+                   dT_static=torch.empty((max(s.n - 1, 1), s.r, s.r), **f32) if s.family == I.HMM else None)
+        self.head.mtpc_window_loss_backward(h, t, num_sequences, sequence_length, gamma, out["slot_loss"], out["loss"],
+                                            out["dh"], out["dW_emit"], out["dW_sum"], out["dT_static"])
+        return out
+
     def close(self):
         self.head.mtpc_destroy()

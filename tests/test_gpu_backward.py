@@ -177,3 +177,37 @@ def test_backward_argument_checks():
     torch.cuda.synchronize()
     assert dh.head.mtpc_get_status() == 0
     dh.close()
+
+
+@pytest.mark.parametrize("family,n,r,v,d,N,L", [(I.CP, 4, 8, 320, 128, 3, 50), (I.CP, 2, 128, 16, 64, 5, 7),
+                                                 (I.HMM, 8, 16, 64, 64, 5, 33), (I.HMM, 1, 4, 32, 64, 2, 9),
+                                                 (I.HMM_CTX, 4, 8, 64, 64, 4, 40), (I.BTREE, 8, 8, 32, 64, 2, 140),
+                                                 (I.BTREE, 2, 4, 32, 64, 3, 11), (I.BTREE, 16, 16, 48, 64, 2, 40)])
+def test_eq6_loss_backward_matches_oracle(family, n, r, v, d, N, L):
+    """The training loss of Eq. 6 and its gradients: one circuit backward pass per prefix length, accumulated, against
+    reverse-mode differentiation of the definition in float64. Windows run past the end of their sequences (masked
+    tails), one sequence has no valid byte in the last slot."""
+    wl = I.make_workload(f"l6_{family}_{n}_{r}", I.HeadShape(family, n, r, v, d), N * L, seed=6000 + n + N + r, weight_std=0.25)
+    t = wl.targets.copy().reshape(N, L, n)
+    for j in range(1, n):
+        t[:, max(L - j, 0):, j] = -1
+    if n > 1:
+        t[0, :, n - 1] = -1
+    t = t.reshape(N * L, n)
+    gamma = 0.8
+    dh = DeviceHead(wl)
+    out = dh.window_loss_backward(N, L, gamma, targets=torch.from_numpy(t).cuda())
+    assert dh.head.mtpc_get_status() == 0
+    ref = og.composite_loss_grad(family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, t, N, gamma)
+    assert np.abs(out["slot_loss"].cpu().numpy() - ref["slot_loss"]).max() <= 2e-3
+    assert abs(float(out["loss"].cpu()[0]) - ref["loss"]) <= 2e-3 * n
+    floor = 2e-5 / N * max(1.0, L ** 0.5)
+    stats = [check("d_hidden", out["dh"], ref["dh"], floor), check("dW_emit", out["dW_emit"], ref["dW_emit"], floor),
+             check("dW_sum", out["dW_sum"], ref["dW_sum"], floor)]
+    if family == I.HMM and n > 1:
+        stats.append(check("dT_static", out["dT_static"][: n - 1], ref["dT_static"], floor))
+    print(f"{wl.name}: (max error / scale, relative L2) per tensor: " + ", ".join(f"({a:.1e}, {b:.1e})" for a, b in stats))
+    # same loss value as the forward-only entry point
+    slot, loss = dh.window_loss(N, L, gamma, targets=torch.from_numpy(t).cuda())
+    assert torch.equal(slot, out["slot_loss"]) and torch.equal(loss, out["loss"])
+    dh.close()
