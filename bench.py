@@ -256,11 +256,46 @@ def measure_backward(torch, dh, wl, hidden, targets, steps: int, peaks):
     dh.head.mtpc_set_timing(0)
     flops = 4.0 * algorithmic_flops(wl)
     tf = flops / (ms * 1e-3) / 1e12
-    return {"call": "mtpc_window_logprob_backward", "ms_per_call": ms, "positions_per_s": wl.T / (ms * 1e-3),
+    eq6 = measure_eq6_step(torch, dh, wl, hidden, targets, out, steps)
+    return {"eq6_training_step": eq6, "call": "mtpc_window_logprob_backward", "ms_per_call": ms, "positions_per_s": wl.T / (ms * 1e-3),
             "phase_ms": {"forward_projection": phase_ms[0], "circuit_backward": phase_ms[1],
                          "projection_gradient_mode": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]},
             "flops_per_call": flops, "achieved_tflops": tf, "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
             "device_status": dh.head.mtpc_get_status()}
+
+
+def measure_eq6_step(torch, dh, wl, hidden, targets, grads, steps: int):
+    """The paper's training loss (Eq. 6, discount 0.8, or 0.9 for n > 8) and its gradients in one call: sequences of 1024
+    positions, windows that run past the end of their sequence masked."""
+    s = wl.shape
+    L = 1024 if wl.T % 1024 == 0 else wl.T
+    N = wl.T // L
+    t = targets.clone().view(N, L, s.n)
+    for j in range(1, s.n):
+        t[:, L - j:, j] = -1
+    t = t.view(wl.T, s.n).contiguous()
+    gamma = 0.9 if s.n > 8 else 0.8
+    f32 = dict(dtype=torch.float32, device="cuda")
+    slot, loss = torch.empty(s.n, **f32), torch.empty(1, **f32)
+    call = lambda: dh.head.mtpc_window_loss_backward(hidden, t, N, L, gamma, slot, loss, *grads[1:])
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    dh.head.mtpc_set_timing(steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    phases = [dh.head.mtpc_get_timing(i) for i in range(steps)]
+    phase_ms = [statistics.mean(p[k] for p in phases) for k in range(len(phases[0]))]
+    dh.head.mtpc_set_timing(0)
+    return {"call": "mtpc_window_loss_backward", "sequences": N, "sequence_length": L, "gamma": gamma, "ms_per_call": ms,
+            "positions_per_s": wl.T / (ms * 1e-3), "loss": float(loss.cpu()[0]),
+            "phase_ms": {"forward_prefix_loss": phase_ms[0], "circuit_backward_passes": phase_ms[1],
+                         "projection_gradient_mode": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]}}
 
 
 def run_ours(args):

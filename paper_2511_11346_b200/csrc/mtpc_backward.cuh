@@ -298,29 +298,46 @@ __global__ void circuit_btree_backward_kernel(const CircuitBackwardArgs a_, unsi
   const int rr = r * r;
   const int ntab = n - 2;
   auto child_of = [&](int t) { return 2 * (first_leaf_node - 1 - (t >> 1)) + 1 + (t & 1); };
+  // A node whose tokens all lie at or after `len` sees no evidence: its subtree evaluates to one, its table has no
+  // gradient, and it is skipped (first token of heap node c: index within its level times the level's width).
+  auto has_evidence = [&](int c) {
+    const int depth = 31 - __clz(c + 1);
+    return ((c + 1 - (1 << depth)) * (n >> depth)) < len;
+  };
   for (int w = next_window(work_counter, lane); w < a_.W; w = next_window(work_counter, lane)) {
     const float* g = a_.G + static_cast<size_t>(w) * n * r;
     const float* lw = a_.logw + static_cast<size_t>(w) * a_.sum_rows;
     const float wt = a_.weight[static_cast<size_t>(w) * a_.weight_stride];
     const size_t drow = static_cast<size_t>(w) * a_.dsum_pitch;
     // ---- upward (tokens >= len are summed out: their input units output one)
-    if (ntab > 0) warp_table_load_async(tabs, lw + r + static_cast<size_t>(child_of(0) - 1) * rr, rr, lane);
     for (int j = n - 2; j >= first_leaf_node; --j) {
       const int t0 = 2 * (j - first_leaf_node);
       if (has) prod[j * r + lane] = (t0 < len ? g[t0 * r + lane] : 0.f) + (t0 + 1 < len ? g[(t0 + 1) * r + lane] : 0.f);
     }
+    auto next_up = [&](int t) {                                          // next table of the upward pass that is needed
+      while (t < ntab && !has_evidence(child_of(t))) ++t;
+      return t;
+    };
+    int buf = 0;
+    int tn = next_up(0);
+    if (tn < ntab) warp_table_load_async(tabs, lw + r + static_cast<size_t>(child_of(tn) - 1) * rr, rr, lane);
     __syncwarp();
     float acc = 0.f;
     for (int t = 0; t < ntab; ++t) {
       const int c = child_of(t);
-      if (t + 1 < ntab) {
-        warp_table_load_async(tabs + ((t + 1) & 1) * rr, lw + r + static_cast<size_t>(child_of(t + 1) - 1) * rr, rr, lane);
-        cp_async_wait<1>();
-      } else {
-        cp_async_wait<0>();
+      float sc = 0.f;                                                    // a subtree without evidence: log 1
+      if (t == tn) {
+        tn = next_up(t + 1);
+        if (tn < ntab) {
+          warp_table_load_async(tabs + (buf ^ 1) * rr, lw + r + static_cast<size_t>(child_of(tn) - 1) * rr, rr, lane);
+          cp_async_wait<1>();
+        } else {
+          cp_async_wait<0>();
+        }
+        __syncwarp();
+        sc = sum_layer_staged(tabs + buf * rr, prod + c * r, lane, r);
+        buf ^= 1;
       }
-      __syncwarp();
-      const float sc = sum_layer_staged(tabs + (t & 1) * rr, prod + c * r, lane, r);
       if (has) S[c * r + lane] = sc;
       acc += sc;
       if (t & 1) {
@@ -336,20 +353,28 @@ __global__ void circuit_btree_backward_kernel(const CircuitBackwardArgs a_, unsi
       U[lane] = lw[lane];
       put_dsum(a_, drow + lane, wt * (__expf(lw[lane] + prod[lane] - logq) - __expf(lw[lane])));
     }
-    if (ntab > 0) warp_table_load_async(tabs, lw + r, rr, lane);
+    auto next_down = [&](int c) {
+      while (c <= ntab && !has_evidence(c)) ++c;
+      return c;
+    };
+    buf = 0;
+    int cn = next_down(1);
+    if (cn <= ntab) warp_table_load_async(tabs, lw + r + static_cast<size_t>(cn - 1) * rr, rr, lane);
     __syncwarp();
-    for (int c = 1; c <= ntab; ++c) {
+    for (int c = cn; c <= ntab; c = cn) {
       const int j = (c - 1) >> 1;
       const int sib = (c & 1) ? c + 1 : c - 1;
-      if (c < ntab) {
-        warp_table_load_async(tabs + (c & 1) * rr, lw + r + static_cast<size_t>(c) * rr, rr, lane);
+      cn = next_down(c + 1);
+      if (cn <= ntab) {
+        warp_table_load_async(tabs + (buf ^ 1) * rr, lw + r + static_cast<size_t>(cn - 1) * rr, rr, lane);
         cp_async_wait<1>();
       } else {
         cp_async_wait<0>();
       }
       if (has) cur[lane] = U[j * r + lane] + S[sib * r + lane];          // in[z]
       __syncwarp();
-      const float* tab = tabs + ((c - 1) & 1) * rr;
+      const float* tab = tabs + buf * rr;
+      buf ^= 1;
       if (has) {
         // message to the child: lane b, over the parent's values z (column of the table)
         float m = -CUDART_INF_F;
