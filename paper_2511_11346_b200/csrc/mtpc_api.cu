@@ -274,6 +274,25 @@ void launch_kernel(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem
 }
 
 // Launch the projection kernel for `rows` positions over the emission groups (with_emit) and / or the sum tiles.
+// Units per work item of the log-likelihood / gradient modes. An item covers its units with 256-column tiles; unless the
+// units end on a tile boundary the last tile is partly wasted (its tail belongs to the next item, which recomputes it).
+// Items are dealt round-robin to `ctas` persistent CTAs, so a launch takes about rounds x tiles-per-item tile times:
+// pick the count that minimises that (v = 320: 4 units = 5 tiles, nothing wasted; v = 272: 8 units = 9 tiles, 6 % wasted
+// but twice as many items as the waste-free 16 units = 17 tiles).
+int choose_group_units(int v, int emit_units, int m_tiles, int ctas) {
+  int best = 1;
+  long long best_cost = -1;
+  const int limit = emit_units < 64 ? emit_units : 64;
+  for (int u = 1; u <= limit; ++u) {
+    const long long tiles = (static_cast<long long>(u) * v + 255) / 256;
+    const long long groups = (emit_units + u - 1) / u;
+    const long long rounds = (groups * m_tiles + ctas - 1) / ctas;
+    const long long cost = rounds * tiles;
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = u; }
+  }
+  return best;
+}
+
 struct GradArgs {            // what the projection kernel needs beyond the forward arguments (backward pass only)
   float* lse_out = nullptr;                  // forward for training: keep the units' log-sum-exps
   const float* lse_in = nullptr;             // gradient mode
@@ -320,6 +339,10 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   p.emit_units = c.n * c.r;
   p.num_groups = with_emit ? tl.num_groups : 0;
   p.group_units = tl.group_units;
+  if (mode != kModeSample && with_emit) {
+    p.group_units = choose_group_units(c.v, p.emit_units, p.m_tiles, h->num_sms);
+    p.num_groups = (p.emit_units + p.group_units - 1) / p.group_units;
+  }
   p.tile_cols = tl.tile_cols;
   p.num_sum_tiles = with_sum ? L.sum_tiles : 0;
   p.sum_cols = L.sum_cols;
