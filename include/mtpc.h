@@ -211,6 +211,9 @@ int mtpc_window_loss(mtpc_head* head, const void* hidden, const int32_t* targets
  *   dT_static     dev [n-1, r, r] fp32: gradient of the static transition logits (MTPC_HMM without the contextual
  *                 flag; required there, ignored otherwise). With MTPC_FLAG_HMM_CONTEXTUAL the gradient of the bias is the
  *                 column sum of the transition-logit gradients and is not returned separately.
+ * Long windows: the circuit backward kernels keep the messages of every step / node of a window in shared memory and use
+ * fewer warps per CTA as n*r grows; a static HMM whose (n-1)*r*r transition-gradient accumulator does not fit beside them
+ * (n = 64 with r = 32) returns MTPC_ERR_UNSUPPORTED.
  * Arithmetic: posteriors in fp32; the logit gradients are rounded to bf16 (the operand type of the tensor cores) before
  * the three weight-sized GEMMs, fp32 accumulation. dT_static is accumulated with atomic adds (order not fixed).
  */

@@ -662,6 +662,20 @@ int launch_plain_gemm(mtpc_head* h, const void* A, size_t lda, const void* Bm, s
   return check_launch();
 }
 
+// Warps per CTA of the circuit backward kernels: as many of 8, 4, 2, 1 as keep the CTA's shared memory within the limit
+// (long windows need n x r floats of messages per warp). 0: not even one warp fits.
+size_t circuit_backward_smem(const mtpc_head* h, int warps) {
+  const mtpc_config& c = h->cfg;
+  if (c.family == MTPC_HMM) return hmm_backward_smem_floats(c.n, c.r, !is_ctx(h), warps) * sizeof(float);
+  if (c.family == MTPC_BTREE) return static_cast<size_t>(warps) * btree_backward_warp_floats(c.n, c.r) * sizeof(float);
+  return 0;
+}
+int circuit_backward_warps(const mtpc_head* h) {
+  for (int w = kCircuitWarps; w >= 1; w >>= 1)
+    if (circuit_backward_smem(h, w) <= static_cast<size_t>(kSmemLimit)) return w;
+  return 0;
+}
+
 int launch_circuit_backward(mtpc_head* h, CircuitBackwardArgs a, float* dT, cudaStream_t st) {
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
@@ -671,17 +685,18 @@ int launch_circuit_backward(mtpc_head* h, CircuitBackwardArgs a, float* dT, cuda
   a.r = c.r;
   a.sum_rows = L.sum_rows;
   unsigned* counter = at<unsigned>(h, L.off_status) + kWorkCounterWord;
-  const int blocks = (a.W + kCircuitWarps - 1) / kCircuitWarps;
-  const int threads = kCircuitWarps * 32;
+  const int warps = c.family == MTPC_CP ? kCircuitWarps : circuit_backward_warps(h);
+  if (warps == 0) return MTPC_ERR_UNSUPPORTED;
+  const int blocks = (a.W + warps - 1) / warps;
+  const int threads = warps * 32;
   const int resident = blocks < 8 * h->num_sms ? blocks : 8 * h->num_sms;
+  const size_t smem = circuit_backward_smem(h, warps);
   if (c.family != MTPC_CP && cudaMemsetAsync(counter, 0, sizeof(unsigned), st) != cudaSuccess) return MTPC_ERR_CUDA;
   if (c.family == MTPC_CP) {
     circuit_cp_backward_kernel<<<blocks, threads, 0, st>>>(a);
   } else if (c.family == MTPC_HMM) {
-    const size_t smem = hmm_backward_smem_floats(c.n, c.r, !is_ctx(h), kCircuitWarps) * sizeof(float);
     circuit_hmm_backward_kernel<<<resident, threads, smem, st>>>(a, hmm_tables(h), hmm_table_stride(h), dT, counter);
   } else {
-    const size_t smem = kCircuitWarps * btree_backward_warp_floats(c.n, c.r) * sizeof(float);
     circuit_btree_backward_kernel<<<resident, threads, smem, st>>>(a, counter);
   }
   h->launches++;
@@ -691,17 +706,16 @@ int launch_circuit_backward(mtpc_head* h, CircuitBackwardArgs a, float* dT, cuda
 // Shared-memory attributes of the circuit backward kernels (per function, set to what this head needs).
 int set_backward_attributes(const mtpc_head* head) {
   const mtpc_config& c = head->cfg;
+  if (c.family == MTPC_CP) return MTPC_OK;
+  const int warps = circuit_backward_warps(head);
+  if (warps == 0) return MTPC_ERR_UNSUPPORTED;
+  const size_t smem = circuit_backward_smem(head, warps);
   bool fail = false;
-  if (c.family == MTPC_HMM) {
-    const size_t smem = hmm_backward_smem_floats(c.n, c.r, !is_ctx(head), kCircuitWarps) * sizeof(float);
-    if (smem > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;
-    if (smem > 48 * 1024)
+  if (smem > 48 * 1024) {
+    if (c.family == MTPC_HMM)
       fail |= cudaFuncSetAttribute(circuit_hmm_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    static_cast<int>(smem)) != cudaSuccess;
-  } else if (c.family == MTPC_BTREE) {
-    const size_t smem = kCircuitWarps * btree_backward_warp_floats(c.n, c.r) * sizeof(float);
-    if (smem > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;
-    if (smem > 48 * 1024)
+    else
       fail |= cudaFuncSetAttribute(circuit_btree_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    static_cast<int>(smem)) != cudaSuccess;
   }

@@ -31,6 +31,10 @@ SMALL = [
     (I.BTREE, 4, 16, 256, 128, 130),
     (I.BTREE, 8, 32, 48, 64, 33),
     (I.BTREE, 16, 8, 32, 64, 70),
+    (I.BTREE, 64, 2, 16, 64, 3),
+    (I.BTREE, 64, 32, 16, 64, 9),          # long windows: fewer warps per CTA so that the messages still fit shared memory
+    (I.HMM, 32, 16, 16, 64, 11),
+    (I.HMM_CTX, 64, 32, 16, 64, 4),
 ]
 
 
@@ -142,6 +146,18 @@ def test_large_vocabulary_heads_evaluate_and_train_but_do_not_draft(family, n, r
     with pytest.raises(B.MtpcError) as e:
         dh.draft_sample(1)
     assert e.value.code == -3
+    dh.close()
+
+
+def test_backward_refuses_what_does_not_fit_shared_memory():
+    from paper_2511_11346_b200 import binding as B
+    # static transitions: the per-CTA accumulator of the transition gradients alone is (n-1) r^2 floats = 258 KB here
+    wl = I.make_workload("bwd_big", I.HeadShape(I.HMM, 64, 32, 16, 64), 4, seed=13, weight_std=0.3)
+    dh = DeviceHead(wl)
+    with pytest.raises(B.MtpcError) as e:
+        dh.window_logprob_backward(torch.ones(4, device="cuda"))
+    assert e.value.code == -3
+    assert np.isfinite(dh.window_logprob().cpu().numpy()).all()      # the forward path is unaffected
     dh.close()
 
 

@@ -307,3 +307,37 @@ def test_padded_vocabulary_every_entry_point(family, n, r, v, vv, d, P, wpp):
         scale = np.abs(want).max()
         assert np.abs(got_t - want).max() <= 1e-2 * scale + 1e-4, name
     dh.close()
+
+
+def test_argument_checks_of_prefix_loss_and_accept_calls():
+    wl = I.make_workload("args2", I.HeadShape(I.CP, 2, 2, 16, 64), 6, seed=3, wpp=2)
+    dh = DeviceHead(wl, max_positions=6, max_wpp=2)
+    lib = B.lib()
+    st = torch.cuda.current_stream().cuda_stream
+    h = dh.hidden_device()
+    t = torch.from_numpy(wl.targets).cuda()
+    u = torch.from_numpy(wl.uniforms).cuda()
+    f32 = dict(dtype=torch.float32, device="cuda")
+    pre, slot, loss = torch.full((6, 2), 7.0, **f32), torch.empty(2, **f32), torch.empty(1, **f32)
+    ob = torch.empty((12, 2), dtype=torch.int32, device="cuda")
+    hd = dh.head.handle
+    assert lib.mtpc_window_prefix_logprob(hd, h.data_ptr(), t.data_ptr(), 0, pre.data_ptr(), st) == 0
+    torch.cuda.synchronize()
+    assert (pre == 7.0).all()                                                          # T = 0 touches nothing
+    assert lib.mtpc_window_prefix_logprob(hd, h.data_ptr(), t.data_ptr(), 7, pre.data_ptr(), st) == -2
+    assert lib.mtpc_window_prefix_logprob(hd, h.data_ptr(), None, 6, pre.data_ptr(), st) == -1
+    assert lib.mtpc_draft_sample_prefix(hd, h.data_ptr(), 6, 3, u.data_ptr(), ob.data_ptr(), pre.data_ptr(), st) == -2
+    assert lib.mtpc_draft_sample_prefix(hd, h.data_ptr(), 6, 2, u.data_ptr(), None, pre.data_ptr(), st) == -1
+    import ctypes
+    g = ctypes.c_float(0.8)
+    assert lib.mtpc_window_loss(hd, h.data_ptr(), t.data_ptr(), 3, 2, g, slot.data_ptr(), loss.data_ptr(), st) == 0
+    assert lib.mtpc_window_loss(hd, h.data_ptr(), t.data_ptr(), 4, 2, g, slot.data_ptr(), loss.data_ptr(), st) == -2   # 8 > 6
+    assert lib.mtpc_window_loss(hd, h.data_ptr(), t.data_ptr(), 0, 2, g, slot.data_ptr(), loss.data_ptr(), st) == -2
+    assert lib.mtpc_window_loss(hd, h.data_ptr(), t.data_ptr(), 3, 2, g, None, loss.data_ptr(), st) == -1
+    assert lib.mtpc_speculative_accept(hd, 6, 3, ob.data_ptr(), pre.data_ptr(), pre.data_ptr(), pre.data_ptr(), ob.data_ptr(),
+                                       ob.data_ptr(), st) == -2
+    assert lib.mtpc_speculative_accept(hd, 6, 2, None, pre.data_ptr(), pre.data_ptr(), pre.data_ptr(), ob.data_ptr(),
+                                       ob.data_ptr(), st) == -1
+    torch.cuda.synchronize()
+    assert dh.head.mtpc_get_status() == 0
+    dh.close()
