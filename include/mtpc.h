@@ -173,8 +173,7 @@ int mtpc_draft_sample_prefix(mtpc_head* head, const void* hidden, int32_t P, int
  * the latent that owns the slot; it is evaluated from the logits the draft call left in the workspace. Hence:
  *   - the call must follow mtpc_draft_sample / mtpc_draft_sample_prefix on this head with the same P and hidden
  *     states, with no other call on the head in between, else MTPC_ERR_STATE;
- *   - only drafts of P <= 128 positions with r <= 32 keep that state (decode-time batches): otherwise
- *     MTPC_ERR_UNSUPPORTED.
+ *   - only drafts of P <= 128 positions keep that state (decode-time batches): otherwise MTPC_ERR_UNSUPPORTED.
  * A uniform outside [0,1) or a draft byte outside [0,v) sets the status bit and yields -1 / -1 for that window.
  */
 int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32_t* draft_bytes,
@@ -269,7 +268,7 @@ int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags);
  *                        [3] transposes and the plain GEMMs.
  *   mtpc_window_loss_backward: [0] forward projection + prefix marginals + loss, [1] the n circuit backward passes,
  *                        [2] and [3] as above.
- *   mtpc_draft_sample, mtpc_draft_sample_prefix:   P <= 128 positions and r <= 32: [0] one pass over all weights (logits of every unit),
+ *   mtpc_draft_sample, mtpc_draft_sample_prefix:   P <= 128 positions: [0] one pass over all weights (logits of every unit),
  *                        [1] per-slot latent + byte draws and evidence, [2] circuit evaluation.
  *                        Otherwise: [0] sum-unit GEMM, [1] latent sampling, [2] GEMM + inverse-CDF epilogue,
  *                        [3] GEMM + gather epilogue on the drafted bytes, [4] circuit evaluation.

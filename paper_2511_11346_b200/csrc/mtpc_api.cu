@@ -143,7 +143,8 @@ int plan(const mtpc_config& c, Layout* L) {
   L->off_G = take(L->max_windows * c.n * c.r * 4);
   L->off_logw = take(static_cast<size_t>(c.max_positions) * L->sum_rows * 4);
   L->off_sel = take(L->max_windows * c.n * 4);
-  L->decode_max_p = (c.r <= 32 && L->can_draft) ? (c.max_positions < kDecodeMaxP ? c.max_positions : kDecodeMaxP) : 0;
+  // (latents of more than 32 values are handled for the mixture only; HMM and BTree are limited to r <= 32 anyway)
+  L->decode_max_p = L->can_draft ? (c.max_positions < kDecodeMaxP ? c.max_positions : kDecodeMaxP) : 0;
   L->off_logits = take(static_cast<size_t>(L->decode_max_p) * emit_units * c.v * 4);
   L->off_unit_lse = take(static_cast<size_t>(L->decode_max_p) * emit_units * 4);
   L->off_prefix = take(static_cast<size_t>(c.max_positions) * c.n * 4);
@@ -381,7 +382,8 @@ size_t btree_smem_bytes(int n, int r, bool with_prefix) {
 // Circuit evaluation of W windows: out[w] = joint log-prob (may be NULL when prefix is given); prefix (may be NULL)
 // [W, n] = log-marginals of the prefixes x_0..x_i.
 // dependent: the launch directly follows draft_slot_kernel, which has zeroed the work counter, and may overlap its tail.
-int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cudaStream_t st, bool dependent = false) {
+int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cudaStream_t st, bool dependent = false,
+                   bool raw_mixture = false) {
   if (W <= 0) return MTPC_OK;
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
@@ -396,7 +398,8 @@ int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cuda
     if (cudaMemsetAsync(counter, 0, sizeof(unsigned), st) != cudaSuccess) return MTPC_ERR_CUDA;
   }
   if (c.family == MTPC_CP) {
-    launch_kernel(circuit_cp_kernel, blocks, threads, 0, st, dependent, G, logw, out, prefix, W, wpp, c.n, c.r, L.sum_rows);
+    launch_kernel(circuit_cp_kernel, blocks, threads, 0, st, dependent, G, logw, out, prefix, W, wpp, c.n, c.r, L.sum_rows,
+                  raw_mixture ? 1 : 0);
   } else if (c.family == MTPC_HMM) {
     launch_kernel(circuit_hmm_stream_kernel, resident, threads, hmm_stream_smem_bytes(c.r), st, dependent, G, logw,
                   hmm_tables(h), hmm_table_stride(h), out, prefix, counter, W, wpp, c.n, c.r, L.sum_rows);
@@ -559,7 +562,7 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
     pt.end();
     if ((rc = check_launch()) != MTPC_OK) return rc;
     pt.begin();
-    rc = launch_circuit(h, W, wpp, out_logprob, out_prefix, st, /*dependent=*/h->ring == 0);
+    rc = launch_circuit(h, W, wpp, out_logprob, out_prefix, st, /*dependent=*/h->ring == 0, /*raw_mixture=*/c.r > 32);
     pt.end();
     return rc;
   }

@@ -37,13 +37,27 @@ __device__ __forceinline__ float warp_lse(float val, bool has) {
 // summed out (Algorithm 3's marginals): for a mixture that is the same log-sum-exp over the first i+1 slots only.
 __global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __restrict__ logw,
                                   float* __restrict__ out, float* __restrict__ prefix, int W, int wpp, int n, int r,
-                                  int sum_rows) {
+                                  int sum_rows, int raw_mixture) {
   grid_dependency_wait();   // G and log omega come from the kernel before this one
   const int w = blockIdx.x * kCircuitWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (w >= W) return;
   const float* g = G + static_cast<size_t>(w) * n * r;
   const float* lw = logw + static_cast<size_t>(w / wpp) * sum_rows;
+  // raw_mixture: logw holds the mixture LOGITS (the few-position draft path with more than 32 components leaves the
+  // softmax to its consumers): log omega_k = logit_k - LSE(logits), so LSE(logits) is subtracted from every result.
+  float norm = 0.f;
+  if (raw_mixture) {
+    float m = -CUDART_INF_F, s = 0.f;
+    for (int k = lane; k < r; k += 32) lse_merge(m, s, lw[k], 1.f);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float m2 = __shfl_xor_sync(kFull, m, off);
+      const float s2 = __shfl_xor_sync(kFull, s, off);
+      lse_merge(m, s, m2, s2);
+    }
+    norm = m + __logf(s);
+  }
   if (prefix != nullptr) {
     // running sums of up to 4 units per lane (r <= 128); one warp log-sum-exp per slot
     float a[4];
@@ -66,7 +80,7 @@ __global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __re
         const float s2 = __shfl_xor_sync(kFull, s, off);
         lse_merge(m, s, m2, s2);
       }
-      last = m + __logf(s);
+      last = m + __logf(s) - norm;
       if (lane == 0) prefix[static_cast<size_t>(w) * n + i] = last;
     }
     if (lane == 0 && out != nullptr) out[w] = last;
@@ -85,7 +99,7 @@ __global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __re
     const float s2 = __shfl_xor_sync(kFull, s, off);
     lse_merge(m, s, m2, s2);
   }
-  if (lane == 0) out[w] = m + __logf(s);
+  if (lane == 0) out[w] = m + __logf(s) - norm;
 }
 
 // Eq. (BTree), bottom-up over the heap-ordered latent tree. Node j >= 1 has the table

@@ -7,7 +7,9 @@
 //                             positions on the N axis (TMEM columns). Emission logits go to a small scratch
 //                             [P, n*r*v] fp32 (P is tiny here, so this is a few MB against hundreds of MB of
 //                             weights); sum-unit logits are log-softmaxed over their groups of r rows (= lanes,
-//                             by warp shuffles) and written as log omega [P, S*r].
+//                             by warp shuffles) and written as log omega [P, S*r]. A mixture of more than 32
+//                             components (CP, r = 64 or 128) spans several warps: its logits are written as they
+//                             are, and the kernels that follow normalise them where they need to.
 //                             Weight rows are cut into tiles of `tile_rows` <= 128 rows, chosen by the host so that
 //                             the tiles divide evenly over the persistent CTAs; each CTA takes a contiguous run
 //                             of tiles and walks K once per pass of up to three tiles, which share one copy of
@@ -207,7 +209,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_decode_gemm_kernel(const
         for (int b = 0; b < (p.P + 15) / 16; ++b) {
           float x[16];
           tmem_ld16(tcol + b * 16, x);
-          if (t.is_sum) {
+          if (t.is_sum && p.r <= 32) {
 #pragma unroll
             for (int c = 0; c < 16; ++c) x[c] += bias;
             // log-softmax over the r rows of a sum unit = r adjacent lanes (r a power of two <= 32); the 16
@@ -269,6 +271,47 @@ __device__ __forceinline__ int warp_inv_cdf_logp(float logp, int r, float u, int
   const float cum = warp_scan_incl(pr, lane);
   const unsigned hit = __ballot_sync(kFull, lane < r && u < cum);
   return hit ? __ffs(hit) - 1 : r - 1;
+}
+
+// The same draw over the softmax of r <= 128 unnormalised logits x[0..r): lane l owns the consecutive indices
+// [l * per, (l + 1) * per), per = ceil(r / 32) <= 4; u * total < running sum, index order, no division.
+__device__ __forceinline__ int warp_inv_cdf_logits_wide(const float* __restrict__ x, int r, float u, int lane) {
+  const int per = (r + 31) / 32;
+  const int k0 = lane * per;
+  float xv[4];
+  float m = -CUDART_INF_F;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    xv[q] = (q < per && k0 + q < r) ? x[k0 + q] : -CUDART_INF_F;
+    m = fmaxf(m, xv[q]);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
+  float part = 0.f;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    xv[q] = __expf(xv[q] - m);       // padding: exp(-inf) = 0
+    part += xv[q];
+  }
+  const float incl = warp_scan_incl(part, lane);
+  const float total = __shfl_sync(kFull, incl, 31);
+  const float thr = u * total;
+  const unsigned hit = __ballot_sync(kFull, thr < incl);
+  if (!hit) return r - 1;
+  const int src = __ffs(hit) - 1;
+  const float before = __shfl_up_sync(kFull, incl, 1);
+  int found = -1;
+  if (lane == src) {
+    float cum = lane == 0 ? 0.f : before;
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (found < 0 && q < per && k0 + q < r) {
+        cum += xv[q];
+        if (thr < cum) found = k0 + q;
+      }
+    if (found < 0) found = min(k0 + per, r) - 1;
+  }
+  return __shfl_sync(kFull, found, src);
 }
 
 // Tables the latent draws of slot i walk through (Algorithm 1 at the sum units), in the order they are used.
@@ -376,7 +419,8 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     if (bad) {
       if (lane == 0) atomicOr(status, 2u);
     } else {
-      int z = warp_inv_cdf_logp(lane < r ? lw[lane] : 0.f, r, u[0], lane);
+      int z = r > 32 ? warp_inv_cdf_logits_wide(lw, r, u[0], lane)     // CP only; the mixture logits are unnormalised
+                     : warp_inv_cdf_logp(lane < r ? lw[lane] : 0.f, r, u[0], lane);
       if (family == 1) {
         for (int st = 0; st < chain; ++st) {
           const float* tab = tables_in_smem ? tabs + st * rr : hmm + static_cast<size_t>(st) * rr;
@@ -427,17 +471,20 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     }
     if (lane == 0) out_bytes[w * n + i] = byte;
     // evidence of the drafted byte under every input unit of the slot (a missing byte is marginalised)
-    if (lane < r) G[(w * n + i) * r + lane] = byte < 0 ? 0.f : row[static_cast<size_t>(lane) * v + byte] - unit_lse[lane];
+    for (int k = lane; k < r; k += 32)
+      G[(w * n + i) * r + k] = byte < 0 ? 0.f : row[static_cast<size_t>(k) * v + byte] - unit_lse[k];
   }
 }
 
 // ---------------------------------------------------------------- acceptance stage (Algorithm 3)
 constexpr int kAcceptWarps = 4;
 
-// Per-warp shared memory of spec_accept_kernel, in floats: the residual weights of the v bytes, and for the binary
-// tree the product and sum-layer vectors of every node, one staged table and one vector.
+// Per-warp shared memory of spec_accept_kernel, in floats: the residual weights of the v bytes, the weight and the
+// log-sum-exp of every input unit of the slot (2 r), and for the binary tree the product and sum-layer vectors of every
+// node, one staged table and one vector.
 __host__ __device__ inline size_t accept_warp_floats(int family, int n, int r, int v) {
-  return static_cast<size_t>(v) + (family == 2 ? 2 * static_cast<size_t>(n - 1) * r + static_cast<size_t>(r) * (r + 1) + r : 0);
+  return static_cast<size_t>(v) + 2 * static_cast<size_t>(r) +
+         (family == 2 ? 2 * static_cast<size_t>(n - 1) * r + static_cast<size_t>(r) * (r + 1) + r : 0);
 }
 
 // One warp per drafted window w (position p = w / wpp). Inputs: the draft's bytes and prefix log-marginals, the
@@ -508,10 +555,43 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
       const size_t unit = (static_cast<size_t>(pos) * n + i) * r + lane;
       return logits[unit * v + x[i]] - unit_lse[unit];
     };
+    float* cw = mres + v;                                // [r] weight of every input unit of slot s
+    float* cl = cw + r;                                  // [r] its log-sum-exp
     float c = 0.f;
     if (family == 0) {
-      c = has ? lw[lane] : 0.f;
-      for (int i = 0; i < s; ++i) c += has ? g_of(i) : 0.f;
+      // mixture of up to 128 components: lane handles k = lane, lane + 32, ...; the weights need no normalisation of
+      // log omega (they are normalised below), so unnormalised mixture logits (r > 32) are as good
+      float cq[4];
+      float m = -CUDART_INF_F, sacc = 0.f;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int k = lane + 32 * q;
+        cq[q] = -CUDART_INF_F;
+        if (k < r) {
+          float a = lw[k];
+          for (int i = 0; i < s; ++i) {
+            const size_t unit = (static_cast<size_t>(pos) * n + i) * r + k;
+            a += logits[unit * v + x[i]] - unit_lse[unit];
+          }
+          cq[q] = a;
+          lse_merge(m, sacc, a, 1.f);
+        }
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        const float m2 = __shfl_xor_sync(kFull, m, off);
+        const float s2 = __shfl_xor_sync(kFull, sacc, off);
+        lse_merge(m, sacc, m2, s2);
+      }
+      const float lse_all = m + __logf(sacc);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int k = lane + 32 * q;
+        if (k < r) {
+          cw[k] = __expf(cq[q] - lse_all);
+          cl[k] = unit_lse[(static_cast<size_t>(pos) * n + s) * r + k];
+        }
+      }
     } else if (family == 1) {
       float alpha = has ? lw[lane] : -CUDART_INF_F;
       for (int i = 0; i < s; ++i) {
@@ -528,7 +608,7 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
       }
       c = alpha;
     } else {
-      float* prod = mres + v;
+      float* prod = cl + r;
       float* S = prod + (n - 1) * r;
       float* table = S + (n - 1) * r;
       float* cur = table + r * (r + 1);
@@ -572,18 +652,20 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
       const int other_leaf = s ^ 1;
       c = up + ((has && other_leaf < s) ? g_of(other_leaf) : 0.f);
     }
-    const float c_lse = warp_lse(c, has);             // every lane takes part in the shuffles
-    const float cprob = has ? __expf(c - c_lse) : 0.f;
-    const float ulse = has ? unit_lse[(static_cast<size_t>(pos) * n + s) * r + lane] : 0.f;
+    if (family != 0) {                                   // HMM, BTree: one weight per lane (r <= 32)
+      const float c_lse = warp_lse(c, has);              // every lane takes part in the shuffles
+      if (has) {
+        cw[lane] = __expf(c - c_lse);
+        cl[lane] = unit_lse[(static_cast<size_t>(pos) * n + s) * r + lane];
+      }
+    }
+    __syncwarp();
     const float* lrow = logits + (static_cast<size_t>(pos) * n + s) * r * v;   // [r, v] logits of slot s
     for (int b0 = 0; b0 < v; b0 += 32) {
       const int b = b0 + lane;
       float q = 0.f;
-      for (int k = 0; k < r; ++k) {
-        const float ck = __shfl_sync(kFull, cprob, k);
-        const float lk = __shfl_sync(kFull, ulse, k);
-        if (b < vv) q = fmaf(ck, __expf(lrow[static_cast<size_t>(k) * v + b] - lk), q);
-      }
+      if (b < vv)
+        for (int k = 0; k < r; ++k) q = fmaf(cw[k], __expf(lrow[static_cast<size_t>(k) * v + b] - cl[k]), q);
       if (b < v) mres[b] = b < vv ? fmaxf(0.f, trow[b] - q) : 0.f;   // padding symbols carry no mass
     }
   }

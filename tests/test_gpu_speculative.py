@@ -158,6 +158,8 @@ ACCEPT_SMALL = [
     (I.CP, 1, 2, 16, 64, 3, 4),
     (I.CP, 4, 8, 320, 128, 5, 16),
     (I.CP, 3, 32, 48, 64, 7, 8),
+    (I.CP, 3, 64, 48, 64, 5, 16),          # more than 32 components: the mixture logits reach the kernels unnormalised
+    (I.CP, 2, 128, 16, 64, 4, 16),
     (I.HMM, 1, 4, 32, 64, 2, 8),
     (I.HMM, 6, 8, 64, 128, 9, 8),
     (I.HMM, 4, 32, 512, 64, 3, 16),
