@@ -401,6 +401,32 @@ def run_ours(args):
     if args.backward and world == 1:
         backward = measure_backward(torch, dh, wl, hidden, targets, steps=max(5, min(args.steps, 30)), peaks=peaks)
 
+    draft_many = None
+    if wl.wpp and world == 1:       # configs[3]: draft one window per position over the whole batch (many-position path)
+        u = torch.from_numpy(wl.uniforms).cuda()
+        W = wl.T * wl.wpp
+        ob = torch.empty((W, s.n), dtype=torch.int32, device="cuda")
+        ol = torch.empty(W, dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            head.mtpc_draft_sample(hidden, wl.wpp, u, ob, ol)
+        torch.cuda.synchronize()
+        dsteps = max(3, min(args.steps, 30))
+        head.mtpc_set_timing(dsteps)
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record()
+        for _ in range(dsteps):
+            head.mtpc_draft_sample(hidden, wl.wpp, u, ob, ol)
+        d1.record()
+        torch.cuda.synchronize()
+        dms = d0.elapsed_time(d1) / dsteps
+        dph = [head.mtpc_get_timing(i) for i in range(dsteps)]
+        head.mtpc_set_timing(0)
+        draft_many = {"call": "mtpc_draft_sample over the whole batch", "windows": W, "ms_per_call": dms,
+                      "windows_per_s": W / (dms * 1e-3),
+                      "phase_ms": [statistics.mean(p[k] for p in dph) for k in range(len(dph[0]))],
+                      "phases": "sum-unit GEMM, latent draws, GEMM + inverse-CDF epilogue, GEMM + gather epilogue on the "
+                                "drafted bytes, circuit", "device_status": head.mtpc_get_status()}
+
     draft, sweep = None, None
     if not args.no_draft and world == 1:
         if args.decode_cells == "all":
@@ -434,6 +460,8 @@ def run_ours(args):
     }
     if backward is not None:
         line["backward"] = backward
+    if draft_many is not None:
+        line["draft_whole_batch"] = draft_many
     if draft is not None:
         line["draft"] = draft
         line["decode_sweep"] = sweep
