@@ -227,3 +227,28 @@ def test_eq6_loss_backward_matches_oracle(family, n, r, v, d, N, L):
     slot, loss = dh.window_loss(N, L, gamma, targets=torch.from_numpy(t).cuda())
     assert torch.equal(slot, out["slot_loss"]) and torch.equal(loss, out["loss"])
     dh.close()
+
+
+def test_per_kernel_timing_of_the_training_calls():
+    wl = I.make_workload("timing", I.HeadShape(I.BTREE, 4, 8, 32, 64), 40, seed=14, wpp=2, weight_std=0.3)
+    dh = DeviceHead(wl)
+    head = dh.head
+    head.mtpc_set_timing(4)
+    w = torch.ones(40, device="cuda")
+    dh.window_logprob_backward(w)
+    ph = head.mtpc_get_timing(0)
+    assert len(ph) == 4 and all(p > 0 for p in ph)            # forward, circuit backward, gradient-mode projection, GEMMs
+    dh.window_loss_backward(4, 10, 0.8)
+    ph = head.mtpc_get_timing(0)
+    assert len(ph) == 4 and all(p > 0 for p in ph)            # forward+prefix+loss, the n circuit passes, projection, GEMMs
+    assert len(head.mtpc_get_timing(1)) == 4                  # the call before is still in the ring
+    b, pre = dh.draft_sample_prefix(2)
+    assert len(head.mtpc_get_timing(0)) == 3                  # few-position draft: weight pass, per-slot kernel, circuit
+    p = torch.from_numpy(I.target_rows(1, 1, (80, 5, 32))).cuda()
+    u = torch.from_numpy(I.uniforms(1, 2, (80, 5))).cuda()
+    dh.speculative_accept(40, 2, b, pre, p, u)
+    assert len(head.mtpc_get_timing(0)) == 1
+    head.mtpc_set_timing(0)
+    assert head.mtpc_get_timing(0) == []
+    assert dh.head.mtpc_get_status() == 0
+    dh.close()
