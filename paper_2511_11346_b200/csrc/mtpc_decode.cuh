@@ -569,7 +569,8 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
         cq[q] = -CUDART_INF_F;
         if (k < r) {
           float a = lw[k];
-          for (int i = 0; i < s; ++i) {
+#pragma unroll 4
+          for (int i = 0; i < s; ++i) {                     // independent gathers: several in flight
             const size_t unit = (static_cast<size_t>(pos) * n + i) * r + k;
             a += logits[unit * v + x[i]] - unit_lse[unit];
           }
@@ -664,8 +665,23 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
     for (int b0 = 0; b0 < v; b0 += 32) {
       const int b = b0 + lane;
       float q = 0.f;
-      if (b < vv)
-        for (int k = 0; k < r; ++k) q = fmaf(cw[k], __expf(lrow[static_cast<size_t>(k) * v + b] - cl[k]), q);
+      if (b < vv) {
+        // the r logits of byte b come from r different rows: eight loads in flight at a time, two accumulation chains
+        float q1 = 0.f;
+        int k = 0;
+        for (; k + 8 <= r; k += 8) {
+          float xv[8];
+#pragma unroll
+          for (int t = 0; t < 8; ++t) xv[t] = lrow[static_cast<size_t>(k + t) * v + b];
+#pragma unroll
+          for (int t = 0; t < 8; t += 2) {
+            q = fmaf(cw[k + t], __expf(xv[t] - cl[k + t]), q);
+            q1 = fmaf(cw[k + t + 1], __expf(xv[t + 1] - cl[k + t + 1]), q1);
+          }
+        }
+        for (; k < r; ++k) q = fmaf(cw[k], __expf(lrow[static_cast<size_t>(k) * v + b] - cl[k]), q);
+        q += q1;
+      }
       if (b < v) mres[b] = b < vv ? fmaxf(0.f, trow[b] - q) : 0.f;   // padding symbols carry no mass
     }
   }
