@@ -257,11 +257,46 @@ def measure_backward(torch, dh, wl, hidden, targets, steps: int, peaks):
     flops = 4.0 * algorithmic_flops(wl)
     tf = flops / (ms * 1e-3) / 1e12
     eq6 = measure_eq6_step(torch, dh, wl, hidden, targets, out, steps)
-    return {"eq6_training_step": eq6, "call": "mtpc_window_logprob_backward", "ms_per_call": ms, "positions_per_s": wl.T / (ms * 1e-3),
+    lowrank = measure_lowrank(torch, wl, out[2], steps, peaks) if s.v <= 1536 else None
+    return {"eq6_training_step": eq6, "lowrank_unembeddings": lowrank, "call": "mtpc_window_logprob_backward", "ms_per_call": ms, "positions_per_s": wl.T / (ms * 1e-3),
             "phase_ms": {"forward_projection": phase_ms[0], "circuit_backward": phase_ms[1],
                          "projection_gradient_mode": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]},
             "flops_per_call": flops, "achieved_tflops": tf, "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
             "device_status": dh.head.mtpc_get_status()}
+
+
+def measure_lowrank(torch, wl, dW_emit, steps: int, peaks, k: int = 16):
+    """Shared unembeddings with rank-k adaptors (App. G) on the workload's head shape: the composition
+    U_ij = W_i + A_ij B_ij and the gradient carried back from dW_emit, each against one pass over its tensors in HBM."""
+    from paper_2511_11346_b200.runner import lowrank_backward, lowrank_compose, to_device_bf16
+    s = wl.shape
+    Wb, A, Bm = I.lowrank_parameters(s.n, s.r, s.v, s.d, k, seed=97)
+    Wb, A, Bm = to_device_bf16(Wb), to_device_bf16(A), to_device_bf16(Bm)
+    units = s.n * s.r
+    nU = units * s.v * s.d
+    small = s.n * s.v * s.d + units * s.v * k + units * k * s.d
+
+    def timed(call):
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    ms_c = timed(lambda: lowrank_compose(Wb, A, Bm))
+    ms_b = timed(lambda: lowrank_backward(A, Bm, dW_emit))
+    bytes_c = 2 * nU + 2 * small                       # write U (bf16), read W, A, B once
+    bytes_b = 4 * nU + 2 * small + 4 * small            # read dW_emit (fp32) once, read A, B, write the three gradients
+    hbm = peaks["hbm_gbs"]
+    return {"rank": k, "compose_ms": ms_c, "compose_algorithmic_bytes": bytes_c,
+            "compose_frac_of_hbm": bytes_c / (ms_c * 1e-3) / 1e9 / hbm, "backward_ms": ms_b, "backward_kernels": 3,
+            "backward_algorithmic_bytes": bytes_b, "backward_frac_of_hbm": bytes_b / (ms_b * 1e-3) / 1e9 / hbm,
+            "note": "the three gradient kernels each stream dW_emit once: at most a third of the one-pass bound"}
 
 
 def measure_eq6_step(torch, dh, wl, hidden, targets, grads, steps: int):

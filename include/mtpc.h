@@ -236,6 +236,25 @@ int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t
                               float* dT_static, void* stream);
 
 /*
+ * Low-rank-adapted unembeddings (App. G, "Unembedding parameter sharing"): U[i, j] = W_base[i] + A[i, j] B[i, j], one
+ * base matrix per token slot shared by its r components plus a rank-k adaptor per component. The head computes on the
+ * composed tensor; these two calls convert between the shared parameters and it. They need no head.
+ *   W_base  device [n, v, d] bf16      A  device [n, r, v, k] bf16      B  device [n, r, k, d] bf16   (row-major)
+ * mtpc_lowrank_compose writes W_emit_out, device [n, r, v, d] bf16 = round-to-nearest of the fp32 sum; pass it to
+ * mtpc_create_head (which converts it again into the layout of its workspace).
+ * mtpc_lowrank_backward takes the gradient of the composed tensor, dW_emit device [n, r, v, d] fp32 (as written by
+ * the backward calls above), and OVERWRITES
+ *   dW_base [n, v, d] = sum_j dW_emit[i, j],  dA [n, r, v, k] = dW_emit[i, j] B[i, j]^T,  dB [n, r, k, d] = A[i, j]^T dW_emit[i, j]
+ * (device fp32, caller-owned). 1 <= k <= 64 (MTPC_ERR_UNSUPPORTED beyond); v <= 65535 and n r <= 65535
+ * (MTPC_ERR_SHAPE). Any d works; with d a multiple of 4 and 16-byte aligned pointers the kernels use vector accesses.
+ * Asynchronous on `stream`.
+ */
+int mtpc_lowrank_compose(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k, const void* W_base, const void* A,
+                         const void* B, void* W_emit_out, void* stream);
+int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k, const void* A, const void* B,
+                          const float* dW_emit, float* dW_base, float* dA, float* dB, void* stream);
+
+/*
  * Host-buffer variants: same results, but hidden / targets / uniforms are HOST pointers (pinned memory for
  * full copy speed) and the outputs are written to HOST buffers. The copies to and from the device go through
  * staging areas in the workspace; the call returns after the stream has been synchronised, so the outputs are

@@ -18,6 +18,7 @@ What follows which passage:
   next_byte_logprob the conditional q(X_{s+1} | x_1..x_s) as a ratio of two such marginals
   speculative_accept Algorithm 3, acceptance loop and the last byte (residual or target distribution)
   composite_loss    Eq. (6): per-slot negative log-likelihood with valid-token normalisation and discount gamma
+  lowrank_unembedding  App. G, "Unembedding parameter sharing": U_ij = W_i + A_ij B_ij
 
 Readings taken where the paper is silent or garbled (each is listed in the design notes too):
   * BTree: the left half is the first floor(n/2) tokens; a child latent depends on its parent's latent
@@ -413,3 +414,22 @@ def composite_loss(prefix_lq: np.ndarray, targets: np.ndarray, num_sequences: in
         slot[j] = -acc / N
     total = float(sum(gamma ** j * slot[j] for j in range(n)))
     return slot, total
+
+
+# ----------------------------------------------------------------------------------------------------
+# shared unembeddings with low-rank adaptors (App. G)
+# ----------------------------------------------------------------------------------------------------
+def lowrank_unembedding(W_base: np.ndarray, A: np.ndarray, B: np.ndarray) -> np.ndarray:
+    """App. G, "Unembedding parameter sharing": the unembedding matrix of token i and component j is
+    U[i, j] = W_base[i] + A[i, j] @ B[i, j], with W_base [n, v, d], A [n, r, v, k], B [n, r, k, d].
+    Returns U [n, r, v, d]; written as the definition, one (i, j) at a time."""
+    W_base = np.asarray(W_base, dtype=np.float64)
+    A = np.asarray(A, dtype=np.float64)
+    B = np.asarray(B, dtype=np.float64)
+    n, r, v, k = A.shape
+    d = B.shape[-1]
+    U = np.empty((n, r, v, d))
+    for i in range(n):
+        for j in range(r):
+            U[i, j] = W_base[i] + A[i, j] @ B[i, j]
+    return U

@@ -17,7 +17,9 @@ equals central finite differences of the NUMPY oracle's log-likelihood (an indep
 closed forms (CP with r = 1: d/dlogit = weight * (onehot - softmax); a masked byte has zero gradient; gradients of
 a normalised circuit's weights sum to zero within each sum unit); the Eq. 6 loss equals the numpy oracle's
 composite_loss and its gradient equals central finite differences of that; with gamma = 1 and every byte valid it is
-the gradient of the mean joint negative log-likelihood. No function here is left unpinned.
+the gradient of the mean joint negative log-likelihood. lowrank_grad (App. G, shared unembeddings with low-rank
+adaptors) is pinned by central finite differences of the numpy oracle's lowrank_unembedding and by the closed forms
+dW_base = sum_j dU_ij, and dA = 0 where B = 0. No function here is left unpinned.
 """
 from __future__ import annotations
 
@@ -141,3 +143,15 @@ def composite_loss_grad(family: int, h, W_emit, W_sum, T_static, targets, num_se
     zero = lambda t: np.zeros(tuple(t.shape)) if t.grad is None else t.grad.numpy()
     return dict(slot_loss=np.array([float(s.detach()) for s in slot]), loss=float(total.detach()), dh=zero(th), dW_emit=zero(tW),
                 dW_sum=zero(tR), dT_static=None if tT is None else zero(tT))
+
+
+def lowrank_grad(W_base, A, B, dU):
+    """App. G, U[i, j] = W_base[i] + A[i, j] B[i, j]: given the gradient dU [n, r, v, d] of a scalar with respect to
+    the composed unembeddings, its gradient with respect to W_base [n, v, d], A [n, r, v, k] and B [n, r, k, d], by reverse
+    mode through the definition. Returns dict(U, dW_base, dA, dB), numpy float64."""
+    tW = torch.tensor(np.asarray(W_base, dtype=np.float64), requires_grad=True)
+    tA = torch.tensor(np.asarray(A, dtype=np.float64), requires_grad=True)
+    tB = torch.tensor(np.asarray(B, dtype=np.float64), requires_grad=True)
+    U = tW[:, None, :, :] + torch.matmul(tA, tB)
+    (U * torch.tensor(np.asarray(dU, dtype=np.float64))).sum().backward()
+    return dict(U=U.detach().numpy(), dW_base=tW.grad.numpy(), dA=tA.grad.numpy(), dB=tB.grad.numpy())

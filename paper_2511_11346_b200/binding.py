@@ -23,6 +23,7 @@ EXPORTS = [
     "mtpc_launch_count", "mtpc_destroy", "mtpc_status_string", "mtpc_window_logprob_static",
     "mtpc_window_prefix_logprob", "mtpc_draft_sample_prefix", "mtpc_speculative_accept", "mtpc_window_loss",
     "mtpc_backward_workspace_bytes", "mtpc_window_logprob_backward", "mtpc_window_loss_backward",
+    "mtpc_lowrank_compose", "mtpc_lowrank_backward",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 ERR_STATIC_SCRATCH = -7
@@ -73,6 +74,8 @@ def lib() -> ctypes.CDLL:
     L.mtpc_backward_workspace_bytes.argtypes = [ctypes.POINTER(MtpcConfig), i32, ctypes.POINTER(sz)]
     L.mtpc_window_logprob_backward.argtypes = [vp, vp, vp, i32, vp, vp, sz, vp, vp, vp, vp, vp, vp]
     L.mtpc_window_loss_backward.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp, sz, vp, vp, vp, vp, vp, vp, vp]
+    L.mtpc_lowrank_compose.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+    L.mtpc_lowrank_backward.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     L.mtpc_status_string.argtypes = [ctypes.c_int]
     L.mtpc_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -84,6 +87,17 @@ def lib() -> ctypes.CDLL:
 
 def status_string(code: int) -> str:
     return lib().mtpc_status_string(code).decode()
+
+
+def mtpc_lowrank_compose(n, r, v, d, k, W_base_ptr, A_ptr, B_ptr, W_emit_out_ptr, stream=0) -> None:
+    """U[i, j] = W_base[i] + A[i, j] B[i, j] (App. G); device pointers, see include/mtpc.h."""
+    _check(lib().mtpc_lowrank_compose(n, r, v, d, k, W_base_ptr, A_ptr, B_ptr, W_emit_out_ptr, stream), "mtpc_lowrank_compose")
+
+
+def mtpc_lowrank_backward(n, r, v, d, k, A_ptr, B_ptr, dW_emit_ptr, dW_base_ptr, dA_ptr, dB_ptr, stream=0) -> None:
+    """Gradient of the composed unembeddings carried back to W_base, A, B; device pointers, see include/mtpc.h."""
+    _check(lib().mtpc_lowrank_backward(n, r, v, d, k, A_ptr, B_ptr, dW_emit_ptr, dW_base_ptr, dA_ptr, dB_ptr, stream),
+           "mtpc_lowrank_backward")
 
 
 def _check(code: int, what: str) -> None:

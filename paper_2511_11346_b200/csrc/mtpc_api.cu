@@ -3,6 +3,7 @@
 // or library fallback.
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <initializer_list>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
@@ -14,6 +15,7 @@
 #include "mtpc_circuit.cuh"
 #include "mtpc_decode.cuh"
 #include "mtpc_gemm.cuh"
+#include "mtpc_lowrank.cuh"
 
 namespace {
 
@@ -1115,6 +1117,58 @@ static int ensure_copy_pipeline(mtpc_head* head, int chunks) {
     head->copy_event_count = chunks + 1;
   }
   return MTPC_OK;
+}
+
+static bool lowrank_vector_ok(int d, std::initializer_list<const void*> ptrs) {
+  if (d % 4) return false;
+  for (const void* p : ptrs)
+    if (reinterpret_cast<uintptr_t>(p) % 16) return false;
+  return true;
+}
+
+int mtpc_lowrank_compose(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k, const void* W_base, const void* A,
+                         const void* B, void* W_emit_out, void* stream) {
+  if (!W_base || !A || !B || !W_emit_out) return MTPC_ERR_NULL;
+  if (n < 1 || r < 1 || v < 1 || d < 1 || k < 1 || static_cast<int64_t>(n) * r > 65535 ||
+      (v + kComposeRows - 1) / kComposeRows > 65535)
+    return MTPC_ERR_SHAPE;
+  if (k > kLowRankMaxK) return MTPC_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const auto* w = static_cast<const __nv_bfloat16*>(W_base);
+  const auto* a = static_cast<const __nv_bfloat16*>(A);
+  const auto* b = static_cast<const __nv_bfloat16*>(B);
+  auto* u = static_cast<__nv_bfloat16*>(W_emit_out);
+  const int rows = (v + kComposeRows - 1) / kComposeRows;
+  if (lowrank_vector_ok(d, {W_base, B, W_emit_out})) {
+    lowrank_compose_kernel<4><<<dim3((d + 4 * kLowRankThreads - 1) / (4 * kLowRankThreads), rows, n * r), kLowRankThreads, 0, st>>>(
+        w, a, b, u, r, v, d, k);
+  } else {
+    lowrank_compose_kernel<1><<<dim3((d + kLowRankThreads - 1) / kLowRankThreads, rows, n * r), kLowRankThreads, 0, st>>>(
+        w, a, b, u, r, v, d, k);
+  }
+  return check_launch();
+}
+
+int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k, const void* A, const void* B,
+                          const float* dW_emit, float* dW_base, float* dA, float* dB, void* stream) {
+  if (!A || !B || !dW_emit || !dW_base || !dA || !dB) return MTPC_ERR_NULL;
+  if (n < 1 || r < 1 || v < 1 || d < 1 || k < 1 || v > 65535 || static_cast<int64_t>(n) * r > 65535) return MTPC_ERR_SHAPE;
+  if (k > kLowRankMaxK) return MTPC_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const auto* a = static_cast<const __nv_bfloat16*>(A);
+  const auto* b = static_cast<const __nv_bfloat16*>(B);
+  const int units = n * r, kchunks = (k + kRankChunk - 1) / kRankChunk;
+  auto blocks = [&](int cv) { return (d + cv * kLowRankThreads - 1) / (cv * kLowRankThreads); };
+  if (lowrank_vector_ok(d, {B, dW_emit, dW_base, dB})) {
+    lowrank_dw_kernel<4><<<dim3(blocks(4), v, n), kLowRankThreads, 0, st>>>(dW_emit, dW_base, r, v, d);
+    lowrank_da_kernel<4><<<dim3((v + 31) / 32, units), kLowRankThreads, 0, st>>>(dW_emit, b, dA, v, d, k);
+    lowrank_db_kernel<2><<<dim3(blocks(2), kchunks, units), kLowRankThreads, 0, st>>>(dW_emit, a, dB, v, d, k);
+  } else {
+    lowrank_dw_kernel<1><<<dim3(blocks(1), v, n), kLowRankThreads, 0, st>>>(dW_emit, dW_base, r, v, d);
+    lowrank_da_kernel<1><<<dim3((v + 31) / 32, units), kLowRankThreads, 0, st>>>(dW_emit, b, dA, v, d, k);
+    lowrank_db_kernel<1><<<dim3(blocks(1), kchunks, units), kLowRankThreads, 0, st>>>(dW_emit, a, dB, v, d, k);
+  }
+  return check_launch();
 }
 
 int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int32_t* targets_host, int32_t T,

@@ -206,6 +206,17 @@ def make_workload(name: str, shape: HeadShape, T: int, seed: int, *, target_kind
     return wl
 
 
+def lowrank_parameters(n: int, r: int, v: int, d: int, k: int, seed: int, *, weight_std: float = 0.02,
+                       adaptor_std: float = 0.05, zero_B: bool = False):
+    """Seeded parameters of the shared-unembedding parametrisation (App. G): W_base [n, v, d], A [n, r, v, k],
+    B [n, r, k, d] as fp32 arrays of bf16-representable values. zero_B gives the initialisation App. G proposes
+    (every adaptor starts at zero)."""
+    W_base = bf16_round(_normal(seed, 11, (n, v, d), weight_std))
+    A = bf16_round(_normal(seed, 12, (n, r, v, k), adaptor_std))
+    B = np.zeros((n, r, k, d), dtype=np.float32) if zero_B else bf16_round(_normal(seed, 13, (n, r, k, d), adaptor_std))
+    return W_base, A, B
+
+
 DECODE_CELLS = [(fam, n, P) for fam in (CP, HMM) for n in (8, 16) for P in (1, 8, 64)]
 
 

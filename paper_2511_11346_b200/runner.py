@@ -20,6 +20,29 @@ def to_host_bf16(x_q: np.ndarray, pinned: bool = True):
     return t.pin_memory() if pinned else t
 
 
+def lowrank_compose(W_base, lora_A, lora_B):
+    """Device bf16 tensors W_base [n, v, d], lora_A [n, r, v, k], lora_B [n, r, k, d] -> composed W_emit [n, r, v, d] (bf16)."""
+    import torch
+    n, r, v, k = lora_A.shape
+    d = lora_B.shape[-1]
+    out = torch.empty((n, r, v, d), dtype=torch.bfloat16, device=lora_A.device)
+    B.mtpc_lowrank_compose(n, r, v, d, k, W_base.data_ptr(), lora_A.data_ptr(), lora_B.data_ptr(), out.data_ptr(),
+                           torch.cuda.current_stream().cuda_stream)
+    return out
+
+
+def lowrank_backward(lora_A, lora_B, dW_emit):
+    """Device tensors lora_A, lora_B (bf16) and dW_emit [n, r, v, d] (fp32) -> (dW_base, dA, dB) as fp32 device tensors."""
+    import torch
+    n, r, v, k = lora_A.shape
+    d = lora_B.shape[-1]
+    f32 = dict(dtype=torch.float32, device=lora_A.device)
+    dW, dA, dB = torch.empty((n, v, d), **f32), torch.empty((n, r, v, k), **f32), torch.empty((n, r, k, d), **f32)
+    B.mtpc_lowrank_backward(n, r, v, d, k, lora_A.data_ptr(), lora_B.data_ptr(), dW_emit.data_ptr(), dW.data_ptr(),
+                            dA.data_ptr(), dB.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    return dW, dA, dB
+
+
 class DeviceHead:
     """Weights of a workload resident in HBM plus a head created on them."""
 

@@ -74,6 +74,12 @@ def test_null_pointers_and_status_strings():
     assert lib.mtpc_window_logprob(None, None, None, 0, None, None) == -1
     assert lib.mtpc_draft_sample(None, None, 0, 1, None, None, None, None) == -1
     assert lib.mtpc_destroy(None) == -1
+    assert lib.mtpc_lowrank_compose(1, 1, 16, 64, 2, None, None, None, None, None) == -1
+    assert lib.mtpc_lowrank_backward(1, 1, 16, 64, 2, None, None, None, None, None, None, None) == -1
+    fake = ctypes.c_void_p(256)           # never dereferenced: the argument checks come first
+    assert lib.mtpc_lowrank_compose(1, 1, 16, 64, 0, fake, fake, fake, fake, None) == -2
+    assert lib.mtpc_lowrank_compose(1, 1, 16, 64, 65, fake, fake, fake, fake, None) == -3
+    assert lib.mtpc_lowrank_backward(1, 1, 2048, 64, 65, fake, fake, fake, fake, fake, fake, None) == -3
     seen = {B.status_string(c) for c in range(0, -8, -1)}
     assert len(seen) == 8 and "ok" in seen
 

@@ -1,0 +1,108 @@
+"""GPU parity of the shared-unembedding parametrisation (App. G: U_ij = W_i + A_ij B_ij): composition and the
+gradient carried back to W, A, B, from the CUDA path (C ABI) against the fp64 oracle on the same seeded inputs.
+
+Bar. The composed tensor is stored in bf16: the device rounds an fp32 sum whose own error is a few 2^-24 relative,
+so it must equal the oracle's value within one bf16 spacing of it (2^-8 relative), and must be the exact bf16 rounding
+of the fp64 value on all but a small fraction of the entries (those that sit at a rounding boundary). The gradients
+are fp32 sums of at most max(v, d, r) products: 1e-5 of the tensor's largest magnitude."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mtpc_oracle as O
+from oracle import mtpc_oracle_grad as OG
+from paper_2511_11346_b200 import binding as B
+from paper_2511_11346_b200 import inputs as I
+from paper_2511_11346_b200.runner import DeviceHead, lowrank_backward, lowrank_compose, to_device_bf16
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [
+    # n, r, v, d, k
+    (1, 1, 16, 64, 1),
+    (2, 3, 48, 100, 3),          # d not a multiple of the CTA width, odd k
+    (3, 4, 320, 300, 8),
+    (2, 2, 272, 520, 16),
+    (1, 5, 33, 257, 9),          # ragged everywhere
+    (2, 2, 64, 256, 64),         # the largest rank
+]
+
+
+def _device(x):
+    return to_device_bf16(np.ascontiguousarray(x))
+
+
+@pytest.mark.parametrize("n,r,v,d,k", SHAPES)
+def test_compose_matches_the_definition(n, r, v, d, k):
+    W, A, Bm = I.lowrank_parameters(n, r, v, d, k, seed=900 + n + r + v + d + k)
+    got = lowrank_compose(_device(W), _device(A), _device(Bm)).float().cpu().numpy().astype(np.float64)
+    ref = O.lowrank_unembedding(W, A, Bm)
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-30)
+    exact = I.bf16_round(ref.astype(np.float32)).astype(np.float64)      # fp64 -> fp32 -> bf16, the value but for double rounding
+    assert np.mean(got != exact) < 1e-3
+
+
+def test_zero_adaptor_reproduces_the_shared_matrix_bit_for_bit():
+    n, r, v, d, k = 2, 3, 48, 128, 4
+    W, A, Bm = I.lowrank_parameters(n, r, v, d, k, seed=77, zero_B=True)
+    got = lowrank_compose(_device(W), _device(A), _device(Bm)).float().cpu().numpy()
+    for j in range(r):
+        np.testing.assert_array_equal(got[:, j], W)
+
+
+@pytest.mark.parametrize("n,r,v,d,k", SHAPES)
+def test_backward_matches_the_gradient_oracle(n, r, v, d, k):
+    W, A, Bm = I.lowrank_parameters(n, r, v, d, k, seed=300 + n + r + v + d + k)
+    dU = np.random.default_rng(k + d).normal(size=(n, r, v, d)).astype(np.float32)
+    dW, dA, dB = lowrank_backward(_device(A), _device(Bm), torch.from_numpy(dU).cuda())
+    torch.cuda.synchronize()
+    ref = OG.lowrank_grad(W, A, Bm, dU)
+    for name, got, want in (("dW_base", dW, ref["dW_base"]), ("dA", dA, ref["dA"]), ("dB", dB, ref["dB"])):
+        got = got.cpu().numpy().astype(np.float64)
+        assert got.shape == want.shape
+        assert np.abs(got - want).max() <= 1e-5 * np.abs(want).max(), name
+
+
+@pytest.mark.parametrize("family", [I.CP, I.BTREE])
+def test_head_on_composed_unembeddings_and_the_gradient_chain(family):
+    """Compose on the device, run the head and its backward on the composed tensor, carry dW_emit back to W, A, B;
+    the oracle does the same chain in fp64 on the bf16 rounding of its own composed tensor."""
+    n, r, v, d, k, T = 4, 4, 64, 128, 4, 150
+    shape = I.HeadShape(family, n, r, v, d)
+    wl = I.make_workload("lowrank_chain", shape, T, seed=4242, weight_std=0.25)
+    W, A, Bm = I.lowrank_parameters(n, r, v, d, k, seed=4243, weight_std=0.25, adaptor_std=0.2)
+    U_q = I.bf16_round(O.lowrank_unembedding(W, A, Bm).astype(np.float32))
+    dA_, dB_ = _device(A), _device(Bm)
+    U_dev = lowrank_compose(_device(W), dA_, dB_)
+    assert np.mean(U_dev.float().cpu().numpy() != U_q) < 1e-3
+    wl.W_emit_q = U_q
+    head = DeviceHead(wl)
+    head.head.mtpc_destroy()
+    head.W_emit = U_dev                                                   # the head under test runs on the device's own composition
+    s = wl.shape
+    head.head = B.MtpcHead(s.family, s.n, s.r, s.v, s.d, s.io_dtype, T, 1, head.W_emit, head.W_sum, head.T_static)
+    weight = np.random.default_rng(5).normal(size=T).astype(np.float32)
+    out = head.window_logprob_backward(torch.from_numpy(weight).cuda())
+    assert head.head.mtpc_get_status() == 0
+    ref = OG.window_logprob_grad(family, wl.hidden_q, U_q, wl.W_sum_q, None, wl.targets, weight)
+    assert np.abs(out["logprob"].cpu().numpy() - ref["logprob"]).max() <= 2e-3
+    dW, dA, dB = lowrank_backward(dA_, dB_, out["dW_emit"])
+    chain = OG.lowrank_grad(W, A, Bm, ref["dW_emit"])
+    for name, got, want in (("dW_base", dW, chain["dW_base"]), ("dA", dA, chain["dA"]), ("dB", dB, chain["dB"])):
+        got = got.cpu().numpy().astype(np.float64)
+        scale = np.abs(want).max()
+        assert np.abs(got - want).max() <= 1e-2 * scale, name            # the bar of the head's own backward pass
+        assert np.linalg.norm(got - want) <= 5e-3 * np.linalg.norm(want), name
+
+
+def test_argument_checks():
+    n, r, v, d = 1, 1, 16, 64
+    W, A, Bm = I.lowrank_parameters(n, r, v, d, 2, seed=1)
+    a, b, w = _device(A), _device(Bm), _device(W)
+    out = torch.empty((n, r, v, d), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.MtpcError) as e:
+        B.mtpc_lowrank_compose(n, r, v, d, 65, w.data_ptr(), a.data_ptr(), b.data_ptr(), out.data_ptr())
+    assert e.value.code == -3      # MTPC_ERR_UNSUPPORTED: rank above 64
+    with pytest.raises(B.MtpcError) as e:
+        B.mtpc_lowrank_compose(n, r, v, d, 0, w.data_ptr(), a.data_ptr(), b.data_ptr(), out.data_ptr())
+    assert e.value.code == -2      # MTPC_ERR_SHAPE

@@ -206,6 +206,22 @@ def loss_gap(orc):
     return float(np.abs(slot - 1.5 * ln(2)).max() + abs(total - 1.5 * ln(2) * 1.8))
 
 
+def lowrank_gap(orc):
+    """Hand example and the scalar formula of App. G's U_ij = W_i + A_ij B_ij, with distinct slots and components."""
+    rng = np.random.default_rng(11)
+    n, r, v, d, k = 2, 3, 4, 5, 2
+    W, A, B = rng.normal(size=(n, v, d)), rng.normal(size=(n, r, v, k)), rng.normal(size=(n, r, k, d))
+    U = orc.lowrank_unembedding(W, A, B)
+    gap = 0.0
+    for i in range(n):
+        for j in range(r):
+            for b in range(v):
+                for c in range(d):
+                    want = W[i, b, c] + sum(A[i, j, b, q] * B[i, j, q, c] for q in range(k))
+                    gap = max(gap, abs(U[i, j, b, c] - want))
+    return gap
+
+
 MUTANTS = [
     # (what is planted, old text, new text, pin that must notice)
     ("mixture weights dropped from Eq. CP", "logsumexp(logw + g.sum(axis=1), axis=-1)", "logsumexp(g.sum(axis=1), axis=-1)", cp_gap),
@@ -265,6 +281,11 @@ MUTANTS = [
     ("discount starts at gamma instead of one", "sum(gamma ** j * slot[j] for j in range(n))",
      "sum(gamma ** (j + 1) * slot[j] for j in range(n))", loss_gap),
     ("loss not averaged over the sequences", "slot[j] = -acc / N", "slot[j] = -acc", loss_gap),
+    ("adaptor added to the base matrix of the wrong slot", "U[i, j] = W_base[i] + A[i, j] @ B[i, j]",
+     "U[i, j] = W_base[0] + A[i, j] @ B[i, j]", lowrank_gap),
+    ("adaptor shared by the components", "U[i, j] = W_base[i] + A[i, j] @ B[i, j]", "U[i, j] = W_base[i] + A[i, 0] @ B[i, 0]",
+     lowrank_gap),
+    ("adaptor dropped", "U[i, j] = W_base[i] + A[i, j] @ B[i, j]", "U[i, j] = W_base[i]", lowrank_gap),
 ]
 
 
