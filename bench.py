@@ -296,7 +296,8 @@ def measure_lowrank(torch, wl, dW_emit, steps: int, peaks, k: int = 16):
     return {"rank": k, "compose_ms": ms_c, "compose_algorithmic_bytes": bytes_c,
             "compose_frac_of_hbm": bytes_c / (ms_c * 1e-3) / 1e9 / hbm, "backward_ms": ms_b, "backward_kernels": 3,
             "backward_algorithmic_bytes": bytes_b, "backward_frac_of_hbm": bytes_b / (ms_b * 1e-3) / 1e9 / hbm,
-            "note": "the three gradient kernels each stream dW_emit once: at most a third of the one-pass bound"}
+            "note": "CUDA-core kernels: k multiply-adds per element keep the fp32 pipes, not HBM, busiest; the three "
+                    "gradient kernels each stream dW_emit once"}
 
 
 def measure_eq6_step(torch, dh, wl, hidden, targets, grads, steps: int):

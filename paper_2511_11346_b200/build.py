@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libmtpc.so")
 SOURCES = ["mtpc_api.cu"]
-HEADERS = ["mtpc_ptx.cuh", "mtpc_gemm.cuh", "mtpc_circuit.cuh", "mtpc_decode.cuh", os.path.join("..", "..", "include", "mtpc.h")]
+HEADERS = sorted(f for f in os.listdir(CSRC) if f.endswith(".cuh")) + [os.path.join("..", "..", "include", "mtpc.h")]
 
 
 def _nvcc() -> str:

@@ -1130,7 +1130,7 @@ int mtpc_lowrank_compose(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k, 
                          const void* B, void* W_emit_out, void* stream) {
   if (!W_base || !A || !B || !W_emit_out) return MTPC_ERR_NULL;
   if (n < 1 || r < 1 || v < 1 || d < 1 || k < 1 || static_cast<int64_t>(n) * r > 65535 ||
-      (v + kComposeRows - 1) / kComposeRows > 65535)
+      (v + kComposeCtaRows - 1) / kComposeCtaRows > 65535)
     return MTPC_ERR_SHAPE;
   if (k > kLowRankMaxK) return MTPC_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1138,12 +1138,17 @@ int mtpc_lowrank_compose(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k, 
   const auto* a = static_cast<const __nv_bfloat16*>(A);
   const auto* b = static_cast<const __nv_bfloat16*>(B);
   auto* u = static_cast<__nv_bfloat16*>(W_emit_out);
-  const int rows = (v + kComposeRows - 1) / kComposeRows;
+  const int rows = (v + kComposeCtaRows - 1) / kComposeCtaRows;
   if (lowrank_vector_ok(d, {W_base, B, W_emit_out})) {
-    lowrank_compose_kernel<4><<<dim3((d + 4 * kLowRankThreads - 1) / (4 * kLowRankThreads), rows, n * r), kLowRankThreads, 0, st>>>(
-        w, a, b, u, r, v, d, k);
+    const size_t smem = compose_smem_bytes(k, 4);
+    if (cudaFuncSetAttribute(lowrank_compose_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) !=
+        cudaSuccess)
+      return MTPC_ERR_CUDA;
+    lowrank_compose_kernel<4><<<dim3((d + 4 * kLowRankThreads - 1) / (4 * kLowRankThreads), rows, n * r), kLowRankThreads, smem,
+                                st>>>(w, a, b, u, r, v, d, k);
   } else {
-    lowrank_compose_kernel<1><<<dim3((d + kLowRankThreads - 1) / kLowRankThreads, rows, n * r), kLowRankThreads, 0, st>>>(
+    const size_t smem = compose_smem_bytes(k, 1);
+    lowrank_compose_kernel<1><<<dim3((d + kLowRankThreads - 1) / kLowRankThreads, rows, n * r), kLowRankThreads, smem, st>>>(
         w, a, b, u, r, v, d, k);
   }
   return check_launch();
@@ -1162,7 +1167,7 @@ int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k,
   if (lowrank_vector_ok(d, {B, dW_emit, dW_base, dB})) {
     lowrank_dw_kernel<4><<<dim3(blocks(4), v, n), kLowRankThreads, 0, st>>>(dW_emit, dW_base, r, v, d);
     lowrank_da_kernel<4><<<dim3((v + 31) / 32, units), kLowRankThreads, 0, st>>>(dW_emit, b, dA, v, d, k);
-    lowrank_db_kernel<2><<<dim3(blocks(2), kchunks, units), kLowRankThreads, 0, st>>>(dW_emit, a, dB, v, d, k);
+    lowrank_db_kernel<4><<<dim3(blocks(4), kchunks, units), kLowRankThreads, 0, st>>>(dW_emit, a, dB, v, d, k);
   } else {
     lowrank_dw_kernel<1><<<dim3(blocks(1), v, n), kLowRankThreads, 0, st>>>(dW_emit, dW_base, r, v, d);
     lowrank_da_kernel<1><<<dim3((v + 31) / 32, units), kLowRankThreads, 0, st>>>(dW_emit, b, dA, v, d, k);

@@ -15,10 +15,15 @@ namespace mtpc {
 
 constexpr int kLowRankThreads = 256;
 constexpr int kLowRankMaxK = 64;
-constexpr int kComposeRows = 8;      // rows of U per thread in the composition
+constexpr int kComposeRows = 8;      // rows of U in a thread's register tile in the composition
+constexpr int kComposeCtaRows = 32;  // rows of U a CTA of the composition walks
 constexpr int kRankChunk = 16;       // ranks per register tile in the gradient kernels
 constexpr int kDaCols = 512;         // columns of B staged per step of lowrank_da_kernel
 constexpr int kDbRows = 256;         // rows of A staged per step of lowrank_db_kernel
+
+inline size_t compose_smem_bytes(int k, int cv) {
+  return static_cast<size_t>(k) * (kLowRankThreads * cv * 2 + kComposeCtaRows * 4);
+}
 
 template <int CV>
 __device__ __forceinline__ void load_bf16(const __nv_bfloat16* p, float (&out)[CV]) {
@@ -60,60 +65,107 @@ __device__ __forceinline__ void store_f32(float* p, const float (&x)[CV]) {
 }
 
 // U[i, j, b, c] = bf16( W[i, b, c] + sum_q A[i, j, b, q] B[i, j, q, c] ), fp32 accumulation in the order q = 0..k-1.
-// grid = (ceil(d / (256 CV)), ceil(v / 8), n r): a thread owns 8 rows x CV columns; the 8 rows of A sit in shared memory.
+// grid = (ceil(d / (256 CV)), ceil(v / 32), n r). A thread owns CV columns: it fetches its k values of B per column
+// once (all loads in flight together, parked in its own slots of shared memory), then walks 4 blocks of 8 rows, the
+// next block's rows of W prefetched while the current one is computed. Dynamic shared memory:
+// compose_smem_bytes(k, CV).
 template <int CV>
 __global__ void __launch_bounds__(kLowRankThreads) lowrank_compose_kernel(const __nv_bfloat16* __restrict__ W,
                                                                          const __nv_bfloat16* __restrict__ A,
                                                                          const __nv_bfloat16* __restrict__ B,
                                                                          __nv_bfloat16* __restrict__ U, int r, int v,
                                                                          int d, int k) {
-  __shared__ __align__(16) float a_s[kLowRankMaxK][kComposeRows];
+  extern __shared__ __align__(16) unsigned char lowrank_smem[];
+  __nv_bfloat16* b_s = reinterpret_cast<__nv_bfloat16*>(lowrank_smem);                       // [k][256 CV]
+  float* a_s = reinterpret_cast<float*>(lowrank_smem + static_cast<size_t>(k) * kLowRankThreads * CV * 2);  // [k][32]
   const int unit = blockIdx.z, i = unit / r;
-  const int b0 = blockIdx.y * kComposeRows;
+  const int row0 = blockIdx.y * kComposeCtaRows;
   const int c = (blockIdx.x * kLowRankThreads + threadIdx.x) * CV;
-  for (int e = threadIdx.x; e < k * kComposeRows; e += kLowRankThreads) {
-    const int q = e / kComposeRows, rr = e % kComposeRows;
-    a_s[q][rr] = b0 + rr < v ? __bfloat162float(A[(static_cast<size_t>(unit) * v + b0 + rr) * k + q]) : 0.f;
-  }
-  __syncthreads();
-  if (c >= d) return;
-  float acc[kComposeRows][CV];
+  const bool in = c < d;
+  {
+    const __nv_bfloat16* Bu = B + static_cast<size_t>(unit) * k * d + c;
+    __nv_bfloat16* mine = b_s + threadIdx.x * CV;
+#pragma unroll 8
+    for (int q = 0; q < k; ++q, Bu += d, mine += kLowRankThreads * CV) {
+      if constexpr (CV == 4) {
+        *reinterpret_cast<uint2*>(mine) = in ? *reinterpret_cast<const uint2*>(Bu) : make_uint2(0u, 0u);
+      } else {
 #pragma unroll
-  for (int rr = 0; rr < kComposeRows; ++rr) {
-    if (b0 + rr < v) {
-      load_bf16<CV>(W + (static_cast<size_t>(i) * v + b0 + rr) * d + c, acc[rr]);
-    } else {
-#pragma unroll
-      for (int t = 0; t < CV; ++t) acc[rr][t] = 0.f;
+        for (int t = 0; t < CV; ++t) mine[t] = in ? Bu[t] : __float2bfloat16_rn(0.f);
+      }
     }
   }
-  const __nv_bfloat16* Bu = B + static_cast<size_t>(unit) * k * d + c;
-#pragma unroll 4
-  for (int q = 0; q < k; ++q) {
-    float bv[CV];
-    load_bf16<CV>(Bu + static_cast<size_t>(q) * d, bv);
-    const float4 a0 = *reinterpret_cast<const float4*>(&a_s[q][0]);
-    const float4 a1 = *reinterpret_cast<const float4*>(&a_s[q][4]);
-    const float av[kComposeRows] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-#pragma unroll
-    for (int rr = 0; rr < kComposeRows; ++rr)
-#pragma unroll
-      for (int t = 0; t < CV; ++t) acc[rr][t] = fmaf(av[rr], bv[t], acc[rr][t]);
+  for (int e = threadIdx.x; e < k * kComposeCtaRows; e += kLowRankThreads) {
+    const int q = e / kComposeCtaRows, rr = e % kComposeCtaRows;
+    a_s[e] = row0 + rr < v ? __bfloat162float(A[(static_cast<size_t>(unit) * v + row0 + rr) * k + q]) : 0.f;
   }
+  __syncthreads();
+  if (!in) return;
+  const __nv_bfloat16* Wi = W + static_cast<size_t>(i) * v * d + c;
+  struct alignas(2 * CV) Raw { __nv_bfloat16 e[CV]; };               // CV bf16 values as they lie in memory
+  auto load_w = [&](int b0, Raw (&w)[kComposeRows]) {
 #pragma unroll
-  for (int rr = 0; rr < kComposeRows; ++rr) {
-    if (b0 + rr >= v) break;
-    __nv_bfloat16* dst = U + (static_cast<size_t>(unit) * v + b0 + rr) * d + c;
-    if constexpr (CV == 4) {
-      const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[rr][0], acc[rr][1]);
-      const __nv_bfloat162 hi = __floats2bfloat162_rn(acc[rr][2], acc[rr][3]);
-      uint2 raw;
-      raw.x = *reinterpret_cast<const uint32_t*>(&lo);
-      raw.y = *reinterpret_cast<const uint32_t*>(&hi);
-      *reinterpret_cast<uint2*>(dst) = raw;
-    } else {
+    for (int rr = 0; rr < kComposeRows; ++rr) {
+      if (b0 + rr < v) {
+        w[rr] = *reinterpret_cast<const Raw*>(Wi + static_cast<size_t>(b0 + rr) * d);
+      } else {
 #pragma unroll
-      for (int t = 0; t < CV; ++t) dst[t] = __float2bfloat16_rn(acc[rr][t]);
+        for (int t = 0; t < CV; ++t) w[rr].e[t] = __float2bfloat16_rn(0.f);
+      }
+    }
+  };
+  Raw wn[kComposeRows];
+  load_w(row0, wn);
+  for (int rb = 0; rb < kComposeCtaRows / kComposeRows; ++rb) {
+    const int b0 = row0 + rb * kComposeRows;
+    if (b0 >= v) break;
+    // Accumulators as pairs of adjacent rows: one packed fp32 multiply-add (two independent round-to-nearest FMAs)
+    // takes the pair of A values as they lie in shared memory and the B value twice.
+    float2 acc[kComposeRows / 2][CV];
+#pragma unroll
+    for (int rr = 0; rr < kComposeRows; ++rr) {
+      float w[CV];
+      load_bf16<CV>(wn[rr].e, w);
+#pragma unroll
+      for (int t = 0; t < CV; ++t) (rr & 1 ? acc[rr / 2][t].y : acc[rr / 2][t].x) = w[t];
+    }
+    load_w(b0 + kComposeRows, wn);                                  // beyond the last row: zeros, never stored
+    const __nv_bfloat16* mine = b_s + threadIdx.x * CV;
+    const float* arow = a_s + rb * kComposeRows;
+#pragma unroll 4
+    for (int q = 0; q < k; ++q, mine += kLowRankThreads * CV, arow += kComposeCtaRows) {
+      float bv[CV];
+      load_bf16<CV>(mine, bv);
+      float2 b2[CV];
+#pragma unroll
+      for (int t = 0; t < CV; ++t) b2[t] = make_float2(bv[t], bv[t]);
+#pragma unroll
+      for (int r4 = 0; r4 < kComposeRows; r4 += 4) {
+        const float4 a = *reinterpret_cast<const float4*>(arow + r4);
+        const float2 a01 = make_float2(a.x, a.y), a23 = make_float2(a.z, a.w);
+#pragma unroll
+        for (int t = 0; t < CV; ++t) {
+          acc[r4 / 2][t] = __ffma2_rn(a01, b2[t], acc[r4 / 2][t]);
+          acc[r4 / 2 + 1][t] = __ffma2_rn(a23, b2[t], acc[r4 / 2 + 1][t]);
+        }
+      }
+    }
+#pragma unroll
+    for (int rr = 0; rr < kComposeRows; ++rr) {
+      if (b0 + rr >= v) break;
+      float o[CV];
+#pragma unroll
+      for (int t = 0; t < CV; ++t) o[t] = rr & 1 ? acc[rr / 2][t].y : acc[rr / 2][t].x;
+      __nv_bfloat16* dst = U + (static_cast<size_t>(unit) * v + b0 + rr) * d + c;
+      if constexpr (CV == 4) {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(o[0], o[1]);
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(o[2], o[3]);
+        *reinterpret_cast<uint2*>(dst) =
+            make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+      } else {
+#pragma unroll
+        for (int t = 0; t < CV; ++t) dst[t] = __float2bfloat16_rn(o[t]);
+      }
     }
   }
 }
@@ -140,60 +192,69 @@ __global__ void __launch_bounds__(kLowRankThreads) lowrank_dw_kernel(const float
 
 // dA[i, j, b, q] = sum_c dU[i, j, b, c] B[i, j, q, c].  grid = (ceil(v / 32), n r); a warp owns 4 rows and every column,
 // a lane CV adjacent columns of each 32 CV-wide stripe; 16 ranks at a time, their rows of B staged 512 columns at a
-// time in shared memory (bf16). The lanes' partial sums meet in a butterfly at the end of each block of ranks.
+// time in shared memory (as fp32). The lanes' partial sums meet in a butterfly at the end of each block of ranks.
 template <int CV>
-__global__ void __launch_bounds__(kLowRankThreads) lowrank_da_kernel(const float* __restrict__ dU,
-                                                                    const __nv_bfloat16* __restrict__ B,
-                                                                    float* __restrict__ dA, int v, int d, int k) {
-  __shared__ __align__(16) __nv_bfloat16 b_s[kRankChunk][kDaCols];
+__global__ void __launch_bounds__(kLowRankThreads, 2) lowrank_da_kernel(const float* __restrict__ dU,
+                                                                       const __nv_bfloat16* __restrict__ B,
+                                                                       float* __restrict__ dA, int v, int d, int k) {
+  __shared__ __align__(16) float b_s[kRankChunk][kDaCols];          // fp32: converted once per stripe, not once per use
+  constexpr int kIters = kDaCols / (32 * CV);                     // column groups of a lane per stripe
   const int unit = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b0 = blockIdx.x * 32 + warp * 4;
+  const float* rows = dU + (static_cast<size_t>(unit) * v + b0) * d;
+  auto load_x = [&](int col, float (&x)[4][CV]) {                  // zeros beyond the last row or column
+#pragma unroll
+    for (int rr = 0; rr < 4; ++rr) {
+      if (b0 + rr < v && col < d) {
+        load_f32<CV>(rows + static_cast<size_t>(rr) * d + col, x[rr]);
+      } else {
+#pragma unroll
+        for (int t = 0; t < CV; ++t) x[rr][t] = 0.f;
+      }
+    }
+  };
   for (int q0 = 0; q0 < k; q0 += kRankChunk) {
     float acc[4][kRankChunk];
 #pragma unroll
     for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
       for (int q = 0; q < kRankChunk; ++q) acc[rr][q] = 0.f;
+    float x[4][CV];
+    load_x(lane * CV, x);
     for (int c0 = 0; c0 < d; c0 += kDaCols) {
       __syncthreads();                                            // the previous stripe has been consumed
       for (int e = threadIdx.x * CV; e < kRankChunk * kDaCols; e += kLowRankThreads * CV) {
         const int q = e / kDaCols, cc = e % kDaCols;
         const bool in = q0 + q < k && c0 + cc < d;               // d is a multiple of CV: the CV columns are in or out together
+        float bv[CV];
         if (in) {
-          const __nv_bfloat16* src = B + (static_cast<size_t>(unit) * k + q0 + q) * d + c0 + cc;
-          if constexpr (CV == 4) {
-            *reinterpret_cast<uint2*>(&b_s[q][cc]) = *reinterpret_cast<const uint2*>(src);
-          } else {
-#pragma unroll
-            for (int t = 0; t < CV; ++t) b_s[q][cc + t] = src[t];
-          }
+          load_bf16<CV>(B + (static_cast<size_t>(unit) * k + q0 + q) * d + c0 + cc, bv);
         } else {
 #pragma unroll
-          for (int t = 0; t < CV; ++t) b_s[q][cc + t] = __float2bfloat16_rn(0.f);
+          for (int t = 0; t < CV; ++t) bv[t] = 0.f;
         }
+        store_f32<CV>(&b_s[q][cc], bv);
       }
       __syncthreads();
-      for (int cc = lane * CV; cc < kDaCols && c0 + cc < d; cc += 32 * CV) {
-        float x[4][CV];
 #pragma unroll
-        for (int rr = 0; rr < 4; ++rr) {
-          if (b0 + rr < v) {
-            load_f32<CV>(dU + (static_cast<size_t>(unit) * v + b0 + rr) * d + c0 + cc, x[rr]);
-          } else {
-#pragma unroll
-            for (int t = 0; t < CV; ++t) x[rr][t] = 0.f;
-          }
-        }
+      for (int it = 0; it < kIters; ++it) {
+        const int cc = (it * 32 + lane) * CV;
+        float xn[4][CV];                                          // the lane's next columns (of this stripe or the next one)
+        load_x(c0 + cc + 32 * CV, xn);
 #pragma unroll
         for (int q = 0; q < kRankChunk; ++q) {
           float bv[CV];
-          load_bf16<CV>(&b_s[q][cc], bv);
+          load_f32<CV>(&b_s[q][cc], bv);
 #pragma unroll
           for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
             for (int t = 0; t < CV; ++t) acc[rr][q] = fmaf(x[rr][t], bv[t], acc[rr][q]);
         }
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr)
+#pragma unroll
+          for (int t = 0; t < CV; ++t) x[rr][t] = xn[rr][t];
       }
     }
 #pragma unroll
@@ -211,7 +272,7 @@ __global__ void __launch_bounds__(kLowRankThreads) lowrank_da_kernel(const float
 // dB[i, j, q, c] = sum_b A[i, j, b, q] dU[i, j, b, c].  grid = (ceil(d / (256 CV)), ceil(k / 16), n r): a thread owns
 // CV columns x 16 ranks and walks the v rows in order; 256 rows of A at a time sit in shared memory (fp32).
 template <int CV>
-__global__ void __launch_bounds__(kLowRankThreads) lowrank_db_kernel(const float* __restrict__ dU,
+__global__ void __launch_bounds__(kLowRankThreads, 2) lowrank_db_kernel(const float* __restrict__ dU,
                                                                     const __nv_bfloat16* __restrict__ A,
                                                                     float* __restrict__ dB, int v, int d, int k) {
   __shared__ __align__(16) float a_s[kDbRows][kRankChunk];
