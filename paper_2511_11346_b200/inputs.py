@@ -217,6 +217,11 @@ def lowrank_parameters(n: int, r: int, v: int, d: int, k: int, seed: int, *, wei
     return W_base, A, B
 
 
+def lowrank_upstream_gradient(n: int, r: int, v: int, d: int, seed: int) -> np.ndarray:
+    """A seeded stand-in for the gradient of the composed unembeddings, [n, r, v, d] fp32."""
+    return _normal(seed, 14, (n, r, v, d), 1.0)
+
+
 DECODE_CELLS = [(fam, n, P) for fam in (CP, HMM) for n in (8, 16) for P in (1, 8, 64)]
 
 
