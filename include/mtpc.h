@@ -258,10 +258,9 @@ int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k,
  * Host-buffer variants: same results, but hidden / targets / uniforms are HOST pointers (pinned memory for
  * full copy speed) and the outputs are written to HOST buffers. The copies to and from the device go through
  * staging areas in the workspace; the call returns after the stream has been synchronised, so the outputs are
- * ready on return. mtpc_window_logprob_host uploads and processes 512, 1024, then 2048 positions at a time: the
- * uploads run on a second stream the head owns, ordered after the work already on `stream`, so that all but the
- * first, short one are hidden behind the kernels (with per-kernel timing on, every chunk is recorded as a call of
- * its own).
+ * ready on return. mtpc_window_logprob_host uploads and processes 2048 positions at a time: the uploads run on a
+ * second stream the head owns, ordered after the work already on `stream`, so that all but the first are hidden
+ * behind the kernels (with per-kernel timing on, every chunk is recorded as a call of its own).
  */
 int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int32_t* targets_host, int32_t T,
                              float* out_logprob_host, void* stream);

@@ -26,7 +26,6 @@ constexpr int kMaxPhases = 5;
 constexpr size_t kSlotSmemLimit = 160 * 1024;   // latent-draw tables of the draft slot kernel kept in shared memory up to this
 constexpr int kMaxDraftVocab = 512;     // draft sampling: the v logits of a unit live in 512 TMEM columns / 16 per lane
 constexpr int kHostChunkPositions = 2048;   // host-buffer calls upload and process this many positions at a time
-constexpr int kMaxHostChunks = 64;          // beyond that the last chunk takes the rest
 constexpr int kWorkCounterWord = 16;   // word of the 256-byte status area used as the circuit kernels' work counter
 constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA on sm_100
 // Hidden states of one rasterisation block of the projection kernel: small enough to stay L2-resident next to the
@@ -1191,23 +1190,15 @@ int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int
   int32_t* dt = at<int32_t>(head, L.off_h_targets);
   float* dout = at<float>(head, L.off_h_out);
   // The positions are uploaded in chunks on a second stream while the kernels of the chunks before run on `stream`:
-  // only the first chunk's upload is not hidden behind compute, so the first chunks are short (a quarter, then half
-  // of the regular size: the upload of each next chunk still ends before the kernels of the chunks before it do).
-  int starts[kMaxHostChunks + 1];
-  int chunks = 0;
-  for (int t0 = 0; t0 < T;) {
-    starts[chunks] = t0;
-    const int want = chunks == 0 ? kHostChunkPositions / 4 : chunks == 1 ? kHostChunkPositions / 2 : kHostChunkPositions;
-    t0 = chunks + 1 == kMaxHostChunks ? T : (T - t0 < want ? T : t0 + want);
-    ++chunks;
-  }
-  starts[chunks] = T;
+  // only the first chunk's upload is not hidden behind compute.
+  const int chunks = (T + kHostChunkPositions - 1) / kHostChunkPositions;
   if ((rc = ensure_copy_pipeline(head, chunks)) != MTPC_OK) return rc;
   cudaStream_t cs = head->copy_stream;
   bool fail = cudaEventRecord(head->copy_events[chunks], st) != cudaSuccess;     // uploads wait for earlier work on `stream`
   fail |= cudaStreamWaitEvent(cs, head->copy_events[chunks], 0) != cudaSuccess;
   for (int k = 0; k < chunks && !fail; ++k) {
-    const size_t t0 = starts[k], tc = starts[k + 1] - starts[k];
+    const size_t t0 = static_cast<size_t>(k) * kHostChunkPositions;
+    const size_t tc = (T - t0) < static_cast<size_t>(kHostChunkPositions) ? (T - t0) : kHostChunkPositions;
     fail |= cudaMemcpyAsync(dh + t0 * c.d * elt, static_cast<const uint8_t*>(hidden_host) + t0 * c.d * elt, tc * c.d * elt,
                             cudaMemcpyHostToDevice, cs) != cudaSuccess;
     fail |= cudaMemcpyAsync(dt + t0 * c.n, targets_host + t0 * c.n, tc * c.n * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess;
@@ -1215,9 +1206,10 @@ int mtpc_window_logprob_host(mtpc_head* head, const void* hidden_host, const int
   }
   if (fail) return MTPC_ERR_CUDA;
   for (int k = 0; k < chunks; ++k) {
-    const size_t t0 = starts[k];
+    const size_t t0 = static_cast<size_t>(k) * kHostChunkPositions;
+    const int tc = static_cast<int>((T - t0) < static_cast<size_t>(kHostChunkPositions) ? (T - t0) : kHostChunkPositions);
     if (cudaStreamWaitEvent(st, head->copy_events[k], 0) != cudaSuccess) return MTPC_ERR_CUDA;
-    rc = window_logprob_impl(head, dh + t0 * c.d * elt, dt + t0 * c.n, starts[k + 1] - starts[k], dout + t0, nullptr, st);
+    rc = window_logprob_impl(head, dh + t0 * c.d * elt, dt + t0 * c.n, tc, dout + t0, nullptr, st);
     if (rc != MTPC_OK) { cudaStreamSynchronize(cs); return rc; }
   }
   fail = cudaMemcpyAsync(out_logprob_host, dout, static_cast<size_t>(T) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess;

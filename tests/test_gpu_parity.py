@@ -236,8 +236,8 @@ def test_max_windows_per_position():
 
 
 def test_chunked_host_call_equals_device_call():
-    """The host-buffer entry point uploads and processes the positions in chunks (512, 1024, then 2048 each); the results
-    are those of one device-buffer call (same arithmetic per position), ragged last chunk included, twice in a row."""
+    """The host-buffer entry point uploads and processes 2048 positions at a time; the results are those of one
+    device-buffer call (same arithmetic per position), ragged last chunk included, twice in a row."""
     wl = I.make_workload("host_chunks", I.HeadShape(I.HMM, 4, 8, 320, 128), 5000, seed=91, weight_std=0.2)
     dh = DeviceHead(wl)
     dev = dh.window_logprob().cpu()
