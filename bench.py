@@ -428,7 +428,11 @@ def run_ours(args):
     # CPU baseline: the oracle as it stands on a bounded sample of the same workload
     cpu_baseline = None
     if not args.no_cpu_baseline:
-        sample = min(wl.T, args.ref_positions)
+        if args.ref_positions:
+            sample = min(wl.T, args.ref_positions)
+        else:                                                                # about 15 s of CPU work, sized by a short probe
+            probe_rate, _ = oracle_positions_per_s(wl, min(wl.T, 256))
+            sample = int(min(wl.T, max(256, (probe_rate * 15.0) // 256 * 256)))
         cpu_value, cpu_s = oracle_positions_per_s(wl, sample)
         cpu_baseline = {"value": cpu_value, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
                         "sample": f"first {sample} of {wl.T} positions, one pass, {cpu_s:.1f} s"}
@@ -514,7 +518,8 @@ def main():
                     help="1 CP (the metric's configuration), 2 HMM, 3 binary tree, 5 HMM with contextual transitions, "
                          "6 CP with the byte-level Llama shape (d=3072, 268 symbols padded to 272)")
     ap.add_argument("--ref-positions", type=int, default=None,
-                    help="positions the CPU oracle processes per step / for the cpu_baseline sample")
+                    help="positions the CPU oracle processes per step (reference arm: default 1024) or for the "
+                         "cpu_baseline sample (default: sized to about 15 s by a short probe)")
     ap.add_argument("--no-draft", action="store_true", help="skip the decode-cell draft measurement")
     ap.add_argument("--decode-cells", default="all",
                     help="draft measurement: 'all' twelve cells of the decode sweep, 'one' (CP n=8 P=64), or a single "
@@ -532,7 +537,6 @@ def main():
     else:
         args.steps = 400 if args.steps is None else args.steps
         args.warmup = max(3, 5 if args.warmup is None else args.warmup)
-        args.ref_positions = args.ref_positions or 4096
         run_ours(args)
 
 
