@@ -112,6 +112,18 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
                      void* workspace, size_t workspace_bytes, void* stream, mtpc_head** out);
 
 /*
+ * After the parameters have changed (an optimiser step between two training calls): rebinds the head to W_emit,
+ * W_sum and T_static, which may be the buffers it was created on, updated in place, or others of the same shapes.
+ * With MTPC_BF16 the kernels read W_emit / W_sum in place, so only what creation derived from the parameters is
+ * redone: the log-softmax of the static HMM transitions or the copy of the contextual transition bias, the tensor
+ * maps, and with MTPC_F32 the rounded copies of the weights. Arguments and ownership as for mtpc_create_head; the
+ * work is enqueued on `stream`, which must also order it after the calls that still use the old parameters. The
+ * logits a draft call left in the workspace are forgotten (mtpc_speculative_accept then needs a new draft).
+ * MTPC_ERR_NULL for a missing pointer (T_static is required exactly where creation requires it).
+ */
+int mtpc_update_parameters(mtpc_head* head, const void* W_emit, const void* W_sum, const float* T_static, void* stream);
+
+/*
  * Window log-likelihood (Eq. 1 evaluated through Eq. CP / Eq. HMM / Eq. BTree):
  *   out_logprob[t] = log q(x_{t,0..n-1} | h_t), natural log, for t in [0,T).
  *   hidden  dev [T, d] io_dtype, row-major.
@@ -240,8 +252,9 @@ int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t
  * base matrix per token slot shared by its r components plus a rank-k adaptor per component. The head computes on the
  * composed tensor; these two calls convert between the shared parameters and it. They need no head.
  *   W_base  device [n, v, d] bf16      A  device [n, r, v, k] bf16      B  device [n, r, k, d] bf16   (row-major)
- * mtpc_lowrank_compose writes W_emit_out, device [n, r, v, d] bf16 = round-to-nearest of the fp32 sum; pass it to
- * mtpc_create_head (which converts it again into the layout of its workspace).
+ * mtpc_lowrank_compose writes W_emit_out, device [n, r, v, d] bf16 = round-to-nearest of the fp32 sum: the W_emit of
+ * mtpc_create_head. A bf16 head reads that buffer in place, so composing into it again after an optimiser step is
+ * all a training loop needs (plus mtpc_update_parameters where T_static changed too).
  * mtpc_lowrank_backward takes the gradient of the composed tensor, dW_emit device [n, r, v, d] fp32 (as written by
  * the backward calls above), and OVERWRITES
  *   dW_base [n, v, d] = sum_j dW_emit[i, j],  dA [n, r, v, k] = dW_emit[i, j] B[i, j]^T,  dB [n, r, k, d] = A[i, j]^T dW_emit[i, j]

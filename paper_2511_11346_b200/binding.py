@@ -23,7 +23,7 @@ EXPORTS = [
     "mtpc_launch_count", "mtpc_destroy", "mtpc_status_string", "mtpc_window_logprob_static",
     "mtpc_window_prefix_logprob", "mtpc_draft_sample_prefix", "mtpc_speculative_accept", "mtpc_window_loss",
     "mtpc_backward_workspace_bytes", "mtpc_window_logprob_backward", "mtpc_window_loss_backward",
-    "mtpc_lowrank_compose", "mtpc_lowrank_backward",
+    "mtpc_lowrank_compose", "mtpc_lowrank_backward", "mtpc_update_parameters",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 ERR_STATIC_SCRATCH = -7
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
     L.mtpc_window_loss_backward.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp, sz, vp, vp, vp, vp, vp, vp, vp]
     L.mtpc_lowrank_compose.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]
     L.mtpc_lowrank_backward.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    L.mtpc_update_parameters.argtypes = [vp, vp, vp, vp, vp]
     L.mtpc_status_string.argtypes = [ctypes.c_int]
     L.mtpc_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -240,6 +241,12 @@ class MtpcHead:
         cnt = ctypes.c_int32(0)
         _check(lib().mtpc_get_timing(self.handle, calls_back, buf, 8, ctypes.byref(cnt)), "mtpc_get_timing")
         return [buf[i] for i in range(cnt.value)]
+
+    def mtpc_update_parameters(self, W_emit, W_sum, T_static=None, stream=None) -> None:
+        """Rebind the head to (possibly updated) parameter tensors; they must outlive the head like the first ones."""
+        _check(lib().mtpc_update_parameters(self.handle, _ptr(W_emit), _ptr(W_sum), _ptr(T_static), _stream(stream)),
+               "mtpc_update_parameters")
+        self._keep = (W_emit, W_sum, T_static)
 
     def mtpc_launch_count(self) -> int:
         out = ctypes.c_uint64(0)

@@ -774,6 +774,53 @@ int check_call(mtpc_head* h, int32_t rows) {
 
 }  // namespace
 
+// Everything the head derives from the parameters: bf16 copies of fp32 weights, the tensor maps on the weight
+// matrices, the log-softmaxed static HMM transitions or the contextual transition bias. Used at creation and again
+// whenever the caller's parameters have changed (mtpc_update_parameters).
+static int bind_parameters(mtpc_head* h, const void* W_emit, const void* W_sum, const float* T_static, cudaStream_t st) {
+  const mtpc_config* cfg = &h->cfg;
+  const Layout& L = h->L;
+  const bool ctx = (cfg->flags & MTPC_FLAG_HMM_CONTEXTUAL) != 0;
+  const size_t emit_count = static_cast<size_t>(cfg->n) * cfg->r * cfg->v * cfg->d;
+  const size_t sum_count = static_cast<size_t>(L.sum_rows) * cfg->d;
+  if (cfg->io_dtype == MTPC_F32) {
+    f32_to_bf16_kernel<<<2048, 256, 0, st>>>(static_cast<const float*>(W_emit), at<__nv_bfloat16>(h, L.off_wemit),
+                                             emit_count);
+    f32_to_bf16_kernel<<<256, 256, 0, st>>>(static_cast<const float*>(W_sum), at<__nv_bfloat16>(h, L.off_wsum),
+                                            sum_count);
+    h->launches += 2;
+    h->W_emit_bf16 = h->ws + L.off_wemit;
+    h->W_sum_bf16 = h->ws + L.off_wsum;
+  } else {
+    h->W_emit_bf16 = W_emit;
+    h->W_sum_bf16 = W_sum;
+  }
+  if (ctx) {
+    // bias of the contextual transition logits, laid out like the sum-unit rows: zeros for the initial unit
+    bool bad = cudaMemsetAsync(h->ws + L.off_sum_bias, 0, static_cast<size_t>(L.sum_rows) * 4, st) != cudaSuccess;
+    if (T_static && cfg->n > 1)
+      bad |= cudaMemcpyAsync(h->ws + L.off_sum_bias + static_cast<size_t>(cfg->r) * 4, T_static,
+                             static_cast<size_t>(cfg->n - 1) * cfg->r * cfg->r * 4, cudaMemcpyDeviceToDevice,
+                             st) != cudaSuccess;
+    if (bad) return MTPC_ERR_CUDA;
+  } else if (cfg->family == MTPC_HMM && cfg->n > 1) {
+    const int rows = (cfg->n - 1) * cfg->r;
+    log_softmax_rows_kernel<<<(rows + 127) / 128, 128, 0, st>>>(T_static, at<float>(h, L.off_logA), rows, cfg->r);
+    h->launches++;
+  }
+  if (check_launch() != MTPC_OK) return MTPC_ERR_CUDA;
+  const uint64_t emit_rows = static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v;
+  int rc = make_tmap(&h->tm_emit_lp, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols);
+  if (rc == MTPC_OK && L.can_draft_many) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
+  if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols);
+  h->decode_tile_rows = decode_tile_rows(static_cast<long long>(emit_rows), h->num_sms);
+  if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_dec, h->W_emit_bf16, emit_rows, cfg->d, h->decode_tile_rows);
+  h->decode_sum_tile_rows = h->decode_tile_rows / 32 * 32;   // whole groups of r <= 32 rows per warp; fits the tile pitch
+  if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum_dec, h->W_sum_bf16, L.sum_rows, cfg->d, h->decode_sum_tile_rows);
+  h->draft_P = 0;                                              // logits left by an earlier draft belong to the old parameters
+  return rc;
+}
+
 extern "C" {
 
 int mtpc_workspace_bytes(const mtpc_config* cfg, size_t* out_bytes) {
@@ -830,45 +877,17 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   fail |= cudaMemsetAsync(h->ws + L.off_status, 0, 256, st) != cudaSuccess;
   if (fail) { delete h; return MTPC_ERR_CUDA; }
 
-  const size_t emit_count = static_cast<size_t>(cfg->n) * cfg->r * cfg->v * cfg->d;
-  const size_t sum_count = static_cast<size_t>(L.sum_rows) * cfg->d;
-  if (cfg->io_dtype == MTPC_F32) {
-    f32_to_bf16_kernel<<<2048, 256, 0, st>>>(static_cast<const float*>(W_emit), at<__nv_bfloat16>(h, L.off_wemit),
-                                             emit_count);
-    f32_to_bf16_kernel<<<256, 256, 0, st>>>(static_cast<const float*>(W_sum), at<__nv_bfloat16>(h, L.off_wsum),
-                                            sum_count);
-    h->launches += 2;
-    h->W_emit_bf16 = h->ws + L.off_wemit;
-    h->W_sum_bf16 = h->ws + L.off_wsum;
-  } else {
-    h->W_emit_bf16 = W_emit;
-    h->W_sum_bf16 = W_sum;
-  }
-  if (ctx) {
-    // bias of the contextual transition logits, laid out like the sum-unit rows: zeros for the initial unit
-    bool bad = cudaMemsetAsync(h->ws + L.off_sum_bias, 0, static_cast<size_t>(L.sum_rows) * 4, st) != cudaSuccess;
-    if (T_static && cfg->n > 1)
-      bad |= cudaMemcpyAsync(h->ws + L.off_sum_bias + static_cast<size_t>(cfg->r) * 4, T_static,
-                             static_cast<size_t>(cfg->n - 1) * cfg->r * cfg->r * 4, cudaMemcpyDeviceToDevice,
-                             st) != cudaSuccess;
-    if (bad) { delete h; return MTPC_ERR_CUDA; }
-  } else if (cfg->family == MTPC_HMM && cfg->n > 1) {
-    const int rows = (cfg->n - 1) * cfg->r;
-    log_softmax_rows_kernel<<<(rows + 127) / 128, 128, 0, st>>>(T_static, at<float>(h, L.off_logA), rows, cfg->r);
-    h->launches++;
-  }
-  if (check_launch() != MTPC_OK) { delete h; return MTPC_ERR_CUDA; }
-  const uint64_t emit_rows = static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v;
-  rc = make_tmap(&h->tm_emit_lp, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols);
-  if (rc == MTPC_OK && L.can_draft_many) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
-  if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols);
-  h->decode_tile_rows = decode_tile_rows(static_cast<long long>(emit_rows), h->num_sms);
-  if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_dec, h->W_emit_bf16, emit_rows, cfg->d, h->decode_tile_rows);
-  h->decode_sum_tile_rows = h->decode_tile_rows / 32 * 32;   // whole groups of r <= 32 rows per warp; fits the tile pitch
-  if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum_dec, h->W_sum_bf16, L.sum_rows, cfg->d, h->decode_sum_tile_rows);
+  rc = bind_parameters(h, W_emit, W_sum, T_static, st);
   if (rc != MTPC_OK) { delete h; return rc; }
   *out = h;
   return MTPC_OK;
+}
+
+int mtpc_update_parameters(mtpc_head* head, const void* W_emit, const void* W_sum, const float* T_static, void* stream) {
+  if (!head || !W_emit || !W_sum) return MTPC_ERR_NULL;
+  const mtpc_config& c = head->cfg;
+  if (c.family == MTPC_HMM && c.n > 1 && !(c.flags & MTPC_FLAG_HMM_CONTEXTUAL) && !T_static) return MTPC_ERR_NULL;
+  return bind_parameters(head, W_emit, W_sum, T_static, static_cast<cudaStream_t>(stream));
 }
 
 int mtpc_window_logprob(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t T, float* out_logprob,

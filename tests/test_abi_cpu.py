@@ -74,6 +74,7 @@ def test_null_pointers_and_status_strings():
     assert lib.mtpc_window_logprob(None, None, None, 0, None, None) == -1
     assert lib.mtpc_draft_sample(None, None, 0, 1, None, None, None, None) == -1
     assert lib.mtpc_destroy(None) == -1
+    assert lib.mtpc_update_parameters(None, None, None, None, None) == -1
     assert lib.mtpc_lowrank_compose(1, 1, 16, 64, 2, None, None, None, None, None) == -1
     assert lib.mtpc_lowrank_backward(1, 1, 16, 64, 2, None, None, None, None, None, None, None) == -1
     fake = ctypes.c_void_p(256)           # never dereferenced: the argument checks come first

@@ -252,3 +252,54 @@ def test_per_kernel_timing_of_the_training_calls():
     assert head.mtpc_get_timing(0) == []
     assert dh.head.mtpc_get_status() == 0
     dh.close()
+
+
+@pytest.mark.parametrize("family,io", [(I.HMM, I.BF16), (I.HMM_CTX, I.BF16), (I.CP, I.F32), (I.BTREE, I.BF16)])
+def test_update_parameters_after_an_optimiser_step(family, io):
+    """A training loop changes the parameters between calls: in place (bf16 heads read the weights where they are) or
+    in new buffers. After mtpc_update_parameters the head computes on the new values - weights, static transitions
+    or transition bias, fp32 weights re-rounded - and a draft made with the old ones can no longer be accepted."""
+    n, r, v, d, T = 4, 8, 64, 128, 70
+    old = I.make_workload("upd_old", I.HeadShape(family, n, r, v, d, io), T, seed=311, weight_std=0.25)
+    new = I.make_workload("upd_new", I.HeadShape(family, n, r, v, d, io), T, seed=312, weight_std=0.25)
+    dh = DeviceHead(old)
+    from oracle import mtpc_oracle as O
+    ref_old = O.window_logprob(family, old.hidden_q, old.W_emit_q, old.W_sum_q, old.T_static, old.targets)
+    assert np.abs(dh.window_logprob().cpu().numpy() - ref_old).max() <= 2e-3
+    fresh = DeviceHead(new)                                     # only to have the new parameters on the device
+    h_new, t_new = fresh.hidden_device(), torch.from_numpy(new.targets).cuda()
+    ref_new = O.window_logprob(family, new.hidden_q, new.W_emit_q, new.W_sum_q, new.T_static, new.targets)
+    # (1) in place: overwrite the tensors the head was created on
+    dh.W_emit.copy_(fresh.W_emit)
+    dh.W_sum.copy_(fresh.W_sum)
+    if dh.T_static is not None:
+        dh.T_static.copy_(fresh.T_static)
+    dh.head.mtpc_update_parameters(dh.W_emit, dh.W_sum, dh.T_static)
+    assert np.abs(dh.window_logprob(hidden=h_new, targets=t_new).cpu().numpy() - ref_new).max() <= 2e-3
+    # (2) other buffers: back to the old values, held in clones
+    back = DeviceHead(old)
+    dh.head.mtpc_update_parameters(back.W_emit, back.W_sum, back.T_static)
+    assert np.abs(dh.window_logprob().cpu().numpy() - ref_old).max() <= 2e-3
+    assert dh.head.mtpc_get_status() == 0
+    # gradients follow the bound parameters too
+    w = torch.full((T,), 1.0 / T, device="cuda")
+    g = dh.window_logprob_backward(w)
+    ref = og.window_logprob_grad(family, old.hidden_q, old.W_emit_q, old.W_sum_q, old.T_static, old.targets,
+                                 np.full(T, 1.0 / T, dtype=np.float32))
+    check("dW_emit after update", g["dW_emit"], ref["dW_emit"], 0.0)
+    for x in (dh, fresh, back):
+        x.close()
+
+
+def test_update_parameters_forgets_the_draft():
+    from paper_2511_11346_b200 import binding as B
+    wl = I.make_workload("upd_draft", I.HeadShape(I.CP, 4, 8, 64, 128), 8, seed=77, wpp=4, weight_std=0.25)
+    dh = DeviceHead(wl, max_wpp=4)
+    bytes_, lq = dh.draft_sample_prefix(wpp=4)
+    dh.head.mtpc_update_parameters(dh.W_emit, dh.W_sum, dh.T_static)
+    p = torch.full((8 * 4, 5, 64), 1.0 / 64, device="cuda")
+    u = torch.full((8 * 4, 5), 0.5, device="cuda")
+    with pytest.raises(B.MtpcError) as e:
+        dh.speculative_accept(8, 4, bytes_, lq, p, u)
+    assert e.value.code == B.ERR_STATE
+    dh.close()
