@@ -303,3 +303,42 @@ def test_update_parameters_forgets_the_draft():
         dh.speculative_accept(8, 4, bytes_, lq, p, u)
     assert e.value.code == B.ERR_STATE
     dh.close()
+
+
+@pytest.mark.parametrize("family", [I.CP, I.HMM, I.BTREE])
+def test_gradient_descent_on_the_device_gradients_lowers_the_loss(family):
+    """Ten plain SGD steps on the Eq. 6 loss with the gradients of mtpc_window_loss_backward (fp32 master weights kept by
+    the test, rounded to bf16 into the head's buffers, mtpc_update_parameters after each step): the loss the device
+    reports must fall at every step, and the fp64 oracle must agree with the last one."""
+    from oracle import mtpc_oracle as O
+    from paper_2511_11346_b200.runner import to_device_bf16
+    n, r, v, d, N, L = 4, 4, 32, 64, 3, 40
+    T = N * L
+    wl = I.make_workload("sgd", I.HeadShape(family, n, r, v, d), T, seed=900 + family, target_kind="zipf", weight_std=0.1)
+    dh = DeviceHead(wl)
+    master = [dh.W_emit.float().clone(), dh.W_sum.float().clone(), None if dh.T_static is None else dh.T_static.clone()]
+    gamma, lr = 0.8, 2.0
+    losses = []
+    for step in range(10):
+        g = dh.window_loss_backward(N, L, gamma)
+        losses.append(float(g["loss"].cpu()[0]))
+        master[0] -= lr * g["dW_emit"]
+        master[1] -= lr * g["dW_sum"]
+        dh.W_emit.copy_(master[0].to(torch.bfloat16))
+        dh.W_sum.copy_(master[1].to(torch.bfloat16))
+        if master[2] is not None:
+            master[2] -= lr * g["dT_static"]
+            dh.T_static.copy_(master[2])
+        dh.head.mtpc_update_parameters(dh.W_emit, dh.W_sum, dh.T_static)
+    slot, loss = dh.window_loss(N, L, gamma)
+    losses.append(float(loss.cpu()[0]))
+    assert dh.head.mtpc_get_status() == 0
+    assert all(b < a for a, b in zip(losses, losses[1:])), losses
+    assert losses[-1] < 0.9 * losses[0], losses
+    We = dh.W_emit.float().cpu().numpy().astype(np.float64)
+    Ws = dh.W_sum.float().cpu().numpy().astype(np.float64)
+    Ts = None if dh.T_static is None else dh.T_static.cpu().numpy().astype(np.float64)
+    pre = O.window_prefix_logprob(family, wl.hidden_q, We, Ws, Ts, wl.targets)
+    _, ref = O.composite_loss(pre, wl.targets, N, gamma)
+    assert abs(losses[-1] - ref) <= 2e-3 * n, (losses[-1], ref)
+    dh.close()
