@@ -232,8 +232,8 @@ def measure_decode_cell(torch, cell, steps: int, warmup: int):
 
 def measure_backward(torch, dh, wl, hidden, targets, steps: int, peaks):
     """One training step of the head = mtpc_window_logprob_backward (forward value + all gradients): ms per call,
-    the per-phase split from the library's event ring, and the tensor throughput over the four weight-sized
-    contractions it runs (forward, recompute, d hidden, dW): 4 x the forward's algorithmic FLOPs."""
+    the per-phase split from the library's event ring, and the tensor throughput over the three weight-sized
+    contractions it runs (forward, d hidden, dW): 3 x the forward's algorithmic FLOPs."""
     s = wl.shape
     f32 = dict(dtype=torch.float32, device="cuda")
     weight = torch.full((wl.T,), -1.0 / wl.T, **f32)
@@ -254,13 +254,13 @@ def measure_backward(torch, dh, wl, hidden, targets, steps: int, peaks):
     phases = [dh.head.mtpc_get_timing(i) for i in range(steps)]
     phase_ms = [statistics.mean(p[k] for p in phases) for k in range(len(phases[0]))]
     dh.head.mtpc_set_timing(0)
-    flops = 4.0 * algorithmic_flops(wl)
+    flops = 3.0 * algorithmic_flops(wl)
     tf = flops / (ms * 1e-3) / 1e12
     eq6 = measure_eq6_step(torch, dh, wl, hidden, targets, out, steps)
     lowrank = measure_lowrank(torch, wl, out[2], steps, peaks) if s.v <= 1536 else None
     return {"eq6_training_step": eq6, "lowrank_unembeddings": lowrank, "call": "mtpc_window_logprob_backward", "ms_per_call": ms, "positions_per_s": wl.T / (ms * 1e-3),
             "phase_ms": {"forward_projection": phase_ms[0], "circuit_backward": phase_ms[1],
-                         "projection_gradient_mode": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]},
+                         "logit_gradient": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]},
             "flops_per_call": flops, "achieved_tflops": tf, "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
             "device_status": dh.head.mtpc_get_status()}
 
@@ -331,7 +331,7 @@ def measure_eq6_step(torch, dh, wl, hidden, targets, grads, steps: int):
     return {"call": "mtpc_window_loss_backward", "sequences": N, "sequence_length": L, "gamma": gamma, "ms_per_call": ms,
             "positions_per_s": wl.T / (ms * 1e-3), "loss": float(loss.cpu()[0]),
             "phase_ms": {"forward_prefix_loss": phase_ms[0], "circuit_backward_passes": phase_ms[1],
-                         "projection_gradient_mode": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]}}
+                         "logit_gradient": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]}}
 
 
 def run_ours(args):

@@ -213,9 +213,10 @@ int mtpc_window_loss(mtpc_head* head, const void* hidden, const int32_t* targets
  *   hidden, targets, T   as for mtpc_window_logprob (a negative target is a marginalised byte: no gradient).
  *   weight        dev [T] fp32.
  *   bwd_workspace dev, 256-byte aligned, >= mtpc_backward_workspace_bytes(cfg, T): holds the units' log-sum-exps and
- *                 posteriors, the bf16 gradient of the logits in both orientations (2 * T * n*r*v * 2 bytes: the one
- *                 large buffer; the fp32 logits themselves are recomputed on chip and never stored) and transposed bf16
- *                 copies of W_emit, W_sum and hidden. Caller-owned, used only during the call's work.
+ *                 posteriors, the fp32 emission logits the forward pass keeps for the backward pass (T * n*r*v * 4
+ *                 bytes), the bf16 gradient of the logits in both orientations (as many bytes again: the large
+ *                 buffers) and transposed bf16 copies of W_emit, W_sum and hidden. Caller-owned, used only during the
+ *                 call's work.
  *   out_logprob   dev [T] fp32 or NULL: the forward value.
  *   d_hidden      dev [T, d] fp32;  dW_emit dev [n, r, v, d] fp32;  dW_sum dev [S*r, d] fp32: overwritten, not
  *                 accumulated.
@@ -296,7 +297,7 @@ int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags);
  *   mtpc_window_logprob: [0] projection GEMM + fused epilogue, [1] circuit evaluation.
  *   mtpc_window_prefix_logprob, mtpc_window_loss: as mtpc_window_logprob (the loss reduction is not timed).
  *   mtpc_speculative_accept: [0] the acceptance kernel.
- *   mtpc_window_logprob_backward: [0] forward projection, [1] circuit backward, [2] projection in gradient mode,
+ *   mtpc_window_logprob_backward: [0] forward projection, [1] circuit backward, [2] gradient of the logits,
  *                        [3] transposes and the plain GEMMs.
  *   mtpc_window_loss_backward: [0] forward projection + prefix marginals + loss, [1] the n circuit backward passes,
  *                        [2] and [3] as above.

@@ -277,7 +277,7 @@ void launch_kernel(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem
 }
 
 // Launch the projection kernel for `rows` positions over the emission groups (with_emit) and / or the sum tiles.
-// Units per work item of the log-likelihood / gradient modes. An item covers its units with 256-column tiles; unless the
+// Units per work item of the log-likelihood mode. An item covers its units with 256-column tiles; unless the
 // units end on a tile boundary the last tile is partly wasted (its tail belongs to the next item, which recomputes it).
 // Items are dealt round-robin to `ctas` persistent CTAs, so a launch takes about rounds x tiles-per-item tile times:
 // pick the count that minimises that (v = 320: 4 units = 5 tiles, nothing wasted; v = 272: 8 units = 9 tiles, 6 % wasted
@@ -296,14 +296,10 @@ int choose_group_units(int v, int emit_units, int m_tiles, int ctas) {
   return best;
 }
 
-struct GradArgs {            // what the projection kernel needs beyond the forward arguments (backward pass only)
-  float* lse_out = nullptr;                  // forward for training: keep the units' log-sum-exps
-  const float* lse_in = nullptr;             // gradient mode
-  const float* post = nullptr;
-  __nv_bfloat16* dlogit = nullptr;
-  __nv_bfloat16* dlogit_t = nullptr;
-  size_t t_pitch = 0;
-  size_t dlogit_pitch = 0;
+struct GradArgs {            // what the projection kernel keeps for the backward pass (training calls only)
+  float* lse_out = nullptr;                  // the units' log-sum-exps [T, n, r]
+  float* logit_out = nullptr;                // the emission logits [T, n r v] fp32
+  size_t logit_pitch = 0;
 };
 
 int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int wpp, bool with_emit, bool with_sum,
@@ -317,12 +313,8 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   memset(&p, 0, sizeof(p));
   if (ga) {
     p.lse_out = ga->lse_out;
-    p.lse_in = ga->lse_in;
-    p.post = ga->post;
-    p.dlogit = ga->dlogit;
-    p.dlogit_t = ga->dlogit_t;
-    p.t_pitch = ga->t_pitch;
-    p.dlogit_pitch = ga->dlogit_pitch;
+    p.logit_out = ga->logit_out;
+    p.logit_pitch = ga->logit_pitch;
   }
   int rc = make_tmap(&p.tm_a, hidden_bf16, static_cast<uint64_t>(rows), static_cast<uint64_t>(c.d), kBlockM);
   if (rc != MTPC_OK) return rc;
@@ -367,8 +359,6 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
   if (mode == kModeLogprob)
     mtpc_gemm_kernel<kModeLogprob><<<grid, kGemmThreads, tl.smem, st>>>(p);
-  else if (mode == kModeGrad)
-    mtpc_gemm_kernel<kModeGrad><<<grid, kGemmThreads, tl.smem, st>>>(p);
   else
     mtpc_gemm_kernel<kModeSample><<<grid, kGemmThreads, tl.smem, st>>>(p);
   h->launches++;
@@ -606,7 +596,7 @@ size_t round64(size_t x) { return (x + 63) / 64 * 64; }
 // and W_sum^T to the right of W_emit^T in [d, Kd], so that d hidden is a single GEMM over K = Nc + S r.
 struct BackwardLayout {
   size_t Nc, Spad, Tpad, Kd;
-  size_t off_lse, off_post, off_dsum_t, off_dlogit, off_dlogit_t, off_wt, off_ht, off_dsum_f32, off_coeff, total;
+  size_t off_lse, off_post, off_logits, off_dsum_t, off_dlogit, off_dlogit_t, off_wt, off_ht, off_dsum_f32, off_coeff, total;
 };
 void plan_backward(const mtpc_config& c, const Layout& L, int T, BackwardLayout* B) {
   B->Nc = static_cast<size_t>(c.n) * c.r * c.v;
@@ -617,6 +607,7 @@ void plan_backward(const mtpc_config& c, const Layout& L, int T, BackwardLayout*
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
   B->off_lse = take(static_cast<size_t>(T) * c.n * c.r * 4);
   B->off_post = take(static_cast<size_t>(T) * c.n * c.r * 4);
+  B->off_logits = take(static_cast<size_t>(T) * B->Nc * 4);              // [T, Nc] fp32: the emission logits of the forward pass
   B->off_dsum_t = take(static_cast<size_t>(L.sum_rows) * B->Tpad * 2);  // [S r, Tpad] bf16
   B->off_dlogit = take(static_cast<size_t>(T) * B->Kd * 2);          // [T, Nc | Spad]
   B->off_dlogit_t = take(B->Nc * B->Tpad * 2);                       // [Nc, Tpad]
@@ -727,7 +718,7 @@ int set_backward_attributes(const mtpc_head* head) {
   return fail ? MTPC_ERR_CUDA : MTPC_OK;
 }
 
-// Phases 3 and 4 of a backward call: the projection kernel in gradient mode (post, lse -> bf16 logit gradients), the
+// Phases 3 and 4 of a backward call: the logit gradients (post, lse and the kept logits -> bf16, both orientations), the
 // transposes and the plain GEMMs. The sum-unit logit gradients are already in place to the right of dlogit.
 int backward_tail(mtpc_head* head, const BackwardLayout& B, uint8_t* bw, const void* hb, const int32_t* targets, int T,
                   float* d_hidden, float* dW_emit, float* dW_sum, PhaseTimer& pt, cudaStream_t st) {
@@ -741,14 +732,19 @@ int backward_tail(mtpc_head* head, const BackwardLayout& B, uint8_t* bw, const v
   void* ht = bw + B.off_ht;
   const int Nc = static_cast<int>(B.Nc);
   pt.begin();
-  GradArgs ga;
-  ga.lse_in = reinterpret_cast<float*>(bw + B.off_lse);
-  ga.post = reinterpret_cast<float*>(bw + B.off_post);
-  ga.dlogit = dlogit;
-  ga.dlogit_t = dlogit_t;
-  ga.t_pitch = B.Tpad;
-  ga.dlogit_pitch = B.Kd;
-  int rc = launch_gemm(head, kModeGrad, hb, T, 1, true, false, targets, nullptr, nullptr, st, &ga);
+  LogitGradArgs la;
+  la.logits = reinterpret_cast<const float*>(bw + B.off_logits);
+  la.lse = reinterpret_cast<const float*>(bw + B.off_lse);
+  la.post = reinterpret_cast<const float*>(bw + B.off_post);
+  la.targets = targets;
+  la.dlogit = dlogit;
+  la.dlogit_t = dlogit_t;
+  la.pitch = B.Kd;
+  la.t_pitch = B.Tpad;
+  la.T = T; la.Nc = Nc; la.n = c.n; la.r = c.r; la.v = c.v;
+  logit_gradient_kernel<<<dim3((Nc + 63) / 64, (T + 63) / 64), 256, 0, st>>>(la);
+  head->launches++;
+  int rc = check_launch();
   pt.end();
   if (rc != MTPC_OK) return rc;
   pt.begin();
@@ -858,8 +854,6 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeSample>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               kSmemLimit) != cudaSuccess;
-  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeGrad>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
   fail |= cudaFuncSetAttribute(plain_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
           cudaSuccess;
@@ -1017,6 +1011,8 @@ int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int3
   pt.begin();
   GradArgs fwd;
   fwd.lse_out = reinterpret_cast<float*>(bw + B.off_lse);
+  fwd.logit_out = reinterpret_cast<float*>(bw + B.off_logits);
+  fwd.logit_pitch = B.Nc;
   rc = launch_gemm(head, kModeLogprob, hb, T, 1, true, true, targets, nullptr, nullptr, st, &fwd);
   pt.end();
   if (rc != MTPC_OK) return rc;
@@ -1038,7 +1034,7 @@ int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int3
   rc = launch_circuit_backward(head, a, dT_static, st);
   pt.end();
   if (rc != MTPC_OK) return rc;
-  // 3., 4. logit gradients from the recomputed logits, then the plain GEMMs
+  // 3., 4. logit gradients from the kept logits, then the plain GEMMs
   return backward_tail(head, B, bw, hb, targets, T, d_hidden, dW_emit, dW_sum, pt, st);
 }
 
@@ -1079,6 +1075,8 @@ int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t
   pt.begin();
   GradArgs fwd;
   fwd.lse_out = reinterpret_cast<float*>(bw + B.off_lse);
+  fwd.logit_out = reinterpret_cast<float*>(bw + B.off_logits);
+  fwd.logit_pitch = B.Nc;
   rc = launch_gemm(head, kModeLogprob, hb, T, 1, true, true, targets, nullptr, nullptr, st, &fwd);
   if (rc == MTPC_OK) rc = launch_circuit(head, T, 1, nullptr, prefix, st);
   if (rc != MTPC_OK) return rc;

@@ -3,15 +3,17 @@
 // with respect to the hidden states, the emission weights, the sum-unit weights and the static transition logits.
 //
 // Stages (host side in mtpc_api.cu):
-//   1. forward projection kernel, also saving the log-sum-exp of every input unit (lse [T, n, r]);
+//   1. forward projection kernel, also keeping the emission logits ([T, n r v] fp32, streamed out of the epilogue) and
+//      the log-sum-exp of every input unit (lse [T, n, r]);
 //   2. circuit backward (this file): one warp per window runs the upward and the downward pass of the circuit and
 //      writes post[w, i, k] = weight * d log q / d G[w, i, k] (the posterior of "token i is emitted by unit k") and
 //      dsum[w, :] = weight * d log q / d (sum-unit logits), i.e. posterior minus prior of every sum unit, in bf16;
-//   3. the projection kernel once more in gradient mode: logits are recomputed tile by tile in tensor memory and turned
-//      into dlogit = post * (onehot(target) - softmax) in the epilogue, written as bf16 in both orientations;
+//   3. logit_gradient_kernel (this file): dlogit = post * (onehot(target) - exp(logit - lse)), one streaming pass over
+//      the kept logits, written as bf16 in both orientations;
 //   4. plain bf16 GEMMs (plain_gemm_kernel, this file) on those: d hidden = dlogit W + dsum R, dW = dlogit^T h,
-//      dR = dsum^T h. The [T, n, r, v] fp32 logit tensor still never exists; its bf16 gradient does, as the operand of
-//      the two weight-sized GEMMs.
+//      dR = dsum^T h.
+// Only the training calls materialise the logits (fp32, and their bf16 gradient, as the operands of the two weight-sized
+// GEMMs); recomputing them on chip instead was measured: a fourth weight-sized contraction against 0.6 ms of streaming.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -452,6 +454,75 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
   for (int e = threadIdx.x; e < 64 * 64; e += 256) {
     const int cc = e / 64, rr_ = e % 64;
     if (r0 + rr_ < rows && c0 + cc < cols) dst[static_cast<size_t>(c0 + cc) * dst_pitch + r0 + rr_] = tile[rr_][cc];
+  }
+}
+
+// ---------------------------------------------------------------- gradient with respect to the emission logits
+// dlogit[t, c] = post[t, u] * (onehot(target[t, i] == c - u v) - exp(logit[t, c] - lse[t, u])),  u = c / v = i r + k,
+// from the logits and log-sum-exps the forward pass kept (padding columns hold -inf: no mass, zero gradient; a
+// marginalised byte has no gradient). Written as bf16 in both orientations, the operands of the two weight-sized
+// GEMMs: dlogit [T, pitch] and dlogit_t [n r v, t_pitch] (columns T..round64(T) zero). 64 x 64 tiles, 256 threads:
+// a thread reads 4 adjacent logits (16 bytes) of 4 rows; the transposed copy goes through shared memory and leaves
+// as 16-byte pieces along t. v is a multiple of 16, so 4 adjacent columns belong to one unit.
+struct LogitGradArgs {
+  const float* logits;       // [T, Nc], pitch Nc
+  const float* lse;          // [T, n r]
+  const float* post;         // [T, n r]
+  const int* targets;        // [T, n]
+  __nv_bfloat16* dlogit;     // [T, pitch]
+  __nv_bfloat16* dlogit_t;   // [Nc, t_pitch]
+  size_t pitch, t_pitch;
+  int T, Nc, n, r, v;
+};
+
+__global__ void __launch_bounds__(256) logit_gradient_kernel(const LogitGradArgs a) {
+  // [column][row]; the rows of column c are rotated by 8 ((c / 4) mod 8) places so that the 16 threads of a row group,
+  // four columns apart, do not all fall on the same two banks
+  __shared__ __align__(16) __nv_bfloat16 tile[64][72];
+  const int c0 = blockIdx.x * 64, t0 = blockIdx.y * 64;
+  const int cg = (threadIdx.x & 15) * 4;                            // the thread's 4 columns within the tile
+  const int tr0 = (threadIdx.x >> 4) * 4;                           // and its 4 rows
+  const int rot = 8 * ((cg >> 2) & 7);
+  const int c = c0 + cg;
+  const int units = a.n * a.r;
+  __align__(8) __nv_bfloat16 o[4][4];                               // [column][row]
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int t = t0 + tr0 + pass;
+    __align__(8) __nv_bfloat16 orow[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) orow[q] = __float2bfloat16_rn(0.f);
+    if (t < a.T && c < a.Nc) {
+      const int u = c / a.v;
+      const int i = u / a.r;
+      const int tgt = a.targets[static_cast<size_t>(t) * a.n + i];
+      const size_t tu = static_cast<size_t>(t) * units + u;
+      const float pst = tgt >= 0 ? a.post[tu] : 0.f;
+      const float lse2 = a.lse[tu] * kLog2e;
+      const float4 x = __ldcs(reinterpret_cast<const float4*>(a.logits + static_cast<size_t>(t) * a.Nc + c));
+      const float xs[4] = {x.x, x.y, x.z, x.w};
+      const int rel = tgt - (c - u * a.v);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        orow[q] = __float2bfloat16_rn(pst * ((rel == q ? 1.f : 0.f) - fast_ex2(fmaf(xs[q], kLog2e, -lse2))));
+      *reinterpret_cast<uint2*>(a.dlogit + static_cast<size_t>(t) * a.pitch + c) = *reinterpret_cast<const uint2*>(orow);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) o[q][pass] = orow[q];
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    *reinterpret_cast<uint2*>(&tile[cg + q][(tr0 + rot) & 63]) = *reinterpret_cast<const uint2*>(o[q]);
+  __syncthreads();
+  // transposed copy: thread -> (column, 16 rows); rows beyond T carry zeros, those beyond the pitch are not written
+  const int cc = threadIdx.x >> 2, seg = (threadIdx.x & 3) * 16;
+  if (c0 + cc < a.Nc) {
+    const int crot = 8 * ((cc >> 2) & 7);
+    __nv_bfloat16* dst = a.dlogit_t + static_cast<size_t>(c0 + cc) * a.t_pitch + t0 + seg;
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+      if (static_cast<size_t>(t0 + seg + 8 * h + 8) <= a.t_pitch)
+        *reinterpret_cast<uint4*>(dst + 8 * h) = *reinterpret_cast<const uint4*>(&tile[cc][(seg + 8 * h + crot) & 63]);
   }
 }
 

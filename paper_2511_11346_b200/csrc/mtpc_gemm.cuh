@@ -1,7 +1,8 @@
 // Projection kernel of the MtPC head (Sec. 3.3): logits = h W^T on the tcgen05 tensor cores, with the softmax
 // over the vocabulary, the evidence gather (log phi at the target byte) or the inverse-CDF byte draw
 // (Algorithm 1, input units), and the log-softmax of the sum-unit logits all done in the epilogue straight
-// out of tensor memory. The [positions, n, r, v] logit tensor never exists in HBM.
+// out of tensor memory. The [positions, n, r, v] logit tensor never exists in HBM, except when a training call asks the
+// epilogue to keep it for the backward pass (logit_out).
 //
 // One persistent CTA per SM, 6 warps:
 //   warp 0      TMA producer: per 64-wide K block, one 128-row tile of h and the v rows of one emission unit
@@ -37,7 +38,7 @@ constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per barr
 constexpr int kABytes = kBlockM * kBlockK * 2;                   // 16 KB
 constexpr uint32_t kStatusBadTarget = 1u, kStatusBadUniform = 2u, kStatusTimeout = 4u;
 
-enum { kModeLogprob = 0, kModeSample = 1, kModeGrad = 2 };
+enum { kModeLogprob = 0, kModeSample = 1 };
 
 struct GemmParams {
   CUtensorMap tm_a;      // hidden  [T, d]        box 64 x 128
@@ -61,13 +62,8 @@ struct GemmParams {
   float* logw;                       // [T, S*r]        log-softmaxed sum-unit weights
   const float* sum_bias;             // [S*r] or NULL   added to the sum-unit logits before their softmax
   float* lse_out;                    // [T, n, r] or NULL: log-sum-exp of every input unit, kept for the backward pass
-  // gradient mode: dlogit[t, col] = post[t, i, k] * (onehot(target) - exp(logit - lse[t, i, k])), bf16, both orientations
-  const float* lse_in;               // [T, n, r]
-  const float* post;                 // [T, n, r]   weight * d log q / d G
-  __nv_bfloat16* dlogit;             // [T, n*r*v] with row pitch dlogit_pitch
-  size_t dlogit_pitch;
-  __nv_bfloat16* dlogit_t;           // [n*r*v, t_pitch]
-  size_t t_pitch;
+  float* logit_out;                  // [T, n*r*v] fp32 with row pitch logit_pitch, or NULL: the emission logits themselves,
+  size_t logit_pitch;                // kept for the backward pass (padding columns as -inf); wpp == 1 only
   const int* unit_sel;               // [T*wpp, n]      selected input unit per token (sample mode)
   const float* uniforms;             // [T*wpp, 2n]
   int* out_bytes;                    // [T*wpp, n]
@@ -412,6 +408,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
             float x[16];
             tmem_ld16(tcol + b * 16, x);
             mask_padding(x, col_in_unit, p.vv);
+            if (p.logit_out != nullptr && valid) {                       // row of W_emit = column of the logit matrix
+              float4* l4 = reinterpret_cast<float4*>(p.logit_out + static_cast<size_t>(row) * p.logit_pitch + tc.brow0 +
+                                                     t * tc.cols + b * 16);
+#pragma unroll
+              for (int q = 0; q < 4; ++q)                                // streaming stores: written once, read once much later
+                __stcs(l4 + q, make_float4(x[4 * q], x[4 * q + 1], x[4 * q + 2], x[4 * q + 3]));
+            }
             float bm = x[0];
 #pragma unroll
             for (int q = 1; q < 16; ++q) bm = fmaxf(bm, x[q]);
@@ -467,65 +470,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
                 slot_i = unit / p.r;
                 k = unit - slot_i * p.r;
                 tgt = (p.wpp == 1 && valid) ? p.targets[wrow0 * p.n + slot_i] : -1;
-              }
-            }
-          }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&ctl->tempty[slot]));
-        }
-        if (!ok) break;
-      } else if (MODE == kModeGrad) {
-        // ---- gradient of the loss with respect to the logits of this item's units, from the recomputed logits:
-        // post * (onehot(target) - softmax). No reduction is needed: the log-sum-exps were kept by the forward pass.
-        const int units_end = tc.unit0 + tc.nunits;
-        int unit = tc.unit0, col_in_unit = 0;
-        int slot_i = unit / p.r, k = unit - slot_i * p.r;
-        const size_t trow = static_cast<size_t>(valid ? row : 0);
-        float pst = 0.f, lse2 = 0.f;
-        int tgt = -1;
-        auto load_unit = [&]() {
-          const size_t u = (trow * p.n + slot_i) * p.r + k;
-          tgt = valid ? p.targets[trow * p.n + slot_i] : -1;
-          pst = (valid && tgt >= 0) ? p.post[u] : 0.f;                  // a marginalised byte has no gradient
-          lse2 = valid ? p.lse_in[u] * kLog2e : 0.f;
-        };
-        load_unit();
-        for (int t = 0; t < tc.ntiles && ok; ++t, ++use) {
-          const uint32_t slot = use % p.num_slots;
-          if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (use / p.num_slots) & 1u, ctl, p.status, lane)) {
-            ok = false;
-            break;
-          }
-          tc_fence_after();
-          const uint32_t tcol = lane_base + slot * p.slot_stride;
-          for (int b = 0; b < nbatch && unit < units_end; ++b) {
-            float x[16];
-            tmem_ld16(tcol + b * 16, x);
-            mask_padding(x, col_in_unit, p.vv);                         // padding columns: softmax 0, gradient 0
-            const int col0 = tc.brow0 + t * tc.cols + b * 16;           // row of W_emit = column of the logit matrix
-            const int rel = tgt - col_in_unit;
-            __align__(16) __nv_bfloat16 o[16];
-#pragma unroll
-            for (int q = 0; q < 16; ++q) {
-              const float sm_ = fast_ex2(fmaf(x[q], kLog2e, -lse2));
-              o[q] = __float2bfloat16_rn(pst * ((rel == q ? 1.f : 0.f) - sm_));
-            }
-            if (valid) {
-              uint4* d4 = reinterpret_cast<uint4*>(p.dlogit + trow * p.dlogit_pitch + col0);
-              d4[0] = *reinterpret_cast<const uint4*>(&o[0]);
-              d4[1] = *reinterpret_cast<const uint4*>(&o[8]);
-#pragma unroll
-              for (int q = 0; q < 16; ++q) p.dlogit_t[static_cast<size_t>(col0 + q) * p.t_pitch + trow] = o[q];
-            }
-            col_in_unit += 16;
-            if (col_in_unit == p.v) {
-              ++unit;
-              col_in_unit = 0;
-              if (unit < units_end) {
-                slot_i = unit / p.r;
-                k = unit - slot_i * p.r;
-                load_unit();
               }
             }
           }

@@ -237,7 +237,7 @@ def test_per_kernel_timing_of_the_training_calls():
     w = torch.ones(40, device="cuda")
     dh.window_logprob_backward(w)
     ph = head.mtpc_get_timing(0)
-    assert len(ph) == 4 and all(p > 0 for p in ph)            # forward, circuit backward, gradient-mode projection, GEMMs
+    assert len(ph) == 4 and all(p > 0 for p in ph)            # forward, circuit backward, logit gradients, GEMMs
     dh.window_loss_backward(4, 10, 0.8)
     ph = head.mtpc_get_timing(0)
     assert len(ph) == 4 and all(p > 0 for p in ph)            # forward+prefix+loss, the n circuit passes, projection, GEMMs
