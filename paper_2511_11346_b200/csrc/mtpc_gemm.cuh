@@ -409,11 +409,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
             tmem_ld16(tcol + b * 16, x);
             mask_padding(x, col_in_unit, p.vv);
             if (p.logit_out != nullptr && valid) {                       // row of W_emit = column of the logit matrix
-              float4* l4 = reinterpret_cast<float4*>(p.logit_out + static_cast<size_t>(row) * p.logit_pitch + tc.brow0 +
-                                                     t * tc.cols + b * 16);
-#pragma unroll
-              for (int q = 0; q < 4; ++q)                                // streaming stores: written once, read once much later
-                __stcs(l4 + q, make_float4(x[4 * q], x[4 * q + 1], x[4 * q + 2], x[4 * q + 3]));
+              float* l = p.logit_out + static_cast<size_t>(row) * p.logit_pitch + tc.brow0 + t * tc.cols + b * 16;
+              st_global_v8(l, x);                                        // 64-byte aligned: v and the tile widths are multiples of 16
+              st_global_v8(l + 8, x + 8);
             }
             float bm = x[0];
 #pragma unroll
