@@ -770,6 +770,14 @@ int check_call(mtpc_head* h, int32_t rows) {
 
 }  // namespace
 
+// The vector paths of the low-rank kernels need d a multiple of 4 and 16-byte aligned pointers.
+static bool lowrank_vector_ok(int d, std::initializer_list<const void*> ptrs) {
+  if (d % 4) return false;
+  for (const void* p : ptrs)
+    if (reinterpret_cast<uintptr_t>(p) % 16) return false;
+  return true;
+}
+
 // Everything the head derives from the parameters: bf16 copies of fp32 weights, the tensor maps on the weight
 // matrices, the log-softmaxed static HMM transitions or the contextual transition bias. Used at creation and again
 // whenever the caller's parameters have changed (mtpc_update_parameters).
@@ -1134,13 +1142,6 @@ static int ensure_copy_pipeline(mtpc_head* head, int chunks) {
     head->copy_event_count = chunks + 1;
   }
   return MTPC_OK;
-}
-
-static bool lowrank_vector_ok(int d, std::initializer_list<const void*> ptrs) {
-  if (d % 4) return false;
-  for (const void* p : ptrs)
-    if (reinterpret_cast<uintptr_t>(p) % 16) return false;
-  return true;
 }
 
 int mtpc_lowrank_compose(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k, const void* W_base, const void* A,
