@@ -672,7 +672,9 @@ int circuit_backward_warps(const mtpc_head* h) {
   return 0;
 }
 
-int launch_circuit_backward(mtpc_head* h, CircuitBackwardArgs a, float* dT, cudaStream_t st) {
+// `loss_coeff` (HMM only): the weights [W, n] of the prefix log-marginals in Eq. 6; the whole gradient in one pass.
+int launch_circuit_backward(mtpc_head* h, CircuitBackwardArgs a, float* dT, cudaStream_t st,
+                            const float* loss_coeff = nullptr) {
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
   a.G = at<float>(h, L.off_G);
@@ -690,6 +692,9 @@ int launch_circuit_backward(mtpc_head* h, CircuitBackwardArgs a, float* dT, cuda
   if (c.family != MTPC_CP && cudaMemsetAsync(counter, 0, sizeof(unsigned), st) != cudaSuccess) return MTPC_ERR_CUDA;
   if (c.family == MTPC_CP) {
     circuit_cp_backward_kernel<<<blocks, threads, 0, st>>>(a);
+  } else if (c.family == MTPC_HMM && loss_coeff != nullptr) {
+    circuit_hmm_loss_backward_kernel<<<resident, threads, smem, st>>>(a, loss_coeff, hmm_tables(h), hmm_table_stride(h), dT,
+                                                                     counter);
   } else if (c.family == MTPC_HMM) {
     circuit_hmm_backward_kernel<<<resident, threads, smem, st>>>(a, hmm_tables(h), hmm_table_stride(h), dT, counter);
   } else {
@@ -708,12 +713,15 @@ int set_backward_attributes(const mtpc_head* head) {
   const size_t smem = circuit_backward_smem(head, warps);
   bool fail = false;
   if (smem > 48 * 1024) {
-    if (c.family == MTPC_HMM)
+    if (c.family == MTPC_HMM) {
       fail |= cudaFuncSetAttribute(circuit_hmm_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    static_cast<int>(smem)) != cudaSuccess;
-    else
+      fail |= cudaFuncSetAttribute(circuit_hmm_loss_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   static_cast<int>(smem)) != cudaSuccess;
+    } else {
       fail |= cudaFuncSetAttribute(circuit_btree_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                    static_cast<int>(smem)) != cudaSuccess;
+    }
   }
   return fail ? MTPC_ERR_CUDA : MTPC_OK;
 }
@@ -1094,27 +1102,39 @@ int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t
   head->launches += 3;
   pt.end();
   if ((rc = check_launch()) != MTPC_OK) return rc;
-  // 2. one circuit backward pass per prefix length, accumulating
+  // 2. circuit backward. HMM: every prefix marginal is a forward message, so one reverse sweep gives the whole gradient.
+  // Mixture and tree: one pass per prefix length, accumulating.
   pt.begin();
-  bool bad = cudaMemsetAsync(post, 0, static_cast<size_t>(T) * c.n * c.r * 4, st) != cudaSuccess;
-  bad |= cudaMemsetAsync(dsum_f32, 0, static_cast<size_t>(T) * L.sum_rows * 4, st) != cudaSuccess;
-  if (static_hmm) bad |= cudaMemsetAsync(dT_static, 0, static_cast<size_t>(c.n - 1) * c.r * c.r * 4, st) != cudaSuccess;
-  if (bad) return MTPC_ERR_CUDA;
-  for (int j = 0; j < c.n; ++j) {
+  if (static_hmm && cudaMemsetAsync(dT_static, 0, static_cast<size_t>(c.n - 1) * c.r * c.r * 4, st) != cudaSuccess)
+    return MTPC_ERR_CUDA;
+  if (c.family == MTPC_HMM) {
     CircuitBackwardArgs a;
     memset(&a, 0, sizeof(a));
     a.targets = targets;
-    a.weight = coeff + j;
-    a.weight_stride = c.n;
     a.post = post;
-    a.dsum_f32 = dsum_f32;
-    a.dsum_pitch = L.sum_rows;
-    a.len = j + 1;
-    a.accumulate = 1;
+    a.dsum = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit) + B.Nc;    // columns [Nc, Nc + S r) of the dlogit rows
+    a.dsum_pitch = static_cast<int>(B.Kd);
+    a.len = c.n;
     a.W = T;
-    if ((rc = launch_circuit_backward(head, a, dT_static, st)) != MTPC_OK) return rc;
-  }
-  {
+    if ((rc = launch_circuit_backward(head, a, dT_static, st, coeff)) != MTPC_OK) return rc;
+  } else {
+    bool bad = cudaMemsetAsync(post, 0, static_cast<size_t>(T) * c.n * c.r * 4, st) != cudaSuccess;
+    bad |= cudaMemsetAsync(dsum_f32, 0, static_cast<size_t>(T) * L.sum_rows * 4, st) != cudaSuccess;
+    if (bad) return MTPC_ERR_CUDA;
+    for (int j = 0; j < c.n; ++j) {
+      CircuitBackwardArgs a;
+      memset(&a, 0, sizeof(a));
+      a.targets = targets;
+      a.weight = coeff + j;
+      a.weight_stride = c.n;
+      a.post = post;
+      a.dsum_f32 = dsum_f32;
+      a.dsum_pitch = L.sum_rows;
+      a.len = j + 1;
+      a.accumulate = 1;
+      a.W = T;
+      if ((rc = launch_circuit_backward(head, a, dT_static, st)) != MTPC_OK) return rc;
+    }
     const size_t total = static_cast<size_t>(T) * L.sum_rows;
     const int blocks = static_cast<int>((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
     f32_rows_to_bf16_kernel<<<blocks, 256, 0, st>>>(dsum_f32, reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit) + B.Nc, T,

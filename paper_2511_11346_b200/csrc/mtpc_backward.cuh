@@ -165,10 +165,12 @@ __device__ __forceinline__ void row_grad(const float* row, const float* pc, floa
 // Tables as in circuit_hmm_stream_kernel (static: stride 0; contextual: one set per position inside log omega).
 // Contextual: the transition-logit gradients go to dsum (bf16, one row per position). Static: they are summed over
 // the windows into dT [n-1, r, r] (fp32): per CTA in shared memory first, then one atomicAdd per entry and CTA.
-// Shared memory: per warp n*r (alpha) + 2*r*r (tables) + 32 floats; static: + (n-1)*r*r floats per CTA.  r <= 32.
+// Shared memory: per warp n*r (alpha) + 2*r*r (tables) + 64 floats; static: + (n-1)*r*r floats per CTA.  r <= 32.
+__host__ __device__ inline size_t hmm_backward_warp_floats(int n, int r) {
+  return static_cast<size_t>(n) * r + 2 * r * r + 64;             // alphas, two tables, two vectors of 32
+}
 __host__ __device__ inline size_t hmm_backward_smem_floats(int n, int r, bool is_static, int warps) {
-  return static_cast<size_t>(warps) * (static_cast<size_t>(n) * r + 2 * r * r + 32) +
-         (is_static ? static_cast<size_t>(n - 1) * r * r : 0);
+  return static_cast<size_t>(warps) * hmm_backward_warp_floats(n, r) + (is_static ? static_cast<size_t>(n - 1) * r * r : 0);
 }
 
 __global__ void circuit_hmm_backward_kernel(const CircuitBackwardArgs a_, const float* __restrict__ tables,
@@ -180,7 +182,7 @@ __global__ void circuit_hmm_backward_kernel(const CircuitBackwardArgs a_, const 
   const int rr = r * r;
   const bool is_static = table_stride == 0;
   float* acc = sm;                                                       // static only: [n-1, r, r]
-  float* mine = sm + (is_static ? (n - 1) * rr : 0) + static_cast<size_t>(wib) * (n * r + 2 * rr + 32);
+  float* mine = sm + (is_static ? (n - 1) * rr : 0) + static_cast<size_t>(wib) * hmm_backward_warp_floats(n, r);
   float* alphas = mine;                                                  // [n, r]
   float* tabs = alphas + n * r;
   float* cvec = tabs + 2 * rr;
@@ -262,6 +264,179 @@ __global__ void circuit_hmm_backward_kernel(const CircuitBackwardArgs a_, const 
         if (!is_static)
           for (int e = (len - 1) * rr + lane; e < (n - 1) * rr; e += r) a_.dsum[drow + r + e] = __float2bfloat16_rn(0.f);
       }
+    }
+    __syncwarp();
+  }
+  if (is_static) {
+    __syncthreads();
+    for (int e = threadIdx.x; e < (n - 1) * rr; e += blockDim.x) {
+      const float v = acc[e];
+      if (v != 0.f) atomicAdd(dT + e, v);
+    }
+  }
+}
+
+// ---------------------------------------------------------------- Eq. 6 through the HMM in one pass
+// The training loss is linear in the prefix log-marginals, L = sum_j coeff[w, j] log p_j, and for the HMM
+// p_j = sum_z exp(alpha_j[z]) is the forward message of step j summed over the state (later steps integrate to one). One
+// forward recursion therefore gives every prefix, and one reverse sweep gives the whole gradient: with
+// abar_i[z] = dL / d alpha_i[z] (plain numbers of either sign, bounded by sum_j |coeff_j|),
+//   abar_{n-1} = coeff_{n-1} softmax(alpha_{n-1}),
+//   prop_{i-1}[a] = sum_b exp(alpha_{i-1}[a] + logA_i[a][b] + G[i][b] - alpha_i[b]) abar_i[b]     (a conditional probability
+//   abar_{i-1}[a] = coeff_{i-1} softmax(alpha_{i-1})[a] + prop_{i-1}[a]                             times abar_i[b])
+// and dL/dG[i] = abar_i, dL/d logA_i[a][b] = the summand of prop_{i-1}[a]; through the row softmax of the transition
+// logits: summand - A_i[a][b] prop_{i-1}[a]; initial unit: abar_0 - omega sum_z abar_0[z]. Same streaming of the tables
+// and the same outputs as circuit_hmm_backward_kernel with accumulate == 0 (post fp32, dsum bf16, static dT by atomics).
+template <int R>
+__device__ __forceinline__ void row_grad_mult_vec(const float* row, const float* pc, const float* mult, float base, float gam,
+                                                  int lane, __nv_bfloat16* dst, float* acc_row) {
+  constexpr int Q = R / 4;
+  const float4* row4 = reinterpret_cast<const float4*>(row);
+  const float4* pc4 = reinterpret_cast<const float4*>(pc);
+  const float4* mu4 = reinterpret_cast<const float4*>(mult);
+#pragma unroll
+  for (int q = 0; q < Q; ++q) {
+    const int j = (q + lane) & (Q - 1);
+    const float4 a = row4[j];
+    const float4 p = pc4[j];
+    const float4 mu = mu4[j];
+    const float ox = __expf(base + a.x + p.x) * mu.x - __expf(a.x) * gam;
+    const float oy = __expf(base + a.y + p.y) * mu.y - __expf(a.y) * gam;
+    const float oz = __expf(base + a.z + p.z) * mu.z - __expf(a.z) * gam;
+    const float ow = __expf(base + a.w + p.w) * mu.w - __expf(a.w) * gam;
+    if (acc_row != nullptr) {
+      atomicAdd(acc_row + 4 * j, ox);
+      atomicAdd(acc_row + 4 * j + 1, oy);
+      atomicAdd(acc_row + 4 * j + 2, oz);
+      atomicAdd(acc_row + 4 * j + 3, ow);
+    } else {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(ox, oy);
+      __nv_bfloat162 hi = __floats2bfloat162_rn(oz, ow);
+      uint2 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(dst + 4 * j) = pk;
+    }
+  }
+}
+// Lane = row a of the table: out[b] = exp(base + row[b] + pc[b]) mult[b] - exp(row[b]) gam, to a bf16 row in global memory
+// or by atomic adds to an fp32 row in shared memory.
+__device__ __forceinline__ void row_grad_mult(const float* row, const float* pc, const float* mult, float base, float gam,
+                                              int lane, int r, __nv_bfloat16* dst, float* acc_row) {
+  switch (r) {
+    case 32: row_grad_mult_vec<32>(row, pc, mult, base, gam, lane, dst, acc_row); return;
+    case 16: row_grad_mult_vec<16>(row, pc, mult, base, gam, lane, dst, acc_row); return;
+    case 8: row_grad_mult_vec<8>(row, pc, mult, base, gam, lane, dst, acc_row); return;
+    case 4: row_grad_mult_vec<4>(row, pc, mult, base, gam, lane, dst, acc_row); return;
+    default: break;
+  }
+  for (int q = 0; q < r; ++q) {
+    int b = q + lane;                                   // start at column `lane`: fewer bank conflicts
+    if (b >= r) b -= r;
+    const float la = row[b];
+    const float o = __expf(base + la + pc[b]) * mult[b] - __expf(la) * gam;
+    if (acc_row != nullptr) atomicAdd(acc_row + b, o);
+    else dst[b] = __float2bfloat16_rn(o);
+  }
+}
+
+__global__ void circuit_hmm_loss_backward_kernel(const CircuitBackwardArgs a_, const float* __restrict__ coeff,
+                                                 const float* __restrict__ tables, int table_stride, float* __restrict__ dT,
+                                                 unsigned* work_counter) {
+  extern __shared__ __align__(16) float sm[];
+  const int lane = threadIdx.x & 31;
+  const int wib = threadIdx.x >> 5;
+  const int n = a_.n, r = a_.r;
+  const int rr = r * r;
+  const bool is_static = table_stride == 0;
+  float* acc = sm;                                                       // static only: [n-1, r, r]
+  float* mine = sm + (is_static ? (n - 1) * rr : 0) + static_cast<size_t>(wib) * hmm_backward_warp_floats(n, r);
+  float* alphas = mine;                                                  // [n, r]
+  float* tabs = alphas + n * r;
+  float* cvec = tabs + 2 * rr;                                           // G[i] - alpha_i (log domain)
+  float* dvec = cvec + 32;                                               // abar_i (plain)
+  const bool has = lane < r;
+  if (is_static) {
+    for (int e = threadIdx.x; e < (n - 1) * rr; e += blockDim.x) acc[e] = 0.f;
+    __syncthreads();
+  }
+  for (int w = next_window(work_counter, lane); w < a_.W; w = next_window(work_counter, lane)) {
+    const float* g = a_.G + static_cast<size_t>(w) * n * r;
+    const float* lw = a_.logw + static_cast<size_t>(w) * a_.sum_rows;
+    const float* tb = tables + static_cast<size_t>(w) * table_stride;
+    const float* cw = coeff + static_cast<size_t>(w) * n;
+    const int* tg = a_.targets + static_cast<size_t>(w) * n;
+    const size_t prow = static_cast<size_t>(w) * n * r;
+    const size_t drow = static_cast<size_t>(w) * a_.dsum_pitch;
+    // ---- forward, keeping every alpha_i
+    if (n > 1) warp_table_load_async(tabs, tb, rr, lane);
+    float alpha = has ? lw[lane] + g[lane] : -CUDART_INF_F;
+    if (has) alphas[lane] = alpha;
+    for (int i = 1; i < n; ++i) {
+      if (i + 1 < n) {
+        warp_table_load_async(tabs + (i & 1) * rr, tb + static_cast<size_t>(i) * rr, rr, lane);
+        cp_async_wait<1>();
+      } else {
+        cp_async_wait<0>();
+      }
+      __syncwarp();
+      const float* A = tabs + ((i - 1) & 1) * rr;
+      float m = alpha;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
+      cvec[lane] = has ? __expf(alpha - m) : 0.f;
+      __syncwarp();
+      if (has) {
+        const float s = hmm_matvec(cvec, A, lane, r);
+        alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : g[i * r + lane] + m + __logf(s);
+        alphas[i * r + lane] = alpha;
+      }
+      __syncwarp();
+    }
+    float lp = warp_lse(alpha, has);                                     // log p_{n-1}: the joint
+    if (lane == 0 && a_.out != nullptr) a_.out[w] = lp;
+    // ---- reverse sweep: tables in reverse order; the table of step n - 1 is still in its buffer
+    float abar = has ? cw[n - 1] * __expf(alpha - lp) : 0.f;
+    for (int i = n - 1; i >= 1; --i) {
+      if (i < n - 1) {
+        cp_async_wait<0>();
+        __syncwarp();
+      }
+      if (i - 1 >= 1) warp_table_load_async(tabs + (i & 1) * rr, tb + static_cast<size_t>(i - 2) * rr, rr, lane);
+      const float* A = tabs + ((i - 1) & 1) * rr;
+      const float al_i = has ? alphas[i * r + lane] : -CUDART_INF_F;
+      if (has) {
+        a_.post[prow + static_cast<size_t>(i) * r + lane] = tg[i] >= 0 ? abar : 0.f;
+        cvec[lane] = al_i == -CUDART_INF_F ? -CUDART_INF_F : g[i * r + lane] - al_i;
+        dvec[lane] = abar;
+      } else {
+        cvec[lane] = -CUDART_INF_F;
+        dvec[lane] = 0.f;
+      }
+      __syncwarp();
+      const float al = has ? alphas[(i - 1) * r + lane] : -CUDART_INF_F;
+      const float lp_prev = warp_lse(al, has);                           // log p_{i-1}
+      float prop = 0.f;
+      if (has) {
+        const float* row = A + lane * r;
+        for (int q = 0; q < r; ++q) {
+          int b = q + lane;
+          if (b >= r) b -= r;
+          prop += __expf(al + row[b] + cvec[b]) * dvec[b];
+        }
+        const size_t off = static_cast<size_t>(r) + static_cast<size_t>(i - 1) * rr + lane * r;
+        row_grad_mult(row, cvec, dvec, al, prop, lane, r, is_static ? nullptr : a_.dsum + drow + off,
+                      is_static ? acc + static_cast<size_t>(i - 1) * rr + lane * r : nullptr);
+      }
+      abar = has ? cw[i - 1] * __expf(al - lp_prev) + prop : 0.f;
+      __syncwarp();                                                      // cvec, dvec and the table buffer are free again
+    }
+    float total = abar;                                                  // sum_z abar_0[z]
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) total += __shfl_xor_sync(kFull, total, off);
+    if (has) {
+      a_.post[prow + lane] = tg[0] >= 0 ? abar : 0.f;
+      a_.dsum[drow + lane] = __float2bfloat16_rn(abar - __expf(lw[lane]) * total);
     }
     __syncwarp();
   }

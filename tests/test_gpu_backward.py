@@ -198,9 +198,13 @@ def test_backward_argument_checks():
 @pytest.mark.parametrize("family,n,r,v,d,N,L", [(I.CP, 4, 8, 320, 128, 3, 50), (I.CP, 2, 128, 16, 64, 5, 7),
                                                  (I.HMM, 8, 16, 64, 64, 5, 33), (I.HMM, 1, 4, 32, 64, 2, 9),
                                                  (I.HMM_CTX, 4, 8, 64, 64, 4, 40), (I.BTREE, 8, 8, 32, 64, 2, 140),
-                                                 (I.BTREE, 2, 4, 32, 64, 3, 11), (I.BTREE, 16, 16, 48, 64, 2, 40)])
+                                                 (I.BTREE, 2, 4, 32, 64, 3, 11), (I.BTREE, 16, 16, 48, 64, 2, 40),
+                                                 (I.HMM, 3, 1, 16, 64, 2, 5), (I.HMM, 16, 32, 32, 64, 2, 20),
+                                                 (I.HMM, 5, 2, 16, 64, 3, 7), (I.HMM_CTX, 3, 2, 16, 64, 3, 7),
+                                                 (I.HMM_CTX, 6, 32, 32, 64, 2, 17), (I.HMM_CTX, 1, 4, 32, 64, 2, 9)])
 def test_eq6_loss_backward_matches_oracle(family, n, r, v, d, N, L):
-    """The training loss of Eq. 6 and its gradients: one circuit backward pass per prefix length, accumulated, against
+    """The training loss of Eq. 6 and its gradients (mixture and tree: one circuit backward pass per prefix length,
+    accumulated; HMM: every prefix is a forward message, one reverse sweep), against
     reverse-mode differentiation of the definition in float64. Windows run past the end of their sequences (masked
     tails), one sequence has no valid byte in the last slot."""
     wl = I.make_workload(f"l6_{family}_{n}_{r}", I.HeadShape(family, n, r, v, d), N * L, seed=6000 + n + N + r, weight_std=0.25)
