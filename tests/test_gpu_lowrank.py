@@ -97,8 +97,9 @@ def test_head_on_composed_unembeddings_and_the_gradient_chain(family):
 
 
 def test_full_size_head_on_sampled_units():
-    """The shape the benchmark times (the mixture head with n=8, r=16, v=320, d=4096; rank 16): whole units of the composed tensor and of the adaptor
-    gradients, and one whole slot of the shared matrix's gradient, against the oracle run on those slices."""
+    """The shape the benchmark times (the mixture head with n=8, r=16, v=320, d=4096; rank 16): whole units of the
+    composed tensor and of the adaptor gradients, and one whole slot of the shared matrix's gradient, against the oracle
+    run on those slices."""
     n, r, v, d, k = 8, 16, 320, 4096, 16
     W, A, Bm = I.lowrank_parameters(n, r, v, d, k, seed=97)
     dU = I.lowrank_upstream_gradient(n, r, v, d, seed=98)
