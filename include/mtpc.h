@@ -299,8 +299,8 @@ int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags);
  *   mtpc_speculative_accept: [0] the acceptance kernel.
  *   mtpc_window_logprob_backward: [0] forward projection, [1] circuit backward, [2] gradient of the logits,
  *                        [3] transposes and the plain GEMMs.
- *   mtpc_window_loss_backward: [0] forward projection + prefix marginals + loss, [1] circuit backward (mixture and
- *                        tree: n passes, one per prefix length; HMM: one reverse sweep for all prefixes),
+ *   mtpc_window_loss_backward: [0] forward projection + prefix marginals + loss, [1] circuit backward (mixture:
+ *                        one pass per prefix length; tree: the same passes in one launch; HMM: one reverse sweep),
  *                        [2] and [3] as above.
  *   mtpc_draft_sample, mtpc_draft_sample_prefix:   P <= 128 positions: [0] one pass over all weights (logits of every unit),
  *                        [1] per-slot latent + byte draws and evidence, [2] circuit evaluation.

@@ -672,7 +672,7 @@ int circuit_backward_warps(const mtpc_head* h) {
   return 0;
 }
 
-// `loss_coeff` (HMM only): the weights [W, n] of the prefix log-marginals in Eq. 6; the whole gradient in one pass.
+// `loss_coeff` (HMM, tree): the weights [W, n] of the prefix log-marginals in Eq. 6; the whole gradient in one launch.
 int launch_circuit_backward(mtpc_head* h, CircuitBackwardArgs a, float* dT, cudaStream_t st,
                             const float* loss_coeff = nullptr) {
   const mtpc_config& c = h->cfg;
@@ -698,7 +698,7 @@ int launch_circuit_backward(mtpc_head* h, CircuitBackwardArgs a, float* dT, cuda
   } else if (c.family == MTPC_HMM) {
     circuit_hmm_backward_kernel<<<resident, threads, smem, st>>>(a, hmm_tables(h), hmm_table_stride(h), dT, counter);
   } else {
-    circuit_btree_backward_kernel<<<resident, threads, smem, st>>>(a, counter);
+    circuit_btree_backward_kernel<<<resident, threads, smem, st>>>(a, loss_coeff, counter);
   }
   h->launches++;
   return check_launch();
@@ -1121,19 +1121,24 @@ int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t
     bool bad = cudaMemsetAsync(post, 0, static_cast<size_t>(T) * c.n * c.r * 4, st) != cudaSuccess;
     bad |= cudaMemsetAsync(dsum_f32, 0, static_cast<size_t>(T) * L.sum_rows * 4, st) != cudaSuccess;
     if (bad) return MTPC_ERR_CUDA;
-    for (int j = 0; j < c.n; ++j) {
-      CircuitBackwardArgs a;
-      memset(&a, 0, sizeof(a));
-      a.targets = targets;
-      a.weight = coeff + j;
-      a.weight_stride = c.n;
-      a.post = post;
-      a.dsum_f32 = dsum_f32;
-      a.dsum_pitch = L.sum_rows;
-      a.len = j + 1;
-      a.accumulate = 1;
-      a.W = T;
-      if ((rc = launch_circuit_backward(head, a, dT_static, st)) != MTPC_OK) return rc;
+    CircuitBackwardArgs a;
+    memset(&a, 0, sizeof(a));
+    a.targets = targets;
+    a.post = post;
+    a.dsum_f32 = dsum_f32;
+    a.dsum_pitch = L.sum_rows;
+    a.accumulate = 1;
+    a.W = T;
+    if (c.family == MTPC_BTREE) {                 // every prefix length of a window by the same warp, back to back
+      a.len = c.n;
+      if ((rc = launch_circuit_backward(head, a, dT_static, st, coeff)) != MTPC_OK) return rc;
+    } else {
+      for (int j = 0; j < c.n; ++j) {               // mixture: one cheap pass per prefix length
+        a.weight = coeff + j;
+        a.weight_stride = c.n;
+        a.len = j + 1;
+        if ((rc = launch_circuit_backward(head, a, dT_static, st)) != MTPC_OK) return rc;
+      }
     }
     const size_t total = static_cast<size_t>(T) * L.sum_rows;
     const int blocks = static_cast<int>((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);

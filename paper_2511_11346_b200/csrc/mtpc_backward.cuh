@@ -460,11 +460,16 @@ __host__ __device__ inline size_t btree_backward_warp_floats(int n, int r) {
   return 3 * static_cast<size_t>(n - 1) * r + 2 * static_cast<size_t>(r) * r + 32;
 }
 
-__global__ void circuit_btree_backward_kernel(const CircuitBackwardArgs a_, unsigned* work_counter) {
+// With `loss_coeff` [W, n] (Eq. 6: L = sum_l coeff[w, l-1] log p_l over the prefix lengths l) the warp runs the pass of
+// every prefix length on its window back to back, accumulating (accumulate == 1): the window's tables and gradient rows
+// are then re-used out of L2 instead of being streamed from HBM once per prefix length.
+__global__ void circuit_btree_backward_kernel(const CircuitBackwardArgs a_, const float* __restrict__ loss_coeff,
+                                              unsigned* work_counter) {
   extern __shared__ __align__(16) float sm[];
   const int wib = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int n = a_.n, r = a_.r, len = a_.len;
+  const int n = a_.n, r = a_.r;
+  int len = a_.len;                                                      // prefix length of the current pass
   float* prod = sm + static_cast<size_t>(wib) * btree_backward_warp_floats(n, r);
   float* S = prod + (n - 1) * r;
   float* U = S + (n - 1) * r;
@@ -484,8 +489,11 @@ __global__ void circuit_btree_backward_kernel(const CircuitBackwardArgs a_, unsi
   for (int w = next_window(work_counter, lane); w < a_.W; w = next_window(work_counter, lane)) {
     const float* g = a_.G + static_cast<size_t>(w) * n * r;
     const float* lw = a_.logw + static_cast<size_t>(w) * a_.sum_rows;
-    const float wt = a_.weight[static_cast<size_t>(w) * a_.weight_stride];
     const size_t drow = static_cast<size_t>(w) * a_.dsum_pitch;
+    for (len = loss_coeff ? 1 : a_.len; len <= (loss_coeff ? n : a_.len); ++len) {
+    const float wt = loss_coeff ? loss_coeff[static_cast<size_t>(w) * n + len - 1]
+                                : a_.weight[static_cast<size_t>(w) * a_.weight_stride];
+    if (loss_coeff != nullptr && wt == 0.f) continue;                    // the same for every lane of the warp
     // ---- upward (tokens >= len are summed out: their input units output one)
     for (int j = n - 2; j >= first_leaf_node; --j) {
       const int t0 = 2 * (j - first_leaf_node);
@@ -579,6 +587,7 @@ __global__ void circuit_btree_backward_kernel(const CircuitBackwardArgs a_, unsi
       }
     }
     __syncwarp();
+    }                                                                    // prefix lengths
   }
 }
 
