@@ -44,12 +44,14 @@ struct CircuitBackwardArgs {
   int len, accumulate;
   int W, n, r, sum_rows;
 };
+// Accumulating passes add by reduction instructions (no value returned, so no wait for the round trip): every address
+// is only ever touched by one lane, in program order, so the sums keep their order and stay reproducible.
 __device__ __forceinline__ void put_post(const CircuitBackwardArgs& a, size_t idx, float v) {
-  if (a.accumulate) a.post[idx] += v;
+  if (a.accumulate) atomicAdd(a.post + idx, v);
   else a.post[idx] = v;
 }
 __device__ __forceinline__ void put_dsum(const CircuitBackwardArgs& a, size_t idx, float v) {
-  if (a.accumulate) a.dsum_f32[idx] += v;
+  if (a.accumulate) atomicAdd(a.dsum_f32 + idx, v);
   else a.dsum[idx] = __float2bfloat16_rn(v);
 }
 
@@ -123,11 +125,10 @@ __device__ __forceinline__ void row_grad_vec(const float* row, const float* pc, 
       atomicAdd(acc_row + 4 * j + 1, oy);
       atomicAdd(acc_row + 4 * j + 2, oz);
       atomicAdd(acc_row + 4 * j + 3, ow);
-    } else if (f32_row != nullptr) {                  // this lane owns the row: plain read-add-write
-      float4* d4 = reinterpret_cast<float4*>(f32_row + 4 * j);
-      float4 o = *d4;
-      o.x += ox; o.y += oy; o.z += oz; o.w += ow;
-      *d4 = o;
+    } else if (f32_row != nullptr) {
+      // this lane owns the row, so the additions to one address keep their order; issued as a reduction (no value comes
+      // back), the warp does not wait for the round trip to L2 that a read-add-write would cost
+      atomicAdd(reinterpret_cast<float4*>(f32_row + 4 * j), make_float4(ox, oy, oz, ow));
     } else {
       __nv_bfloat162 lo = __floats2bfloat162_rn(ox, oy);
       __nv_bfloat162 hi = __floats2bfloat162_rn(oz, ow);
@@ -152,7 +153,7 @@ __device__ __forceinline__ void row_grad(const float* row, const float* pc, floa
     const float la = row[b];
     const float o = wt * (__expf(base + la + pc[b]) - __expf(la) * gam);
     if (acc_row != nullptr) atomicAdd(acc_row + b, o);
-    else if (f32_row != nullptr) f32_row[b] += o;
+    else if (f32_row != nullptr) atomicAdd(f32_row + b, o);
     else dst[b] = __float2bfloat16_rn(o);
   }
 }
