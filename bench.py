@@ -34,7 +34,7 @@ UNIT = "positions/s"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one projection-kernel launch, from the ncu capture
 # summarised in profiles/ (captured on the full configuration). None = not captured.
-NCU_TRAFFIC_BYTES = {1: 931_400_000, 2: None, 3: None, 5: None, 6: None}   # configs[1]: mean of 933.4 and 929.4 MB (profiles/)
+NCU_TRAFFIC_BYTES = {1: 938_600_000, 2: None, 3: None, 5: None, 6: None}   # configs[1]: mean of 940.7 and 936.6 MB (profiles/)
 
 
 def workload_name(idx: int, wl) -> str:
