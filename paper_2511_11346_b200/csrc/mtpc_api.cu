@@ -630,9 +630,9 @@ int launch_transpose(mtpc_head* h, const void* src, void* dst, int rows, int col
   return check_launch();
 }
 
-// C[M, N] fp32 (pitch ldc) = A[M, K] B[N, K]^T (+ C): A, B bf16 with K contiguous and row pitches lda, ldb (elements).
+// C[M, N] fp32 (pitch ldc) = A[M, K] B[N, K]^T: A, B bf16 with K contiguous and row pitches lda, ldb (elements).
 int launch_plain_gemm(mtpc_head* h, const void* A, size_t lda, const void* Bm, size_t ldb, float* C, size_t ldc, int M,
-                      int N, int K, bool accumulate, cudaStream_t st) {
+                      int N, int K, cudaStream_t st) {
   if (M <= 0 || N <= 0 || K <= 0) return MTPC_OK;
   PlainGemmParams p;
   memset(&p, 0, sizeof(p));
@@ -647,7 +647,7 @@ int launch_plain_gemm(mtpc_head* h, const void* A, size_t lda, const void* Bm, s
   const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
   p.stages = (kSmemLimit - ctl) / p.stage_bytes;
   if (p.stages > kMaxStages) p.stages = kMaxStages;
-  p.accumulate = accumulate ? 1 : 0;
+  p.wide_stores = (reinterpret_cast<uintptr_t>(C) % 32 == 0 && ldc % 8 == 0) ? 1 : 0;
   p.C = C;
   p.ldc = ldc;
   p.status = at<unsigned>(h, h->L.off_status);
@@ -762,10 +762,10 @@ int backward_tail(mtpc_head* head, const BackwardLayout& B, uint8_t* bw, const v
   if (rc == MTPC_OK) rc = launch_transpose(head, dsum, dsum_t, T, L.sum_rows, B.Kd, B.Tpad, st);
   // d hidden [T, d] = [dlogit | dsum] [T, Nc + S r] [W_emit ; W_sum] [Nc + S r, d]
   if (rc == MTPC_OK)
-    rc = launch_plain_gemm(head, dlogit, B.Kd, wt, B.Kd, d_hidden, c.d, T, c.d, Nc + L.sum_rows, false, st);
+    rc = launch_plain_gemm(head, dlogit, B.Kd, wt, B.Kd, d_hidden, c.d, T, c.d, Nc + L.sum_rows, st);
   // dW_emit [Nc, d] = dlogit^T [Nc, T] hidden [T, d];  dW_sum [S r, d] = dsum^T [S r, T] hidden [T, d]
-  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dlogit_t, B.Tpad, ht, B.Tpad, dW_emit, c.d, Nc, c.d, T, false, st);
-  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dsum_t, B.Tpad, ht, B.Tpad, dW_sum, c.d, L.sum_rows, c.d, T, false, st);
+  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dlogit_t, B.Tpad, ht, B.Tpad, dW_emit, c.d, Nc, c.d, T, st);
+  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dsum_t, B.Tpad, ht, B.Tpad, dW_sum, c.d, L.sum_rows, c.d, T, st);
   pt.end();
   return rc;
 }

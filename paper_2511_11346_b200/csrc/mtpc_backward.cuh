@@ -712,7 +712,7 @@ __global__ void __launch_bounds__(256) logit_gradient_kernel(const LogitGradArgs
 }
 
 // ---------------------------------------------------------------- plain bf16 GEMM on the tcgen05 tensor cores
-// C[M, N] (fp32, row-major, pitch ldc) = A[M, K] B[N, K]^T (+ C if accumulate); A and B bf16, K contiguous (K-major), read
+// C[M, N] (fp32, row-major, pitch ldc) = A[M, K] B[N, K]^T; A and B bf16, K contiguous (K-major), read
 // through TMA descriptors with 64-element boxes (out-of-range rows and K columns read as zero). Same pipeline as the
 // projection kernel: one persistent CTA per SM, warp 0 TMA producer, warp 1 MMA issuer (M=128, N=256 tiles, two TMEM
 // slots), warps 2..5 epilogue (one thread per row, 16 fp32 columns per step).
@@ -722,7 +722,7 @@ struct PlainGemmParams {
   int M, N, kblocks;
   int m_tiles, n_tiles;
   int stages, stage_bytes;
-  int accumulate;
+  int wide_stores;       // C and ldc allow 32-byte stores
   float* C;
   size_t ldc;
   unsigned* status;
@@ -845,15 +845,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
         tmem_ld16(tcol + b * 16, x);
         const int col0 = nt * kPlainTileN + b * 16;
         if (row < p.M && col0 < p.N) {                 // N is a multiple of 16
-          float4* c4 = reinterpret_cast<float4*>(crow + col0);
+          if (p.wide_stores) {                         // 32-byte aligned rows: one full sector per store
+            st_global_v8(crow + col0, x);
+            st_global_v8(crow + col0 + 8, x + 8);
+          } else {
+            float4* c4 = reinterpret_cast<float4*>(crow + col0);
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            float4 v = make_float4(x[4 * q], x[4 * q + 1], x[4 * q + 2], x[4 * q + 3]);
-            if (p.accumulate) {
-              const float4 o = c4[q];
-              v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-            }
-            c4[q] = v;
+            for (int q = 0; q < 4; ++q) c4[q] = make_float4(x[4 * q], x[4 * q + 1], x[4 * q + 2], x[4 * q + 3]);
           }
         }
       }
