@@ -371,10 +371,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
                 for (int q = 0; q < 16; ++q) x[q] += p.sum_bias[gcol + b * 16 + q];
               }
               if (valid && gcol < p.sum_rows) {
-                float4* d4 = reinterpret_cast<float4*>(dst + gcol + b * 16);
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                  d4[q] = make_float4(x[4 * q] - lse, x[4 * q + 1] - lse, x[4 * q + 2] - lse, x[4 * q + 3] - lse);
+                for (int q = 0; q < 16; ++q) x[q] -= lse;
+                // r is a multiple of 16 here, so the rows of log omega (S r floats) and this offset are 64-byte aligned
+                st_global_v8(dst + gcol + b * 16, x);
+                st_global_v8(dst + gcol + b * 16 + 8, x + 8);
               }
             }
           }
