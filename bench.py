@@ -427,6 +427,7 @@ def run_ours(args):
 
     # CPU baseline: the oracle as it stands on a bounded sample of the same workload
     cpu_baseline = None
+    parity = None
     if not args.no_cpu_baseline:
         if args.ref_positions:
             sample = min(wl.T, args.ref_positions)
@@ -436,6 +437,13 @@ def run_ours(args):
         cpu_value, cpu_s = oracle_positions_per_s(wl, sample)
         cpu_baseline = {"value": cpu_value, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
                         "sample": f"first {sample} of {wl.T} positions, one pass, {cpu_s:.1f} s"}
+        # the timed launches' own output (device path and host-buffer path) against the oracle on the first positions
+        from oracle import mtpc_oracle as orc
+        k = min(wl.T, 256)
+        ref = orc.window_logprob(wl.shape.family, wl.hidden_q[:k], wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets[:k])
+        parity = {"positions": k, "tolerance": 2e-3,
+                  "max_abs_err_device_call": float(np.abs(out[:k].cpu().numpy().astype(np.float64) - ref).max()),
+                  "max_abs_err_host_call": float(np.abs(oh[:k].numpy().astype(np.float64) - ref).max())}
 
     backward = None
     if args.backward and world == 1:
@@ -496,6 +504,7 @@ def run_ours(args):
         "roofline": roofline,
         "kernels": kernels,
         "cpu_baseline": cpu_baseline,
+        "parity": parity,
         "device_status": status,
     }
     if backward is not None:
