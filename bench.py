@@ -428,7 +428,7 @@ def run_ours(args):
     # CPU baseline: the oracle as it stands on a bounded sample of the same workload
     cpu_baseline = None
     parity = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:          # rank 0 of a single-GPU run only
         if args.ref_positions:
             sample = min(wl.T, args.ref_positions)
         else:                                                                # about 15 s of CPU work, sized by a short probe
