@@ -32,9 +32,11 @@ from paper_2511_11346_b200 import replicas             # noqa: E402
 METRIC = "window_loglik_positions_per_s"
 UNIT = "positions/s"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one projection-kernel launch, from the ncu capture
-# summarised in profiles/ (captured on the full configuration). None = not captured.
-NCU_TRAFFIC_BYTES = {1: 938_600_000, 2: None, 3: None, 5: None, 6: None}   # configs[1]: mean of 940.7 and 936.6 MB (profiles/)
+# dram__bytes_read.sum + dram__bytes_write.sum of one projection-kernel launch, from the ncu captures
+# summarised in profiles/ (captured on the full configuration). None = not captured, or the kernel has changed since.
+NCU_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 5: None, 6: None}
+BURST_REGION_S = 1.0      # a timed loop shorter than this runs at boost clocks: its tensor roofline is the burst peak
+SUSTAINED_LOOP_S = 2.5    # length of the second, power-capped loop whose roofline is the sustained peak
 
 
 def workload_name(idx: int, wl) -> str:
@@ -60,7 +62,8 @@ def load_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
 
-    def __init__(self, index: int):
+    def __init__(self, index: int, period_s: float = 0.001):
+        self.period_s = period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thread = None
@@ -86,7 +89,7 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            time.sleep(0.02)
+            time.sleep(self.period_s)
 
     def start(self):
         if self.nv is not None:
@@ -144,8 +147,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(args.workload, wl),
-                   "sample": f"each step = the fp64 numpy oracle on the first {sample} of {wl.T} positions"},
+        "config": config_block(args.workload, wl, world),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"first {sample} of {wl.T} positions per step, {args.steps} steps"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -334,6 +336,146 @@ def measure_eq6_step(torch, dh, wl, hidden, targets, grads, steps: int):
                          "logit_gradient": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]}}
 
 
+CIRCUIT_KERNEL = {I.CP: "circuit_cp_kernel", I.HMM: "circuit_hmm_stream_kernel", I.BTREE: "circuit_btree_kernel",
+                  I.HMM_CTX: "circuit_hmm_stream_kernel (per-position tables)"}
+
+
+def config_block(idx: int, wl, world: int) -> dict:
+    """The `config` object of the JSON line; the same for this arm and for the reference arm."""
+    s = wl.shape
+    in_bytes = ((s.n * s.r * s.v + s.sum_rows) * s.d + wl.T * s.d) * 2
+    return {"workload": workload_name(idx, wl), "parallelism": f"replicas x{world} (no collective)",
+            "l2": f"inputs larger than L2: {in_bytes / 1e6:.0f} MB of weights and hidden states per step against 126 MB, "
+                  "no flush between steps",
+            "step": "one mtpc_window_logprob call: projection GEMM + fused epilogue, then circuit evaluation"}
+
+
+def timed_logprob_loop(torch, head, hidden, targets, out, steps: int, dev_index: int, sync_ranks: bool = False):
+    """`steps` back-to-back mtpc_window_logprob calls between two CUDA events on the launching stream, the SM clock
+    sampled meanwhile; per-kernel means from the library's event ring (recorded on the same stream in the same loop)."""
+    kept = min(steps, 4096)
+    head.mtpc_set_timing(kept)
+    launches0 = head.mtpc_launch_count()
+    sampler = ClockSampler(dev_index)
+    stream = torch.cuda.current_stream()
+    if sync_ranks:
+        replicas.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        head.mtpc_window_logprob(hidden, targets, out)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if sync_ranks:
+        replicas.barrier()
+    elapsed_s = e0.elapsed_time(e1) * 1e-3
+    phases = [head.mtpc_get_timing(i) for i in range(kept)]
+    head.mtpc_set_timing(0)
+    return {"elapsed_s": elapsed_s, "steps": steps, "gemm_ms": statistics.mean(p[0] for p in phases),
+            "circuit_ms": statistics.mean(p[1] for p in phases), "clocks": clocks, "timed_launches": kept,
+            "launches": head.mtpc_launch_count() - launches0}
+
+
+def tensor_roofline(flops: float, loop: dict, peaks: dict, peak_src: str) -> dict:
+    """Projection kernel against the measured cuBLAS bf16 peak that matches the loop it was timed in: the burst figure
+    for a loop shorter than BURST_REGION_S (boost clocks), the sustained one for a longer, power-capped loop."""
+    achieved = flops / (loop["gemm_ms"] * 1e-3) / 1e12
+    burst = loop["elapsed_s"] < BURST_REGION_S
+    key = "bf16_tflops" if burst else "bf16_tflops_sustained"
+    peak = peaks[key]
+    c = loop["clocks"]
+    return {"achieved": achieved, "peak": peak, "frac": achieved / peak,
+            "peak_source": f"{peak_src}: {key} ({'burst' if burst else 'sustained'} figure: the kernel was timed inside a "
+                           f"{loop['elapsed_s']:.3f} s loop of {loop['steps']} back-to-back steps)",
+            "avg_launch_ms": loop["gemm_ms"], "timed_launches": loop["timed_launches"], "loop_s": loop["elapsed_s"],
+            "sm_mhz_median": c["sm_mhz"], "clock_samples": c["samples"], "reasons": c["reasons"]}
+
+
+def sustained_steps(ms_per_step: float) -> int:
+    return int(max(20, min(4096, SUSTAINED_LOOP_S / (ms_per_step * 1e-3))))
+
+
+def circuit_roofline(wl, circuit_ms: float, peaks: dict) -> dict:
+    cbytes = circuit_bytes(wl)
+    gbs = cbytes / (circuit_ms * 1e-3) / 1e9
+    return {"kernel": CIRCUIT_KERNEL[wl.shape.family], "avg_ms": circuit_ms, "bound": "hbm", "algorithmic_bytes": cbytes,
+            "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"]}
+
+
+def oracle_parity(wl, out, k: int = 256) -> dict:
+    """The timed launches' own output against the fp64 oracle on the first k positions."""
+    from oracle import mtpc_oracle as orc
+    k = min(wl.T, k)
+    ref = orc.window_logprob(wl.shape.family, wl.hidden_q[:k], wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets[:k])
+    return {"positions": k, "tolerance": 2e-3,
+            "max_abs_err": float(np.abs(out[:k].cpu().numpy().astype(np.float64) - ref).max())}
+
+
+def measure_draft_whole_batch(torch, head, wl, hidden, steps: int) -> dict:
+    """configs[3]: draft one window per position over the whole batch (the many-position path)."""
+    s = wl.shape
+    u = torch.from_numpy(wl.uniforms).cuda()
+    W = wl.T * wl.wpp
+    ob = torch.empty((W, s.n), dtype=torch.int32, device="cuda")
+    ol = torch.empty(W, dtype=torch.float32, device="cuda")
+    for _ in range(3):
+        head.mtpc_draft_sample(hidden, wl.wpp, u, ob, ol)
+    torch.cuda.synchronize()
+    head.mtpc_set_timing(steps)
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    d0.record()
+    for _ in range(steps):
+        head.mtpc_draft_sample(hidden, wl.wpp, u, ob, ol)
+    d1.record()
+    torch.cuda.synchronize()
+    dms = d0.elapsed_time(d1) / steps
+    dph = [head.mtpc_get_timing(i) for i in range(steps)]
+    head.mtpc_set_timing(0)
+    return {"call": "mtpc_draft_sample over the whole batch", "windows": W, "ms_per_call": dms,
+            "windows_per_s": W / (dms * 1e-3),
+            "phase_ms": [statistics.mean(p[k] for p in dph) for k in range(len(dph[0]))],
+            "device_status": head.mtpc_get_status()}
+
+
+def measure_other_workload(torch, idx: int, dev_index: int, peaks: dict, peak_src: str, with_oracle: bool) -> dict:
+    """configs[2] / configs[3] measured like the headline workload, in shorter loops: a burst loop of a few hundred
+    milliseconds, a sustained loop, the circuit kernel against HBM and the parity of the timed output."""
+    from paper_2511_11346_b200.runner import DeviceHead
+    wl = I.config_workload(idx)
+    dh = DeviceHead(wl)
+    head = dh.head
+    hidden = dh.hidden_device()
+    targets = torch.from_numpy(wl.targets).cuda()
+    out = torch.empty(wl.T, dtype=torch.float32, device="cuda")
+    for _ in range(5):
+        head.mtpc_window_logprob(hidden, targets, out)
+    torch.cuda.synchronize()
+    flops = algorithmic_flops(wl)
+    burst = timed_logprob_loop(torch, head, hidden, targets, out, 60, dev_index)
+    ms = burst["elapsed_s"] / burst["steps"] * 1e3
+    sus = timed_logprob_loop(torch, head, hidden, targets, out, sustained_steps(ms), dev_index)
+    res = {"workload": workload_name(idx, wl), "positions_per_s": wl.T * burst["steps"] / burst["elapsed_s"],
+           "ms_per_step": ms, "steps": burst["steps"],
+           "positions_per_s_sustained": wl.T * sus["steps"] / sus["elapsed_s"],
+           "roofline": dict(bound="tensor", kernel="mtpc_gemm_kernel<logprob>", unit="TFLOP/s", flops_per_launch=flops,
+                            traffic=NCU_TRAFFIC_BYTES.get(idx), **tensor_roofline(flops, burst, peaks, peak_src)),
+           "roofline_sustained": tensor_roofline(flops, sus, peaks, peak_src),
+           "circuit_kernel": circuit_roofline(wl, burst["circuit_ms"], peaks),
+           "device_status": head.mtpc_get_status()}
+    if with_oracle:
+        res["parity"] = oracle_parity(wl, out)
+    if wl.wpp:
+        res["draft_whole_batch"] = measure_draft_whole_batch(torch, head, wl, hidden, 20)
+    res["gpu_launches"] = int(burst["launches"] + sus["launches"])
+    dh.close()
+    del dh, hidden, targets, out
+    torch.cuda.empty_cache()
+    return res
+
+
 def run_ours(args):
     import torch
     from paper_2511_11346_b200.runner import DeviceHead
@@ -352,35 +494,24 @@ def run_ours(args):
     hidden = dh.hidden_device()
     targets = torch.from_numpy(wl.targets).cuda()
     out = torch.empty(wl.T, dtype=torch.float32, device="cuda")
-    stream = torch.cuda.current_stream()
 
     # ---------------- device-resident throughput: K steps back to back, per-kernel events kept by the library
     for _ in range(args.warmup):
         head.mtpc_window_logprob(hidden, targets, out)
     torch.cuda.synchronize()
-    head.mtpc_set_timing(min(args.steps, 4096))
-    launches0 = head.mtpc_launch_count()
-    sampler = ClockSampler(dev_index)
-    replicas.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(args.steps):
-        head.mtpc_window_logprob(hidden, targets, out)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    replicas.barrier()
-    clocks = sampler.stop()
-    elapsed_s = replicas.max_over_ranks(e0.elapsed_time(e1) * 1e-3, device="cuda")
-    launches = head.mtpc_launch_count() - launches0
-    kept = min(args.steps, 4096)
-    phases = [head.mtpc_get_timing(i) for i in range(kept)]
-    gemm_ms = statistics.mean(p[0] for p in phases)
-    circuit_ms = statistics.mean(p[1] for p in phases)
-    head.mtpc_set_timing(0)
+    main = timed_logprob_loop(torch, head, hidden, targets, out, args.steps, dev_index, sync_ranks=True)
+    elapsed_s = replicas.max_over_ranks(main["elapsed_s"], device="cuda")
+    main["elapsed_s"] = elapsed_s
     status = head.mtpc_get_status()
     value = replicas.aggregate_throughput(wl.T, args.steps, world, elapsed_s)
+    gemm_ms, circuit_ms = main["gemm_ms"], main["circuit_ms"]
+
+    # ---------------- the same call in a loop long enough to sit under the power cap (sustained clocks)
+    sus = None
+    if not args.no_sustained:
+        sus = timed_logprob_loop(torch, head, hidden, targets, out, sustained_steps(elapsed_s / args.steps * 1e3), dev_index,
+                                 sync_ranks=True)
+    out_main = out.clone()
 
     # ---------------- end to end through the host-buffer entry point (pinned host memory, copies timed)
     hh = dh.hidden_host()
@@ -405,30 +536,28 @@ def run_ours(args):
 
     peaks, peak_src = load_peaks()
     flops = algorithmic_flops(wl)
-    achieved = flops / (gemm_ms * 1e-3) / 1e12
-    peak = peaks["bf16_tflops_sustained"]
-    traffic = NCU_TRAFFIC_BYTES.get(args.workload)
-    roofline = {"bound": "tensor", "kernel": "mtpc_gemm_kernel<logprob>", "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic,
-                "peak_source": f"{peak_src}: bf16_tflops_sustained (kernel timed inside a {elapsed_s:.2f} s back-to-back loop)",
-                "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "burst_peak": peaks["bf16_tflops"],
-                "flops_per_launch": flops, "avg_launch_ms": gemm_ms, "circuit_kernel_avg_ms": circuit_ms,
-                "timed_launches": kept}
-    cbytes = circuit_bytes(wl)
-    cgbs = cbytes / (circuit_ms * 1e-3) / 1e9
+    roofline = dict(bound="tensor", kernel="mtpc_gemm_kernel<logprob>", unit="TFLOP/s", flops_per_launch=flops,
+                    traffic=NCU_TRAFFIC_BYTES.get(args.workload), **tensor_roofline(flops, main, peaks, peak_src))
+    roofline["frac_of_burst_peak"] = roofline["achieved"] / peaks["bf16_tflops"]
+    roofline["frac_of_sustained_peak"] = roofline["achieved"] / peaks["bf16_tflops_sustained"]
+    roofline["circuit_kernel_avg_ms"] = circuit_ms
+    if sus is not None:
+        roofline["sustained"] = tensor_roofline(flops, sus, peaks, peak_src)
+        roofline["sustained"]["positions_per_s"] = wl.T * sus["steps"] / sus["elapsed_s"]
+    achieved = roofline["achieved"]
+    ck = circuit_roofline(wl, circuit_ms, peaks)
+    ck["share_of_step"] = circuit_ms / (gemm_ms + circuit_ms)
     kernels = [
         {"kernel": "mtpc_gemm_kernel<logprob>", "avg_ms": gemm_ms, "bound": "tensor", "achieved_tflops": achieved,
-         "frac_of_sustained_peak": achieved / peak, "share_of_step": gemm_ms / (gemm_ms + circuit_ms)},
-        {"kernel": {I.CP: "circuit_cp_kernel", I.HMM: "circuit_hmm_kernel", I.BTREE: "circuit_btree_kernel",
-                    I.HMM_CTX: "circuit_hmm_kernel (per-position tables)"}[s.family], "avg_ms": circuit_ms, "bound": "hbm",
-         "algorithmic_bytes": cbytes, "achieved_gbs": cgbs, "peak_gbs": peaks["hbm_gbs"],
-         "frac": cgbs / peaks["hbm_gbs"], "share_of_step": circuit_ms / (gemm_ms + circuit_ms)},
+         "frac": roofline["frac"], "share_of_step": gemm_ms / (gemm_ms + circuit_ms)},
+        ck,
     ]
 
     # CPU baseline: the oracle as it stands on a bounded sample of the same workload
     cpu_baseline = None
     parity = None
-    if not args.no_cpu_baseline and world == 1:          # rank 0 of a single-GPU run only
+    with_oracle = not args.no_cpu_baseline and world == 1          # rank 0 of a single-GPU run only
+    if with_oracle:
         if args.ref_positions:
             sample = min(wl.T, args.ref_positions)
         else:                                                                # about 15 s of CPU work, sized by a short probe
@@ -438,12 +567,9 @@ def run_ours(args):
         cpu_baseline = {"value": cpu_value, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
                         "sample": f"first {sample} of {wl.T} positions, one pass, {cpu_s:.1f} s"}
         # the timed launches' own output (device path and host-buffer path) against the oracle on the first positions
-        from oracle import mtpc_oracle as orc
-        k = min(wl.T, 256)
-        ref = orc.window_logprob(wl.shape.family, wl.hidden_q[:k], wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets[:k])
-        parity = {"positions": k, "tolerance": 2e-3,
-                  "max_abs_err_device_call": float(np.abs(out[:k].cpu().numpy().astype(np.float64) - ref).max()),
-                  "max_abs_err_host_call": float(np.abs(oh[:k].numpy().astype(np.float64) - ref).max())}
+        parity = oracle_parity(wl, out_main)
+        parity["max_abs_err_device_call"] = parity.pop("max_abs_err")
+        parity["max_abs_err_host_call"] = oracle_parity(wl, oh)["max_abs_err"]
 
     backward = None
     if args.backward and world == 1:
@@ -451,29 +577,19 @@ def run_ours(args):
 
     draft_many = None
     if wl.wpp and world == 1:       # configs[3]: draft one window per position over the whole batch (many-position path)
-        u = torch.from_numpy(wl.uniforms).cuda()
-        W = wl.T * wl.wpp
-        ob = torch.empty((W, s.n), dtype=torch.int32, device="cuda")
-        ol = torch.empty(W, dtype=torch.float32, device="cuda")
-        for _ in range(3):
-            head.mtpc_draft_sample(hidden, wl.wpp, u, ob, ol)
-        torch.cuda.synchronize()
-        dsteps = max(3, min(args.steps, 30))
-        head.mtpc_set_timing(dsteps)
-        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        d0.record()
-        for _ in range(dsteps):
-            head.mtpc_draft_sample(hidden, wl.wpp, u, ob, ol)
-        d1.record()
-        torch.cuda.synchronize()
-        dms = d0.elapsed_time(d1) / dsteps
-        dph = [head.mtpc_get_timing(i) for i in range(dsteps)]
-        head.mtpc_set_timing(0)
-        draft_many = {"call": "mtpc_draft_sample over the whole batch", "windows": W, "ms_per_call": dms,
-                      "windows_per_s": W / (dms * 1e-3),
-                      "phase_ms": [statistics.mean(p[k] for p in dph) for k in range(len(dph[0]))],
-                      "phases": "sum-unit GEMM, latent draws, GEMM + inverse-CDF epilogue, GEMM + gather epilogue on the "
-                                "drafted bytes, circuit", "device_status": head.mtpc_get_status()}
+        draft_many = measure_draft_whole_batch(torch, head, wl, hidden, max(3, min(args.steps, 30)))
+
+    launches = main["launches"] + (sus["launches"] if sus else 0)
+    dh.close()
+    del dh, hidden, targets, out
+    torch.cuda.empty_cache()
+
+    # ---------------- the other heads the throughput target names (default run: configs[2] and configs[3])
+    others = []
+    if world == 1 and args.workload == 1 and args.positions is None and not args.no_other_workloads:
+        for idx in (2, 3):
+            others.append(measure_other_workload(torch, idx, dev_index, peaks, peak_src, with_oracle))
+            launches += others[-1]["gpu_launches"]
 
     draft, sweep = None, None
     if not args.no_draft and world == 1:
@@ -484,29 +600,35 @@ def run_ours(args):
         else:                                   # "cp:8:64", "hmm:16:1", ...
             fam, n_, p_ = args.decode_cells.split(":")
             cells = [({"cp": I.CP, "hmm": I.HMM}[fam], int(n_), int(p_))]
-        sweep = [measure_decode_cell(torch, cell, steps=200, warmup=5)[0] for cell in cells]
+        sweep = []
+        for cell in cells:
+            res, cell_launches = measure_decode_cell(torch, cell, steps=200, warmup=5)
+            sweep.append(res)
+            launches += cell_launches
         draft = next((c for c in sweep if "decode_cp_n8_P64" in c["workload"]), sweep[0])
 
+    c = main["clocks"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": elapsed_s / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": workload_name(args.workload, wl), "parallelism": f"replicas x{world} (no collective)",
-                   "l2": "inputs larger than L2 (336 MB of weights + 67 MB of hidden states per step vs 126 MB)"
-                   if args.workload == 1 else "inputs larger than L2",
-                   "step": "one mtpc_window_logprob call: projection GEMM + fused epilogue, then circuit evaluation"},
-        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                   "samples": clocks["samples"]},
+        "config": config_block(args.workload, wl, world),
+        "clocks": {"sm_mhz": c["sm_mhz"], "sm_max_mhz": c["sm_max_mhz"], "reasons": c["reasons"], "samples": c["samples"],
+                   "region": f"the {args.steps} timed steps ({elapsed_s * 1e3:.1f} ms); the sustained loop has its own record "
+                             "under roofline.sustained"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3,
                 "call": "mtpc_window_logprob_host (pinned host buffers, copies inside the call)"},
-        "gpu_launches": int(launches),
+        "gpu_launches": int(main["launches"]),
+        "gpu_launches_all_loops": int(launches),
         "roofline": roofline,
         "kernels": kernels,
         "cpu_baseline": cpu_baseline,
         "parity": parity,
         "device_status": status,
     }
+    if others:
+        line["workloads"] = others
     if backward is not None:
         line["backward"] = backward
     if draft_many is not None:
@@ -534,6 +656,9 @@ def main():
                     help="draft measurement: 'all' twelve cells of the decode sweep, 'one' (CP n=8 P=64), or a single "
                          "cell as family:n:P, e.g. hmm:16:1")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiling runs)")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the second, seconds-long loop (profiling runs)")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="default run only: skip configs[2] and configs[3] after the headline workload")
     ap.add_argument("--backward", action="store_true", help="also time mtpc_window_logprob_backward on the workload")
     ap.add_argument("--positions", type=int, default=None,
                     help="override the number of positions (scaled-down profiler captures; not a bench value)")

@@ -60,7 +60,8 @@ enum {
 /* Bits of the device status word. */
 enum {
   MTPC_STATUS_BAD_TARGET = 1u,  /* a target >= v was seen; that window's log-prob is NaN               */
-  MTPC_STATUS_BAD_UNIFORM = 2u, /* a uniform outside [0,1) was seen; that draw returned -1             */
+  MTPC_STATUS_BAD_UNIFORM = 2u, /* a uniform outside [0,1) was seen; that draw returned -1 and the log-prob
+                                   (or the prefix log-marginals from that byte on) of its window is NaN */
   MTPC_STATUS_TIMEOUT = 4u      /* a bounded barrier wait expired; the outputs of that call are invalid */
 };
 
@@ -314,6 +315,17 @@ int mtpc_get_timing(mtpc_head* head, int32_t calls_back, float* out_ms, int32_t 
 int mtpc_launch_count(mtpc_head* head, uint64_t* out_count);
 
 /*
+ * Test hook, not part of the method (no passage of the paper): sets the time limit of the pipeline waits inside
+ * the tensor-core kernels of this head (waits on shared-memory barriers for a TMA copy, an MMA batch or a free
+ * accumulator). The default is 1 s, far beyond any healthy wait; limit_ns == 0 restores it. With a limit shorter
+ * than a memory round trip a healthy call gives up: the CTA that saw the wait expire raises MTPC_STATUS_TIMEOUT,
+ * waits (up to the fixed 1 s) for its copies and MMAs in flight, frees its tensor memory and returns, the
+ * outputs of that call are unspecified and the next mtpc_get_status returns MTPC_ERR_TIMEOUT. That is how the tests
+ * exercise the give-up path without withholding anything from a kernel. Host-side only; takes effect at the next call.
+ */
+int mtpc_debug_set_wait_limit_ns(mtpc_head* head, uint64_t limit_ns);
+
+/*
  * Window log-likelihood without any allocation (the paper has no counterpart: this is a packaging variant of
  * mtpc_window_logprob, same arithmetic, same kernels, same results).
  *
@@ -327,9 +339,10 @@ int mtpc_launch_count(mtpc_head* head, uint64_t* out_count);
  * holds those bytes until the process exits, whether or not this function is ever called. It calls no
  * cudaMalloc / cudaFree and no allocating library routine.
  *
- *   cfg        family, n, r, v, d as for mtpc_create_head; io_dtype must be MTPC_BF16 and flags 0
- *              (MTPC_ERR_UNSUPPORTED otherwise: fp32 inputs would need a rounded copy of the weights, contextual
- *              transitions a copy of their bias); max_positions, max_windows_per_pos are ignored.
+ *   cfg        family, n, r, v, v_valid, d as for mtpc_create_head (v_valid: a padded vocabulary, 0 = none);
+ *              io_dtype must be MTPC_BF16 and flags 0 (MTPC_ERR_UNSUPPORTED otherwise: fp32 inputs would need a
+ *              rounded copy of the weights, contextual transitions a copy of their bias); max_positions,
+ *              max_windows_per_pos are ignored.
  *   W_emit, W_sum, T_static, hidden, targets, out_logprob: dev, exactly as for mtpc_create_head and
  *              mtpc_window_logprob; all caller-owned, read or written only by the work this call enqueues.
  *   out_status dev uint32 or NULL: receives this call's MTPC_STATUS_* bits (stream-ordered, like the outputs).

@@ -23,11 +23,12 @@ EXPORTS = [
     "mtpc_launch_count", "mtpc_destroy", "mtpc_status_string", "mtpc_window_logprob_static",
     "mtpc_window_prefix_logprob", "mtpc_draft_sample_prefix", "mtpc_speculative_accept", "mtpc_window_loss",
     "mtpc_backward_workspace_bytes", "mtpc_window_logprob_backward", "mtpc_window_loss_backward",
-    "mtpc_lowrank_compose", "mtpc_lowrank_backward", "mtpc_update_parameters",
+    "mtpc_lowrank_compose", "mtpc_lowrank_backward", "mtpc_update_parameters", "mtpc_debug_set_wait_limit_ns",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 ERR_STATIC_SCRATCH = -7
 ERR_STATE = -8
+ERR_TIMEOUT = -6
 
 
 class MtpcConfig(ctypes.Structure):
@@ -77,6 +78,7 @@ def lib() -> ctypes.CDLL:
     L.mtpc_lowrank_compose.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]
     L.mtpc_lowrank_backward.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     L.mtpc_update_parameters.argtypes = [vp, vp, vp, vp, vp]
+    L.mtpc_debug_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
     L.mtpc_status_string.argtypes = [ctypes.c_int]
     L.mtpc_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -123,13 +125,13 @@ def mtpc_workspace_bytes(cfg: MtpcConfig) -> int:
 
 
 def mtpc_window_logprob_static(family: int, n: int, r: int, v: int, d: int, W_emit, W_sum, T_static, hidden, targets,
-                               out_logprob, out_status=None, stream=None) -> None:
+                               out_logprob, out_status=None, stream=None, v_valid: int = 0) -> None:
     """Window log-likelihood through the entry point that allocates nothing: no head, no workspace. For callers
     that cannot allocate device memory where they need the result (inside another component's memory pool, on
     a thread where a synchronising cudaMalloc is forbidden). The library's one static scratch array per device is
     shared by all such calls, so do not let two of them overlap on the GPU. bf16 tensors only; raises MtpcError
     with code ERR_STATIC_SCRATCH when the positions do not fit the array (split them over several calls)."""
-    cfg = MtpcConfig(family, n, r, v, d, MTPC_BF16, 1, 1, 0)
+    cfg = MtpcConfig(family, n, r, v, d, MTPC_BF16, 1, 1, 0, v_valid)
     T = hidden.shape[0]
     _check(lib().mtpc_window_logprob_static(ctypes.byref(cfg), _ptr(W_emit), _ptr(W_sum), _ptr(T_static), _ptr(hidden),
                                             _ptr(targets), T, _ptr(out_logprob), _ptr(out_status), _stream(stream)),
@@ -226,12 +228,18 @@ class MtpcHead:
                                             _ptr(out_bytes_host), _ptr(out_logprob_host), _stream(stream)),
                "mtpc_draft_sample_host")
 
-    def mtpc_get_status(self, stream=None) -> int:
+    def mtpc_get_status(self, stream=None, with_code: bool = False):
+        """The status bits raised since the last query (and cleared by it); with_code: (return code, bits), the code
+        being MTPC_ERR_TIMEOUT when a bounded wait gave up on the device."""
         flags = ctypes.c_uint32(0)
         code = lib().mtpc_get_status(self.handle, _stream(stream), ctypes.byref(flags))
-        if code not in (MTPC_OK, -6):
+        if code not in (MTPC_OK, ERR_TIMEOUT):
             raise MtpcError(code, "mtpc_get_status")
-        return flags.value
+        return (code, flags.value) if with_code else flags.value
+
+    def mtpc_debug_set_wait_limit_ns(self, limit_ns: int) -> None:
+        """Test hook: time limit of the pipeline waits inside the tensor-core kernels (0 = the default of 1 s)."""
+        _check(lib().mtpc_debug_set_wait_limit_ns(self.handle, int(limit_ns)), "mtpc_debug_set_wait_limit_ns")
 
     def mtpc_set_timing(self, ring: int) -> None:
         _check(lib().mtpc_set_timing(self.handle, int(ring)), "mtpc_set_timing")

@@ -215,6 +215,7 @@ struct mtpc_head {
   int* ring_phases;         // [ring] phases recorded by the call in that slot
   uint64_t calls;           // timed calls so far
   uint64_t launches;
+  uint64_t wait_limit_ns;   // limit of the pipeline waits inside the tcgen05 kernels (kWaitLimitNs; a test may shorten it)
 };
 
 namespace {
@@ -304,7 +305,7 @@ struct GradArgs {            // what the projection kernel keeps for the backwar
 
 int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int wpp, bool with_emit, bool with_sum,
                 const int* targets, const float* uniforms, int* out_bytes, cudaStream_t st,
-                const GradArgs* ga = nullptr) {
+                const GradArgs* ga = nullptr, bool targets_are_drafts = false) {
   if (rows <= 0 || (!with_emit && !with_sum)) return MTPC_OK;
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
@@ -322,6 +323,7 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   p.tm_sum = h->tm_sum;
   p.T = rows;
   p.m_tiles = (rows + kBlockM - 1) / kBlockM;
+  p.m_units = p.m_tiles;
   p.kblocks = c.d / kBlockK;
   {
     const size_t tile_bytes = static_cast<size_t>(kBlockM) * c.d * 2;
@@ -348,6 +350,7 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   p.stage_bytes = tl.stage_bytes;
   p.wpp = wpp;
   p.targets = targets;
+  p.missing_is_nan = targets_are_drafts ? 1 : 0;
   p.G = at<float>(h, L.off_G);
   p.logw = at<float>(h, L.off_logw);
   p.sum_bias = sum_bias(h);
@@ -355,12 +358,13 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   p.uniforms = uniforms;
   p.out_bytes = out_bytes;
   p.status = at<unsigned>(h, L.off_status);
+  p.wait_limit_ns = h->wait_limit_ns;
   const long long items = static_cast<long long>(p.m_tiles) * (p.num_groups + p.num_sum_tiles);
   const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
   if (mode == kModeLogprob)
-    mtpc_gemm_kernel<kModeLogprob><<<grid, kGemmThreads, tl.smem, st>>>(p);
+    mtpc_gemm_kernel<kModeLogprob, 1><<<grid, kGemmThreads, tl.smem, st>>>(p);
   else
-    mtpc_gemm_kernel<kModeSample><<<grid, kGemmThreads, tl.smem, st>>>(p);
+    mtpc_gemm_kernel<kModeSample, 1><<<grid, kGemmThreads, tl.smem, st>>>(p);
   h->launches++;
   return check_launch();
 }
@@ -406,24 +410,18 @@ int launch_circuit(mtpc_head* h, int W, int wpp, float* out, float* prefix, cuda
   return check_launch();
 }
 
-// Kernel attributes that depend on the head's shape; they are per function, so every head (and the static entry
-// point) sets them to what it needs or more.
-bool set_circuit_attributes(const mtpc_config& c) {
-  bool fail = false;
-  if (c.family == MTPC_HMM && hmm_stream_smem_bytes(c.r) > 48 * 1024)
-    fail |= cudaFuncSetAttribute(circuit_hmm_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(hmm_stream_smem_bytes(c.r))) != cudaSuccess;
-  if (c.family == MTPC_BTREE) {
-    const int plain = static_cast<int>(btree_smem_bytes(c.n, c.r, false));
-    const int pre = static_cast<int>(btree_smem_bytes(c.n, c.r, true));
-    if (plain > 48 * 1024)
-      fail |= cudaFuncSetAttribute(circuit_btree_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, plain) !=
-              cudaSuccess;
-    if (pre > 48 * 1024)
-      fail |= cudaFuncSetAttribute(circuit_btree_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, pre) !=
-              cudaSuccess;
-  }
-  return !fail;
+// cudaFuncAttributeMaxDynamicSharedMemorySize belongs to the function, not to a head or a call: whoever sets it last
+// wins. So every kernel that may ask for more than 48 KB gets the device's full limit, once and for all, and heads of
+// different shapes (or a head and the static entry point) cannot lower it under each other.
+template <typename K>
+bool allow_full_smem(K kernel) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) == cudaSuccess;
+}
+bool set_circuit_attributes() {
+  bool ok = allow_full_smem(circuit_hmm_stream_kernel);
+  ok &= allow_full_smem(circuit_btree_kernel<false>);
+  ok &= allow_full_smem(circuit_btree_kernel<true>);
+  return ok;
 }
 
 // Rows per emission tile of the few-position draft path: the height in [64, 128] (multiple of 8) that leaves the
@@ -476,6 +474,7 @@ int launch_decode_gemm(mtpc_head* h, const void* hidden_bf16, int P, cudaStream_
   p.logw = at<float>(h, L.off_logw);
   p.sum_bias = sum_bias(h);
   p.status = at<unsigned>(h, L.off_status);
+  p.wait_limit_ns = h->wait_limit_ns;
   const int tiles = p.emit_tiles + p.sum_tiles;
   const int grid = tiles < h->num_sms ? tiles : h->num_sms;
   mtpc_decode_gemm_kernel<<<grid, kGemmThreads, p.stages * p.stage_bytes + ctl, st>>>(p);
@@ -579,7 +578,8 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   if (rc != MTPC_OK) return rc;
   // 4. evidence of the drafted bytes under every unit -> 5. joint log-prob with the latents summed out
   pt.begin();
-  rc = launch_gemm(h, kModeLogprob, hb, P, wpp, true, false, out_bytes, nullptr, nullptr, st);
+  rc = launch_gemm(h, kModeLogprob, hb, P, wpp, true, false, out_bytes, nullptr, nullptr, st, nullptr,
+                   /*targets_are_drafts=*/true);
   pt.end();
   if (rc != MTPC_OK) return rc;
   pt.begin();
@@ -651,6 +651,7 @@ int launch_plain_gemm(mtpc_head* h, const void* A, size_t lda, const void* Bm, s
   p.C = C;
   p.ldc = ldc;
   p.status = at<unsigned>(h, h->L.off_status);
+  p.wait_limit_ns = h->wait_limit_ns;
   const long long items = static_cast<long long>(p.m_tiles) * p.n_tiles;
   const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
   plain_gemm_kernel<<<grid, kGemmThreads, p.stages * p.stage_bytes + ctl, st>>>(p);
@@ -704,26 +705,14 @@ int launch_circuit_backward(mtpc_head* h, CircuitBackwardArgs a, float* dT, cuda
   return check_launch();
 }
 
-// Shared-memory attributes of the circuit backward kernels (per function, set to what this head needs).
+// Shared-memory attributes of the circuit backward kernels (per function: always the full limit, see allow_full_smem).
 int set_backward_attributes(const mtpc_head* head) {
-  const mtpc_config& c = head->cfg;
-  if (c.family == MTPC_CP) return MTPC_OK;
-  const int warps = circuit_backward_warps(head);
-  if (warps == 0) return MTPC_ERR_UNSUPPORTED;
-  const size_t smem = circuit_backward_smem(head, warps);
-  bool fail = false;
-  if (smem > 48 * 1024) {
-    if (c.family == MTPC_HMM) {
-      fail |= cudaFuncSetAttribute(circuit_hmm_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   static_cast<int>(smem)) != cudaSuccess;
-      fail |= cudaFuncSetAttribute(circuit_hmm_loss_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   static_cast<int>(smem)) != cudaSuccess;
-    } else {
-      fail |= cudaFuncSetAttribute(circuit_btree_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   static_cast<int>(smem)) != cudaSuccess;
-    }
-  }
-  return fail ? MTPC_ERR_CUDA : MTPC_OK;
+  if (head->cfg.family == MTPC_CP) return MTPC_OK;
+  if (circuit_backward_warps(head) == 0) return MTPC_ERR_UNSUPPORTED;
+  bool ok = allow_full_smem(circuit_hmm_backward_kernel);
+  ok &= allow_full_smem(circuit_hmm_loss_backward_kernel);
+  ok &= allow_full_smem(circuit_btree_backward_kernel);
+  return ok ? MTPC_OK : MTPC_ERR_CUDA;
 }
 
 // Phases 3 and 4 of a backward call: the logit gradients (post, lse and the kept logits -> bf16, both orientations), the
@@ -864,12 +853,13 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   h->cfg = *cfg;
   h->L = L;
   h->ws = static_cast<uint8_t*>(workspace);
+  h->wait_limit_ns = kWaitLimitNs;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   bool fail = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess;
   // the attribute is per function, not per head: always ask for the full 227 KB so that heads do not undo each other
-  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
-  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeSample>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeSample, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
   fail |= cudaFuncSetAttribute(plain_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
           cudaSuccess;
@@ -877,13 +867,8 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
           cudaSuccess;
   fail |= cudaFuncSetAttribute(draft_slot_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                static_cast<int>(kSlotSmemLimit)) != cudaSuccess;
-  fail |= !set_circuit_attributes(*cfg);
-  {
-    const size_t smem = kAcceptWarps * accept_warp_floats(cfg->family, cfg->n, cfg->r, cfg->v) * sizeof(float);
-    if (L.can_draft && smem > 48 * 1024)
-      fail |= cudaFuncSetAttribute(spec_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   static_cast<int>(smem)) != cudaSuccess;
-  }
+  fail |= !set_circuit_attributes();
+  fail |= !allow_full_smem(spec_accept_kernel);
   fail |= cudaMemsetAsync(h->ws + L.off_status, 0, 256, st) != cudaSuccess;
   if (fail) { delete h; return MTPC_ERR_CUDA; }
 
@@ -1345,6 +1330,12 @@ int mtpc_get_timing(mtpc_head* head, int32_t calls_back, float* out_ms, int32_t 
   return MTPC_OK;
 }
 
+int mtpc_debug_set_wait_limit_ns(mtpc_head* head, uint64_t limit_ns) {
+  if (!head) return MTPC_ERR_NULL;
+  head->wait_limit_ns = limit_ns == 0 ? kWaitLimitNs : limit_ns;
+  return MTPC_OK;
+}
+
 int mtpc_launch_count(mtpc_head* head, uint64_t* out_count) {
   if (!head || !out_count) return MTPC_ERR_NULL;
   *out_count = head->launches;
@@ -1452,11 +1443,12 @@ extern "C" int mtpc_window_logprob_static(const mtpc_config* cfg, const void* W_
   h.ws = scratch;
   h.W_emit_bf16 = W_emit;
   h.W_sum_bf16 = W_sum;
+  h.wait_limit_ns = kWaitLimitNs;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   bool fail = cudaDeviceGetAttribute(&h.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess;
-  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeLogprob, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
-  fail |= !set_circuit_attributes(c);
+  fail |= !set_circuit_attributes();
   // The array keeps whatever the previous call left in it. Only the status word has to start at zero; G, log omega
   // and logA are fully rewritten for the rows this call reads.
   fail |= cudaMemsetAsync(scratch + L.off_status, 0, 256, st) != cudaSuccess;

@@ -726,6 +726,7 @@ struct PlainGemmParams {
   float* C;
   size_t ldc;
   unsigned* status;
+  uint64_t wait_limit_ns;   // limit of every pipeline wait
 };
 constexpr int kPlainTileN = 256;
 
@@ -754,6 +755,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
     }
     mbar_init(smem_u32(&ctl->drain), 1);
     ctl->abort = 0;
+    ctl->wait_limit_ns = p.wait_limit_ns;
     fence_mbar_init();
     tma_prefetch_desc(&p.tm_a);
     tma_prefetch_desc(&p.tm_b);
@@ -785,15 +787,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
           if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) {
-        for (int s = 0; s < p.stages; ++s)
-          if (issued_mask & (1u << s)) {
-            const uint32_t bar = smem_u32(&ctl->full[s]);
-            const uint32_t par = (phase_mask >> s) & 1u;
-            const uint64_t t0 = global_timer_ns();
-            while (!mbar_try_wait(bar, par) && global_timer_ns() - t0 < kWaitLimitNs) {}
-          }
-      }
+      // no copy may still be in flight when the CTA goes away (they have all landed unless some warp gave up)
+      for (int s = 0; s < p.stages; ++s)
+        if (issued_mask & (1u << s)) {
+          const uint32_t bar = smem_u32(&ctl->full[s]);
+          const uint32_t par = (phase_mask >> s) & 1u;
+          const uint64_t t0 = global_timer_ns();
+          while (!mbar_try_wait(bar, par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+        }
     }
     __syncwarp();
   } else if (warp == 1) {

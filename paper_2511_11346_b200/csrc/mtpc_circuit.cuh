@@ -368,6 +368,7 @@ __global__ void circuit_hmm_stream_kernel(const float* __restrict__ G, const flo
       const float* A = tabs + ((i - 1) % kHmmDepth) * rr;
       const float gi = has ? g[i * r + lane] : 0.f;
       float m = alpha;
+      const bool poisoned = __any_sync(kFull, alpha != alpha);   // NaN evidence (a target or a draw that was refused)
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
       // e[a] = exp(alpha[a] - m) goes through shared memory: every lane then reads four of them per request
@@ -377,6 +378,7 @@ __global__ void circuit_hmm_stream_kernel(const float* __restrict__ G, const flo
       if (has) {
         const float s = hmm_matvec(evec, A, lane, r);
         alpha = (m == -CUDART_INF_F) ? -CUDART_INF_F : gi + m + __logf(s);
+        if (poisoned) alpha = CUDART_NAN_F;              // the max above skips NaN: it would be lost when every state is NaN
       }
       __syncwarp();                                      // the buffers may be overwritten
     }

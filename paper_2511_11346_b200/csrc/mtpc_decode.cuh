@@ -46,6 +46,7 @@ struct DecodeParams {
   float* logw;           // [P, sum_rows]
   const float* sum_bias; // [sum_rows] or NULL: added to the sum-unit logits before their softmax
   unsigned* status;
+  uint64_t wait_limit_ns;   // limit of every pipeline wait
 };
 
 // Tile `t` of the launch: emission tiles first, then sum tiles.
@@ -91,6 +92,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_decode_gemm_kernel(const
     }
     mbar_init(smem_u32(&ctl->drain), 1);
     ctl->abort = 0;
+    ctl->wait_limit_ns = p.wait_limit_ns;
     fence_mbar_init();
     tma_prefetch_desc(&p.tm_h);
     tma_prefetch_desc(&p.tm_emit);
@@ -131,15 +133,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_decode_gemm_kernel(const
         }
         cur += ntiles;
       }
-      if (!ok) {
-        for (int s = 0; s < p.stages; ++s)
-          if (issued_mask & (1u << s)) {
-            const uint32_t bar = smem_u32(&ctl->full[s]);
-            const uint32_t par = (phase_mask >> s) & 1u;
-            const uint64_t t0 = global_timer_ns();
-            while (!mbar_try_wait(bar, par) && global_timer_ns() - t0 < kWaitLimitNs) {}
-          }
-      }
+      // no copy may still be in flight when the CTA goes away (they have all landed unless some warp gave up)
+      for (int s = 0; s < p.stages; ++s)
+        if (issued_mask & (1u << s)) {
+          const uint32_t bar = smem_u32(&ctl->full[s]);
+          const uint32_t par = (phase_mask >> s) & 1u;
+          const uint64_t t0 = global_timer_ns();
+          while (!mbar_try_wait(bar, par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+        }
     }
     __syncwarp();
   } else if (warp == 1) {
@@ -470,9 +471,10 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
       }
     }
     if (lane == 0) out_bytes[w * n + i] = byte;
-    // evidence of the drafted byte under every input unit of the slot (a missing byte is marginalised)
+    // evidence of the drafted byte under every input unit of the slot; a draw that was refused (byte -1) has none:
+    // NaN, so that the window's log-prob comes out as NaN rather than as the joint of its other bytes
     for (int k = lane; k < r; k += 32)
-      G[(w * n + i) * r + k] = byte < 0 ? 0.f : row[static_cast<size_t>(k) * v + byte] - unit_lse[k];
+      G[(w * n + i) * r + k] = byte < 0 ? CUDART_NAN_F : row[static_cast<size_t>(k) * v + byte] - unit_lse[k];
   }
 }
 

@@ -34,7 +34,8 @@ constexpr int kMaxStages = 8;
 constexpr int kMaxSlots = 16;
 constexpr int kTmemCols = 512;
 constexpr int kGemmThreads = 192;
-constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per barrier wait
+constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per barrier wait (the default, and always the limit of the drain waits)
+constexpr uint64_t kAbortSettleNs = 200ull * 1000ull;            // 0.2 ms: far longer than any copy or MMA in flight takes
 constexpr int kABytes = kBlockM * kBlockK * 2;                   // 16 KB
 constexpr uint32_t kStatusBadTarget = 1u, kStatusBadUniform = 2u, kStatusTimeout = 4u;
 
@@ -45,7 +46,8 @@ struct GemmParams {
   CUtensorMap tm_emit;   // W_emit  [n*r*v, d]    box 64 x tile_cols
   CUtensorMap tm_sum;    // W_sum   [S*r, d]      box 64 x sum_cols
   int T, m_tiles, kblocks;
-  int m_block;                       // m-tiles per rasterisation block (see tile_coord)
+  int m_units;                       // M work units: m-tiles, or pairs of m-tiles when two CTAs share every MMA
+  int m_block;                       // M work units per rasterisation block (see tile_coord)
   int n, r, v;
   int vv;                            // symbols that exist (<= v, > v - 16): the columns [vv, v) of every unit are padding
   int emit_units;                    // n * r
@@ -58,6 +60,7 @@ struct GemmParams {
   int stages, stage_bytes;
   int wpp;                           // windows (target rows) per position
   const int* targets;                // [T*wpp, n]
+  int missing_is_nan;                // a negative target is a refused draw (G = NaN), not a byte to sum out (G = 0)
   float* G;                          // [T*wpp, n, r]   log phi at the target
   float* logw;                       // [T, S*r]        log-softmaxed sum-unit weights
   const float* sum_bias;             // [S*r] or NULL   added to the sum-unit logits before their softmax
@@ -68,6 +71,7 @@ struct GemmParams {
   const float* uniforms;             // [T*wpp, 2n]
   int* out_bytes;                    // [T*wpp, n]
   unsigned* status;
+  uint64_t wait_limit_ns;            // limit of every pipeline wait (kWaitLimitNs unless a test shortened it)
 };
 
 struct GemmControl {
@@ -76,6 +80,7 @@ struct GemmControl {
   uint64_t tfull[kMaxSlots];
   uint64_t tempty[kMaxSlots];
   uint64_t drain;
+  uint64_t wait_limit_ns;
   uint32_t tmem_base;
   volatile int abort;
 };
@@ -101,7 +106,7 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Gemm
     if (mbar_try_wait(bar, parity)) return true;
     if ((++it & 63u) == 0) {
       if (ctl->abort) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > ctl->wait_limit_ns) {
         ctl->abort = 1;
         atomicOr(status, kStatusTimeout);
         return false;
@@ -120,27 +125,28 @@ __device__ __forceinline__ bool bounded_wait_warp(uint32_t bar, uint32_t parity,
 struct TileCoord {
   int mt, is_sum, ntiles, cols, brow0, unit0, nunits;
 };
-// Work items. Emission items come first, in blocks of m_block m-tiles: inside a block the m-tile runs fastest and
+// Work items (c.mt counts M work units: m-tiles, or pairs of m-tiles in the CTA-pair kernel). Emission items come
+// first, in blocks of m_block units: inside a block the unit runs fastest and
 // the group next, so the CTAs that run at the same time share a few groups' weights through L2 while the block's
 // hidden states (m_block x 128 rows) stay L2-resident for every group; a block is finished before the next one
 // starts, so the weights are streamed from HBM once per block and the hidden states once. Sum items follow,
 // m-tile fastest.
 __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int item) {
   TileCoord c;
-  const int emit_items = p.num_groups * p.m_tiles;
+  const int emit_items = p.num_groups * p.m_units;
   int g;
   if (item < emit_items) {
     const int per_block = p.m_block * p.num_groups;
     const int blk = item / per_block;
     const int rem = item - blk * per_block;
     const int m0 = blk * p.m_block;
-    const int mcount = min(p.m_block, p.m_tiles - m0);   // only the last block can be short
+    const int mcount = min(p.m_block, p.m_units - m0);   // only the last block can be short
     g = rem / mcount;
     c.mt = m0 + (rem - g * mcount);
   } else {
     const int rem = item - emit_items;
-    g = p.num_groups + rem / p.m_tiles;
-    c.mt = rem % p.m_tiles;
+    g = p.num_groups + rem / p.m_units;
+    c.mt = rem % p.m_units;
   }
   c.is_sum = g >= p.num_groups;
   if (c.is_sum) {
@@ -187,7 +193,14 @@ __device__ __forceinline__ void sum_groups_in_batch(const float (&x)[16], float*
   }
 }
 
-template <int MODE>
+// CTAS = 1: every CTA works alone (cta_group::1). CTAS = 2: the kernel is launched in clusters of two CTAs that share
+// every MMA (cta_group::2, M = 256): the pair covers 256 positions, each CTA stages its own 128 rows of h and HALF of the
+// weight tile (the leader, cluster rank 0, the first half of the tile's columns), so a CTA moves a third less data from
+// L2 to shared memory per MMA; the leader's warp 1 issues the MMAs for both, each CTA's epilogue warps read their own
+// 128 accumulator rows. Barriers: full[s] lives in the leader and counts the bytes of both CTAs' copies; empty[s] and
+// tfull[slot] exist in both CTAs and are signalled together by the leader's commits; tempty[slot] lives in the leader
+// and collects the arrivals of both CTAs' epilogue warps.
+template <int MODE, int CTAS>
 __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -197,7 +210,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int num_items = (p.num_groups + p.num_sum_tiles) * p.m_tiles;
+  const int num_items = (p.num_groups + p.num_sum_tiles) * p.m_units;
+  const uint32_t cta_rank = CTAS == 2 ? cluster_cta_rank() : 0u;      // 0 = the pair's leader
+  const int first_item = CTAS == 2 ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int item_step = CTAS == 2 ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -206,21 +222,28 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
     }
     for (int s = 0; s < p.num_slots; ++s) {
       mbar_init(smem_u32(&ctl->tfull[s]), 1);
-      mbar_init(smem_u32(&ctl->tempty[s]), 4);
+      mbar_init(smem_u32(&ctl->tempty[s]), 4 * CTAS);
     }
     mbar_init(smem_u32(&ctl->drain), 1);
     ctl->abort = 0;
+    ctl->wait_limit_ns = p.wait_limit_ns;
     fence_mbar_init();
     tma_prefetch_desc(&p.tm_a);
     tma_prefetch_desc(&p.tm_emit);
     tma_prefetch_desc(&p.tm_sum);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
-    tmem_relinquish();
+    if (CTAS == 2) {
+      tmem_alloc_pair(smem_u32(&ctl->tmem_base), kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
+      tmem_relinquish();
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();   // the peer's barriers are initialised before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
 
@@ -229,25 +252,37 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+      for (int item = first_item; item < num_items && ok; item += item_step) {
         const TileCoord tc = tile_coord(p, item);
         const CUtensorMap* tmb = tc.is_sum ? &p.tm_sum : &p.tm_emit;
-        const uint32_t bytes = kABytes + tc.cols * (kBlockK * 2);
+        const int brows = tc.cols / CTAS;                                 // weight rows this CTA stages per tile
+        const uint32_t bytes = CTAS * (kABytes + brows * (kBlockK * 2));   // of both CTAs' copies when paired
+        const int arow = (tc.mt * CTAS + static_cast<int>(cta_rank)) * kBlockM;
         for (int t = 0; t < tc.ntiles && ok; ++t) {
           for (int kb = 0; kb < p.kblocks; ++kb) {
             if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
-            const uint32_t full = smem_u32(&ctl->full[stage]);
             const uint32_t a_dst = tiles_addr + stage * p.stage_bytes;
-            mbar_arrive_expect_tx(full, bytes);
-            tma_load_2d(a_dst, &p.tm_a, full, kb * kBlockK, tc.mt * kBlockM);
-            tma_load_2d(a_dst + kABytes, tmb, full, kb * kBlockK, tc.brow0 + t * tc.cols);
+            const int brow = tc.brow0 + t * tc.cols + static_cast<int>(cta_rank) * brows;
+            if (CTAS == 2) {
+              const uint32_t full = cluster_map_shared(smem_u32(&ctl->full[stage]), 0);   // the leader's barrier
+              if (cta_rank == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[stage]), bytes);
+              tma_load_2d_pair(a_dst, &p.tm_a, full, kb * kBlockK, arow);
+              tma_load_2d_pair(a_dst + kABytes, tmb, full, kb * kBlockK, brow);
+            } else {
+              const uint32_t full = smem_u32(&ctl->full[stage]);
+              mbar_arrive_expect_tx(full, bytes);
+              tma_load_2d(a_dst, &p.tm_a, full, kb * kBlockK, arow);
+              tma_load_2d(a_dst + kABytes, tmb, full, kb * kBlockK, brow);
+            }
             issued_mask |= 1u << stage;
             phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
             if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
           }
         }
       }
-      if (!ok) {   // give the copies still in flight a bounded chance to land before the CTA goes away
+      // The CTA must not go away with copies in flight. After a full run they have all landed already (the MMA warp
+      // consumed them); after an abort, by this warp or by another one, give them a bounded chance to land.
+      if (CTAS == 1 || cta_rank == 0) {
         for (int s = 0; s < p.stages; ++s)
           if (issued_mask & (1u << s)) {
             const uint32_t bar = smem_u32(&ctl->full[s]);
@@ -260,12 +295,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && cta_rank == 0) {
       uint32_t stage = 0, phase = 0, use = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+      for (int item = first_item; item < num_items && ok; item += item_step) {
         const TileCoord tc = tile_coord(p, item);
-        const uint32_t idesc = umma_idesc_bf16(kBlockM, tc.cols);
+        const uint32_t idesc = umma_idesc_bf16(kBlockM * CTAS, tc.cols);
         for (int t = 0; t < tc.ntiles && ok; ++t, ++use) {
           const uint32_t slot = use % p.num_slots;
           if (!bounded_wait(smem_u32(&ctl->tempty[slot]), ((use / p.num_slots) & 1u) ^ 1u, ctl, p.status)) {
@@ -281,17 +316,22 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
             const uint64_t a_desc = umma_smem_desc_sw128(a_addr);
             const uint64_t b_desc = umma_smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
-            for (int kk = 0; kk < kBlockK / 16; ++kk)   // +32 bytes per K=16 step inside the swizzled row
-              umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
-            umma_commit(smem_u32(&ctl->empty[stage]));
+            for (int kk = 0; kk < kBlockK / 16; ++kk) {   // +32 bytes per K=16 step inside the swizzled row
+              if (CTAS == 2) umma_bf16_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+              else umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+            }
+            if (CTAS == 2) umma_commit_pair(smem_u32(&ctl->empty[stage]));   // frees the stage in both CTAs
+            else umma_commit(smem_u32(&ctl->empty[stage]));
             if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
           }
           if (!ok) break;
-          umma_commit(smem_u32(&ctl->tfull[slot]));
+          if (CTAS == 2) umma_commit_pair(smem_u32(&ctl->tfull[slot]));      // the accumulators of both CTAs are ready
+          else umma_commit(smem_u32(&ctl->tfull[slot]));
         }
       }
       if (!ok) {   // wait (bounded) for the MMAs already issued before TMEM is freed
-        umma_commit(smem_u32(&ctl->drain));
+        if (CTAS == 2) umma_commit_pair(smem_u32(&ctl->drain));
+        else umma_commit(smem_u32(&ctl->drain));
         const uint64_t t0 = global_timer_ns();
         while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
       }
@@ -303,9 +343,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     uint32_t use = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+    // a drained accumulator slot is handed back to the MMA issuer: the leader's, also from the peer's epilogue warps
+    auto release_slot = [&](uint32_t slot) {
+      if (CTAS == 2) mbar_arrive_cluster(cluster_map_shared(smem_u32(&ctl->tempty[slot]), 0));
+      else mbar_arrive(smem_u32(&ctl->tempty[slot]));
+    };
+    for (int item = first_item; item < num_items && ok; item += item_step) {
       const TileCoord tc = tile_coord(p, item);
-      const int row = tc.mt * kBlockM + quarter * 32 + lane;
+      const int row = (tc.mt * CTAS + static_cast<int>(cta_rank)) * kBlockM + quarter * 32 + lane;
       const bool valid = row < p.T;
       const int nbatch = tc.cols / 16;
 
@@ -382,7 +427,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&ctl->tempty[slot]));
+        if (lane == 0) release_slot(slot);
         use += 1;
         continue;
       }
@@ -453,7 +498,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
                   const int tj = (p.wpp == 1) ? tgt : p.targets[(wrow0 + j) * p.n + slot_i];
                   float* g = p.G + ((wrow0 + j) * p.n + slot_i) * p.r + k;
                   if (tj < 0) {
-                    *g = 0.f;                                  // marginalised byte: the input unit sums to 1
+                    *g = p.missing_is_nan ? CUDART_NAN_F : 0.f;   // marginalised byte: the input unit sums to 1
                   } else if (tj >= p.vv) {
                     *g = CUDART_NAN_F;
                     atomicOr(p.status, kStatusBadTarget);
@@ -474,7 +519,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
           }
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&ctl->tempty[slot]));
+          if (lane == 0) release_slot(slot);
         }
         if (!ok) break;
       } else {
@@ -554,7 +599,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
         tc_fence_before();
         __syncwarp();
         if (lane == 0)
-          for (int c = 0; c < tc.ntiles; ++c) mbar_arrive(smem_u32(&ctl->tempty[(use + c) % p.num_slots]));
+          for (int c = 0; c < tc.ntiles; ++c) release_slot((use + c) % p.num_slots);
         use += tc.ntiles;
       }
     }
@@ -562,9 +607,20 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
 
   tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) {
+    // A CTA of a pair may leave only when its partner no longer needs it (MMAs read both CTAs' shared memory and write
+    // both CTAs' tensor memory; copies and arrivals cross over). After a run in which some wait gave up, first let
+    // whatever is still in flight land: the peer's copies are counted on the leader's barriers and cannot be awaited here.
+    if (ctl->abort && threadIdx.x == 0) {
+      const uint64_t t0 = global_timer_ns();
+      while (global_timer_ns() - t0 < kAbortSettleNs) {}
+    }
+    cluster_sync_all();
+  }
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (CTAS == 2) tmem_dealloc_pair(tmem_base, kTmemCols);
+    else tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 

@@ -168,12 +168,29 @@ def test_bad_uniform_is_flagged_not_sampled():
     u[3, 2 + 1] = 1.0                 # byte draw of slot 1, window 3
     u[7, 0] = -0.25                   # latent draw of window 7
     dh = DeviceHead(wl)
-    out_bytes, _ = dh.draft_sample(uniforms=torch.from_numpy(u).cuda())
+    out_bytes, out_lp = dh.draft_sample(uniforms=torch.from_numpy(u).cuda())
     assert dh.head.mtpc_get_status() == B.STATUS_BAD_UNIFORM
-    gb = out_bytes.cpu().numpy()
+    gb, gl = out_bytes.cpu().numpy(), out_lp.cpu().numpy()
     assert gb[3, 1] == -1 and gb[3, 0] >= 0
     assert (gb[7] == -1).all()
     assert (np.delete(gb, [3, 7], axis=0) >= 0).all()
+    # a window with a refused draw has no log-prob (NaN), the others are untouched
+    assert np.isnan(gl[3]) and np.isnan(gl[7]) and np.isfinite(np.delete(gl, [3, 7])).all()
+    dh.close()
+
+
+def test_bad_uniform_many_position_path_gives_nan_logprob():
+    shape = I.HeadShape(I.HMM, 4, 8, 64, 64)
+    wl = I.make_workload("badu_many", shape, 150, seed=16, wpp=1, weight_std=0.3)     # 150 > 128 positions
+    u = wl.uniforms.copy()
+    u[20, 4 + 2] = 1.5                # byte draw of slot 2, window 20
+    u[140, 1] = float("nan")          # latent draw of window 140
+    dh = DeviceHead(wl)
+    out_bytes, out_lp = dh.draft_sample(uniforms=torch.from_numpy(u).cuda())
+    assert dh.head.mtpc_get_status() == B.STATUS_BAD_UNIFORM
+    gb, gl = out_bytes.cpu().numpy(), out_lp.cpu().numpy()
+    assert gb[20, 2] == -1 and (gb[140] == -1).all()
+    assert np.isnan(gl[20]) and np.isnan(gl[140]) and np.isfinite(np.delete(gl, [20, 140])).all()
     dh.close()
 
 

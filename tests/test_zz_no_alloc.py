@@ -2,8 +2,8 @@
 running inside another component's memory pool, or on a thread where a synchronising cudaMalloc is not
 allowed). It takes no head and no workspace: its scratch is a static array inside the library.
 
-The check: through the C ABI, its output must equal what mtpc_window_logprob gives on the same inputs, within the
-log-prob tolerance of the parity tests, on two calls in a row - the second on fewer positions and other targets,
+The check: through the C ABI, its output must equal what mtpc_window_logprob gives on the same inputs (and what the
+fp64 oracle gives), within the log-prob tolerance of the parity tests, on two calls in a row - the second on fewer positions and other targets,
 so that whatever the first call left in the shared array would show if it were read. This file is collected last
 on purpose: a run that stops at the first failure has then already run every other test."""
 import ctypes
@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import mtpc_oracle as orc
 from paper_2511_11346_b200 import binding as B
 from paper_2511_11346_b200 import inputs as I
 from paper_2511_11346_b200.runner import DeviceHead
@@ -26,7 +27,7 @@ def static_logprob(dh, hidden, targets):
     out = torch.full((hidden.shape[0],), float("nan"), dtype=torch.float32, device="cuda")
     status = torch.full((1,), 99, dtype=torch.int32, device="cuda")
     B.mtpc_window_logprob_static(s.family, s.n, s.r, s.v, s.d, dh.W_emit, dh.W_sum, dh.T_static, hidden, targets, out,
-                                 status)
+                                 status, v_valid=s.v_valid)
     torch.cuda.synchronize()
     return out.cpu().numpy(), int(status.item())
 
@@ -44,6 +45,8 @@ def test_static_scratch_call_matches_the_workspace_call_twice_in_a_row(family, n
     got, status = static_logprob(dh, hidden, targets)
     assert status == 0
     assert np.abs(got - want).max() <= LOGPROB_TOL
+    ref = orc.window_logprob(family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets)
+    assert np.abs(got - ref).max() <= LOGPROB_TOL
 
     # second call: a ragged subset of the positions, shuffled targets with one byte marginalised and one bad
     T2 = T - 37
@@ -59,6 +62,24 @@ def test_static_scratch_call_matches_the_workspace_call_twice_in_a_row(family, n
     assert np.isnan(got2[5]) and np.isnan(want2[5])
     keep = np.arange(T2) != 5
     assert np.abs(got2[keep] - want2[keep]).max() <= LOGPROB_TOL
+    ref2 = orc.window_logprob(family, wl.hidden_q[:T2][keep], wl.W_emit_q, wl.W_sum_q, wl.T_static, t2[keep])
+    assert np.abs(got2[keep] - ref2).max() <= LOGPROB_TOL
+    dh.close()
+
+
+def test_static_scratch_call_with_a_padded_vocabulary():
+    # 44 symbols stored as 48 columns: the padding rows of W_emit hold large values that must carry no mass
+    shape = I.HeadShape(I.CP, 3, 4, 48, 128, I.BF16, v_valid=44)
+    wl = I.make_workload("noalloc_pad", shape, 140, seed=931, weight_std=0.25)
+    dh = DeviceHead(wl)
+    hidden = dh.hidden_device()
+    targets = torch.from_numpy(wl.targets).cuda()
+    want = dh.window_logprob(hidden, targets).cpu().numpy()
+    ref = orc.window_logprob(I.CP, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.targets)
+    for _ in range(2):
+        got, status = static_logprob(dh, hidden, targets)
+        assert status == 0
+        assert np.abs(got - want).max() <= LOGPROB_TOL and np.abs(got - ref).max() <= LOGPROB_TOL
     dh.close()
 
 
