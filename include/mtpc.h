@@ -326,6 +326,22 @@ int mtpc_launch_count(mtpc_head* head, uint64_t* out_count);
 int mtpc_debug_set_wait_limit_ns(mtpc_head* head, uint64_t limit_ns);
 
 /*
+ * Test and measurement hook (no passage of the paper): which build of the projection kernel this head launches.
+ * 0 (default): chosen per launch; 1: every CTA works alone (tcgen05 cta_group::1); 2: clusters of two CTAs share every
+ * MMA (cta_group::2), MTPC_ERR_UNSUPPORTED if the device cannot hold such a cluster. The results are the same numbers
+ * either way (same products, same order of accumulation); the tests run both.
+ */
+int mtpc_debug_set_projection_variant(mtpc_head* head, int32_t variant);
+
+/*
+ * Test and measurement hook (no passage of the paper): how mtpc_draft_sample on more than 128 positions runs the byte
+ * draws of Algorithm 1. 0 (default): chosen per call; 1: one pass of every position against every input unit;
+ * 2: the (window, slot) pairs are first sorted by the unit they sample from, and each is multiplied by that unit only
+ * (MTPC_ERR_UNSUPPORTED if the head was created for at most 128 positions). Same uniforms, same bytes either way.
+ */
+int mtpc_debug_set_draft_grouping(mtpc_head* head, int32_t mode);
+
+/*
  * Window log-likelihood without any allocation (the paper has no counterpart: this is a packaging variant of
  * mtpc_window_logprob, same arithmetic, same kernels, same results).
  *

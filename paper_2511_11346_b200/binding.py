@@ -24,6 +24,7 @@ EXPORTS = [
     "mtpc_window_prefix_logprob", "mtpc_draft_sample_prefix", "mtpc_speculative_accept", "mtpc_window_loss",
     "mtpc_backward_workspace_bytes", "mtpc_window_logprob_backward", "mtpc_window_loss_backward",
     "mtpc_lowrank_compose", "mtpc_lowrank_backward", "mtpc_update_parameters", "mtpc_debug_set_wait_limit_ns",
+    "mtpc_debug_set_projection_variant", "mtpc_debug_set_draft_grouping",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 ERR_STATIC_SCRATCH = -7
@@ -79,6 +80,8 @@ def lib() -> ctypes.CDLL:
     L.mtpc_lowrank_backward.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     L.mtpc_update_parameters.argtypes = [vp, vp, vp, vp, vp]
     L.mtpc_debug_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
+    L.mtpc_debug_set_projection_variant.argtypes = [vp, i32]
+    L.mtpc_debug_set_draft_grouping.argtypes = [vp, i32]
     L.mtpc_status_string.argtypes = [ctypes.c_int]
     L.mtpc_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -240,6 +243,14 @@ class MtpcHead:
     def mtpc_debug_set_wait_limit_ns(self, limit_ns: int) -> None:
         """Test hook: time limit of the pipeline waits inside the tensor-core kernels (0 = the default of 1 s)."""
         _check(lib().mtpc_debug_set_wait_limit_ns(self.handle, int(limit_ns)), "mtpc_debug_set_wait_limit_ns")
+
+    def mtpc_debug_set_projection_variant(self, variant: int) -> None:
+        """Test hook: 0 = projection kernel chosen per launch, 1 = single CTAs, 2 = CTA pairs (cta_group::2)."""
+        _check(lib().mtpc_debug_set_projection_variant(self.handle, int(variant)), "mtpc_debug_set_projection_variant")
+
+    def mtpc_debug_set_draft_grouping(self, mode: int) -> None:
+        """Test hook, many-position draft: 0 = chosen per call, 1 = all units for all positions, 2 = draws sorted by unit."""
+        _check(lib().mtpc_debug_set_draft_grouping(self.handle, int(mode)), "mtpc_debug_set_draft_grouping")
 
     def mtpc_set_timing(self, ring: int) -> None:
         _check(lib().mtpc_set_timing(self.handle, int(ring)), "mtpc_set_timing")

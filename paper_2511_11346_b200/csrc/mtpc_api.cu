@@ -31,6 +31,9 @@ constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA 
 // Hidden states of one rasterisation block of the projection kernel: small enough to stay L2-resident next to the
 // weight tiles streaming past (data read by all SMs ends up in both halves of the 126 MB L2).
 constexpr size_t kHiddenBlockBytes = 36u << 20;
+// Many-position draft, sampling pass grouped by unit: hidden states staged per (window, slot) pair, at most this much
+// at a time (longer calls are processed in chunks of positions).
+constexpr size_t kGroupStageBytes = 1u << 30;
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
@@ -42,6 +45,7 @@ struct Tiling {
   int group_tiles;      // tiles of a full group
   int num_groups;       // groups covering all n*r units
   int slot_stride, num_slots, stages, stage_bytes, smem;
+  int pair_stages, pair_stage_bytes, pair_smem;   // the same ring when two CTAs share every MMA (half a weight tile per CTA)
 };
 
 struct Layout {
@@ -57,6 +61,9 @@ struct Layout {
   bool can_draft;       // v <= 512: the sampling kernels hold a whole input unit on chip
   bool can_draft_many;  // the sampling epilogue of the projection kernel can tile a unit (draft of more than 128 positions)
   size_t off_h_hidden, off_h_targets, off_h_uniforms, off_h_bytes, off_h_out;
+  // grouped sampling pass of the many-position draft (0 entries: not available)
+  size_t group_entries;   // (window, slot) pairs that can be staged at once
+  size_t off_grp_ints, off_grp_tiles, off_grp_perm, off_grp_stage;
   size_t total;
 };
 
@@ -74,6 +81,10 @@ bool fit_tiling(Tiling* t, int sum_cols) {
   if (stages > kMaxStages) stages = kMaxStages;
   t->stages = stages;
   t->smem = stages * t->stage_bytes + ctl;
+  t->pair_stage_bytes = (kABytes + widest / 2 * kBlockK * 2 + 1023) / 1024 * 1024;   // A tile + half a B tile
+  t->pair_stages = (kSmemLimit - ctl) / t->pair_stage_bytes;
+  if (t->pair_stages > kMaxStages) t->pair_stages = kMaxStages;
+  t->pair_smem = t->pair_stages * t->pair_stage_bytes + ctl;
   return stages >= 2 && t->num_slots >= 2;
 }
 
@@ -156,6 +167,19 @@ int plan(const mtpc_config& c, Layout* L) {
   L->off_h_uniforms = take(L->max_windows * 2 * c.n * 4);
   L->off_h_bytes = take(L->max_windows * c.n * 4);
   L->off_h_out = take(L->max_windows * 4);
+  // grouped sampling: only heads that can be asked for a many-position draft carry the staging area
+  L->group_entries = 0;
+  if (L->can_draft_many && c.max_positions > L->decode_max_p && emit_units <= kGroupMaxUnits) {
+    const size_t cap = kGroupStageBytes / (static_cast<size_t>(c.d) * 2);
+    const size_t all = L->max_windows * c.n;
+    L->group_entries = all < cap ? all : cap;
+    if (L->group_entries < static_cast<size_t>(c.max_windows_per_pos) * c.n) L->group_entries = 0;   // not even one position
+  }
+  const size_t ge = L->group_entries;
+  L->off_grp_ints = take(ge ? (3 * static_cast<size_t>(emit_units) + 64) * 4 : 0);     // counts | cursors | offsets | tile count
+  L->off_grp_tiles = take(ge ? (emit_units + ge / 128 + 1) * sizeof(GroupTile) : 0);
+  L->off_grp_perm = take(ge * 4);
+  L->off_grp_stage = take(ge * c.d * 2);
   L->total = off;
   return MTPC_OK;
 }
@@ -203,6 +227,10 @@ struct mtpc_head {
   const void* W_emit_bf16;
   const void* W_sum_bf16;
   CUtensorMap tm_emit_lp, tm_emit_sm, tm_sum;   // W_emit with the box of either tiling; W_sum
+  CUtensorMap tm_emit_lp2, tm_emit_sm2, tm_sum2; // the same with boxes of half the rows: what one CTA of a pair stages
+  int projection_variant;                       // 0: chosen per launch; 1: every CTA alone; 2: CTA pairs (cta_group::2)
+  int draft_grouping;                           // many-position draft: 0 chosen per call; 1 never sort the draws by unit; 2 always
+  int max_pairs;                                // clusters of two projection CTAs that can be resident at once
   CUtensorMap tm_emit_dec, tm_sum_dec;          // the same matrices in the few-position draft path's tiles
   int decode_tile_rows, decode_sum_tile_rows;
   int num_sms;
@@ -297,6 +325,16 @@ int choose_group_units(int v, int emit_units, int m_tiles, int ctas) {
   return best;
 }
 
+struct GroupArgs {           // grouped sampling pass: the staged hidden states and their tiles (mtpc_group.cuh)
+  const void* stage = nullptr;
+  int entries = 0;                           // rows of the staging buffer in use
+  const GroupTile* tiles = nullptr;
+  const int* num_tiles = nullptr;
+  const int* perm = nullptr;
+  const int* unit_sel = nullptr;             // this chunk's rows of the selected units
+  int max_tiles = 0;
+};
+
 struct GradArgs {            // what the projection kernel keeps for the backward pass (training calls only)
   float* lse_out = nullptr;                  // the units' log-sum-exps [T, n, r]
   float* logit_out = nullptr;                // the emission logits [T, n r v] fp32
@@ -305,11 +343,12 @@ struct GradArgs {            // what the projection kernel keeps for the backwar
 
 int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int wpp, bool with_emit, bool with_sum,
                 const int* targets, const float* uniforms, int* out_bytes, cudaStream_t st,
-                const GradArgs* ga = nullptr, bool targets_are_drafts = false) {
+                const GradArgs* ga = nullptr, bool targets_are_drafts = false, const GroupArgs* grp = nullptr) {
   if (rows <= 0 || (!with_emit && !with_sum)) return MTPC_OK;
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
   const Tiling& tl = mode == kModeSample ? L.sm : L.lp;
+  if (grp != nullptr && mode != kModeSample) return MTPC_ERR_SHAPE;
   GemmParams p;
   memset(&p, 0, sizeof(p));
   if (ga) {
@@ -317,19 +356,25 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
     p.logit_out = ga->logit_out;
     p.logit_pitch = ga->logit_pitch;
   }
-  int rc = make_tmap(&p.tm_a, hidden_bf16, static_cast<uint64_t>(rows), static_cast<uint64_t>(c.d), kBlockM);
+  int rc = grp ? make_tmap(&p.tm_a, grp->stage, static_cast<uint64_t>(grp->entries), static_cast<uint64_t>(c.d), kBlockM)
+               : make_tmap(&p.tm_a, hidden_bf16, static_cast<uint64_t>(rows), static_cast<uint64_t>(c.d), kBlockM);
   if (rc != MTPC_OK) return rc;
   p.tm_emit = mode == kModeSample ? h->tm_emit_sm : h->tm_emit_lp;
   p.tm_sum = h->tm_sum;
   p.T = rows;
   p.m_tiles = (rows + kBlockM - 1) / kBlockM;
-  p.m_units = p.m_tiles;
+  // Two CTAs per MMA when there are at least two m-tiles to pair up (and the device can hold a cluster at all)
+  const bool pair = grp == nullptr &&
+                    (h->projection_variant == 2 || (h->projection_variant == 0 && p.m_tiles >= 2 && h->max_pairs > 0));
+  const int ctas = pair ? 2 : 1;
+  const int workers = pair ? h->max_pairs : h->num_sms;               // CTAs, or CTA pairs, resident at once
+  p.m_units = (p.m_tiles + ctas - 1) / ctas;
   p.kblocks = c.d / kBlockK;
   {
-    const size_t tile_bytes = static_cast<size_t>(kBlockM) * c.d * 2;
-    const int cap_tiles = kHiddenBlockBytes / tile_bytes > 0 ? static_cast<int>(kHiddenBlockBytes / tile_bytes) : 1;
-    const int nblocks = (p.m_tiles + cap_tiles - 1) / cap_tiles;
-    p.m_block = (p.m_tiles + nblocks - 1) / nblocks;
+    const size_t unit_bytes = static_cast<size_t>(kBlockM) * ctas * c.d * 2;
+    const int cap_units = kHiddenBlockBytes / unit_bytes > 0 ? static_cast<int>(kHiddenBlockBytes / unit_bytes) : 1;
+    const int nblocks = (p.m_units + cap_units - 1) / cap_units;
+    p.m_block = (p.m_units + nblocks - 1) / nblocks;
   }
   p.n = c.n; p.r = c.r; p.v = c.v;
   p.vv = valid_symbols(c);
@@ -337,7 +382,7 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   p.num_groups = with_emit ? tl.num_groups : 0;
   p.group_units = tl.group_units;
   if (mode != kModeSample && with_emit) {
-    p.group_units = choose_group_units(c.v, p.emit_units, p.m_tiles, h->num_sms);
+    p.group_units = choose_group_units(c.v, p.emit_units, p.m_units, workers);
     p.num_groups = (p.emit_units + p.group_units - 1) / p.group_units;
   }
   p.tile_cols = tl.tile_cols;
@@ -346,8 +391,12 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   p.sum_rows = L.sum_rows;
   p.slot_stride = tl.slot_stride;
   p.num_slots = tl.num_slots;
-  p.stages = tl.stages;
-  p.stage_bytes = tl.stage_bytes;
+  p.stages = pair ? tl.pair_stages : tl.stages;
+  p.stage_bytes = pair ? tl.pair_stage_bytes : tl.stage_bytes;
+  if (pair) {
+    p.tm_emit = mode == kModeSample ? h->tm_emit_sm2 : h->tm_emit_lp2;
+    p.tm_sum = h->tm_sum2;
+  }
   p.wpp = wpp;
   p.targets = targets;
   p.missing_is_nan = targets_are_drafts ? 1 : 0;
@@ -355,16 +404,43 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   p.logw = at<float>(h, L.off_logw);
   p.sum_bias = sum_bias(h);
   p.unit_sel = at<int>(h, L.off_sel);
+  if (grp) {
+    p.group_tiles = grp->tiles;
+    p.group_num_tiles = grp->num_tiles;
+    p.group_perm = grp->perm;
+    p.unit_sel = grp->unit_sel;
+  }
   p.uniforms = uniforms;
   p.out_bytes = out_bytes;
   p.status = at<unsigned>(h, L.off_status);
   p.wait_limit_ns = h->wait_limit_ns;
-  const long long items = static_cast<long long>(p.m_tiles) * (p.num_groups + p.num_sum_tiles);
-  const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
-  if (mode == kModeLogprob)
-    mtpc_gemm_kernel<kModeLogprob, 1><<<grid, kGemmThreads, tl.smem, st>>>(p);
-  else
-    mtpc_gemm_kernel<kModeSample, 1><<<grid, kGemmThreads, tl.smem, st>>>(p);
+  const long long items = grp ? grp->max_tiles : static_cast<long long>(p.m_units) * (p.num_groups + p.num_sum_tiles);
+  const int grid = ctas * static_cast<int>(items < workers ? items : workers);
+  const size_t smem = pair ? tl.pair_smem : tl.smem;
+  if (grp) {
+    mtpc_gemm_kernel<kModeSampleGrouped, 1><<<grid, kGemmThreads, smem, st>>>(p);
+  } else if (!pair) {
+    if (mode == kModeLogprob)
+      mtpc_gemm_kernel<kModeLogprob, 1><<<grid, kGemmThreads, smem, st>>>(p);
+    else
+      mtpc_gemm_kernel<kModeSample, 1><<<grid, kGemmThreads, smem, st>>>(p);
+  } else {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (mode == kModeLogprob) cudaLaunchKernelEx(&cfg, mtpc_gemm_kernel<kModeLogprob, 2>, p);
+    else cudaLaunchKernelEx(&cfg, mtpc_gemm_kernel<kModeSample, 2>, p);
+  }
   h->launches++;
   return check_launch();
 }
@@ -422,6 +498,28 @@ bool set_circuit_attributes() {
   ok &= allow_full_smem(circuit_btree_kernel<false>);
   ok &= allow_full_smem(circuit_btree_kernel<true>);
   return ok;
+}
+
+// How many clusters of two projection CTAs the device holds at once (0: none, the single-CTA kernel is used).
+int resident_pairs(int smem_bytes) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(2);
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&clusters, mtpc_gemm_kernel<kModeLogprob, 2>, &cfg) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return clusters;
 }
 
 // Rows per emission tile of the few-position draft path: the height in [64, 128] (multiple of 8) that leaves the
@@ -571,11 +669,53 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   h->launches++;
   pt.end();
   if ((rc = check_launch()) != MTPC_OK) return rc;
-  // 3. byte draws at the selected input units
-  pt.begin();
-  rc = launch_gemm(h, kModeSample, hb, P, wpp, true, false, nullptr, uniforms, out_bytes, st);
-  pt.end();
-  if (rc != MTPC_OK) return rc;
+  // 3. byte draws at the selected input units. With few windows per position against many units per slot the draws
+  // are first sorted by unit, so that every window is multiplied by the one unit it samples from.
+  const bool grouped = L.group_entries > 0 && h->draft_grouping != 1 && (h->draft_grouping == 2 || wpp * 4 <= c.r);
+  if (grouped) {
+    const int units = c.n * c.r;
+    int* ints = at<int>(h, L.off_grp_ints);
+    int* counts = ints, *cursors = ints + units, *offsets = ints + 2 * units, *num_tiles = ints + 3 * units;
+    GroupTile* tiles = at<GroupTile>(h, L.off_grp_tiles);
+    int* perm = at<int>(h, L.off_grp_perm);
+    __nv_bfloat16* stage = at<__nv_bfloat16>(h, L.off_grp_stage);
+    const int chunk_pos = static_cast<int>(L.group_entries / (static_cast<size_t>(wpp) * c.n));   // >= 1 by construction
+    for (int p0 = 0; p0 < P; p0 += chunk_pos) {
+      const int pc = P - p0 < chunk_pos ? P - p0 : chunk_pos;
+      const int entries = pc * wpp * c.n;
+      const size_t w0 = static_cast<size_t>(p0) * wpp;
+      const int* sel = at<int>(h, L.off_sel) + w0 * c.n;
+      pt.begin();
+      if (cudaMemsetAsync(ints, 0, static_cast<size_t>(2 * units) * 4, st) != cudaSuccess) return MTPC_ERR_CUDA;
+      const int cblocks = (entries + kGroupThreads - 1) / kGroupThreads;
+      group_count_kernel<<<cblocks < 4 * h->num_sms ? cblocks : 4 * h->num_sms, kGroupThreads, units * sizeof(int), st>>>(
+          sel, counts, entries, c.n, c.r);
+      group_scan_kernel<<<1, kGroupScanThreads, 0, st>>>(counts, offsets, tiles, num_tiles, units);
+      const int gblocks = (entries + kGroupThreads / 32 - 1) / (kGroupThreads / 32);
+      group_gather_kernel<<<gblocks < 16 * h->num_sms ? gblocks : 16 * h->num_sms, kGroupThreads, 0, st>>>(
+          sel, static_cast<const __nv_bfloat16*>(hb) + static_cast<size_t>(p0) * c.d, offsets, cursors, perm, stage, entries,
+          c.n, c.r, wpp, c.d);
+      h->launches += 3;
+      if ((rc = check_launch()) != MTPC_OK) return rc;
+      GroupArgs ga;
+      ga.stage = stage;
+      ga.entries = entries;
+      ga.tiles = tiles;
+      ga.num_tiles = num_tiles;
+      ga.perm = perm;
+      ga.unit_sel = sel;
+      ga.max_tiles = units + entries / 128 + 1;
+      rc = launch_gemm(h, kModeSample, hb, pc, wpp, true, false, nullptr, uniforms + w0 * 2 * c.n, out_bytes + w0 * c.n, st,
+                       nullptr, false, &ga);
+      pt.end();
+      if (rc != MTPC_OK) return rc;
+    }
+  } else {
+    pt.begin();
+    rc = launch_gemm(h, kModeSample, hb, P, wpp, true, false, nullptr, uniforms, out_bytes, st);
+    pt.end();
+    if (rc != MTPC_OK) return rc;
+  }
   // 4. evidence of the drafted bytes under every unit -> 5. joint log-prob with the latents summed out
   pt.begin();
   rc = launch_gemm(h, kModeLogprob, hb, P, wpp, true, false, out_bytes, nullptr, nullptr, st, nullptr,
@@ -814,6 +954,9 @@ static int bind_parameters(mtpc_head* h, const void* W_emit, const void* W_sum, 
   int rc = make_tmap(&h->tm_emit_lp, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols);
   if (rc == MTPC_OK && L.can_draft_many) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols);
+  if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_lp2, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols / 2);
+  if (rc == MTPC_OK && L.can_draft_many) rc = make_tmap(&h->tm_emit_sm2, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols / 2);
+  if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum2, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols / 2);
   h->decode_tile_rows = decode_tile_rows(static_cast<long long>(emit_rows), h->num_sms);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_dec, h->W_emit_bf16, emit_rows, cfg->d, h->decode_tile_rows);
   h->decode_sum_tile_rows = h->decode_tile_rows / 32 * 32;   // whole groups of r <= 32 rows per warp; fits the tile pitch
@@ -861,6 +1004,10 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
                                kSmemLimit) != cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeSample, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
+  fail |= !allow_full_smem(mtpc_gemm_kernel<kModeSampleGrouped, 1>);
+  fail |= !allow_full_smem(mtpc_gemm_kernel<kModeLogprob, 2>);
+  fail |= !allow_full_smem(mtpc_gemm_kernel<kModeSample, 2>);
+  h->max_pairs = fail ? 0 : resident_pairs(L.lp.pair_smem);
   fail |= cudaFuncSetAttribute(plain_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
           cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
@@ -1333,6 +1480,22 @@ int mtpc_get_timing(mtpc_head* head, int32_t calls_back, float* out_ms, int32_t 
 int mtpc_debug_set_wait_limit_ns(mtpc_head* head, uint64_t limit_ns) {
   if (!head) return MTPC_ERR_NULL;
   head->wait_limit_ns = limit_ns == 0 ? kWaitLimitNs : limit_ns;
+  return MTPC_OK;
+}
+
+int mtpc_debug_set_projection_variant(mtpc_head* head, int32_t variant) {
+  if (!head) return MTPC_ERR_NULL;
+  if (variant < 0 || variant > 2) return MTPC_ERR_SHAPE;
+  if (variant == 2 && head->max_pairs <= 0) return MTPC_ERR_UNSUPPORTED;
+  head->projection_variant = variant;
+  return MTPC_OK;
+}
+
+int mtpc_debug_set_draft_grouping(mtpc_head* head, int32_t mode) {
+  if (!head) return MTPC_ERR_NULL;
+  if (mode < 0 || mode > 2) return MTPC_ERR_SHAPE;
+  if (mode == 2 && head->L.group_entries == 0) return MTPC_ERR_UNSUPPORTED;
+  head->draft_grouping = mode;
   return MTPC_OK;
 }
 

@@ -24,6 +24,7 @@
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
+#include "mtpc_group.cuh"
 #include "mtpc_ptx.cuh"
 
 namespace mtpc {
@@ -39,7 +40,9 @@ constexpr uint64_t kAbortSettleNs = 200ull * 1000ull;            // 0.2 ms: far 
 constexpr int kABytes = kBlockM * kBlockK * 2;                   // 16 KB
 constexpr uint32_t kStatusBadTarget = 1u, kStatusBadUniform = 2u, kStatusTimeout = 4u;
 
-enum { kModeLogprob = 0, kModeSample = 1 };
+// kModeSampleGrouped: the byte draws again, on rows that were sorted by the unit they sample from (mtpc_group.cuh):
+// a work item is one GroupTile instead of (m-tile, unit).
+enum { kModeLogprob = 0, kModeSample = 1, kModeSampleGrouped = 2 };
 
 struct GemmParams {
   CUtensorMap tm_a;      // hidden  [T, d]        box 64 x 128
@@ -70,6 +73,9 @@ struct GemmParams {
   const int* unit_sel;               // [T*wpp, n]      selected input unit per token (sample mode)
   const float* uniforms;             // [T*wpp, 2n]
   int* out_bytes;                    // [T*wpp, n]
+  const GroupTile* group_tiles;      // grouped sampling: the work items, ...
+  const int* group_num_tiles;        // ... how many there are (device memory: written by the kernel that made them), ...
+  const int* group_perm;             // ... and which (window, slot) pair every row of the staged hidden states (tm_a) holds
   unsigned* status;
   uint64_t wait_limit_ns;            // limit of every pipeline wait (kWaitLimitNs unless a test shortened it)
 };
@@ -124,7 +130,23 @@ __device__ __forceinline__ bool bounded_wait_warp(uint32_t bar, uint32_t parity,
 
 struct TileCoord {
   int mt, is_sum, ntiles, cols, brow0, unit0, nunits;
+  int arow, count;   // first row of the A operand and the rows that count (set by the caller for ungrouped items)
 };
+// A grouped item: `count` staged rows from `row0` on, against the tiles of the one unit they sample from.
+__device__ __forceinline__ TileCoord group_coord(const GemmParams& p, int item) {
+  const GroupTile g = p.group_tiles[item];
+  TileCoord c;
+  c.mt = 0;
+  c.is_sum = 0;
+  c.unit0 = g.unit;
+  c.nunits = 1;
+  c.cols = p.tile_cols;
+  c.brow0 = g.unit * p.v;
+  c.ntiles = p.v / p.tile_cols;
+  c.arow = g.row0;
+  c.count = g.count;
+  return c;
+}
 // Work items (c.mt counts M work units: m-tiles, or pairs of m-tiles in the CTA-pair kernel). Emission items come
 // first, in blocks of m_block units: inside a block the unit runs fastest and
 // the group next, so the CTAs that run at the same time share a few groups' weights through L2 while the block's
@@ -210,8 +232,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int num_items = (p.num_groups + p.num_sum_tiles) * p.m_units;
+  static_assert(MODE != kModeSampleGrouped || CTAS == 1, "grouped tiles are ragged: no pairing");
+  const int num_items = MODE == kModeSampleGrouped ? *p.group_num_tiles : (p.num_groups + p.num_sum_tiles) * p.m_units;
   const uint32_t cta_rank = CTAS == 2 ? cluster_cta_rank() : 0u;      // 0 = the pair's leader
+  auto coord = [&](int item) {
+    if (MODE == kModeSampleGrouped) return group_coord(p, item);
+    TileCoord c = tile_coord(p, item);
+    c.arow = (c.mt * CTAS + static_cast<int>(cta_rank)) * kBlockM;
+    c.count = min(kBlockM, p.T - c.arow);                             // <= 0: a pair's second CTA past the last position
+    return c;
+  };
   const int first_item = CTAS == 2 ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
   const int item_step = CTAS == 2 ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
 
@@ -253,11 +283,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
       uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
       bool ok = true;
       for (int item = first_item; item < num_items && ok; item += item_step) {
-        const TileCoord tc = tile_coord(p, item);
+        const TileCoord tc = coord(item);
         const CUtensorMap* tmb = tc.is_sum ? &p.tm_sum : &p.tm_emit;
         const int brows = tc.cols / CTAS;                                 // weight rows this CTA stages per tile
         const uint32_t bytes = CTAS * (kABytes + brows * (kBlockK * 2));   // of both CTAs' copies when paired
-        const int arow = (tc.mt * CTAS + static_cast<int>(cta_rank)) * kBlockM;
+        const int arow = tc.arow;
         for (int t = 0; t < tc.ntiles && ok; ++t) {
           for (int kb = 0; kb < p.kblocks; ++kb) {
             if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
@@ -299,7 +329,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
       uint32_t stage = 0, phase = 0, use = 0;
       bool ok = true;
       for (int item = first_item; item < num_items && ok; item += item_step) {
-        const TileCoord tc = tile_coord(p, item);
+        const TileCoord tc = coord(item);
         const uint32_t idesc = umma_idesc_bf16(kBlockM * CTAS, tc.cols);
         for (int t = 0; t < tc.ntiles && ok; ++t, ++use) {
           const uint32_t slot = use % p.num_slots;
@@ -349,9 +379,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
       else mbar_arrive(smem_u32(&ctl->tempty[slot]));
     };
     for (int item = first_item; item < num_items && ok; item += item_step) {
-      const TileCoord tc = tile_coord(p, item);
-      const int row = (tc.mt * CTAS + static_cast<int>(cta_rank)) * kBlockM + quarter * 32 + lane;
-      const bool valid = row < p.T;
+      const TileCoord tc = coord(item);
+      const int row = tc.arow + quarter * 32 + lane;
+      const bool valid = quarter * 32 + lane < tc.count;
       const int nbatch = tc.cols / 16;
 
       if (tc.is_sum) {
@@ -528,10 +558,18 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
         const int slot_i = tc.unit0 / p.r;
         const int k = tc.unit0 - slot_i * p.r;
         unsigned long long pending = 0ull;
-        const size_t wrow0 = static_cast<size_t>(valid ? row : 0) * p.wpp;
-        if (valid)
-          for (int j = 0; j < p.wpp; ++j)
-            if (p.unit_sel[(wrow0 + j) * p.n + slot_i] == k) pending |= 1ull << j;
+        size_t wrow0 = 0;
+        int nwin = p.wpp;
+        if (MODE == kModeSampleGrouped) {
+          // the row holds one (window, slot) pair, and the slot is this tile's
+          if (valid) { wrow0 = static_cast<size_t>(p.group_perm[row] / p.n); pending = 1ull; }
+          nwin = 1;
+        } else {
+          wrow0 = static_cast<size_t>(valid ? row : 0) * p.wpp;
+          if (valid)
+            for (int j = 0; j < nwin; ++j)
+              if (p.unit_sel[(wrow0 + j) * p.n + slot_i] == k) pending |= 1ull << j;
+        }
         for (int c = 0; c < tc.ntiles && ok; ++c) {
           const uint32_t u = use + c;
           if (!bounded_wait_warp(smem_u32(&ctl->tfull[u % p.num_slots]), (u / p.num_slots) & 1u, ctl, p.status,
@@ -615,6 +653,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
       const uint64_t t0 = global_timer_ns();
       while (global_timer_ns() - t0 < kAbortSettleNs) {}
     }
+    __syncthreads();      // every warp converged again before the cluster-wide barrier
     cluster_sync_all();
   }
   if (warp == 1) {

@@ -56,17 +56,91 @@ def test_heads_of_different_shapes_do_not_lower_each_others_shared_memory_limit(
         dh.close()
 
 
-@pytest.mark.parametrize("path", ["logprob", "draft_few", "draft_many", "backward"])
+@pytest.mark.parametrize("family,n,r,v,d,T,wpp", [
+    (I.CP, 3, 16, 320, 128, 700, 1),        # 6 m-tiles: three pairs; v = 320 tiles straddle units
+    (I.HMM, 4, 8, 64, 192, 385, 2),         # odd number of m-tiles and a ragged last one: the last pair's second CTA is empty
+    (I.BTREE, 8, 32, 256, 64, 290, 1),      # 193 sum units: several sum tiles
+    (I.CP, 2, 4, 48, 64, 100, 3),           # a single m-tile run by a pair
+])
+def test_both_builds_of_the_projection_kernel_give_the_same_numbers(family, n, r, v, d, T, wpp):
+    """Single CTAs (cta_group::1) and CTA pairs (cta_group::2) form the same products in the same order: log-probs,
+    drafted bytes and gradients must agree bit for bit, and with the oracle."""
+    wl = I.make_workload("variants", I.HeadShape(family, n, r, v, d), T, seed=300 + n + r, wpp=wpp, weight_std=0.25)
+    dh = DeviceHead(wl)
+    ref = oracle_logprob(wl)
+    weight = torch.full((wl.T,), -1.0 / wl.T, dtype=torch.float32, device="cuda")
+    results = []
+    for variant in (1, 2):
+        dh.head.mtpc_debug_set_projection_variant(variant)
+        lp = dh.window_logprob().cpu().numpy()
+        assert np.abs(lp - ref).max() <= LOGPROB_TOL, variant
+        out_bytes, out_lp = dh.draft_sample()
+        g = dh.window_logprob_backward(weight)
+        assert dh.head.mtpc_get_status(with_code=True) == (B.MTPC_OK, 0)
+        results.append((lp, out_bytes.cpu().numpy(), out_lp.cpu().numpy(), g["dh"].cpu().numpy(), g["dW_emit"].cpu().numpy()))
+    for a, b in zip(*results):
+        np.testing.assert_array_equal(a, b)
+    d = orc.draft_sample(family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wl.wpp, wl.uniforms)
+    differ = (results[0][1] != d["bytes"]).any(axis=1)
+    assert not (differ & (d["margin"] >= 1e-6)).any()
+    dh.close()
+
+
+@pytest.mark.parametrize("family,n,r,v,d,T,wpp", [
+    (I.CP, 3, 4, 320, 128, 2000, 1),        # 12 units, ~500 windows each: every unit spans several 128-row tiles
+    (I.CP, 2, 64, 64, 64, 150, 1),          # 128 units for 300 draws: units with one window, units with none
+    (I.HMM, 4, 8, 48, 64, 300, 2),          # two windows per position, padded-free odd vocabulary tile (48 columns)
+    (I.BTREE, 8, 32, 256, 64, 290, 1),      # tree latents
+    (I.HMM_CTX, 3, 16, 320, 64, 200, 1),    # contextual transitions; a unit's 320 columns in two accumulator tiles
+])
+def test_draws_sorted_by_unit_give_the_same_bytes(family, n, r, v, d, T, wpp):
+    """Many-position draft (Algorithm 1): running every position against every unit, or sorting the (window, slot) pairs
+    by the unit they sample from and multiplying each by that unit only, must return the same bytes and log-probs -
+    the order in which windows are processed must not matter - and they must be the oracle's."""
+    wl = I.make_workload("grouped", I.HeadShape(family, n, r, v, d), T, seed=500 + n + r, wpp=wpp, weight_std=0.25)
+    dh = DeviceHead(wl)
+    u = wl.uniforms.copy()
+    u[5, n + 1] = 2.0                        # a refused byte draw ...
+    u[9, 0] = -1.0                           # ... and a refused latent draw keep their meaning in both modes
+    ud = torch.from_numpy(u).cuda()
+    got = []
+    for mode in (1, 2, 2):                   # the sorted pass twice: its internal row order differs from run to run
+        dh.head.mtpc_debug_set_draft_grouping(mode)
+        out_bytes, out_lp = dh.draft_sample(uniforms=ud)
+        assert dh.head.mtpc_get_status(with_code=True) == (B.MTPC_OK, B.STATUS_BAD_UNIFORM)
+        got.append((out_bytes.cpu().numpy(), out_lp.cpu().numpy()))
+    for b, lp in got[1:]:
+        np.testing.assert_array_equal(b, got[0][0])
+        np.testing.assert_array_equal(lp, got[0][1])
+    gb, gl = got[1]
+    assert gb[5, 1] == -1 and (gb[9] == -1).all() and np.isnan(gl[5]) and np.isnan(gl[9])
+    ok = np.ones(len(gb), dtype=bool)
+    ok[[5, 9]] = False
+    fam = wl.shape.family
+    ref = orc.draft_sample(fam, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wpp, wl.uniforms)
+    differ = (gb != ref["bytes"]).any(axis=1) & ok
+    assert not (differ & (ref["margin"] >= 1e-6)).any()
+    same = ok & ~differ
+    assert np.abs(gl[same] - ref["logprob"][same]).max() <= LOGPROB_TOL
+    dh.close()
+
+
+@pytest.mark.parametrize("path", ["logprob", "logprob_single_ctas", "draft_few", "draft_many", "draft_many_ungrouped", "backward"])
 def test_a_wait_that_runs_out_is_reported_and_the_head_recovers(path):
     """Projection kernel (log-likelihood and sampling epilogues), the few-position draft kernel and the plain GEMMs of
     the backward pass: with a 50 ns limit the first wait for a copy gives up in every CTA."""
-    T = {"logprob": 300, "draft_few": 8, "draft_many": 200, "backward": 300}[path]
+    T = {"logprob": 300, "logprob_single_ctas": 300, "draft_few": 8, "draft_many": 200, "draft_many_ungrouped": 200,
+         "backward": 300}[path]
     wl = I.make_workload("timeout_" + path, I.HeadShape(I.HMM, 4, 8, 64, 4096), T, seed=77, wpp=2, weight_std=0.2)
     dh = DeviceHead(wl)
     weight = torch.full((wl.T,), -1.0 / wl.T, dtype=torch.float32, device="cuda")
+    if path == "logprob_single_ctas":
+        dh.head.mtpc_debug_set_projection_variant(1)      # the other paths pair their CTAs (more than one m-tile)
+    if path == "draft_many_ungrouped":
+        dh.head.mtpc_debug_set_draft_grouping(1)          # wpp = 2 against r = 8 units: sorted by unit otherwise
 
     def call():
-        if path == "logprob":
+        if path.startswith("logprob"):
             return dh.window_logprob()
         if path == "backward":
             return dh.window_logprob_backward(weight)["logprob"]
@@ -82,7 +156,7 @@ def test_a_wait_that_runs_out_is_reported_and_the_head_recovers(path):
     assert "wait" in B.status_string(code)
     assert dh.head.mtpc_get_status(with_code=True) == (B.MTPC_OK, 0)      # reading cleared the word
     dh.head.mtpc_debug_set_wait_limit_ns(0)               # back to the default
-    if path in ("logprob", "backward"):
+    if path.startswith("logprob") or path == "backward":
         got = call().cpu().numpy()
         assert np.abs(got - oracle_logprob(wl)).max() <= LOGPROB_TOL
     else:
