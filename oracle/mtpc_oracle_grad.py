@@ -61,8 +61,15 @@ def forward(family: int, h, W_emit, W_sum, T_static, targets):
     n, r, v, d = W_emit.shape
     T = h.shape[0]
     logits = (h @ W_emit.reshape(n * r * v, d).T).reshape(T, n, r, v)
-    logphi = torch.log_softmax(logits, dim=-1)
     slog = (h @ W_sum.T).reshape(T, W_sum.shape[0] // r, r)
+    return forward_from_logits(family, logits, slog, T_static, targets)
+
+
+def forward_from_logits(family: int, logits, slog, T_static, targets):
+    """The same definition from the two projections on: logits [T, n, r, v] of the input units, slog [T, S, r] of the sum
+    units (Sec. 3.3), then the softmaxes and the circuit."""
+    T, n, r, v = logits.shape
+    logphi = torch.log_softmax(logits, dim=-1)
     if family == HMM_CTX and T_static is not None:
         slog = torch.cat([slog[:, :1, :], slog[:, 1:, :] + T_static.reshape(1, -1, r)], dim=1)
     logw = torch.log_softmax(slog, dim=-1)
@@ -83,6 +90,28 @@ def forward(family: int, h, W_emit, W_sum, T_static, targets):
     if family == BTREE:
         return _lse(logw[:, 0, :] + _btree_product(0, 0, n, logw, g, r), dim=-1)
     raise ValueError(family)
+
+
+def window_logprob_logit_grad(family: int, h, W_emit, W_sum, T_static, targets, weight):
+    """Gradient of L = sum_t weight[t] * log q_t with respect to the two projections themselves: dlogit [T, n, r, v]
+    (input units) and dslog [T, S, r] (sum units), numpy float64. By the chain rule through the projections,
+    dW_emit = dlogit^T h, dW_sum = dslog^T h and dh = dlogit W_emit + dslog W_sum (pinned that way); a test uses the
+    magnitudes |dlogit|, |dslog| to bound, entry by entry, what rounding dlogit to 16 bits may cost a gradient."""
+    th = torch.tensor(np.asarray(h, dtype=np.float64))
+    tW = torch.tensor(np.asarray(W_emit, dtype=np.float64))
+    tR = torch.tensor(np.asarray(W_sum, dtype=np.float64))
+    n, r, v, d = tW.shape
+    T = th.shape[0]
+    logits = (th @ tW.reshape(n * r * v, d).T).reshape(T, n, r, v).requires_grad_(True)
+    slog = (th @ tR.T).reshape(T, tR.shape[0] // r, r).requires_grad_(True)
+    tT = None
+    if T_static is not None and family in (HMM, HMM_CTX):
+        tT = torch.tensor(np.asarray(T_static, dtype=np.float64))
+    tx = torch.tensor(np.asarray(targets, dtype=np.int64))
+    tw = torch.tensor(np.asarray(weight, dtype=np.float64))
+    lp = forward_from_logits(family, logits, slog, tT, tx)
+    (lp * tw).sum().backward()
+    return dict(dlogit=logits.grad.numpy(), dslog=np.zeros(tuple(slog.shape)) if slog.grad is None else slog.grad.numpy())
 
 
 def window_logprob_grad(family: int, h, W_emit, W_sum, T_static, targets, weight):

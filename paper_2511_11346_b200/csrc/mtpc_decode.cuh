@@ -26,7 +26,10 @@
 namespace mtpc {
 
 constexpr int kDecodeMaxP = 128;                   // positions per call on this path
-constexpr int kDecodeMaxTiles = 3;                 // weight tiles that share one copy of the hidden states
+#ifndef MTPC_DECODE_MAX_TILES
+#define MTPC_DECODE_MAX_TILES 3
+#endif
+constexpr int kDecodeMaxTiles = MTPC_DECODE_MAX_TILES;   // weight tiles that share one copy of the hidden states
 constexpr int kSlotThreads = 512;
 
 struct DecodeParams {

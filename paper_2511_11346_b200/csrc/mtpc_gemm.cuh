@@ -31,7 +31,10 @@ namespace mtpc {
 
 constexpr int kBlockM = 128;         // positions per tile (= TMEM lanes)
 constexpr int kBlockK = 64;          // bf16 elements per 128-byte swizzled row
-constexpr int kMaxStages = 8;
+#ifndef MTPC_MAX_STAGES
+#define MTPC_MAX_STAGES 8
+#endif
+constexpr int kMaxStages = MTPC_MAX_STAGES;
 constexpr int kMaxSlots = 16;
 constexpr int kTmemCols = 512;
 constexpr int kGemmThreads = 192;

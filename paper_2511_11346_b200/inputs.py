@@ -12,7 +12,8 @@ weights and data that are not available offline):
   3  BTree              T=4096 d=3072 n=16 r=32 v=256  bf16, uniform targets, + draft wpp=1
   4  decode sweep cells P in {1,8,64}, d=4096, v=320, CP r=16 / HMM r=32, n in {8,16}, wpp=16
   5  HMM with contextual transitions: as 2, plus (n-1) r r = 7168 transition rows in W_sum and a bias ~N(0,1) + 4 I
-  6  CP head shaped like the paper's byte-level Llama-3.2-3B (Table 4): d=3072, 268 symbols stored as v=272, n=8, r=16
+  6  CP head shaped like the paper's byte-level Llama-3.2-3B (Table 4): d=3072, 268 symbols stored as v=272, n=8, r=16,
+     fp32 io (the dtype Table 4 gives for that model)
 Hidden states ~N(0,1); every weight ~N(0, std=0.02); uniforms in [0,1) as fp32. For the acceptance stage the
 target model's conditionals are Dirichlet rows (target_rows) and its uniforms come from the same generator.
 """
@@ -240,7 +241,8 @@ def config_workload(idx: int, *, cell: tuple[int, int, int] | None = None, T: in
         return make_workload("btree_train", HeadShape(BTREE, 16, 32, 256, 3072), T or 4096, seed,
                              target_kind="uniform", wpp=1)
     if idx == 6:
-        return make_workload("cp_llama_byte", HeadShape(CP, 8, 16, 272, 3072, v_valid=268), T or 8192, seed, target_kind="zipf")
+        return make_workload("cp_llama_byte", HeadShape(CP, 8, 16, 272, 3072, F32, v_valid=268), T or 8192, seed,
+                             target_kind="zipf")      # fp32 tensors in, as the paper runs its byte-level Llama (Table 4)
     if idx == 5:
         return make_workload("hmmctx_train", HeadShape(HMM_CTX, 8, 32, 320, 4096), T or 8192, seed, target_kind="zipf")
     if idx == 4:

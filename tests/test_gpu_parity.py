@@ -68,7 +68,7 @@ def test_config0_cp_tiny_whole():
     dh.close()
 
 
-@pytest.mark.parametrize("idx,nsample", [(1, 256), (2, 256), (3, 128), (5, 128)])
+@pytest.mark.parametrize("idx,nsample", [(1, 256), (2, 256), (3, 128), (5, 128), (6, 256)])
 def test_full_size_configs_on_sampled_positions(idx, nsample):
     """Full-size launch (the configuration the benchmark times); the oracle checks a seeded sample of
     positions, always including the first and last rows of the first and last 128-row tiles."""
@@ -124,6 +124,17 @@ def test_small_shapes_span_tiles_and_ragged_tails(family, n, r, v, d, T, wpp):
                          weight_std=0.25)        # logits of order one even at small d
     dh = DeviceHead(wl)
     rows = np.arange(T)
+    check_logprob(dh, wl, rows)
+    check_draft(dh, wl, rows)
+    dh.close()
+
+
+def test_fp32_io_at_the_training_width():
+    """fp32 hidden states and weights at d = 4096 (the library rounds them on the device), several m-tiles, ragged tail."""
+    shape = I.HeadShape(I.CP, 2, 4, 320, 4096, I.F32)
+    wl = I.make_workload("f32io_wide", shape, 300, seed=78, wpp=1)
+    dh = DeviceHead(wl)
+    rows = np.arange(wl.T)
     check_logprob(dh, wl, rows)
     check_draft(dh, wl, rows)
     dh.close()

@@ -20,6 +20,7 @@ pytestmark = pytest.mark.gpu
 
 LOGPROB_TOL = 2e-3
 BOUNDARY_BAND = 1e-6       # draft draws (as in test_gpu_parity.py)
+OWN_ALPHA_BAND = 1e-5
 ALPHA_BAND = 2e-4          # |alpha - p/q| of an acceptance test
 FINAL_BAND = 1e-4          # distance of the last draw to a boundary of the residual CDF, times Z
 FULL_BAND = 1e-5           # the same for a draw from a target row (both sides read the same fp32 row)
@@ -148,6 +149,21 @@ def check_accept(wl, wpp):
     assert not bad.any(), (np.nonzero(bad)[0][:5], acc_g[bad][:5], ref["accepted"][bad][:5], next_g[bad][:5],
                            ref["next_byte"][bad][:5])
     assert comparable.sum() >= 0.9 * W
+    # The same decisions taken by the oracle from the DEVICE's own draft and prefix marginals: both sides then test
+    # alpha against the same 32-bit numbers, the device as alpha * q > p in fp32, the oracle as alpha > p / q in fp64, so
+    # the length of the accepted prefix must agree for every window whose closest test is further than 1e-5 from flipping
+    # (two fp32 roundings of numbers below 1); only the last byte's draw keeps the wider band of the residual weights.
+    own = orc.speculative_accept(prefix_g.cpu().numpy().astype(np.float64), gb, p, ua,
+                                 lambda r_, s_: orc.next_byte_logprob(s.family, logw, logphi, wl.T_static, gb[r_], s_, pos[r_]))
+    tight = own["margin_alpha"] >= OWN_ALPHA_BAND
+    assert (acc_g[tight] == own["accepted"][tight]).all(), np.nonzero(tight & (acc_g != own["accepted"]))[0][:5]
+    own_final = np.where(own["accepted"] == n, own["margin_final"] < FULL_BAND,
+                         own["margin_final"] * own["resid_mass"] < FINAL_BAND)
+    cmp_byte = tight & ~own_final
+    assert (next_g[cmp_byte] == own["next_byte"][cmp_byte]).all()
+    print(f"{wl.name}: against the oracle run on the device's own marginals: {int((~tight).sum())} of {W} windows within "
+          f"{OWN_ALPHA_BAND} of flipping a test, {int((tight & own_final).sum())} more with the last draw inside its band")
+    assert tight.sum() >= 0.98 * W
     if W >= 64:
         assert hist[n] > 0 and hist[:n].sum() > 0        # the case exercises full acceptance and rejection
     dh.close()

@@ -149,3 +149,32 @@ def test_undiscounted_eq6_gradient_is_the_mean_nll_gradient(family):
     gj = og.window_logprob_grad(family, h, W, R, Ts, x, np.full(N * L, -1.0 / (N * L)))
     for name in ("dh", "dW_emit", "dW_sum"):
         np.testing.assert_allclose(g6[name], gj[name], atol=1e-12)
+
+
+@pytest.mark.parametrize("family,n,r,v", CASES)
+def test_logit_gradients_chain_to_the_parameter_gradients(family, n, r, v):
+    """window_logprob_logit_grad: pushed through the two projections by hand (dW = dlogit^T h, dh = dlogit W + dslog R), the
+    gradients with respect to the logits must give the parameter gradients that finite differences already pin; and
+    for a rank-one mixture they have the closed form weight * (onehot - softmax)."""
+    rng = np.random.default_rng(1700 + 10 * family + n)
+    h, W, R, Ts, x, wt = tiny(rng, family, n, r, v)
+    x[1, 0] = -1
+    full = og.window_logprob_grad(family, h, W, R, Ts, x, wt)
+    lg = og.window_logprob_logit_grad(family, h, W, R, Ts, x, wt)
+    T, d = h.shape
+    dl = lg["dlogit"].reshape(T, n * r * v)
+    ds = lg["dslog"].reshape(T, -1)
+    np.testing.assert_allclose(dl.T @ h, full["dW_emit"].reshape(n * r * v, d), atol=1e-12)
+    np.testing.assert_allclose(ds.T @ h, full["dW_sum"], atol=1e-12)
+    np.testing.assert_allclose(dl @ W.reshape(n * r * v, d) + ds @ R, full["dh"], atol=1e-12)
+    assert np.abs(lg["dlogit"][1, 0]).max() == 0.0            # the marginalised byte: no gradient into its logits
+    if family == CP and r == 1:
+        logits = np.einsum("td,nvd->tnv", h, W[:, 0])
+        soft = scipy.special.softmax(logits, axis=-1)
+        onehot = np.zeros_like(soft)
+        for t in range(T):
+            for i in range(n):
+                if x[t, i] >= 0:
+                    onehot[t, i, x[t, i]] = 1.0
+        want = wt[:, None, None] * (onehot - soft) * (x >= 0)[:, :, None]
+        np.testing.assert_allclose(lg["dlogit"][:, :, 0, :], want, atol=1e-12)
