@@ -70,10 +70,11 @@ typedef struct {
   int32_t n;                   /* window length. BTREE: a power of two >= 2                            */
   int32_t r;                   /* units per layer (mixture components / hidden states): a power of two,
                                   <= 128 for CP, <= 32 for HMM and BTREE                               */
-  int32_t v;                   /* vocabulary: a multiple of 16. Up to 512 (splittable into equal chunks of
-                                  <= 256 columns that are multiples of 16: 256 and 320 are) everything
-                                  works; larger vocabularies evaluate and train (the softmax runs online
-                                  across accumulator tiles) but the draft calls return UNSUPPORTED        */
+  int32_t v;                   /* vocabulary: a multiple of 16, any size the n*r*v <= 2^30 limit admits (a unit of
+                                  up to 512 symbols is sampled out of tensor memory in one go; wider units are
+                                  streamed through it twice and, on more than 128 positions, always with the
+                                  draws sorted by unit). v = 272 and the like (no split into equal 16-aligned
+                                  tiles of <= 256 columns) draft on up to 128 positions per call only              */
   int32_t d;                   /* hidden size: a multiple of 64                                        */
   int32_t io_dtype;            /* MTPC_F32 | MTPC_BF16: dtype of hidden, W_emit and W_sum              */
   int32_t max_positions;       /* upper bound on T (log-prob) and P (draft) per call                   */

@@ -24,7 +24,7 @@ using namespace mtpc;
 constexpr size_t kAlign = 256;
 constexpr int kMaxPhases = 5;
 constexpr size_t kSlotSmemLimit = 160 * 1024;   // latent-draw tables of the draft slot kernel kept in shared memory up to this
-constexpr int kMaxDraftVocab = 512;     // draft sampling: the v logits of a unit live in 512 TMEM columns / 16 per lane
+constexpr int kMaxDraftVocab = 512;     // many-position draft: the v logits of a unit live in 512 TMEM columns
 constexpr int kHostChunkPositions = 2048;   // host-buffer calls upload and process this many positions at a time
 constexpr int kWorkCounterWord = 16;   // word of the 256-byte status area used as the circuit kernels' work counter
 constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA on sm_100
@@ -60,6 +60,7 @@ struct Layout {
   int decode_max_p;     // positions the few-position draft path can take (0: path not available)
   bool can_draft;       // v <= 512: the sampling kernels hold a whole input unit on chip
   bool can_draft_many;  // the sampling epilogue of the projection kernel can tile a unit (draft of more than 128 positions)
+  bool sample_two_pass; // ... but only by streaming the unit's tiles through tensor memory twice (v > 512): draws sorted by unit
   size_t off_h_hidden, off_h_targets, off_h_uniforms, off_h_bytes, off_h_out;
   // grouped sampling pass of the many-position draft (0 entries: not available)
   size_t group_entries;   // (window, slot) pairs that can be staged at once
@@ -115,9 +116,10 @@ int plan(const mtpc_config& c, Layout* L) {
   L->sum_tiles = (L->sum_rows + sum_cols - 1) / sum_cols;
   const int emit_units = c.n * c.r;
   // sampling: emission unit -> equal tiles of <= 256 columns, each a multiple of 16, all in TMEM at once
-  // (a unit of more than 512 bytes does not fit tensor memory: such heads evaluate and train, but do not draft)
-  L->can_draft = c.v <= kMaxDraftVocab;
-  if (L->can_draft) {
+  // (a unit of more than 512 symbols does not fit tensor memory: such heads draft through the few-position path only)
+  L->can_draft = true;
+  L->sample_two_pass = c.v > kMaxDraftVocab;
+  if (!L->sample_two_pass) {
     int chunks = (c.v + 255) / 256;
     while (c.v % chunks != 0 || (c.v / chunks) % 16 != 0) ++chunks;
     L->sm.tile_cols = c.v / chunks;
@@ -127,7 +129,12 @@ int plan(const mtpc_config& c, Layout* L) {
     // (no such split, e.g. v = 272 = 17 x 16: only the few-position draft path, which needs none, is available)
     L->can_draft_many = fit_tiling(&L->sm, sum_cols) && L->sm.num_slots >= chunks;
   } else {
-    L->can_draft_many = false;
+    // 256-column tiles, the last one ragged (its tail columns are masked), streamed through two accumulator slots
+    L->sm.tile_cols = 256;
+    L->sm.group_units = 1;
+    L->sm.group_tiles = (c.v + 255) / 256;
+    L->sm.num_groups = emit_units;
+    L->can_draft_many = fit_tiling(&L->sm, sum_cols);
   }
   if (!L->can_draft_many) memset(&L->sm, 0, sizeof(L->sm));
   // log-likelihood: 256-column tiles; a group is the shortest run of whole units that is a whole number of tiles
@@ -408,6 +415,7 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
     p.group_tiles = grp->tiles;
     p.group_num_tiles = grp->num_tiles;
     p.group_perm = grp->perm;
+    p.group_two_pass = L.sample_two_pass ? 1 : 0;
     p.unit_sel = grp->unit_sel;
   }
   p.uniforms = uniforms;
@@ -640,7 +648,8 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
       const size_t base = static_cast<size_t>((2 * c.r + 3) & ~3) * sizeof(float);
       const size_t with_tables = base + static_cast<size_t>(chain) * c.r * c.r * sizeof(float);
       const int in_smem = chain > 0 && with_tables <= kSlotSmemLimit;
-      launch_kernel(draft_slot_kernel, dim3(c.n, P), kSlotThreads, in_smem ? with_tables : base, st, h->ring == 0, c.family,
+      launch_kernel(c.v > kMaxDraftVocab ? draft_slot_kernel<true> : draft_slot_kernel<false>, dim3(c.n, P), kSlotThreads,
+                    in_smem ? with_tables : base, st, h->ring == 0, c.family,
                     at<float>(h, L.off_logits), at<float>(h, L.off_logw), hmm_tables(h), uniforms, out_bytes,
                     at<float>(h, L.off_G), at<float>(h, L.off_unit_lse), at<unsigned>(h, L.off_status),
                     at<unsigned>(h, L.off_status) + kWorkCounterWord, wpp, c.n, c.r, c.v, valid_symbols(c), L.sum_rows,
@@ -671,7 +680,9 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   if ((rc = check_launch()) != MTPC_OK) return rc;
   // 3. byte draws at the selected input units. With few windows per position against many units per slot the draws
   // are first sorted by unit, so that every window is multiplied by the one unit it samples from.
-  const bool grouped = L.group_entries > 0 && h->draft_grouping != 1 && (h->draft_grouping == 2 || wpp * 4 <= c.r);
+  if (L.sample_two_pass && L.group_entries == 0) return MTPC_ERR_UNSUPPORTED;
+  const bool grouped = L.sample_two_pass ||
+                       (L.group_entries > 0 && h->draft_grouping != 1 && (h->draft_grouping == 2 || wpp * 4 <= c.r));
   if (grouped) {
     const int units = c.n * c.r;
     int* ints = at<int>(h, L.off_grp_ints);
@@ -1012,7 +1023,9 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
           cudaSuccess;
   fail |= cudaFuncSetAttribute(mtpc_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
           cudaSuccess;
-  fail |= cudaFuncSetAttribute(draft_slot_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  fail |= cudaFuncSetAttribute(draft_slot_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               static_cast<int>(kSlotSmemLimit)) != cudaSuccess;
+  fail |= cudaFuncSetAttribute(draft_slot_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                static_cast<int>(kSlotSmemLimit)) != cudaSuccess;
   fail |= !set_circuit_attributes();
   fail |= !allow_full_smem(spec_accept_kernel);
@@ -1087,10 +1100,14 @@ int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32
   const Layout& L = head->L;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int W = P * wpp;
-  const size_t smem = kAcceptWarps * accept_warp_floats(c.family, c.n, c.r, c.v) * sizeof(float);
+  const size_t per_warp = accept_warp_floats(c.family, c.n, c.r, c.v) * sizeof(float);
+  int warps = kAcceptWarps;                               // wide vocabularies: fewer warps share the CTA's shared memory
+  while (warps > 1 && warps * per_warp > static_cast<size_t>(kSmemLimit)) warps >>= 1;
+  if (warps * per_warp > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;
+  const size_t smem = warps * per_warp;
   PhaseTimer pt(head, st);
   pt.begin();
-  spec_accept_kernel<<<(W + kAcceptWarps - 1) / kAcceptWarps, kAcceptWarps * 32, smem, st>>>(
+  spec_accept_kernel<<<(W + warps - 1) / warps, warps * 32, smem, st>>>(
       c.family, at<float>(head, L.off_logits), at<float>(head, L.off_unit_lse), at<float>(head, L.off_logw),
       hmm_tables(head), draft_bytes, prefix_logprob, target_probs, accept_uniforms, out_accepted,
       out_next_byte, at<unsigned>(head, L.off_status), W, wpp, c.n, c.r, c.v, valid_symbols(c), L.sum_rows,

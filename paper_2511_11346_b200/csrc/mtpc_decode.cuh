@@ -337,13 +337,69 @@ __device__ __forceinline__ const float* slot_chain_table(int family, const float
   return lw + r + static_cast<size_t>(node - 1) * r * r;
 }
 
+constexpr int kSlotMaxPerLane = 16;   // symbols a lane holds at a time: 512 per warp pass
+// Sum of exp(x[b] - m) over the symbols [c0, c0 + 512) that exist (b < vv); lane l takes l, l + 32, ... of the chunk.
+__device__ __forceinline__ float warp_chunk_sum(const float* __restrict__ x, int c0, int vv, float m, int lane) {
+  float xv[kSlotMaxPerLane];
+#pragma unroll
+  for (int q = 0; q < kSlotMaxPerLane; ++q) {
+    const int b = c0 + lane + 32 * q;
+    xv[q] = b < vv ? x[b] : -CUDART_INF_F;
+  }
+  float s = 0.f;
+#pragma unroll
+  for (int q = 0; q < kSlotMaxPerLane; ++q) s += __expf(xv[q] - m);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(kFull, s, off);
+  return s;
+}
+// Inverse CDF inside one chunk of 32 * per symbols starting at c0, on the weights exp(x[b] - m): lane l owns the
+// consecutive symbols [c0 + l*per, c0 + (l+1)*per). The threshold is u * (the chunk's total) when `relative`, else
+// `thr` itself. Returns the smallest symbol whose running sum exceeds the threshold; the last existing symbol of
+// the chunk if rounding leaves none. All lanes return the same value.
+__device__ __forceinline__ int warp_inv_cdf_chunk(const float* __restrict__ x, int c0, int per, int vv, float m, float thr,
+                                                  bool relative, int lane) {
+  const int b0 = c0 + lane * per;
+  float ev[kSlotMaxPerLane];
+#pragma unroll
+  for (int q = 0; q < kSlotMaxPerLane; ++q) ev[q] = (q < per && b0 + q < vv) ? x[b0 + q] : -CUDART_INF_F;
+  float part = 0.f;
+#pragma unroll
+  for (int q = 0; q < kSlotMaxPerLane; ++q) {
+    ev[q] = __expf(ev[q] - m);
+    part += ev[q];
+  }
+  const float incl = warp_scan_incl(part, lane);
+  if (relative) thr *= __shfl_sync(kFull, incl, 31);
+  const unsigned hit = __ballot_sync(kFull, thr < incl);
+  int byte = min(c0 + 32 * per, vv) - 1;
+  if (hit) {
+    const int src = __ffs(hit) - 1;
+    int found = -1;
+    const float before = __shfl_up_sync(kFull, incl, 1);
+    if (lane == src) {
+      float cum = lane == 0 ? 0.f : before;
+#pragma unroll
+      for (int q = 0; q < kSlotMaxPerLane; ++q)
+        if (found < 0 && q < per && b0 + q < vv) {
+          cum += ev[q];
+          if (thr < cum) found = b0 + q;
+        }
+      if (found < 0) found = min(b0 + per, vv) - 1;   // the lane's total passed the threshold: its last byte
+    }
+    byte = __shfl_sync(kFull, found, src);
+  }
+  return byte;
+}
+
 // logA: HMM transition log-probabilities [n-1, r, r]; position p reads them at logA + p * logA_stride (stride 0:
 // one static set for all positions; stride sum_rows with logA = log omega + r: contextual tables, App. H).
 // grid = (n, P), 16 warps. Shared memory: 2 * r floats (max and log-sum-exp of each unit of the slot), then, when
 // tables_in_smem, the chain's tables (slot_chain_length * r * r floats), fetched by cp.async while the log-sum-exps
 // are computed, so that the data-dependent row reads of the latent draws do not each cost a trip to L2.
 // The log-sum-exps also go to unit_lse_out [P, n, r], so that later calls can turn the retained logits into log phi.
-constexpr int kSlotMaxPerLane = 16;   // v <= 512
+// WIDE: vocabularies of more than 512 symbols (a separate build: the narrow one keeps a unit's logits in 16 registers per lane).
+template <bool WIDE>
 __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     int family, const float* __restrict__ logits, const float* __restrict__ logw, const float* __restrict__ logA,
     const float* __restrict__ uniforms, int* __restrict__ out_bytes, float* __restrict__ G,
@@ -381,25 +437,33 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     cp_async_commit();
   }
 
-  // ---- log-sum-exp of every input unit of the slot: a lane's logits are fetched in one batch of independent loads
+  // ---- log-sum-exp of every input unit of the slot: a lane's logits are fetched in batches of independent loads
+  // (one batch covers 512 symbols; wider vocabularies take several, merged online)
+  constexpr int kChunk = kSlotMaxPerLane * 32;
   for (int k = warp; k < r; k += nwarps) {
     const float* x = row + static_cast<size_t>(k) * v;
-    float xv[kSlotMaxPerLane];
+    float m = -CUDART_INF_F, s = 0.f;
+    for (int c0 = 0; c0 < (WIDE ? v : 1); c0 += kChunk) {
+      float xv[kSlotMaxPerLane];
 #pragma unroll
-    for (int q = 0; q < kSlotMaxPerLane; ++q) {
-      const int b = lane + 32 * q;
-      xv[q] = b < vv ? x[b] : -CUDART_INF_F;   // [vv, v): padding symbols
+      for (int q = 0; q < kSlotMaxPerLane; ++q) {
+        const int b = c0 + lane + 32 * q;
+        xv[q] = b < vv ? x[b] : -CUDART_INF_F;   // [vv, v): padding symbols
+      }
+      float cm = xv[0];
+#pragma unroll
+      for (int q = 1; q < kSlotMaxPerLane; ++q) cm = fmaxf(cm, xv[q]);
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) cm = fmaxf(cm, __shfl_xor_sync(kFull, cm, off));
+      const float mn = fmaxf(m, cm);           // finite from the first chunk on (symbol 0 always exists)
+      float cs = 0.f;
+#pragma unroll
+      for (int q = 0; q < kSlotMaxPerLane; ++q) cs += __expf(xv[q] - mn);   // padding: exp(-inf) = 0
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) cs += __shfl_xor_sync(kFull, cs, off);
+      s = s * __expf(m - mn) + cs;             // first chunk: 0 * exp(-inf) = 0
+      m = mn;
     }
-    float m = xv[0];
-#pragma unroll
-    for (int q = 1; q < kSlotMaxPerLane; ++q) m = fmaxf(m, xv[q]);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, off));
-    float s = 0.f;
-#pragma unroll
-    for (int q = 0; q < kSlotMaxPerLane; ++q) s += __expf(xv[q] - m);   // padding: exp(-inf) = 0
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(kFull, s, off);
     if (lane == 0) {
       unit_max[k] = m;
       unit_lse[k] = m + __logf(s);
@@ -438,39 +502,27 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
           z = warp_inv_cdf_logp(lane < r ? tab[z * r + lane] : 0.f, r, u[node], lane);
         }
       }
-      // ---- inverse CDF over the v bytes of unit z: lane l owns bytes [l*per, (l+1)*per)
       const float* x = row + static_cast<size_t>(z) * v;
       const float m = unit_max[z];
-      const int b0 = lane * per;
-      float ev[kSlotMaxPerLane];
-#pragma unroll
-      for (int q = 0; q < kSlotMaxPerLane; ++q) ev[q] = (q < per && b0 + q < vv) ? x[b0 + q] : -CUDART_INF_F;
-      float part = 0.f;
-#pragma unroll
-      for (int q = 0; q < kSlotMaxPerLane; ++q) {
-        ev[q] = __expf(ev[q] - m);
-        part += ev[q];
-      }
-      const float incl = warp_scan_incl(part, lane);
-      const float total = __shfl_sync(kFull, incl, 31);
-      const float thr = ub * total;
-      const unsigned hit = __ballot_sync(kFull, thr < incl);
-      byte = vv - 1;   // rounding may leave no index: the last one
-      if (hit) {
-        const int src = __ffs(hit) - 1;
-        int found = -1;
-        const float before = __shfl_up_sync(kFull, incl, 1);
-        if (lane == src) {
-          float cum = lane == 0 ? 0.f : before;
-#pragma unroll
-          for (int q = 0; q < kSlotMaxPerLane; ++q)
-            if (found < 0 && q < per && b0 + q < vv) {
-              cum += ev[q];
-              if (thr < cum) found = b0 + q;
-            }
-          if (found < 0) found = min(b0 + per, vv) - 1;   // the lane's total passed the threshold: its last byte
+      if (!WIDE) {
+        // ---- inverse CDF over the v bytes of unit z: lane l owns bytes [l*per, (l+1)*per)
+        byte = warp_inv_cdf_chunk(x, 0, per, vv, m, ub, true, lane);
+      } else {
+        // ---- wide vocabulary: 512 symbols at a time. First the total (chunk sums in fp32, added up in fp64), then
+        // the chunk the threshold u * total falls into, then the draw inside that chunk.
+        double total = 0.0;
+        for (int c0 = 0; c0 < v; c0 += kChunk) total += static_cast<double>(warp_chunk_sum(x, c0, vv, m, lane));
+        const double thr = static_cast<double>(ub) * total;
+        double before = 0.0;
+        byte = vv - 1;                           // rounding may leave no index: the last one
+        for (int c0 = 0; c0 < v; c0 += kChunk) {
+          const float cs = warp_chunk_sum(x, c0, vv, m, lane);
+          if (thr < before + static_cast<double>(cs)) {
+            byte = warp_inv_cdf_chunk(x, c0, kSlotMaxPerLane, vv, m, static_cast<float>(thr - before), false, lane);
+            break;
+          }
+          before += static_cast<double>(cs);
         }
-        byte = __shfl_sync(kFull, found, src);
       }
     }
     if (lane == 0) out_bytes[w * n + i] = byte;
@@ -512,7 +564,7 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
     int logA_stride) {
   extern __shared__ float sm[];
   const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int w = blockIdx.x * kAcceptWarps + wib;
+  const int w = blockIdx.x * (blockDim.x >> 5) + wib;    // up to kAcceptWarps warps per CTA (fewer for wide vocabularies)
   if (w >= W) return;
   float* mres = sm + static_cast<size_t>(wib) * accept_warp_floats(family, n, r, v);
   const int pos = w / wpp;

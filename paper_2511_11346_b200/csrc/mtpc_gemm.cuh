@@ -79,6 +79,7 @@ struct GemmParams {
   const GroupTile* group_tiles;      // grouped sampling: the work items, ...
   const int* group_num_tiles;        // ... how many there are (device memory: written by the kernel that made them), ...
   const int* group_perm;             // ... and which (window, slot) pair every row of the staged hidden states (tm_a) holds
+  int group_two_pass;                // grouped sampling of a unit too wide for tensor memory: its tiles are computed twice
   unsigned* status;
   uint64_t wait_limit_ns;            // limit of every pipeline wait (kWaitLimitNs unless a test shortened it)
 };
@@ -134,6 +135,7 @@ __device__ __forceinline__ bool bounded_wait_warp(uint32_t bar, uint32_t parity,
 struct TileCoord {
   int mt, is_sum, ntiles, cols, brow0, unit0, nunits;
   int arow, count;   // first row of the A operand and the rows that count (set by the caller for ungrouped items)
+  int wrap;          // tiles per sweep over the item's weight rows: tile t reads the rows of tile t % wrap
 };
 // A grouped item: `count` staged rows from `row0` on, against the tiles of the one unit they sample from.
 __device__ __forceinline__ TileCoord group_coord(const GemmParams& p, int item) {
@@ -145,7 +147,8 @@ __device__ __forceinline__ TileCoord group_coord(const GemmParams& p, int item) 
   c.nunits = 1;
   c.cols = p.tile_cols;
   c.brow0 = g.unit * p.v;
-  c.ntiles = p.v / p.tile_cols;
+  c.wrap = (p.v + p.tile_cols - 1) / p.tile_cols;
+  c.ntiles = p.group_two_pass ? 2 * c.wrap : c.wrap;
   c.arow = g.row0;
   c.count = g.count;
   return c;
@@ -243,6 +246,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
     TileCoord c = tile_coord(p, item);
     c.arow = (c.mt * CTAS + static_cast<int>(cta_rank)) * kBlockM;
     c.count = min(kBlockM, p.T - c.arow);                             // <= 0: a pair's second CTA past the last position
+    c.wrap = c.ntiles;
     return c;
   };
   const int first_item = CTAS == 2 ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
@@ -295,7 +299,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
           for (int kb = 0; kb < p.kblocks; ++kb) {
             if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
             const uint32_t a_dst = tiles_addr + stage * p.stage_bytes;
-            const int brow = tc.brow0 + t * tc.cols + static_cast<int>(cta_rank) * brows;
+            const int brow = tc.brow0 + (t % tc.wrap) * tc.cols + static_cast<int>(cta_rank) * brows;
             if (CTAS == 2) {
               const uint32_t full = cluster_map_shared(smem_u32(&ctl->full[stage]), 0);   // the leader's barrier
               if (cta_rank == 0) mbar_arrive_expect_tx(smem_u32(&ctl->full[stage]), bytes);
@@ -572,6 +576,70 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
           if (valid)
             for (int j = 0; j < nwin; ++j)
               if (p.unit_sel[(wrow0 + j) * p.n + slot_i] == k) pending |= 1ull << j;
+        }
+        if (MODE == kModeSampleGrouped && p.group_two_pass) {
+          // ---- a unit wider than tensor memory: its tiles stream through the accumulator ring twice. Sweep 1: running
+          // maximum and sum of exponentials (the sum in fp64, 16 terms at a time, so that tens of thousands of terms
+          // keep the precision the draw needs). Sweep 2: the scan u * total < running sum over the recomputed tiles.
+          const float uval = valid ? p.uniforms[wrow0 * (2 * p.n) + p.n + slot_i] : 0.f;
+          float m = -CUDART_INF_F;
+          double total = 0.0, cum = 0.0, thr = 0.0;
+          int found = p.vv - 1;   // rounding may leave no index: the last one
+          bool hit = false;
+          for (int t = 0; t < tc.ntiles && ok; ++t, ++use) {
+            const uint32_t slot = use % p.num_slots;
+            if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (use / p.num_slots) & 1u, ctl, p.status, lane)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t tcol = lane_base + slot * p.slot_stride;
+            const bool second = t >= tc.wrap;
+            if (t == tc.wrap) thr = static_cast<double>(uval) * total;
+            const int col_tile = (t % tc.wrap) * tc.cols;
+            for (int b = 0; b < nbatch && col_tile + b * 16 < p.vv; ++b) {
+              float x[16];
+              tmem_ld16(tcol + b * 16, x);
+              const int col0 = col_tile + b * 16;
+              mask_padding(x, col0, p.vv);
+              if (!second) {
+                float bm = x[0];
+#pragma unroll
+                for (int q = 1; q < 16; ++q) bm = fmaxf(bm, x[q]);
+                if (bm > m) {                                   // rescale what was summed so far to the new maximum
+                  total *= static_cast<double>(fast_ex2((m - bm) * kLog2e));
+                  m = bm;
+                }
+                const float m2 = m * kLog2e;
+                float part = 0.f;
+#pragma unroll
+                for (int q = 0; q < 16; ++q) part += fast_ex2(fmaf(x[q], kLog2e, -m2));
+                total += static_cast<double>(part);
+              } else if (!hit) {
+                const float m2 = m * kLog2e;
+                const float rest = static_cast<float>(thr - cum);   // what the threshold still needs inside this batch
+                float part = 0.f;
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                  part += fast_ex2(fmaf(x[q], kLog2e, -m2));
+                  if (!hit && rest < part) { hit = true; found = col0 + q; }
+                }
+                cum += static_cast<double>(part);
+              }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) release_slot(slot);
+          }
+          if (!ok) break;
+          if (valid) {
+            if (!(uval >= 0.f && uval < 1.f)) {
+              found = -1;
+              atomicOr(p.status, kStatusBadUniform);
+            }
+            p.out_bytes[wrow0 * p.n + slot_i] = found;
+          }
+          continue;
         }
         for (int c = 0; c < tc.ntiles && ok; ++c) {
           const uint32_t u = use + c;

@@ -129,6 +129,26 @@ def test_small_shapes_span_tiles_and_ragged_tails(family, n, r, v, d, T, wpp):
     dh.close()
 
 
+@pytest.mark.parametrize("family,n,r,v,vv,d,T,wpp", [
+    (I.CP, 2, 4, 1024, 0, 64, 6, 4),          # few positions: the per-slot kernel walks the unit 512 symbols at a time
+    (I.HMM, 2, 2, 4112, 4100, 64, 5, 3),      # padded vocabulary, 4100 symbols stored as 4112
+    (I.CP, 1, 2, 32768, 0, 64, 3, 4),         # a subword-sized vocabulary
+    (I.CP, 2, 4, 1024, 0, 64, 200, 1),        # many positions: units streamed through tensor memory twice, draws sorted by unit
+    (I.BTREE, 2, 2, 4112, 4100, 64, 150, 2),
+    (I.HMM, 2, 2, 32768, 0, 64, 140, 1),
+])
+def test_drafting_from_vocabularies_wider_than_tensor_memory(family, n, r, v, vv, d, T, wpp):
+    """More than 512 symbols per unit (App. G's subword case): log-likelihood, drafted bytes and draft log-probs against
+    the oracle, on the few-position and on the many-position path."""
+    wl = I.make_workload(f"widev_{v}_{T}", I.HeadShape(family, n, r, v, d, v_valid=vv), T, seed=2000 + v % 97 + T, wpp=wpp,
+                         weight_std=0.25)
+    dh = DeviceHead(wl)
+    rows = np.arange(T)
+    check_logprob(dh, wl, rows)
+    check_draft(dh, wl, rows)
+    dh.close()
+
+
 def test_fp32_io_at_the_training_width():
     """fp32 hidden states and weights at d = 4096 (the library rounds them on the device), several m-tiles, ragged tail."""
     shape = I.HeadShape(I.CP, 2, 4, 320, 4096, I.F32)
