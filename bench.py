@@ -262,7 +262,7 @@ def measure_backward(torch, dh, wl, hidden, targets, steps: int, peaks):
     lowrank = measure_lowrank(torch, wl, out[2], steps, peaks) if s.v <= 1536 else None
     return {"eq6_training_step": eq6, "lowrank_unembeddings": lowrank, "call": "mtpc_window_logprob_backward", "ms_per_call": ms, "positions_per_s": wl.T / (ms * 1e-3),
             "phase_ms": {"forward_projection": phase_ms[0], "circuit_backward": phase_ms[1],
-                         "logit_gradient": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]},
+                         "logit_gradient": phase_ms[2], "plain_gemms": phase_ms[3]},
             "flops_per_call": flops, "achieved_tflops": tf, "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
             "device_status": dh.head.mtpc_get_status()}
 
@@ -333,7 +333,7 @@ def measure_eq6_step(torch, dh, wl, hidden, targets, grads, steps: int):
     return {"call": "mtpc_window_loss_backward", "sequences": N, "sequence_length": L, "gamma": gamma, "ms_per_call": ms,
             "positions_per_s": wl.T / (ms * 1e-3), "loss": float(loss.cpu()[0]),
             "phase_ms": {"forward_prefix_loss": phase_ms[0], "circuit_backward_passes": phase_ms[1],
-                         "logit_gradient": phase_ms[2], "transposes_and_plain_gemms": phase_ms[3]}}
+                         "logit_gradient": phase_ms[2], "plain_gemms": phase_ms[3]}}
 
 
 CIRCUIT_KERNEL = {I.CP: "circuit_cp_kernel", I.HMM: "circuit_hmm_stream_kernel", I.BTREE: "circuit_btree_kernel",

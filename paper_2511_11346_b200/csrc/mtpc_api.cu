@@ -225,6 +225,22 @@ int make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, u
   return r == CUDA_SUCCESS ? MTPC_OK : MTPC_ERR_CUDA;
 }
 
+// bf16 matrix [rows, cols] row-major read as an MN-major operand (its columns are the operand's M or N index, its rows
+// the K index): boxes of 64 columns x 64 rows, 128-byte swizzle, zero fill outside.
+int make_tmap_mn(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return MTPC_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0 || (pitch * 2) % 16 != 0) return MTPC_ERR_WORKSPACE;
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstride[1] = {pitch * 2};
+  cuuint32_t box[2] = {64, static_cast<cuuint32_t>(kBlockK)};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MTPC_OK : MTPC_ERR_CUDA;
+}
+
 }  // namespace
 
 struct mtpc_head {
@@ -743,55 +759,54 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
 size_t round64(size_t x) { return (x + 63) / 64 * 64; }
 
 // Carving of the backward workspace for T positions (all buffers 256-byte aligned).
-// The sum-unit logit gradients sit to the right of the emission logit gradients in one matrix [T, Kd], Kd = Nc + Spad,
-// and W_sum^T to the right of W_emit^T in [d, Kd], so that d hidden is a single GEMM over K = Nc + S r.
+// The sum-unit logit gradients sit to the right of the emission logit gradients in one matrix [T, Kd], Kd = Nc + Spad.
 struct BackwardLayout {
-  size_t Nc, Spad, Tpad, Kd;
-  size_t off_lse, off_post, off_logits, off_dsum_t, off_dlogit, off_dlogit_t, off_wt, off_ht, off_dsum_f32, off_coeff, total;
+  size_t Nc, Spad, Kd;
+  size_t off_lse, off_post, off_logits, off_dlogit, off_dsum_f32, off_coeff, total;
 };
 void plan_backward(const mtpc_config& c, const Layout& L, int T, BackwardLayout* B) {
   B->Nc = static_cast<size_t>(c.n) * c.r * c.v;
   B->Spad = round64(L.sum_rows);
-  B->Tpad = round64(T);
   B->Kd = B->Nc + B->Spad;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
   B->off_lse = take(static_cast<size_t>(T) * c.n * c.r * 4);
   B->off_post = take(static_cast<size_t>(T) * c.n * c.r * 4);
   B->off_logits = take(static_cast<size_t>(T) * B->Nc * 4);              // [T, Nc] fp32: the emission logits of the forward pass
-  B->off_dsum_t = take(static_cast<size_t>(L.sum_rows) * B->Tpad * 2);  // [S r, Tpad] bf16
-  B->off_dlogit = take(static_cast<size_t>(T) * B->Kd * 2);          // [T, Nc | Spad]
-  B->off_dlogit_t = take(B->Nc * B->Tpad * 2);                       // [Nc, Tpad]
-  B->off_wt = take(static_cast<size_t>(c.d) * B->Kd * 2);            // [d, Nc | Spad]: W_emit^T | W_sum^T
-  B->off_ht = take(static_cast<size_t>(c.d) * B->Tpad * 2);          // hidden^T [d, Tpad]
+  B->off_dlogit = take(static_cast<size_t>(T) * B->Kd * 2);          // [T, Nc | Spad] bf16
   B->off_dsum_f32 = take(static_cast<size_t>(T) * L.sum_rows * 4);   // Eq. 6: sum-unit logit gradients accumulated over the passes
   B->off_coeff = take(static_cast<size_t>(T) * c.n * 4);             // Eq. 6: weights of the prefix marginals
   B->total = off;
 }
 
-int launch_transpose(mtpc_head* h, const void* src, void* dst, int rows, int cols, size_t src_pitch, size_t dst_pitch,
-                     cudaStream_t st) {
-  if (rows <= 0 || cols <= 0) return MTPC_OK;
-  dim3 grid((cols + 63) / 64, (rows + 63) / 64);
-  const int vec_ok = src_pitch % 8 == 0 && dst_pitch % 8 == 0 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0 &&
-                     (reinterpret_cast<uintptr_t>(dst) & 15u) == 0;
-  transpose_bf16_kernel<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), static_cast<__nv_bfloat16*>(dst),
-                                              rows, cols, src_pitch, dst_pitch, vec_ok);
-  h->launches++;
-  return check_launch();
-}
+// One operand of a plain GEMM: a bf16 matrix in device memory, either [rows = M or N, K] with K contiguous (K-major) or
+// [rows = K, M or N] with the M / N index contiguous (MN-major); pitch in elements.
+struct GemmOperand {
+  const void* ptr;
+  size_t pitch;
+  bool mn_major;
+};
 
-// C[M, N] fp32 (pitch ldc) = A[M, K] B[N, K]^T: A, B bf16 with K contiguous and row pitches lda, ldb (elements).
-int launch_plain_gemm(mtpc_head* h, const void* A, size_t lda, const void* Bm, size_t ldb, float* C, size_t ldc, int M,
-                      int N, int K, cudaStream_t st) {
-  if (M <= 0 || N <= 0 || K <= 0) return MTPC_OK;
+// C[M, N] fp32 (pitch ldc) = A B^T over K = K0 + K1: segment 0 multiplies A's K range [0, K0) with B0, segment 1 (K1 > 0)
+// A's K range [a_k1, a_k1 + K1) with B1.
+int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmOperand B1, int K1, int a_k1, float* C,
+                      size_t ldc, int M, int N, cudaStream_t st) {
+  if (M <= 0 || N <= 0 || K0 <= 0) return MTPC_OK;
+  if (K1 > 0 && (A.mn_major || B1.mn_major != B0.mn_major)) return MTPC_ERR_SHAPE;
   PlainGemmParams p;
   memset(&p, 0, sizeof(p));
-  int rc = make_tmap(&p.tm_a, A, M, K, kBlockM, lda);
-  if (rc == MTPC_OK) rc = make_tmap(&p.tm_b, Bm, N, K, kPlainTileN, ldb);
+  const int Ka = K1 > 0 ? a_k1 + K1 : K0;                      // extent of A along K
+  int rc = A.mn_major ? make_tmap_mn(&p.tm_a, A.ptr, Ka, M, A.pitch) : make_tmap(&p.tm_a, A.ptr, M, Ka, kBlockM, A.pitch);
+  if (rc == MTPC_OK)
+    rc = B0.mn_major ? make_tmap_mn(&p.tm_b[0], B0.ptr, K0, N, B0.pitch) : make_tmap(&p.tm_b[0], B0.ptr, N, K0, kPlainTileN, B0.pitch);
+  if (rc == MTPC_OK && K1 > 0)
+    rc = B1.mn_major ? make_tmap_mn(&p.tm_b[1], B1.ptr, K1, N, B1.pitch) : make_tmap(&p.tm_b[1], B1.ptr, N, K1, kPlainTileN, B1.pitch);
   if (rc != MTPC_OK) return rc;
   p.M = M; p.N = N;
-  p.kblocks = (K + kBlockK - 1) / kBlockK;
+  p.a_k0[0] = 0;
+  p.a_k0[1] = a_k1;
+  p.seg_kblocks[0] = (K0 + kBlockK - 1) / kBlockK;
+  p.seg_kblocks[1] = K1 > 0 ? (K1 + kBlockK - 1) / kBlockK : 0;
   p.m_tiles = (M + kBlockM - 1) / kBlockM;
   p.n_tiles = (N + kPlainTileN - 1) / kPlainTileN;
   p.stage_bytes = kABytes + kPlainTileN * kBlockK * 2;
@@ -805,7 +820,11 @@ int launch_plain_gemm(mtpc_head* h, const void* A, size_t lda, const void* Bm, s
   p.wait_limit_ns = h->wait_limit_ns;
   const long long items = static_cast<long long>(p.m_tiles) * p.n_tiles;
   const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
-  plain_gemm_kernel<<<grid, kGemmThreads, p.stages * p.stage_bytes + ctl, st>>>(p);
+  const size_t smem = p.stages * p.stage_bytes + ctl;
+  if (A.mn_major && B0.mn_major) plain_gemm_kernel<true, true><<<grid, kGemmThreads, smem, st>>>(p);
+  else if (!A.mn_major && B0.mn_major) plain_gemm_kernel<false, true><<<grid, kGemmThreads, smem, st>>>(p);
+  else if (!A.mn_major && !B0.mn_major) plain_gemm_kernel<false, false><<<grid, kGemmThreads, smem, st>>>(p);
+  else return MTPC_ERR_SHAPE;
   h->launches++;
   return check_launch();
 }
@@ -866,18 +885,15 @@ int set_backward_attributes(const mtpc_head* head) {
   return ok ? MTPC_OK : MTPC_ERR_CUDA;
 }
 
-// Phases 3 and 4 of a backward call: the logit gradients (post, lse and the kept logits -> bf16, both orientations), the
-// transposes and the plain GEMMs. The sum-unit logit gradients are already in place to the right of dlogit.
+// Phases 3 and 4 of a backward call: the logit gradients (post, lse and the kept logits -> bf16 rows) and the plain GEMMs.
+// The sum-unit logit gradients are already in place to the right of dlogit. Every GEMM operand is read where it lies:
+// the weights and the hidden states in the caller's buffers, the gradient matrix along its rows or down its columns.
 int backward_tail(mtpc_head* head, const BackwardLayout& B, uint8_t* bw, const void* hb, const int32_t* targets, int T,
                   float* d_hidden, float* dW_emit, float* dW_sum, PhaseTimer& pt, cudaStream_t st) {
   const mtpc_config& c = head->cfg;
   const Layout& L = head->L;
-  __nv_bfloat16* dsum_t = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dsum_t);
   __nv_bfloat16* dlogit = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit);
   __nv_bfloat16* dsum = dlogit + B.Nc;
-  __nv_bfloat16* dlogit_t = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit_t);
-  __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(bw + B.off_wt);
-  void* ht = bw + B.off_ht;
   const int Nc = static_cast<int>(B.Nc);
   pt.begin();
   LogitGradArgs la;
@@ -886,26 +902,31 @@ int backward_tail(mtpc_head* head, const BackwardLayout& B, uint8_t* bw, const v
   la.post = reinterpret_cast<const float*>(bw + B.off_post);
   la.targets = targets;
   la.dlogit = dlogit;
-  la.dlogit_t = dlogit_t;
   la.pitch = B.Kd;
-  la.t_pitch = B.Tpad;
   la.T = T; la.Nc = Nc; la.n = c.n; la.r = c.r; la.v = c.v;
-  logit_gradient_kernel<<<dim3((Nc + 63) / 64, (T + 63) / 64), 256, 0, st>>>(la);
+  {
+    const int col_blocks = (Nc / 8 + 255) / 256;
+    int row_blocks = (16 * head->num_sms + col_blocks - 1) / col_blocks;   // enough CTAs to fill the device, each walks rows
+    if (row_blocks > T) row_blocks = T;
+    if (row_blocks > 65535) row_blocks = 65535;
+    logit_gradient_kernel<<<dim3(col_blocks, row_blocks), 256, 0, st>>>(la);
+  }
   head->launches++;
   int rc = check_launch();
   pt.end();
   if (rc != MTPC_OK) return rc;
   pt.begin();
-  rc = launch_transpose(head, head->W_emit_bf16, wt, Nc, c.d, c.d, B.Kd, st);
-  if (rc == MTPC_OK) rc = launch_transpose(head, head->W_sum_bf16, wt + B.Nc, L.sum_rows, c.d, c.d, B.Kd, st);
-  if (rc == MTPC_OK) rc = launch_transpose(head, hb, ht, T, c.d, c.d, B.Tpad, st);
-  if (rc == MTPC_OK) rc = launch_transpose(head, dsum, dsum_t, T, L.sum_rows, B.Kd, B.Tpad, st);
-  // d hidden [T, d] = [dlogit | dsum] [T, Nc + S r] [W_emit ; W_sum] [Nc + S r, d]
-  if (rc == MTPC_OK)
-    rc = launch_plain_gemm(head, dlogit, B.Kd, wt, B.Kd, d_hidden, c.d, T, c.d, Nc + L.sum_rows, st);
+  const GemmOperand g_rows{dlogit, B.Kd, false};            // [T, Nc | S r] along its rows: K = the logit index
+  const GemmOperand g_cols{dlogit, B.Kd, true};             // the same matrix down its columns: K = the position
+  const GemmOperand s_cols{dsum, B.Kd, true};
+  const GemmOperand w_emit{head->W_emit_bf16, static_cast<size_t>(c.d), true};   // [Nc, d]: N = d contiguous
+  const GemmOperand w_sum{head->W_sum_bf16, static_cast<size_t>(c.d), true};
+  const GemmOperand hid{hb, static_cast<size_t>(c.d), true};                     // [T, d]: N = d contiguous, K = the position
+  // d hidden [T, d] = dlogit [T, Nc] W_emit [Nc, d] + dsum [T, S r] W_sum [S r, d]
+  rc = launch_plain_gemm(head, g_rows, w_emit, Nc, w_sum, L.sum_rows, Nc, d_hidden, c.d, T, c.d, st);
   // dW_emit [Nc, d] = dlogit^T [Nc, T] hidden [T, d];  dW_sum [S r, d] = dsum^T [S r, T] hidden [T, d]
-  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dlogit_t, B.Tpad, ht, B.Tpad, dW_emit, c.d, Nc, c.d, T, st);
-  if (rc == MTPC_OK) rc = launch_plain_gemm(head, dsum_t, B.Tpad, ht, B.Tpad, dW_sum, c.d, L.sum_rows, c.d, T, st);
+  if (rc == MTPC_OK) rc = launch_plain_gemm(head, g_cols, hid, T, hid, 0, 0, dW_emit, c.d, Nc, c.d, st);
+  if (rc == MTPC_OK) rc = launch_plain_gemm(head, s_cols, hid, T, hid, 0, 0, dW_sum, c.d, L.sum_rows, c.d, st);
   pt.end();
   return rc;
 }
@@ -1019,8 +1040,9 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   fail |= !allow_full_smem(mtpc_gemm_kernel<kModeLogprob, 2>);
   fail |= !allow_full_smem(mtpc_gemm_kernel<kModeSample, 2>);
   h->max_pairs = fail ? 0 : resident_pairs(L.lp.pair_smem);
-  fail |= cudaFuncSetAttribute(plain_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
-          cudaSuccess;
+  fail |= !allow_full_smem(plain_gemm_kernel<false, false>);
+  fail |= !allow_full_smem(plain_gemm_kernel<false, true>);
+  fail |= !allow_full_smem(plain_gemm_kernel<true, true>);
   fail |= cudaFuncSetAttribute(mtpc_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
           cudaSuccess;
   fail |= cudaFuncSetAttribute(draft_slot_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,

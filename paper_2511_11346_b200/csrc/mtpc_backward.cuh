@@ -9,9 +9,9 @@
 //      writes post[w, i, k] = weight * d log q / d G[w, i, k] (the posterior of "token i is emitted by unit k") and
 //      dsum[w, :] = weight * d log q / d (sum-unit logits), i.e. posterior minus prior of every sum unit, in bf16;
 //   3. logit_gradient_kernel (this file): dlogit = post * (onehot(target) - exp(logit - lse)), one streaming pass over
-//      the kept logits, written as bf16 in both orientations;
-//   4. plain bf16 GEMMs (plain_gemm_kernel, this file) on those: d hidden = dlogit W + dsum R, dW = dlogit^T h,
-//      dR = dsum^T h.
+//      the kept logits, written once as bf16 rows;
+//   4. plain bf16 GEMMs (plain_gemm_kernel, this file) on those, every operand read where it lies (the tensor cores
+//      take either orientation): d hidden = dlogit W + dsum R, dW = dlogit^T h, dR = dsum^T h.
 // Only the training calls materialise the logits (fp32, and their bf16 gradient, as the operands of the two weight-sized
 // GEMMs); recomputing them on chip instead was measured: a fourth weight-sized contraction against 0.6 ms of streaming.
 #pragma once
@@ -604,122 +604,60 @@ __global__ void f32_rows_to_bf16_kernel(const float* __restrict__ src, __nv_bflo
   }
 }
 
-// ---------------------------------------------------------------- bf16 transpose with a padded pitch
-// dst[c, r] = src[r, c] for r < rows, c < cols; dst rows have `dst_pitch` elements (>= rows; the padding is not written).
-// 64 x 64 tiles through shared memory, 256 threads. Inner tiles move 16 bytes per thread and request on both sides
-// (pitches and base addresses allow it: multiples of 8 elements); edge tiles fall back to element-wise copies.
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src,
-                                                             __nv_bfloat16* __restrict__ dst, int rows, int cols,
-                                                             size_t src_pitch, size_t dst_pitch, int vec_ok) {
-  __shared__ __align__(16) __nv_bfloat16 tile[64][72];
-  const int c0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
-  const bool inner = vec_ok && r0 + 64 <= rows && c0 + 64 <= cols;
-  if (inner) {
-    for (int e = threadIdx.x; e < 64 * 8; e += 256) {
-      const int rr_ = e >> 3, ch = e & 7;
-      *reinterpret_cast<uint4*>(&tile[rr_][ch * 8]) =
-          *reinterpret_cast<const uint4*>(src + static_cast<size_t>(r0 + rr_) * src_pitch + c0 + ch * 8);
-    }
-    __syncthreads();
-    for (int e = threadIdx.x; e < 64 * 8; e += 256) {
-      const int cc = e & 63, ch = e >> 6;              // consecutive threads: consecutive columns of the tile
-      __align__(16) __nv_bfloat16 v[8];
-#pragma unroll
-      for (int q = 0; q < 8; ++q) v[q] = tile[ch * 8 + q][cc];
-      *reinterpret_cast<uint4*>(dst + static_cast<size_t>(c0 + cc) * dst_pitch + r0 + ch * 8) =
-          *reinterpret_cast<const uint4*>(v);
-    }
-    return;
-  }
-  for (int e = threadIdx.x; e < 64 * 64; e += 256) {
-    const int rr_ = e / 64, cc = e % 64;
-    if (r0 + rr_ < rows && c0 + cc < cols) tile[rr_][cc] = src[static_cast<size_t>(r0 + rr_) * src_pitch + c0 + cc];
-  }
-  __syncthreads();
-  for (int e = threadIdx.x; e < 64 * 64; e += 256) {
-    const int cc = e / 64, rr_ = e % 64;
-    if (r0 + rr_ < rows && c0 + cc < cols) dst[static_cast<size_t>(c0 + cc) * dst_pitch + r0 + rr_] = tile[rr_][cc];
-  }
-}
-
 // ---------------------------------------------------------------- gradient with respect to the emission logits
 // dlogit[t, c] = post[t, u] * (onehot(target[t, i] == c - u v) - exp(logit[t, c] - lse[t, u])),  u = c / v = i r + k,
 // from the logits and log-sum-exps the forward pass kept (padding columns hold -inf: no mass, zero gradient; a
-// marginalised byte has no gradient). Written as bf16 in both orientations, the operands of the two weight-sized
-// GEMMs: dlogit [T, pitch] and dlogit_t [n r v, t_pitch] (columns T..round64(T) zero). 64 x 64 tiles, 256 threads:
-// a thread reads 4 adjacent logits (16 bytes) of 4 rows; the transposed copy goes through shared memory and leaves
-// as 16-byte pieces along t. v is a multiple of 16, so 4 adjacent columns belong to one unit.
+// marginalised byte has no gradient). Written once, as bf16 rows [T, pitch]: both weight-sized GEMMs read this one
+// matrix, d hidden along its rows (K-major) and dW down its columns (MN-major). One streaming pass: a thread converts
+// 8 adjacent logits (two 16-byte loads, one 16-byte store); v is a multiple of 16, so they belong to one unit.
 struct LogitGradArgs {
   const float* logits;       // [T, Nc], pitch Nc
   const float* lse;          // [T, n r]
   const float* post;         // [T, n r]
   const int* targets;        // [T, n]
   __nv_bfloat16* dlogit;     // [T, pitch]
-  __nv_bfloat16* dlogit_t;   // [Nc, t_pitch]
-  size_t pitch, t_pitch;
+  size_t pitch;
   int T, Nc, n, r, v;
 };
 
 __global__ void __launch_bounds__(256) logit_gradient_kernel(const LogitGradArgs a) {
-  // [column][row]; the rows of column c are rotated by 8 ((c / 4) mod 8) places so that the 16 threads of a row group,
-  // four columns apart, do not all fall on the same two banks
-  __shared__ __align__(16) __nv_bfloat16 tile[64][72];
-  const int c0 = blockIdx.x * 64, t0 = blockIdx.y * 64;
-  const int cg = (threadIdx.x & 15) * 4;                            // the thread's 4 columns within the tile
-  const int tr0 = (threadIdx.x >> 4) * 4;                           // and its 4 rows
-  const int rot = 8 * ((cg >> 2) & 7);
-  const int c = c0 + cg;
+  const int c = (blockIdx.x * 256 + threadIdx.x) * 8;
+  if (c >= a.Nc) return;
   const int units = a.n * a.r;
-  __align__(8) __nv_bfloat16 o[4][4];                               // [column][row]
+  const int u = c / a.v;
+  const int i = u / a.r;
+  const int col_in_unit = c - u * a.v;
+  for (int t = blockIdx.y; t < a.T; t += gridDim.y) {
+    const int tgt = a.targets[static_cast<size_t>(t) * a.n + i];
+    const size_t tu = static_cast<size_t>(t) * units + u;
+    const float pst = tgt >= 0 ? a.post[tu] : 0.f;
+    const float lse2 = a.lse[tu] * kLog2e;
+    const float4* src = reinterpret_cast<const float4*>(a.logits + static_cast<size_t>(t) * a.Nc + c);
+    const float4 x0 = __ldcs(src), x1 = __ldcs(src + 1);
+    const float xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+    const int rel = tgt - col_in_unit;
+    __align__(16) __nv_bfloat16 o[8];
 #pragma unroll
-  for (int pass = 0; pass < 4; ++pass) {
-    const int t = t0 + tr0 + pass;
-    __align__(8) __nv_bfloat16 orow[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) orow[q] = __float2bfloat16_rn(0.f);
-    if (t < a.T && c < a.Nc) {
-      const int u = c / a.v;
-      const int i = u / a.r;
-      const int tgt = a.targets[static_cast<size_t>(t) * a.n + i];
-      const size_t tu = static_cast<size_t>(t) * units + u;
-      const float pst = tgt >= 0 ? a.post[tu] : 0.f;
-      const float lse2 = a.lse[tu] * kLog2e;
-      const float4 x = __ldcs(reinterpret_cast<const float4*>(a.logits + static_cast<size_t>(t) * a.Nc + c));
-      const float xs[4] = {x.x, x.y, x.z, x.w};
-      const int rel = tgt - (c - u * a.v);
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        orow[q] = __float2bfloat16_rn(pst * ((rel == q ? 1.f : 0.f) - fast_ex2(fmaf(xs[q], kLog2e, -lse2))));
-      *reinterpret_cast<uint2*>(a.dlogit + static_cast<size_t>(t) * a.pitch + c) = *reinterpret_cast<const uint2*>(orow);
-    }
-#pragma unroll
-    for (int q = 0; q < 4; ++q) o[q][pass] = orow[q];
-  }
-#pragma unroll
-  for (int q = 0; q < 4; ++q)
-    *reinterpret_cast<uint2*>(&tile[cg + q][(tr0 + rot) & 63]) = *reinterpret_cast<const uint2*>(o[q]);
-  __syncthreads();
-  // transposed copy: thread -> (column, 16 rows); rows beyond T carry zeros, those beyond the pitch are not written
-  const int cc = threadIdx.x >> 2, seg = (threadIdx.x & 3) * 16;
-  if (c0 + cc < a.Nc) {
-    const int crot = 8 * ((cc >> 2) & 7);
-    __nv_bfloat16* dst = a.dlogit_t + static_cast<size_t>(c0 + cc) * a.t_pitch + t0 + seg;
-#pragma unroll
-    for (int h = 0; h < 2; ++h)
-      if (static_cast<size_t>(t0 + seg + 8 * h + 8) <= a.t_pitch)
-        *reinterpret_cast<uint4*>(dst + 8 * h) = *reinterpret_cast<const uint4*>(&tile[cc][(seg + 8 * h + crot) & 63]);
+    for (int q = 0; q < 8; ++q)
+      o[q] = __float2bfloat16_rn(pst * ((rel == q ? 1.f : 0.f) - fast_ex2(fmaf(xs[q], kLog2e, -lse2))));
+    *reinterpret_cast<uint4*>(a.dlogit + static_cast<size_t>(t) * a.pitch + c) = *reinterpret_cast<const uint4*>(o);
   }
 }
 
 // ---------------------------------------------------------------- plain bf16 GEMM on the tcgen05 tensor cores
-// C[M, N] (fp32, row-major, pitch ldc) = A[M, K] B[N, K]^T; A and B bf16, K contiguous (K-major), read
-// through TMA descriptors with 64-element boxes (out-of-range rows and K columns read as zero). Same pipeline as the
+// C[M, N] (fp32, row-major, pitch ldc) = A[M, K] B[N, K]^T with bf16 operands read where they lie, in either
+// orientation: K-major (K contiguous in memory: 64-element K boxes of 128 or 256 rows) or MN-major (the M / N index
+// contiguous: 64 x 64 boxes, two for the 128 rows of A, four for the 256 columns of B). Out-of-range rows and
+// columns read as zero. The K axis may consist of two segments with a B matrix each (d hidden sums over the emission
+// rows and the sum-unit rows, which are separate matrices); A then continues at column a_k0[1]. Same pipeline as the
 // projection kernel: one persistent CTA per SM, warp 0 TMA producer, warp 1 MMA issuer (M=128, N=256 tiles, two TMEM
 // slots), warps 2..5 epilogue (one thread per row, 16 fp32 columns per step).
 struct PlainGemmParams {
-  CUtensorMap tm_a;      // A [M, K]  box 64 x 128
-  CUtensorMap tm_b;      // B [N, K]  box 64 x 256
-  int M, N, kblocks;
+  CUtensorMap tm_a;      // K-major: A [M, K], box 64 (k) x 128; MN-major: A^T [K, M], box 64 (m) x 64 (k)
+  CUtensorMap tm_b[2];   // per K segment. K-major: B [N, K], box 64 (k) x 256; MN-major: B^T [K, N], box 64 (n) x 64 (k)
+  int a_k0[2];           // K coordinate of A at which each segment starts (multiples of 8)
+  int seg_kblocks[2];    // 64-wide K blocks per segment (segment 1: 0 if unused)
+  int M, N;
   int m_tiles, n_tiles;
   int stages, stage_bytes;
   int wide_stores;       // C and ldc allow 32-byte stores
@@ -729,7 +667,9 @@ struct PlainGemmParams {
   uint64_t wait_limit_ns;   // limit of every pipeline wait
 };
 constexpr int kPlainTileN = 256;
+constexpr uint32_t kMnBoxBytes = 64 * kBlockK * 2;   // one 64 x 64 bf16 box: 8 KB
 
+template <bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __grid_constant__ PlainGemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -741,6 +681,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
   // n-tile fastest: the CTAs running together cover a few m-tiles x all n-tiles, so the (larger) A operand is
   // streamed from HBM once and the B operand once per wave of m-tiles
   const int num_items = p.m_tiles * p.n_tiles;
+  const int kblocks = p.seg_kblocks[0] + p.seg_kblocks[1];
   constexpr uint32_t kSlots = 2;
   constexpr uint32_t kBBytes = kPlainTileN * kBlockK * 2;
 
@@ -758,7 +699,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
     ctl->wait_limit_ns = p.wait_limit_ns;
     fence_mbar_init();
     tma_prefetch_desc(&p.tm_a);
-    tma_prefetch_desc(&p.tm_b);
+    tma_prefetch_desc(&p.tm_b[0]);
+    if (p.seg_kblocks[1] > 0) tma_prefetch_desc(&p.tm_b[1]);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
@@ -775,13 +717,27 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
       bool ok = true;
       for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
         const int nt = item % p.n_tiles, mt = item / p.n_tiles;
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        for (int kb = 0; kb < kblocks; ++kb) {
           if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
           const uint32_t full = smem_u32(&ctl->full[stage]);
           const uint32_t a_dst = tiles_addr + stage * p.stage_bytes;
+          const int seg = kb >= p.seg_kblocks[0] ? 1 : 0;
+          const int kloc = (kb - (seg ? p.seg_kblocks[0] : 0)) * kBlockK;      // K offset inside the segment
           mbar_arrive_expect_tx(full, kABytes + kBBytes);
-          tma_load_2d(a_dst, &p.tm_a, full, kb * kBlockK, mt * kBlockM);
-          tma_load_2d(a_dst + kABytes, &p.tm_b, full, kb * kBlockK, nt * kPlainTileN);
+          if (A_MN) {
+#pragma unroll
+            for (int q = 0; q < kBlockM / 64; ++q)
+              tma_load_2d(a_dst + q * kMnBoxBytes, &p.tm_a, full, mt * kBlockM + q * 64, p.a_k0[seg] + kloc);
+          } else {
+            tma_load_2d(a_dst, &p.tm_a, full, p.a_k0[seg] + kloc, mt * kBlockM);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int q = 0; q < kPlainTileN / 64; ++q)
+              tma_load_2d(a_dst + kABytes + q * kMnBoxBytes, &p.tm_b[seg], full, nt * kPlainTileN + q * 64, kloc);
+          } else {
+            tma_load_2d(a_dst + kABytes, &p.tm_b[seg], full, kloc, nt * kPlainTileN);
+          }
           issued_mask |= 1u << stage;
           phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
           if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
@@ -801,21 +757,25 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, use = 0;
       bool ok = true;
-      const uint32_t idesc = umma_idesc_bf16(kBlockM, kPlainTileN);
+      const uint32_t idesc = umma_idesc_bf16(kBlockM, kPlainTileN, A_MN, B_MN);
+      // descriptor advance per K=16 step, in 16-byte units: 32 bytes along a swizzled K-major row, two 8-row groups
+      // (2048 bytes) down an MN-major box
+      constexpr uint32_t kStepA = A_MN ? 128u : 2u, kStepB = B_MN ? 128u : 2u;
       for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++use) {
         const uint32_t slot = use % kSlots;
         if (!bounded_wait(smem_u32(&ctl->tempty[slot]), ((use / kSlots) & 1u) ^ 1u, ctl, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + slot * kPlainTileN;
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        for (int kb = 0; kb < kblocks; ++kb) {
           if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = tiles_addr + stage * p.stage_bytes;
-          const uint64_t a_desc = umma_smem_desc_sw128(a_addr);
-          const uint64_t b_desc = umma_smem_desc_sw128(a_addr + kABytes);
+          const uint64_t a_desc = A_MN ? umma_smem_desc_mn_sw128(a_addr, kMnBoxBytes) : umma_smem_desc_sw128(a_addr);
+          const uint64_t b_desc = B_MN ? umma_smem_desc_mn_sw128(a_addr + kABytes, kMnBoxBytes)
+                                       : umma_smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
           for (int kk = 0; kk < kBlockK / 16; ++kk)
-            umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+            umma_bf16(d_tmem, a_desc + kStepA * kk, b_desc + kStepB * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
           umma_commit(smem_u32(&ctl->empty[stage]));
           if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
         }

@@ -195,10 +195,25 @@ __device__ __forceinline__ uint64_t umma_smem_desc_sw128(uint32_t smem_addr) {
   d |= static_cast<uint64_t>(2) << 61;
   return d;
 }
+// The same for an MN-major bf16 tile (the M or N index is the contiguous one) as 64 x 64 TMA boxes with the 128-byte
+// swizzle: a box holds 64 K rows of 128 bytes (64 consecutive M/N elements), so groups of 8 K rows are 1024 bytes
+// apart (stride byte offset) and the boxes that continue the M/N axis follow each other at `mn_box_bytes` (leading
+// byte offset; 8192 for 64 K rows). One K=16 instruction step covers two groups of 8 rows: +2048 bytes.
+__device__ __forceinline__ uint64_t umma_smem_desc_mn_sw128(uint32_t smem_addr, uint32_t mn_box_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>(mn_box_bytes >> 4) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
 // Instruction descriptor, kind::f16: D fp32 (bits [4,6) = 1), A and B bf16 (bits [7,10) = [10,13) = 1),
-// both K-major (bits 15, 16 = 0), N>>3 in bits [17,23), M>>4 in bits [24,29).
-__host__ __device__ constexpr uint32_t umma_idesc_bf16(uint32_t M, uint32_t N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+// bit 15 / 16 = 1: A / B is MN-major (0: K-major), N>>3 in bits [17,23), M>>4 in bits [24,29).
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(uint32_t M, uint32_t N, bool a_mn_major = false,
+                                                       bool b_mn_major = false) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
+         ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
 // 32-byte global store (eight fp32 values to a 32-byte aligned address): one full sector per request.
