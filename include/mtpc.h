@@ -216,9 +216,8 @@ int mtpc_window_loss(mtpc_head* head, const void* hidden, const int32_t* targets
  *   weight        dev [T] fp32.
  *   bwd_workspace dev, 256-byte aligned, >= mtpc_backward_workspace_bytes(cfg, T): holds the units' log-sum-exps and
  *                 posteriors, the fp32 emission logits the forward pass keeps for the backward pass (T * n*r*v * 4
- *                 bytes), the bf16 gradient of the logits in both orientations (as many bytes again: the large
- *                 buffers) and transposed bf16 copies of W_emit, W_sum and hidden. Caller-owned, used only during the
- *                 call's work.
+ *                 bytes) and their bf16 gradient (half as many bytes again). The weights and hidden states are read
+ *                 where they lie (no transposed copies). Caller-owned, used only during the call's work.
  *   out_logprob   dev [T] fp32 or NULL: the forward value.
  *   d_hidden      dev [T, d] fp32;  dW_emit dev [n, r, v, d] fp32;  dW_sum dev [S*r, d] fp32: overwritten, not
  *                 accumulated.
@@ -300,13 +299,14 @@ int mtpc_get_status(mtpc_head* head, void* stream, uint32_t* out_flags);
  *   mtpc_window_prefix_logprob, mtpc_window_loss: as mtpc_window_logprob (the loss reduction is not timed).
  *   mtpc_speculative_accept: [0] the acceptance kernel.
  *   mtpc_window_logprob_backward: [0] forward projection, [1] circuit backward, [2] gradient of the logits,
- *                        [3] transposes and the plain GEMMs.
+ *                        [3] the three plain GEMMs.
  *   mtpc_window_loss_backward: [0] forward projection + prefix marginals + loss, [1] circuit backward (mixture:
  *                        one pass per prefix length; tree: the same passes in one launch; HMM: one reverse sweep),
  *                        [2] and [3] as above.
  *   mtpc_draft_sample, mtpc_draft_sample_prefix:   P <= 128 positions: [0] one pass over all weights (logits of every unit),
  *                        [1] per-slot latent + byte draws and evidence, [2] circuit evaluation.
- *                        Otherwise: [0] sum-unit GEMM, [1] latent sampling, [2] GEMM + inverse-CDF epilogue,
+ *                        Otherwise: [0] sum-unit GEMM, [1] latent sampling, [2] byte draws (GEMM + inverse-CDF
+ *                        epilogue; when the draws are sorted by unit: the sort, the staging copy and that GEMM),
  *                        [3] GEMM + gather epilogue on the drafted bytes, [4] circuit evaluation.
  */
 int mtpc_set_timing(mtpc_head* head, int32_t ring);
