@@ -487,9 +487,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
           }
           tc_fence_after();
           const uint32_t tcol = lane_base + slot * p.slot_stride;
-          for (int b = 0; b < nbatch && unit < units_end; ++b) {
+          // one batch of 16 accumulator columns of this row; false once the item's last unit has been closed
+          auto consume = [&](const uint32_t (&raw)[16], int b) -> bool {
             float x[16];
-            tmem_ld16(tcol + b * 16, x);
+#pragma unroll
+            for (int q = 0; q < 16; ++q) x[q] = __uint_as_float(raw[q]);
             mask_padding(x, col_in_unit, p.vv);
             if (p.logit_out != nullptr && valid) {                       // row of W_emit = column of the logit matrix
               float* l = p.logit_out + static_cast<size_t>(row) * p.logit_pitch + tc.brow0 + t * tc.cols + b * 16;
@@ -553,6 +555,25 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
                 tgt = (p.wpp == 1 && valid) ? p.targets[wrow0 * p.n + slot_i] : -1;
               }
             }
+            return unit < units_end;
+          };
+          // The load of the next batch is in flight while this one goes through the exponentials (two register buffers).
+          uint32_t ra[16], rb[16];
+          tmem_ld16_issue(tcol, ra);
+          tmem_ld_wait16(ra);
+          for (int b = 0;;) {
+            const bool more_b = b + 1 < nbatch;
+            if (more_b) tmem_ld16_issue(tcol + (b + 1) * 16, rb);
+            const bool go_a = consume(ra, b);
+            if (more_b) tmem_ld_wait16(rb);
+            if (!go_a || !more_b) break;
+            ++b;
+            const bool more_a = b + 1 < nbatch;
+            if (more_a) tmem_ld16_issue(tcol + (b + 1) * 16, ra);
+            const bool go_b = consume(rb, b);
+            if (more_a) tmem_ld_wait16(ra);
+            if (!go_b || !more_a) break;
+            ++b;
           }
           tc_fence_before();
           __syncwarp();

@@ -182,6 +182,25 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&x)[16]) {
   for (int i = 0; i < 16; ++i) x[i] = __uint_as_float(r[i]);
 }
 
+// The same load without the wait, and the wait on its own: a second load can be in flight while the first batch is
+// consumed. The wait takes the registers as operands so that nothing that reads them is scheduled ahead of it.
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
+      "%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait16(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :
+               : "memory");
+}
+
 // Shared-memory matrix descriptor for a K-major bf16 tile stored as rows of 128 bytes (64 elements) with the
 // 128-byte swizzle TMA writes: 8-row groups are 1024 bytes apart (stride byte offset); the leading byte
 // offset is not used by swizzled K-major layouts. Bits: [0,14) address>>4, [16,30) LBO>>4, [32,46) SBO>>4,
