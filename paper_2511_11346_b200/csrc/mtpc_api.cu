@@ -1122,14 +1122,11 @@ int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32
   const Layout& L = head->L;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int W = P * wpp;
-  const size_t per_warp = accept_warp_floats(c.family, c.n, c.r, c.v) * sizeof(float);
-  int warps = kAcceptWarps;                               // wide vocabularies: fewer warps share the CTA's shared memory
-  while (warps > 1 && warps * per_warp > static_cast<size_t>(kSmemLimit)) warps >>= 1;
-  if (warps * per_warp > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;
-  const size_t smem = warps * per_warp;
+  const size_t smem = accept_warp_floats(c.family, c.n, c.r, c.v) * sizeof(float);
+  if (smem > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;      // a residual row of more than ~56k symbols
   PhaseTimer pt(head, st);
   pt.begin();
-  spec_accept_kernel<<<(W + warps - 1) / warps, warps * 32, smem, st>>>(
+  spec_accept_kernel<<<W, kAcceptThreads, smem, st>>>(
       c.family, at<float>(head, L.off_logits), at<float>(head, L.off_unit_lse), at<float>(head, L.off_logw),
       hmm_tables(head), draft_bytes, prefix_logprob, target_probs, accept_uniforms, out_accepted,
       out_next_byte, at<unsigned>(head, L.off_status), W, wpp, c.n, c.r, c.v, valid_symbols(c), L.sum_rows,

@@ -534,17 +534,18 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
 }
 
 // ---------------------------------------------------------------- acceptance stage (Algorithm 3)
-constexpr int kAcceptWarps = 4;
+constexpr int kAcceptThreads = 256;
 
-// Per-warp shared memory of spec_accept_kernel, in floats: the residual weights of the v bytes, the weight and the
+// Shared memory of one CTA (= one window) of spec_accept_kernel, in floats: the residual weights of the v bytes, the weight and the
 // log-sum-exp of every input unit of the slot (2 r), and for the binary tree the product and sum-layer vectors of every
 // node, one staged table and one vector.
 __host__ __device__ inline size_t accept_warp_floats(int family, int n, int r, int v) {
-  return static_cast<size_t>(v) + 2 * static_cast<size_t>(r) +
+  return 4 + static_cast<size_t>(v) + 2 * static_cast<size_t>(r) +                // 4: the accepted length, for all warps
          (family == 2 ? 2 * static_cast<size_t>(n - 1) * r + static_cast<size_t>(r) * (r + 1) + r : 0);
 }
 
-// One warp per drafted window w (position p = w / wpp). Inputs: the draft's bytes and prefix log-marginals, the
+// One CTA per drafted window w (position p = w / wpp): warp 0 runs the tests and the short latent recursions, all
+// warps share the residual row (v bytes x r units of exponentials, the bulk of the work), warp 0 draws. Inputs: the draft's bytes and prefix log-marginals, the
 // target model's conditionals along the draft, one uniform per test plus one for the last byte; the logits and
 // per-unit log-sum-exps the draft call left in the workspace.
 //   1. s = 0; while s < n: the draft's conditional of byte s is q_s = exp(prefix[s] - prefix[s-1]) (prefix[-1] = 0);
@@ -556,17 +557,18 @@ __host__ __device__ inline size_t accept_warp_floats(int family, int n, int r, i
 //      from alpha_{s-1}; BTree: the upward pass with the bytes >= s summed out, then the downward pass along the
 //      path from the root to the node that owns token s.
 //   Both draws are inverse-CDF on unnormalised weights (u * total < running sum, index order, no division).
-__global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
+__global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
     int family, const float* __restrict__ logits, const float* __restrict__ unit_lse, const float* __restrict__ logw,
     const float* __restrict__ logA, const int* __restrict__ bytes, const float* __restrict__ prefix,
     const float* __restrict__ target, const float* __restrict__ uniforms, int* __restrict__ out_accepted,
     int* __restrict__ out_next, unsigned* status, int W, int wpp, int n, int r, int v, int vv, int sum_rows,
     int logA_stride) {
   extern __shared__ float sm[];
+  int& accepted_len = *reinterpret_cast<int*>(sm);       // s, or -1: the window's inputs were refused
   const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int w = blockIdx.x * (blockDim.x >> 5) + wib;    // up to kAcceptWarps warps per CTA (fewer for wide vocabularies)
+  const int w = blockIdx.x;
   if (w >= W) return;
-  float* mres = sm + static_cast<size_t>(wib) * accept_warp_floats(family, n, r, v);
+  float* mres = sm + 4;
   const int pos = w / wpp;
   const int* x = bytes + static_cast<size_t>(w) * n;
   const float* pre = prefix + static_cast<size_t>(w) * n;
@@ -575,6 +577,9 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
   const float* lw = logw + static_cast<size_t>(pos) * sum_rows;
   const bool has = lane < r;
 
+  float* cw = mres + v;                                  // [r] weight of every input unit of slot s
+  float* cl = cw + r;                                    // [r] its log-sum-exp
+  if (wib == 0) {
   // ---- 1. acceptance tests
   bool bad_u = false, bad_x = false;
   for (int c = lane; c <= n; c += 32) bad_u |= !(u[c] >= 0.f && u[c] < 1.f);
@@ -586,9 +591,9 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
       atomicOr(status, bad_u ? 2u : 1u);
       out_accepted[w] = -1;
       out_next[w] = -1;
+      accepted_len = -1;
     }
-    return;
-  }
+  } else {
   // lane i runs the test of byte i (all loads in flight at once); the first rejecting lane ends the accepted run
   int s = n;
   for (int base = 0; base < n && s == n; base += 32) {
@@ -601,19 +606,16 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
     const unsigned m = __ballot_sync(kFull, rej);
     if (m) s = base + __ffs(m) - 1;
   }
-  if (lane == 0) out_accepted[w] = s;
-  const float* trow = tp + static_cast<size_t>(s) * v;
-
-  if (s == n) {
-    for (int b = lane; b < v; b += 32) mres[b] = b < vv ? trow[b] : 0.f;
-  } else {
+  if (lane == 0) {
+    out_accepted[w] = s;
+    accepted_len = s;
+  }
+  if (s < n) {
     // ---- 2. c[k]: log-weight of input unit k of slot s given the accepted bytes (lane = k)
     auto g_of = [&](int i) -> float {   // log phi_{i,lane}(x_i)
       const size_t unit = (static_cast<size_t>(pos) * n + i) * r + lane;
       return logits[unit * v + x[i]] - unit_lse[unit];
     };
-    float* cw = mres + v;                                // [r] weight of every input unit of slot s
-    float* cl = cw + r;                                  // [r] its log-sum-exp
     float c = 0.f;
     if (family == 0) {
       // mixture of up to 128 components: lane handles k = lane, lane + 32, ...; the weights need no normalisation of
@@ -717,10 +719,19 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
         cl[lane] = unit_lse[(static_cast<size_t>(pos) * n + s) * r + lane];
       }
     }
-    __syncwarp();
+  }
+  }
+  }   // warp 0
+  __syncthreads();
+  const int s = accepted_len;
+  if (s < 0) return;
+  const float* trow = tp + static_cast<size_t>(s) * v;
+  // ---- residual weights of the v bytes, all warps
+  if (s == n) {
+    for (int b = threadIdx.x; b < v; b += kAcceptThreads) mres[b] = b < vv ? trow[b] : 0.f;
+  } else {
     const float* lrow = logits + (static_cast<size_t>(pos) * n + s) * r * v;   // [r, v] logits of slot s
-    for (int b0 = 0; b0 < v; b0 += 32) {
-      const int b = b0 + lane;
+    for (int b = threadIdx.x; b < v; b += kAcceptThreads) {
       float q = 0.f;
       if (b < vv) {
         // the r logits of byte b come from r different rows: eight loads in flight at a time, two accumulation chains
@@ -739,12 +750,13 @@ __global__ void __launch_bounds__(kAcceptWarps * 32) spec_accept_kernel(
         for (; k < r; ++k) q = fmaf(cw[k], __expf(lrow[static_cast<size_t>(k) * v + b] - cl[k]), q);
         q += q1;
       }
-      if (b < v) mres[b] = b < vv ? fmaxf(0.f, trow[b] - q) : 0.f;   // padding symbols carry no mass
+      mres[b] = b < vv ? fmaxf(0.f, trow[b] - q) : 0.f;   // padding symbols carry no mass
     }
   }
-  __syncwarp();
+  __syncthreads();
+  if (wib != 0) return;
 
-  // ---- 3. inverse CDF over the weights in mres: lane l owns bytes [l*per, (l+1)*per)
+  // ---- 3. inverse CDF over the weights in mres (warp 0): lane l owns bytes [l*per, (l+1)*per)
   const int per = (v + 31) / 32;
   const int b0 = lane * per;
   float part = 0.f;
