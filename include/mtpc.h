@@ -270,6 +270,29 @@ int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k,
                           const float* dW_emit, float* dW_base, float* dA, float* dB, void* stream);
 
 /*
+ * A head that keeps the shared unembeddings of App. G FACTORED: the emission logits are evaluated as
+ *   logit[t, i, j, :] = W_base[i] h_t + A[i, j] (B[i, j] h_t)
+ * without ever forming the composed [n, r, v, d] tensor: one contraction over d per slot (shared by its r components), a
+ * small one for z = B h, and a rank-k correction per component, 2 d (n v + n r k) + 4 n r v k FLOPs per position instead
+ * of 2 d n r v. z is handed to the tensor cores as two bf16 halves (z = hi + lo), so the result differs from exact
+ * arithmetic on the bf16 parameters only by fp32 accumulation (no rounding of a composed U to bf16).
+ *   cfg, W_sum, T_static, workspace, stream, out: as mtpc_create_head; cfg->io_dtype must be MTPC_BF16.
+ *   k        the adaptors' rank: 16 or 32 (MTPC_ERR_UNSUPPORTED otherwise; so are shapes whose base accumulator and two
+ *            correction slots do not fit the 512 columns of tensor memory: v up to 448).
+ *   W_base   dev [n, v, d] bf16;  A dev [n, r, v, k] bf16;  B dev [n, r, k, d] bf16: caller-owned, read in place, must
+ *            outlive the head (after an optimiser step no call is needed unless W_sum / T_static moved:
+ *            mtpc_update_parameters with W_emit = NULL then).
+ *   workspace >= mtpc_lowrank_workspace_bytes(cfg, k): the dense head's workspace plus z in fp32 and in bf16 halves.
+ * Such a head serves mtpc_window_logprob, mtpc_window_prefix_logprob, mtpc_window_loss and mtpc_window_logprob_host.
+ * Drafting, acceptance and the backward calls return MTPC_ERR_UNSUPPORTED on it: they run on the composed tensor
+ * (mtpc_lowrank_compose + mtpc_create_head, gradients carried back by mtpc_lowrank_backward).
+ */
+int mtpc_lowrank_workspace_bytes(const mtpc_config* cfg, int32_t k, size_t* out_bytes);
+int mtpc_create_head_lowrank(const mtpc_config* cfg, int32_t k, const void* W_base, const void* A, const void* B,
+                             const void* W_sum, const float* T_static, void* workspace, size_t workspace_bytes,
+                             void* stream, mtpc_head** out);
+
+/*
  * Host-buffer variants: same results, but hidden / targets / uniforms are HOST pointers (pinned memory for
  * full copy speed) and the outputs are written to HOST buffers. The copies to and from the device go through
  * staging areas in the workspace; the call returns after the stream has been synchronised, so the outputs are

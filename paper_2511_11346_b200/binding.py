@@ -24,7 +24,8 @@ EXPORTS = [
     "mtpc_window_prefix_logprob", "mtpc_draft_sample_prefix", "mtpc_speculative_accept", "mtpc_window_loss",
     "mtpc_backward_workspace_bytes", "mtpc_window_logprob_backward", "mtpc_window_loss_backward",
     "mtpc_lowrank_compose", "mtpc_lowrank_backward", "mtpc_update_parameters", "mtpc_debug_set_wait_limit_ns",
-    "mtpc_debug_set_projection_variant", "mtpc_debug_set_draft_grouping",
+    "mtpc_debug_set_projection_variant", "mtpc_debug_set_draft_grouping", "mtpc_lowrank_workspace_bytes",
+    "mtpc_create_head_lowrank",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 ERR_STATIC_SCRATCH = -7
@@ -82,6 +83,8 @@ def lib() -> ctypes.CDLL:
     L.mtpc_debug_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
     L.mtpc_debug_set_projection_variant.argtypes = [vp, i32]
     L.mtpc_debug_set_draft_grouping.argtypes = [vp, i32]
+    L.mtpc_lowrank_workspace_bytes.argtypes = [ctypes.POINTER(MtpcConfig), i32, ctypes.POINTER(sz)]
+    L.mtpc_create_head_lowrank.argtypes = [ctypes.POINTER(MtpcConfig), i32, vp, vp, vp, vp, vp, vp, sz, vp, ctypes.POINTER(vp)]
     L.mtpc_status_string.argtypes = [ctypes.c_int]
     L.mtpc_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -145,16 +148,30 @@ class MtpcHead:
     """Owns the opaque head handle and keeps the tensors the head points into alive."""
 
     def __init__(self, family: int, n: int, r: int, v: int, d: int, io_dtype: int, max_positions: int,
-                 max_windows_per_pos: int, W_emit, W_sum, T_static=None, stream=None, flags: int = 0, v_valid: int = 0):
+                 max_windows_per_pos: int, W_emit, W_sum, T_static=None, stream=None, flags: int = 0, v_valid: int = 0,
+                 lowrank=None):
+        """lowrank = (W_base, A, B) device bf16 tensors instead of W_emit (None): a factored head (mtpc_create_head_lowrank)."""
         import torch
         self.cfg = MtpcConfig(family, n, r, v, d, io_dtype, max_positions, max_windows_per_pos, flags, v_valid)
-        nbytes = mtpc_workspace_bytes(self.cfg)
-        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=W_emit.device)
-        self._keep = (W_emit, W_sum, T_static)
         handle = ctypes.c_void_p(0)
-        _check(lib().mtpc_create_head(ctypes.byref(self.cfg), _ptr(W_emit), _ptr(W_sum), _ptr(T_static),
-                                      self.workspace.data_ptr(), nbytes, _stream(stream), ctypes.byref(handle)),
-               "mtpc_create_head")
+        if lowrank is None:
+            nbytes = mtpc_workspace_bytes(self.cfg)
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=W_emit.device)
+            self._keep = (W_emit, W_sum, T_static)
+            _check(lib().mtpc_create_head(ctypes.byref(self.cfg), _ptr(W_emit), _ptr(W_sum), _ptr(T_static),
+                                          self.workspace.data_ptr(), nbytes, _stream(stream), ctypes.byref(handle)),
+                   "mtpc_create_head")
+        else:
+            W_base, A, Bm = lowrank
+            k = A.shape[-1]
+            need = ctypes.c_size_t(0)
+            _check(lib().mtpc_lowrank_workspace_bytes(ctypes.byref(self.cfg), k, ctypes.byref(need)),
+                   "mtpc_lowrank_workspace_bytes")
+            self.workspace = torch.empty(need.value, dtype=torch.uint8, device=W_sum.device)
+            self._keep = (W_base, A, Bm, W_sum, T_static)
+            _check(lib().mtpc_create_head_lowrank(ctypes.byref(self.cfg), k, _ptr(W_base), _ptr(A), _ptr(Bm), _ptr(W_sum),
+                                                  _ptr(T_static), self.workspace.data_ptr(), need.value, _stream(stream),
+                                                  ctypes.byref(handle)), "mtpc_create_head_lowrank")
         self.handle = handle
 
     # -- device-buffer calls

@@ -16,6 +16,7 @@
 #include "mtpc_decode.cuh"
 #include "mtpc_gemm.cuh"
 #include "mtpc_lowrank.cuh"
+#include "mtpc_lowrank_gemm.cuh"
 
 namespace {
 
@@ -225,6 +226,21 @@ int make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, u
   return r == CUDA_SUCCESS ? MTPC_OK : MTPC_ERR_CUDA;
 }
 
+// bf16 matrix [rows, cols] row-major -> tiles of box_rows x 16 elements (32-byte rows), 32-byte swizzle, zero fill outside.
+int make_tmap_sw32(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return MTPC_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0 || (cols * 2) % 16 != 0) return MTPC_ERR_WORKSPACE;
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstride[1] = {cols * 2};
+  cuuint32_t box[2] = {16, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MTPC_OK : MTPC_ERR_CUDA;
+}
+
 // bf16 matrix [rows, cols] row-major read as an MN-major operand (its columns are the operand's M or N index, its rows
 // the K index): boxes of 64 columns x 64 rows, 128-byte swizzle, zero fill outside.
 int make_tmap_mn(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch) {
@@ -253,6 +269,13 @@ struct mtpc_head {
   CUtensorMap tm_emit_lp2, tm_emit_sm2, tm_sum2; // the same with boxes of half the rows: what one CTA of a pair stages
   int projection_variant;                       // 0: chosen per launch; 1: every CTA alone; 2: CTA pairs (cta_group::2)
   int draft_grouping;                           // many-position draft: 0 chosen per call; 1 never sort the draws by unit; 2 always
+  // factored low-rank head (App. G; mtpc_create_head_lowrank): rank k > 0, no composed W_emit
+  int lr_k;
+  const void* lr_W_base;                        // [n, v, d] bf16
+  const void* lr_A;                             // [n, r, v, k] bf16
+  const void* lr_B;                             // [n, r, k, d] bf16
+  size_t lr_off_z32, lr_off_zhl;                // workspace: z = B h as fp32 [T, n r k], then split into bf16 halves [T, n r, 2, k]
+  LowRankGemmParams lr_params;                  // everything of the factored projection launch that does not depend on the call
   int max_pairs;                                // clusters of two projection CTAs that can be resident at once
   CUtensorMap tm_emit_dec, tm_sum_dec;          // the same matrices in the few-position draft path's tiles
   int decode_tile_rows, decode_sum_tile_rows;
@@ -619,6 +642,18 @@ int stage_hidden(mtpc_head* h, const void* hidden, int rows, const void** out_bf
   return MTPC_OK;
 }
 
+// One operand of a plain GEMM: a bf16 matrix in device memory, either [rows = M or N, K] with K contiguous (K-major) or
+// [rows = K, M or N] with the M / N index contiguous (MN-major); pitch in elements.
+struct GemmOperand {
+  const void* ptr;
+  size_t pitch;
+  bool mn_major;
+};
+
+int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmOperand B1, int K1, int a_k1, float* C,
+                      size_t ldc, int M, int N, cudaStream_t st);
+int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, const int* targets, cudaStream_t st);
+
 // out [T] (joint) and / or prefix [T, n] (prefix log-marginals); either may be NULL, not both.
 int window_logprob_impl(mtpc_head* h, const void* hidden, const int32_t* targets, int32_t T, float* out, float* prefix,
                         cudaStream_t st) {
@@ -628,7 +663,8 @@ int window_logprob_impl(mtpc_head* h, const void* hidden, const int32_t* targets
   if (rc != MTPC_OK) return rc;
   PhaseTimer pt(h, st);
   pt.begin();
-  rc = launch_gemm(h, kModeLogprob, hb, T, 1, true, true, targets, nullptr, nullptr, st);
+  if (h->lr_k > 0) rc = launch_lowrank_projection(h, hb, T, targets, st);
+  else rc = launch_gemm(h, kModeLogprob, hb, T, 1, true, true, targets, nullptr, nullptr, st);
   pt.end();
   if (rc != MTPC_OK) return rc;
   pt.begin();
@@ -643,7 +679,7 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
   const int W = P * wpp;
-  if (!L.can_draft) return MTPC_ERR_UNSUPPORTED;
+  if (!L.can_draft || h->lr_k > 0) return MTPC_ERR_UNSUPPORTED;   // (a factored low-rank head evaluates; drafting wants W_emit)
   const void* hb = nullptr;
   int rc = stage_hidden(h, hidden, P, &hb, st);
   if (rc != MTPC_OK) return rc;
@@ -779,14 +815,6 @@ void plan_backward(const mtpc_config& c, const Layout& L, int T, BackwardLayout*
   B->total = off;
 }
 
-// One operand of a plain GEMM: a bf16 matrix in device memory, either [rows = M or N, K] with K contiguous (K-major) or
-// [rows = K, M or N] with the M / N index contiguous (MN-major); pitch in elements.
-struct GemmOperand {
-  const void* ptr;
-  size_t pitch;
-  bool mn_major;
-};
-
 // C[M, N] fp32 (pitch ldc) = A B^T over K = K0 + K1: segment 0 multiplies A's K range [0, K0) with B0, segment 1 (K1 > 0)
 // A's K range [a_k1, a_k1 + K1) with B1.
 int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmOperand B1, int K1, int a_k1, float* C,
@@ -826,6 +854,69 @@ int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmO
   else if (!A.mn_major && !B0.mn_major) plain_gemm_kernel<false, false><<<grid, kGemmThreads, smem, st>>>(p);
   else return MTPC_ERR_SHAPE;
   h->launches++;
+  return check_launch();
+}
+
+// Tiling of the factored projection (mtpc_lowrank_gemm.cuh) for a head shape; false: the shape does not fit.
+bool plan_lowrank(const mtpc_config& c, int k, LowRankGemmParams* p) {
+  if (k < 16 || k > kLrMaxRank || k % 16 != 0 || c.v % 16 != 0) return false;
+  const int base_cols = (c.v + 31) / 32 * 32;
+  int chunk = (kTmemCols - base_cols) / 2 / 32 * 32;          // two correction slots beside the base accumulator
+  if (chunk > 256) chunk = 256;
+  if (chunk < 32) return false;
+  if (chunk > c.v) chunk = c.v;                                // (v < 32 never gets here with chunk < 16: v is a multiple of 16)
+  p->n = c.n; p->r = c.r; p->v = c.v; p->k = k;
+  p->vv = c.v_valid > 0 ? c.v_valid : c.v;
+  p->kblocks = c.d / kBlockK;
+  p->base_boxes = (c.v + 255) / 256;
+  if (c.v % p->base_boxes != 0 || (c.v / p->base_boxes) % 16 != 0) return false;
+  p->base_box_rows = c.v / p->base_boxes;
+  p->chunk_cols = chunk;
+  p->nchunk = (c.v + chunk - 1) / chunk;
+  p->corr_col0 = base_cols;
+  const int kq = k / 16;
+  const int base_entry = kABytes + c.v * kBlockK * 2;
+  const int corr_entry = 2 * kq * kBlockM * 32 + kq * p->nchunk * chunk * 32;
+  const int entry = base_entry > corr_entry ? base_entry : corr_entry;
+  p->stage_bytes = (entry + 1023) / 1024 * 1024;
+  const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
+  p->stages = (kSmemLimit - ctl) / p->stage_bytes;
+  if (p->stages > kMaxStages) p->stages = kMaxStages;
+  return p->stages >= 2;
+}
+
+// Factored projection of a low-rank head: log omega by the dense kernel's sum tiles, z = B h by a plain GEMM, its split
+// into bf16 halves, then the factored kernel writes G.
+int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, const int* targets, cudaStream_t st) {
+  const mtpc_config& c = h->cfg;
+  const Layout& L = h->L;
+  const int units = c.n * c.r, k = h->lr_k;
+  int rc = launch_gemm(h, kModeLogprob, hidden_bf16, T, 1, false, true, targets, nullptr, nullptr, st);
+  if (rc != MTPC_OK) return rc;
+  float* z32 = reinterpret_cast<float*>(h->ws + h->lr_off_z32);
+  __nv_bfloat16* zhl = reinterpret_cast<__nv_bfloat16*>(h->ws + h->lr_off_zhl);
+  const GemmOperand hid{hidden_bf16, static_cast<size_t>(c.d), false};
+  const GemmOperand bmat{h->lr_B, static_cast<size_t>(c.d), false};          // [n r k, d], K = d contiguous
+  rc = launch_plain_gemm(h, hid, bmat, c.d, bmat, 0, 0, z32, static_cast<size_t>(units) * k, T, units * k, st);
+  if (rc != MTPC_OK) return rc;
+  const size_t total = static_cast<size_t>(T) * units * k;
+  const int blocks = static_cast<int>((total + 255) / 256 < 8192 ? (total + 255) / 256 : 8192);
+  lowrank_split_kernel<<<blocks, 256, 0, st>>>(z32, zhl, static_cast<size_t>(T) * units, k);
+  LowRankGemmParams p = h->lr_params;
+  rc = make_tmap(&p.tm_h, hidden_bf16, static_cast<uint64_t>(T), static_cast<uint64_t>(c.d), kBlockM);
+  if (rc == MTPC_OK) rc = make_tmap_sw32(&p.tm_z, zhl, static_cast<uint64_t>(T), static_cast<uint64_t>(units) * 2 * k, kBlockM);
+  if (rc != MTPC_OK) return rc;
+  p.T = T;
+  p.m_tiles = (T + kBlockM - 1) / kBlockM;
+  p.targets = targets;
+  p.G = at<float>(h, L.off_G);
+  p.status = at<unsigned>(h, L.off_status);
+  p.wait_limit_ns = h->wait_limit_ns;
+  const long long items = static_cast<long long>(p.m_tiles) * c.n;
+  const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
+  const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
+  mtpc_lowrank_gemm_kernel<<<grid, kGemmThreads, p.stages * p.stage_bytes + ctl, st>>>(p);
+  h->launches += 2;
   return check_launch();
 }
 
@@ -983,14 +1074,16 @@ static int bind_parameters(mtpc_head* h, const void* W_emit, const void* W_sum, 
   }
   if (check_launch() != MTPC_OK) return MTPC_ERR_CUDA;
   const uint64_t emit_rows = static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v;
-  int rc = make_tmap(&h->tm_emit_lp, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols);
-  if (rc == MTPC_OK && L.can_draft_many) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
+  const bool dense = h->lr_k == 0;      // a factored low-rank head has no composed W_emit: only the sum-unit maps
+  int rc = MTPC_OK;
+  if (dense) rc = make_tmap(&h->tm_emit_lp, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols);
+  if (rc == MTPC_OK && dense && L.can_draft_many) rc = make_tmap(&h->tm_emit_sm, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols);
-  if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_lp2, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols / 2);
-  if (rc == MTPC_OK && L.can_draft_many) rc = make_tmap(&h->tm_emit_sm2, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols / 2);
+  if (rc == MTPC_OK && dense) rc = make_tmap(&h->tm_emit_lp2, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols / 2);
+  if (rc == MTPC_OK && dense && L.can_draft_many) rc = make_tmap(&h->tm_emit_sm2, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols / 2);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum2, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols / 2);
   h->decode_tile_rows = decode_tile_rows(static_cast<long long>(emit_rows), h->num_sms);
-  if (rc == MTPC_OK) rc = make_tmap(&h->tm_emit_dec, h->W_emit_bf16, emit_rows, cfg->d, h->decode_tile_rows);
+  if (rc == MTPC_OK && dense) rc = make_tmap(&h->tm_emit_dec, h->W_emit_bf16, emit_rows, cfg->d, h->decode_tile_rows);
   h->decode_sum_tile_rows = h->decode_tile_rows / 32 * 32;   // whole groups of r <= 32 rows per warp; fits the tile pitch
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum_dec, h->W_sum_bf16, L.sum_rows, cfg->d, h->decode_sum_tile_rows);
   h->draft_P = 0;                                              // logits left by an earlier draft belong to the old parameters
@@ -1008,13 +1101,42 @@ int mtpc_workspace_bytes(const mtpc_config* cfg, size_t* out_bytes) {
   return MTPC_OK;
 }
 
-int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_sum, const float* T_static,
-                     void* workspace, size_t workspace_bytes, void* stream, mtpc_head** out) {
-  if (!cfg || !W_emit || !W_sum || !workspace || !out) return MTPC_ERR_NULL;
+// lowrank: NULL for a dense head; else the rank and the three parameter tensors of App. G (W_emit is NULL then).
+struct LowRankSpec {
+  int k;
+  const void* W_base;
+  const void* A;
+  const void* B;
+};
+
+static int lowrank_extra_bytes(const mtpc_config& c, int k, size_t base_total, size_t* off_z32, size_t* off_zhl, size_t* total) {
+  const size_t units = static_cast<size_t>(c.n) * c.r;
+  size_t off = align_up(base_total);
+  *off_z32 = off;
+  off += align_up(static_cast<size_t>(c.max_positions) * units * k * 4);
+  *off_zhl = off;
+  off += align_up(static_cast<size_t>(c.max_positions) * units * 2 * k * 2);
+  *total = off;
+  return MTPC_OK;
+}
+
+static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const LowRankSpec* lowrank, const void* W_sum,
+                            const float* T_static, void* workspace, size_t workspace_bytes, void* stream, mtpc_head** out) {
+  if (!cfg || !W_sum || !workspace || !out) return MTPC_ERR_NULL;
+  if (!lowrank && !W_emit) return MTPC_ERR_NULL;
+  if (lowrank && (!lowrank->W_base || !lowrank->A || !lowrank->B)) return MTPC_ERR_NULL;
   *out = nullptr;
   Layout L;
   int rc = plan(*cfg, &L);
   if (rc != MTPC_OK) return rc;
+  LowRankGemmParams lrp;
+  memset(&lrp, 0, sizeof(lrp));
+  size_t lr_z32 = 0, lr_zhl = 0;
+  if (lowrank) {
+    if (cfg->io_dtype != MTPC_BF16) return MTPC_ERR_UNSUPPORTED;
+    if (!plan_lowrank(*cfg, lowrank->k, &lrp)) return MTPC_ERR_UNSUPPORTED;
+    lowrank_extra_bytes(*cfg, lowrank->k, L.total, &lr_z32, &lr_zhl, &L.total);
+  }
   const bool ctx = (cfg->flags & MTPC_FLAG_HMM_CONTEXTUAL) != 0;
   if (cfg->family == MTPC_HMM && cfg->n > 1 && !ctx && !T_static) return MTPC_ERR_NULL;
   if (workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0) return MTPC_ERR_WORKSPACE;
@@ -1029,6 +1151,15 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   h->L = L;
   h->ws = static_cast<uint8_t*>(workspace);
   h->wait_limit_ns = kWaitLimitNs;
+  if (lowrank) {
+    h->lr_k = lowrank->k;
+    h->lr_W_base = lowrank->W_base;
+    h->lr_A = lowrank->A;
+    h->lr_B = lowrank->B;
+    h->lr_off_z32 = lr_z32;
+    h->lr_off_zhl = lr_zhl;
+    h->lr_params = lrp;
+  }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   bool fail = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess;
   // the attribute is per function, not per head: always ask for the full 227 KB so that heads do not undo each other
@@ -1055,13 +1186,47 @@ int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_s
   if (fail) { delete h; return MTPC_ERR_CUDA; }
 
   rc = bind_parameters(h, W_emit, W_sum, T_static, st);
+  if (rc == MTPC_OK && lowrank) {
+    fail = !allow_full_smem(mtpc_lowrank_gemm_kernel);
+    rc = fail ? MTPC_ERR_CUDA
+              : make_tmap(&h->lr_params.tm_w, lowrank->W_base, static_cast<uint64_t>(cfg->n) * cfg->v, cfg->d,
+                          h->lr_params.base_box_rows);
+    if (rc == MTPC_OK)
+      rc = make_tmap_sw32(&h->lr_params.tm_a, lowrank->A, static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v, lowrank->k,
+                          h->lr_params.chunk_cols);
+  }
   if (rc != MTPC_OK) { delete h; return rc; }
   *out = h;
   return MTPC_OK;
 }
 
+int mtpc_create_head(const mtpc_config* cfg, const void* W_emit, const void* W_sum, const float* T_static,
+                     void* workspace, size_t workspace_bytes, void* stream, mtpc_head** out) {
+  if (!W_emit) return MTPC_ERR_NULL;
+  return create_head_impl(cfg, W_emit, nullptr, W_sum, T_static, workspace, workspace_bytes, stream, out);
+}
+
+int mtpc_lowrank_workspace_bytes(const mtpc_config* cfg, int32_t k, size_t* out_bytes) {
+  if (!cfg || !out_bytes) return MTPC_ERR_NULL;
+  Layout L;
+  int rc = plan(*cfg, &L);
+  if (rc != MTPC_OK) return rc;
+  LowRankGemmParams lrp;
+  if (cfg->io_dtype != MTPC_BF16 || !plan_lowrank(*cfg, k, &lrp)) return MTPC_ERR_UNSUPPORTED;
+  size_t a = 0, b = 0;
+  return lowrank_extra_bytes(*cfg, k, L.total, &a, &b, out_bytes);
+}
+
+int mtpc_create_head_lowrank(const mtpc_config* cfg, int32_t k, const void* W_base, const void* A, const void* B,
+                             const void* W_sum, const float* T_static, void* workspace, size_t workspace_bytes,
+                             void* stream, mtpc_head** out) {
+  const LowRankSpec spec{k, W_base, A, B};
+  return create_head_impl(cfg, nullptr, &spec, W_sum, T_static, workspace, workspace_bytes, stream, out);
+}
+
+
 int mtpc_update_parameters(mtpc_head* head, const void* W_emit, const void* W_sum, const float* T_static, void* stream) {
-  if (!head || !W_emit || !W_sum) return MTPC_ERR_NULL;
+  if (!head || !W_sum || (!W_emit && head->lr_k == 0)) return MTPC_ERR_NULL;   // a factored head has no W_emit to rebind
   const mtpc_config& c = head->cfg;
   if (c.family == MTPC_HMM && c.n > 1 && !(c.flags & MTPC_FLAG_HMM_CONTEXTUAL) && !T_static) return MTPC_ERR_NULL;
   return bind_parameters(head, W_emit, W_sum, T_static, static_cast<cudaStream_t>(stream));
@@ -1176,6 +1341,7 @@ int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int3
   if (rc != MTPC_OK) return rc;
   if (T == 0) return MTPC_OK;
   if (!hidden || !targets || !weight || !bwd_workspace || !d_hidden || !dW_emit || !dW_sum) return MTPC_ERR_NULL;
+  if (head->lr_k > 0) return MTPC_ERR_UNSUPPORTED;
   const mtpc_config& c = head->cfg;
   const bool static_hmm = c.family == MTPC_HMM && !is_ctx(head) && c.n > 1;
   if (static_hmm && !dT_static) return MTPC_ERR_NULL;
@@ -1232,6 +1398,7 @@ int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t
   if (T64 > head->cfg.max_positions) return MTPC_ERR_SHAPE;
   if (!hidden || !targets || !bwd_workspace || !out_slot_loss || !out_loss || !d_hidden || !dW_emit || !dW_sum)
     return MTPC_ERR_NULL;
+  if (head->lr_k > 0) return MTPC_ERR_UNSUPPORTED;
   const int T = static_cast<int>(T64);
   const mtpc_config& c = head->cfg;
   const Layout& L = head->L;

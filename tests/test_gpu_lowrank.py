@@ -132,3 +132,87 @@ def test_argument_checks():
     with pytest.raises(B.MtpcError) as e:
         B.mtpc_lowrank_compose(n, r, v, d, 0, w.data_ptr(), a.data_ptr(), b.data_ptr(), out.data_ptr())
     assert e.value.code == -2      # MTPC_ERR_SHAPE
+
+
+# --------------------------------------------------------------------------- the factored head (no composed tensor)
+FACTORED = [
+    # family, n, r, v, vv, d, k, T
+    (I.CP, 2, 4, 320, 0, 128, 16, 300),        # v = 320: the base in two 160-column halves, corrections in 96-column chunks
+    (I.CP, 3, 16, 256, 0, 192, 16, 129),       # v = 256: one base box, 128-column chunks
+    (I.HMM, 4, 8, 64, 0, 64, 32, 257),         # rank 32: two K steps per half
+    (I.BTREE, 4, 4, 48, 44, 64, 16, 70),       # padded vocabulary, tree circuit
+    (I.HMM_CTX, 3, 8, 320, 0, 128, 16, 200),   # contextual transitions: many sum tiles beside the factored projection
+    (I.CP, 1, 1, 16, 0, 64, 16, 5),            # the smallest everything
+]
+
+
+def _factored_case(family, n, r, v, vv, d, k, T, seed):
+    shape = I.HeadShape(family, n, r, v, d, v_valid=vv)
+    wl = I.make_workload(f"lr_{family}_{v}_{k}", shape, T, seed=seed, weight_std=0.25)
+    W, A, Bm = I.lowrank_parameters(n, r, v, d, k, seed=seed + 1, weight_std=0.25, adaptor_std=0.2)
+    return wl, W, A, Bm
+
+
+@pytest.mark.parametrize("family,n,r,v,vv,d,k,T", FACTORED)
+def test_factored_head_matches_the_composed_definition(family, n, r, v, vv, d, k, T):
+    """logit = W_i h + A_ij (B_ij h) evaluated without composing U: the window log-likelihood and the prefix marginals
+    must equal the oracle's on U = W_i + A_ij B_ij (fp64, composed from the same bf16 parameters) within 2e-3."""
+    wl, W, A, Bm = _factored_case(family, n, r, v, vv, d, k, T, seed=4100 + v + k + T)
+    sym = vv or v
+    U = O.lowrank_unembedding(W, A, Bm)[:, :, :sym, :]                     # the oracle never sees padding rows
+    fam = wl.shape.family
+    ref = O.window_logprob(fam, wl.hidden_q, U, wl.W_sum_q, wl.T_static, wl.targets)
+    ctx = family == I.HMM_CTX
+    W_sum = to_device_bf16(wl.W_sum_q)
+    Ts = torch.from_numpy(np.ascontiguousarray(wl.T_static)).cuda() if wl.T_static is not None else None
+    head = B.MtpcHead(B.MTPC_HMM if ctx else family, n, r, v, d, B.MTPC_BF16, T, 1, None, W_sum, Ts,
+                      flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0, v_valid=vv, lowrank=(_device(W), _device(A), _device(Bm)))
+    hidden = to_device_bf16(wl.hidden_q)
+    t = wl.targets.copy()
+    if T > 8 and n > 1:
+        t[3, 1] = -1                                                       # a marginalised byte
+        ref = O.window_logprob(fam, wl.hidden_q, U, wl.W_sum_q, wl.T_static, t)
+    targets = torch.from_numpy(t).cuda()
+    out = torch.empty(T, dtype=torch.float32, device="cuda")
+    for _ in range(2):                                                     # twice: the accumulator ring wraps between calls
+        head.mtpc_window_logprob(hidden, targets, out)
+        assert head.mtpc_get_status() == 0
+        err = np.abs(out.cpu().numpy() - ref).max()
+        assert err <= 2e-3, err
+    pre = torch.empty((T, n), dtype=torch.float32, device="cuda")
+    head.mtpc_window_prefix_logprob(hidden, targets, pre)
+    assert np.abs(pre[:, -1].cpu().numpy() - ref).max() <= 2e-3
+    # what the factored head does not do is refused, not approximated
+    with pytest.raises(B.MtpcError) as e:
+        head.mtpc_draft_sample(hidden, 1, torch.zeros((T, 2 * n), device="cuda"), torch.empty((T, n), dtype=torch.int32, device="cuda"), out)
+    assert e.value.code == -3
+    head.mtpc_destroy()
+
+
+def test_factored_head_agrees_with_the_dense_head_on_the_composed_tensor_and_refuses_other_ranks():
+    family, n, r, v, d, k, T = I.CP, 2, 4, 320, 256, 16, 260
+    wl, W, A, Bm = _factored_case(family, n, r, v, 0, d, k, T, seed=4999)
+    Wd, Ad, Bd = _device(W), _device(A), _device(Bm)
+    W_sum = to_device_bf16(wl.W_sum_q)
+    hidden = to_device_bf16(wl.hidden_q)
+    targets = torch.from_numpy(wl.targets).cuda()
+    fact = B.MtpcHead(family, n, r, v, d, B.MTPC_BF16, T, 1, None, W_sum, None, lowrank=(Wd, Ad, Bd))
+    U = lowrank_compose(Wd, Ad, Bd)                                        # bf16-rounded composition
+    dense = B.MtpcHead(family, n, r, v, d, B.MTPC_BF16, T, 1, U, W_sum, None)
+    a, b = torch.empty(T, device="cuda"), torch.empty(T, device="cuda")
+    fact.mtpc_window_logprob(hidden, targets, a)
+    dense.mtpc_window_logprob(hidden, targets, b)
+    # the dense head computes on U rounded to bf16 (2^-9 relative per entry, d = 256 terms per logit): a looser agreement
+    assert float((a - b).abs().max()) <= 5e-2
+    exact = O.window_logprob(family, wl.hidden_q, O.lowrank_unembedding(W, A, Bm), wl.W_sum_q, None, wl.targets)
+    assert np.abs(a.cpu().numpy() - exact).max() <= 2e-3
+    assert np.abs(a.cpu().numpy() - exact).max() <= np.abs(b.cpu().numpy() - exact).max() + 1e-4
+    fact.mtpc_destroy()
+    dense.mtpc_destroy()
+    cfg = B.MtpcConfig(family, n, r, v, d, B.MTPC_BF16, T, 1, 0, 0)
+    import ctypes
+    need = ctypes.c_size_t(0)
+    assert B.lib().mtpc_lowrank_workspace_bytes(ctypes.byref(cfg), 8, ctypes.byref(need)) == -3      # rank not 16 or 32
+    assert B.lib().mtpc_lowrank_workspace_bytes(ctypes.byref(cfg), 16, ctypes.byref(need)) == 0 and need.value > 0
+    big = B.MtpcConfig(family, n, r, 480, d, B.MTPC_BF16, T, 1, 0, 0)                                 # no room for the corrections
+    assert B.lib().mtpc_lowrank_workspace_bytes(ctypes.byref(big), 16, ctypes.byref(need)) == -3
