@@ -295,11 +295,53 @@ def measure_lowrank(torch, wl, dW_emit, steps: int, peaks, k: int = 16):
     bytes_c = 2 * nU + 2 * small                       # write U (bf16), read W, A, B once
     bytes_b = 4 * nU + 2 * small + 4 * small            # read dW_emit (fp32) once, read A, B, write the three gradients
     hbm = peaks["hbm_gbs"]
-    return {"rank": k, "compose_ms": ms_c, "compose_algorithmic_bytes": bytes_c,
-            "compose_frac_of_hbm": bytes_c / (ms_c * 1e-3) / 1e9 / hbm, "backward_ms": ms_b, "backward_kernels": 3,
-            "backward_algorithmic_bytes": bytes_b, "backward_frac_of_hbm": bytes_b / (ms_b * 1e-3) / 1e9 / hbm,
-            "note": "CUDA-core kernels: k multiply-adds per element keep the fp32 pipes, not HBM, busiest; the three "
-                    "gradient kernels each stream dW_emit once"}
+    out = {"rank": k, "compose_ms": ms_c, "compose_algorithmic_bytes": bytes_c,
+           "compose_frac_of_hbm": bytes_c / (ms_c * 1e-3) / 1e9 / hbm, "backward_ms": ms_b, "backward_kernels": 3,
+           "backward_algorithmic_bytes": bytes_b, "backward_frac_of_hbm": bytes_b / (ms_b * 1e-3) / 1e9 / hbm,
+           "note": "CUDA-core kernels: k multiply-adds per element keep the fp32 pipes, not HBM, busiest; the three "
+                   "gradient kernels each stream dW_emit once"}
+    if wl.shape.io_dtype == I.BF16 and s.v % 32 == 0 and s.v <= 448:
+        out["factored_forward"] = measure_factored_forward(torch, wl, (Wb, A, Bm), steps)
+    return out
+
+
+def measure_factored_forward(torch, wl, lowrank, steps: int):
+    """mtpc_window_logprob on a head that keeps the shared unembeddings factored (no composed tensor): time per call, the
+    projection phase alone, and its own (smaller) FLOP count 2 d (n v + n r k) + 4 n r v k per position."""
+    from paper_2511_11346_b200 import binding as B
+    from paper_2511_11346_b200.runner import to_device_bf16
+    s = wl.shape
+    k = lowrank[1].shape[-1]
+    ctx = s.family == I.HMM_CTX
+    W_sum = to_device_bf16(wl.W_sum_q)
+    Ts = torch.from_numpy(np.ascontiguousarray(wl.T_static)).cuda() if wl.T_static is not None else None
+    head = B.MtpcHead(B.MTPC_HMM if ctx else s.family, s.n, s.r, s.v, s.d, B.MTPC_BF16, wl.T, 1, None, W_sum, Ts,
+                      flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0, v_valid=s.v_valid, lowrank=lowrank)
+    hidden = to_device_bf16(wl.hidden_q)
+    targets = torch.from_numpy(wl.targets).cuda()
+    out = torch.empty(wl.T, dtype=torch.float32, device="cuda")
+    for _ in range(3):
+        head.mtpc_window_logprob(hidden, targets, out)
+    torch.cuda.synchronize()
+    head.mtpc_set_timing(steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        head.mtpc_window_logprob(hidden, targets, out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    phases = [head.mtpc_get_timing(i) for i in range(steps)]
+    proj_ms = statistics.mean(p[0] for p in phases)
+    head.mtpc_set_timing(0)
+    status = head.mtpc_get_status()
+    head.mtpc_destroy()
+    flops = (2.0 * s.d * (s.n * s.symbols + s.n * s.r * k + s.sum_rows) + 4.0 * s.n * s.r * s.symbols * k) * wl.T
+    return {"call": "mtpc_window_logprob on a factored head", "ms_per_call": ms, "projection_phase_ms": proj_ms,
+            "positions_per_s": wl.T / (ms * 1e-3), "flops_per_call": flops, "achieved_tflops": flops / (proj_ms * 1e-3) / 1e12,
+            "dense_flops_per_call": algorithmic_flops(wl), "device_status": status,
+            "note": "projection phase = sum-unit tiles + z = B h (plain GEMM) + split + factored kernel; the softmax over "
+                    "n r v logits per position is the same as in the dense head and now dominates"}
 
 
 def measure_eq6_step(torch, dh, wl, hidden, targets, grads, steps: int):

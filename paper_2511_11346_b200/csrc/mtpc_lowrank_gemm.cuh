@@ -232,28 +232,59 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_lowrank_gemm_kernel(cons
           const int col_chunk = c * p.chunk_cols;
           const int width = min(p.chunk_cols, p.v - col_chunk);
           const uint32_t ccol = lane_base + p.corr_col0 + slot * p.chunk_cols;
-          for (int b = 0; b < width / 16; ++b) {
-            float x[16], y[16];
-            tmem_ld16(ccol + b * 16, x);
-            tmem_ld16(lane_base + col_chunk + b * 16, y);
+          // one batch of 16 columns: correction + base, then the dense kernel's online log-sum-exp and target gather
+          auto consume = [&](const uint32_t (&rc)[16], const uint32_t (&rb)[16], int b) {
+            float x[16];
 #pragma unroll
-            for (int q = 0; q < 16; ++q) x[q] += y[q];
+            for (int q = 0; q < 16; ++q) x[q] = __uint_as_float(rc[q]) + __uint_as_float(rb[q]);
             const int col0 = col_chunk + b * 16;
             mask_padding(x, col0, p.vv);
-            float bm = x[0];
+            // the epilogue warp is alone on its scheduler, so dependent chains cost their full latency: reduce as trees
+            float t8[8];
 #pragma unroll
-            for (int q = 1; q < 16; ++q) bm = fmaxf(bm, x[q]);
+            for (int q = 0; q < 8; ++q) t8[q] = fmaxf(x[q], x[q + 8]);
+            const float bm = fmaxf(fmaxf(fmaxf(t8[0], t8[1]), fmaxf(t8[2], t8[3])), fmaxf(fmaxf(t8[4], t8[5]), fmaxf(t8[6], t8[7])));
             const float mn = fmaxf(m, bm);
             const float mn2 = mn * kLog2e;
-            s *= fast_ex2((m - mn) * kLog2e);
+            const float rescale = fast_ex2((m - mn) * kLog2e);
+            float e[16];
 #pragma unroll
-            for (int q = 0; q < 16; ++q) s += fast_ex2(fmaf(x[q], kLog2e, -mn2));
+            for (int q = 0; q < 16; ++q) e[q] = fast_ex2(fmaf(x[q], kLog2e, -mn2));
+#pragma unroll
+            for (int q = 0; q < 8; ++q) e[q] += e[q + 8];
+            s = fmaf(s, rescale, ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7])));
             m = mn;
             const int rel = tgt - col0;
             if (static_cast<unsigned>(rel) < 16u) {
 #pragma unroll
               for (int q = 0; q < 16; ++q)
                 if (rel == q) tval = x[q];
+            }
+          };
+          // both loads of the next batch are in flight while this one goes through the exponentials
+          const int nb = width / 16;
+          uint32_t c0[16], b0[16], c1[16], b1[16];
+          tmem_ld16_issue(ccol, c0);
+          tmem_ld16_issue(lane_base + col_chunk, b0);
+          tmem_ld_wait16(c0);
+          tmem_ld_wait16(b0);
+          for (int b = 0; b < nb; b += 2) {
+            if (b + 1 < nb) {
+              tmem_ld16_issue(ccol + (b + 1) * 16, c1);
+              tmem_ld16_issue(lane_base + col_chunk + (b + 1) * 16, b1);
+            }
+            consume(c0, b0, b);
+            if (b + 1 >= nb) break;
+            tmem_ld_wait16(c1);
+            tmem_ld_wait16(b1);
+            if (b + 2 < nb) {
+              tmem_ld16_issue(ccol + (b + 2) * 16, c0);
+              tmem_ld16_issue(lane_base + col_chunk + (b + 2) * 16, b0);
+            }
+            consume(c1, b1, b + 1);
+            if (b + 2 < nb) {
+              tmem_ld_wait16(c0);
+              tmem_ld_wait16(b0);
             }
           }
           tc_fence_before();
