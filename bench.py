@@ -34,7 +34,7 @@ UNIT = "positions/s"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one projection-kernel launch, from the ncu captures
 # summarised in profiles/ (captured on the full configuration). None = not captured, or the kernel has changed since.
-NCU_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 5: None, 6: None}
+NCU_TRAFFIC_BYTES = {1: 1_094_800_000, 2: 2_533_300_000, 3: 1_196_800_000, 5: None, 6: None}   # profiles/gemm_logprob_cfg1_cfg2_cfg3_ncu.txt
 BURST_REGION_S = 1.0      # a timed loop shorter than this runs at boost clocks: its tensor roofline is the burst peak
 SUSTAINED_LOOP_S = 2.5    # length of the second, power-capped loop whose roofline is the sustained peak
 
