@@ -20,7 +20,7 @@ What follows which passage:
   composite_loss    Eq. (6): per-slot negative log-likelihood with valid-token normalisation and discount gamma
   lowrank_unembedding  App. G, "Unembedding parameter sharing": U_ij = W_i + A_ij B_ij
 
-Readings taken where the paper is silent or garbled (each is listed in the design notes too):
+Readings taken where the paper is silent or garbled:
   * BTree: the left half is the first floor(n/2) tokens; a child latent depends on its parent's latent
     only; products are element-wise in the latent; n must be a power of two here. Internal nodes are in
     heap order (root 0, children 2j+1 and 2j+2); the deepest internal node n/2-1+m owns tokens 2m, 2m+1.

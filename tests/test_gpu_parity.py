@@ -1,6 +1,6 @@
 """GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded inputs.
 
-Bars (the benchmark spec): window log-probs within 2e-3 absolute; drafted bytes bit-exact for every window whose
+Bars: window log-probs within 2e-3 absolute; drafted bytes bit-exact for every window whose
 draws all lie further than 1e-6 from an oracle CDF boundary (the others are counted and printed); draft
 log-probs are checked for EVERY window against the oracle's joint of the bytes the GPU returned."""
 import numpy as np
