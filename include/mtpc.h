@@ -184,10 +184,15 @@ int mtpc_draft_sample_prefix(mtpc_head* head, const void* hidden, int32_t P, int
  *                   as in mtpc_draft_sample. (With zero residual mass, which exact arithmetic excludes after a
  *                   rejection, the last byte v-1 is returned.)
  * The conditional q(. | x_0..x_{s-1}) is a mixture of the r input units of slot s whose weights are the posterior of
- * the latent that owns the slot; it is evaluated from the logits the draft call left in the workspace. Hence:
- *   - the call must follow mtpc_draft_sample / mtpc_draft_sample_prefix on this head with the same P and hidden
- *     states, with no other call on the head in between, else MTPC_ERR_STATE;
- *   - only drafts of P <= 128 positions keep that state (decode-time batches): otherwise MTPC_ERR_UNSUPPORTED.
+ * the latent that owns the slot; it is evaluated from what the draft call left in the workspace. Hence:
+ *   - the call must follow mtpc_draft_sample / mtpc_draft_sample_prefix on this head with the same P and wpp, with no
+ *     other call on the head in between, else MTPC_ERR_STATE;
+ *   - a draft of P <= 128 positions (decode-time batches) leaves every logit of those positions: one kernel;
+ *   - a draft of more positions (a verification batch) leaves only the evidence of the drafted bytes. The call then
+ *     runs the tests, sorts the rejected windows by the slot of their first rejected byte, recomputes that slot's
+ *     r*v logits for them in one projection pass over staged hidden states, and draws. It reads the hidden states the
+ *     DRAFT call was given (bf16 heads: the caller's buffer, which must still hold them); heads created for at most 128
+ *     positions have no scratch for this (MTPC_ERR_UNSUPPORTED).
  * A uniform outside [0,1) or a draft byte outside [0,v) sets the status bit and yields -1 / -1 for that window.
  */
 int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32_t* draft_bytes,

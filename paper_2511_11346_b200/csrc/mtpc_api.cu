@@ -66,6 +66,10 @@ struct Layout {
   // grouped sampling pass of the many-position draft (0 entries: not available)
   size_t group_entries;   // (window, slot) pairs that can be staged at once
   size_t off_grp_ints, off_grp_tiles, off_grp_perm, off_grp_stage;
+  // acceptance stage after a many-position draft: first rejected slot and staging row per window, the recomputed logits
+  // [accept_rows, r v] and unit log-sum-exps [accept_rows, r] of that slot
+  size_t accept_rows;     // windows that can be handled at once (0: not available)
+  size_t off_acc_rej, off_acc_row, off_acc_logits, off_acc_lse;
   size_t total;
 };
 
@@ -188,6 +192,18 @@ int plan(const mtpc_config& c, Layout* L) {
   L->off_grp_tiles = take(ge ? (emit_units + ge / 128 + 1) * sizeof(GroupTile) : 0);
   L->off_grp_perm = take(ge * 4);
   L->off_grp_stage = take(ge * c.d * 2);
+  L->accept_rows = 0;
+  if (ge > 0) {
+    const size_t cap = kGroupStageBytes / (static_cast<size_t>(c.r) * c.v * 4);
+    L->accept_rows = L->max_windows < cap ? L->max_windows : cap;
+    if (L->accept_rows > ge) L->accept_rows = ge;                               // they share the staging rows
+    if (L->accept_rows < static_cast<size_t>(c.max_windows_per_pos)) L->accept_rows = 0;
+  }
+  const size_t ar = L->accept_rows;
+  L->off_acc_rej = take(ar ? L->max_windows * 4 : 0);
+  L->off_acc_row = take(ar ? L->max_windows * 4 : 0);
+  L->off_acc_logits = take(ar * c.r * c.v * 4);
+  L->off_acc_lse = take(ar * c.r * 4);
   L->total = off;
   return MTPC_OK;
 }
@@ -283,7 +299,9 @@ struct mtpc_head {
   cudaStream_t copy_stream; // host-buffer calls: uploads run here, ahead of the kernels (created on first use)
   cudaEvent_t* copy_events; // [copy_event_count]: "chunk c is on the device"; [0] doubles as "the call may start"
   int copy_event_count;
-  int draft_P;              // positions whose logits the few-position draft path left in the workspace (0: none)
+  int draft_P;              // positions whose draft state (logits, or after a many-position draft G and log omega) is in the workspace (0: none)
+  int draft_wpp;            // windows per position of that draft
+  const void* draft_hidden; // many-position draft: the bf16 hidden states it read (the acceptance stage stages rows of them)
   int ring;                 // calls whose per-kernel events are retained (0 = timing off)
   cudaEvent_t* ev;          // [ring][kMaxPhases][2]
   int* ring_phases;         // [ring] phases recorded by the call in that slot
@@ -379,6 +397,7 @@ struct GroupArgs {           // grouped sampling pass: the staged hidden states 
   const int* perm = nullptr;
   const int* unit_sel = nullptr;             // this chunk's rows of the selected units
   int max_tiles = 0;
+  bool by_slot = false;                      // rows sorted by slot; the kernel writes the slot's logits (acceptance stage)
 };
 
 struct GradArgs {            // what the projection kernel keeps for the backward pass (training calls only)
@@ -394,7 +413,7 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
   const Tiling& tl = mode == kModeSample ? L.sm : L.lp;
-  if (grp != nullptr && mode != kModeSample) return MTPC_ERR_SHAPE;
+  if (grp != nullptr && (grp->by_slot ? mode != kModeLogprob : mode != kModeSample)) return MTPC_ERR_SHAPE;
   GemmParams p;
   memset(&p, 0, sizeof(p));
   if (ga) {
@@ -454,7 +473,7 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
     p.group_tiles = grp->tiles;
     p.group_num_tiles = grp->num_tiles;
     p.group_perm = grp->perm;
-    p.group_two_pass = L.sample_two_pass ? 1 : 0;
+    p.group_two_pass = (L.sample_two_pass && !grp->by_slot) ? 1 : 0;
     p.unit_sel = grp->unit_sel;
   }
   p.uniforms = uniforms;
@@ -464,7 +483,9 @@ int launch_gemm(mtpc_head* h, int mode, const void* hidden_bf16, int rows, int w
   const long long items = grp ? grp->max_tiles : static_cast<long long>(p.m_units) * (p.num_groups + p.num_sum_tiles);
   const int grid = ctas * static_cast<int>(items < workers ? items : workers);
   const size_t smem = pair ? tl.pair_smem : tl.smem;
-  if (grp) {
+  if (grp && grp->by_slot) {
+    mtpc_gemm_kernel<kModeLogitsGrouped, 1><<<grid, kGemmThreads, smem, st>>>(p);
+  } else if (grp) {
     mtpc_gemm_kernel<kModeSampleGrouped, 1><<<grid, kGemmThreads, smem, st>>>(p);
   } else if (!pair) {
     if (mode == kModeLogprob)
@@ -709,6 +730,7 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
     }
     h->launches++;
     h->draft_P = P;
+    h->draft_wpp = wpp;
     pt.end();
     if ((rc = check_launch()) != MTPC_OK) return rc;
     pt.begin();
@@ -757,7 +779,7 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
       const int gblocks = (entries + kGroupThreads / 32 - 1) / (kGroupThreads / 32);
       group_gather_kernel<<<gblocks < 16 * h->num_sms ? gblocks : 16 * h->num_sms, kGroupThreads, 0, st>>>(
           sel, static_cast<const __nv_bfloat16*>(hb) + static_cast<size_t>(p0) * c.d, offsets, cursors, perm, stage, entries,
-          c.n, c.r, wpp, c.d);
+          c.n, c.r, wpp, c.d, static_cast<int*>(nullptr));
       h->launches += 3;
       if ((rc = check_launch()) != MTPC_OK) return rc;
       GroupArgs ga;
@@ -788,6 +810,11 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   pt.begin();
   rc = launch_circuit(h, W, wpp, out_logprob, out_prefix, st);
   pt.end();
+  if (rc == MTPC_OK) {                 // G, log omega and the hidden states stay in place for an acceptance call
+    h->draft_P = P;
+    h->draft_wpp = wpp;
+    h->draft_hidden = hb;
+  }
   return rc;
 }
 
@@ -1168,6 +1195,7 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
   fail |= cudaFuncSetAttribute(mtpc_gemm_kernel<kModeSample, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSmemLimit) != cudaSuccess;
   fail |= !allow_full_smem(mtpc_gemm_kernel<kModeSampleGrouped, 1>);
+  fail |= !allow_full_smem(mtpc_gemm_kernel<kModeLogitsGrouped, 1>);
   fail |= !allow_full_smem(mtpc_gemm_kernel<kModeLogprob, 2>);
   fail |= !allow_full_smem(mtpc_gemm_kernel<kModeSample, 2>);
   h->max_pairs = fail ? 0 : resident_pairs(L.lp.pair_smem);
@@ -1281,8 +1309,7 @@ int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32
   if (P == 0) return MTPC_OK;
   if (!draft_bytes || !prefix_logprob || !target_probs || !accept_uniforms || !out_accepted || !out_next_byte)
     return MTPC_ERR_NULL;
-  if (P > head->L.decode_max_p) return MTPC_ERR_UNSUPPORTED;
-  if (head->draft_P != P) return MTPC_ERR_STATE;
+  if (head->draft_P != P || head->draft_wpp != wpp) return MTPC_ERR_STATE;
   const mtpc_config& c = head->cfg;
   const Layout& L = head->L;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1290,15 +1317,85 @@ int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32
   const size_t smem = accept_warp_floats(c.family, c.n, c.r, c.v) * sizeof(float);
   if (smem > static_cast<size_t>(kSmemLimit)) return MTPC_ERR_UNSUPPORTED;      // a residual row of more than ~56k symbols
   PhaseTimer pt(head, st);
-  pt.begin();
-  spec_accept_kernel<<<W, kAcceptThreads, smem, st>>>(
-      c.family, at<float>(head, L.off_logits), at<float>(head, L.off_unit_lse), at<float>(head, L.off_logw),
-      hmm_tables(head), draft_bytes, prefix_logprob, target_probs, accept_uniforms, out_accepted,
-      out_next_byte, at<unsigned>(head, L.off_status), W, wpp, c.n, c.r, c.v, valid_symbols(c), L.sum_rows,
-      hmm_table_stride(head));
-  head->launches++;
-  pt.end();
-  return check_launch();
+  if (P <= L.decode_max_p) {
+    // after a few-position draft: every logit of the drafted positions is still in the workspace
+    pt.begin();
+    spec_accept_kernel<<<W, kAcceptThreads, smem, st>>>(
+        c.family, at<float>(head, L.off_logits), at<float>(head, L.off_unit_lse), at<float>(head, L.off_logw),
+        hmm_tables(head), draft_bytes, prefix_logprob, target_probs, accept_uniforms, out_accepted,
+        out_next_byte, at<unsigned>(head, L.off_status), W, wpp, c.n, c.r, c.v, valid_symbols(c), L.sum_rows,
+        hmm_table_stride(head), static_cast<const float*>(nullptr), static_cast<const int*>(nullptr));
+    head->launches++;
+    pt.end();
+    return check_launch();
+  }
+  // After a many-position draft no logits were kept. The evidence of the drafted bytes (G) and log omega are still in
+  // the workspace; what is missing is, for every window rejected at byte s, the r v logits of slot s. So: run the tests,
+  // sort the rejected windows by s, stage their hidden states, recompute those logits with one sorted projection pass,
+  // then run the acceptance kernel on them. In chunks of positions whose windows fit the scratch.
+  if (L.accept_rows == 0 || !head->draft_hidden) return MTPC_ERR_UNSUPPORTED;
+  int* ints = at<int>(head, L.off_grp_ints);
+  int* counts = ints, *cursors = ints + c.n, *offsets = ints + 2 * c.n, *num_tiles = ints + 3 * c.n;
+  GroupTile* tiles = at<GroupTile>(head, L.off_grp_tiles);
+  int* perm = at<int>(head, L.off_grp_perm);
+  __nv_bfloat16* stage = at<__nv_bfloat16>(head, L.off_grp_stage);
+  int* rej = at<int>(head, L.off_acc_rej);
+  int* row_of = at<int>(head, L.off_acc_row);
+  float* lg = at<float>(head, L.off_acc_logits);
+  float* lse = at<float>(head, L.off_acc_lse);
+  const int chunk_pos = static_cast<int>(L.accept_rows / wpp);                  // >= 1 by construction
+  const float* tables = hmm_tables(head);
+  const int tstride = hmm_table_stride(head);
+  for (int p0 = 0; p0 < P; p0 += chunk_pos) {
+    const int pc = P - p0 < chunk_pos ? P - p0 : chunk_pos;
+    const int wc = pc * wpp;
+    const size_t w0 = static_cast<size_t>(p0) * wpp;
+    const int32_t* xb = draft_bytes + w0 * c.n;
+    const float* pre = prefix_logprob + w0 * c.n;
+    const float* tp = target_probs + w0 * (c.n + 1) * c.v;
+    const float* ua = accept_uniforms + w0 * (c.n + 1);
+    pt.begin();
+    accept_test_kernel<<<(wc + 7) / 8, 256, 0, st>>>(xb, pre, tp, ua, rej, wc, c.n, c.v, valid_symbols(c));
+    if (cudaMemsetAsync(ints, 0, static_cast<size_t>(2 * c.n) * 4, st) != cudaSuccess) return MTPC_ERR_CUDA;
+    const int cblocks = (wc + kGroupThreads - 1) / kGroupThreads;
+    group_count_kernel<<<cblocks < 4 * head->num_sms ? cblocks : 4 * head->num_sms, kGroupThreads, c.n * sizeof(int), st>>>(
+        rej, counts, wc, 1, c.n);
+    group_scan_kernel<<<1, kGroupScanThreads, 0, st>>>(counts, offsets, tiles, num_tiles, c.n);
+    const int gblocks = (wc + kGroupThreads / 32 - 1) / (kGroupThreads / 32);
+    group_gather_kernel<<<gblocks < 16 * head->num_sms ? gblocks : 16 * head->num_sms, kGroupThreads, 0, st>>>(
+        rej, static_cast<const __nv_bfloat16*>(head->draft_hidden) + static_cast<size_t>(p0) * c.d, offsets, cursors, perm,
+        stage, wc, 1, c.n, wpp, c.d, row_of);
+    head->launches += 4;
+    int rc2 = check_launch();
+    if (rc2 != MTPC_OK) return rc2;
+    GroupArgs ga;
+    ga.stage = stage;
+    ga.entries = wc;
+    ga.tiles = tiles;
+    ga.num_tiles = num_tiles;
+    ga.perm = perm;
+    ga.unit_sel = rej;
+    ga.max_tiles = c.n + wc / 128 + 1;
+    ga.by_slot = true;
+    GradArgs out;
+    out.lse_out = lse;
+    out.logit_out = lg;
+    out.logit_pitch = static_cast<size_t>(c.r) * c.v;
+    rc2 = launch_gemm(head, kModeLogprob, head->draft_hidden, pc, wpp, true, false, nullptr, nullptr, nullptr, st, &out, false,
+                      &ga);
+    pt.end();
+    if (rc2 != MTPC_OK) return rc2;
+    pt.begin();
+    spec_accept_kernel<<<wc, kAcceptThreads, smem, st>>>(
+        c.family, lg, lse, at<float>(head, L.off_logw) + static_cast<size_t>(p0) * L.sum_rows,
+        tables + static_cast<size_t>(p0) * tstride, xb, pre, tp, ua, out_accepted + w0, out_next_byte + w0,
+        at<unsigned>(head, L.off_status), wc, wpp, c.n, c.r, c.v, valid_symbols(c), L.sum_rows, tstride,
+        at<float>(head, L.off_G) + w0 * c.n * c.r, row_of);
+    head->launches++;
+    pt.end();
+    if ((rc2 = check_launch()) != MTPC_OK) return rc2;
+  }
+  return MTPC_OK;
 }
 
 int mtpc_window_loss(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,

@@ -562,7 +562,10 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
     const float* __restrict__ logA, const int* __restrict__ bytes, const float* __restrict__ prefix,
     const float* __restrict__ target, const float* __restrict__ uniforms, int* __restrict__ out_accepted,
     int* __restrict__ out_next, unsigned* status, int W, int wpp, int n, int r, int v, int vv, int sum_rows,
-    int logA_stride) {
+    int logA_stride, const float* __restrict__ evidence, const int* __restrict__ row_of) {
+  // evidence != NULL (after a many-position draft): log phi of the drafted bytes comes from evidence [W, n, r] (the G the
+  // draft left), and `logits` [rows, r v] / `unit_lse` [rows, r] hold only the slot of each rejected window's first
+  // rejected byte, at row row_of[w].
   extern __shared__ float sm[];
   int& accepted_len = *reinterpret_cast<int*>(sm);       // s, or -1: the window's inputs were refused
   const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -612,9 +615,16 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
   }
   if (s < n) {
     // ---- 2. c[k]: log-weight of input unit k of slot s given the accepted bytes (lane = k)
-    auto g_of = [&](int i) -> float {   // log phi_{i,lane}(x_i)
-      const size_t unit = (static_cast<size_t>(pos) * n + i) * r + lane;
+    auto g_at = [&](int i, int k) -> float {   // log phi_{i,k}(x_i)
+      if (evidence != nullptr) return evidence[(static_cast<size_t>(w) * n + i) * r + k];
+      const size_t unit = (static_cast<size_t>(pos) * n + i) * r + k;
       return logits[unit * v + x[i]] - unit_lse[unit];
+    };
+    auto g_of = [&](int i) -> float { return g_at(i, lane); };
+    // log-sum-exp of unit k of slot s
+    auto lse_of = [&](int k) -> float {
+      return evidence != nullptr ? unit_lse[static_cast<size_t>(row_of[w]) * r + k]
+                                 : unit_lse[(static_cast<size_t>(pos) * n + s) * r + k];
     };
     float c = 0.f;
     if (family == 0) {
@@ -629,10 +639,7 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
         if (k < r) {
           float a = lw[k];
 #pragma unroll 4
-          for (int i = 0; i < s; ++i) {                     // independent gathers: several in flight
-            const size_t unit = (static_cast<size_t>(pos) * n + i) * r + k;
-            a += logits[unit * v + x[i]] - unit_lse[unit];
-          }
+          for (int i = 0; i < s; ++i) a += g_at(i, k);      // independent gathers: several in flight
           cq[q] = a;
           lse_merge(m, sacc, a, 1.f);
         }
@@ -649,7 +656,7 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
         const int k = lane + 32 * q;
         if (k < r) {
           cw[k] = __expf(cq[q] - lse_all);
-          cl[k] = unit_lse[(static_cast<size_t>(pos) * n + s) * r + k];
+          cl[k] = lse_of(k);
         }
       }
     } else if (family == 1) {
@@ -716,7 +723,7 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
       const float c_lse = warp_lse(c, has);              // every lane takes part in the shuffles
       if (has) {
         cw[lane] = __expf(c - c_lse);
-        cl[lane] = unit_lse[(static_cast<size_t>(pos) * n + s) * r + lane];
+        cl[lane] = lse_of(lane);
       }
     }
   }
@@ -730,7 +737,8 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
   if (s == n) {
     for (int b = threadIdx.x; b < v; b += kAcceptThreads) mres[b] = b < vv ? trow[b] : 0.f;
   } else {
-    const float* lrow = logits + (static_cast<size_t>(pos) * n + s) * r * v;   // [r, v] logits of slot s
+    const float* lrow = evidence != nullptr ? logits + static_cast<size_t>(row_of[w]) * r * v
+                                            : logits + (static_cast<size_t>(pos) * n + s) * r * v;   // [r, v] logits of slot s
     for (int b = threadIdx.x; b < v; b += kAcceptThreads) {
       float q = 0.f;
       if (b < vv) {
@@ -783,6 +791,39 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
     byte = __shfl_sync(kFull, found, src);
   }
   if (lane == 0) out_next[w] = byte;
+}
+
+// The tests of Algorithm 3 alone, one warp per window: first_rejected[w] = s if the draft is rejected at byte s < n, else -1
+// (everything accepted, or inputs that the acceptance kernel will refuse). Decides which slot's logits the acceptance
+// stage after a many-position draft has to recompute for the window.
+__global__ void accept_test_kernel(const int* __restrict__ bytes, const float* __restrict__ prefix,
+                                   const float* __restrict__ target, const float* __restrict__ uniforms,
+                                   int* __restrict__ first_rejected, int W, int n, int v, int vv) {
+  const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (w >= W) return;
+  const int* x = bytes + static_cast<size_t>(w) * n;
+  const float* pre = prefix + static_cast<size_t>(w) * n;
+  const float* u = uniforms + static_cast<size_t>(w) * (n + 1);
+  const float* tp = target + static_cast<size_t>(w) * (n + 1) * v;
+  bool bad = false;
+  for (int c = lane; c <= n; c += 32) bad |= !(u[c] >= 0.f && u[c] < 1.f);
+  for (int c = lane; c < n; c += 32) bad |= static_cast<unsigned>(x[c]) >= static_cast<unsigned>(vv);
+  bad = __any_sync(kFull, bad);
+  int s = n;
+  if (!bad) {
+    for (int base = 0; base < n && s == n; base += 32) {
+      const int i = base + lane;
+      bool rej = false;
+      if (i < n) {
+        const float q = __expf(pre[i] - (i > 0 ? pre[i - 1] : 0.f));
+        rej = u[i] * q > tp[static_cast<size_t>(i) * v + x[i]];
+      }
+      const unsigned m = __ballot_sync(kFull, rej);
+      if (m) s = base + __ffs(m) - 1;
+    }
+  }
+  if (lane == 0) first_rejected[w] = (bad || s == n) ? -1 : s;
 }
 
 }  // namespace mtpc

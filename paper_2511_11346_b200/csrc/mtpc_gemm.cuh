@@ -45,7 +45,9 @@ constexpr uint32_t kStatusBadTarget = 1u, kStatusBadUniform = 2u, kStatusTimeout
 
 // kModeSampleGrouped: the byte draws again, on rows that were sorted by the unit they sample from (mtpc_group.cuh):
 // a work item is one GroupTile instead of (m-tile, unit).
-enum { kModeLogprob = 0, kModeSample = 1, kModeSampleGrouped = 2 };
+// kModeLogitsGrouped: rows sorted by SLOT (the acceptance stage after a many-position draft): a work item is a GroupTile
+// whose `unit` is a slot; the logits of the slot's r units and their log-sum-exps are written out per staged row.
+enum { kModeLogprob = 0, kModeSample = 1, kModeSampleGrouped = 2, kModeLogitsGrouped = 3 };
 
 struct GemmParams {
   CUtensorMap tm_a;      // hidden  [T, d]        box 64 x 128
@@ -137,17 +139,18 @@ struct TileCoord {
   int arow, count;   // first row of the A operand and the rows that count (set by the caller for ungrouped items)
   int wrap;          // tiles per sweep over the item's weight rows: tile t reads the rows of tile t % wrap
 };
-// A grouped item: `count` staged rows from `row0` on, against the tiles of the one unit they sample from.
-__device__ __forceinline__ TileCoord group_coord(const GemmParams& p, int item) {
+// A grouped item: `count` staged rows from `row0` on, against the tiles of the one unit they sample from (by_slot: of the
+// r units of the one slot whose logits they need).
+__device__ __forceinline__ TileCoord group_coord(const GemmParams& p, int item, bool by_slot) {
   const GroupTile g = p.group_tiles[item];
   TileCoord c;
   c.mt = 0;
   c.is_sum = 0;
-  c.unit0 = g.unit;
-  c.nunits = 1;
+  c.unit0 = by_slot ? g.unit * p.r : g.unit;
+  c.nunits = by_slot ? p.r : 1;
   c.cols = p.tile_cols;
-  c.brow0 = g.unit * p.v;
-  c.wrap = (p.v + p.tile_cols - 1) / p.tile_cols;
+  c.brow0 = c.unit0 * p.v;
+  c.wrap = (c.nunits * p.v + p.tile_cols - 1) / p.tile_cols;
   c.ntiles = p.group_two_pass ? 2 * c.wrap : c.wrap;
   c.arow = g.row0;
   c.count = g.count;
@@ -238,11 +241,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  static_assert(MODE != kModeSampleGrouped || CTAS == 1, "grouped tiles are ragged: no pairing");
-  const int num_items = MODE == kModeSampleGrouped ? *p.group_num_tiles : (p.num_groups + p.num_sum_tiles) * p.m_units;
+  constexpr bool kGrouped = MODE == kModeSampleGrouped || MODE == kModeLogitsGrouped;
+  static_assert(!kGrouped || CTAS == 1, "grouped tiles are ragged: no pairing");
+  const int num_items = kGrouped ? *p.group_num_tiles : (p.num_groups + p.num_sum_tiles) * p.m_units;
   const uint32_t cta_rank = CTAS == 2 ? cluster_cta_rank() : 0u;      // 0 = the pair's leader
   auto coord = [&](int item) {
-    if (MODE == kModeSampleGrouped) return group_coord(p, item);
+    if (kGrouped) return group_coord(p, item, MODE == kModeLogitsGrouped);
     TileCoord c = tile_coord(p, item);
     c.arow = (c.mt * CTAS + static_cast<int>(cta_rank)) * kBlockM;
     c.count = min(kBlockM, p.T - c.arow);                             // <= 0: a pair's second CTA past the last position
@@ -469,7 +473,50 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_gemm_kernel(const __grid
         continue;
       }
 
-      if (MODE == kModeLogprob) {
+      if (MODE == kModeLogitsGrouped) {
+        // ---- the slot's logits and unit log-sum-exps per staged row (logit_out [rows, r v], lse_out [rows, r]): what the
+        // acceptance stage needs to form the circuit's conditional of the first rejected byte
+        int col = 0, k = 0;                                       // column inside the slot's r v columns; unit index
+        float m = -CUDART_INF_F, s = 0.f;
+        for (int t = 0; t < tc.ntiles && ok; ++t, ++use) {
+          const uint32_t slot = use % p.num_slots;
+          if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (use / p.num_slots) & 1u, ctl, p.status, lane)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t tcol = lane_base + slot * p.slot_stride;
+          for (int b = 0; b < nbatch && k < p.r; ++b) {
+            float x[16];
+            tmem_ld16(tcol + b * 16, x);
+            mask_padding(x, col - k * p.v, p.vv);
+            if (valid) {
+              float* l = p.logit_out + static_cast<size_t>(row) * p.logit_pitch + col;
+              st_global_v8(l, x);
+              st_global_v8(l + 8, x + 8);
+            }
+            float bm = x[0];
+#pragma unroll
+            for (int q = 1; q < 16; ++q) bm = fmaxf(bm, x[q]);
+            const float mn = fmaxf(m, bm);
+            const float mn2 = mn * kLog2e;
+            s *= fast_ex2((m - mn) * kLog2e);
+#pragma unroll
+            for (int q = 0; q < 16; ++q) s += fast_ex2(fmaf(x[q], kLog2e, -mn2));
+            m = mn;
+            col += 16;
+            if (col == (k + 1) * p.v) {
+              if (valid) p.lse_out[static_cast<size_t>(row) * p.r + k] = m + fast_lg2(s) * kLn2;
+              ++k;
+              m = -CUDART_INF_F; s = 0.f;
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) release_slot(slot);
+        }
+        if (!ok) break;
+      } else if (MODE == kModeLogprob) {
         // ---- log phi at the target byte: online log-sum-exp over the v columns of each unit + gather. The
         // running (m, s) and the gathered logit live across tile boundaries; a unit is closed when its v-th
         // column has been consumed.

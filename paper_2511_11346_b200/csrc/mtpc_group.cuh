@@ -100,13 +100,14 @@ __global__ void __launch_bounds__(kGroupScanThreads) group_scan_kernel(const int
 }
 
 // One warp per (window, slot) pair: lane 0 takes the next free staging row of the pair's unit, the warp copies the
-// window's hidden state (d bf16, d a multiple of 8, rows 16-byte aligned) there and records which pair the row holds.
+// window's hidden state (d bf16, d a multiple of 8, rows 16-byte aligned) there and records which pair the row holds
+// (and, where row_of is given, which row a pair got).
 __global__ void __launch_bounds__(kGroupThreads) group_gather_kernel(const int* __restrict__ unit_sel,
                                                                      const __nv_bfloat16* __restrict__ hidden,
                                                                      const int* __restrict__ offsets,
                                                                      int* __restrict__ cursors, int* __restrict__ perm,
                                                                      __nv_bfloat16* __restrict__ stage, int entries, int n,
-                                                                     int r, int wpp, int d) {
+                                                                     int r, int wpp, int d, int* __restrict__ row_of) {
   const int lane = threadIdx.x & 31;
   const int warps = gridDim.x * (kGroupThreads / 32);
   const int vecs = d / 8;                                      // 16-byte pieces per row
@@ -118,6 +119,7 @@ __global__ void __launch_bounds__(kGroupThreads) group_gather_kernel(const int* 
       const int u = (e % n) * r + z;
       row = offsets[u] + atomicAdd(&cursors[u], 1);
       perm[row] = e;
+      if (row_of != nullptr) row_of[e] = row;                  // the inverse map, for callers that look a pair's row up
     }
     row = __shfl_sync(0xffffffffu, row, 0);
     const uint4* src = reinterpret_cast<const uint4*>(hidden + static_cast<size_t>((e / n) / wpp) * d);

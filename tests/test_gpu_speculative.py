@@ -112,7 +112,8 @@ def check_accept(wl, wpp):
     rows = np.arange(P)
     pos = np.repeat(rows, wpp)
     dh = DeviceHead(wl)
-    bytes_g, prefix_g = dh.draft_sample_prefix(wpp)
+    hidden_d = dh.hidden_device()            # kept alive: after a many-position draft the acceptance stage reads it again
+    bytes_g, prefix_g = dh.draft_sample_prefix(wpp, hidden=hidden_d)
     assert dh.head.mtpc_get_status() == 0
     # oracle: its own draft, its own prefix marginals
     logphi, logw = oracle_params(wl, rows)
@@ -188,6 +189,12 @@ ACCEPT_SMALL = [
     (I.BTREE, 16, 8, 32, 64, 128, 2),
     (I.CP, 2, 4, 1024, 64, 3, 4),          # vocabularies wider than 512 symbols
     (I.HMM, 2, 2, 4112, 64, 2, 8),
+    # more than 128 positions: the many-position draft keeps no logits, the acceptance stage recomputes the slot it needs
+    (I.CP, 3, 8, 64, 64, 150, 2),
+    (I.HMM, 4, 8, 48, 64, 140, 1),
+    (I.BTREE, 4, 4, 32, 64, 200, 1),
+    (I.HMM_CTX, 3, 4, 320, 64, 130, 2),
+    (I.CP, 2, 16, 320, 128, 300, 1),       # r v = 5120 logit columns per rejected window, 20 accumulator tiles per row tile
 ]
 
 
@@ -227,10 +234,10 @@ def test_accept_needs_the_draft_state_and_flags_bad_inputs():
     with pytest.raises(B.MtpcError) as e:
         dh.speculative_accept(6, 2, bytes_g, prefix_g, p, ua)
     assert e.value.code == B.ERR_STATE
-    # more positions than the few-position path keeps logits for
+    # more positions than were drafted (a many-position draft would have had to come first)
     with pytest.raises(B.MtpcError) as e:
         dh.speculative_accept(129, 1, bytes_g, prefix_g, p, ua)
-    assert e.value.code == -3
+    assert e.value.code == B.ERR_STATE
     # a uniform outside [0,1) and a byte outside [0,v): flagged, -1 / -1 for those windows only
     bytes_g, prefix_g = dh.draft_sample_prefix(2)
     ua2 = ua.clone()
