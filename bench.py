@@ -476,10 +476,32 @@ def measure_draft_whole_batch(torch, head, wl, hidden, steps: int) -> dict:
     dms = d0.elapsed_time(d1) / steps
     dph = [head.mtpc_get_timing(i) for i in range(steps)]
     head.mtpc_set_timing(0)
-    return {"call": "mtpc_draft_sample over the whole batch", "windows": W, "ms_per_call": dms,
-            "windows_per_s": W / (dms * 1e-3),
-            "phase_ms": [statistics.mean(p[k] for p in dph) for k in range(len(dph[0]))],
-            "device_status": head.mtpc_get_status()}
+    res = {"call": "mtpc_draft_sample over the whole batch", "windows": W, "ms_per_call": dms,
+           "windows_per_s": W / (dms * 1e-3),
+           "phase_ms": [statistics.mean(p[k] for p in dph) for k in range(len(dph[0]))],
+           "phases": "sum-unit GEMM, latent draws, byte draws (sorted by unit: sort + staging + GEMM), GEMM + gather "
+                     "epilogue on the drafted bytes, circuit"}
+    # draft with prefix marginals + acceptance stage (Algorithm 3) on the whole batch, synthetic target-model rows
+    tp = torch.from_numpy(I.target_rows(I.BASE_SEED + 77, 9, (W, s.n + 1, s.v))).cuda()
+    ua = torch.from_numpy(I.uniforms(I.BASE_SEED + 78, 10, (W, s.n + 1))).cuda()
+    opre = torch.empty((W, s.n), dtype=torch.float32, device="cuda")
+    oacc = torch.empty(W, dtype=torch.int32, device="cuda")
+    onxt = torch.empty(W, dtype=torch.int32, device="cuda")
+    cyc = []
+    for it in range(3 + steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        head.mtpc_draft_sample_prefix(hidden, wl.wpp, u, ob, opre)
+        head.mtpc_speculative_accept(wl.T, wl.wpp, ob, opre, tp, ua, oacc, onxt)
+        e1.record()
+        e1.synchronize()
+        if it >= 3:
+            cyc.append(e0.elapsed_time(e1))
+    res["draft_plus_accept"] = {"ms_per_cycle": statistics.median(cyc),
+                                "mean_accepted_bytes_vs_synthetic_target": float(oacc.float().mean().cpu()),
+                                "calls": "mtpc_draft_sample_prefix + mtpc_speculative_accept"}
+    res["device_status"] = head.mtpc_get_status()
+    return res
 
 
 def measure_other_workload(torch, idx: int, dev_index: int, peaks: dict, peak_src: str, with_oracle: bool) -> dict:
