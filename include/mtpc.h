@@ -283,11 +283,11 @@ int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k,
  * arithmetic on the bf16 parameters only by fp32 accumulation (no rounding of a composed U to bf16).
  *   cfg, W_sum, T_static, workspace, stream, out: as mtpc_create_head; cfg->io_dtype must be MTPC_BF16.
  *   k        the adaptors' rank: 16 or 32 (MTPC_ERR_UNSUPPORTED otherwise; so are shapes whose base accumulator and two
- *            correction slots do not fit the 512 columns of tensor memory: v up to 448).
+ *            correction slots do not fit the 512 columns of tensor memory: v up to 480).
  *   W_base   dev [n, v, d] bf16;  A dev [n, r, v, k] bf16;  B dev [n, r, k, d] bf16: caller-owned, read in place, must
  *            outlive the head (after an optimiser step no call is needed unless W_sum / T_static moved:
  *            mtpc_update_parameters with W_emit = NULL then).
- *   workspace >= mtpc_lowrank_workspace_bytes(cfg, k): the dense head's workspace plus z in fp32 and in bf16 halves.
+ *   workspace >= mtpc_lowrank_workspace_bytes(cfg, k): the dense head's workspace plus z = B h as two bf16 halves.
  * Such a head serves mtpc_window_logprob, mtpc_window_prefix_logprob, mtpc_window_loss and mtpc_window_logprob_host.
  * Drafting, acceptance and the backward calls return MTPC_ERR_UNSUPPORTED on it: they run on the composed tensor
  * (mtpc_lowrank_compose + mtpc_create_head, gradients carried back by mtpc_lowrank_backward).

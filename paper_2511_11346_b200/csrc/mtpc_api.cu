@@ -672,7 +672,7 @@ struct GemmOperand {
 };
 
 int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmOperand B1, int K1, int a_k1, float* C,
-                      size_t ldc, int M, int N, cudaStream_t st);
+                      size_t ldc, int M, int N, cudaStream_t st, void* C_hilo = nullptr, int split_k = 0);
 int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, const int* targets, cudaStream_t st);
 
 // out [T] (joint) and / or prefix [T, n] (prefix log-marginals); either may be NULL, not both.
@@ -844,8 +844,9 @@ void plan_backward(const mtpc_config& c, const Layout& L, int T, BackwardLayout*
 
 // C[M, N] fp32 (pitch ldc) = A B^T over K = K0 + K1: segment 0 multiplies A's K range [0, K0) with B0, segment 1 (K1 > 0)
 // A's K range [a_k1, a_k1 + K1) with B1.
+// C_hilo != NULL (then C is NULL): the result leaves as two bf16 halves per entry, see PlainGemmParams.
 int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmOperand B1, int K1, int a_k1, float* C,
-                      size_t ldc, int M, int N, cudaStream_t st) {
+                      size_t ldc, int M, int N, cudaStream_t st, void* C_hilo, int split_k) {
   if (M <= 0 || N <= 0 || K0 <= 0) return MTPC_OK;
   if (K1 > 0 && (A.mn_major || B1.mn_major != B0.mn_major)) return MTPC_ERR_SHAPE;
   PlainGemmParams p;
@@ -871,6 +872,10 @@ int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmO
   p.wide_stores = (reinterpret_cast<uintptr_t>(C) % 32 == 0 && ldc % 8 == 0) ? 1 : 0;
   p.C = C;
   p.ldc = ldc;
+  p.C_hilo = static_cast<__nv_bfloat16*>(C_hilo);
+  p.split_k = split_k;
+  if ((C == nullptr) == (C_hilo == nullptr)) return MTPC_ERR_NULL;
+  if (C_hilo != nullptr && (split_k < 16 || split_k % 16 != 0 || N % split_k != 0)) return MTPC_ERR_SHAPE;
   p.status = at<unsigned>(h, h->L.off_status);
   p.wait_limit_ns = h->wait_limit_ns;
   const long long items = static_cast<long long>(p.m_tiles) * p.n_tiles;
@@ -884,14 +889,24 @@ int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmO
   return check_launch();
 }
 
+#ifndef MTPC_LR_GROUPS
+#define MTPC_LR_GROUPS 2
+#endif
+constexpr int kLrGroups = MTPC_LR_GROUPS;   // epilogue groups of the factored projection kernel (<= kLrMaxGroups)
 // Tiling of the factored projection (mtpc_lowrank_gemm.cuh) for a head shape; false: the shape does not fit.
 bool plan_lowrank(const mtpc_config& c, int k, LowRankGemmParams* p) {
   if (k < 16 || k > kLrMaxRank || k % 16 != 0 || c.v % 16 != 0) return false;
   const int base_cols = (c.v + 31) / 32 * 32;
-  int chunk = (kTmemCols - base_cols) / 2 / 32 * 32;          // two correction slots beside the base accumulator
-  if (chunk > 256) chunk = 256;
-  if (chunk < 32) return false;
-  if (chunk > c.v) chunk = c.v;                                // (v < 32 never gets here with chunk < 16: v is a multiple of 16)
+  // beside the base accumulator: two correction slots for each of `groups` epilogue groups; as many groups (up to
+  // kLrGroups, and no more than there are components) as leave chunks of at least 32 columns, else narrower chunks
+  const int spare = kTmemCols - base_cols;
+  int groups = kLrGroups < c.r ? kLrGroups : c.r;
+  while (groups > 1 && spare / (2 * groups) < 32) --groups;
+  int chunk = spare / (2 * groups) / 16 * 16;
+  if (chunk > 96) chunk = 96;
+  if (chunk < 16) return false;
+  if (chunk > c.v) chunk = c.v;
+  p->groups = groups;
   p->n = c.n; p->r = c.r; p->v = c.v; p->k = k;
   p->vv = c.v_valid > 0 ? c.v_valid : c.v;
   p->kblocks = c.d / kBlockK;
@@ -909,7 +924,7 @@ bool plan_lowrank(const mtpc_config& c, int k, LowRankGemmParams* p) {
   const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
   p->stages = (kSmemLimit - ctl) / p->stage_bytes;
   if (p->stages > kMaxStages) p->stages = kMaxStages;
-  return p->stages >= 2;
+  return p->stages >= groups + 1;       // the operands of `groups` components are resident together
 }
 
 // Factored projection of a low-rank head: log omega by the dense kernel's sum tiles, z = B h by a plain GEMM, its split
@@ -920,15 +935,12 @@ int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, cons
   const int units = c.n * c.r, k = h->lr_k;
   int rc = launch_gemm(h, kModeLogprob, hidden_bf16, T, 1, false, true, targets, nullptr, nullptr, st);
   if (rc != MTPC_OK) return rc;
-  float* z32 = reinterpret_cast<float*>(h->ws + h->lr_off_z32);
   __nv_bfloat16* zhl = reinterpret_cast<__nv_bfloat16*>(h->ws + h->lr_off_zhl);
   const GemmOperand hid{hidden_bf16, static_cast<size_t>(c.d), false};
   const GemmOperand bmat{h->lr_B, static_cast<size_t>(c.d), false};          // [n r k, d], K = d contiguous
-  rc = launch_plain_gemm(h, hid, bmat, c.d, bmat, 0, 0, z32, static_cast<size_t>(units) * k, T, units * k, st);
+  // z = B h, leaving the GEMM's epilogue already split into its two bf16 halves [T, n r, 2, k]
+  rc = launch_plain_gemm(h, hid, bmat, c.d, bmat, 0, 0, nullptr, 0, T, units * k, st, zhl, k);
   if (rc != MTPC_OK) return rc;
-  const size_t total = static_cast<size_t>(T) * units * k;
-  const int blocks = static_cast<int>((total + 255) / 256 < 8192 ? (total + 255) / 256 : 8192);
-  lowrank_split_kernel<<<blocks, 256, 0, st>>>(z32, zhl, static_cast<size_t>(T) * units, k);
   LowRankGemmParams p = h->lr_params;
   rc = make_tmap(&p.tm_h, hidden_bf16, static_cast<uint64_t>(T), static_cast<uint64_t>(c.d), kBlockM);
   if (rc == MTPC_OK) rc = make_tmap_sw32(&p.tm_z, zhl, static_cast<uint64_t>(T), static_cast<uint64_t>(units) * 2 * k, kBlockM);
@@ -942,8 +954,8 @@ int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, cons
   const long long items = static_cast<long long>(p.m_tiles) * c.n;
   const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
   const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
-  mtpc_lowrank_gemm_kernel<<<grid, kGemmThreads, p.stages * p.stage_bytes + ctl, st>>>(p);
-  h->launches += 2;
+  mtpc_lowrank_gemm_kernel<<<grid, 64 + 128 * p.groups, p.stages * p.stage_bytes + ctl, st>>>(p);
+  h->launches += 1;
   return check_launch();
 }
 
@@ -1139,8 +1151,7 @@ struct LowRankSpec {
 static int lowrank_extra_bytes(const mtpc_config& c, int k, size_t base_total, size_t* off_z32, size_t* off_zhl, size_t* total) {
   const size_t units = static_cast<size_t>(c.n) * c.r;
   size_t off = align_up(base_total);
-  *off_z32 = off;
-  off += align_up(static_cast<size_t>(c.max_positions) * units * k * 4);
+  *off_z32 = off;                       // (no fp32 copy of z: the GEMM writes the halves itself)
   *off_zhl = off;
   off += align_up(static_cast<size_t>(c.max_positions) * units * 2 * k * 2);
   *total = off;

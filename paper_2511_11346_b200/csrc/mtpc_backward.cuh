@@ -663,6 +663,10 @@ struct PlainGemmParams {
   int wide_stores;       // C and ldc allow 32-byte stores
   float* C;
   size_t ldc;
+  // Instead of C (C == NULL): the result split into two bf16 halves, x = hi + lo, written as [M, N / split_k, 2, split_k]
+  // (group g of split_k columns: hi at column (2 g) split_k, lo at (2 g + 1) split_k; split_k a multiple of 16).
+  __nv_bfloat16* C_hilo;
+  int split_k;
   unsigned* status;
   uint64_t wait_limit_ns;   // limit of every pipeline wait
 };
@@ -805,7 +809,21 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
         float x[16];
         tmem_ld16(tcol + b * 16, x);
         const int col0 = nt * kPlainTileN + b * 16;
-        if (row < p.M && col0 < p.N) {                 // N is a multiple of 16
+        if (row < p.M && col0 < p.N && p.C == nullptr) {
+          // 16 columns of one group: 32 bytes of high halves and 32 bytes of low halves
+          const int grp = col0 / p.split_k, q0 = col0 - grp * p.split_k;
+          __align__(16) __nv_bfloat16 hi[16], lo[16];
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            hi[q] = __float2bfloat16_rn(x[q]);
+            lo[q] = __float2bfloat16_rn(x[q] - __bfloat162float(hi[q]));
+          }
+          __nv_bfloat16* dst = p.C_hilo + static_cast<size_t>(row) * (2 * p.N) + static_cast<size_t>(2 * grp) * p.split_k + q0;
+          reinterpret_cast<uint4*>(dst)[0] = reinterpret_cast<const uint4*>(hi)[0];
+          reinterpret_cast<uint4*>(dst)[1] = reinterpret_cast<const uint4*>(hi)[1];
+          reinterpret_cast<uint4*>(dst + p.split_k)[0] = reinterpret_cast<const uint4*>(lo)[0];
+          reinterpret_cast<uint4*>(dst + p.split_k)[1] = reinterpret_cast<const uint4*>(lo)[1];
+        } else if (row < p.M && col0 < p.N) {          // N is a multiple of 16
           if (p.wide_stores) {                         // 32-byte aligned rows: one full sector per store
             st_global_v8(crow + col0, x);
             st_global_v8(crow + col0 + 8, x + 8);

@@ -3,13 +3,17 @@
 // tensor is never formed. Per (128 positions, slot i):
 //   base    = h W_i^T            one weight-sized-over-r contraction (K = d), v accumulator columns kept in tensor memory;
 //   corr_j  = z_j A_ij^T         for each of the r components one K = k contraction on z_j = B_ij h (computed by a plain
-//                                GEMM beforehand and split into two bf16 halves, z = hi + lo, so that rounding z to the
+//                                GEMM beforehand whose epilogue splits it into two bf16 halves, z = hi + lo, so that rounding z to the
 //                                tensor cores' operand type costs 2^-17 instead of 2^-9), in chunks of `chunk_cols` columns
-//                                through two accumulator slots;
+//                                through a few accumulator slots (enough of them in flight to cover the round trip
+//                                slot released -> MMAs issued -> commit seen, which is longer than a chunk's epilogue);
 //   epilogue: x = base + corr_j, then exactly the log-likelihood epilogue of the dense kernel (online log-sum-exp over the
 //             unit's v columns, target gather, G = logit[target] - LSE).
 // FLOPs per position: 2 d (n v + n r k) + 4 n r v k instead of 2 d n r v.
-// Same roles as the dense kernel: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue (one thread per position).
+// Roles: warp 0 TMA producer, warp 1 MMA issuer, then `groups` epilogue groups of four warps (one thread per position):
+// group g takes the components j = g, g + groups, ... of a slot and owns two correction slots. The epilogue (one
+// exponential per logit, n r v of them per position) is what bounds this kernel once the contraction has shrunk, and a
+// lone warp per scheduler cannot keep the special-function pipe busy: several groups can.
 // One shared-memory ring carries both kinds of entries: a 64-wide K block of (h, W_i), or the operands of one component's
 // correction (z_hi, z_lo: k/16 boxes of 128 rows x 16 each; A_ij: k/16 x nchunk boxes of chunk_cols rows x 16), all as
 // 32-byte rows with the 32-byte swizzle, so every correction MMA (K = 16) starts at the base of its own box.
@@ -22,7 +26,8 @@
 namespace mtpc {
 
 constexpr int kLrMaxRank = 32;          // k <= 32 (a multiple of 16)
-constexpr int kLrBaseSlot = 2;          // barrier index of the base accumulator (0, 1: the correction slots)
+constexpr int kLrMaxGroups = 3;         // epilogue groups: 64 + 128 * groups threads per CTA
+constexpr int kLrBaseSlot = kMaxSlots - 1;   // barrier index of the base accumulator (0 .. corr_slots - 1: the correction slots)
 
 struct LowRankGemmParams {
   CUtensorMap tm_h;      // hidden [T, d]              box 64 x 128, 128-byte swizzle
@@ -33,7 +38,8 @@ struct LowRankGemmParams {
   int n, r, v, vv, k;
   int base_boxes, base_box_rows;     // W_i is fetched as base_boxes boxes of base_box_rows rows (v > 256: two halves)
   int chunk_cols, nchunk;            // correction chunks: nchunk = ceil(v / chunk_cols)
-  int corr_col0;                     // first tensor-memory column of correction slot 0 (slot 1 follows at + chunk_cols)
+  int corr_col0;                     // first tensor-memory column of correction slot 0 (slot s follows at + s * chunk_cols)
+  int groups;                        // epilogue groups (1 .. kLrMaxGroups), each with two correction slots of chunk_cols columns
   int stages, stage_bytes;
   const int* targets;                // [T, n]
   float* G;                          // [T, n, r]
@@ -54,7 +60,7 @@ __device__ __forceinline__ uint64_t umma_smem_desc_kmajor(uint32_t smem_addr, ui
   return d;
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 1) mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
+__global__ void __launch_bounds__(64 + 128 * kLrMaxGroups, 1) mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
@@ -75,12 +81,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_lowrank_gemm_kernel(cons
       mbar_init(smem_u32(&ctl->full[s]), 1);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < 2 * p.groups; ++s) {
       mbar_init(smem_u32(&ctl->tfull[s]), 1);
       mbar_init(smem_u32(&ctl->tempty[s]), 4);
     }
     mbar_init(smem_u32(&ctl->tfull[kLrBaseSlot]), 1);
-    mbar_init(smem_u32(&ctl->tempty[kLrBaseSlot]), 4);
+    mbar_init(smem_u32(&ctl->tempty[kLrBaseSlot]), 4 * p.groups);
     mbar_init(smem_u32(&ctl->drain), 1);
     ctl->abort = 0;
     ctl->wait_limit_ns = p.wait_limit_ns;
@@ -152,7 +158,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_lowrank_gemm_kernel(cons
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      uint32_t stage = 0, phase = 0, it = 0, cuse = 0;
+      uint32_t stage = 0, phase = 0, it = 0;
+      uint32_t cuse[kLrMaxGroups] = {0, 0, 0};                      // chunks issued so far for each epilogue group
       bool ok = true;
       const int base_n = p.base_box_rows;                           // columns per base MMA (v, or v / 2)
       const uint32_t idesc_base = umma_idesc_bf16(kBlockM, base_n);
@@ -177,30 +184,40 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_lowrank_gemm_kernel(cons
         }
         if (!ok) break;
         umma_commit(smem_u32(&ctl->tfull[kLrBaseSlot]));
-        // ---- corrections: component j, chunk c -> correction slot (cuse & 1)
-        for (int j = 0; j < p.r && ok; ++j) {
-          if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t addr = tiles_addr + stage * p.stage_bytes;
-          for (int c = 0; c < p.nchunk; ++c, ++cuse) {
-            const uint32_t slot = cuse & 1u;
-            if (!bounded_wait(smem_u32(&ctl->tempty[slot]), ((cuse >> 1) & 1u) ^ 1u, ctl, p.status)) { ok = false; break; }
-            tc_fence_after();
-            const int width = min(p.chunk_cols, p.v - c * p.chunk_cols);
-            const uint32_t idesc = umma_idesc_bf16(kBlockM, width);
-            const uint32_t d_tmem = tmem_base + p.corr_col0 + slot * p.chunk_cols;
-            uint32_t acc = 0;
-            for (int part = 0; part < 2; ++part)
-              for (int q = 0; q < kq; ++q) {
-                umma_bf16(d_tmem, umma_smem_desc_kmajor(addr + (part * kq + q) * zbox, 32),
-                          umma_smem_desc_kmajor(addr + a_off + (q * p.nchunk + c) * abox, 32), idesc, acc);
-                acc = 1;
-              }
-            umma_commit(smem_u32(&ctl->tfull[slot]));
+        // ---- corrections, `groups` components at a time (component j0 + g belongs to epilogue group g): their chunks
+        // are issued in turn, chunk c of component j0 + g into slot 2 g + (that group's chunk count & 1)
+        for (int j0 = 0; j0 < p.r && ok; j0 += p.groups) {
+          const int ng = min(p.groups, p.r - j0);
+          uint32_t addr[kLrMaxGroups], estage[kLrMaxGroups];
+          for (int g = 0; g < ng && ok; ++g) {
+            if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
+            addr[g] = tiles_addr + stage * p.stage_bytes;
+            estage[g] = stage;
+            next_stage();
           }
           if (!ok) break;
-          umma_commit(smem_u32(&ctl->empty[stage]));
-          next_stage();
+          tc_fence_after();
+          for (int c = 0; c < p.nchunk && ok; ++c) {
+            const int width = min(p.chunk_cols, p.v - c * p.chunk_cols);
+            const uint32_t idesc = umma_idesc_bf16(kBlockM, width);
+            for (int g = 0; g < ng; ++g) {
+              const uint32_t slot = 2 * g + (cuse[g] & 1u);
+              if (!bounded_wait(smem_u32(&ctl->tempty[slot]), ((cuse[g] >> 1) & 1u) ^ 1u, ctl, p.status)) { ok = false; break; }
+              tc_fence_after();
+              const uint32_t d_tmem = tmem_base + p.corr_col0 + slot * p.chunk_cols;
+              uint32_t acc = 0;
+              for (int part = 0; part < 2; ++part)
+                for (int q = 0; q < kq; ++q) {
+                  umma_bf16(d_tmem, umma_smem_desc_kmajor(addr[g] + (part * kq + q) * zbox, 32),
+                            umma_smem_desc_kmajor(addr[g] + a_off + (q * p.nchunk + c) * abox, 32), idesc, acc);
+                  acc = 1;
+                }
+              umma_commit(smem_u32(&ctl->tfull[slot]));
+              ++cuse[g];
+            }
+          }
+          if (!ok) break;
+          for (int g = 0; g < ng; ++g) umma_commit(smem_u32(&ctl->empty[estage[g]]));
         }
       }
       if (!ok) {   // wait (bounded) for the MMAs already issued before tensor memory is freed
@@ -213,6 +230,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_lowrank_gemm_kernel(cons
   } else {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;
+    const int group = (warp - 2) >> 2;                        // this warp's epilogue group: components group, group + groups, ...
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     uint32_t it = 0, cuse = 0;
     bool ok = true;
@@ -223,10 +241,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_lowrank_gemm_kernel(cons
       const int tgt = valid ? p.targets[static_cast<size_t>(row) * p.n + slot_i] : -1;
       if (!bounded_wait_warp(smem_u32(&ctl->tfull[kLrBaseSlot]), it & 1u, ctl, p.status, lane)) { ok = false; break; }
       tc_fence_after();
-      for (int j = 0; j < p.r && ok; ++j) {
+      for (int j = group; j < p.r && ok; j += p.groups) {
         float m = -CUDART_INF_F, s = 0.f, tval = 0.f;
         for (int c = 0; c < p.nchunk; ++c, ++cuse) {
-          const uint32_t slot = cuse & 1u;
+          const uint32_t slot = 2 * group + (cuse & 1u);
           if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (cuse >> 1) & 1u, ctl, p.status, lane)) { ok = false; break; }
           tc_fence_after();
           const int col_chunk = c * p.chunk_cols;
@@ -239,7 +257,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_lowrank_gemm_kernel(cons
             for (int q = 0; q < 16; ++q) x[q] = __uint_as_float(rc[q]) + __uint_as_float(rb[q]);
             const int col0 = col_chunk + b * 16;
             mask_padding(x, col0, p.vv);
-            // the epilogue warp is alone on its scheduler, so dependent chains cost their full latency: reduce as trees
+            // short dependent chains: reduce as trees
             float t8[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q) t8[q] = fmaxf(x[q], x[q + 8]);
@@ -316,20 +334,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_lowrank_gemm_kernel(cons
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
-  }
-}
-
-// z [T, units, k] fp32 (the plain GEMM's output) -> [T, units, 2, k] bf16: hi = bf16(z), lo = bf16(z - hi).
-__global__ void lowrank_split_kernel(const float* __restrict__ z, __nv_bfloat16* __restrict__ out, size_t rows_units, int k) {
-  const size_t total = rows_units * k;
-  for (size_t e = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; e < total;
-       e += static_cast<size_t>(gridDim.x) * blockDim.x) {
-    const size_t ru = e / k;
-    const int q = static_cast<int>(e - ru * k);
-    const float x = z[e];
-    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-    out[(ru * 2) * k + q] = hi;
-    out[(ru * 2 + 1) * k + q] = __float2bfloat16_rn(x - __bfloat162float(hi));
   }
 }
 

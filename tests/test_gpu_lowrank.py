@@ -143,6 +143,7 @@ FACTORED = [
     (I.BTREE, 4, 4, 48, 44, 64, 16, 70),       # padded vocabulary, tree circuit
     (I.HMM_CTX, 3, 8, 320, 0, 128, 16, 200),   # contextual transitions: many sum tiles beside the factored projection
     (I.CP, 1, 1, 16, 0, 64, 16, 5),            # the smallest everything
+    (I.CP, 2, 4, 480, 0, 64, 16, 140),         # the widest unit that leaves room for corrections: two 16-column slots
 ]
 
 
@@ -214,5 +215,5 @@ def test_factored_head_agrees_with_the_dense_head_on_the_composed_tensor_and_ref
     need = ctypes.c_size_t(0)
     assert B.lib().mtpc_lowrank_workspace_bytes(ctypes.byref(cfg), 8, ctypes.byref(need)) == -3      # rank not 16 or 32
     assert B.lib().mtpc_lowrank_workspace_bytes(ctypes.byref(cfg), 16, ctypes.byref(need)) == 0 and need.value > 0
-    big = B.MtpcConfig(family, n, r, 480, d, B.MTPC_BF16, T, 1, 0, 0)                                 # no room for the corrections
+    big = B.MtpcConfig(family, n, r, 512, d, B.MTPC_BF16, T, 1, 0, 0)                                 # no room for the corrections
     assert B.lib().mtpc_lowrank_workspace_bytes(ctypes.byref(big), 16, ctypes.byref(need)) == -3
