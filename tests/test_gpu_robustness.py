@@ -168,3 +168,52 @@ def test_a_wait_that_runs_out_is_reported_and_the_head_recovers(path):
         assert np.abs(out_lp.cpu().numpy()[same] - ref["logprob"][same]).max() <= LOGPROB_TOL
     assert dh.head.mtpc_get_status(with_code=True) == (B.MTPC_OK, 0)
     dh.close()
+
+
+@pytest.mark.parametrize("family,n,r,v,d,P,wpp", [
+    (I.CP, 8, 16, 320, 256, 8, 16),         # few positions: weight pass, per-slot kernel and circuit as dependent launches
+    (I.HMM, 4, 8, 64, 128, 5, 3),
+    (I.BTREE, 8, 8, 64, 64, 200, 2),        # many positions: sorted draws, projection passes, circuit
+])
+def test_draft_and_acceptance_calls_can_be_captured_into_a_cuda_graph(family, n, r, v, d, P, wpp):
+    """The calls only enqueue work on the caller's stream (no synchronisation, no allocation), so a serving loop may
+    capture draft + acceptance once and replay the graph: the replay must return what the plain calls return, and they
+    what the oracle returns."""
+    wl = I.make_workload("graph", I.HeadShape(family, n, r, v, d), P, seed=900 + n + r, wpp=wpp, weight_std=0.25)
+    dh = DeviceHead(wl)
+    W = P * wpp
+    hidden = dh.hidden_device()
+    u = torch.from_numpy(wl.uniforms).cuda()
+    tp = torch.from_numpy(I.target_rows(I.BASE_SEED + 5, 9, (W, n + 1, v))).cuda()
+    ua = torch.from_numpy(I.uniforms(I.BASE_SEED + 6, 10, (W, n + 1))).cuda()
+
+    def buffers():
+        return (torch.zeros((W, n), dtype=torch.int32, device="cuda"), torch.zeros((W, n), dtype=torch.float32, device="cuda"),
+                torch.zeros(W, dtype=torch.int32, device="cuda"), torch.zeros(W, dtype=torch.int32, device="cuda"))
+
+    def cycle(ob, opre, oacc, onxt, stream=None):
+        dh.head.mtpc_draft_sample_prefix(hidden, wpp, u, ob, opre, stream=stream)
+        dh.head.mtpc_speculative_accept(P, wpp, ob, opre, tp, ua, oacc, onxt, stream=stream)
+
+    plain = buffers()
+    cycle(*plain)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    replayed = buffers()
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            cycle(*replayed, stream=side)
+        for t in replayed:
+            t.zero_()
+        graph.replay()
+        graph.replay()
+        side.synchronize()
+    assert dh.head.mtpc_get_status(with_code=True) == (B.MTPC_OK, 0)
+    for a, b in zip(plain, replayed):
+        np.testing.assert_array_equal(a.cpu().numpy(), b.cpu().numpy())
+    ref = orc.draft_sample(wl.shape.family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wpp, wl.uniforms)
+    differ = (replayed[0].cpu().numpy() != ref["bytes"]).any(axis=1)
+    assert not (differ & (ref["margin"] >= 1e-6)).any()
+    del graph
+    dh.close()
