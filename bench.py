@@ -162,7 +162,33 @@ def circuit_bytes(wl) -> int:
     return 4 * wl.T * (s.n * s.r + s.sum_rows + 1)
 
 
-def measure_decode_cell(torch, cell, steps: int, warmup: int):
+def graph_replay_times(torch, enqueue, outputs, steps: int, warmup: int):
+    """Capture enqueue(stream) once into a CUDA graph on a side stream, zero `outputs`, replay it `warmup` times untimed
+    and `steps` times timed (CUDA events on that stream, one replay each): the per-replay times in ms. The outputs hold
+    the last replay's results when it returns."""
+    side = torch.cuda.Stream()
+    times = []
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            enqueue(side)
+        for t in outputs:
+            t.zero_()
+        for _ in range(warmup):
+            graph.replay()
+        side.synchronize()
+        for _ in range(steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay()
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1))
+    del graph
+    return times
+
+
+def measure_decode_cell(torch, cell, steps: int, warmup: int, with_graph: bool = True):
     """Draft windows/s and p50 latency on one decode cell (family, n, P) with 16 windows per position. Every call
     is timed on its own (CUDA events on the launching stream); the library's event ring gives the per-kernel split."""
     from paper_2511_11346_b200.runner import DeviceHead
@@ -188,26 +214,11 @@ def measure_decode_cell(torch, cell, steps: int, warmup: int):
     # the same call captured once into a CUDA graph and replayed: what a serving loop pays once the host side of the
     # three launches (tensor-map encode, launch attributes, the binding) is out of the way; results must be identical
     ref_b, ref_l = ob.clone(), ol.clone()
-    side = torch.cuda.Stream()
-    graph_lat = []
-    with torch.cuda.stream(side):
-        graph = torch.cuda.CUDAGraph()
-        ob.zero_()
-        ol.zero_()
-        with torch.cuda.graph(graph, stream=side):
-            dh.head.mtpc_draft_sample(h, wl.wpp, u, ob, ol, stream=side)
-        for _ in range(warmup):
-            graph.replay()
-        side.synchronize()
+    graph_lat, graph_identical = [], None
+    if with_graph:
+        graph_lat = graph_replay_times(torch, lambda st: dh.head.mtpc_draft_sample(h, wl.wpp, u, ob, ol, stream=st),
+                                       (ob, ol), steps, warmup)
         graph_identical = bool((ob == ref_b).all()) and bool(((ol == ref_l) | (ol.isnan() & ref_l.isnan())).all())
-        for _ in range(steps):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            graph.replay()
-            e1.record()
-            e1.synchronize()
-            graph_lat.append(e0.elapsed_time(e1))
-    del graph
     # per-kernel split from the library's event ring (a second pass: the events serialise the kernels)
     ksteps = min(steps, 50)
     dh.head.mtpc_set_timing(ksteps)
@@ -236,50 +247,39 @@ def measure_decode_cell(torch, cell, steps: int, warmup: int):
             cyc.append(e0.elapsed_time(e1))
     mean_accepted = float(oacc.float().mean().cpu())
     ref_acc, ref_nxt = oacc.clone(), onxt.clone()
-    graph_cyc = []
-    with torch.cuda.stream(side):
-        graph = torch.cuda.CUDAGraph()
-        oacc.zero_()
-        onxt.zero_()
-        with torch.cuda.graph(graph, stream=side):
-            dh.head.mtpc_draft_sample_prefix(h, wl.wpp, u, ob, opre, stream=side)
-            dh.head.mtpc_speculative_accept(wl.T, wl.wpp, ob, opre, tp, ua, oacc, onxt, stream=side)
-        for _ in range(warmup):
-            graph.replay()
-        side.synchronize()
+    graph_cyc, cycle_identical = [], None
+    if with_graph:
+        def cycle(st):
+            dh.head.mtpc_draft_sample_prefix(h, wl.wpp, u, ob, opre, stream=st)
+            dh.head.mtpc_speculative_accept(wl.T, wl.wpp, ob, opre, tp, ua, oacc, onxt, stream=st)
+        graph_cyc = graph_replay_times(torch, cycle, (oacc, onxt), steps, warmup)
         cycle_identical = bool((oacc == ref_acc).all()) and bool((onxt == ref_nxt).all())
-        for _ in range(steps):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            graph.replay()
-            e1.record()
-            e1.synchronize()
-            graph_cyc.append(e0.elapsed_time(e1))
-    del graph
     status = dh.head.mtpc_get_status()
     p50 = statistics.median(lat)
     weight_bytes = (s.n * s.r * s.v + s.sum_rows) * s.d * 2
     peaks, src = load_peaks()
     gbs = weight_bytes / (p50 * 1e-3) / 1e9
-    graph_p50 = statistics.median(graph_lat)
+    graph_p50 = statistics.median(graph_lat) if with_graph else None
     gemm_gbs = weight_bytes / (phase_p50[0] * 1e-3) / 1e9
     out = {"workload": f"configs[4] {wl.name}: P={wl.T} wpp={wl.wpp} d={s.d} n={s.n} r={s.r} v={s.v}",
            "windows_per_s": W / (p50 * 1e-3), "p50_ms": p50, "calls": steps, "kernels_per_call": launches,
            "kernel_p50_ms": phase_p50, "device_status": status,
-           "cuda_graph_replay": {"p50_ms": graph_p50, "hbm_frac": weight_bytes / (graph_p50 * 1e-3) / 1e9 / peaks["hbm_gbs"],
+           "cuda_graph_replay": None if graph_p50 is None else {
+                                 "p50_ms": graph_p50, "hbm_frac": weight_bytes / (graph_p50 * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                  "results_identical_to_plain_call": graph_identical,
                                  "note": "mtpc_draft_sample captured once by the caller (torch.cuda.graph), replayed"},
            "draft_plus_accept": {"p50_ms": statistics.median(cyc), "kernels_per_call": launches + 1,
                                  "mean_accepted_bytes_vs_synthetic_target": mean_accepted,
                                  "calls": "mtpc_draft_sample_prefix + mtpc_speculative_accept",
-                                 "cuda_graph_replay_p50_ms": statistics.median(graph_cyc),
+                                 "cuda_graph_replay_p50_ms": statistics.median(graph_cyc) if with_graph else None,
                                  "cuda_graph_results_identical": cycle_identical},
            "hbm_roofline": {"algorithmic_bytes": weight_bytes, "note": "one pass over the emission and sum-unit weights",
                             "achieved_gbs": gbs, "peak_gbs": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
                             "weight_pass_kernel_gbs": gemm_gbs, "weight_pass_kernel_frac": gemm_gbs / peaks["hbm_gbs"],
                             "peak_source": src}}
     dh.close()
-    return out, launches * (2 * (steps + warmup) + 1 + min(steps, 50)) + (launches + 1) * (2 * (steps + warmup) + 1)
+    calls = (steps + warmup) + ((steps + warmup + 1) if with_graph else 0)        # plain loop; capture + replays
+    return out, launches * (calls + min(steps, 50)) + (launches + 1) * calls
 
 
 def measure_backward(torch, dh, wl, hidden, targets, steps: int, peaks):
@@ -716,7 +716,7 @@ def run_ours(args):
             cells = [({"cp": I.CP, "hmm": I.HMM}[fam], int(n_), int(p_))]
         sweep = []
         for cell in cells:
-            res, cell_launches = measure_decode_cell(torch, cell, steps=200, warmup=5)
+            res, cell_launches = measure_decode_cell(torch, cell, steps=200, warmup=5, with_graph=not args.no_graph)
             sweep.append(res)
             launches += cell_launches
         draft = next((c for c in sweep if "decode_cp_n8_P64" in c["workload"]), sweep[0])
@@ -770,6 +770,7 @@ def main():
                     help="draft measurement: 'all' twelve cells of the decode sweep, 'one' (CP n=8 P=64), or a single "
                          "cell as family:n:P, e.g. hmm:16:1")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiling runs)")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay of the draft calls (profiling runs)")
     ap.add_argument("--no-sustained", action="store_true", help="skip the second, seconds-long loop (profiling runs)")
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="default run only: skip configs[2] and configs[3] after the headline workload")

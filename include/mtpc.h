@@ -16,6 +16,10 @@
  *     allocates no device memory: all scratch lives in the caller's workspace.
  *   - Calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*) and return without
  *     waiting, except where stated. A head must not be used from two streams at once: its workspace is shared.
+ *     mtpc_window_logprob, mtpc_window_prefix_logprob, the two draft calls and mtpc_speculative_accept do nothing
+ *     else (no synchronisation, no allocation, nothing read back), so they may be recorded into a CUDA graph by
+ *     stream capture and replayed; the pointers they were given are then fixed for the life of the graph. With the
+ *     timing ring switched on (mtpc_set_timing) a call also records events and is not meant for capture.
  *   - Return value: MTPC_OK (0) or a negative MTPC_ERR_* code. Nothing throws or aborts across this ABI and
  *     the device code never traps: data errors only the device can see (target >= v, uniform outside [0,1),
  *     a bounded wait that ran out) set bits in a device status word, read with mtpc_get_status, and put

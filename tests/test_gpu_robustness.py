@@ -187,13 +187,18 @@ def test_draft_and_acceptance_calls_can_be_captured_into_a_cuda_graph(family, n,
     tp = torch.from_numpy(I.target_rows(I.BASE_SEED + 5, 9, (W, n + 1, v))).cuda()
     ua = torch.from_numpy(I.uniforms(I.BASE_SEED + 6, 10, (W, n + 1))).cuda()
 
+    targets = torch.from_numpy(wl.targets).cuda()
+
     def buffers():
         return (torch.zeros((W, n), dtype=torch.int32, device="cuda"), torch.zeros((W, n), dtype=torch.float32, device="cuda"),
-                torch.zeros(W, dtype=torch.int32, device="cuda"), torch.zeros(W, dtype=torch.int32, device="cuda"))
+                torch.zeros(W, dtype=torch.int32, device="cuda"), torch.zeros(W, dtype=torch.int32, device="cuda"),
+                torch.zeros(P, dtype=torch.float32, device="cuda"), torch.zeros((P, n), dtype=torch.float32, device="cuda"))
 
-    def cycle(ob, opre, oacc, onxt, stream=None):
+    def cycle(ob, opre, oacc, onxt, lp, pre, stream=None):
         dh.head.mtpc_draft_sample_prefix(hidden, wpp, u, ob, opre, stream=stream)
         dh.head.mtpc_speculative_accept(P, wpp, ob, opre, tp, ua, oacc, onxt, stream=stream)
+        dh.head.mtpc_window_logprob(hidden, targets, lp, stream=stream)           # the likelihood calls as well
+        dh.head.mtpc_window_prefix_logprob(hidden, targets, pre, stream=stream)
 
     plain = buffers()
     cycle(*plain)
@@ -215,5 +220,7 @@ def test_draft_and_acceptance_calls_can_be_captured_into_a_cuda_graph(family, n,
     ref = orc.draft_sample(wl.shape.family, wl.hidden_q, wl.W_emit_q, wl.W_sum_q, wl.T_static, wpp, wl.uniforms)
     differ = (replayed[0].cpu().numpy() != ref["bytes"]).any(axis=1)
     assert not (differ & (ref["margin"] >= 1e-6)).any()
+    assert np.abs(replayed[4].cpu().numpy() - oracle_logprob(wl)).max() <= LOGPROB_TOL
+    assert np.abs(replayed[5].cpu().numpy()[:, -1] - oracle_logprob(wl)).max() <= LOGPROB_TOL
     del graph
     dh.close()
