@@ -390,7 +390,7 @@ def measure_factored_forward(torch, wl, lowrank, steps: int):
     return {"call": "mtpc_window_logprob on a factored head", "ms_per_call": ms, "projection_phase_ms": proj_ms,
             "positions_per_s": wl.T / (ms * 1e-3), "flops_per_call": flops, "achieved_tflops": flops / (proj_ms * 1e-3) / 1e12,
             "dense_flops_per_call": algorithmic_flops(wl), "device_status": status,
-            "note": "projection phase = sum-unit tiles + z = B h (plain GEMM) + split + factored kernel; the softmax over "
+            "note": "projection phase = sum-unit tiles + z = B h (a plain GEMM that writes z as two bf16 halves) + factored kernel; the softmax over "
                     "n r v logits per position is the same as in the dense head and now dominates"}
 
 
