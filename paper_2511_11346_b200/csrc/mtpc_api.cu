@@ -290,7 +290,7 @@ struct mtpc_head {
   const void* lr_W_base;                        // [n, v, d] bf16
   const void* lr_A;                             // [n, r, v, k] bf16
   const void* lr_B;                             // [n, r, k, d] bf16
-  size_t lr_off_z32, lr_off_zhl;                // workspace: z = B h as fp32 [T, n r k], then split into bf16 halves [T, n r, 2, k]
+  size_t lr_off_zhl, lr_off_partial;            // workspace: z = B h as bf16 halves [T, n r, 2, k]; per-panel partial log-sum-exps
   LowRankGemmParams lr_params;                  // everything of the factored projection launch that does not depend on the call
   int max_pairs;                                // clusters of two projection CTAs that can be resident at once
   CUtensorMap tm_emit_dec, tm_sum_dec;          // the same matrices in the few-position draft path's tiles
@@ -896,35 +896,47 @@ constexpr int kLrGroups = MTPC_LR_GROUPS;   // epilogue groups of the factored p
 // Tiling of the factored projection (mtpc_lowrank_gemm.cuh) for a head shape; false: the shape does not fit.
 bool plan_lowrank(const mtpc_config& c, int k, LowRankGemmParams* p) {
   if (k < 16 || k > kLrMaxRank || k % 16 != 0 || c.v % 16 != 0) return false;
-  const int base_cols = (c.v + 31) / 32 * 32;
-  // beside the base accumulator: two correction slots for each of `groups` epilogue groups; as many groups (up to
-  // kLrGroups, and no more than there are components) as leave chunks of at least 32 columns, else narrower chunks
-  const int spare = kTmemCols - base_cols;
+  // the fewest panels whose two base buffers leave room for the correction slots (two per epilogue group, chunks of at
+  // least 16 columns; as many groups, up to kLrGroups and the number of components, as leave chunks of at least 32)
+  int panels = 0, pc = 0, stride = 0, spare = 0;
+  for (int np = 1; np <= kLrMaxPanels; ++np) {
+    pc = ((c.v + np - 1) / np + 15) / 16 * 16;          // the last panel may be narrower
+    stride = (pc + 31) / 32 * 32;
+    spare = kTmemCols - 2 * stride;
+    if (pc <= 256 && spare >= 32) { panels = (c.v + pc - 1) / pc; break; }
+  }
+  if (panels == 0) return false;
   int groups = kLrGroups < c.r ? kLrGroups : c.r;
   while (groups > 1 && spare / (2 * groups) < 32) --groups;
   int chunk = spare / (2 * groups) / 16 * 16;
   if (chunk > 96) chunk = 96;
-  if (chunk < 16) return false;
-  if (chunk > c.v) chunk = c.v;
+  if (chunk > pc) chunk = pc;
   p->groups = groups;
   p->n = c.n; p->r = c.r; p->v = c.v; p->k = k;
   p->vv = c.v_valid > 0 ? c.v_valid : c.v;
   p->kblocks = c.d / kBlockK;
-  p->base_boxes = (c.v + 255) / 256;
-  if (c.v % p->base_boxes != 0 || (c.v / p->base_boxes) % 16 != 0) return false;
-  p->base_box_rows = c.v / p->base_boxes;
+  p->panels = panels;
+  p->panel_cols = pc;
+  p->acc_stride = stride;
   p->chunk_cols = chunk;
-  p->nchunk = (c.v + chunk - 1) / chunk;
-  p->corr_col0 = base_cols;
+  p->nchunk = (pc + chunk - 1) / chunk;
+  p->corr_col0 = 2 * stride;
   const int kq = k / 16;
-  const int base_entry = kABytes + c.v * kBlockK * 2;
-  const int corr_entry = 2 * kq * kBlockM * 32 + kq * p->nchunk * chunk * 32;
-  const int entry = base_entry > corr_entry ? base_entry : corr_entry;
-  p->stage_bytes = (entry + 1023) / 1024 * 1024;
-  const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
-  p->stages = (kSmemLimit - ctl) / p->stage_bytes;
-  if (p->stages > kMaxStages) p->stages = kMaxStages;
-  return p->stages >= groups + 1;       // the operands of `groups` components are resident together
+  p->base_stage_bytes = kABytes + pc * kBlockK * 2;                                  // a multiple of 1024 (pc % 16 == 0)
+  p->corr_stage_bytes = (2 * kq * kBlockM * 32 + kq * p->nchunk * chunk * 32 + 1023) / 1024 * 1024;
+  const int ctl = 1024 + static_cast<int>(sizeof(LowRankControl));
+  // the operands of `groups` components are resident together and the next ones on their way; the base ring takes the rest
+  for (int cs = kLrCorrStages; cs >= groups + 1; --cs) {
+    const int left = kSmemLimit - ctl - cs * p->corr_stage_bytes;
+    int bs = left / p->base_stage_bytes;
+    if (bs > kMaxStages) bs = kMaxStages;
+    if (bs >= 3 || (bs == 2 && cs == groups + 1)) {
+      p->corr_stages = cs;
+      p->base_stages = bs;
+      return true;
+    }
+  }
+  return false;
 }
 
 // Factored projection of a low-rank head: log omega by the dense kernel's sum tiles, z = B h by a plain GEMM, its split
@@ -951,11 +963,21 @@ int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, cons
   p.G = at<float>(h, L.off_G);
   p.status = at<unsigned>(h, L.off_status);
   p.wait_limit_ns = h->wait_limit_ns;
-  const long long items = static_cast<long long>(p.m_tiles) * c.n;
+  const size_t entries = static_cast<size_t>(T) * units;
+  p.partial = reinterpret_cast<float2*>(h->ws + h->lr_off_partial);
+  p.target_logit = reinterpret_cast<float*>(h->ws + h->lr_off_partial +
+                                            static_cast<size_t>(p.panels) * c.max_positions * units * sizeof(float2));
+  const long long items = static_cast<long long>(p.m_tiles) * c.n * p.panels;
   const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
-  const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
-  mtpc_lowrank_gemm_kernel<<<grid, 64 + 128 * p.groups, p.stages * p.stage_bytes + ctl, st>>>(p);
+  const int ctl = 1024 + static_cast<int>(sizeof(LowRankControl));
+  mtpc_lowrank_gemm_kernel<<<grid, kLrRoleThreads + 128 * p.groups,
+                             p.base_stages * p.base_stage_bytes + p.corr_stages * p.corr_stage_bytes + ctl, st>>>(p);
   h->launches += 1;
+  if (p.panels > 1) {     // several panels per unit: their partial log-sum-exps are combined into G
+    lowrank_merge_kernel<<<static_cast<unsigned>((entries + 255) / 256), 256, 0, st>>>(
+        p.partial, p.target_logit, targets, p.G, p.status, entries, c.r, p.vv, p.panels);
+    h->launches += 1;
+  }
   return check_launch();
 }
 
@@ -1148,12 +1170,16 @@ struct LowRankSpec {
   const void* B;
 };
 
-static int lowrank_extra_bytes(const mtpc_config& c, int k, size_t base_total, size_t* off_z32, size_t* off_zhl, size_t* total) {
+// Workspace of a factored head beyond the dense layout: z = B h as two bf16 halves [T, n r, 2, k] (written by the GEMM
+// that computes it), and, where a unit is cut into panels, the panels' (maximum, sum) pairs and the targets' logits.
+static int lowrank_extra_bytes(const mtpc_config& c, int k, int panels, size_t base_total, size_t* off_zhl,
+                               size_t* off_partial, size_t* total) {
   const size_t units = static_cast<size_t>(c.n) * c.r;
   size_t off = align_up(base_total);
-  *off_z32 = off;                       // (no fp32 copy of z: the GEMM writes the halves itself)
   *off_zhl = off;
   off += align_up(static_cast<size_t>(c.max_positions) * units * 2 * k * 2);
+  *off_partial = off;
+  if (panels > 1) off += align_up(static_cast<size_t>(c.max_positions) * units * (panels * sizeof(float2) + sizeof(float)));
   *total = off;
   return MTPC_OK;
 }
@@ -1169,11 +1195,11 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
   if (rc != MTPC_OK) return rc;
   LowRankGemmParams lrp;
   memset(&lrp, 0, sizeof(lrp));
-  size_t lr_z32 = 0, lr_zhl = 0;
+  size_t lr_zhl = 0, lr_partial = 0;
   if (lowrank) {
     if (cfg->io_dtype != MTPC_BF16) return MTPC_ERR_UNSUPPORTED;
     if (!plan_lowrank(*cfg, lowrank->k, &lrp)) return MTPC_ERR_UNSUPPORTED;
-    lowrank_extra_bytes(*cfg, lowrank->k, L.total, &lr_z32, &lr_zhl, &L.total);
+    lowrank_extra_bytes(*cfg, lowrank->k, lrp.panels, L.total, &lr_zhl, &lr_partial, &L.total);
   }
   const bool ctx = (cfg->flags & MTPC_FLAG_HMM_CONTEXTUAL) != 0;
   if (cfg->family == MTPC_HMM && cfg->n > 1 && !ctx && !T_static) return MTPC_ERR_NULL;
@@ -1194,8 +1220,8 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
     h->lr_W_base = lowrank->W_base;
     h->lr_A = lowrank->A;
     h->lr_B = lowrank->B;
-    h->lr_off_z32 = lr_z32;
     h->lr_off_zhl = lr_zhl;
+    h->lr_off_partial = lr_partial;
     h->lr_params = lrp;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1229,7 +1255,7 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
     fail = !allow_full_smem(mtpc_lowrank_gemm_kernel);
     rc = fail ? MTPC_ERR_CUDA
               : make_tmap(&h->lr_params.tm_w, lowrank->W_base, static_cast<uint64_t>(cfg->n) * cfg->v, cfg->d,
-                          h->lr_params.base_box_rows);
+                          h->lr_params.panel_cols);
     if (rc == MTPC_OK)
       rc = make_tmap_sw32(&h->lr_params.tm_a, lowrank->A, static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v, lowrank->k,
                           h->lr_params.chunk_cols);
@@ -1253,7 +1279,7 @@ int mtpc_lowrank_workspace_bytes(const mtpc_config* cfg, int32_t k, size_t* out_
   LowRankGemmParams lrp;
   if (cfg->io_dtype != MTPC_BF16 || !plan_lowrank(*cfg, k, &lrp)) return MTPC_ERR_UNSUPPORTED;
   size_t a = 0, b = 0;
-  return lowrank_extra_bytes(*cfg, k, L.total, &a, &b, out_bytes);
+  return lowrank_extra_bytes(*cfg, k, lrp.panels, L.total, &a, &b, out_bytes);
 }
 
 int mtpc_create_head_lowrank(const mtpc_config* cfg, int32_t k, const void* W_base, const void* A, const void* B,

@@ -1,50 +1,68 @@
 // Projection kernel of a head whose unembeddings are shared across the components of a slot and adapted by low-rank
 // terms (App. G): U_ij = W_i + A_ij B_ij, so logit[t, i, j, :] = W_i h_t + A_ij (B_ij h_t). The composed [n, r, v, d]
-// tensor is never formed. Per (128 positions, slot i):
-//   base    = h W_i^T            one weight-sized-over-r contraction (K = d), v accumulator columns kept in tensor memory;
-//   corr_j  = z_j A_ij^T         for each of the r components one K = k contraction on z_j = B_ij h (computed by a plain
-//                                GEMM beforehand whose epilogue splits it into two bf16 halves, z = hi + lo, so that rounding z to the
-//                                tensor cores' operand type costs 2^-17 instead of 2^-9), in chunks of `chunk_cols` columns
-//                                through a few accumulator slots (enough of them in flight to cover the round trip
-//                                slot released -> MMAs issued -> commit seen, which is longer than a chunk's epilogue);
-//   epilogue: x = base + corr_j, then exactly the log-likelihood epilogue of the dense kernel (online log-sum-exp over the
-//             unit's v columns, target gather, G = logit[target] - LSE).
+// tensor is never formed. A unit's v columns are cut into `panels` panels of panel_cols columns (the last one may be
+// narrower); a work item is (128 positions, slot i, panel):
+//   base    = h W_i^T            the panel's columns of the one weight-sized-over-r contraction (K = d), accumulated into one
+//                                of TWO tensor-memory buffers, so that the next item's base runs while this item's
+//                                corrections and epilogue are under way;
+//   corr_j  = z_j A_ij^T         for each of the r components one K = 2k contraction on z_j = B_ij h (computed by a plain
+//                                GEMM beforehand whose epilogue splits it into two bf16 halves, z = hi + lo, so that rounding z to
+//                                the tensor cores' operand type costs 2^-17 instead of 2^-9), in chunks of chunk_cols columns
+//                                through two accumulator slots per epilogue group;
+//   epilogue: x = base + corr_j, then the log-likelihood epilogue of the dense kernel on the panel (online log-sum-exp,
+//             target gather). One panel: G = logit[target] - LSE directly. Several: every panel leaves (max, sum of
+//             exponentials) per (position, slot, component), the panel that holds the target leaves its logit, and
+//             lowrank_merge_kernel combines them - so the items are independent and deal out evenly.
 // FLOPs per position: 2 d (n v + n r k) + 4 n r v k instead of 2 d n r v.
-// Roles: warp 0 TMA producer, warp 1 MMA issuer, then `groups` epilogue groups of four warps (one thread per position):
-// group g takes the components j = g, g + groups, ... of a slot and owns two correction slots. The epilogue (one
-// exponential per logit, n r v of them per position) is what bounds this kernel once the contraction has shrunk, and a
-// lone warp per scheduler cannot keep the special-function pipe busy: several groups can.
-// One shared-memory ring carries both kinds of entries: a 64-wide K block of (h, W_i), or the operands of one component's
-// correction (z_hi, z_lo: k/16 boxes of 128 rows x 16 each; A_ij: k/16 x nchunk boxes of chunk_cols rows x 16), all as
-// 32-byte rows with the 32-byte swizzle, so every correction MMA (K = 16) starts at the base of its own box.
+// Roles: warp 0 TMA producer of the base operands, warp 1 MMA issuer of the base, warp 2 TMA producer of the correction
+// operands, warp 3 MMA issuer of the corrections, then `groups` epilogue groups of four warps (one thread per position):
+// group g takes the components j = g, g + groups, ... The two pipelines share nothing but the tensor cores: each has its
+// own shared-memory ring (base: a 64-wide K block of h and of the panel's rows of W_i, 128-byte swizzle; corrections: z_hi,
+// z_lo as k/16 boxes of 128 rows x 16 and A_ij as k/16 x nchunk boxes of chunk_cols rows x 16, 32-byte rows with the
+// 32-byte swizzle, so every correction MMA (K = 16) starts at the base of its own box) and its own barriers.
 #pragma once
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
+#include "mtpc_circuit.cuh"
 #include "mtpc_gemm.cuh"
 
 namespace mtpc {
 
 constexpr int kLrMaxRank = 32;          // k <= 32 (a multiple of 16)
-constexpr int kLrMaxGroups = 3;         // epilogue groups: 64 + 128 * groups threads per CTA
-constexpr int kLrBaseSlot = kMaxSlots - 1;   // barrier index of the base accumulator (0 .. corr_slots - 1: the correction slots)
+constexpr int kLrMaxGroups = 3;         // epilogue groups: 128 + 128 * groups threads per CTA
+constexpr int kLrMaxPanels = 8;
+constexpr int kLrCorrStages = 4;        // entries of the correction operand ring (at most)
+constexpr int kLrRoleThreads = 128;     // the four single-thread roles, one warp each
 
 struct LowRankGemmParams {
   CUtensorMap tm_h;      // hidden [T, d]              box 64 x 128, 128-byte swizzle
-  CUtensorMap tm_w;      // W_base [n*v, d]            box 64 x base_box_rows, 128-byte swizzle
+  CUtensorMap tm_w;      // W_base [n*v, d]            box 64 x panel_cols, 128-byte swizzle
   CUtensorMap tm_z;      // z      [T, n*r*2*k]        box 16 x 128, 32-byte swizzle (unit u: hi at (2u)k, lo at (2u+1)k)
   CUtensorMap tm_a;      // A      [n*r*v, k]          box 16 x chunk_cols, 32-byte swizzle
   int T, m_tiles, kblocks;
   int n, r, v, vv, k;
-  int base_boxes, base_box_rows;     // W_i is fetched as base_boxes boxes of base_box_rows rows (v > 256: two halves)
-  int chunk_cols, nchunk;            // correction chunks: nchunk = ceil(v / chunk_cols)
+  int panels, panel_cols;            // panel q covers the columns [q panel_cols, min(v, (q + 1) panel_cols)) of a unit
+  int acc_stride;                    // tensor-memory columns between the two base buffers (panel_cols rounded up to 32)
+  int chunk_cols, nchunk;            // correction chunks of a full panel: nchunk = ceil(panel_cols / chunk_cols)
   int corr_col0;                     // first tensor-memory column of correction slot 0 (slot s follows at + s * chunk_cols)
   int groups;                        // epilogue groups (1 .. kLrMaxGroups), each with two correction slots of chunk_cols columns
-  int stages, stage_bytes;
+  int base_stages, base_stage_bytes, corr_stages, corr_stage_bytes;
   const int* targets;                // [T, n]
   float* G;                          // [T, n, r]
+  float2* partial;                   // panels > 1: [panels, T n r] (running maximum, sum of exponentials) of each panel
+  float* target_logit;               // panels > 1: [T n r] logit of the target, written by the panel that holds it
   unsigned* status;
   uint64_t wait_limit_ns;
+};
+
+struct LowRankControl {
+  GemmControl g;                     // full / empty: base ring; tfull / tempty: correction slots; abort, limits, tmem_base
+  uint64_t cfull[kLrCorrStages];     // correction operand ring
+  uint64_t cempty[kLrCorrStages];
+  uint64_t afull[2];                 // base accumulators
+  uint64_t aempty[2];
+  uint64_t drain2;
 };
 
 // K-major operand tile whose rows are `row_bytes` (32, 64 or 128) wide and swizzled with that span: 8-row groups are
@@ -60,34 +78,72 @@ __device__ __forceinline__ uint64_t umma_smem_desc_kmajor(uint32_t smem_addr, ui
   return d;
 }
 
-__global__ void __launch_bounds__(64 + 128 * kLrMaxGroups, 1) mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
+// Wait (bounded) until the copies a producer still has in flight have landed: no copy may be in flight when the CTA goes.
+__device__ __forceinline__ void lowrank_drain_ring(uint64_t* full, int stages, uint32_t issued_mask, uint32_t phase_mask) {
+  for (int s = 0; s < stages; ++s)
+    if (issued_mask & (1u << s)) {
+      const uint32_t bar = smem_u32(&full[s]);
+      const uint32_t par = (phase_mask >> s) & 1u;
+      const uint64_t t0 = global_timer_ns();
+      while (!mbar_try_wait(bar, par) && global_timer_ns() - t0 < kWaitLimitNs) {}
+    }
+}
+
+struct LowRankItem {
+  int mt, slot, panel;
+  int width;     // columns of this panel (the last panel of a unit may be narrower), a multiple of 16
+  int nchunk;    // correction chunks that cover them
+};
+// panel fastest, then slot: the CTAs that run together share the hidden tile (and the slot's W_i) through L2
+__device__ __forceinline__ LowRankItem lowrank_item(const LowRankGemmParams& p, int item) {
+  LowRankItem c;
+  c.panel = item % p.panels;
+  const int rest = item / p.panels;
+  c.slot = rest % p.n;
+  c.mt = rest / p.n;
+  c.width = min(p.panel_cols, p.v - c.panel * p.panel_cols);
+  c.nchunk = (c.width + p.chunk_cols - 1) / p.chunk_cols;
+  return c;
+}
+
+__global__ void __launch_bounds__(kLrRoleThreads + 128 * kLrMaxGroups, 1)
+mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
-  const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
-  uint8_t* tiles = smem_raw + (tiles_addr - raw_addr);
-  GemmControl* ctl = reinterpret_cast<GemmControl*>(tiles + static_cast<size_t>(p.stages) * p.stage_bytes);
+  const uint32_t base_ring = (raw_addr + 1023u) & ~1023u;
+  const uint32_t corr_ring = base_ring + static_cast<uint32_t>(p.base_stages * p.base_stage_bytes);
+  uint8_t* tiles = smem_raw + (base_ring - raw_addr);
+  LowRankControl* lc = reinterpret_cast<LowRankControl*>(tiles + static_cast<size_t>(p.base_stages) * p.base_stage_bytes +
+                                                         static_cast<size_t>(p.corr_stages) * p.corr_stage_bytes);
+  GemmControl* ctl = &lc->g;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int num_items = p.m_tiles * p.n;                 // slot fastest: the CTAs running together share the hidden tiles
-  const int kq = p.k / 16;                                // K = 16 steps of one correction
+  const int num_items = p.m_tiles * p.n * p.panels;
+  const int kq = p.k / 16;                                // K = 16 steps of one half of a correction
   const uint32_t zbox = kBlockM * 32;                     // bytes of one z box (128 rows x 32 bytes)
   const uint32_t abox = static_cast<uint32_t>(p.chunk_cols) * 32;
   const uint32_t a_off = 2 * kq * zbox;                   // correction entry: [z_hi boxes | z_lo boxes | A boxes (q, c)]
-  const uint32_t base_b_off = kABytes;                    // base entry: [h tile | W_i boxes]
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) {
+    for (int s = 0; s < p.base_stages; ++s) {
       mbar_init(smem_u32(&ctl->full[s]), 1);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
+    }
+    for (int s = 0; s < p.corr_stages; ++s) {
+      mbar_init(smem_u32(&lc->cfull[s]), 1);
+      mbar_init(smem_u32(&lc->cempty[s]), 1);
     }
     for (int s = 0; s < 2 * p.groups; ++s) {
       mbar_init(smem_u32(&ctl->tfull[s]), 1);
       mbar_init(smem_u32(&ctl->tempty[s]), 4);
     }
-    mbar_init(smem_u32(&ctl->tfull[kLrBaseSlot]), 1);
-    mbar_init(smem_u32(&ctl->tempty[kLrBaseSlot]), 4 * p.groups);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&lc->afull[s]), 1);
+      mbar_init(smem_u32(&lc->aempty[s]), 4 * p.groups);
+    }
     mbar_init(smem_u32(&ctl->drain), 1);
+    mbar_init(smem_u32(&lc->drain2), 1);
     ctl->abort = 0;
     ctl->wait_limit_ns = p.wait_limit_ns;
     fence_mbar_init();
@@ -106,99 +162,117 @@ __global__ void __launch_bounds__(64 + 128 * kLrMaxGroups, 1) mtpc_lowrank_gemm_
   const uint32_t tmem_base = ctl->tmem_base;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer, base operands
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
       bool ok = true;
-      const uint32_t base_bytes = kABytes + static_cast<uint32_t>(p.base_boxes * p.base_box_rows) * (kBlockK * 2);
-      const uint32_t corr_bytes = 2 * kq * zbox + static_cast<uint32_t>(kq * p.nchunk) * abox;
-      auto advance = [&]() {
-        issued_mask |= 1u << stage;
-        phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
-        if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; }
-      };
+      const uint32_t bytes = kABytes + static_cast<uint32_t>(p.panel_cols) * (kBlockK * 2);
       for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
-        const int mt = item / p.n, slot_i = item - mt * p.n;
-        for (int kb = 0; kb < p.kblocks && ok; ++kb) {
+        const LowRankItem w = lowrank_item(p, item);
+        for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
           const uint32_t full = smem_u32(&ctl->full[stage]);
-          const uint32_t dst = tiles_addr + stage * p.stage_bytes;
-          mbar_arrive_expect_tx(full, base_bytes);
-          tma_load_2d(dst, &p.tm_h, full, kb * kBlockK, mt * kBlockM);
-          for (int q = 0; q < p.base_boxes; ++q)
-            tma_load_2d(dst + base_b_off + q * p.base_box_rows * (kBlockK * 2), &p.tm_w, full, kb * kBlockK,
-                        slot_i * p.v + q * p.base_box_rows);
-          advance();
-        }
-        for (int j = 0; j < p.r && ok; ++j) {
-          if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
-          const uint32_t full = smem_u32(&ctl->full[stage]);
-          const uint32_t dst = tiles_addr + stage * p.stage_bytes;
-          const int unit = slot_i * p.r + j;
-          mbar_arrive_expect_tx(full, corr_bytes);
-          for (int part = 0; part < 2; ++part)
-            for (int q = 0; q < kq; ++q)
-              tma_load_2d(dst + (part * kq + q) * zbox, &p.tm_z, full, (2 * unit + part) * p.k + 16 * q, mt * kBlockM);
-          for (int q = 0; q < kq; ++q)
-            for (int c = 0; c < p.nchunk; ++c)
-              tma_load_2d(dst + a_off + (q * p.nchunk + c) * abox, &p.tm_a, full, 16 * q, unit * p.v + c * p.chunk_cols);
-          advance();
+          const uint32_t dst = base_ring + stage * p.base_stage_bytes;
+          mbar_arrive_expect_tx(full, bytes);
+          tma_load_2d(dst, &p.tm_h, full, kb * kBlockK, w.mt * kBlockM);
+          // the box is panel_cols rows high also for a narrower last panel: the rows past it (the next slot's, or
+          // zeros past the end of W_base) are not multiplied
+          tma_load_2d(dst + kABytes, &p.tm_w, full, kb * kBlockK, w.slot * p.v + w.panel * p.panel_cols);
+          issued_mask |= 1u << stage;
+          phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
+          if (++stage == static_cast<uint32_t>(p.base_stages)) { stage = 0; phase ^= 1u; }
         }
       }
-      // no copy may still be in flight when the CTA goes away
-      for (int s = 0; s < p.stages; ++s)
-        if (issued_mask & (1u << s)) {
-          const uint32_t bar = smem_u32(&ctl->full[s]);
-          const uint32_t par = (phase_mask >> s) & 1u;
-          const uint64_t t0 = global_timer_ns();
-          while (!mbar_try_wait(bar, par) && global_timer_ns() - t0 < kWaitLimitNs) {}
-        }
+      lowrank_drain_ring(ctl->full, p.base_stages, issued_mask, phase_mask);
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ MMA issuer, base: item `it` into buffer it & 1
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, it = 0;
-      uint32_t cuse[kLrMaxGroups] = {0, 0, 0};                      // chunks issued so far for each epilogue group
       bool ok = true;
-      const int base_n = p.base_box_rows;                           // columns per base MMA (v, or v / 2)
-      const uint32_t idesc_base = umma_idesc_bf16(kBlockM, base_n);
-      auto next_stage = [&]() { if (++stage == static_cast<uint32_t>(p.stages)) { stage = 0; phase ^= 1u; } };
       for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++it) {
-        // ---- base: all K blocks into columns [0, v)
-        if (!bounded_wait(smem_u32(&ctl->tempty[kLrBaseSlot]), (it & 1u) ^ 1u, ctl, p.status)) { ok = false; break; }
+        const uint32_t idesc = umma_idesc_bf16(kBlockM, lowrank_item(p, item).width);
+        const uint32_t buf = it & 1u;
+        if (!bounded_wait(smem_u32(&lc->aempty[buf]), ((it >> 1) & 1u) ^ 1u, ctl, p.status)) { ok = false; break; }
         tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * p.acc_stride;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t addr = tiles_addr + stage * p.stage_bytes;
+          const uint32_t addr = base_ring + stage * p.base_stage_bytes;
           const uint64_t a_desc = umma_smem_desc_sw128(addr);
-          for (int q = 0; q < p.base_boxes; ++q) {
-            const uint64_t b_desc = umma_smem_desc_sw128(addr + base_b_off + q * base_n * (kBlockK * 2));
+          const uint64_t b_desc = umma_smem_desc_sw128(addr + kABytes);
 #pragma unroll
-            for (int kk = 0; kk < kBlockK / 16; ++kk)
-              umma_bf16(tmem_base + q * base_n, a_desc + 2 * kk, b_desc + 2 * kk, idesc_base, (kb | kk) != 0 ? 1u : 0u);
-          }
+          for (int kk = 0; kk < kBlockK / 16; ++kk)
+            umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
           umma_commit(smem_u32(&ctl->empty[stage]));
-          next_stage();
+          if (++stage == static_cast<uint32_t>(p.base_stages)) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(smem_u32(&ctl->tfull[kLrBaseSlot]));
-        // ---- corrections, `groups` components at a time (component j0 + g belongs to epilogue group g): their chunks
-        // are issued in turn, chunk c of component j0 + g into slot 2 g + (that group's chunk count & 1)
+        umma_commit(smem_u32(&lc->afull[buf]));
+      }
+      if (!ok || ctl->abort) {   // wait (bounded) for the MMAs already issued before tensor memory is freed
+        umma_commit(smem_u32(&ctl->drain));
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+    __syncwarp();
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ TMA producer, correction operands
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
+      bool ok = true;
+      const uint32_t bytes = 2 * kq * zbox + static_cast<uint32_t>(kq * p.nchunk) * abox;
+      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+        const LowRankItem w = lowrank_item(p, item);
+        for (int j = 0; j < p.r; ++j) {
+          if (!bounded_wait(smem_u32(&lc->cempty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
+          const uint32_t full = smem_u32(&lc->cfull[stage]);
+          const uint32_t dst = corr_ring + stage * p.corr_stage_bytes;
+          const int unit = w.slot * p.r + j;
+          mbar_arrive_expect_tx(full, bytes);
+          for (int part = 0; part < 2; ++part)
+            for (int q = 0; q < kq; ++q)
+              tma_load_2d(dst + (part * kq + q) * zbox, &p.tm_z, full, (2 * unit + part) * p.k + 16 * q, w.mt * kBlockM);
+          // all nchunk boxes of a full panel are fetched; boxes may run past the panel (into the next panel, unit, or
+          // the end of A: zero-filled): the MMAs cover only the panel's own columns
+          for (int q = 0; q < kq; ++q)
+            for (int c = 0; c < p.nchunk; ++c)
+              tma_load_2d(dst + a_off + (q * p.nchunk + c) * abox, &p.tm_a, full, 16 * q,
+                          unit * p.v + w.panel * p.panel_cols + c * p.chunk_cols);
+          issued_mask |= 1u << stage;
+          phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
+          if (++stage == static_cast<uint32_t>(p.corr_stages)) { stage = 0; phase ^= 1u; }
+        }
+      }
+      lowrank_drain_ring(lc->cfull, p.corr_stages, issued_mask, phase_mask);
+    }
+    __syncwarp();
+  } else if (warp == 3) {
+    // ------------------------------------------------------------------ MMA issuer, corrections: `groups` components
+    // at a time (component j0 + g belongs to epilogue group g); their chunks are issued in turn, chunk c of component
+    // j0 + g into slot 2 g + (that group's chunk count & 1)
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      uint32_t cuse[kLrMaxGroups] = {0, 0, 0};
+      bool ok = true;
+      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
+        const LowRankItem w = lowrank_item(p, item);
         for (int j0 = 0; j0 < p.r && ok; j0 += p.groups) {
           const int ng = min(p.groups, p.r - j0);
           uint32_t addr[kLrMaxGroups], estage[kLrMaxGroups];
           for (int g = 0; g < ng && ok; ++g) {
-            if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
-            addr[g] = tiles_addr + stage * p.stage_bytes;
+            if (!bounded_wait(smem_u32(&lc->cfull[stage]), phase, ctl, p.status)) { ok = false; break; }
+            addr[g] = corr_ring + stage * p.corr_stage_bytes;
             estage[g] = stage;
-            next_stage();
+            if (++stage == static_cast<uint32_t>(p.corr_stages)) { stage = 0; phase ^= 1u; }
           }
           if (!ok) break;
           tc_fence_after();
-          for (int c = 0; c < p.nchunk && ok; ++c) {
-            const int width = min(p.chunk_cols, p.v - c * p.chunk_cols);
+          for (int c = 0; c < w.nchunk && ok; ++c) {
+            const int width = min(p.chunk_cols, w.width - c * p.chunk_cols);
             const uint32_t idesc = umma_idesc_bf16(kBlockM, width);
             for (int g = 0; g < ng; ++g) {
               const uint32_t slot = 2 * g + (cuse[g] & 1u);
@@ -217,45 +291,49 @@ __global__ void __launch_bounds__(64 + 128 * kLrMaxGroups, 1) mtpc_lowrank_gemm_
             }
           }
           if (!ok) break;
-          for (int g = 0; g < ng; ++g) umma_commit(smem_u32(&ctl->empty[estage[g]]));
+          for (int g = 0; g < ng; ++g) umma_commit(smem_u32(&lc->cempty[estage[g]]));
         }
       }
-      if (!ok) {   // wait (bounded) for the MMAs already issued before tensor memory is freed
-        umma_commit(smem_u32(&ctl->drain));
+      if (!ok || ctl->abort) {
+        umma_commit(smem_u32(&lc->drain2));
         const uint64_t t0 = global_timer_ns();
-        while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(smem_u32(&lc->drain2), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
       }
     }
     __syncwarp();
   } else {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;
-    const int group = (warp - 2) >> 2;                        // this warp's epilogue group: components group, group + groups, ...
+    const int group = (warp - kLrRoleThreads / 32) >> 2;      // this warp's epilogue group: components group, group + groups, ...
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    const size_t entries = static_cast<size_t>(p.T) * p.n * p.r;
     uint32_t it = 0, cuse = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++it) {
-      const int mt = item / p.n, slot_i = item - mt * p.n;
-      const int row = mt * kBlockM + quarter * 32 + lane;
+      const LowRankItem w = lowrank_item(p, item);
+      const int row = w.mt * kBlockM + quarter * 32 + lane;
       const bool valid = row < p.T;
-      const int tgt = valid ? p.targets[static_cast<size_t>(row) * p.n + slot_i] : -1;
-      if (!bounded_wait_warp(smem_u32(&ctl->tfull[kLrBaseSlot]), it & 1u, ctl, p.status, lane)) { ok = false; break; }
+      const int tgt = valid ? p.targets[static_cast<size_t>(row) * p.n + w.slot] : -1;
+      const int panel_col0 = w.panel * p.panel_cols;
+      const uint32_t buf = it & 1u;
+      if (!bounded_wait_warp(smem_u32(&lc->afull[buf]), (it >> 1) & 1u, ctl, p.status, lane)) { ok = false; break; }
       tc_fence_after();
+      const uint32_t bcol = lane_base + buf * p.acc_stride;
       for (int j = group; j < p.r && ok; j += p.groups) {
         float m = -CUDART_INF_F, s = 0.f, tval = 0.f;
-        for (int c = 0; c < p.nchunk; ++c, ++cuse) {
+        for (int c = 0; c < w.nchunk; ++c, ++cuse) {
           const uint32_t slot = 2 * group + (cuse & 1u);
           if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (cuse >> 1) & 1u, ctl, p.status, lane)) { ok = false; break; }
           tc_fence_after();
-          const int col_chunk = c * p.chunk_cols;
-          const int width = min(p.chunk_cols, p.v - col_chunk);
+          const int col_chunk = c * p.chunk_cols;             // first column of the chunk inside the panel
+          const int width = min(p.chunk_cols, w.width - col_chunk);
           const uint32_t ccol = lane_base + p.corr_col0 + slot * p.chunk_cols;
           // one batch of 16 columns: correction + base, then the dense kernel's online log-sum-exp and target gather
           auto consume = [&](const uint32_t (&rc)[16], const uint32_t (&rb)[16], int b) {
             float x[16];
 #pragma unroll
             for (int q = 0; q < 16; ++q) x[q] = __uint_as_float(rc[q]) + __uint_as_float(rb[q]);
-            const int col0 = col_chunk + b * 16;
+            const int col0 = panel_col0 + col_chunk + b * 16; // column inside the unit
             mask_padding(x, col0, p.vv);
             // short dependent chains: reduce as trees
             float t8[8];
@@ -283,13 +361,13 @@ __global__ void __launch_bounds__(64 + 128 * kLrMaxGroups, 1) mtpc_lowrank_gemm_
           const int nb = width / 16;
           uint32_t c0[16], b0[16], c1[16], b1[16];
           tmem_ld16_issue(ccol, c0);
-          tmem_ld16_issue(lane_base + col_chunk, b0);
+          tmem_ld16_issue(bcol + col_chunk, b0);
           tmem_ld_wait16(c0);
           tmem_ld_wait16(b0);
           for (int b = 0; b < nb; b += 2) {
             if (b + 1 < nb) {
               tmem_ld16_issue(ccol + (b + 1) * 16, c1);
-              tmem_ld16_issue(lane_base + col_chunk + (b + 1) * 16, b1);
+              tmem_ld16_issue(bcol + col_chunk + (b + 1) * 16, b1);
             }
             consume(c0, b0, b);
             if (b + 1 >= nb) break;
@@ -297,7 +375,7 @@ __global__ void __launch_bounds__(64 + 128 * kLrMaxGroups, 1) mtpc_lowrank_gemm_
             tmem_ld_wait16(b1);
             if (b + 2 < nb) {
               tmem_ld16_issue(ccol + (b + 2) * 16, c0);
-              tmem_ld16_issue(lane_base + col_chunk + (b + 2) * 16, b0);
+              tmem_ld16_issue(bcol + col_chunk + (b + 2) * 16, b0);
             }
             consume(c1, b1, b + 1);
             if (b + 2 < nb) {
@@ -311,21 +389,27 @@ __global__ void __launch_bounds__(64 + 128 * kLrMaxGroups, 1) mtpc_lowrank_gemm_
         }
         if (!ok) break;
         if (valid) {
-          float* g = p.G + (static_cast<size_t>(row) * p.n + slot_i) * p.r + j;
-          if (tgt < 0) {
-            *g = 0.f;                                  // marginalised byte: the input unit sums to 1
-          } else if (tgt >= p.vv) {
-            *g = CUDART_NAN_F;
-            atomicOr(p.status, kStatusBadTarget);
+          const size_t e = (static_cast<size_t>(row) * p.n + w.slot) * p.r + j;
+          if (p.panels == 1) {
+            if (tgt < 0) {
+              p.G[e] = 0.f;                                  // marginalised byte: the input unit sums to 1
+            } else if (tgt >= p.vv) {
+              p.G[e] = CUDART_NAN_F;
+              atomicOr(p.status, kStatusBadTarget);
+            } else {
+              p.G[e] = tval - (m + fast_lg2(s) * kLn2);
+            }
           } else {
-            *g = tval - (m + fast_lg2(s) * kLn2);
+            // (padding is less than 16 columns and a panel at least 16 wide: every panel has existing symbols)
+            p.partial[static_cast<size_t>(w.panel) * entries + e] = make_float2(m, s);
+            if (static_cast<unsigned>(tgt - panel_col0) < static_cast<unsigned>(w.width)) p.target_logit[e] = tval;
           }
         }
       }
       if (!ok) break;
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctl->tempty[kLrBaseSlot]));   // the next item's base may overwrite the columns
+      if (lane == 0) mbar_arrive(smem_u32(&lc->aempty[buf]));   // the base of the item after next may overwrite the buffer
     }
   }
 
@@ -335,6 +419,28 @@ __global__ void __launch_bounds__(64 + 128 * kLrMaxGroups, 1) mtpc_lowrank_gemm_
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
+}
+
+// G[t, i, j] = logit[target] - LSE over the unit, from the per-panel (maximum, sum of exponentials) the factored projection
+// left: one thread per (position, slot, component). Targets < 0 (marginalised): 0; targets >= vv: NaN and the status bit.
+__global__ void lowrank_merge_kernel(const float2* __restrict__ partial, const float* __restrict__ target_logit,
+                                     const int* __restrict__ targets, float* __restrict__ G, unsigned* status,
+                                     size_t entries, int r, int vv, int panels) {
+  const size_t e = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (e >= entries) return;
+  const int tgt = targets[e / r];
+  if (tgt < 0) { G[e] = 0.f; return; }
+  if (tgt >= vv) {
+    G[e] = CUDART_NAN_F;
+    atomicOr(status, kStatusBadTarget);
+    return;
+  }
+  float m = -CUDART_INF_F, s = 0.f;
+  for (int q = 0; q < panels; ++q) {
+    const float2 ms = partial[static_cast<size_t>(q) * entries + e];
+    lse_merge(m, s, ms.x, ms.y);
+  }
+  G[e] = target_logit[e] - (m + __logf(s));
 }
 
 }  // namespace mtpc

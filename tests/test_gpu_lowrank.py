@@ -143,7 +143,10 @@ FACTORED = [
     (I.BTREE, 4, 4, 48, 44, 64, 16, 70),       # padded vocabulary, tree circuit
     (I.HMM_CTX, 3, 8, 320, 0, 128, 16, 200),   # contextual transitions: many sum tiles beside the factored projection
     (I.CP, 1, 1, 16, 0, 64, 16, 5),            # the smallest everything
-    (I.CP, 2, 4, 480, 0, 64, 16, 140),         # the widest unit that leaves room for corrections: two 16-column slots
+    (I.CP, 2, 4, 480, 0, 64, 16, 140),         # three panels of 160 columns
+    (I.HMM, 2, 4, 320, 306, 64, 16, 100),      # padded vocabulary, two panels, static transitions
+    (I.CP, 1, 2, 1024, 1010, 64, 16, 40),      # eight panels of 128 columns
+    (I.CP, 2, 4, 272, 268, 64, 16, 90),        # panels of 144 and 128 columns
 ]
 
 
@@ -215,5 +218,33 @@ def test_factored_head_agrees_with_the_dense_head_on_the_composed_tensor_and_ref
     need = ctypes.c_size_t(0)
     assert B.lib().mtpc_lowrank_workspace_bytes(ctypes.byref(cfg), 8, ctypes.byref(need)) == -3      # rank not 16 or 32
     assert B.lib().mtpc_lowrank_workspace_bytes(ctypes.byref(cfg), 16, ctypes.byref(need)) == 0 and need.value > 0
-    big = B.MtpcConfig(family, n, r, 512, d, B.MTPC_BF16, T, 1, 0, 0)                                 # no room for the corrections
-    assert B.lib().mtpc_lowrank_workspace_bytes(ctypes.byref(big), 16, ctypes.byref(need)) == -3
+    for bad_v in (40, 9616):        # 40: not a multiple of 16; 9616: more than eight panels
+        big = B.MtpcConfig(family, n, r, bad_v, d, B.MTPC_BF16, T, 1, 0, 0)
+        assert B.lib().mtpc_lowrank_workspace_bytes(ctypes.byref(big), 16, ctypes.byref(need)) == -3, bad_v
+
+
+def test_a_wait_that_runs_out_in_the_factored_kernel_is_reported_and_the_head_recovers():
+    """Both pipelines of the factored projection (base and corrections, each with its own producer and MMA issuer) give up
+    at their first wait under a 50 ns limit: the status must say so, the context must stay usable, and the next call
+    with the default limit must be right again."""
+    family, n, r, v, d, k, T = I.CP, 3, 8, 320, 4096, 16, 400      # d = 4096: the first copies take longer than 64 polls
+    wl, W, A, Bm = _factored_case(family, n, r, v, 0, d, k, T, seed=4500)
+    head = B.MtpcHead(family, n, r, v, d, B.MTPC_BF16, T, 1, None, to_device_bf16(wl.W_sum_q), None,
+                      lowrank=(_device(W), _device(A), _device(Bm)))
+    hidden = to_device_bf16(wl.hidden_q)
+    targets = torch.from_numpy(wl.targets).cuda()
+    out = torch.empty(T, device="cuda")
+    ref = O.window_logprob(family, wl.hidden_q, O.lowrank_unembedding(W, A, Bm), wl.W_sum_q, None, wl.targets)
+    head.mtpc_window_logprob(hidden, targets, out)
+    assert head.mtpc_get_status(with_code=True) == (B.MTPC_OK, 0)
+    assert np.abs(out.cpu().numpy() - ref).max() <= 2e-3
+    head.mtpc_debug_set_wait_limit_ns(50)
+    head.mtpc_window_logprob(hidden, targets, out)            # gives up; outputs unspecified
+    torch.cuda.synchronize()
+    code, bits = head.mtpc_get_status(with_code=True)
+    assert code == B.ERR_TIMEOUT and bits & B.STATUS_TIMEOUT
+    head.mtpc_debug_set_wait_limit_ns(0)
+    head.mtpc_window_logprob(hidden, targets, out)
+    assert head.mtpc_get_status(with_code=True) == (B.MTPC_OK, 0)
+    assert np.abs(out.cpu().numpy() - ref).max() <= 2e-3
+    head.mtpc_destroy()
