@@ -242,21 +242,6 @@ int make_tmap(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, u
   return r == CUDA_SUCCESS ? MTPC_OK : MTPC_ERR_CUDA;
 }
 
-// bf16 matrix [rows, cols] row-major -> tiles of box_rows x 16 elements (32-byte rows), 32-byte swizzle, zero fill outside.
-int make_tmap_sw32(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return MTPC_ERR_CUDA;
-  if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0 || (cols * 2) % 16 != 0) return MTPC_ERR_WORKSPACE;
-  cuuint64_t gdim[2] = {cols, rows};
-  cuuint64_t gstride[1] = {cols * 2};
-  cuuint32_t box[2] = {16, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? MTPC_OK : MTPC_ERR_CUDA;
-}
-
 // bf16 matrix [rows, cols] row-major read as an MN-major operand (its columns are the operand's M or N index, its rows
 // the K index): boxes of 64 columns x 64 rows, 128-byte swizzle, zero fill outside.
 int make_tmap_mn(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch) {
@@ -290,6 +275,7 @@ struct mtpc_head {
   const void* lr_W_base;                        // [n, v, d] bf16
   const void* lr_A;                             // [n, r, v, k] bf16
   const void* lr_B;                             // [n, r, k, d] bf16
+  size_t lr_off_arep;                           // workspace: A as [n, v, r, k]
   size_t lr_off_zhl, lr_off_partial;            // workspace: z = B h as bf16 halves [T, n r, 2, k]; per-panel partial log-sum-exps
   LowRankGemmParams lr_params;                  // everything of the factored projection launch that does not depend on the call
   int max_pairs;                                // clusters of two projection CTAs that can be resident at once
@@ -921,16 +907,15 @@ bool plan_lowrank(const mtpc_config& c, int k, LowRankGemmParams* p) {
   p->chunk_cols = chunk;
   p->nchunk = (pc + chunk - 1) / chunk;
   p->corr_col0 = 2 * stride;
-  const int kq = k / 16;
   p->base_stage_bytes = kABytes + pc * kBlockK * 2;                                  // a multiple of 1024 (pc % 16 == 0)
-  p->corr_stage_bytes = (2 * kq * kBlockM * 32 + kq * p->nchunk * chunk * 32 + 1023) / 1024 * 1024;
+  p->corr_stage_bytes = 2 * kBlockM * 128 + p->nchunk * chunk * 128;                 // two z boxes and the A' boxes of 64 / k components
   const int ctl = 1024 + static_cast<int>(sizeof(LowRankControl));
-  // the operands of `groups` components are resident together and the next ones on their way; the base ring takes the rest
-  for (int cs = kLrCorrStages; cs >= groups + 1; --cs) {
+  // at least two correction entries (one in use, the next on its way); the base ring takes the rest, at least two K blocks
+  for (int cs = kLrCorrStages; cs >= 2; --cs) {
     const int left = kSmemLimit - ctl - cs * p->corr_stage_bytes;
     int bs = left / p->base_stage_bytes;
     if (bs > kMaxStages) bs = kMaxStages;
-    if (bs >= 3 || (bs == 2 && cs == groups + 1)) {
+    if (bs >= 3 || (bs == 2 && cs == 2)) {
       p->corr_stages = cs;
       p->base_stages = bs;
       return true;
@@ -955,8 +940,14 @@ int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, cons
   if (rc != MTPC_OK) return rc;
   LowRankGemmParams p = h->lr_params;
   rc = make_tmap(&p.tm_h, hidden_bf16, static_cast<uint64_t>(T), static_cast<uint64_t>(c.d), kBlockM);
-  if (rc == MTPC_OK) rc = make_tmap_sw32(&p.tm_z, zhl, static_cast<uint64_t>(T), static_cast<uint64_t>(units) * 2 * k, kBlockM);
+  if (rc == MTPC_OK) rc = make_tmap(&p.tm_z, zhl, static_cast<uint64_t>(T), static_cast<uint64_t>(units) * 2 * k, kBlockM);
   if (rc != MTPC_OK) return rc;
+  {   // A as [n, v, r, k]: the adaptor columns of adjacent components side by side (remade every call: A may have changed)
+    const size_t pieces = static_cast<size_t>(units) * c.v * (k / 8);
+    lowrank_repack_kernel<<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, st>>>(
+        static_cast<const uint4*>(h->lr_A), reinterpret_cast<uint4*>(h->ws + h->lr_off_arep), c.n, c.r, c.v, k / 8);
+    h->launches += 1;
+  }
   p.T = T;
   p.m_tiles = (T + kBlockM - 1) / kBlockM;
   p.targets = targets;
@@ -1171,15 +1162,18 @@ struct LowRankSpec {
 };
 
 // Workspace of a factored head beyond the dense layout: z = B h as two bf16 halves [T, n r, 2, k] (written by the GEMM
-// that computes it), and, where a unit is cut into panels, the panels' (maximum, sum) pairs and the targets' logits.
+// that computes it), where a unit is cut into panels the panels' (maximum, sum) pairs and the targets' logits, and the
+// copy of A the factored kernel reads.
 static int lowrank_extra_bytes(const mtpc_config& c, int k, int panels, size_t base_total, size_t* off_zhl,
-                               size_t* off_partial, size_t* total) {
+                               size_t* off_partial, size_t* off_arep, size_t* total) {
   const size_t units = static_cast<size_t>(c.n) * c.r;
   size_t off = align_up(base_total);
   *off_zhl = off;
   off += align_up(static_cast<size_t>(c.max_positions) * units * 2 * k * 2);
   *off_partial = off;
   if (panels > 1) off += align_up(static_cast<size_t>(c.max_positions) * units * (panels * sizeof(float2) + sizeof(float)));
+  *off_arep = off;                      // the copy of A laid out [n, v, r, k]
+  off += align_up(units * c.v * k * 2);
   *total = off;
   return MTPC_OK;
 }
@@ -1195,11 +1189,11 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
   if (rc != MTPC_OK) return rc;
   LowRankGemmParams lrp;
   memset(&lrp, 0, sizeof(lrp));
-  size_t lr_zhl = 0, lr_partial = 0;
+  size_t lr_zhl = 0, lr_partial = 0, lr_arep = 0;
   if (lowrank) {
     if (cfg->io_dtype != MTPC_BF16) return MTPC_ERR_UNSUPPORTED;
     if (!plan_lowrank(*cfg, lowrank->k, &lrp)) return MTPC_ERR_UNSUPPORTED;
-    lowrank_extra_bytes(*cfg, lowrank->k, lrp.panels, L.total, &lr_zhl, &lr_partial, &L.total);
+    lowrank_extra_bytes(*cfg, lowrank->k, lrp.panels, L.total, &lr_zhl, &lr_partial, &lr_arep, &L.total);
   }
   const bool ctx = (cfg->flags & MTPC_FLAG_HMM_CONTEXTUAL) != 0;
   if (cfg->family == MTPC_HMM && cfg->n > 1 && !ctx && !T_static) return MTPC_ERR_NULL;
@@ -1222,6 +1216,7 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
     h->lr_B = lowrank->B;
     h->lr_off_zhl = lr_zhl;
     h->lr_off_partial = lr_partial;
+    h->lr_off_arep = lr_arep;
     h->lr_params = lrp;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1257,8 +1252,8 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
               : make_tmap(&h->lr_params.tm_w, lowrank->W_base, static_cast<uint64_t>(cfg->n) * cfg->v, cfg->d,
                           h->lr_params.panel_cols);
     if (rc == MTPC_OK)
-      rc = make_tmap_sw32(&h->lr_params.tm_a, lowrank->A, static_cast<uint64_t>(cfg->n) * cfg->r * cfg->v, lowrank->k,
-                          h->lr_params.chunk_cols);
+      rc = make_tmap(&h->lr_params.tm_a, h->ws + h->lr_off_arep, static_cast<uint64_t>(cfg->n) * cfg->v,
+                     static_cast<uint64_t>(cfg->r) * lowrank->k, h->lr_params.chunk_cols);
   }
   if (rc != MTPC_OK) { delete h; return rc; }
   *out = h;
@@ -1278,8 +1273,8 @@ int mtpc_lowrank_workspace_bytes(const mtpc_config* cfg, int32_t k, size_t* out_
   if (rc != MTPC_OK) return rc;
   LowRankGemmParams lrp;
   if (cfg->io_dtype != MTPC_BF16 || !plan_lowrank(*cfg, k, &lrp)) return MTPC_ERR_UNSUPPORTED;
-  size_t a = 0, b = 0;
-  return lowrank_extra_bytes(*cfg, k, lrp.panels, L.total, &a, &b, out_bytes);
+  size_t a = 0, b = 0, c3 = 0;
+  return lowrank_extra_bytes(*cfg, k, lrp.panels, L.total, &a, &b, &c3, out_bytes);
 }
 
 int mtpc_create_head_lowrank(const mtpc_config* cfg, int32_t k, const void* W_base, const void* A, const void* B,

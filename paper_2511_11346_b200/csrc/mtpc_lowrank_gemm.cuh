@@ -15,11 +15,16 @@
 //             lowrank_merge_kernel combines them - so the items are independent and deal out evenly.
 // FLOPs per position: 2 d (n v + n r k) + 4 n r v k instead of 2 d n r v.
 // Roles: warp 0 TMA producer of the base operands, warp 1 MMA issuer of the base, warp 2 TMA producer of the correction
-// operands, warp 3 MMA issuer of the corrections, then `groups` epilogue groups of four warps (one thread per position):
-// group g takes the components j = g, g + groups, ... The two pipelines share nothing but the tensor cores: each has its
-// own shared-memory ring (base: a 64-wide K block of h and of the panel's rows of W_i, 128-byte swizzle; corrections: z_hi,
-// z_lo as k/16 boxes of 128 rows x 16 and A_ij as k/16 x nchunk boxes of chunk_cols rows x 16, 32-byte rows with the
-// 32-byte swizzle, so every correction MMA (K = 16) starts at the base of its own box) and its own barriers.
+// operands, warps 3 .. 2 + groups one MMA issuer of corrections per epilogue group (issuing one of these small MMAs holds
+// its thread for a few hundred cycles although the tensor pipe is nearly idle: the issuers must not queue behind each
+// other), then from warp 8 on `groups` epilogue groups of four warps (one thread per position): group g takes the
+// components j = g, g + groups, ... The two pipelines share nothing but the tensor cores: each has its
+// own shared-memory ring and its own barriers. Base ring: a 64-wide K block of h and of the panel's rows of W_i. Correction
+// ring: one entry holds the operands of 64 / k components, all as 128-byte rows with the 128-byte swizzle (the tensor cores
+// read 32-byte-row tiles several times slower): z as boxes of 128 positions x 64 values = [hi | lo] of 32 / k adjacent
+// components, and A as boxes of chunk_cols vocabulary rows x 64 values = the k adaptor columns of 64 / k adjacent components,
+// read from a copy of A laid out [n, v, r, k] (lowrank_repack_kernel, made on every call: A is small and may have changed).
+// A correction MMA (K = 16) addresses its operands inside those rows, 32 bytes apart, like the K steps of the base.
 #pragma once
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -30,16 +35,16 @@
 namespace mtpc {
 
 constexpr int kLrMaxRank = 32;          // k <= 32 (a multiple of 16)
-constexpr int kLrMaxGroups = 3;         // epilogue groups: 128 + 128 * groups threads per CTA
+constexpr int kLrMaxGroups = 2;         // epilogue groups: 256 + 128 * groups threads per CTA (512: 128 registers each)
 constexpr int kLrMaxPanels = 8;
 constexpr int kLrCorrStages = 4;        // entries of the correction operand ring (at most)
-constexpr int kLrRoleThreads = 128;     // the four single-thread roles, one warp each
+constexpr int kLrRoleThreads = 256;     // the single-thread roles, one warp each: warps 0 .. 2 + groups (the rest idle)
 
 struct LowRankGemmParams {
   CUtensorMap tm_h;      // hidden [T, d]              box 64 x 128, 128-byte swizzle
   CUtensorMap tm_w;      // W_base [n*v, d]            box 64 x panel_cols, 128-byte swizzle
-  CUtensorMap tm_z;      // z      [T, n*r*2*k]        box 16 x 128, 32-byte swizzle (unit u: hi at (2u)k, lo at (2u+1)k)
-  CUtensorMap tm_a;      // A      [n*r*v, k]          box 16 x chunk_cols, 32-byte swizzle
+  CUtensorMap tm_z;      // z      [T, n*r*2*k]        box 64 x 128, 128-byte swizzle (unit u: hi at (2u)k, lo at (2u+1)k)
+  CUtensorMap tm_a;      // A'     [n*v, r*k]          box 64 x chunk_cols, 128-byte swizzle (row (i, b): A[i, 0..r-1, b, :])
   int T, m_tiles, kblocks;
   int n, r, v, vv, k;
   int panels, panel_cols;            // panel q covers the columns [q panel_cols, min(v, (q + 1) panel_cols)) of a unit
@@ -62,21 +67,8 @@ struct LowRankControl {
   uint64_t cempty[kLrCorrStages];
   uint64_t afull[2];                 // base accumulators
   uint64_t aempty[2];
-  uint64_t drain2;
+  uint64_t drain2[kLrMaxGroups];
 };
-
-// K-major operand tile whose rows are `row_bytes` (32, 64 or 128) wide and swizzled with that span: 8-row groups are
-// 8 * row_bytes apart.
-__device__ __forceinline__ uint64_t umma_smem_desc_kmajor(uint32_t smem_addr, uint32_t row_bytes) {
-  const uint64_t layout = row_bytes == 128 ? 2 : (row_bytes == 64 ? 4 : 6);
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>(1) << 16;
-  d |= static_cast<uint64_t>((8 * row_bytes) >> 4) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= layout << 61;
-  return d;
-}
 
 // Wait (bounded) until the copies a producer still has in flight have landed: no copy may be in flight when the CTA goes.
 __device__ __forceinline__ void lowrank_drain_ring(uint64_t* full, int stages, uint32_t issued_mask, uint32_t phase_mask) {
@@ -121,9 +113,12 @@ mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
   const int lane = threadIdx.x & 31;
   const int num_items = p.m_tiles * p.n * p.panels;
   const int kq = p.k / 16;                                // K = 16 steps of one half of a correction
-  const uint32_t zbox = kBlockM * 32;                     // bytes of one z box (128 rows x 32 bytes)
-  const uint32_t abox = static_cast<uint32_t>(p.chunk_cols) * 32;
-  const uint32_t a_off = 2 * kq * zbox;                   // correction entry: [z_hi boxes | z_lo boxes | A boxes (q, c)]
+  const int ca = 64 / p.k;                                // components per correction entry (= per box of A')
+  const int cz = 32 / p.k;                                // components per box of z; an entry has ca / cz = 2 of them
+  const int nent = (p.r + ca - 1) / ca;                   // correction entries per item
+  const uint32_t zbox = kBlockM * 128;                    // bytes of one z box (128 rows x 128 bytes)
+  const uint32_t abox = static_cast<uint32_t>(p.chunk_cols) * 128;
+  const uint32_t a_off = 2 * zbox;                        // correction entry: [z box 0 | z box 1 | A' boxes c = 0 .. nchunk - 1]
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.base_stages; ++s) {
@@ -132,7 +127,7 @@ mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
     }
     for (int s = 0; s < p.corr_stages; ++s) {
       mbar_init(smem_u32(&lc->cfull[s]), 1);
-      mbar_init(smem_u32(&lc->cempty[s]), 1);
+      mbar_init(smem_u32(&lc->cempty[s]), p.groups);        // every correction issuer hands an entry back
     }
     for (int s = 0; s < 2 * p.groups; ++s) {
       mbar_init(smem_u32(&ctl->tfull[s]), 1);
@@ -143,7 +138,7 @@ mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
       mbar_init(smem_u32(&lc->aempty[s]), 4 * p.groups);
     }
     mbar_init(smem_u32(&ctl->drain), 1);
-    mbar_init(smem_u32(&lc->drain2), 1);
+    for (int g = 0; g < p.groups; ++g) mbar_init(smem_u32(&lc->drain2[g]), 1);
     ctl->abort = 0;
     ctl->wait_limit_ns = p.wait_limit_ns;
     fence_mbar_init();
@@ -224,24 +219,22 @@ mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
       bool ok = true;
-      const uint32_t bytes = 2 * kq * zbox + static_cast<uint32_t>(kq * p.nchunk) * abox;
+      const uint32_t bytes = 2 * zbox + static_cast<uint32_t>(p.nchunk) * abox;
       for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
         const LowRankItem w = lowrank_item(p, item);
-        for (int j = 0; j < p.r; ++j) {
+        for (int e = 0; e < nent; ++e) {
           if (!bounded_wait(smem_u32(&lc->cempty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
           const uint32_t full = smem_u32(&lc->cfull[stage]);
           const uint32_t dst = corr_ring + stage * p.corr_stage_bytes;
-          const int unit = w.slot * p.r + j;
+          const int unit0 = w.slot * p.r + e * ca;           // first component of the entry
           mbar_arrive_expect_tx(full, bytes);
-          for (int part = 0; part < 2; ++part)
-            for (int q = 0; q < kq; ++q)
-              tma_load_2d(dst + (part * kq + q) * zbox, &p.tm_z, full, (2 * unit + part) * p.k + 16 * q, w.mt * kBlockM);
-          // all nchunk boxes of a full panel are fetched; boxes may run past the panel (into the next panel, unit, or
-          // the end of A: zero-filled): the MMAs cover only the panel's own columns
-          for (int q = 0; q < kq; ++q)
-            for (int c = 0; c < p.nchunk; ++c)
-              tma_load_2d(dst + a_off + (q * p.nchunk + c) * abox, &p.tm_a, full, 16 * q,
-                          unit * p.v + w.panel * p.panel_cols + c * p.chunk_cols);
+          // boxes may cover components past the slot's last (the next slot's, or zeros past the end) and, for A',
+          // rows past the panel: none of that is multiplied
+          for (int bx = 0; bx < 2; ++bx)
+            tma_load_2d(dst + bx * zbox, &p.tm_z, full, (unit0 + bx * cz) * 2 * p.k, w.mt * kBlockM);
+          for (int c = 0; c < p.nchunk; ++c)
+            tma_load_2d(dst + a_off + c * abox, &p.tm_a, full, e * ca * p.k,
+                        w.slot * p.v + w.panel * p.panel_cols + c * p.chunk_cols);
           issued_mask |= 1u << stage;
           phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
           if (++stage == static_cast<uint32_t>(p.corr_stages)) { stage = 0; phase ^= 1u; }
@@ -250,58 +243,55 @@ mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
       lowrank_drain_ring(lc->cfull, p.corr_stages, issued_mask, phase_mask);
     }
     __syncwarp();
-  } else if (warp == 3) {
-    // ------------------------------------------------------------------ MMA issuer, corrections: `groups` components
-    // at a time (component j0 + g belongs to epilogue group g); their chunks are issued in turn, chunk c of component
-    // j0 + g into slot 2 g + (that group's chunk count & 1)
+  } else if (warp >= 3 && warp < 3 + p.groups) {
+    // ------------------------------------------------------------------ MMA issuer of the corrections of one epilogue
+    // group: its components in turn, chunk c of the group's u-th chunk overall into slot 2 g + (u & 1)
     if (lane == 0) {
-      uint32_t stage = 0, phase = 0;
-      uint32_t cuse[kLrMaxGroups] = {0, 0, 0};
+      const int g = warp - 3;
+      uint32_t stage = 0, phase = 0, cuse = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
         const LowRankItem w = lowrank_item(p, item);
-        for (int j0 = 0; j0 < p.r && ok; j0 += p.groups) {
-          const int ng = min(p.groups, p.r - j0);
-          uint32_t addr[kLrMaxGroups], estage[kLrMaxGroups];
-          for (int g = 0; g < ng && ok; ++g) {
-            if (!bounded_wait(smem_u32(&lc->cfull[stage]), phase, ctl, p.status)) { ok = false; break; }
-            addr[g] = corr_ring + stage * p.corr_stage_bytes;
-            estage[g] = stage;
-            if (++stage == static_cast<uint32_t>(p.corr_stages)) { stage = 0; phase ^= 1u; }
-          }
-          if (!ok) break;
+        for (int e = 0; e < nent && ok; ++e) {
+          if (!bounded_wait(smem_u32(&lc->cfull[stage]), phase, ctl, p.status)) { ok = false; break; }
           tc_fence_after();
-          for (int c = 0; c < w.nchunk && ok; ++c) {
-            const int width = min(p.chunk_cols, w.width - c * p.chunk_cols);
-            const uint32_t idesc = umma_idesc_bf16(kBlockM, width);
-            for (int g = 0; g < ng; ++g) {
-              const uint32_t slot = 2 * g + (cuse[g] & 1u);
-              if (!bounded_wait(smem_u32(&ctl->tempty[slot]), ((cuse[g] >> 1) & 1u) ^ 1u, ctl, p.status)) { ok = false; break; }
+          const uint32_t entry = corr_ring + stage * p.corr_stage_bytes;
+          for (int l = 0; l < ca && ok; ++l) {
+            const int j = e * ca + l;
+            if (j >= p.r) break;
+            if (j % p.groups != g) continue;
+            // descriptors step in 16-byte units: the component's [hi | lo] inside its z box, its k columns inside the A' box
+            const uint64_t z_desc = umma_smem_desc_sw128(entry + (l / cz) * zbox) + ((l % cz) * 2 * p.k) / 8;
+            for (int c = 0; c < w.nchunk; ++c, ++cuse) {
+              const int width = min(p.chunk_cols, w.width - c * p.chunk_cols);
+              const uint32_t idesc = umma_idesc_bf16(kBlockM, width);
+              const uint64_t a_desc = umma_smem_desc_sw128(entry + a_off + c * abox) + (l * p.k) / 8;
+              const uint32_t slot = 2 * g + (cuse & 1u);
+              if (!bounded_wait(smem_u32(&ctl->tempty[slot]), ((cuse >> 1) & 1u) ^ 1u, ctl, p.status)) { ok = false; break; }
               tc_fence_after();
               const uint32_t d_tmem = tmem_base + p.corr_col0 + slot * p.chunk_cols;
               uint32_t acc = 0;
               for (int part = 0; part < 2; ++part)
                 for (int q = 0; q < kq; ++q) {
-                  umma_bf16(d_tmem, umma_smem_desc_kmajor(addr[g] + (part * kq + q) * zbox, 32),
-                            umma_smem_desc_kmajor(addr[g] + a_off + (q * p.nchunk + c) * abox, 32), idesc, acc);
+                  umma_bf16(d_tmem, z_desc + (part * p.k + 16 * q) / 8, a_desc + (16 * q) / 8, idesc, acc);
                   acc = 1;
                 }
               umma_commit(smem_u32(&ctl->tfull[slot]));
-              ++cuse[g];
             }
           }
           if (!ok) break;
-          for (int g = 0; g < ng; ++g) umma_commit(smem_u32(&lc->cempty[estage[g]]));
+          umma_commit(smem_u32(&lc->cempty[stage]));           // (also for an entry none of whose components are this group's)
+          if (++stage == static_cast<uint32_t>(p.corr_stages)) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok || ctl->abort) {
-        umma_commit(smem_u32(&lc->drain2));
+        umma_commit(smem_u32(&lc->drain2[g]));
         const uint64_t t0 = global_timer_ns();
-        while (!mbar_try_wait(smem_u32(&lc->drain2), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(smem_u32(&lc->drain2[g]), 0) && global_timer_ns() - t0 < kWaitLimitNs) {}
       }
     }
     __syncwarp();
-  } else {
+  } else if (warp >= kLrRoleThreads / 32) {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;
     const int group = (warp - kLrRoleThreads / 32) >> 2;      // this warp's epilogue group: components group, group + groups, ...
@@ -441,6 +431,20 @@ __global__ void lowrank_merge_kernel(const float2* __restrict__ partial, const f
     lse_merge(m, s, ms.x, ms.y);
   }
   G[e] = target_logit[e] - (m + __logf(s));
+}
+
+// A [n, r, v, k] -> A' [n, v, r, k] (bf16, k a multiple of 8): one 16-byte piece per thread.
+__global__ void lowrank_repack_kernel(const uint4* __restrict__ A, uint4* __restrict__ out, int n, int r, int v, int kv) {
+  const size_t total = static_cast<size_t>(n) * r * v * kv;      // kv = k / 8 pieces per row
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int q = static_cast<int>(idx % kv);
+  size_t rest = idx / kv;
+  const int j = static_cast<int>(rest % r);
+  rest /= r;
+  const int b = static_cast<int>(rest % v);
+  const int i = static_cast<int>(rest / v);
+  out[idx] = A[((static_cast<size_t>(i) * r + j) * v + b) * kv + q];
 }
 
 }  // namespace mtpc
