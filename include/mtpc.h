@@ -286,12 +286,15 @@ int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k,
  * of 2 d n r v. z is handed to the tensor cores as two bf16 halves (z = hi + lo), so the result differs from exact
  * arithmetic on the bf16 parameters only by fp32 accumulation (no rounding of a composed U to bf16).
  *   cfg, W_sum, T_static, workspace, stream, out: as mtpc_create_head; cfg->io_dtype must be MTPC_BF16.
- *   k        the adaptors' rank: 16 or 32 (MTPC_ERR_UNSUPPORTED otherwise; so are shapes whose base accumulator and two
- *            correction slots do not fit the 512 columns of tensor memory: v up to 480).
+ *   k        the adaptors' rank: 16 or 32 (MTPC_ERR_UNSUPPORTED otherwise). v must be a multiple of 16 that splits into
+ *            at most eight panels of at most 224 columns (a panel's two accumulators and the correction slots share the
+ *            512 columns of tensor memory): every such v up to 1792; MTPC_ERR_UNSUPPORTED otherwise.
  *   W_base   dev [n, v, d] bf16;  A dev [n, r, v, k] bf16;  B dev [n, r, k, d] bf16: caller-owned, read in place, must
  *            outlive the head (after an optimiser step no call is needed unless W_sum / T_static moved:
  *            mtpc_update_parameters with W_emit = NULL then).
- *   workspace >= mtpc_lowrank_workspace_bytes(cfg, k): the dense head's workspace plus z = B h as two bf16 halves.
+ *   workspace >= mtpc_lowrank_workspace_bytes(cfg, k): the dense head's workspace plus z = B h as two bf16 halves, a copy
+ *            of A in the layout the kernel reads (remade on every call, so A is always read as it is then) and, for
+ *            v > 224, the per-panel partial log-sum-exps.
  * Such a head serves mtpc_window_logprob, mtpc_window_prefix_logprob, mtpc_window_loss and mtpc_window_logprob_host.
  * Drafting, acceptance and the backward calls return MTPC_ERR_UNSUPPORTED on it: they run on the composed tensor
  * (mtpc_lowrank_compose + mtpc_create_head, gradients carried back by mtpc_lowrank_backward).
