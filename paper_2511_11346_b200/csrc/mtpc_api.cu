@@ -924,8 +924,8 @@ bool plan_lowrank(const mtpc_config& c, int k, LowRankGemmParams* p) {
   return false;
 }
 
-// Factored projection of a low-rank head: log omega by the dense kernel's sum tiles, z = B h by a plain GEMM, its split
-// into bf16 halves, then the factored kernel writes G.
+// Factored projection of a low-rank head: log omega by the dense kernel's sum tiles, z = B h by a plain GEMM that writes
+// it as two bf16 halves, A repacked, then the factored kernel (and the merge of its panels) writes G.
 int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, const int* targets, cudaStream_t st) {
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
