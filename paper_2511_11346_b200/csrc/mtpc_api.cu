@@ -276,6 +276,8 @@ struct mtpc_head {
   const void* lr_A;                             // [n, r, v, k] bf16
   const void* lr_B;                             // [n, r, k, d] bf16
   size_t lr_off_arep;                           // workspace: A as [n, v, r, k]
+  size_t lr_off_dec;                            // workspace: few-position draft products base [P, n v] | z [P, n r k]
+  CUtensorMap tm_lrB_dec;                       // B [n r k, d] for the few-position draft path
   size_t lr_off_zhl, lr_off_partial;            // workspace: z = B h as bf16 halves [T, n r, 2, k]; per-panel partial log-sum-exps
   LowRankGemmParams lr_params;                  // everything of the factored projection launch that does not depend on the call
   int max_pairs;                                // clusters of two projection CTAs that can be resident at once
@@ -604,12 +606,23 @@ int launch_decode_gemm(mtpc_head* h, const void* hidden_bf16, int P, cudaStream_
   p.tm_sum = h->tm_sum_dec;
   p.kblocks = c.d / kBlockK;
   p.emit_rows = c.n * c.r * c.v;
+  p.logits = at<float>(h, L.off_logits);
+  if (h->lr_k > 0) {
+    // a factored low-rank head streams W_base and B instead of the composed tensor: base = W_base h and z = B h, from
+    // which lowrank_expand_kernel forms the logits
+    p.tm_emit2 = h->tm_lrB_dec;
+    p.emit_rows = c.n * c.v;
+    p.emit2_rows = c.n * c.r * h->lr_k;
+    p.logits = reinterpret_cast<float*>(h->ws + h->lr_off_dec);
+    p.logits2 = p.logits + static_cast<size_t>(L.decode_max_p) * p.emit_rows;
+  }
   p.sum_rows = L.sum_rows;
   p.r = c.r;
   p.tile_rows = h->decode_tile_rows;
   p.sum_tile_rows = h->decode_sum_tile_rows;
   p.tile_bytes = p.tile_rows * kBlockK * 2;
   p.emit_tiles = (p.emit_rows + p.tile_rows - 1) / p.tile_rows;
+  p.emit2_tiles = (p.emit2_rows + p.tile_rows - 1) / p.tile_rows;
   p.sum_tiles = (p.sum_rows + p.sum_tile_rows - 1) / p.sum_tile_rows;
   p.tile_stride = (p.Ppad + 31) / 32 * 32;
   p.pass_tiles = kTmemCols / (2 * p.tile_stride);                     // two slots of pass_tiles accumulators
@@ -622,15 +635,20 @@ int launch_decode_gemm(mtpc_head* h, const void* hidden_bf16, int P, cudaStream_
   const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
   p.stages = (kSmemLimit - ctl) / p.stage_bytes;
   if (p.stages > kMaxStages) p.stages = kMaxStages;
-  p.logits = at<float>(h, L.off_logits);
   p.logw = at<float>(h, L.off_logw);
   p.sum_bias = sum_bias(h);
   p.status = at<unsigned>(h, L.off_status);
   p.wait_limit_ns = h->wait_limit_ns;
-  const int tiles = p.emit_tiles + p.sum_tiles;
+  const int tiles = p.emit_tiles + p.emit2_tiles + p.sum_tiles;
   const int grid = tiles < h->num_sms ? tiles : h->num_sms;
   mtpc_decode_gemm_kernel<<<grid, kGemmThreads, p.stages * p.stage_bytes + ctl, st>>>(p);
   h->launches++;
+  if (h->lr_k > 0) {
+    launch_kernel(lowrank_expand_kernel, dim3(c.n * c.r, (c.v + kExpandThreads - 1) / kExpandThreads), kExpandThreads,
+                  static_cast<size_t>(P) * h->lr_k * sizeof(float), st, h->ring == 0, p.logits, p.logits2,
+                  static_cast<const __nv_bfloat16*>(h->lr_A), at<float>(h, L.off_logits), P, c.n, c.r, c.v, h->lr_k);
+    h->launches++;
+  }
   return check_launch();
 }
 
@@ -686,7 +704,8 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
   const int W = P * wpp;
-  if (!L.can_draft || h->lr_k > 0) return MTPC_ERR_UNSUPPORTED;   // (a factored low-rank head evaluates; drafting wants W_emit)
+  if (!L.can_draft) return MTPC_ERR_UNSUPPORTED;
+  if (h->lr_k > 0 && P > L.decode_max_p) return MTPC_ERR_UNSUPPORTED;   // a factored head drafts on the few-position path only
   const void* hb = nullptr;
   int rc = stage_hidden(h, hidden, P, &hb, st);
   if (rc != MTPC_OK) return rc;
@@ -1134,8 +1153,11 @@ static int bind_parameters(mtpc_head* h, const void* W_emit, const void* W_sum, 
   if (rc == MTPC_OK && dense) rc = make_tmap(&h->tm_emit_lp2, h->W_emit_bf16, emit_rows, cfg->d, L.lp.tile_cols / 2);
   if (rc == MTPC_OK && dense && L.can_draft_many) rc = make_tmap(&h->tm_emit_sm2, h->W_emit_bf16, emit_rows, cfg->d, L.sm.tile_cols / 2);
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum2, h->W_sum_bf16, L.sum_rows, cfg->d, L.sum_cols / 2);
-  h->decode_tile_rows = decode_tile_rows(static_cast<long long>(emit_rows), h->num_sms);
+  const uint64_t base_rows = static_cast<uint64_t>(cfg->n) * cfg->v, adapt_rows = static_cast<uint64_t>(cfg->n) * cfg->r * h->lr_k;
+  h->decode_tile_rows = decode_tile_rows(static_cast<long long>(dense ? emit_rows : base_rows + adapt_rows), h->num_sms);
   if (rc == MTPC_OK && dense) rc = make_tmap(&h->tm_emit_dec, h->W_emit_bf16, emit_rows, cfg->d, h->decode_tile_rows);
+  if (rc == MTPC_OK && !dense) rc = make_tmap(&h->tm_emit_dec, h->lr_W_base, base_rows, cfg->d, h->decode_tile_rows);
+  if (rc == MTPC_OK && !dense) rc = make_tmap(&h->tm_lrB_dec, h->lr_B, adapt_rows, cfg->d, h->decode_tile_rows);
   h->decode_sum_tile_rows = h->decode_tile_rows / 32 * 32;   // whole groups of r <= 32 rows per warp; fits the tile pitch
   if (rc == MTPC_OK) rc = make_tmap(&h->tm_sum_dec, h->W_sum_bf16, L.sum_rows, cfg->d, h->decode_sum_tile_rows);
   h->draft_P = 0;                                              // logits left by an earlier draft belong to the old parameters
@@ -1165,7 +1187,7 @@ struct LowRankSpec {
 // that computes it), where a unit is cut into panels the panels' (maximum, sum) pairs and the targets' logits, and the
 // copy of A the factored kernel reads.
 static int lowrank_extra_bytes(const mtpc_config& c, int k, int panels, size_t base_total, size_t* off_zhl,
-                               size_t* off_partial, size_t* off_arep, size_t* total) {
+                               size_t* off_partial, size_t* off_arep, size_t* off_dec, size_t* total) {
   const size_t units = static_cast<size_t>(c.n) * c.r;
   size_t off = align_up(base_total);
   *off_zhl = off;
@@ -1174,6 +1196,9 @@ static int lowrank_extra_bytes(const mtpc_config& c, int k, int panels, size_t b
   if (panels > 1) off += align_up(static_cast<size_t>(c.max_positions) * units * (panels * sizeof(float2) + sizeof(float)));
   *off_arep = off;                      // the copy of A laid out [n, v, r, k]
   off += align_up(units * c.v * k * 2);
+  *off_dec = off;                       // few-position draft: base = W_base h [P, n v] and z = B h [P, n r k], fp32
+  off += align_up(static_cast<size_t>(c.max_positions < kDecodeMaxP ? c.max_positions : kDecodeMaxP) *
+                  (static_cast<size_t>(c.n) * c.v + units * k) * 4);
   *total = off;
   return MTPC_OK;
 }
@@ -1189,11 +1214,11 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
   if (rc != MTPC_OK) return rc;
   LowRankGemmParams lrp;
   memset(&lrp, 0, sizeof(lrp));
-  size_t lr_zhl = 0, lr_partial = 0, lr_arep = 0;
+  size_t lr_zhl = 0, lr_partial = 0, lr_arep = 0, lr_dec = 0;
   if (lowrank) {
     if (cfg->io_dtype != MTPC_BF16) return MTPC_ERR_UNSUPPORTED;
     if (!plan_lowrank(*cfg, lowrank->k, &lrp)) return MTPC_ERR_UNSUPPORTED;
-    lowrank_extra_bytes(*cfg, lowrank->k, lrp.panels, L.total, &lr_zhl, &lr_partial, &lr_arep, &L.total);
+    lowrank_extra_bytes(*cfg, lowrank->k, lrp.panels, L.total, &lr_zhl, &lr_partial, &lr_arep, &lr_dec, &L.total);
   }
   const bool ctx = (cfg->flags & MTPC_FLAG_HMM_CONTEXTUAL) != 0;
   if (cfg->family == MTPC_HMM && cfg->n > 1 && !ctx && !T_static) return MTPC_ERR_NULL;
@@ -1217,6 +1242,7 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
     h->lr_off_zhl = lr_zhl;
     h->lr_off_partial = lr_partial;
     h->lr_off_arep = lr_arep;
+    h->lr_off_dec = lr_dec;
     h->lr_params = lrp;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1273,8 +1299,8 @@ int mtpc_lowrank_workspace_bytes(const mtpc_config* cfg, int32_t k, size_t* out_
   if (rc != MTPC_OK) return rc;
   LowRankGemmParams lrp;
   if (cfg->io_dtype != MTPC_BF16 || !plan_lowrank(*cfg, k, &lrp)) return MTPC_ERR_UNSUPPORTED;
-  size_t a = 0, b = 0, c3 = 0;
-  return lowrank_extra_bytes(*cfg, k, lrp.panels, L.total, &a, &b, &c3, out_bytes);
+  size_t a = 0, b = 0, c3 = 0, c4 = 0;
+  return lowrank_extra_bytes(*cfg, k, lrp.panels, L.total, &a, &b, &c3, &c4, out_bytes);
 }
 
 int mtpc_create_head_lowrank(const mtpc_config* cfg, int32_t k, const void* W_base, const void* A, const void* B,

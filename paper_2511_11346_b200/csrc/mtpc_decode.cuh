@@ -36,8 +36,11 @@ struct DecodeParams {
   CUtensorMap tm_h;      // hidden [P, d]       box 64 x Ppad
   CUtensorMap tm_emit;   // W_emit [n*r*v, d]   box 64 x tile_rows
   CUtensorMap tm_sum;    // W_sum  [S*r, d]     box 64 x sum_tile_rows
+  CUtensorMap tm_emit2;  // a second matrix of emission-like rows [emit2_rows, d], box 64 x tile_rows (a factored
+                         // low-rank head: tm_emit = W_base, tm_emit2 = B); unused when emit2_tiles == 0
   int P, Ppad, kblocks;
   int emit_rows, sum_rows, r;
+  int emit2_rows, emit2_tiles;
   int tile_rows;                 // rows of an emission tile (a multiple of 8, <= 128)
   int sum_tile_rows;             // rows of a sum tile (a multiple of 32, <= tile_rows rounded up to 32)
   int tile_bytes;                // shared-memory pitch of a weight tile
@@ -46,20 +49,22 @@ struct DecodeParams {
   int tile_stride;               // TMEM columns per tile
   int stages, stage_bytes;
   float* logits;         // [P, emit_rows]
+  float* logits2;        // [P, emit2_rows]
   float* logw;           // [P, sum_rows]
   const float* sum_bias; // [sum_rows] or NULL: added to the sum-unit logits before their softmax
   unsigned* status;
   uint64_t wait_limit_ns;   // limit of every pipeline wait
 };
 
-// Tile `t` of the launch: emission tiles first, then sum tiles.
+// Tile `t` of the launch: emission tiles first, then those of the second matrix, then sum tiles.
 struct DecodeTile {
-  int is_sum, index, rows;   // which matrix, tile index within it, rows per tile
+  int is_sum, second, index, rows;   // which matrix, tile index within it, rows per tile
 };
 __device__ __forceinline__ DecodeTile decode_tile(const DecodeParams& p, int t) {
   DecodeTile d;
-  d.is_sum = t >= p.emit_tiles;
-  d.index = d.is_sum ? t - p.emit_tiles : t;
+  d.is_sum = t >= p.emit_tiles + p.emit2_tiles;
+  d.second = !d.is_sum && t >= p.emit_tiles;
+  d.index = d.is_sum ? t - p.emit_tiles - p.emit2_tiles : (d.second ? t - p.emit_tiles : t);
   d.rows = d.is_sum ? p.sum_tile_rows : p.tile_rows;
   return d;
 }
@@ -78,7 +83,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_decode_gemm_kernel(const
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int total_tiles = p.emit_tiles + p.sum_tiles;
+  const int total_tiles = p.emit_tiles + p.emit2_tiles + p.sum_tiles;
   const int tile_begin = static_cast<int>(static_cast<long long>(blockIdx.x) * total_tiles / gridDim.x);
   const int tile_end = static_cast<int>(static_cast<long long>(blockIdx.x + 1) * total_tiles / gridDim.x);
   const uint32_t hidden_off = p.pass_tiles * p.tile_bytes;
@@ -100,6 +105,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_decode_gemm_kernel(const
     tma_prefetch_desc(&p.tm_h);
     tma_prefetch_desc(&p.tm_emit);
     tma_prefetch_desc(&p.tm_sum);
+    if (p.emit2_tiles > 0) tma_prefetch_desc(&p.tm_emit2);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
@@ -127,7 +133,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_decode_gemm_kernel(const
           mbar_arrive_expect_tx(full, bytes);
           for (int q = 0; q < ntiles; ++q) {
             const DecodeTile t = decode_tile(p, cur + q);
-            tma_load_2d(dst + q * p.tile_bytes, t.is_sum ? &p.tm_sum : &p.tm_emit, full, kb * kBlockK, t.index * t.rows);
+            tma_load_2d(dst + q * p.tile_bytes, t.is_sum ? &p.tm_sum : (t.second ? &p.tm_emit2 : &p.tm_emit), full,
+                        kb * kBlockK, t.index * t.rows);
           }
           tma_load_2d(dst + hidden_off, &p.tm_h, full, kb * kBlockK, 0);
           issued_mask |= 1u << stage;
@@ -203,8 +210,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) mtpc_decode_gemm_kernel(const
       for (int q = 0; q < ntiles; ++q) {
         const DecodeTile t = decode_tile(p, cur + q);
         if (quarter * 32 >= t.rows) continue;                      // warp-uniform: none of this warp's lanes is a row
-        const int nrows = t.is_sum ? p.sum_rows : p.emit_rows;
-        float* dst = t.is_sum ? p.logw : p.logits;
+        const int nrows = t.is_sum ? p.sum_rows : (t.second ? p.emit2_rows : p.emit_rows);
+        float* dst = t.is_sum ? p.logw : (t.second ? p.logits2 : p.logits);
         const uint32_t tcol = lane_base + slot * slot_cols + q * p.tile_stride;
         const int local = quarter * 32 + lane;
         const int row = t.index * t.rows + local;

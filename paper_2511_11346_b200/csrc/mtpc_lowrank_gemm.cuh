@@ -447,4 +447,51 @@ __global__ void lowrank_repack_kernel(const uint4* __restrict__ A, uint4* __rest
   out[idx] = A[((static_cast<size_t>(i) * r + j) * v + b) * kv + q];
 }
 
+// Few-position draft on a factored head: logits[p, i, j, b] = base[p, i, b] + sum_q A[i, j, b, q] z[p, i, j, q], from the
+// two small products the weight pass left (base = W_base h [P, n v], z = B h [P, n r k], fp32). One CTA per (unit,
+// 256 symbols): a thread keeps its symbol's adaptor row in registers and walks the positions, whose z rows sit in shared
+// memory. Launched as a programmatic dependent of the weight pass.
+constexpr int kExpandThreads = 256;
+__global__ void __launch_bounds__(kExpandThreads) lowrank_expand_kernel(const float* __restrict__ base,
+                                                                        const float* __restrict__ z,
+                                                                        const __nv_bfloat16* __restrict__ A,
+                                                                        float* __restrict__ logits, int P, int n, int r,
+                                                                        int v, int k) {
+  extern __shared__ float zs[];                                 // [P, k]
+  grid_launch_dependents();
+  grid_dependency_wait();
+  const int unit = blockIdx.x, i = unit / r;
+  const int b = blockIdx.y * kExpandThreads + threadIdx.x;
+  const size_t units = static_cast<size_t>(n) * r;
+  for (int e = threadIdx.x; e < P * k; e += kExpandThreads) zs[e] = z[(static_cast<size_t>(e / k) * units + unit) * k + e % k];
+  __syncthreads();
+  if (b >= v) return;
+  float a[kLrMaxRank];
+  const uint4* arow = reinterpret_cast<const uint4*>(A + (static_cast<size_t>(unit) * v + b) * k);   // k bf16 = k / 8 pieces
+#pragma unroll
+  for (int q = 0; q < kLrMaxRank / 8; ++q) {
+    if (q * 8 < k) {
+      const uint4 piece = arow[q];
+      const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&piece);
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const float2 f = __bfloat1622float2(h2[t]);
+        a[q * 8 + 2 * t] = f.x;
+        a[q * 8 + 2 * t + 1] = f.y;
+      }
+    } else {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) a[q * 8 + t] = 0.f;
+    }
+  }
+  for (int pos = 0; pos < P; ++pos) {
+    float acc = base[(static_cast<size_t>(pos) * n + i) * v + b];
+    const float* zp = zs + pos * k;
+#pragma unroll
+    for (int q = 0; q < kLrMaxRank; ++q)
+      if (q < k) acc = fmaf(a[q], zp[q], acc);
+    logits[(static_cast<size_t>(pos) * units + unit) * v + b] = acc;
+  }
+}
+
 }  // namespace mtpc

@@ -46,12 +46,20 @@ def lowrank_backward(lora_A, lora_B, dW_emit):
 class DeviceHead:
     """Weights of a workload resident in HBM plus a head created on them."""
 
-    def __init__(self, wl: I.Workload, max_positions: int | None = None, max_wpp: int | None = None, device="cuda"):
+    def __init__(self, wl: I.Workload, max_positions: int | None = None, max_wpp: int | None = None, device="cuda",
+                 lowrank=None):
+        """lowrank = (W_base, A, B) as fp32 arrays of bf16-representable values: a head that keeps the shared
+        unembeddings factored (wl.W_emit_q is then not uploaded)."""
         import torch
         s = wl.shape
         self.wl = wl
         self.device = device
-        if s.io_dtype == I.F32:
+        self.lowrank = None
+        if lowrank is not None:
+            self.lowrank = tuple(to_device_bf16(np.ascontiguousarray(x), device) for x in lowrank)
+            self.W_emit = None
+            self.W_sum = to_device_bf16(wl.W_sum_q, device)
+        elif s.io_dtype == I.F32:
             self.W_emit = torch.from_numpy(wl.W_emit_raw).to(device)
             self.W_sum = torch.from_numpy(wl.W_sum_raw).to(device)
         else:
@@ -61,7 +69,8 @@ class DeviceHead:
         ctx = s.family == I.HMM_CTX
         self.head = B.MtpcHead(B.MTPC_HMM if ctx else s.family, s.n, s.r, s.v, s.d, s.io_dtype,
                                max_positions or max(wl.T, 1), max_wpp or max(wl.wpp, 1), self.W_emit, self.W_sum,
-                               self.T_static, flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0, v_valid=s.v_valid)
+                               self.T_static, flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0, v_valid=s.v_valid,
+                               lowrank=self.lowrank)
 
     def hidden_device(self, rows=None):
         import torch

@@ -105,13 +105,14 @@ def target_rows_for(wl, W, bytes_o, logphi, logw, pos):
     return p.astype(np.float32)
 
 
-def check_accept(wl, wpp):
+def check_accept(wl, wpp, lowrank=None):
+    """lowrank = (W_base, A, B): the device head keeps them factored; wl.W_emit_q must then be their exact composition."""
     s = wl.shape
     P, n = wl.T, s.n
     W = P * wpp
     rows = np.arange(P)
     pos = np.repeat(rows, wpp)
-    dh = DeviceHead(wl)
+    dh = DeviceHead(wl, lowrank=lowrank)
     hidden_d = dh.hidden_device()            # kept alive: after a many-position draft the acceptance stage reads it again
     bytes_g, prefix_g = dh.draft_sample_prefix(wpp, hidden=hidden_d)
     assert dh.head.mtpc_get_status() == 0
@@ -203,6 +204,24 @@ def test_accept_small_shapes(family, n, r, v, d, P, wpp):
     wl = I.make_workload(f"acc_{family}_{n}_{r}_{v}", I.HeadShape(family, n, r, v, d), P, seed=3000 + 5 * n + r + v + P,
                          wpp=wpp, weight_std=0.25)
     check_accept(wl, wpp)
+
+
+@pytest.mark.parametrize("family,n,r,v,d,k,P,wpp", [
+    (I.CP, 4, 8, 320, 128, 16, 5, 16),
+    (I.HMM, 6, 8, 64, 128, 32, 9, 8),
+    (I.BTREE, 4, 16, 256, 128, 16, 6, 8),
+    (I.HMM_CTX, 4, 4, 48, 64, 16, 128, 2),     # the most positions the few-position path takes
+    (I.CP, 2, 4, 1024, 64, 16, 3, 4),          # a vocabulary wider than 512 symbols
+])
+def test_draft_and_accept_on_a_factored_low_rank_head(family, n, r, v, d, k, P, wpp):
+    """App. G's shared unembeddings kept factored (U_ij = W_i + A_ij B_ij never formed): the few-position draft streams
+    W_base and B once, forms the logits from the two small products, and everything after is the dense head's path. Bytes,
+    prefix marginals and acceptance decisions must be the oracle's on the exactly composed tensor."""
+    wl = I.make_workload(f"lr_draft_{family}_{n}_{r}", I.HeadShape(family, n, r, v, d), P, seed=5200 + n + r + v + P,
+                         wpp=wpp, weight_std=0.25)
+    Wb, A, Bm = I.lowrank_parameters(n, r, v, d, k, seed=5300 + n + r, weight_std=0.25, adaptor_std=0.2)
+    wl.W_emit_q = orc.lowrank_unembedding(Wb, A, Bm)       # fp64, exact: what the factored head computes on
+    check_accept(wl, wpp, lowrank=(Wb, A, Bm))
 
 
 @pytest.mark.parametrize("cell", [(I.CP, 8, 8), (I.CP, 16, 1), (I.HMM, 8, 64), (I.HMM, 16, 8)])
