@@ -350,9 +350,55 @@ def measure_lowrank(torch, wl, dW_emit, steps: int, peaks, k: int = 16):
            "backward_algorithmic_bytes": bytes_b, "backward_frac_of_hbm": bytes_b / (ms_b * 1e-3) / 1e9 / hbm,
            "note": "CUDA-core kernels: k multiply-adds per element keep the fp32 pipes, not HBM, busiest; the three "
                    "gradient kernels each stream dW_emit once"}
-    if wl.shape.io_dtype == I.BF16 and s.v % 32 == 0 and s.v <= 448:
+    if wl.shape.io_dtype == I.BF16 and s.v % 16 == 0:
         out["factored_forward"] = measure_factored_forward(torch, wl, (Wb, A, Bm), steps)
+        out["factored_draft"] = measure_factored_draft(torch, wl, (Wb, A, Bm), peaks)
     return out
+
+
+def measure_factored_draft(torch, wl, lowrank, peaks, P: int = 8, wpp: int = 16, calls: int = 200):
+    """mtpc_draft_sample for a few positions on a head that keeps the shared unembeddings factored: the weight pass streams
+    W_base and B (and the sum-unit weights) instead of the composed tensor, so "one pass over the weights" is
+    2 d (n v + n r k + sum rows) + 2 n r v k bytes."""
+    from paper_2511_11346_b200 import binding as B
+    from paper_2511_11346_b200.runner import to_device_bf16
+    s = wl.shape
+    k = lowrank[1].shape[-1]
+    ctx = s.family == I.HMM_CTX
+    W_sum = to_device_bf16(wl.W_sum_q)
+    Ts = torch.from_numpy(np.ascontiguousarray(wl.T_static)).cuda() if wl.T_static is not None else None
+    head = B.MtpcHead(B.MTPC_HMM if ctx else s.family, s.n, s.r, s.v, s.d, B.MTPC_BF16, P, wpp, None, W_sum, Ts,
+                      flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0, v_valid=s.v_valid, lowrank=lowrank)
+    hidden = to_device_bf16(np.ascontiguousarray(wl.hidden_q[:P]))
+    W = P * wpp
+    u = torch.from_numpy(I.uniforms(I.BASE_SEED + 91, 7, (W, 2 * s.n))).cuda()
+    ob = torch.empty((W, s.n), dtype=torch.int32, device="cuda")
+    ol = torch.empty(W, dtype=torch.float32, device="cuda")
+    for _ in range(5):
+        head.mtpc_draft_sample(hidden, wpp, u, ob, ol)
+    torch.cuda.synchronize()
+    lat = []
+    for _ in range(calls):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        head.mtpc_draft_sample(hidden, wpp, u, ob, ol)
+        e1.record()
+        e1.synchronize()
+        lat.append(e0.elapsed_time(e1))
+    ref_b = ob.clone()
+    graph_lat = graph_replay_times(torch, lambda st: head.mtpc_draft_sample(hidden, wpp, u, ob, ol, stream=st), (ob, ol), calls, 5)
+    identical = bool((ob == ref_b).all())
+    status = head.mtpc_get_status()
+    head.mtpc_destroy()
+    p50, g50 = statistics.median(lat), statistics.median(graph_lat)
+    weight_bytes = 2 * s.d * (s.n * s.v + s.n * s.r * k + s.sum_rows) + 2 * s.n * s.r * s.v * k
+    dense_bytes = 2 * s.d * (s.n * s.r * s.v + s.sum_rows)
+    return {"call": f"mtpc_draft_sample on a factored head, P={P} wpp={wpp}", "p50_ms": p50, "cuda_graph_replay_p50_ms": g50,
+            "graph_results_identical": identical, "windows_per_s": W / (p50 * 1e-3), "kernels_per_call": 4,
+            "weight_bytes": weight_bytes, "dense_weight_bytes": dense_bytes,
+            "hbm_frac": weight_bytes / (g50 * 1e-3) / 1e9 / peaks["hbm_gbs"], "device_status": status,
+            "note": "weight pass (W_base, B, sum units) + logits from the two small products + per-slot kernel + circuit; "
+                    "at these sizes the call is a chain of four short kernels, not a bandwidth problem"}
 
 
 def measure_factored_forward(torch, wl, lowrank, steps: int):
