@@ -726,7 +726,12 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
       const size_t base = static_cast<size_t>((2 * c.r + 3) & ~3) * sizeof(float);
       const size_t with_tables = base + static_cast<size_t>(chain) * c.r * c.r * sizeof(float);
       const int in_smem = chain > 0 && with_tables <= kSlotSmemLimit;
-      launch_kernel(c.v > kMaxDraftVocab ? draft_slot_kernel<true> : draft_slot_kernel<false>, dim3(c.n, P), kSlotThreads,
+      // builds of the narrow kernel that unroll 4, 8, 10 or 16 batches of 32 symbols: the smallest that covers v
+      auto* slot_kernel = c.v > kMaxDraftVocab ? draft_slot_kernel<true, 16>
+                          : c.v <= 128 ? draft_slot_kernel<false, 4>
+                          : c.v <= 256 ? draft_slot_kernel<false, 8>
+                          : c.v <= 320 ? draft_slot_kernel<false, 10> : draft_slot_kernel<false, 16>;
+      launch_kernel(slot_kernel, dim3(c.n, P), kSlotThreads,
                     in_smem ? with_tables : base, st, h->ring == 0, c.family,
                     at<float>(h, L.off_logits), at<float>(h, L.off_logw), hmm_tables(h), uniforms, out_bytes,
                     at<float>(h, L.off_G), at<float>(h, L.off_unit_lse), at<unsigned>(h, L.off_status),
@@ -1262,10 +1267,12 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
   fail |= !allow_full_smem(plain_gemm_kernel<true, true>);
   fail |= cudaFuncSetAttribute(mtpc_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
           cudaSuccess;
-  fail |= cudaFuncSetAttribute(draft_slot_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               static_cast<int>(kSlotSmemLimit)) != cudaSuccess;
-  fail |= cudaFuncSetAttribute(draft_slot_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               static_cast<int>(kSlotSmemLimit)) != cudaSuccess;
+  const int slot_smem = static_cast<int>(kSlotSmemLimit);
+  fail |= cudaFuncSetAttribute(draft_slot_kernel<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, slot_smem) != cudaSuccess;
+  fail |= cudaFuncSetAttribute(draft_slot_kernel<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, slot_smem) != cudaSuccess;
+  fail |= cudaFuncSetAttribute(draft_slot_kernel<false, 10>, cudaFuncAttributeMaxDynamicSharedMemorySize, slot_smem) != cudaSuccess;
+  fail |= cudaFuncSetAttribute(draft_slot_kernel<false, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, slot_smem) != cudaSuccess;
+  fail |= cudaFuncSetAttribute(draft_slot_kernel<true, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, slot_smem) != cudaSuccess;
   fail |= !set_circuit_attributes();
   fail |= !allow_full_smem(spec_accept_kernel);
   fail |= cudaMemsetAsync(h->ws + L.off_status, 0, 256, st) != cudaSuccess;

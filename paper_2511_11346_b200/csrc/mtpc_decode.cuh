@@ -364,15 +364,16 @@ __device__ __forceinline__ float warp_chunk_sum(const float* __restrict__ x, int
 // consecutive symbols [c0 + l*per, c0 + (l+1)*per). The threshold is u * (the chunk's total) when `relative`, else
 // `thr` itself. Returns the smallest symbol whose running sum exceeds the threshold; the last existing symbol of
 // the chunk if rounding leaves none. All lanes return the same value.
+template <int NQ>   // per <= NQ <= kSlotMaxPerLane: the steps that are unrolled
 __device__ __forceinline__ int warp_inv_cdf_chunk(const float* __restrict__ x, int c0, int per, int vv, float m, float thr,
                                                   bool relative, int lane) {
   const int b0 = c0 + lane * per;
-  float ev[kSlotMaxPerLane];
+  float ev[NQ];
 #pragma unroll
-  for (int q = 0; q < kSlotMaxPerLane; ++q) ev[q] = (q < per && b0 + q < vv) ? x[b0 + q] : -CUDART_INF_F;
+  for (int q = 0; q < NQ; ++q) ev[q] = (q < per && b0 + q < vv) ? x[b0 + q] : -CUDART_INF_F;
   float part = 0.f;
 #pragma unroll
-  for (int q = 0; q < kSlotMaxPerLane; ++q) {
+  for (int q = 0; q < NQ; ++q) {
     ev[q] = __expf(ev[q] - m);
     part += ev[q];
   }
@@ -387,7 +388,7 @@ __device__ __forceinline__ int warp_inv_cdf_chunk(const float* __restrict__ x, i
     if (lane == src) {
       float cum = lane == 0 ? 0.f : before;
 #pragma unroll
-      for (int q = 0; q < kSlotMaxPerLane; ++q)
+      for (int q = 0; q < NQ; ++q)
         if (found < 0 && q < per && b0 + q < vv) {
           cum += ev[q];
           if (thr < cum) found = b0 + q;
@@ -406,8 +407,8 @@ __device__ __forceinline__ int warp_inv_cdf_chunk(const float* __restrict__ x, i
 // are computed, so that the data-dependent row reads of the latent draws do not each cost a trip to L2.
 // The log-sum-exps also go to unit_lse_out [P, n, r], so that later calls can turn the retained logits into log phi.
 // WIDE: vocabularies of more than 512 symbols (a separate build: the narrow one keeps a unit's logits in 16 registers per lane).
-template <bool WIDE>
-__global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
+template <bool WIDE, int NQ>   // NQ: batches of 32 symbols of a unit that are unrolled (v <= 32 NQ; WIDE: 16)
+__global__ void __launch_bounds__(kSlotThreads, 2) draft_slot_kernel(
     int family, const float* __restrict__ logits, const float* __restrict__ logw, const float* __restrict__ logA,
     const float* __restrict__ uniforms, int* __restrict__ out_bytes, float* __restrict__ G,
     float* __restrict__ unit_lse_out, unsigned* status, unsigned* work_counter, int wpp, int n, int r, int v, int vv,
@@ -451,21 +452,21 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
     const float* x = row + static_cast<size_t>(k) * v;
     float m = -CUDART_INF_F, s = 0.f;
     for (int c0 = 0; c0 < (WIDE ? v : 1); c0 += kChunk) {
-      float xv[kSlotMaxPerLane];
+      float xv[NQ];
 #pragma unroll
-      for (int q = 0; q < kSlotMaxPerLane; ++q) {
+      for (int q = 0; q < NQ; ++q) {
         const int b = c0 + lane + 32 * q;
         xv[q] = b < vv ? x[b] : -CUDART_INF_F;   // [vv, v): padding symbols
       }
       float cm = xv[0];
 #pragma unroll
-      for (int q = 1; q < kSlotMaxPerLane; ++q) cm = fmaxf(cm, xv[q]);
+      for (int q = 1; q < NQ; ++q) cm = fmaxf(cm, xv[q]);
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) cm = fmaxf(cm, __shfl_xor_sync(kFull, cm, off));
       const float mn = fmaxf(m, cm);           // finite from the first chunk on (symbol 0 always exists)
       float cs = 0.f;
 #pragma unroll
-      for (int q = 0; q < kSlotMaxPerLane; ++q) cs += __expf(xv[q] - mn);   // padding: exp(-inf) = 0
+      for (int q = 0; q < NQ; ++q) cs += __expf(xv[q] - mn);   // padding: exp(-inf) = 0
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) cs += __shfl_xor_sync(kFull, cs, off);
       s = s * __expf(m - mn) + cs;             // first chunk: 0 * exp(-inf) = 0
@@ -513,7 +514,7 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
       const float m = unit_max[z];
       if (!WIDE) {
         // ---- inverse CDF over the v bytes of unit z: lane l owns bytes [l*per, (l+1)*per)
-        byte = warp_inv_cdf_chunk(x, 0, per, vv, m, ub, true, lane);
+        byte = warp_inv_cdf_chunk<NQ>(x, 0, per, vv, m, ub, true, lane);
       } else {
         // ---- wide vocabulary: 512 symbols at a time. First the total (chunk sums in fp32, added up in fp64), then
         // the chunk the threshold u * total falls into, then the draw inside that chunk.
@@ -525,7 +526,7 @@ __global__ void __launch_bounds__(kSlotThreads) draft_slot_kernel(
         for (int c0 = 0; c0 < v; c0 += kChunk) {
           const float cs = warp_chunk_sum(x, c0, vv, m, lane);
           if (thr < before + static_cast<double>(cs)) {
-            byte = warp_inv_cdf_chunk(x, c0, kSlotMaxPerLane, vv, m, static_cast<float>(thr - before), false, lane);
+            byte = warp_inv_cdf_chunk<kSlotMaxPerLane>(x, c0, kSlotMaxPerLane, vv, m, static_cast<float>(thr - before), false, lane);
             break;
           }
           before += static_cast<double>(cs);
