@@ -298,11 +298,30 @@ int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k,
  * Such a head serves mtpc_window_logprob, mtpc_window_prefix_logprob, mtpc_window_loss, mtpc_window_logprob_host, and,
  * for up to 128 positions per call, mtpc_draft_sample, mtpc_draft_sample_prefix and mtpc_speculative_accept: the draft's
  * weight pass then streams W_base and B (n v + n r k rows) instead of n r v composed rows, and the logits are formed
- * from the two small products. Drafts of more than 128 positions and the backward calls return MTPC_ERR_UNSUPPORTED on
- * it: they run on the composed tensor (mtpc_lowrank_compose + mtpc_create_head, gradients carried back by
- * mtpc_lowrank_backward).
+ * from the two small products. Its training call is mtpc_lowrank_window_logprob_backward (below). Drafts of more than
+ * 128 positions, mtpc_window_logprob_backward and mtpc_window_loss_backward return MTPC_ERR_UNSUPPORTED on it: those run
+ * on the composed tensor (mtpc_lowrank_compose + mtpc_create_head, gradients carried back by mtpc_lowrank_backward).
  */
 int mtpc_lowrank_workspace_bytes(const mtpc_config* cfg, int32_t k, size_t* out_bytes);
+
+/*
+ * Training call of a factored head (App. G): out_logprob[t] = log q(targets[t]) as mtpc_window_logprob, and the gradients
+ * of sum_t weight[t] out_logprob[t] with respect to the hidden states and to the parameters the head was built on, without
+ * the [n, r, v, d] gradient of a composed tensor ever existing: with g = d / d logit [T, n r v],
+ *   dW_base[i] = (sum_j g_ij)^T h,   dA[i,j] = g_ij^T (B[i,j] h),   dB[i,j] = (g_ij A[i,j])^T h,
+ *   d_hidden   = sum_i (sum_j g_ij) W_base[i] + sum_ij (g_ij A[i,j]) B[i,j] + the sum units' part.
+ *   hidden, targets, T, weight, out_logprob, d_hidden [T, d], dW_sum, dT_static: as mtpc_window_logprob_backward.
+ *   dW_base dev [n, v, d] fp32;  dA dev [n, r, v, k] fp32;  dB dev [n, r, k, d] fp32: OVERWRITTEN.
+ *   bwd_workspace  dev, 256-byte aligned, >= mtpc_lowrank_backward_workspace_bytes(cfg, k, T): the kept logits
+ *                  [T, n r v] fp32, their gradients in bf16, and the small operands derived from them.
+ * g is rounded to bf16 before the tensor cores contract it (as in mtpc_window_logprob_backward), dA uses the bf16 high
+ * half of B h. MTPC_ERR_STATE on a head that was not created by mtpc_create_head_lowrank. Asynchronous on `stream`.
+ */
+int mtpc_lowrank_backward_workspace_bytes(const mtpc_config* cfg, int32_t k, int32_t T, size_t* out_bytes);
+int mtpc_lowrank_window_logprob_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t T,
+                                         const float* weight, void* bwd_workspace, size_t bwd_workspace_bytes,
+                                         float* out_logprob, float* d_hidden, float* dW_base, float* dA, float* dB,
+                                         float* dW_sum, float* dT_static, void* stream);
 int mtpc_create_head_lowrank(const mtpc_config* cfg, int32_t k, const void* W_base, const void* A, const void* B,
                              const void* W_sum, const float* T_static, void* workspace, size_t workspace_bytes,
                              void* stream, mtpc_head** out);

@@ -675,9 +675,19 @@ struct GemmOperand {
   bool mn_major;
 };
 
+// Optional extras of a plain GEMM launch: bf16 output instead of fp32, and several products of one shape in a launch
+// (see PlainGemmParams); a_* / b_* extents: the whole matrices the batched operands are windows of (M or N, then K).
+struct PlainGemmExtra {
+  void* C_bf16 = nullptr;
+  int batches = 1, a_m_step = 0, a_k_step = 0, b_n_step = 0, b_k_step = 0;
+  size_t c_step = 0;
+  long long a_extent_m = 0, a_extent_k = 0, b_extent_n = 0, b_extent_k = 0;
+};
 int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmOperand B1, int K1, int a_k1, float* C,
-                      size_t ldc, int M, int N, cudaStream_t st, void* C_hilo = nullptr, int split_k = 0);
-int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, const int* targets, cudaStream_t st);
+                      size_t ldc, int M, int N, cudaStream_t st, void* C_hilo = nullptr, int split_k = 0,
+                      const PlainGemmExtra* extra = nullptr);
+int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, const int* targets, cudaStream_t st,
+                              const GradArgs* ga = nullptr);
 
 // out [T] (joint) and / or prefix [T, n] (prefix log-marginals); either may be NULL, not both.
 int window_logprob_impl(mtpc_head* h, const void* hidden, const int32_t* targets, int32_t T, float* out, float* prefix,
@@ -856,15 +866,20 @@ void plan_backward(const mtpc_config& c, const Layout& L, int T, BackwardLayout*
 // A's K range [a_k1, a_k1 + K1) with B1.
 // C_hilo != NULL (then C is NULL): the result leaves as two bf16 halves per entry, see PlainGemmParams.
 int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmOperand B1, int K1, int a_k1, float* C,
-                      size_t ldc, int M, int N, cudaStream_t st, void* C_hilo, int split_k) {
+                      size_t ldc, int M, int N, cudaStream_t st, void* C_hilo, int split_k, const PlainGemmExtra* extra) {
   if (M <= 0 || N <= 0 || K0 <= 0) return MTPC_OK;
   if (K1 > 0 && (A.mn_major || B1.mn_major != B0.mn_major)) return MTPC_ERR_SHAPE;
+  const PlainGemmExtra none;
+  const PlainGemmExtra& x = extra ? *extra : none;
+  if (x.batches < 1 || (x.batches > 1 && K1 > 0)) return MTPC_ERR_SHAPE;
   PlainGemmParams p;
   memset(&p, 0, sizeof(p));
   const int Ka = K1 > 0 ? a_k1 + K1 : K0;                      // extent of A along K
-  int rc = A.mn_major ? make_tmap_mn(&p.tm_a, A.ptr, Ka, M, A.pitch) : make_tmap(&p.tm_a, A.ptr, M, Ka, kBlockM, A.pitch);
+  const uint64_t a_m = x.a_extent_m ? x.a_extent_m : M, a_k = x.a_extent_k ? x.a_extent_k : Ka;
+  const uint64_t b_n = x.b_extent_n ? x.b_extent_n : N, b_k = x.b_extent_k ? x.b_extent_k : K0;
+  int rc = A.mn_major ? make_tmap_mn(&p.tm_a, A.ptr, a_k, a_m, A.pitch) : make_tmap(&p.tm_a, A.ptr, a_m, a_k, kBlockM, A.pitch);
   if (rc == MTPC_OK)
-    rc = B0.mn_major ? make_tmap_mn(&p.tm_b[0], B0.ptr, K0, N, B0.pitch) : make_tmap(&p.tm_b[0], B0.ptr, N, K0, kPlainTileN, B0.pitch);
+    rc = B0.mn_major ? make_tmap_mn(&p.tm_b[0], B0.ptr, b_k, b_n, B0.pitch) : make_tmap(&p.tm_b[0], B0.ptr, b_n, b_k, kPlainTileN, B0.pitch);
   if (rc == MTPC_OK && K1 > 0)
     rc = B1.mn_major ? make_tmap_mn(&p.tm_b[1], B1.ptr, K1, N, B1.pitch) : make_tmap(&p.tm_b[1], B1.ptr, N, K1, kPlainTileN, B1.pitch);
   if (rc != MTPC_OK) return rc;
@@ -879,16 +894,22 @@ int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmO
   const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
   p.stages = (kSmemLimit - ctl) / p.stage_bytes;
   if (p.stages > kMaxStages) p.stages = kMaxStages;
-  p.wide_stores = (reinterpret_cast<uintptr_t>(C) % 32 == 0 && ldc % 8 == 0) ? 1 : 0;
+  p.wide_stores = (reinterpret_cast<uintptr_t>(C) % 32 == 0 && ldc % 8 == 0 && x.c_step % 8 == 0) ? 1 : 0;
   p.C = C;
   p.ldc = ldc;
   p.C_hilo = static_cast<__nv_bfloat16*>(C_hilo);
   p.split_k = split_k;
-  if ((C == nullptr) == (C_hilo == nullptr)) return MTPC_ERR_NULL;
+  p.C_bf16 = static_cast<__nv_bfloat16*>(x.C_bf16);
+  if ((C != nullptr) + (C_hilo != nullptr) + (x.C_bf16 != nullptr) != 1) return MTPC_ERR_NULL;
   if (C_hilo != nullptr && (split_k < 16 || split_k % 16 != 0 || N % split_k != 0)) return MTPC_ERR_SHAPE;
+  if (x.C_bf16 != nullptr && (reinterpret_cast<uintptr_t>(x.C_bf16) % 32 != 0 || ldc % 16 != 0 || x.c_step % 16 != 0))
+    return MTPC_ERR_WORKSPACE;
+  p.batches = x.batches;
+  p.a_m_step = x.a_m_step; p.a_k_step = x.a_k_step; p.b_n_step = x.b_n_step; p.b_k_step = x.b_k_step;
+  p.c_step = x.c_step;
   p.status = at<unsigned>(h, h->L.off_status);
   p.wait_limit_ns = h->wait_limit_ns;
-  const long long items = static_cast<long long>(p.m_tiles) * p.n_tiles;
+  const long long items = static_cast<long long>(p.m_tiles) * p.n_tiles * p.batches;
   const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
   const size_t smem = p.stages * p.stage_bytes + ctl;
   if (A.mn_major && B0.mn_major) plain_gemm_kernel<true, true><<<grid, kGemmThreads, smem, st>>>(p);
@@ -950,7 +971,8 @@ bool plan_lowrank(const mtpc_config& c, int k, LowRankGemmParams* p) {
 
 // Factored projection of a low-rank head: log omega by the dense kernel's sum tiles, z = B h by a plain GEMM that writes
 // it as two bf16 halves, A repacked, then the factored kernel (and the merge of its panels) writes G.
-int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, const int* targets, cudaStream_t st) {
+int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, const int* targets, cudaStream_t st,
+                              const GradArgs* ga) {
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
   const int units = c.n * c.r, k = h->lr_k;
@@ -978,6 +1000,11 @@ int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, cons
   p.G = at<float>(h, L.off_G);
   p.status = at<unsigned>(h, L.off_status);
   p.wait_limit_ns = h->wait_limit_ns;
+  if (ga != nullptr) {                 // a training call keeps every logit and every unit's log-sum-exp
+    p.logit_out = ga->logit_out;
+    p.logit_pitch = ga->logit_pitch;
+    p.lse_out = ga->lse_out;
+  }
   const size_t entries = static_cast<size_t>(T) * units;
   p.partial = reinterpret_cast<float2*>(h->ws + h->lr_off_partial);
   p.target_logit = reinterpret_cast<float*>(h->ws + h->lr_off_partial +
@@ -990,7 +1017,7 @@ int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, cons
   h->launches += 1;
   if (p.panels > 1) {     // several panels per unit: their partial log-sum-exps are combined into G
     lowrank_merge_kernel<<<static_cast<unsigned>((entries + 255) / 256), 256, 0, st>>>(
-        p.partial, p.target_logit, targets, p.G, p.status, entries, c.r, p.vv, p.panels);
+        p.partial, p.target_logit, targets, p.G, p.lse_out, p.status, entries, c.r, p.vv, p.panels);
     h->launches += 1;
   }
   return check_launch();
@@ -1096,6 +1123,30 @@ int backward_tail(mtpc_head* head, const BackwardLayout& B, uint8_t* bw, const v
   if (rc == MTPC_OK) rc = launch_plain_gemm(head, s_cols, hid, T, hid, 0, 0, dW_sum, c.d, L.sum_rows, c.d, st);
   pt.end();
   return rc;
+}
+
+// Backward workspace of a factored head: the dense layout (log-sum-exps, posteriors, kept logits, logit gradients), then
+//   sy    [T, n v | n r k | S r padded] bf16: the logit gradients summed over a slot's components, multiplied by the
+//         adaptors A, and those of the sum units: the A operand of d hidden and of the three weight-gradient GEMMs;
+//   wcat  [n v + n r k, d] bf16: W_base and B one after the other (one K segment of d hidden);
+//   apad  [n r, v rounded up to 64, k] bf16: A with zero rows between the units.
+struct LowRankBackwardLayout {
+  BackwardLayout B;
+  size_t Ksy, pitch, v64;
+  size_t off_sy, off_wcat, off_apad, total;
+};
+void plan_lowrank_backward(const mtpc_config& c, const Layout& L, int k, int T, LowRankBackwardLayout* R) {
+  plan_backward(c, L, T, &R->B);
+  const size_t units = static_cast<size_t>(c.n) * c.r;
+  R->Ksy = static_cast<size_t>(c.n) * c.v + units * k;
+  R->pitch = R->Ksy + R->B.Spad;
+  R->v64 = round64(c.v);
+  size_t off = R->B.total;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  R->off_sy = take(static_cast<size_t>(T) * R->pitch * 2);
+  R->off_wcat = take(R->Ksy * c.d * 2);
+  R->off_apad = take(units * R->v64 * k * 2);
+  R->total = off;
 }
 
 int check_call(mtpc_head* h, int32_t rows) {
@@ -1548,6 +1599,151 @@ int mtpc_window_logprob_backward(mtpc_head* head, const void* hidden, const int3
   if (rc != MTPC_OK) return rc;
   // 3., 4. logit gradients from the kept logits, then the plain GEMMs
   return backward_tail(head, B, bw, hb, targets, T, d_hidden, dW_emit, dW_sum, pt, st);
+}
+
+int mtpc_lowrank_backward_workspace_bytes(const mtpc_config* cfg, int32_t k, int32_t T, size_t* out_bytes) {
+  if (!cfg || !out_bytes) return MTPC_ERR_NULL;
+  if (T < 1) return MTPC_ERR_SHAPE;
+  Layout L;
+  int rc = plan(*cfg, &L);
+  if (rc != MTPC_OK) return rc;
+  LowRankGemmParams lrp;
+  if (cfg->io_dtype != MTPC_BF16 || !plan_lowrank(*cfg, k, &lrp)) return MTPC_ERR_UNSUPPORTED;
+  LowRankBackwardLayout R;
+  plan_lowrank_backward(*cfg, L, k, T, &R);
+  *out_bytes = R.total;
+  return MTPC_OK;
+}
+
+int mtpc_lowrank_window_logprob_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t T,
+                                         const float* weight, void* bwd_workspace, size_t bwd_workspace_bytes,
+                                         float* out_logprob, float* d_hidden, float* dW_base, float* dA, float* dB,
+                                         float* dW_sum, float* dT_static, void* stream) {
+  int rc = check_call(head, T);
+  if (rc != MTPC_OK) return rc;
+  if (T == 0) return MTPC_OK;
+  if (!hidden || !targets || !weight || !bwd_workspace || !d_hidden || !dW_base || !dA || !dB || !dW_sum) return MTPC_ERR_NULL;
+  if (head->lr_k == 0) return MTPC_ERR_STATE;                  // a head on a composed tensor: mtpc_window_logprob_backward
+  const mtpc_config& c = head->cfg;
+  const Layout& L = head->L;
+  const int k = head->lr_k, units = c.n * c.r;
+  const bool static_hmm = c.family == MTPC_HMM && !is_ctx(head) && c.n > 1;
+  if (static_hmm && !dT_static) return MTPC_ERR_NULL;
+  LowRankBackwardLayout R;
+  plan_lowrank_backward(c, L, k, T, &R);
+  const BackwardLayout& B = R.B;
+  if (bwd_workspace_bytes < R.total || (reinterpret_cast<uintptr_t>(bwd_workspace) % kAlign) != 0) return MTPC_ERR_WORKSPACE;
+  if ((rc = set_backward_attributes(head)) != MTPC_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* bw = static_cast<uint8_t*>(bwd_workspace);
+  const void* hb = hidden;                                     // (factored heads are bf16)
+  head->draft_P = 0;
+  PhaseTimer pt(head, st);
+  // 1. factored forward projection, keeping every logit and every unit's log-sum-exp
+  pt.begin();
+  GradArgs fwd;
+  fwd.lse_out = reinterpret_cast<float*>(bw + B.off_lse);
+  fwd.logit_out = reinterpret_cast<float*>(bw + B.off_logits);
+  fwd.logit_pitch = B.Nc;
+  rc = launch_lowrank_projection(head, hb, T, targets, st, &fwd);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  // 2. circuit backward: posteriors of the input units; the sum units' logit gradients go to the right of sy
+  pt.begin();
+  if (static_hmm && cudaMemsetAsync(dT_static, 0, static_cast<size_t>(c.n - 1) * c.r * c.r * 4, st) != cudaSuccess)
+    return MTPC_ERR_CUDA;
+  __nv_bfloat16* sy = reinterpret_cast<__nv_bfloat16*>(bw + R.off_sy);
+  CircuitBackwardArgs a;
+  memset(&a, 0, sizeof(a));
+  a.targets = targets;
+  a.weight = weight;
+  a.weight_stride = 1;
+  a.out = out_logprob;
+  a.post = reinterpret_cast<float*>(bw + B.off_post);
+  a.dsum = sy + R.Ksy;
+  a.dsum_pitch = static_cast<int>(R.pitch);
+  a.len = c.n;
+  a.W = T;
+  rc = launch_circuit_backward(head, a, dT_static, st);
+  pt.end();
+  if (rc != MTPC_OK) return rc;
+  // 3. logit gradients g [T, n r v] (bf16), their sum over a slot's components, the zero-padded A, W_base and B in a row
+  pt.begin();
+  __nv_bfloat16* dlogit = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit);
+  const int Nc = static_cast<int>(B.Nc);
+  LogitGradArgs la;
+  la.logits = reinterpret_cast<const float*>(bw + B.off_logits);
+  la.lse = reinterpret_cast<const float*>(bw + B.off_lse);
+  la.post = reinterpret_cast<const float*>(bw + B.off_post);
+  la.targets = targets;
+  la.dlogit = dlogit;
+  la.pitch = B.Kd;
+  la.T = T; la.Nc = Nc; la.n = c.n; la.r = c.r; la.v = c.v;
+  {
+    const int col_blocks = (Nc / 8 + 255) / 256;
+    int row_blocks = (16 * head->num_sms + col_blocks - 1) / col_blocks;
+    if (row_blocks > T) row_blocks = T;
+    if (row_blocks > 65535) row_blocks = 65535;
+    logit_gradient_kernel<<<dim3(col_blocks, row_blocks), 256, 0, st>>>(la);
+  }
+  {
+    const size_t pieces = static_cast<size_t>(T) * (c.n * c.v / 8);
+    lowrank_component_sum_kernel<<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, st>>>(dlogit, B.Kd, sy, R.pitch, T,
+                                                                                               c.n, c.r, c.v);
+    const size_t pad_pieces = static_cast<size_t>(units) * R.v64 * (k / 8);
+    lowrank_pad_kernel<<<static_cast<unsigned>((pad_pieces + 255) / 256), 256, 0, st>>>(
+        static_cast<const uint4*>(head->lr_A), reinterpret_cast<uint4*>(bw + R.off_apad), units, c.v, static_cast<int>(R.v64), k / 8);
+  }
+  head->launches += 3;
+  uint8_t* wcat = bw + R.off_wcat;
+  const size_t base_bytes = static_cast<size_t>(c.n) * c.v * c.d * 2;
+  bool fail = cudaMemcpyAsync(wcat, head->lr_W_base, base_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess;
+  fail |= cudaMemcpyAsync(wcat + base_bytes, head->lr_B, static_cast<size_t>(units) * k * c.d * 2, cudaMemcpyDeviceToDevice, st) != cudaSuccess;
+  if (fail || (rc = check_launch()) != MTPC_OK) return MTPC_ERR_CUDA;
+  pt.end();
+  // 4. the GEMMs
+  pt.begin();
+  const GemmOperand none{nullptr, 0, false};
+  const GemmOperand hid{hb, static_cast<size_t>(c.d), true};
+  {   // y_ij = g_ij A_ij [T, k], one product per unit, into the middle columns of sy
+    PlainGemmExtra x;
+    x.C_bf16 = sy + static_cast<size_t>(c.n) * c.v;
+    x.batches = units;
+    x.a_k_step = c.v;
+    x.b_k_step = static_cast<int>(R.v64);
+    x.c_step = k;
+    x.a_extent_m = T; x.a_extent_k = Nc;
+    x.b_extent_n = k; x.b_extent_k = static_cast<long long>(units) * R.v64;
+    rc = launch_plain_gemm(head, GemmOperand{dlogit, B.Kd, false}, GemmOperand{bw + R.off_apad, static_cast<size_t>(k), true},
+                           static_cast<int>(R.v64), none, 0, 0, nullptr, R.pitch, T, k, st, nullptr, 0, &x);
+  }
+  // d hidden [T, d] = [s | y] [W_base ; B] + dsum W_sum
+  if (rc == MTPC_OK)
+    rc = launch_plain_gemm(head, GemmOperand{sy, R.pitch, false}, GemmOperand{wcat, static_cast<size_t>(c.d), true},
+                           static_cast<int>(R.Ksy), GemmOperand{head->W_sum_bf16, static_cast<size_t>(c.d), true}, L.sum_rows,
+                           static_cast<int>(R.Ksy), d_hidden, c.d, T, c.d, st);
+  // dW_base = s^T h, dB = y^T h, dW_sum = dsum^T h: sy down its columns
+  if (rc == MTPC_OK)
+    rc = launch_plain_gemm(head, GemmOperand{sy, R.pitch, true}, hid, T, hid, 0, 0, dW_base, c.d, c.n * c.v, c.d, st);
+  if (rc == MTPC_OK)
+    rc = launch_plain_gemm(head, GemmOperand{sy + static_cast<size_t>(c.n) * c.v, R.pitch, true}, hid, T, hid, 0, 0, dB, c.d,
+                           units * k, c.d, st);
+  if (rc == MTPC_OK)
+    rc = launch_plain_gemm(head, GemmOperand{sy + R.Ksy, R.pitch, true}, hid, T, hid, 0, 0, dW_sum, c.d, L.sum_rows, c.d, st);
+  if (rc == MTPC_OK) {   // dA_ij [v, k] = g_ij^T z_ij, one product per unit, on the bf16 high half of z the forward pass left
+    PlainGemmExtra x;
+    x.batches = units;
+    x.a_m_step = c.v;
+    x.b_n_step = 2 * k;
+    x.c_step = static_cast<size_t>(c.v) * k;
+    x.a_extent_m = Nc; x.a_extent_k = T;
+    x.b_extent_n = static_cast<long long>(units) * 2 * k; x.b_extent_k = T;
+    rc = launch_plain_gemm(head, GemmOperand{dlogit, B.Kd, true},
+                           GemmOperand{head->ws + head->lr_off_zhl, static_cast<size_t>(units) * 2 * k, true}, T, none, 0, 0, dA,
+                           k, c.v, k, st, nullptr, 0, &x);
+  }
+  pt.end();
+  return rc;
 }
 
 int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,

@@ -667,6 +667,15 @@ struct PlainGemmParams {
   // (group g of split_k columns: hi at column (2 g) split_k, lo at (2 g + 1) split_k; split_k a multiple of 16).
   __nv_bfloat16* C_hilo;
   int split_k;
+  // Instead of C (C == NULL, C_hilo == NULL): the result rounded to bf16, [M, N] at a pitch of ldc elements.
+  __nv_bfloat16* C_bf16;
+  // Several independent products of the same shape in one launch (batches > 1; one K segment): product q reads A at
+  // its M / K coordinates plus q * a_m_step / q * a_k_step, B at its N / K coordinates plus q * b_n_step / q * b_k_step,
+  // and writes at C (or C_bf16) + q * c_step elements. Rows of A and columns of B past M and N are then another product's
+  // data, not zeros: they reach accumulator rows and columns that are not written. Along K the operands must agree on
+  // zeros past the product's own extent (the caller pads one of them).
+  int batches, a_m_step, a_k_step, b_n_step, b_k_step;
+  size_t c_step;
   unsigned* status;
   uint64_t wait_limit_ns;   // limit of every pipeline wait
 };
@@ -684,7 +693,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
   const int lane = threadIdx.x & 31;
   // n-tile fastest: the CTAs running together cover a few m-tiles x all n-tiles, so the (larger) A operand is
   // streamed from HBM once and the B operand once per wave of m-tiles
-  const int num_items = p.m_tiles * p.n_tiles;
+  const int per_batch = p.m_tiles * p.n_tiles;
+  const int num_items = per_batch * p.batches;
   const int kblocks = p.seg_kblocks[0] + p.seg_kblocks[1];
   constexpr uint32_t kSlots = 2;
   constexpr uint32_t kBBytes = kPlainTileN * kBlockK * 2;
@@ -720,7 +730,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
       uint32_t stage = 0, phase = 0, issued_mask = 0, phase_mask = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
-        const int nt = item % p.n_tiles, mt = item / p.n_tiles;
+        const int bt = item / per_batch, rest = item - bt * per_batch;
+        const int nt = rest % p.n_tiles, mt = rest / p.n_tiles;
+        const int am = mt * kBlockM + bt * p.a_m_step, ak = bt * p.a_k_step;    // this product's corner of A ...
+        const int bn = nt * kPlainTileN + bt * p.b_n_step, bk = bt * p.b_k_step;   // ... and of B
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
           const uint32_t full = smem_u32(&ctl->full[stage]);
@@ -731,16 +744,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
           if (A_MN) {
 #pragma unroll
             for (int q = 0; q < kBlockM / 64; ++q)
-              tma_load_2d(a_dst + q * kMnBoxBytes, &p.tm_a, full, mt * kBlockM + q * 64, p.a_k0[seg] + kloc);
+              tma_load_2d(a_dst + q * kMnBoxBytes, &p.tm_a, full, am + q * 64, p.a_k0[seg] + kloc + ak);
           } else {
-            tma_load_2d(a_dst, &p.tm_a, full, p.a_k0[seg] + kloc, mt * kBlockM);
+            tma_load_2d(a_dst, &p.tm_a, full, p.a_k0[seg] + kloc + ak, am);
           }
           if (B_MN) {
 #pragma unroll
             for (int q = 0; q < kPlainTileN / 64; ++q)
-              tma_load_2d(a_dst + kABytes + q * kMnBoxBytes, &p.tm_b[seg], full, nt * kPlainTileN + q * 64, kloc);
+              tma_load_2d(a_dst + kABytes + q * kMnBoxBytes, &p.tm_b[seg], full, bn + q * 64, kloc + bk);
           } else {
-            tma_load_2d(a_dst + kABytes, &p.tm_b[seg], full, kloc, nt * kPlainTileN);
+            tma_load_2d(a_dst + kABytes, &p.tm_b[seg], full, kloc + bk, bn);
           }
           issued_mask |= 1u << stage;
           phase_mask = (phase_mask & ~(1u << stage)) | (phase << stage);
@@ -798,18 +811,28 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
     const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
     uint32_t use = 0;
     for (int item = blockIdx.x; item < num_items; item += gridDim.x, ++use) {
-      const int nt = item % p.n_tiles, mt = item / p.n_tiles;
+      const int bt = item / per_batch, rest = item - bt * per_batch;
+      const int nt = rest % p.n_tiles, mt = rest / p.n_tiles;
       const uint32_t slot = use % kSlots;
       if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (use / kSlots) & 1u, ctl, p.status, lane)) break;
       tc_fence_after();
       const int row = mt * kBlockM + quarter * 32 + lane;
       const uint32_t tcol = lane_base + slot * kPlainTileN;
-      float* crow = p.C + static_cast<size_t>(row < p.M ? row : 0) * p.ldc;
+      const size_t coff = static_cast<size_t>(row < p.M ? row : 0) * p.ldc + static_cast<size_t>(bt) * p.c_step;
+      float* crow = p.C + coff;
       for (int b = 0; b < kPlainTileN / 16; ++b) {
+        const int col0 = nt * kPlainTileN + b * 16;
+        if (col0 >= p.N) break;                          // (warp-uniform) the rest of the tile lies past the last column
         float x[16];
         tmem_ld16(tcol + b * 16, x);
-        const int col0 = nt * kPlainTileN + b * 16;
-        if (row < p.M && col0 < p.N && p.C == nullptr) {
+        if (row < p.M && p.C == nullptr && p.C_hilo == nullptr) {
+          __align__(16) __nv_bfloat16 o[16];
+#pragma unroll
+          for (int q = 0; q < 16; ++q) o[q] = __float2bfloat16_rn(x[q]);
+          uint4* dst = reinterpret_cast<uint4*>(p.C_bf16 + coff + col0);      // ldc, c_step and C_bf16 keep 16 columns 32-byte aligned
+          dst[0] = reinterpret_cast<const uint4*>(o)[0];
+          dst[1] = reinterpret_cast<const uint4*>(o)[1];
+        } else if (row < p.M && col0 < p.N && p.C == nullptr) {
           // 16 columns of one group: 32 bytes of high halves and 32 bytes of low halves
           const int grp = col0 / p.split_k, q0 = col0 - grp * p.split_k;
           __align__(16) __nv_bfloat16 hi[16], lo[16];

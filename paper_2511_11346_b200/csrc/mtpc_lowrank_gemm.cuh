@@ -57,6 +57,9 @@ struct LowRankGemmParams {
   float* G;                          // [T, n, r]
   float2* partial;                   // panels > 1: [panels, T n r] (running maximum, sum of exponentials) of each panel
   float* target_logit;               // panels > 1: [T n r] logit of the target, written by the panel that holds it
+  float* logit_out;                  // training: every logit [T, n r v] fp32 at a pitch of logit_pitch (NULL: not kept) ...
+  size_t logit_pitch;
+  float* lse_out;                    // ... and every unit's log-sum-exp [T, n r] (with several panels: by the merge kernel)
   unsigned* status;
   uint64_t wait_limit_ns;
 };
@@ -325,6 +328,11 @@ mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
             for (int q = 0; q < 16; ++q) x[q] = __uint_as_float(rc[q]) + __uint_as_float(rb[q]);
             const int col0 = panel_col0 + col_chunk + b * 16; // column inside the unit
             mask_padding(x, col0, p.vv);
+            if (p.logit_out != nullptr && valid) {            // row of the logit matrix: (slot, component, symbol)
+              float* l = p.logit_out + static_cast<size_t>(row) * p.logit_pitch + (static_cast<size_t>(w.slot) * p.r + j) * p.v + col0;
+              st_global_v8(l, x);
+              st_global_v8(l + 8, x + 8);
+            }
             // short dependent chains: reduce as trees
             float t8[8];
 #pragma unroll
@@ -381,6 +389,7 @@ mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
         if (valid) {
           const size_t e = (static_cast<size_t>(row) * p.n + w.slot) * p.r + j;
           if (p.panels == 1) {
+            if (p.lse_out != nullptr) p.lse_out[e] = m + fast_lg2(s) * kLn2;
             if (tgt < 0) {
               p.G[e] = 0.f;                                  // marginalised byte: the input unit sums to 1
             } else if (tgt >= p.vv) {
@@ -414,10 +423,17 @@ mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
 // G[t, i, j] = logit[target] - LSE over the unit, from the per-panel (maximum, sum of exponentials) the factored projection
 // left: one thread per (position, slot, component). Targets < 0 (marginalised): 0; targets >= vv: NaN and the status bit.
 __global__ void lowrank_merge_kernel(const float2* __restrict__ partial, const float* __restrict__ target_logit,
-                                     const int* __restrict__ targets, float* __restrict__ G, unsigned* status,
-                                     size_t entries, int r, int vv, int panels) {
+                                     const int* __restrict__ targets, float* __restrict__ G, float* __restrict__ lse_out,
+                                     unsigned* status, size_t entries, int r, int vv, int panels) {
   const size_t e = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (e >= entries) return;
+  float m = -CUDART_INF_F, s = 0.f;
+  for (int q = 0; q < panels; ++q) {
+    const float2 ms = partial[static_cast<size_t>(q) * entries + e];
+    lse_merge(m, s, ms.x, ms.y);
+  }
+  const float lse = m + __logf(s);
+  if (lse_out != nullptr) lse_out[e] = lse;
   const int tgt = targets[e / r];
   if (tgt < 0) { G[e] = 0.f; return; }
   if (tgt >= vv) {
@@ -425,12 +441,7 @@ __global__ void lowrank_merge_kernel(const float2* __restrict__ partial, const f
     atomicOr(status, kStatusBadTarget);
     return;
   }
-  float m = -CUDART_INF_F, s = 0.f;
-  for (int q = 0; q < panels; ++q) {
-    const float2 ms = partial[static_cast<size_t>(q) * entries + e];
-    lse_merge(m, s, ms.x, ms.y);
-  }
-  G[e] = target_logit[e] - (m + __logf(s));
+  G[e] = target_logit[e] - lse;
 }
 
 // A [n, r, v, k] -> A' [n, v, r, k] (bf16, k a multiple of 8): one 16-byte piece per thread.
@@ -492,6 +503,50 @@ __global__ void __launch_bounds__(kExpandThreads) lowrank_expand_kernel(const fl
       if (q < k) acc = fmaf(a[q], zp[q], acc);
     logits[(static_cast<size_t>(pos) * units + unit) * v + b] = acc;
   }
+}
+
+// Backward pass of a factored head (App. G): with g = d loss / d logit [T, n r v] (bf16), the gradients are
+//   dW_base[i] = (sum_j g_ij)^T h,   dA_ij = g_ij^T (B_ij h),   dB_ij = (g_ij A_ij)^T h,
+//   d hidden   = (sum_j g_ij) W_base[i] + (g_ij A_ij) B_ij  summed over the slots and components.
+// lowrank_component_sum_kernel: S[t, i, b] = sum_j g[t, i, j, b], written as bf16 into a matrix of pitch out_pitch (where
+// it is the A operand of the GEMMs that follow). Eight symbols per thread, 16-byte loads and stores.
+__global__ void __launch_bounds__(256) lowrank_component_sum_kernel(const __nv_bfloat16* __restrict__ g, size_t g_pitch,
+                                                                    __nv_bfloat16* __restrict__ out, size_t out_pitch, int T,
+                                                                    int n, int r, int v) {
+  const int per_row = n * v / 8;                                 // 16-byte pieces of one row of S
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(T) * per_row) return;
+  const int t = static_cast<int>(idx / per_row), c = static_cast<int>(idx % per_row) * 8;
+  const int i = c / v, b = c - i * v;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  const __nv_bfloat16* src = g + static_cast<size_t>(t) * g_pitch + static_cast<size_t>(i) * r * v + b;
+  for (int j = 0; j < r; ++j) {
+    const uint4 piece = *reinterpret_cast<const uint4*>(src + static_cast<size_t>(j) * v);
+    const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&piece);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float2 f = __bfloat1622float2(h2[q]);
+      acc[2 * q] += f.x;
+      acc[2 * q + 1] += f.y;
+    }
+  }
+  __align__(16) __nv_bfloat16 o[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) o[q] = __float2bfloat16_rn(acc[q]);
+  *reinterpret_cast<uint4*>(out + static_cast<size_t>(t) * out_pitch + c) = *reinterpret_cast<const uint4*>(o);
+}
+
+// A [n r, v, k] -> [n r, v64, k] with v64 = v rounded up to 64 and zero rows past v: the batched GEMM g_ij A_ij walks K in
+// blocks of 64 symbols, and what it reads of g past a unit's own columns must meet zeros.
+__global__ void lowrank_pad_kernel(const uint4* __restrict__ A, uint4* __restrict__ out, int units, int v, int v64, int kv) {
+  const size_t total = static_cast<size_t>(units) * v64 * kv;    // kv = k / 8 pieces per row
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int q = static_cast<int>(idx % kv);
+  const size_t rest = idx / kv;
+  const int b = static_cast<int>(rest % v64);
+  const size_t u = rest / v64;
+  out[idx] = b < v ? A[(u * v + b) * kv + q] : make_uint4(0u, 0u, 0u, 0u);
 }
 
 }  // namespace mtpc

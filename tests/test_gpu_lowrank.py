@@ -254,3 +254,90 @@ def test_a_wait_that_runs_out_in_the_factored_kernel_is_reported_and_the_head_re
     assert head.mtpc_get_status(with_code=True) == (B.MTPC_OK, 0)
     assert np.abs(out.cpu().numpy() - ref).max() <= 2e-3
     head.mtpc_destroy()
+
+
+# --------------------------------------------------------------------------- training call of the factored head
+def _check_tensor(name, got, ref, magnitude_sum, floor):
+    """Entry by entry |got - ref| <= 2.2 * 2^-8 * (sum of the magnitudes of the products behind the entry) + floor: every
+    product has at most two factors that the device rounded to bf16 (the logit gradient, and its sum over the components,
+    its product with A, or the high half of B h); as a whole: relative L2 error below 1e-2."""
+    got = got.cpu().numpy().astype(np.float64).reshape(ref.shape)
+    assert np.isfinite(got).all(), name
+    bound = 2.2 * 2.0 ** -8 * magnitude_sum.reshape(ref.shape) + floor
+    excess = np.abs(got - ref) - bound
+    worst = np.unravel_index(np.argmax(excess), excess.shape)
+    assert excess[worst] <= 0, f"{name}: entry {worst} differs by {abs(got[worst] - ref[worst])}, bound {bound[worst]}"
+    rel2 = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    assert rel2 <= 1e-2 or np.abs(ref).max() < 100 * floor, f"{name}: relative L2 error {rel2}"
+    return float((np.abs(got - ref) / bound).max()), rel2
+
+
+@pytest.mark.parametrize("family,n,r,v,vv,d,k,T", [
+    (I.CP, 2, 4, 320, 0, 128, 16, 300),        # two panels; v a multiple of 64
+    (I.HMM, 4, 8, 64, 0, 64, 32, 257),         # rank 32, static transitions (dT_static)
+    (I.BTREE, 4, 4, 48, 44, 64, 16, 70),       # padded vocabulary, v not a multiple of 64: the zero rows of the padded A
+    (I.HMM_CTX, 3, 8, 320, 0, 128, 16, 200),   # contextual transitions: the sum units carry most of d hidden
+    (I.CP, 2, 4, 272, 268, 64, 16, 90),        # ragged panels and a ragged K block per unit
+    (I.CP, 1, 1, 16, 0, 64, 16, 5),
+])
+def test_factored_backward_is_the_chain_rule_through_the_composition(family, n, r, v, vv, d, k, T):
+    """mtpc_lowrank_window_logprob_backward against the oracle: the gradient of sum_t weight[t] log q_t with respect to the
+    exactly composed U (fp64), carried back to W_base, A and B by the oracle's reverse mode through U = W + A B."""
+    wl, W, A, Bm = _factored_case(family, n, r, v, vv, d, k, T, seed=6100 + v + k + T)
+    sym = vv or v
+    fam = wl.shape.family
+    U = O.lowrank_unembedding(W, A, Bm)[:, :, :sym, :]
+    t = wl.targets.copy()
+    if T > 8 and n > 1:
+        t[3, 1] = -1
+    weight = np.random.default_rng(T).normal(size=T).astype(np.float32)
+    if T > 4:
+        weight[2] = 0.0
+    ref = OG.window_logprob_grad(fam, wl.hidden_q, U, wl.W_sum_q, wl.T_static, t, weight)
+    dU = np.zeros((n, r, v, d))
+    dU[:, :, :sym] = ref["dW_emit"]
+    lr = OG.lowrank_grad(W, A, Bm, dU)
+    ctx = family == I.HMM_CTX
+    Ts = torch.from_numpy(np.ascontiguousarray(wl.T_static)).cuda() if wl.T_static is not None else None
+    head = B.MtpcHead(B.MTPC_HMM if ctx else family, n, r, v, d, B.MTPC_BF16, T, 1, None, to_device_bf16(wl.W_sum_q), Ts,
+                      flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0, v_valid=vv, lowrank=(_device(W), _device(A), _device(Bm)))
+    f32 = dict(dtype=torch.float32, device="cuda")
+    S = wl.W_sum_q.shape[0]
+    out = dict(logprob=torch.empty(T, **f32), dh=torch.empty((T, d), **f32), dW_base=torch.empty((n, v, d), **f32),
+               dA=torch.empty((n, r, v, k), **f32), dB=torch.empty((n, r, k, d), **f32), dW_sum=torch.empty((S, d), **f32),
+               dT=torch.empty((max(n - 1, 1), r, r), **f32) if fam == I.HMM else None)
+    hidden = to_device_bf16(wl.hidden_q)
+    for _ in range(2):                       # twice: nothing of the first call may leak into the second
+        head.mtpc_lowrank_window_logprob_backward(hidden, torch.from_numpy(t).cuda(), torch.from_numpy(weight).cuda(),
+                                                  out["logprob"], out["dh"], out["dW_base"], out["dA"], out["dB"],
+                                                  out["dW_sum"], out["dT"])
+    assert head.mtpc_get_status() == 0
+    assert np.abs(out["logprob"].cpu().numpy() - ref["logprob"]).max() <= 2e-3
+    # magnitudes behind every entry, from the oracle's logit gradients
+    lg = OG.window_logprob_logit_grad(fam, wl.hidden_q, U, wl.W_sum_q, wl.T_static, t, weight)
+    g = np.zeros((T, n, r, v))
+    g[..., :sym] = np.abs(lg["dlogit"]).reshape(T, n, r, sym)
+    ds = np.abs(lg["dslog"]).reshape(T, -1)
+    ah = np.abs(wl.hidden_q.astype(np.float64))
+    aW, aA, aB = np.abs(W.astype(np.float64)), np.abs(A.astype(np.float64)), np.abs(Bm.astype(np.float64))
+    gs = g.sum(axis=2)                                             # [T, n, v]
+    gy = np.einsum("tijb,ijbq->tijq", g, aA)                       # [T, n, r, k]
+    z = np.abs(np.einsum("ijqd,td->tijq", Bm.astype(np.float64), wl.hidden_q.astype(np.float64)))
+    mags = dict(dh=np.einsum("tib,ibd->td", gs, aW) + np.einsum("tijq,ijqd->td", gy, aB) + ds @ np.abs(wl.W_sum_q.astype(np.float64)),
+                dW_base=np.einsum("tib,td->ibd", gs, ah), dB=np.einsum("tijq,td->ijqd", gy, ah),
+                dA=np.einsum("tijb,tijq->ijbq", g, z), dW_sum=ds.T @ ah)
+    floor = 2e-5 * float(np.abs(weight).max()) * max(1.0, T ** 0.5)
+    refs = dict(dh=ref["dh"], dW_base=lr["dW_base"], dA=lr["dA"], dB=lr["dB"], dW_sum=ref["dW_sum"])
+    used = {name: _check_tensor(name, out[name], refs[name], mags[name], floor) for name in refs}
+    if fam == I.HMM and n > 1:
+        got = out["dT"][: n - 1].cpu().numpy().astype(np.float64)
+        assert np.abs(got - ref["dT_static"]).max() <= 1e-2 * np.abs(ref["dT_static"]).max() + floor
+    print(f"{wl.name}: share of the entry-wise bound used / relative L2: " + ", ".join(f"{n_} {u:.2f} / {l:.1e}" for n_, (u, l) in used.items()))
+    # the padding rows of dA and dW_base receive no gradient
+    if vv:
+        assert float(out["dA"][:, :, vv:].abs().max()) <= floor and float(out["dW_base"][:, vv:].abs().max()) <= floor
+    # the forward entry point still gives the same value
+    fwd = torch.empty(T, **f32)
+    head.mtpc_window_logprob(hidden, torch.from_numpy(t).cuda(), fwd)
+    assert torch.equal(fwd, out["logprob"])
+    head.mtpc_destroy()
