@@ -353,7 +353,54 @@ def measure_lowrank(torch, wl, dW_emit, steps: int, peaks, k: int = 16):
     if wl.shape.io_dtype == I.BF16 and s.v % 16 == 0:
         out["factored_forward"] = measure_factored_forward(torch, wl, (Wb, A, Bm), steps)
         out["factored_draft"] = measure_factored_draft(torch, wl, (Wb, A, Bm), peaks)
+        out["factored_backward"] = measure_factored_backward(torch, wl, (Wb, A, Bm), steps)
     return out
+
+
+def measure_factored_backward(torch, wl, lowrank, steps: int):
+    """mtpc_lowrank_window_logprob_backward: the training call of a head that keeps the shared unembeddings factored
+    (value + gradients with respect to the hidden states, W_base, A, B and the sum-unit weights), per call and per phase."""
+    from paper_2511_11346_b200 import binding as B
+    from paper_2511_11346_b200.runner import to_device_bf16
+    s = wl.shape
+    k = lowrank[1].shape[-1]
+    ctx = s.family == I.HMM_CTX
+    W_sum = to_device_bf16(wl.W_sum_q)
+    Ts = torch.from_numpy(np.ascontiguousarray(wl.T_static)).cuda() if wl.T_static is not None else None
+    head = B.MtpcHead(B.MTPC_HMM if ctx else s.family, s.n, s.r, s.v, s.d, B.MTPC_BF16, wl.T, 1, None, W_sum, Ts,
+                      flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0, v_valid=s.v_valid, lowrank=lowrank)
+    hidden = to_device_bf16(wl.hidden_q)
+    targets = torch.from_numpy(wl.targets).cuda()
+    f32 = dict(dtype=torch.float32, device="cuda")
+    weight = torch.full((wl.T,), -1.0 / wl.T, **f32)
+    out = [torch.empty(wl.T, **f32), torch.empty((wl.T, s.d), **f32), torch.empty((s.n, s.v, s.d), **f32),
+           torch.empty((s.n, s.r, s.v, k), **f32), torch.empty((s.n, s.r, k, s.d), **f32), torch.empty((s.sum_rows, s.d), **f32),
+           torch.empty((max(s.n - 1, 1), s.r, s.r), **f32) if s.family == I.HMM else None]
+    call = lambda: head.mtpc_lowrank_window_logprob_backward(hidden, targets, weight, *out)
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    fwd = torch.empty(wl.T, **f32)
+    head.mtpc_window_logprob(hidden, targets, fwd)
+    same_value = bool(torch.equal(fwd, out[0]))
+    head.mtpc_set_timing(steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    phases = [head.mtpc_get_timing(i) for i in range(steps)]
+    phase_ms = [statistics.mean(p[q] for p in phases) for q in range(len(phases[0]))]
+    head.mtpc_set_timing(0)
+    status = head.mtpc_get_status()
+    head.mtpc_destroy()
+    return {"call": "mtpc_lowrank_window_logprob_backward", "ms_per_call": ms, "phase_ms": phase_ms,
+            "phases": "factored forward keeping the logits, circuit backward, logit gradients + their sums + operand "
+                      "copies, GEMMs (g A, d hidden, dW_base, dB, dW_sum, dA)",
+            "value_equals_forward_call": same_value, "device_status": status,
+            "note": "the route through the composed tensor costs compose_ms + the dense backward call + backward_ms"}
 
 
 def measure_factored_draft(torch, wl, lowrank, peaks, P: int = 8, wpp: int = 16, calls: int = 200):
