@@ -298,7 +298,7 @@ int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k,
  * Such a head serves mtpc_window_logprob, mtpc_window_prefix_logprob, mtpc_window_loss, mtpc_window_logprob_host, and,
  * for up to 128 positions per call, mtpc_draft_sample, mtpc_draft_sample_prefix and mtpc_speculative_accept: the draft's
  * weight pass then streams W_base and B (n v + n r k rows) instead of n r v composed rows, and the logits are formed
- * from the two small products. Its training call is mtpc_lowrank_window_logprob_backward (below). Drafts of more than
+ * from the two small products. Its training calls are mtpc_lowrank_window_logprob_backward and mtpc_lowrank_window_loss_backward (below). Drafts of more than
  * 128 positions, mtpc_window_logprob_backward and mtpc_window_loss_backward return MTPC_ERR_UNSUPPORTED on it: those run
  * on the composed tensor (mtpc_lowrank_compose + mtpc_create_head, gradients carried back by mtpc_lowrank_backward).
  */
@@ -322,6 +322,15 @@ int mtpc_lowrank_window_logprob_backward(mtpc_head* head, const void* hidden, co
                                          const float* weight, void* bwd_workspace, size_t bwd_workspace_bytes,
                                          float* out_logprob, float* d_hidden, float* dW_base, float* dA, float* dB,
                                          float* dW_sum, float* dT_static, void* stream);
+/*
+ * The training loss of Eq. 6 and its gradients on a factored head: arguments as mtpc_window_loss_backward, with dW_base, dA,
+ * dB (as above) in place of dW_emit; the same workspace size as mtpc_lowrank_window_logprob_backward for
+ * T = num_sequences * sequence_length.
+ */
+int mtpc_lowrank_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,
+                                      int32_t sequence_length, float gamma, void* bwd_workspace, size_t bwd_workspace_bytes,
+                                      float* out_slot_loss, float* out_loss, float* d_hidden, float* dW_base, float* dA,
+                                      float* dB, float* dW_sum, float* dT_static, void* stream);
 int mtpc_create_head_lowrank(const mtpc_config* cfg, int32_t k, const void* W_base, const void* A, const void* B,
                              const void* W_sum, const float* T_static, void* workspace, size_t workspace_bytes,
                              void* stream, mtpc_head** out);

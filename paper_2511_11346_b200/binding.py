@@ -26,6 +26,7 @@ EXPORTS = [
     "mtpc_lowrank_compose", "mtpc_lowrank_backward", "mtpc_update_parameters", "mtpc_debug_set_wait_limit_ns",
     "mtpc_debug_set_projection_variant", "mtpc_debug_set_draft_grouping", "mtpc_lowrank_workspace_bytes",
     "mtpc_create_head_lowrank", "mtpc_lowrank_backward_workspace_bytes", "mtpc_lowrank_window_logprob_backward",
+    "mtpc_lowrank_window_loss_backward",
 ]
 STATIC_SCRATCH_BYTES = 16 << 20
 ERR_STATIC_SCRATCH = -7
@@ -86,6 +87,8 @@ def lib() -> ctypes.CDLL:
     L.mtpc_lowrank_workspace_bytes.argtypes = [ctypes.POINTER(MtpcConfig), i32, ctypes.POINTER(sz)]
     L.mtpc_lowrank_backward_workspace_bytes.argtypes = [ctypes.POINTER(MtpcConfig), i32, i32, ctypes.POINTER(sz)]
     L.mtpc_lowrank_window_logprob_backward.argtypes = [vp, vp, vp, i32, vp, vp, sz, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.mtpc_lowrank_window_loss_backward.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp, sz, vp, vp, vp, vp, vp, vp, vp,
+                                                    vp, vp]
     L.mtpc_create_head_lowrank.argtypes = [ctypes.POINTER(MtpcConfig), i32, vp, vp, vp, vp, vp, vp, sz, vp, ctypes.POINTER(vp)]
     L.mtpc_status_string.argtypes = [ctypes.c_int]
     L.mtpc_status_string.restype = ctypes.c_char_p
@@ -237,18 +240,32 @@ class MtpcHead:
                                                   ws.numel(), _ptr(out_logprob), _ptr(d_hidden), _ptr(dW_emit), _ptr(dW_sum),
                                                   _ptr(dT_static), _stream(stream)), "mtpc_window_logprob_backward")
 
-    def mtpc_lowrank_window_logprob_backward(self, hidden, targets, weight, out_logprob, d_hidden, dW_base, dA, dB, dW_sum,
-                                             dT_static=None, stream=None) -> None:
-        """Training call of a factored head: gradients with respect to W_base, A and B; workspace allocated here (torch)."""
+    def _lowrank_backward_workspace(self, T: int, k: int, device):
         import torch
-        T = hidden.shape[0]
-        k = dA.shape[-1]
         need = ctypes.c_size_t(0)
         _check(lib().mtpc_lowrank_backward_workspace_bytes(ctypes.byref(self.cfg), k, T, ctypes.byref(need)),
                "mtpc_lowrank_backward_workspace_bytes")
         ws = getattr(self, "_bwd_ws", None)
         if ws is None or ws.numel() < need.value:
-            ws = self._bwd_ws = torch.empty(need.value, dtype=torch.uint8, device=hidden.device)
+            ws = self._bwd_ws = torch.empty(need.value, dtype=torch.uint8, device=device)
+        return ws
+
+    def mtpc_lowrank_window_loss_backward(self, hidden, targets, num_sequences: int, sequence_length: int, gamma: float,
+                                          out_slot_loss, out_loss, d_hidden, dW_base, dA, dB, dW_sum, dT_static=None,
+                                          stream=None) -> None:
+        """Eq. 6 loss and its gradients on a factored head; workspace allocated here (torch)."""
+        ws = self._lowrank_backward_workspace(hidden.shape[0], dA.shape[-1], hidden.device)
+        _check(lib().mtpc_lowrank_window_loss_backward(self.handle, _ptr(hidden), _ptr(targets), num_sequences, sequence_length,
+                                                       ctypes.c_float(gamma), ws.data_ptr(), ws.numel(), _ptr(out_slot_loss),
+                                                       _ptr(out_loss), _ptr(d_hidden), _ptr(dW_base), _ptr(dA), _ptr(dB),
+                                                       _ptr(dW_sum), _ptr(dT_static), _stream(stream)),
+               "mtpc_lowrank_window_loss_backward")
+
+    def mtpc_lowrank_window_logprob_backward(self, hidden, targets, weight, out_logprob, d_hidden, dW_base, dA, dB, dW_sum,
+                                             dT_static=None, stream=None) -> None:
+        """Training call of a factored head: gradients with respect to W_base, A and B; workspace allocated here (torch)."""
+        T = hidden.shape[0]
+        ws = self._lowrank_backward_workspace(T, dA.shape[-1], hidden.device)
         _check(lib().mtpc_lowrank_window_logprob_backward(self.handle, _ptr(hidden), _ptr(targets), T, _ptr(weight),
                                                           ws.data_ptr(), ws.numel(), _ptr(out_logprob), _ptr(d_hidden),
                                                           _ptr(dW_base), _ptr(dA), _ptr(dB), _ptr(dW_sum), _ptr(dT_static),

@@ -1149,6 +1149,96 @@ void plan_lowrank_backward(const mtpc_config& c, const Layout& L, int k, int T, 
   R->total = off;
 }
 
+// Phases 3 and 4 of a training call on a factored head: logit gradients g [T, n r v] (bf16), their sum over a slot's
+// components, the zero-padded A, W_base and B in a row; then the GEMMs. The sum units' logit gradients are already in the
+// right-hand columns of sy.
+int lowrank_backward_tail(mtpc_head* head, const LowRankBackwardLayout& R, uint8_t* bw, const void* hb, const int32_t* targets,
+                          int T, float* d_hidden, float* dW_base, float* dA, float* dB, float* dW_sum, PhaseTimer& pt,
+                          cudaStream_t st) {
+  const mtpc_config& c = head->cfg;
+  const Layout& L = head->L;
+  const BackwardLayout& B = R.B;
+  const int k = head->lr_k, units = c.n * c.r;
+  __nv_bfloat16* sy = reinterpret_cast<__nv_bfloat16*>(bw + R.off_sy);
+  int rc = MTPC_OK;
+  pt.begin();
+  __nv_bfloat16* dlogit = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit);
+  const int Nc = static_cast<int>(B.Nc);
+  LogitGradArgs la;
+  la.logits = reinterpret_cast<const float*>(bw + B.off_logits);
+  la.lse = reinterpret_cast<const float*>(bw + B.off_lse);
+  la.post = reinterpret_cast<const float*>(bw + B.off_post);
+  la.targets = targets;
+  la.dlogit = dlogit;
+  la.pitch = B.Kd;
+  la.T = T; la.Nc = Nc; la.n = c.n; la.r = c.r; la.v = c.v;
+  {
+    const int col_blocks = (Nc / 8 + 255) / 256;
+    int row_blocks = (16 * head->num_sms + col_blocks - 1) / col_blocks;
+    if (row_blocks > T) row_blocks = T;
+    if (row_blocks > 65535) row_blocks = 65535;
+    logit_gradient_kernel<<<dim3(col_blocks, row_blocks), 256, 0, st>>>(la);
+  }
+  {
+    const size_t pieces = static_cast<size_t>(T) * (c.n * c.v / 8);
+    lowrank_component_sum_kernel<<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, st>>>(dlogit, B.Kd, sy, R.pitch, T,
+                                                                                               c.n, c.r, c.v);
+    const size_t pad_pieces = static_cast<size_t>(units) * R.v64 * (k / 8);
+    lowrank_pad_kernel<<<static_cast<unsigned>((pad_pieces + 255) / 256), 256, 0, st>>>(
+        static_cast<const uint4*>(head->lr_A), reinterpret_cast<uint4*>(bw + R.off_apad), units, c.v, static_cast<int>(R.v64), k / 8);
+  }
+  head->launches += 3;
+  uint8_t* wcat = bw + R.off_wcat;
+  const size_t base_bytes = static_cast<size_t>(c.n) * c.v * c.d * 2;
+  bool fail = cudaMemcpyAsync(wcat, head->lr_W_base, base_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess;
+  fail |= cudaMemcpyAsync(wcat + base_bytes, head->lr_B, static_cast<size_t>(units) * k * c.d * 2, cudaMemcpyDeviceToDevice, st) != cudaSuccess;
+  if (fail || (rc = check_launch()) != MTPC_OK) return MTPC_ERR_CUDA;
+  pt.end();
+  // 4. the GEMMs
+  pt.begin();
+  const GemmOperand none{nullptr, 0, false};
+  const GemmOperand hid{hb, static_cast<size_t>(c.d), true};
+  {   // y_ij = g_ij A_ij [T, k], one product per unit, into the middle columns of sy
+    PlainGemmExtra x;
+    x.C_bf16 = sy + static_cast<size_t>(c.n) * c.v;
+    x.batches = units;
+    x.a_k_step = c.v;
+    x.b_k_step = static_cast<int>(R.v64);
+    x.c_step = k;
+    x.a_extent_m = T; x.a_extent_k = Nc;
+    x.b_extent_n = k; x.b_extent_k = static_cast<long long>(units) * R.v64;
+    rc = launch_plain_gemm(head, GemmOperand{dlogit, B.Kd, false}, GemmOperand{bw + R.off_apad, static_cast<size_t>(k), true},
+                           static_cast<int>(R.v64), none, 0, 0, nullptr, R.pitch, T, k, st, nullptr, 0, &x);
+  }
+  // d hidden [T, d] = [s | y] [W_base ; B] + dsum W_sum
+  if (rc == MTPC_OK)
+    rc = launch_plain_gemm(head, GemmOperand{sy, R.pitch, false}, GemmOperand{wcat, static_cast<size_t>(c.d), true},
+                           static_cast<int>(R.Ksy), GemmOperand{head->W_sum_bf16, static_cast<size_t>(c.d), true}, L.sum_rows,
+                           static_cast<int>(R.Ksy), d_hidden, c.d, T, c.d, st);
+  // dW_base = s^T h, dB = y^T h, dW_sum = dsum^T h: sy down its columns
+  if (rc == MTPC_OK)
+    rc = launch_plain_gemm(head, GemmOperand{sy, R.pitch, true}, hid, T, hid, 0, 0, dW_base, c.d, c.n * c.v, c.d, st);
+  if (rc == MTPC_OK)
+    rc = launch_plain_gemm(head, GemmOperand{sy + static_cast<size_t>(c.n) * c.v, R.pitch, true}, hid, T, hid, 0, 0, dB, c.d,
+                           units * k, c.d, st);
+  if (rc == MTPC_OK)
+    rc = launch_plain_gemm(head, GemmOperand{sy + R.Ksy, R.pitch, true}, hid, T, hid, 0, 0, dW_sum, c.d, L.sum_rows, c.d, st);
+  if (rc == MTPC_OK) {   // dA_ij [v, k] = g_ij^T z_ij, one product per unit, on the bf16 high half of z the forward pass left
+    PlainGemmExtra x;
+    x.batches = units;
+    x.a_m_step = c.v;
+    x.b_n_step = 2 * k;
+    x.c_step = static_cast<size_t>(c.v) * k;
+    x.a_extent_m = Nc; x.a_extent_k = T;
+    x.b_extent_n = static_cast<long long>(units) * 2 * k; x.b_extent_k = T;
+    rc = launch_plain_gemm(head, GemmOperand{dlogit, B.Kd, true},
+                           GemmOperand{head->ws + head->lr_off_zhl, static_cast<size_t>(units) * 2 * k, true}, T, none, 0, 0, dA,
+                           k, c.v, k, st, nullptr, 0, &x);
+  }
+  pt.end();
+  return rc;
+}
+
 int check_call(mtpc_head* h, int32_t rows) {
   if (!h) return MTPC_ERR_NULL;
   if (rows < 0 || rows > h->cfg.max_positions) return MTPC_ERR_SHAPE;
@@ -1626,7 +1716,7 @@ int mtpc_lowrank_window_logprob_backward(mtpc_head* head, const void* hidden, co
   if (head->lr_k == 0) return MTPC_ERR_STATE;                  // a head on a composed tensor: mtpc_window_logprob_backward
   const mtpc_config& c = head->cfg;
   const Layout& L = head->L;
-  const int k = head->lr_k, units = c.n * c.r;
+  const int k = head->lr_k;
   const bool static_hmm = c.family == MTPC_HMM && !is_ctx(head) && c.n > 1;
   if (static_hmm && !dT_static) return MTPC_ERR_NULL;
   LowRankBackwardLayout R;
@@ -1667,104 +1757,36 @@ int mtpc_lowrank_window_logprob_backward(mtpc_head* head, const void* hidden, co
   rc = launch_circuit_backward(head, a, dT_static, st);
   pt.end();
   if (rc != MTPC_OK) return rc;
-  // 3. logit gradients g [T, n r v] (bf16), their sum over a slot's components, the zero-padded A, W_base and B in a row
-  pt.begin();
-  __nv_bfloat16* dlogit = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit);
-  const int Nc = static_cast<int>(B.Nc);
-  LogitGradArgs la;
-  la.logits = reinterpret_cast<const float*>(bw + B.off_logits);
-  la.lse = reinterpret_cast<const float*>(bw + B.off_lse);
-  la.post = reinterpret_cast<const float*>(bw + B.off_post);
-  la.targets = targets;
-  la.dlogit = dlogit;
-  la.pitch = B.Kd;
-  la.T = T; la.Nc = Nc; la.n = c.n; la.r = c.r; la.v = c.v;
-  {
-    const int col_blocks = (Nc / 8 + 255) / 256;
-    int row_blocks = (16 * head->num_sms + col_blocks - 1) / col_blocks;
-    if (row_blocks > T) row_blocks = T;
-    if (row_blocks > 65535) row_blocks = 65535;
-    logit_gradient_kernel<<<dim3(col_blocks, row_blocks), 256, 0, st>>>(la);
-  }
-  {
-    const size_t pieces = static_cast<size_t>(T) * (c.n * c.v / 8);
-    lowrank_component_sum_kernel<<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, st>>>(dlogit, B.Kd, sy, R.pitch, T,
-                                                                                               c.n, c.r, c.v);
-    const size_t pad_pieces = static_cast<size_t>(units) * R.v64 * (k / 8);
-    lowrank_pad_kernel<<<static_cast<unsigned>((pad_pieces + 255) / 256), 256, 0, st>>>(
-        static_cast<const uint4*>(head->lr_A), reinterpret_cast<uint4*>(bw + R.off_apad), units, c.v, static_cast<int>(R.v64), k / 8);
-  }
-  head->launches += 3;
-  uint8_t* wcat = bw + R.off_wcat;
-  const size_t base_bytes = static_cast<size_t>(c.n) * c.v * c.d * 2;
-  bool fail = cudaMemcpyAsync(wcat, head->lr_W_base, base_bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess;
-  fail |= cudaMemcpyAsync(wcat + base_bytes, head->lr_B, static_cast<size_t>(units) * k * c.d * 2, cudaMemcpyDeviceToDevice, st) != cudaSuccess;
-  if (fail || (rc = check_launch()) != MTPC_OK) return MTPC_ERR_CUDA;
-  pt.end();
-  // 4. the GEMMs
-  pt.begin();
-  const GemmOperand none{nullptr, 0, false};
-  const GemmOperand hid{hb, static_cast<size_t>(c.d), true};
-  {   // y_ij = g_ij A_ij [T, k], one product per unit, into the middle columns of sy
-    PlainGemmExtra x;
-    x.C_bf16 = sy + static_cast<size_t>(c.n) * c.v;
-    x.batches = units;
-    x.a_k_step = c.v;
-    x.b_k_step = static_cast<int>(R.v64);
-    x.c_step = k;
-    x.a_extent_m = T; x.a_extent_k = Nc;
-    x.b_extent_n = k; x.b_extent_k = static_cast<long long>(units) * R.v64;
-    rc = launch_plain_gemm(head, GemmOperand{dlogit, B.Kd, false}, GemmOperand{bw + R.off_apad, static_cast<size_t>(k), true},
-                           static_cast<int>(R.v64), none, 0, 0, nullptr, R.pitch, T, k, st, nullptr, 0, &x);
-  }
-  // d hidden [T, d] = [s | y] [W_base ; B] + dsum W_sum
-  if (rc == MTPC_OK)
-    rc = launch_plain_gemm(head, GemmOperand{sy, R.pitch, false}, GemmOperand{wcat, static_cast<size_t>(c.d), true},
-                           static_cast<int>(R.Ksy), GemmOperand{head->W_sum_bf16, static_cast<size_t>(c.d), true}, L.sum_rows,
-                           static_cast<int>(R.Ksy), d_hidden, c.d, T, c.d, st);
-  // dW_base = s^T h, dB = y^T h, dW_sum = dsum^T h: sy down its columns
-  if (rc == MTPC_OK)
-    rc = launch_plain_gemm(head, GemmOperand{sy, R.pitch, true}, hid, T, hid, 0, 0, dW_base, c.d, c.n * c.v, c.d, st);
-  if (rc == MTPC_OK)
-    rc = launch_plain_gemm(head, GemmOperand{sy + static_cast<size_t>(c.n) * c.v, R.pitch, true}, hid, T, hid, 0, 0, dB, c.d,
-                           units * k, c.d, st);
-  if (rc == MTPC_OK)
-    rc = launch_plain_gemm(head, GemmOperand{sy + R.Ksy, R.pitch, true}, hid, T, hid, 0, 0, dW_sum, c.d, L.sum_rows, c.d, st);
-  if (rc == MTPC_OK) {   // dA_ij [v, k] = g_ij^T z_ij, one product per unit, on the bf16 high half of z the forward pass left
-    PlainGemmExtra x;
-    x.batches = units;
-    x.a_m_step = c.v;
-    x.b_n_step = 2 * k;
-    x.c_step = static_cast<size_t>(c.v) * k;
-    x.a_extent_m = Nc; x.a_extent_k = T;
-    x.b_extent_n = static_cast<long long>(units) * 2 * k; x.b_extent_k = T;
-    rc = launch_plain_gemm(head, GemmOperand{dlogit, B.Kd, true},
-                           GemmOperand{head->ws + head->lr_off_zhl, static_cast<size_t>(units) * 2 * k, true}, T, none, 0, 0, dA,
-                           k, c.v, k, st, nullptr, 0, &x);
-  }
-  pt.end();
-  return rc;
+  // 3., 4. logit gradients and what is derived from them, then the GEMMs
+  return lowrank_backward_tail(head, R, bw, hb, targets, T, d_hidden, dW_base, dA, dB, dW_sum, pt, st);
 }
 
-int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,
-                              int32_t sequence_length, float gamma, void* bwd_workspace, size_t bwd_workspace_bytes,
-                              float* out_slot_loss, float* out_loss, float* d_hidden, float* dW_emit, float* dW_sum,
-                              float* dT_static, void* stream) {
+}  // extern "C"
+
+// Eq. 6 loss and its gradients, on a head built on a composed tensor (dW_emit) or on a factored one (dW_base, dA, dB): the
+// two differ in the projection that keeps the logits and in the GEMMs at the end.
+static int window_loss_backward_impl(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,
+                                     int32_t sequence_length, float gamma, void* bwd_workspace, size_t bwd_workspace_bytes,
+                                     float* out_slot_loss, float* out_loss, float* d_hidden, float* dW_emit, float* dW_base,
+                                     float* dA, float* dB, float* dW_sum, float* dT_static, void* stream) {
   if (!head) return MTPC_ERR_NULL;
   if (num_sequences < 1 || sequence_length < 1) return MTPC_ERR_SHAPE;
   const int64_t T64 = static_cast<int64_t>(num_sequences) * sequence_length;
   if (T64 > head->cfg.max_positions) return MTPC_ERR_SHAPE;
-  if (!hidden || !targets || !bwd_workspace || !out_slot_loss || !out_loss || !d_hidden || !dW_emit || !dW_sum)
-    return MTPC_ERR_NULL;
-  if (head->lr_k > 0) return MTPC_ERR_UNSUPPORTED;
+  if (!hidden || !targets || !bwd_workspace || !out_slot_loss || !out_loss || !d_hidden || !dW_sum) return MTPC_ERR_NULL;
+  const bool factored = head->lr_k > 0;
+  if (factored ? (!dW_base || !dA || !dB) : !dW_emit) return MTPC_ERR_NULL;
   const int T = static_cast<int>(T64);
   const mtpc_config& c = head->cfg;
   const Layout& L = head->L;
   const bool static_hmm = c.family == MTPC_HMM && !is_ctx(head) && c.n > 1;
   if (static_hmm && !dT_static) return MTPC_ERR_NULL;
-  BackwardLayout B;
-  plan_backward(c, L, T, &B);
-  if (bwd_workspace_bytes < B.total || (reinterpret_cast<uintptr_t>(bwd_workspace) % kAlign) != 0)
+  LowRankBackwardLayout R;
+  memset(&R, 0, sizeof(R));
+  if (factored) plan_lowrank_backward(c, L, head->lr_k, T, &R);
+  else plan_backward(c, L, T, &R.B);
+  const BackwardLayout& B = R.B;
+  if (bwd_workspace_bytes < (factored ? R.total : B.total) || (reinterpret_cast<uintptr_t>(bwd_workspace) % kAlign) != 0)
     return MTPC_ERR_WORKSPACE;
   int rc = set_backward_attributes(head);
   if (rc != MTPC_OK) return rc;
@@ -1786,9 +1808,14 @@ int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t
   fwd.lse_out = reinterpret_cast<float*>(bw + B.off_lse);
   fwd.logit_out = reinterpret_cast<float*>(bw + B.off_logits);
   fwd.logit_pitch = B.Nc;
-  rc = launch_gemm(head, kModeLogprob, hb, T, 1, true, true, targets, nullptr, nullptr, st, &fwd);
+  rc = factored ? launch_lowrank_projection(head, hb, T, targets, st, &fwd)
+                : launch_gemm(head, kModeLogprob, hb, T, 1, true, true, targets, nullptr, nullptr, st, &fwd);
   if (rc == MTPC_OK) rc = launch_circuit(head, T, 1, nullptr, prefix, st);
   if (rc != MTPC_OK) return rc;
+  // the sum units' logit gradients (bf16): to the right of dlogit, or of [s | y] on a factored head
+  __nv_bfloat16* dsum_bf16 = factored ? reinterpret_cast<__nv_bfloat16*>(bw + R.off_sy) + R.Ksy
+                                      : reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit) + B.Nc;
+  const size_t dsum_bf16_pitch = factored ? R.pitch : B.Kd;
   loss_partial_kernel<<<num_sequences, kLossThreads, 0, st>>>(prefix, targets, partial, sequence_length, c.n);
   loss_final_kernel<<<1, kLossThreads, 0, st>>>(partial, out_slot_loss, out_loss, num_sequences, c.n, gamma);
   loss_coeff_kernel<<<num_sequences, kLossThreads, 0, st>>>(targets, coeff, sequence_length, c.n, num_sequences, gamma);
@@ -1805,8 +1832,8 @@ int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t
     memset(&a, 0, sizeof(a));
     a.targets = targets;
     a.post = post;
-    a.dsum = reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit) + B.Nc;    // columns [Nc, Nc + S r) of the dlogit rows
-    a.dsum_pitch = static_cast<int>(B.Kd);
+    a.dsum = dsum_bf16;
+    a.dsum_pitch = static_cast<int>(dsum_bf16_pitch);
     a.len = c.n;
     a.W = T;
     if ((rc = launch_circuit_backward(head, a, dT_static, st, coeff)) != MTPC_OK) return rc;
@@ -1835,13 +1862,35 @@ int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t
     }
     const size_t total = static_cast<size_t>(T) * L.sum_rows;
     const int blocks = static_cast<int>((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
-    f32_rows_to_bf16_kernel<<<blocks, 256, 0, st>>>(dsum_f32, reinterpret_cast<__nv_bfloat16*>(bw + B.off_dlogit) + B.Nc, T,
-                                                    L.sum_rows, L.sum_rows, B.Kd);
+    f32_rows_to_bf16_kernel<<<blocks, 256, 0, st>>>(dsum_f32, dsum_bf16, T, L.sum_rows, L.sum_rows, dsum_bf16_pitch);
     head->launches++;
   }
   pt.end();
   if ((rc = check_launch()) != MTPC_OK) return rc;
+  if (factored) return lowrank_backward_tail(head, R, bw, hb, targets, T, d_hidden, dW_base, dA, dB, dW_sum, pt, st);
   return backward_tail(head, B, bw, hb, targets, T, d_hidden, dW_emit, dW_sum, pt, st);
+}
+
+extern "C" {
+
+int mtpc_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,
+                              int32_t sequence_length, float gamma, void* bwd_workspace, size_t bwd_workspace_bytes,
+                              float* out_slot_loss, float* out_loss, float* d_hidden, float* dW_emit, float* dW_sum,
+                              float* dT_static, void* stream) {
+  if (head && head->lr_k > 0) return MTPC_ERR_UNSUPPORTED;     // a factored head: mtpc_lowrank_window_loss_backward
+  return window_loss_backward_impl(head, hidden, targets, num_sequences, sequence_length, gamma, bwd_workspace,
+                                   bwd_workspace_bytes, out_slot_loss, out_loss, d_hidden, dW_emit, nullptr, nullptr, nullptr,
+                                   dW_sum, dT_static, stream);
+}
+
+int mtpc_lowrank_window_loss_backward(mtpc_head* head, const void* hidden, const int32_t* targets, int32_t num_sequences,
+                                      int32_t sequence_length, float gamma, void* bwd_workspace, size_t bwd_workspace_bytes,
+                                      float* out_slot_loss, float* out_loss, float* d_hidden, float* dW_base, float* dA,
+                                      float* dB, float* dW_sum, float* dT_static, void* stream) {
+  if (head && head->lr_k == 0) return MTPC_ERR_STATE;          // a head on a composed tensor: mtpc_window_loss_backward
+  return window_loss_backward_impl(head, hidden, targets, num_sequences, sequence_length, gamma, bwd_workspace,
+                                   bwd_workspace_bytes, out_slot_loss, out_loss, d_hidden, nullptr, dW_base, dA, dB, dW_sum,
+                                   dT_static, stream);
 }
 
 // Streams and events of the chunked host-buffer path; no device memory is allocated.

@@ -341,3 +341,68 @@ def test_factored_backward_is_the_chain_rule_through_the_composition(family, n, 
     head.mtpc_window_logprob(hidden, torch.from_numpy(t).cuda(), fwd)
     assert torch.equal(fwd, out["logprob"])
     head.mtpc_destroy()
+
+
+def _whole_tensor(name, got, ref, floor):
+    """Largest error below 1e-2 of the tensor's largest magnitude, relative L2 error below 1e-2 (two bf16-rounded factors
+    per product)."""
+    got = got.cpu().numpy().astype(np.float64).reshape(ref.shape)
+    assert np.isfinite(got).all(), name
+    scale = np.abs(ref).max()
+    err = np.abs(got - ref).max()
+    rel2 = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    assert err <= 1e-2 * scale + floor, f"{name}: max error {err} against scale {scale}"
+    assert rel2 <= 1e-2 or scale < 100 * floor, f"{name}: relative L2 error {rel2}"
+    return err / max(scale, 1e-30), rel2
+
+
+@pytest.mark.parametrize("family,n,r,v,d,k,N,L", [(I.CP, 4, 8, 320, 128, 16, 3, 50), (I.HMM, 8, 16, 64, 64, 16, 5, 33),
+                                                   (I.HMM_CTX, 4, 8, 64, 64, 32, 4, 40), (I.BTREE, 8, 8, 32, 64, 16, 2, 140),
+                                                   (I.HMM, 1, 4, 32, 64, 16, 2, 9)])
+def test_eq6_loss_backward_on_a_factored_head(family, n, r, v, d, k, N, L):
+    """The training loss of Eq. 6 and its gradients with respect to W_base, A and B, against reverse-mode differentiation of
+    the definition on the exactly composed tensor, carried through U = W + A B. Windows run past the end of their sequences."""
+    T = N * L
+    wl, W, A, Bm = _factored_case(family, n, r, v, 0, d, k, T, seed=6400 + n + N + r)
+    fam = wl.shape.family
+    U = O.lowrank_unembedding(W, A, Bm)
+    t = wl.targets.copy().reshape(N, L, n)
+    for j in range(1, n):
+        t[:, max(L - j, 0):, j] = -1
+    if n > 1:
+        t[0, :, n - 1] = -1
+    t = t.reshape(T, n)
+    gamma = 0.8
+    ref = OG.composite_loss_grad(fam, wl.hidden_q, U, wl.W_sum_q, wl.T_static, t, N, gamma)
+    lr = OG.lowrank_grad(W, A, Bm, ref["dW_emit"])
+    ctx = family == I.HMM_CTX
+    Ts = torch.from_numpy(np.ascontiguousarray(wl.T_static)).cuda() if wl.T_static is not None else None
+    head = B.MtpcHead(B.MTPC_HMM if ctx else family, n, r, v, d, B.MTPC_BF16, T, 1, None, to_device_bf16(wl.W_sum_q), Ts,
+                      flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0, lowrank=(_device(W), _device(A), _device(Bm)))
+    f32 = dict(dtype=torch.float32, device="cuda")
+    S = wl.W_sum_q.shape[0]
+    slot, loss = torch.empty(n, **f32), torch.empty(1, **f32)
+    out = dict(dh=torch.empty((T, d), **f32), dW_base=torch.empty((n, v, d), **f32), dA=torch.empty((n, r, v, k), **f32),
+               dB=torch.empty((n, r, k, d), **f32), dW_sum=torch.empty((S, d), **f32))
+    dT = torch.empty((max(n - 1, 1), r, r), **f32) if fam == I.HMM else None
+    hidden = to_device_bf16(wl.hidden_q)
+    td = torch.from_numpy(t).cuda()
+    head.mtpc_lowrank_window_loss_backward(hidden, td, N, L, gamma, slot, loss, out["dh"], out["dW_base"], out["dA"], out["dB"],
+                                           out["dW_sum"], dT)
+    assert head.mtpc_get_status() == 0
+    assert np.abs(slot.cpu().numpy() - ref["slot_loss"]).max() <= 2e-3
+    assert abs(float(loss.cpu()[0]) - ref["loss"]) <= 2e-3 * n
+    floor = 2e-5 / N * max(1.0, L ** 0.5)
+    refs = dict(dh=ref["dh"], dW_base=lr["dW_base"], dA=lr["dA"], dB=lr["dB"], dW_sum=ref["dW_sum"])
+    stats = {name: _whole_tensor(name, out[name], refs[name], floor) for name in refs}
+    if fam == I.HMM and n > 1:
+        stats["dT_static"] = _whole_tensor("dT_static", dT[: n - 1], ref["dT_static"], floor)
+    print(f"{wl.name}: (max error / scale, relative L2): " + ", ".join(f"{n_} ({a:.1e}, {b:.1e})" for n_, (a, b) in stats.items()))
+    # the forward-only entry point gives the same loss; the composed-tensor entry point refuses a factored head
+    slot2, loss2 = torch.empty(n, **f32), torch.empty(1, **f32)
+    head.mtpc_window_loss(hidden, td, N, L, gamma, slot2, loss2)
+    assert torch.equal(slot, slot2) and torch.equal(loss, loss2)
+    with pytest.raises(B.MtpcError) as e:
+        head.mtpc_window_loss_backward(hidden, td, N, L, gamma, slot, loss, out["dh"], torch.empty((n, r, v, d), **f32), out["dW_sum"], dT)
+    assert e.value.code == -3
+    head.mtpc_destroy()
