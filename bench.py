@@ -394,9 +394,29 @@ def measure_factored_backward(torch, wl, lowrank, steps: int):
     phases = [head.mtpc_get_timing(i) for i in range(steps)]
     phase_ms = [statistics.mean(p[q] for p in phases) for q in range(len(phases[0]))]
     head.mtpc_set_timing(0)
+    # the paper's training loss (Eq. 6): sequences of 1024 positions, windows past the end of a sequence masked
+    L = 1024 if wl.T % 1024 == 0 else wl.T
+    N = wl.T // L
+    t6 = targets.clone().view(N, L, s.n)
+    for j in range(1, s.n):
+        t6[:, L - j:, j] = -1
+    t6 = t6.view(wl.T, s.n).contiguous()
+    gamma = 0.8 if s.n <= 8 else 0.9
+    slot, loss = torch.empty(s.n, **f32), torch.empty(1, **f32)
+    call6 = lambda: head.mtpc_lowrank_window_loss_backward(hidden, t6, N, L, gamma, slot, loss, *out[1:])
+    for _ in range(3):
+        call6()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        call6()
+    e1.record()
+    torch.cuda.synchronize()
+    ms6 = e0.elapsed_time(e1) / steps
     status = head.mtpc_get_status()
     head.mtpc_destroy()
     return {"call": "mtpc_lowrank_window_logprob_backward", "ms_per_call": ms, "phase_ms": phase_ms,
+            "eq6_call": "mtpc_lowrank_window_loss_backward", "eq6_ms_per_call": ms6, "eq6_loss": float(loss.cpu()[0]),
             "phases": "factored forward keeping the logits, circuit backward, logit gradients + their sums + operand "
                       "copies, GEMMs (g A, d hidden, dW_base, dB, dW_sum, dA)",
             "value_equals_forward_call": same_value, "device_status": status,
