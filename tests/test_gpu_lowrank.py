@@ -406,3 +406,51 @@ def test_eq6_loss_backward_on_a_factored_head(family, n, r, v, d, k, N, L):
         head.mtpc_window_loss_backward(hidden, td, N, L, gamma, slot, loss, out["dh"], torch.empty((n, r, v, d), **f32), out["dW_sum"], dT)
     assert e.value.code == -3
     head.mtpc_destroy()
+
+
+def test_factored_training_call_at_full_size_on_sampled_positions():
+    """configs[1]'s shape, rank 16, the launch configuration the benchmark times (64 row tiles, 128 products per batched
+    launch). The loss weights are non-zero on a seeded sample of positions, so every gradient is a sum over exactly those
+    positions, which the oracle can afford; d hidden must vanish everywhere else. A second launch with every weight non-zero
+    checks what holds at any size: the logit gradients of a unit sum to zero over its symbols, so dA summed over the symbols
+    and dW_base summed over the symbols vanish."""
+    wl = I.config_workload(1)
+    s = wl.shape
+    k = 16
+    W, A, Bm = I.lowrank_parameters(s.n, s.r, s.v, s.d, k, seed=97)
+    rng = np.random.default_rng(61)
+    rows = np.unique(np.concatenate([[0, 127, 128, wl.T - 129, wl.T - 128, wl.T - 1], rng.choice(wl.T, 40, replace=False)]))
+    weight = np.zeros(wl.T, dtype=np.float32)
+    weight[rows] = rng.normal(size=len(rows)).astype(np.float32)
+    U = O.lowrank_unembedding(W, A, Bm)
+    ref = OG.window_logprob_grad(s.family, wl.hidden_q[rows], U, wl.W_sum_q, wl.T_static, wl.targets[rows], weight[rows])
+    lr = OG.lowrank_grad(W, A, Bm, ref["dW_emit"])
+    del U
+    head = B.MtpcHead(s.family, s.n, s.r, s.v, s.d, B.MTPC_BF16, wl.T, 1, None, to_device_bf16(wl.W_sum_q), None,
+                      lowrank=(_device(W), _device(A), _device(Bm)))
+    f32 = dict(dtype=torch.float32, device="cuda")
+    out = dict(logprob=torch.empty(wl.T, **f32), dh=torch.empty((wl.T, s.d), **f32), dW_base=torch.empty((s.n, s.v, s.d), **f32),
+               dA=torch.empty((s.n, s.r, s.v, k), **f32), dB=torch.empty((s.n, s.r, k, s.d), **f32),
+               dW_sum=torch.empty((wl.W_sum_q.shape[0], s.d), **f32))
+    hidden = to_device_bf16(wl.hidden_q)
+    targets = torch.from_numpy(wl.targets).cuda()
+    call = lambda w: head.mtpc_lowrank_window_logprob_backward(hidden, targets, w, out["logprob"], out["dh"], out["dW_base"],
+                                                               out["dA"], out["dB"], out["dW_sum"], None)
+    call(torch.from_numpy(weight).cuda())
+    assert head.mtpc_get_status() == 0
+    floor = 2e-5 * float(np.abs(weight).max()) * len(rows) ** 0.5
+    assert np.abs(out["logprob"].cpu().numpy()[rows] - ref["logprob"]).max() <= 2e-3
+    got_dh = out["dh"].cpu().numpy()
+    _whole_tensor("d_hidden", torch.from_numpy(got_dh[rows]), ref["dh"], floor)
+    others = np.setdiff1d(np.arange(wl.T), rows)
+    assert np.abs(got_dh[others]).max() == 0.0
+    for name, want in (("dW_base", lr["dW_base"]), ("dA", lr["dA"]), ("dB", lr["dB"]), ("dW_sum", ref["dW_sum"])):
+        _whole_tensor(name, out[name], want, floor)
+    call(torch.full((wl.T,), -1.0 / wl.T, device="cuda"))
+    assert head.mtpc_get_status() == 0
+    dA, dWb = out["dA"], out["dW_base"]
+    assert float(dA.abs().max()) > 0 and torch.isfinite(out["dh"]).all() and torch.isfinite(out["dB"]).all()
+    # sum over the symbols b of g[t, i, j, b] = 0  =>  sum_b dW_base[i, b, :] = 0; dA[i, j, b, :] = sum_t g z sums to 0 over b
+    assert float(dWb.sum(dim=1).abs().max()) <= 2e-2 * float(dWb.abs().max())
+    assert float(dA.sum(dim=2).abs().max()) <= 2e-2 * float(dA.abs().max())
+    head.mtpc_destroy()
