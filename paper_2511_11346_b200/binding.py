@@ -123,10 +123,16 @@ def _ptr(t) -> int:
     return 0 if t is None else t.data_ptr()
 
 
-def _stream(stream) -> int:
+def _stream(stream, device_index=None) -> int:
+    """The raw cudaStream_t of `stream`, or of torch's current stream on the device (asked for through the raw-handle
+    call: building a torch.cuda.Stream object costs microseconds, which a 70 us draft call notices)."""
     import torch
-    s = stream if stream is not None else torch.cuda.current_stream()
-    return s.cuda_stream
+    if stream is not None:
+        return stream.cuda_stream
+    raw = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+    if raw is None:
+        return torch.cuda.current_stream().cuda_stream
+    return raw(torch.cuda.current_device() if device_index is None else device_index)
 
 
 def mtpc_workspace_bytes(cfg: MtpcConfig) -> int:
@@ -159,12 +165,13 @@ class MtpcHead:
         import torch
         self.cfg = MtpcConfig(family, n, r, v, d, io_dtype, max_positions, max_windows_per_pos, flags, v_valid)
         handle = ctypes.c_void_p(0)
+        self._dev = W_sum.device.index                        # the head lives on the device of its weights
         if lowrank is None:
             nbytes = mtpc_workspace_bytes(self.cfg)
             self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=W_emit.device)
             self._keep = (W_emit, W_sum, T_static)
             _check(lib().mtpc_create_head(ctypes.byref(self.cfg), _ptr(W_emit), _ptr(W_sum), _ptr(T_static),
-                                          self.workspace.data_ptr(), nbytes, _stream(stream), ctypes.byref(handle)),
+                                          self.workspace.data_ptr(), nbytes, _stream(stream, self._dev), ctypes.byref(handle)),
                    "mtpc_create_head")
         else:
             W_base, A, Bm = lowrank
@@ -175,7 +182,7 @@ class MtpcHead:
             self.workspace = torch.empty(need.value, dtype=torch.uint8, device=W_sum.device)
             self._keep = (W_base, A, Bm, W_sum, T_static)
             _check(lib().mtpc_create_head_lowrank(ctypes.byref(self.cfg), k, _ptr(W_base), _ptr(A), _ptr(Bm), _ptr(W_sum),
-                                                  _ptr(T_static), self.workspace.data_ptr(), need.value, _stream(stream),
+                                                  _ptr(T_static), self.workspace.data_ptr(), need.value, _stream(stream, self._dev),
                                                   ctypes.byref(handle)), "mtpc_create_head_lowrank")
         self.handle = handle
 
@@ -183,33 +190,33 @@ class MtpcHead:
     def mtpc_window_logprob(self, hidden, targets, out_logprob, stream=None) -> None:
         T = hidden.shape[0]
         _check(lib().mtpc_window_logprob(self.handle, _ptr(hidden), _ptr(targets), T, _ptr(out_logprob),
-                                         _stream(stream)), "mtpc_window_logprob")
+                                         _stream(stream, self._dev)), "mtpc_window_logprob")
 
     def mtpc_draft_sample(self, hidden, wpp: int, uniforms, out_bytes, out_logprob, stream=None) -> None:
         P = hidden.shape[0]
         _check(lib().mtpc_draft_sample(self.handle, _ptr(hidden), P, wpp, _ptr(uniforms), _ptr(out_bytes),
-                                       _ptr(out_logprob), _stream(stream)), "mtpc_draft_sample")
+                                       _ptr(out_logprob), _stream(stream, self._dev)), "mtpc_draft_sample")
 
     def mtpc_window_prefix_logprob(self, hidden, targets, out_prefix_logprob, stream=None) -> None:
         T = hidden.shape[0]
         _check(lib().mtpc_window_prefix_logprob(self.handle, _ptr(hidden), _ptr(targets), T, _ptr(out_prefix_logprob),
-                                                _stream(stream)), "mtpc_window_prefix_logprob")
+                                                _stream(stream, self._dev)), "mtpc_window_prefix_logprob")
 
     def mtpc_draft_sample_prefix(self, hidden, wpp: int, uniforms, out_bytes, out_prefix_logprob, stream=None) -> None:
         P = hidden.shape[0]
         _check(lib().mtpc_draft_sample_prefix(self.handle, _ptr(hidden), P, wpp, _ptr(uniforms), _ptr(out_bytes),
-                                              _ptr(out_prefix_logprob), _stream(stream)), "mtpc_draft_sample_prefix")
+                                              _ptr(out_prefix_logprob), _stream(stream, self._dev)), "mtpc_draft_sample_prefix")
 
     def mtpc_speculative_accept(self, P: int, wpp: int, draft_bytes, prefix_logprob, target_probs, accept_uniforms,
                                 out_accepted, out_next_byte, stream=None) -> None:
         _check(lib().mtpc_speculative_accept(self.handle, P, wpp, _ptr(draft_bytes), _ptr(prefix_logprob),
                                              _ptr(target_probs), _ptr(accept_uniforms), _ptr(out_accepted),
-                                             _ptr(out_next_byte), _stream(stream)), "mtpc_speculative_accept")
+                                             _ptr(out_next_byte), _stream(stream, self._dev)), "mtpc_speculative_accept")
 
     def mtpc_window_loss(self, hidden, targets, num_sequences: int, sequence_length: int, gamma: float, out_slot_loss,
                          out_loss, stream=None) -> None:
         _check(lib().mtpc_window_loss(self.handle, _ptr(hidden), _ptr(targets), num_sequences, sequence_length,
-                                      ctypes.c_float(gamma), _ptr(out_slot_loss), _ptr(out_loss), _stream(stream)),
+                                      ctypes.c_float(gamma), _ptr(out_slot_loss), _ptr(out_loss), _stream(stream, self._dev)),
                "mtpc_window_loss")
 
     def _backward_workspace(self, T: int, device):
@@ -229,7 +236,7 @@ class MtpcHead:
         _check(lib().mtpc_window_loss_backward(self.handle, _ptr(hidden), _ptr(targets), num_sequences, sequence_length,
                                                ctypes.c_float(gamma), ws.data_ptr(), ws.numel(), _ptr(out_slot_loss),
                                                _ptr(out_loss), _ptr(d_hidden), _ptr(dW_emit), _ptr(dW_sum), _ptr(dT_static),
-                                               _stream(stream)), "mtpc_window_loss_backward")
+                                               _stream(stream, self._dev)), "mtpc_window_loss_backward")
 
     def mtpc_window_logprob_backward(self, hidden, targets, weight, out_logprob, d_hidden, dW_emit, dW_sum, dT_static=None,
                                      stream=None) -> None:
@@ -238,7 +245,7 @@ class MtpcHead:
         ws = self._backward_workspace(T, hidden.device)
         _check(lib().mtpc_window_logprob_backward(self.handle, _ptr(hidden), _ptr(targets), T, _ptr(weight), ws.data_ptr(),
                                                   ws.numel(), _ptr(out_logprob), _ptr(d_hidden), _ptr(dW_emit), _ptr(dW_sum),
-                                                  _ptr(dT_static), _stream(stream)), "mtpc_window_logprob_backward")
+                                                  _ptr(dT_static), _stream(stream, self._dev)), "mtpc_window_logprob_backward")
 
     def _lowrank_backward_workspace(self, T: int, k: int, device):
         import torch
@@ -258,7 +265,7 @@ class MtpcHead:
         _check(lib().mtpc_lowrank_window_loss_backward(self.handle, _ptr(hidden), _ptr(targets), num_sequences, sequence_length,
                                                        ctypes.c_float(gamma), ws.data_ptr(), ws.numel(), _ptr(out_slot_loss),
                                                        _ptr(out_loss), _ptr(d_hidden), _ptr(dW_base), _ptr(dA), _ptr(dB),
-                                                       _ptr(dW_sum), _ptr(dT_static), _stream(stream)),
+                                                       _ptr(dW_sum), _ptr(dT_static), _stream(stream, self._dev)),
                "mtpc_lowrank_window_loss_backward")
 
     def mtpc_lowrank_window_logprob_backward(self, hidden, targets, weight, out_logprob, d_hidden, dW_base, dA, dB, dW_sum,
@@ -269,26 +276,26 @@ class MtpcHead:
         _check(lib().mtpc_lowrank_window_logprob_backward(self.handle, _ptr(hidden), _ptr(targets), T, _ptr(weight),
                                                           ws.data_ptr(), ws.numel(), _ptr(out_logprob), _ptr(d_hidden),
                                                           _ptr(dW_base), _ptr(dA), _ptr(dB), _ptr(dW_sum), _ptr(dT_static),
-                                                          _stream(stream)), "mtpc_lowrank_window_logprob_backward")
+                                                          _stream(stream, self._dev)), "mtpc_lowrank_window_logprob_backward")
 
     # -- host-buffer calls (copies inside; outputs ready on return)
     def mtpc_window_logprob_host(self, hidden_host, targets_host, out_logprob_host, stream=None) -> None:
         T = hidden_host.shape[0]
         _check(lib().mtpc_window_logprob_host(self.handle, _ptr(hidden_host), _ptr(targets_host), T,
-                                              _ptr(out_logprob_host), _stream(stream)), "mtpc_window_logprob_host")
+                                              _ptr(out_logprob_host), _stream(stream, self._dev)), "mtpc_window_logprob_host")
 
     def mtpc_draft_sample_host(self, hidden_host, wpp: int, uniforms_host, out_bytes_host, out_logprob_host,
                                stream=None) -> None:
         P = hidden_host.shape[0]
         _check(lib().mtpc_draft_sample_host(self.handle, _ptr(hidden_host), P, wpp, _ptr(uniforms_host),
-                                            _ptr(out_bytes_host), _ptr(out_logprob_host), _stream(stream)),
+                                            _ptr(out_bytes_host), _ptr(out_logprob_host), _stream(stream, self._dev)),
                "mtpc_draft_sample_host")
 
     def mtpc_get_status(self, stream=None, with_code: bool = False):
         """The status bits raised since the last query (and cleared by it); with_code: (return code, bits), the code
         being MTPC_ERR_TIMEOUT when a bounded wait gave up on the device."""
         flags = ctypes.c_uint32(0)
-        code = lib().mtpc_get_status(self.handle, _stream(stream), ctypes.byref(flags))
+        code = lib().mtpc_get_status(self.handle, _stream(stream, self._dev), ctypes.byref(flags))
         if code not in (MTPC_OK, ERR_TIMEOUT):
             raise MtpcError(code, "mtpc_get_status")
         return (code, flags.value) if with_code else flags.value
@@ -316,7 +323,7 @@ class MtpcHead:
 
     def mtpc_update_parameters(self, W_emit, W_sum, T_static=None, stream=None) -> None:
         """Rebind the head to (possibly updated) parameter tensors; they must outlive the head like the first ones."""
-        _check(lib().mtpc_update_parameters(self.handle, _ptr(W_emit), _ptr(W_sum), _ptr(T_static), _stream(stream)),
+        _check(lib().mtpc_update_parameters(self.handle, _ptr(W_emit), _ptr(W_sum), _ptr(T_static), _stream(stream, self._dev)),
                "mtpc_update_parameters")
         self._keep = (W_emit, W_sum, T_static)
 
