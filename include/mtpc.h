@@ -295,12 +295,14 @@ int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k,
  *   workspace >= mtpc_lowrank_workspace_bytes(cfg, k): the dense head's workspace plus z = B h as two bf16 halves, a copy
  *            of A in the layout the kernel reads (remade on every call, so A is always read as it is then) and, for
  *            v > 224, the per-panel partial log-sum-exps.
- * Such a head serves mtpc_window_logprob, mtpc_window_prefix_logprob, mtpc_window_loss, mtpc_window_logprob_host, and,
- * for up to 128 positions per call, mtpc_draft_sample, mtpc_draft_sample_prefix and mtpc_speculative_accept: the draft's
- * weight pass then streams W_base and B (n v + n r k rows) instead of n r v composed rows, and the logits are formed
- * from the two small products. Its training calls are mtpc_lowrank_window_logprob_backward and mtpc_lowrank_window_loss_backward (below). Drafts of more than
- * 128 positions, mtpc_window_logprob_backward and mtpc_window_loss_backward return MTPC_ERR_UNSUPPORTED on it: those run
- * on the composed tensor (mtpc_lowrank_compose + mtpc_create_head, gradients carried back by mtpc_lowrank_backward).
+ * Such a head serves mtpc_window_logprob, mtpc_window_prefix_logprob, mtpc_window_loss, mtpc_window_logprob_host,
+ * mtpc_draft_sample, mtpc_draft_sample_prefix and, after a draft of up to 128 positions, mtpc_speculative_accept: the
+ * draft's weight pass streams W_base and B (n v + n r k rows) instead of n r v composed rows, and the logits are formed
+ * from the two small products; longer drafts run 128 positions at a time (the acceptance stage then returns
+ * MTPC_ERR_STATE: only the last chunk's logits remain). Its training calls are mtpc_lowrank_window_logprob_backward and
+ * mtpc_lowrank_window_loss_backward (below); mtpc_window_logprob_backward and mtpc_window_loss_backward return
+ * MTPC_ERR_UNSUPPORTED on it (they produce the gradient of a composed tensor: mtpc_lowrank_compose + mtpc_create_head,
+ * carried back by mtpc_lowrank_backward).
  */
 int mtpc_lowrank_workspace_bytes(const mtpc_config* cfg, int32_t k, size_t* out_bytes);
 

@@ -715,7 +715,21 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   const Layout& L = h->L;
   const int W = P * wpp;
   if (!L.can_draft) return MTPC_ERR_UNSUPPORTED;
-  if (h->lr_k > 0 && P > L.decode_max_p) return MTPC_ERR_UNSUPPORTED;   // a factored head drafts on the few-position path only
+  if (h->lr_k > 0 && P > L.decode_max_p) {
+    // A factored head has no composed tensor for the many-position path, and needs none: W_base, B and A are small enough
+    // to stay in L2, so the few-position path runs chunk after chunk of positions. Only the last chunk's logits remain:
+    // no acceptance stage after such a draft.
+    for (int p0 = 0; p0 < P; p0 += L.decode_max_p) {
+      const int pc = P - p0 < L.decode_max_p ? P - p0 : L.decode_max_p;
+      const size_t w0 = static_cast<size_t>(p0) * wpp;
+      const int rc = draft_sample_impl(h, static_cast<const uint8_t*>(hidden) + static_cast<size_t>(p0) * c.d * 2, pc, wpp,
+                                       uniforms + w0 * 2 * c.n, out_bytes + w0 * c.n, out_logprob ? out_logprob + w0 : nullptr,
+                                       out_prefix ? out_prefix + w0 * c.n : nullptr, st);
+      if (rc != MTPC_OK) return rc;
+    }
+    h->draft_P = 0;
+    return MTPC_OK;
+  }
   const void* hb = nullptr;
   int rc = stage_hidden(h, hidden, P, &hb, st);
   if (rc != MTPC_OK) return rc;

@@ -188,14 +188,27 @@ def test_factored_head_matches_the_composed_definition(family, n, r, v, vv, d, k
     assert np.abs(pre[:, -1].cpu().numpy() - ref).max() <= 2e-3
     # what the factored head does not do is refused, not approximated: it drafts on the few-position path only
     # (tests/test_gpu_speculative.py checks those drafts), and has no backward pass
-    draft_args = (hidden, 1, torch.full((T, 2 * n), 0.5, device="cuda"), torch.empty((T, n), dtype=torch.int32, device="cuda"), out)
-    if T > 128:
+    # it drafts too, 128 positions at a time (tests/test_gpu_speculative.py checks drafts and acceptance); the backward call of a
+    # head on a composed tensor is refused, not approximated
+    u = wl.uniforms if wl.uniforms is not None else I.uniforms(I.BASE_SEED + 3, 5, (T, 2 * n))
+    drafted = torch.empty((T, n), dtype=torch.int32, device="cuda")
+    head.mtpc_draft_sample(hidden, 1, torch.from_numpy(np.ascontiguousarray(u[:T])).cuda(), drafted, out)
+    assert head.mtpc_get_status() == 0
+    d_ref = O.draft_sample(fam, wl.hidden_q, U, wl.W_sum_q, wl.T_static, 1, u[:T])
+    differ = (drafted.cpu().numpy() != d_ref["bytes"]).any(axis=1)
+    assert not (differ & (d_ref["margin"] >= 1e-6)).any()
+    assert np.abs(out.cpu().numpy()[~differ] - d_ref["logprob"][~differ]).max() <= 2e-3
+    if T > 128:                                                            # only the last chunk's logits remain
         with pytest.raises(B.MtpcError) as e:
-            head.mtpc_draft_sample(*draft_args)
-        assert e.value.code == -3
-    else:
-        head.mtpc_draft_sample(*draft_args)
-        assert head.mtpc_get_status() == 0
+            head.mtpc_speculative_accept(T, 1, drafted, pre, torch.zeros((T, n + 1, v), device="cuda"),
+                                         torch.zeros((T, n + 1), device="cuda"), torch.empty(T, dtype=torch.int32, device="cuda"),
+                                         torch.empty(T, dtype=torch.int32, device="cuda"))
+        assert e.value.code == B.ERR_STATE
+    with pytest.raises(B.MtpcError) as e:
+        head.mtpc_window_logprob_backward(hidden, targets, torch.ones(T, device="cuda"), out, torch.empty((T, d), device="cuda"),
+                                          torch.empty((n, r, v, d), device="cuda"), torch.empty((wl.W_sum_q.shape[0], d), device="cuda"),
+                                          torch.empty((max(n - 1, 1), r, r), device="cuda"))
+    assert e.value.code == -3
     head.mtpc_destroy()
 
 
