@@ -903,8 +903,10 @@ int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmO
   p.seg_kblocks[0] = (K0 + kBlockK - 1) / kBlockK;
   p.seg_kblocks[1] = K1 > 0 ? (K1 + kBlockK - 1) / kBlockK : 0;
   p.m_tiles = (M + kBlockM - 1) / kBlockM;
-  p.n_tiles = (N + kPlainTileN - 1) / kPlainTileN;
-  p.stage_bytes = kABytes + kPlainTileN * kBlockK * 2;
+  // batched products with a rank for N: 64-column accumulator tiles
+  const int tile_n = (x.batches > 1 && N <= 64 && B0.mn_major) ? 64 : kPlainTileN;
+  p.n_tiles = (N + tile_n - 1) / tile_n;
+  p.stage_bytes = kABytes + tile_n * kBlockK * 2;
   const int ctl = 1024 + static_cast<int>(sizeof(GemmControl));
   p.stages = (kSmemLimit - ctl) / p.stage_bytes;
   if (p.stages > kMaxStages) p.stages = kMaxStages;
@@ -926,7 +928,9 @@ int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmO
   const long long items = static_cast<long long>(p.m_tiles) * p.n_tiles * p.batches;
   const int grid = static_cast<int>(items < h->num_sms ? items : h->num_sms);
   const size_t smem = p.stages * p.stage_bytes + ctl;
-  if (A.mn_major && B0.mn_major) plain_gemm_kernel<true, true><<<grid, kGemmThreads, smem, st>>>(p);
+  if (tile_n == 64 && A.mn_major) plain_gemm_kernel<true, true, 64><<<grid, kGemmThreads, smem, st>>>(p);
+  else if (tile_n == 64) plain_gemm_kernel<false, true, 64><<<grid, kGemmThreads, smem, st>>>(p);
+  else if (A.mn_major && B0.mn_major) plain_gemm_kernel<true, true><<<grid, kGemmThreads, smem, st>>>(p);
   else if (!A.mn_major && B0.mn_major) plain_gemm_kernel<false, true><<<grid, kGemmThreads, smem, st>>>(p);
   else if (!A.mn_major && !B0.mn_major) plain_gemm_kernel<false, false><<<grid, kGemmThreads, smem, st>>>(p);
   else return MTPC_ERR_SHAPE;
@@ -1420,6 +1424,8 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
   fail |= !allow_full_smem(plain_gemm_kernel<false, false>);
   fail |= !allow_full_smem(plain_gemm_kernel<false, true>);
   fail |= !allow_full_smem(plain_gemm_kernel<true, true>);
+  fail |= !allow_full_smem(plain_gemm_kernel<true, true, 64>);
+  fail |= !allow_full_smem(plain_gemm_kernel<false, true, 64>);
   fail |= cudaFuncSetAttribute(mtpc_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) !=
           cudaSuccess;
   const int slot_smem = static_cast<int>(kSlotSmemLimit);

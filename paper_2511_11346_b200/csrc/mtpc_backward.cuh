@@ -682,7 +682,9 @@ struct PlainGemmParams {
 constexpr int kPlainTileN = 256;
 constexpr uint32_t kMnBoxBytes = 64 * kBlockK * 2;   // one 64 x 64 bf16 box: 8 KB
 
-template <bool A_MN, bool B_MN>
+// TN: columns of an accumulator tile: 256, or 64 for the batched products whose N is a rank (MN-major B only: the boxes
+// of the tensor map are 64 wide) - what is fetched, multiplied and read back for columns that do not exist is a quarter.
+template <bool A_MN, bool B_MN, int TN = 256>
 __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __grid_constant__ PlainGemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -697,7 +699,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
   const int num_items = per_batch * p.batches;
   const int kblocks = p.seg_kblocks[0] + p.seg_kblocks[1];
   constexpr uint32_t kSlots = 2;
-  constexpr uint32_t kBBytes = kPlainTileN * kBlockK * 2;
+  constexpr uint32_t kBBytes = TN * kBlockK * 2;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -733,7 +735,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
         const int bt = item / per_batch, rest = item - bt * per_batch;
         const int nt = rest % p.n_tiles, mt = rest / p.n_tiles;
         const int am = mt * kBlockM + bt * p.a_m_step, ak = bt * p.a_k_step;    // this product's corner of A ...
-        const int bn = nt * kPlainTileN + bt * p.b_n_step, bk = bt * p.b_k_step;   // ... and of B
+        const int bn = nt * TN + bt * p.b_n_step, bk = bt * p.b_k_step;   // ... and of B
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!bounded_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, p.status)) { ok = false; break; }
           const uint32_t full = smem_u32(&ctl->full[stage]);
@@ -750,7 +752,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
           }
           if (B_MN) {
 #pragma unroll
-            for (int q = 0; q < kPlainTileN / 64; ++q)
+            for (int q = 0; q < TN / 64; ++q)
               tma_load_2d(a_dst + kABytes + q * kMnBoxBytes, &p.tm_b[seg], full, bn + q * 64, kloc + bk);
           } else {
             tma_load_2d(a_dst + kABytes, &p.tm_b[seg], full, kloc + bk, bn);
@@ -774,7 +776,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, use = 0;
       bool ok = true;
-      const uint32_t idesc = umma_idesc_bf16(kBlockM, kPlainTileN, A_MN, B_MN);
+      const uint32_t idesc = umma_idesc_bf16(kBlockM, TN, A_MN, B_MN);
       // descriptor advance per K=16 step, in 16-byte units: 32 bytes along a swizzled K-major row, two 8-row groups
       // (2048 bytes) down an MN-major box
       constexpr uint32_t kStepA = A_MN ? 128u : 2u, kStepB = B_MN ? 128u : 2u;
@@ -782,7 +784,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
         const uint32_t slot = use % kSlots;
         if (!bounded_wait(smem_u32(&ctl->tempty[slot]), ((use / kSlots) & 1u) ^ 1u, ctl, p.status)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + slot * kPlainTileN;
+        const uint32_t d_tmem = tmem_base + slot * TN;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!bounded_wait(smem_u32(&ctl->full[stage]), phase, ctl, p.status)) { ok = false; break; }
           tc_fence_after();
@@ -817,11 +819,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) plain_gemm_kernel(const __gri
       if (!bounded_wait_warp(smem_u32(&ctl->tfull[slot]), (use / kSlots) & 1u, ctl, p.status, lane)) break;
       tc_fence_after();
       const int row = mt * kBlockM + quarter * 32 + lane;
-      const uint32_t tcol = lane_base + slot * kPlainTileN;
+      const uint32_t tcol = lane_base + slot * TN;
       const size_t coff = static_cast<size_t>(row < p.M ? row : 0) * p.ldc + static_cast<size_t>(bt) * p.c_step;
       float* crow = p.C + coff;
-      for (int b = 0; b < kPlainTileN / 16; ++b) {
-        const int col0 = nt * kPlainTileN + b * 16;
+      for (int b = 0; b < TN / 16; ++b) {
+        const int col0 = nt * TN + b * 16;
         if (col0 >= p.N) break;                          // (warp-uniform) the rest of the tile lies past the last column
         float x[16];
         tmem_ld16(tcol + b * 16, x);
