@@ -147,6 +147,8 @@ FACTORED = [
     (I.HMM, 2, 4, 320, 306, 64, 16, 100),      # padded vocabulary, two panels, static transitions
     (I.CP, 1, 2, 1024, 1010, 64, 16, 40),      # eight panels of 128 columns
     (I.CP, 2, 4, 272, 268, 64, 16, 90),        # panels of 144 and 128 columns
+    (I.CP, 1, 2, 1792, 0, 64, 16, 30),         # the widest unit: eight panels of 224 columns, one epilogue group, two-entry rings
+    (I.HMM, 2, 4, 224, 0, 128, 32, 131),       # one panel of 224 columns, rank 32
 ]
 
 
