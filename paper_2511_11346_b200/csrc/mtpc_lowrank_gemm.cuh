@@ -20,8 +20,8 @@
 // other), then from warp 8 on `groups` epilogue groups of four warps (one thread per position): group g takes the
 // components j = g, g + groups, ... The two pipelines share nothing but the tensor cores: each has its
 // own shared-memory ring and its own barriers. Base ring: a 64-wide K block of h and of the panel's rows of W_i. Correction
-// ring: one entry holds the operands of 64 / k components, all as 128-byte rows with the 128-byte swizzle (the tensor cores
-// read 32-byte-row tiles several times slower): z as boxes of 128 positions x 64 values = [hi | lo] of 32 / k adjacent
+// ring: one entry holds the operands of 64 / k components, all as 128-byte rows with the 128-byte swizzle (few large boxes
+// instead of many 32-byte-row ones): z as boxes of 128 positions x 64 values = [hi | lo] of 32 / k adjacent
 // components, and A as boxes of chunk_cols vocabulary rows x 64 values = the k adaptor columns of 64 / k adjacent components,
 // read from a copy of A laid out [n, v, r, k] (lowrank_repack_kernel, made on every call: A is small and may have changed).
 // A correction MMA (K = 16) addresses its operands inside those rows, 32 bytes apart, like the K steps of the base.
