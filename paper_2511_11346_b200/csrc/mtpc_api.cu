@@ -277,6 +277,7 @@ struct mtpc_head {
   const void* lr_B;                             // [n, r, k, d] bf16
   size_t lr_off_arep;                           // workspace: A as [n, v, r, k]
   size_t lr_off_dec;                            // workspace: few-position draft products base [P, n v] | z [P, n r k]
+  size_t lr_off_base;                           // workspace: long drafts: W_base h [T, n v] fp32 (0: not reserved)
   CUtensorMap tm_lrB_dec;                       // B [n r k, d] for the few-position draft path
   size_t lr_off_zhl, lr_off_partial;            // workspace: z = B h as bf16 halves [T, n r, 2, k]; per-panel partial log-sum-exps
   LowRankGemmParams lr_params;                  // everything of the factored projection launch that does not depend on the call
@@ -686,8 +687,9 @@ struct PlainGemmExtra {
 int launch_plain_gemm(mtpc_head* h, GemmOperand A, GemmOperand B0, int K0, GemmOperand B1, int K1, int a_k1, float* C,
                       size_t ldc, int M, int N, cudaStream_t st, void* C_hilo = nullptr, int split_k = 0,
                       const PlainGemmExtra* extra = nullptr);
+// parts: 1 = sum-unit tiles (log omega), 2 = z = B h and the repacked A, 4 = the factored kernel (and its merge)
 int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, const int* targets, cudaStream_t st,
-                              const GradArgs* ga = nullptr);
+                              const GradArgs* ga = nullptr, int parts = 7, bool targets_are_drafts = false);
 
 // out [T] (joint) and / or prefix [T, n] (prefix log-marginals); either may be NULL, not both.
 int window_logprob_impl(mtpc_head* h, const void* hidden, const int32_t* targets, int32_t T, float* out, float* prefix,
@@ -715,10 +717,56 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
   const Layout& L = h->L;
   const int W = P * wpp;
   if (!L.can_draft) return MTPC_ERR_UNSUPPORTED;
+  if (h->lr_k > 0 && P > L.decode_max_p && wpp == 1 && c.v <= kMaxDraftVocab && h->lr_off_base != 0) {
+    // A long draft on a factored head, one window per position: log omega, the latent draws, then every (window, slot)
+    // forms the logits of its one selected unit from W_base h and B h (lowrank_draw_kernel) and draws its byte; the
+    // evidence of the drafted bytes under every unit is the factored projection with them as targets. No logits are
+    // kept: no acceptance stage after such a draft.
+    const int k = h->lr_k;
+    h->draft_P = 0;
+    PhaseTimer pt(h, st);
+    pt.begin();
+    int rc = launch_lowrank_projection(h, hidden, P, nullptr, st, nullptr, /*parts=*/1 | 2);
+    pt.end();
+    if (rc != MTPC_OK) return rc;
+    pt.begin();
+    latent_sample_kernel<<<(W + 127) / 128, 128, 0, st>>>(c.family, at<float>(h, L.off_logw), hmm_tables(h), uniforms,
+                                                          at<int>(h, L.off_sel), out_bytes, at<unsigned>(h, L.off_status), W,
+                                                          wpp, c.n, c.r, L.sum_rows, hmm_table_stride(h));
+    h->launches++;
+    pt.end();
+    if ((rc = check_launch()) != MTPC_OK) return rc;
+    pt.begin();
+    float* base = reinterpret_cast<float*>(h->ws + h->lr_off_base);
+    rc = launch_plain_gemm(h, GemmOperand{hidden, static_cast<size_t>(c.d), false},
+                           GemmOperand{h->lr_W_base, static_cast<size_t>(c.d), false}, c.d,
+                           GemmOperand{h->lr_W_base, static_cast<size_t>(c.d), false}, 0, 0, base,
+                           static_cast<size_t>(c.n) * c.v, P, c.n * c.v, st);
+    if (rc != MTPC_OK) return rc;
+    {
+      const int pairs = W * c.n;
+      int blocks = (pairs + kDrawWarps - 1) / kDrawWarps;
+      if (blocks > 32 * h->num_sms) blocks = 32 * h->num_sms;
+      lowrank_draw_kernel<<<blocks, 32 * kDrawWarps, static_cast<size_t>(kDrawWarps) * c.v * sizeof(float), st>>>(
+          base, reinterpret_cast<const __nv_bfloat16*>(h->ws + h->lr_off_zhl), static_cast<const __nv_bfloat16*>(h->lr_A),
+          at<int>(h, L.off_sel), uniforms, out_bytes, at<unsigned>(h, L.off_status), W, wpp, c.n, c.r, c.v, valid_symbols(c), k);
+      h->launches++;
+    }
+    pt.end();
+    if ((rc = check_launch()) != MTPC_OK) return rc;
+    pt.begin();
+    rc = launch_lowrank_projection(h, hidden, P, out_bytes, st, nullptr, /*parts=*/4, /*targets_are_drafts=*/true);
+    pt.end();
+    if (rc != MTPC_OK) return rc;
+    pt.begin();
+    rc = launch_circuit(h, W, wpp, out_logprob, out_prefix, st);
+    pt.end();
+    return rc;
+  }
   if (h->lr_k > 0 && P > L.decode_max_p) {
-    // A factored head has no composed tensor for the many-position path, and needs none: W_base, B and A are small enough
-    // to stay in L2, so the few-position path runs chunk after chunk of positions. Only the last chunk's logits remain:
-    // no acceptance stage after such a draft.
+    // Otherwise (several windows per position, or units wider than 512 symbols) the few-position path runs chunk after
+    // chunk of positions: W_base, B and A are small enough to stay in L2. Only the last chunk's logits remain: no
+    // acceptance stage after such a draft either.
     for (int p0 = 0; p0 < P; p0 += L.decode_max_p) {
       const int pc = P - p0 < L.decode_max_p ? P - p0 : L.decode_max_p;
       const size_t w0 = static_cast<size_t>(p0) * wpp;
@@ -990,34 +1038,38 @@ bool plan_lowrank(const mtpc_config& c, int k, LowRankGemmParams* p) {
 // Factored projection of a low-rank head: log omega by the dense kernel's sum tiles, z = B h by a plain GEMM that writes
 // it as two bf16 halves, A repacked, then the factored kernel (and the merge of its panels) writes G.
 int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, const int* targets, cudaStream_t st,
-                              const GradArgs* ga) {
+                              const GradArgs* ga, int parts, bool targets_are_drafts) {
   const mtpc_config& c = h->cfg;
   const Layout& L = h->L;
   const int units = c.n * c.r, k = h->lr_k;
-  int rc = launch_gemm(h, kModeLogprob, hidden_bf16, T, 1, false, true, targets, nullptr, nullptr, st);
+  int rc = MTPC_OK;
+  if (parts & 1) rc = launch_gemm(h, kModeLogprob, hidden_bf16, T, 1, false, true, targets, nullptr, nullptr, st);
   if (rc != MTPC_OK) return rc;
   __nv_bfloat16* zhl = reinterpret_cast<__nv_bfloat16*>(h->ws + h->lr_off_zhl);
-  const GemmOperand hid{hidden_bf16, static_cast<size_t>(c.d), false};
-  const GemmOperand bmat{h->lr_B, static_cast<size_t>(c.d), false};          // [n r k, d], K = d contiguous
-  // z = B h, leaving the GEMM's epilogue already split into its two bf16 halves [T, n r, 2, k]
-  rc = launch_plain_gemm(h, hid, bmat, c.d, bmat, 0, 0, nullptr, 0, T, units * k, st, zhl, k);
-  if (rc != MTPC_OK) return rc;
-  LowRankGemmParams p = h->lr_params;
-  rc = make_tmap(&p.tm_h, hidden_bf16, static_cast<uint64_t>(T), static_cast<uint64_t>(c.d), kBlockM);
-  if (rc == MTPC_OK) rc = make_tmap(&p.tm_z, zhl, static_cast<uint64_t>(T), static_cast<uint64_t>(units) * 2 * k, kBlockM);
-  if (rc != MTPC_OK) return rc;
-  {   // A as [n, v, r, k]: the adaptor columns of adjacent components side by side (remade every call: A may have changed)
+  if (parts & 2) {
+    const GemmOperand hid{hidden_bf16, static_cast<size_t>(c.d), false};
+    const GemmOperand bmat{h->lr_B, static_cast<size_t>(c.d), false};          // [n r k, d], K = d contiguous
+    // z = B h, leaving the GEMM's epilogue already split into its two bf16 halves [T, n r, 2, k]
+    rc = launch_plain_gemm(h, hid, bmat, c.d, bmat, 0, 0, nullptr, 0, T, units * k, st, zhl, k);
+    if (rc != MTPC_OK) return rc;
+    // A as [n, v, r, k]: the adaptor columns of adjacent components side by side (remade every call: A may have changed)
     const size_t pieces = static_cast<size_t>(units) * c.v * (k / 8);
     lowrank_repack_kernel<<<static_cast<unsigned>((pieces + 255) / 256), 256, 0, st>>>(
         static_cast<const uint4*>(h->lr_A), reinterpret_cast<uint4*>(h->ws + h->lr_off_arep), c.n, c.r, c.v, k / 8);
     h->launches += 1;
   }
+  if (!(parts & 4)) return check_launch();
+  LowRankGemmParams p = h->lr_params;
+  rc = make_tmap(&p.tm_h, hidden_bf16, static_cast<uint64_t>(T), static_cast<uint64_t>(c.d), kBlockM);
+  if (rc == MTPC_OK) rc = make_tmap(&p.tm_z, zhl, static_cast<uint64_t>(T), static_cast<uint64_t>(units) * 2 * k, kBlockM);
+  if (rc != MTPC_OK) return rc;
   p.T = T;
   p.m_tiles = (T + kBlockM - 1) / kBlockM;
   p.targets = targets;
   p.G = at<float>(h, L.off_G);
   p.status = at<unsigned>(h, L.off_status);
   p.wait_limit_ns = h->wait_limit_ns;
+  p.missing_is_nan = targets_are_drafts ? 1 : 0;
   if (ga != nullptr) {                 // a training call keeps every logit and every unit's log-sum-exp
     p.logit_out = ga->logit_out;
     p.logit_pitch = ga->logit_pitch;
@@ -1035,7 +1087,7 @@ int launch_lowrank_projection(mtpc_head* h, const void* hidden_bf16, int T, cons
   h->launches += 1;
   if (p.panels > 1) {     // several panels per unit: their partial log-sum-exps are combined into G
     lowrank_merge_kernel<<<static_cast<unsigned>((entries + 255) / 256), 256, 0, st>>>(
-        p.partial, p.target_logit, targets, p.G, p.lse_out, p.status, entries, c.r, p.vv, p.panels);
+        p.partial, p.target_logit, targets, p.G, p.lse_out, p.status, entries, c.r, p.vv, p.panels, p.missing_is_nan);
     h->launches += 1;
   }
   return check_launch();
@@ -1351,7 +1403,7 @@ struct LowRankSpec {
 // that computes it), where a unit is cut into panels the panels' (maximum, sum) pairs and the targets' logits, and the
 // copy of A the factored kernel reads.
 static int lowrank_extra_bytes(const mtpc_config& c, int k, int panels, size_t base_total, size_t* off_zhl,
-                               size_t* off_partial, size_t* off_arep, size_t* off_dec, size_t* total) {
+                               size_t* off_partial, size_t* off_arep, size_t* off_dec, size_t* off_base, size_t* total) {
   const size_t units = static_cast<size_t>(c.n) * c.r;
   size_t off = align_up(base_total);
   *off_zhl = off;
@@ -1363,6 +1415,11 @@ static int lowrank_extra_bytes(const mtpc_config& c, int k, int panels, size_t b
   *off_dec = off;                       // few-position draft: base = W_base h [P, n v] and z = B h [P, n r k], fp32
   off += align_up(static_cast<size_t>(c.max_positions < kDecodeMaxP ? c.max_positions : kDecodeMaxP) *
                   (static_cast<size_t>(c.n) * c.v + units * k) * 4);
+  *off_base = 0;                        // long drafts (more positions than that path takes): W_base h [T, n v] fp32
+  if (c.max_positions > kDecodeMaxP && c.v <= kMaxDraftVocab) {
+    *off_base = off;
+    off += align_up(static_cast<size_t>(c.max_positions) * c.n * c.v * 4);
+  }
   *total = off;
   return MTPC_OK;
 }
@@ -1378,11 +1435,11 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
   if (rc != MTPC_OK) return rc;
   LowRankGemmParams lrp;
   memset(&lrp, 0, sizeof(lrp));
-  size_t lr_zhl = 0, lr_partial = 0, lr_arep = 0, lr_dec = 0;
+  size_t lr_zhl = 0, lr_partial = 0, lr_arep = 0, lr_dec = 0, lr_base = 0;
   if (lowrank) {
     if (cfg->io_dtype != MTPC_BF16) return MTPC_ERR_UNSUPPORTED;
     if (!plan_lowrank(*cfg, lowrank->k, &lrp)) return MTPC_ERR_UNSUPPORTED;
-    lowrank_extra_bytes(*cfg, lowrank->k, lrp.panels, L.total, &lr_zhl, &lr_partial, &lr_arep, &lr_dec, &L.total);
+    lowrank_extra_bytes(*cfg, lowrank->k, lrp.panels, L.total, &lr_zhl, &lr_partial, &lr_arep, &lr_dec, &lr_base, &L.total);
   }
   const bool ctx = (cfg->flags & MTPC_FLAG_HMM_CONTEXTUAL) != 0;
   if (cfg->family == MTPC_HMM && cfg->n > 1 && !ctx && !T_static) return MTPC_ERR_NULL;
@@ -1407,6 +1464,7 @@ static int create_head_impl(const mtpc_config* cfg, const void* W_emit, const Lo
     h->lr_off_partial = lr_partial;
     h->lr_off_arep = lr_arep;
     h->lr_off_dec = lr_dec;
+    h->lr_off_base = lr_base;
     h->lr_params = lrp;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1467,8 +1525,8 @@ int mtpc_lowrank_workspace_bytes(const mtpc_config* cfg, int32_t k, size_t* out_
   if (rc != MTPC_OK) return rc;
   LowRankGemmParams lrp;
   if (cfg->io_dtype != MTPC_BF16 || !plan_lowrank(*cfg, k, &lrp)) return MTPC_ERR_UNSUPPORTED;
-  size_t a = 0, b = 0, c3 = 0, c4 = 0;
-  return lowrank_extra_bytes(*cfg, k, lrp.panels, L.total, &a, &b, &c3, &c4, out_bytes);
+  size_t a = 0, b = 0, c3 = 0, c4 = 0, c5 = 0;
+  return lowrank_extra_bytes(*cfg, k, lrp.panels, L.total, &a, &b, &c3, &c4, &c5, out_bytes);
 }
 
 int mtpc_create_head_lowrank(const mtpc_config* cfg, int32_t k, const void* W_base, const void* A, const void* B,

@@ -30,6 +30,7 @@
 #include <math_constants.h>
 
 #include "mtpc_circuit.cuh"
+#include "mtpc_decode.cuh"
 #include "mtpc_gemm.cuh"
 
 namespace mtpc {
@@ -60,6 +61,7 @@ struct LowRankGemmParams {
   float* logit_out;                  // training: every logit [T, n r v] fp32 at a pitch of logit_pitch (NULL: not kept) ...
   size_t logit_pitch;
   float* lse_out;                    // ... and every unit's log-sum-exp [T, n r] (with several panels: by the merge kernel)
+  int missing_is_nan;                // the targets are drafted bytes: -1 is a refused draw (G = NaN), not a marginalised byte (G = 0)
   unsigned* status;
   uint64_t wait_limit_ns;
 };
@@ -391,7 +393,7 @@ mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
           if (p.panels == 1) {
             if (p.lse_out != nullptr) p.lse_out[e] = m + fast_lg2(s) * kLn2;
             if (tgt < 0) {
-              p.G[e] = 0.f;                                  // marginalised byte: the input unit sums to 1
+              p.G[e] = p.missing_is_nan ? CUDART_NAN_F : 0.f;   // marginalised byte: the input unit sums to 1
             } else if (tgt >= p.vv) {
               p.G[e] = CUDART_NAN_F;
               atomicOr(p.status, kStatusBadTarget);
@@ -424,7 +426,7 @@ mtpc_lowrank_gemm_kernel(const __grid_constant__ LowRankGemmParams p) {
 // left: one thread per (position, slot, component). Targets < 0 (marginalised): 0; targets >= vv: NaN and the status bit.
 __global__ void lowrank_merge_kernel(const float2* __restrict__ partial, const float* __restrict__ target_logit,
                                      const int* __restrict__ targets, float* __restrict__ G, float* __restrict__ lse_out,
-                                     unsigned* status, size_t entries, int r, int vv, int panels) {
+                                     unsigned* status, size_t entries, int r, int vv, int panels, int missing_is_nan) {
   const size_t e = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (e >= entries) return;
   float m = -CUDART_INF_F, s = 0.f;
@@ -435,7 +437,7 @@ __global__ void lowrank_merge_kernel(const float2* __restrict__ partial, const f
   const float lse = m + __logf(s);
   if (lse_out != nullptr) lse_out[e] = lse;
   const int tgt = targets[e / r];
-  if (tgt < 0) { G[e] = 0.f; return; }
+  if (tgt < 0) { G[e] = missing_is_nan ? CUDART_NAN_F : 0.f; return; }
   if (tgt >= vv) {
     G[e] = CUDART_NAN_F;
     atomicOr(status, kStatusBadTarget);
@@ -547,6 +549,69 @@ __global__ void lowrank_pad_kernel(const uint4* __restrict__ A, uint4* __restric
   const int b = static_cast<int>(rest % v64);
   const size_t u = rest / v64;
   out[idx] = b < v ? A[(u * v + b) * kv + q] : make_uint4(0u, 0u, 0u, 0u);
+}
+
+// Byte draws of a long draft on a factored head (Algorithm 1, input-unit step): one warp per (window, slot) forms the v
+// logits of the one unit the window's latent draw selected, base[t, i, :] + A[i, z] (B[i, z] h_t), in shared memory and draws
+// the byte by inverse CDF on exp(logit - max) - v k multiply-adds per draw, no tensor cores and no pass over the other
+// units. base = W_base h [P, n v] fp32 and z = B h (two bf16 halves [P, n r, 2, k]) come from two plain GEMMs.
+// v <= 512. A refused latent draw (unit_sel < 0) or byte uniform leaves the byte at -1 (preset by the latent kernel).
+constexpr int kDrawWarps = 8;
+__global__ void __launch_bounds__(32 * kDrawWarps) lowrank_draw_kernel(
+    const float* __restrict__ base, const __nv_bfloat16* __restrict__ zhl, const __nv_bfloat16* __restrict__ A,
+    const int* __restrict__ unit_sel, const float* __restrict__ uniforms, int* __restrict__ out_bytes, unsigned* status, int W,
+    int wpp, int n, int r, int v, int vv, int k) {
+  extern __shared__ float draw_sm[];                              // kDrawWarps x v logits
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float* x = draw_sm + warp * v;
+  const size_t units = static_cast<size_t>(n) * r;
+  const int pairs = W * n;
+  const int per = (v + 31) / 32;
+  for (int e = blockIdx.x * kDrawWarps + warp; e < pairs; e += gridDim.x * kDrawWarps) {
+    const int w = e / n, i = e - w * n;
+    const int z = unit_sel[e];
+    if (z < 0) continue;                                          // warp-uniform
+    const float ub = uniforms[static_cast<size_t>(w) * 2 * n + n + i];
+    if (!(ub >= 0.f && ub < 1.f)) {
+      if (lane == 0) atomicOr(status, 2u);
+      continue;
+    }
+    const size_t t = static_cast<size_t>(w / wpp);
+    const size_t unit = static_cast<size_t>(i) * r + z;
+    const __nv_bfloat16* zrow = zhl + (t * units + unit) * 2 * k;
+    const float zmine = lane < k ? __bfloat162float(zrow[lane]) + __bfloat162float(zrow[k + lane]) : 0.f;
+    float zq[kLrMaxRank];
+#pragma unroll
+    for (int q = 0; q < kLrMaxRank; ++q) zq[q] = __shfl_sync(0xffffffffu, zmine, q);
+    const float* brow = base + (t * n + i) * v;
+    float m = -CUDART_INF_F;
+    for (int b = lane; b < v; b += 32) {
+      float acc = brow[b];
+      const uint4* arow = reinterpret_cast<const uint4*>(A + (unit * v + b) * k);
+#pragma unroll
+      for (int q8 = 0; q8 < kLrMaxRank / 8; ++q8) {
+        if (q8 * 8 < k) {
+          const uint4 piece = arow[q8];
+          const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&piece);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float2 f = __bfloat1622float2(h2[u]);
+            acc = fmaf(f.x, zq[q8 * 8 + 2 * u], acc);
+            acc = fmaf(f.y, zq[q8 * 8 + 2 * u + 1], acc);
+          }
+        }
+      }
+      if (b >= vv) acc = -CUDART_INF_F;                           // [vv, v): padding symbols
+      x[b] = acc;
+      m = fmaxf(m, acc);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    __syncwarp();
+    const int byte = warp_inv_cdf_chunk<kSlotMaxPerLane>(x, 0, per, vv, m, ub, true, lane);
+    if (lane == 0) out_bytes[e] = byte;
+    __syncwarp();                                                 // x is reused by the warp's next pair
+  }
 }
 
 }  // namespace mtpc

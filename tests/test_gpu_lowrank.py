@@ -469,3 +469,41 @@ def test_factored_training_call_at_full_size_on_sampled_positions():
     assert float(dWb.sum(dim=1).abs().max()) <= 2e-2 * float(dWb.abs().max())
     assert float(dA.sum(dim=2).abs().max()) <= 2e-2 * float(dA.abs().max())
     head.mtpc_destroy()
+
+
+@pytest.mark.parametrize("family,n,r,v,d,k,P,wpp", [
+    (I.HMM, 4, 8, 48, 64, 16, 300, 1),         # one window per position: every (window, slot) forms its one unit's logits
+    (I.BTREE, 4, 4, 32, 64, 32, 200, 1),
+    (I.HMM_CTX, 3, 4, 320, 64, 16, 130, 1),    # two panels in the evidence pass
+    (I.CP, 3, 8, 64, 64, 16, 150, 2),          # two windows per position: the few-position path, 128 positions at a time
+])
+def test_long_drafts_on_a_factored_head(family, n, r, v, d, k, P, wpp):
+    """More positions than the few-position path takes (Algorithm 1 on a verification batch): bytes and log-probs against the
+    oracle on the exactly composed tensor; refused draws keep their meaning (byte -1, log-prob NaN, status bit)."""
+    wl = I.make_workload(f"lr_long_{family}_{n}_{r}", I.HeadShape(family, n, r, v, d), P, seed=6600 + n + r + v + P, wpp=wpp,
+                         weight_std=0.25)
+    W_, A, Bm = I.lowrank_parameters(n, r, v, d, k, seed=6700 + n + r, weight_std=0.25, adaptor_std=0.2)
+    U = O.lowrank_unembedding(W_, A, Bm)
+    fam = wl.shape.family
+    dh = DeviceHead(wl, lowrank=(W_, A, Bm))
+    u = wl.uniforms.copy()
+    u[5, n + 1 if n > 1 else n] = 2.0          # a refused byte draw ...
+    u[9, 0] = -1.0                             # ... and a refused latent draw
+    out_bytes, out_lp = dh.draft_sample(uniforms=torch.from_numpy(u).cuda())
+    assert dh.head.mtpc_get_status(with_code=True) == (B.MTPC_OK, B.STATUS_BAD_UNIFORM)
+    gb, gl = out_bytes.cpu().numpy(), out_lp.cpu().numpy()
+    assert gb[5, 1 if n > 1 else 0] == -1 and (gb[9] == -1).all() and np.isnan(gl[5]) and np.isnan(gl[9])
+    ok = np.ones(len(gb), dtype=bool)
+    ok[[5, 9]] = False
+    ref = O.draft_sample(fam, wl.hidden_q, U, wl.W_sum_q, wl.T_static, wpp, wl.uniforms)
+    differ = (gb != ref["bytes"]).any(axis=1) & ok
+    assert not (differ & (ref["margin"] >= 1e-6)).any()
+    same = ok & ~differ
+    assert np.abs(gl[same] - ref["logprob"][same]).max() <= 2e-3
+    # prefix marginals of the same draft
+    b2, pre = dh.draft_sample_prefix()
+    assert torch.equal(b2, dh.draft_sample()[0])
+    want = O.prefix_logprob(fam, O.head_logw(fam, wl.hidden_q, wl.W_sum_q, wl.T_static, r), O.emission_logphi(wl.hidden_q, U),
+                            wl.T_static, b2.cpu().numpy(), np.repeat(np.arange(P), wpp))
+    assert np.abs(pre.cpu().numpy() - want).max() <= 2e-3
+    dh.close()
