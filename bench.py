@@ -457,7 +457,7 @@ def measure_factored_draft(torch, wl, lowrank, peaks, P: int = 8, wpp: int = 16,
     identical = bool((ob == ref_b).all())
     status = head.mtpc_get_status()
     head.mtpc_destroy()
-    # the whole batch of the workload, one window per position: 128 positions at a time through the same path
+    # the whole batch of the workload, one window per position
     big = B.MtpcHead(B.MTPC_HMM if ctx else s.family, s.n, s.r, s.v, s.d, B.MTPC_BF16, wl.T, 1, None, W_sum, Ts,
                      flags=B.MTPC_FLAG_HMM_CONTEXTUAL if ctx else 0, v_valid=s.v_valid, lowrank=lowrank)
     hid_all = to_device_bf16(wl.hidden_q)
@@ -484,7 +484,8 @@ def measure_factored_draft(torch, wl, lowrank, peaks, P: int = 8, wpp: int = 16,
             "weight_bytes": weight_bytes, "dense_weight_bytes": dense_bytes,
             "hbm_frac": weight_bytes / (g50 * 1e-3) / 1e9 / peaks["hbm_gbs"], "device_status": status,
             "whole_batch": {"windows": wl.T, "ms_per_call": whole_ms, "windows_per_s": wl.T / (whole_ms * 1e-3),
-                            "note": "mtpc_draft_sample over all positions of the workload, one window each: chunks of 128"},
+                            "note": "mtpc_draft_sample over all positions of the workload, one window each: log omega, latent draws, one unit's "
+                                    "logits per (window, slot) from W_base h and B h, evidence by the factored projection, circuit"},
             "note": "weight pass (W_base, B, sum units) + logits from the two small products + per-slot kernel + circuit; "
                     "at these sizes the call is a chain of four short kernels, not a bandwidth problem"}
 
