@@ -761,6 +761,11 @@ int draft_sample_impl(mtpc_head* h, const void* hidden, int32_t P, int32_t wpp, 
     pt.begin();
     rc = launch_circuit(h, W, wpp, out_logprob, out_prefix, st);
     pt.end();
+    if (rc == MTPC_OK) {               // G, log omega, W_base h and B h stay in place for an acceptance call
+      h->draft_P = P;
+      h->draft_wpp = wpp;
+      h->draft_hidden = nullptr;
+    }
     return rc;
   }
   if (h->lr_k > 0 && P > L.decode_max_p) {
@@ -1617,7 +1622,9 @@ int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32
   // the workspace; what is missing is, for every window rejected at byte s, the r v logits of slot s. So: run the tests,
   // sort the rejected windows by s, stage their hidden states, recompute those logits with one sorted projection pass,
   // then run the acceptance kernel on them. In chunks of positions whose windows fit the scratch.
-  if (L.accept_rows == 0 || !head->draft_hidden) return MTPC_ERR_UNSUPPORTED;
+  const bool factored = head->lr_k > 0;     // (a long draft on a factored head left W_base h and B h instead of needing the hidden states)
+  if (L.accept_rows == 0 || (!factored && !head->draft_hidden)) return MTPC_ERR_UNSUPPORTED;
+  if (factored && head->lr_off_base == 0) return MTPC_ERR_UNSUPPORTED;
   int* ints = at<int>(head, L.off_grp_ints);
   int* counts = ints, *cursors = ints + c.n, *offsets = ints + 2 * c.n, *num_tiles = ints + 3 * c.n;
   GroupTile* tiles = at<GroupTile>(head, L.off_grp_tiles);
@@ -1640,6 +1647,30 @@ int mtpc_speculative_accept(mtpc_head* head, int32_t P, int32_t wpp, const int32
     const float* ua = accept_uniforms + w0 * (c.n + 1);
     pt.begin();
     accept_test_kernel<<<(wc + 7) / 8, 256, 0, st>>>(xb, pre, tp, ua, rej, wc, c.n, c.v, valid_symbols(c));
+    if (factored) {
+      // the slot's logits from W_base h and B h, window by window: no sort, no staging, no projection pass
+      const int pairs = wc * c.r;
+      int blocks = (pairs + kDrawWarps - 1) / kDrawWarps;
+      if (blocks > 32 * head->num_sms) blocks = 32 * head->num_sms;
+      lowrank_slot_logits_kernel<<<blocks, 32 * kDrawWarps, 0, st>>>(
+          reinterpret_cast<const float*>(head->ws + head->lr_off_base), reinterpret_cast<const __nv_bfloat16*>(head->ws + head->lr_off_zhl),
+          static_cast<const __nv_bfloat16*>(head->lr_A), rej, lg, lse, row_of, wc, static_cast<int>(w0), wpp, c.n, c.r, c.v,
+          valid_symbols(c), head->lr_k);
+      head->launches += 2;
+      pt.end();
+      int rcf = check_launch();
+      if (rcf != MTPC_OK) return rcf;
+      pt.begin();
+      spec_accept_kernel<<<wc, kAcceptThreads, smem, st>>>(
+          c.family, lg, lse, at<float>(head, L.off_logw) + static_cast<size_t>(p0) * L.sum_rows,
+          tables + static_cast<size_t>(p0) * tstride, xb, pre, tp, ua, out_accepted + w0, out_next_byte + w0,
+          at<unsigned>(head, L.off_status), wc, wpp, c.n, c.r, c.v, valid_symbols(c), L.sum_rows, tstride,
+          at<float>(head, L.off_G) + w0 * c.n * c.r, row_of);
+      head->launches++;
+      pt.end();
+      if ((rcf = check_launch()) != MTPC_OK) return rcf;
+      continue;
+    }
     if (cudaMemsetAsync(ints, 0, static_cast<size_t>(2 * c.n) * 4, st) != cudaSuccess) return MTPC_ERR_CUDA;
     const int cblocks = (wc + kGroupThreads - 1) / kGroupThreads;
     group_count_kernel<<<cblocks < 4 * head->num_sms ? cblocks : 4 * head->num_sms, kGroupThreads, c.n * sizeof(int), st>>>(

@@ -614,4 +614,60 @@ __global__ void __launch_bounds__(32 * kDrawWarps) lowrank_draw_kernel(
   }
 }
 
+// Acceptance stage after a long draft on a factored head (Algorithm 3): for every window whose draft was rejected at byte s
+// (first_rejected[w] = s >= 0) the r v logits of slot s and the r log-sum-exps, which no call kept:
+// logits[w, j, :] = base[t, s, :] + A[s, j] (B[s, j] h_t). One warp per (window, component); rows of the outputs are the
+// windows themselves (row_of[w] = w). Padding symbols get -inf, as in the projection kernels.
+__global__ void __launch_bounds__(32 * kDrawWarps) lowrank_slot_logits_kernel(
+    const float* __restrict__ base, const __nv_bfloat16* __restrict__ zhl, const __nv_bfloat16* __restrict__ A,
+    const int* __restrict__ first_rejected, float* __restrict__ logits, float* __restrict__ unit_lse, int* __restrict__ row_of,
+    int W, int w_first, int wpp, int n, int r, int v, int vv, int k) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const size_t units = static_cast<size_t>(n) * r;
+  const int pairs = W * r;
+  for (int e = blockIdx.x * kDrawWarps + warp; e < pairs; e += gridDim.x * kDrawWarps) {
+    const int w = e / r, j = e - w * r;
+    if (j == 0 && lane == 0) row_of[w] = w;
+    const int s = first_rejected[w];
+    if (s < 0) continue;                                          // warp-uniform: everything accepted, no residual draw
+    const size_t t = static_cast<size_t>((w_first + w) / wpp);
+    const size_t unit = static_cast<size_t>(s) * r + j;
+    const __nv_bfloat16* zrow = zhl + (t * units + unit) * 2 * k;
+    const float zmine = lane < k ? __bfloat162float(zrow[lane]) + __bfloat162float(zrow[k + lane]) : 0.f;
+    float zq[kLrMaxRank];
+#pragma unroll
+    for (int q = 0; q < kLrMaxRank; ++q) zq[q] = __shfl_sync(0xffffffffu, zmine, q);
+    const float* brow = base + (t * n + s) * v;
+    float* out = logits + (static_cast<size_t>(w) * r + j) * v;
+    float m = -CUDART_INF_F, sum = 0.f;
+    for (int b = lane; b < v; b += 32) {
+      float acc = brow[b];
+      const uint4* arow = reinterpret_cast<const uint4*>(A + (unit * v + b) * k);
+#pragma unroll
+      for (int q8 = 0; q8 < kLrMaxRank / 8; ++q8) {
+        if (q8 * 8 < k) {
+          const uint4 piece = arow[q8];
+          const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&piece);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float2 f = __bfloat1622float2(h2[u]);
+            acc = fmaf(f.x, zq[q8 * 8 + 2 * u], acc);
+            acc = fmaf(f.y, zq[q8 * 8 + 2 * u + 1], acc);
+          }
+        }
+      }
+      if (b >= vv) acc = -CUDART_INF_F;
+      out[b] = acc;
+      lse_merge(m, sum, acc, 1.f);                                // running (maximum, sum of exponentials) of this lane's symbols
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m, off);
+      const float s2 = __shfl_xor_sync(0xffffffffu, sum, off);
+      lse_merge(m, sum, m2, s2);
+    }
+    if (lane == 0) unit_lse[static_cast<size_t>(w) * r + j] = m + __logf(sum);
+  }
+}
+
 }  // namespace mtpc

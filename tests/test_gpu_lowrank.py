@@ -200,12 +200,6 @@ def test_factored_head_matches_the_composed_definition(family, n, r, v, vv, d, k
     differ = (drafted.cpu().numpy() != d_ref["bytes"]).any(axis=1)
     assert not (differ & (d_ref["margin"] >= 1e-6)).any()
     assert np.abs(out.cpu().numpy()[~differ] - d_ref["logprob"][~differ]).max() <= 2e-3
-    if T > 128:                                                            # only the last chunk's logits remain
-        with pytest.raises(B.MtpcError) as e:
-            head.mtpc_speculative_accept(T, 1, drafted, pre, torch.zeros((T, n + 1, v), device="cuda"),
-                                         torch.zeros((T, n + 1), device="cuda"), torch.empty(T, dtype=torch.int32, device="cuda"),
-                                         torch.empty(T, dtype=torch.int32, device="cuda"))
-        assert e.value.code == B.ERR_STATE
     with pytest.raises(B.MtpcError) as e:
         head.mtpc_window_logprob_backward(hidden, targets, torch.ones(T, device="cuda"), out, torch.empty((T, d), device="cuda"),
                                           torch.empty((n, r, v, d), device="cuda"), torch.empty((wl.W_sum_q.shape[0], d), device="cuda"),
@@ -506,4 +500,11 @@ def test_long_drafts_on_a_factored_head(family, n, r, v, d, k, P, wpp):
     want = O.prefix_logprob(fam, O.head_logw(fam, wl.hidden_q, wl.W_sum_q, wl.T_static, r), O.emission_logphi(wl.hidden_q, U),
                             wl.T_static, b2.cpu().numpy(), np.repeat(np.arange(P), wpp))
     assert np.abs(pre.cpu().numpy() - want).max() <= 2e-3
+    if wpp > 1:                                # drafted 128 positions at a time: only the last chunk's logits remain
+        W = P * wpp
+        with pytest.raises(B.MtpcError) as e:
+            dh.head.mtpc_speculative_accept(P, wpp, b2, pre, torch.zeros((W, n + 1, v), device="cuda"),
+                                            torch.zeros((W, n + 1), device="cuda"), torch.empty(W, dtype=torch.int32, device="cuda"),
+                                            torch.empty(W, dtype=torch.int32, device="cuda"))
+        assert e.value.code == B.ERR_STATE
     dh.close()

@@ -212,6 +212,12 @@ def test_accept_small_shapes(family, n, r, v, d, P, wpp):
     (I.BTREE, 4, 16, 256, 128, 16, 6, 8),
     (I.HMM_CTX, 4, 4, 48, 64, 16, 128, 2),     # the most positions the few-position path takes
     (I.CP, 2, 4, 1024, 64, 16, 3, 4),          # a vocabulary wider than 512 symbols
+    # more than 128 positions, one window each: bytes drawn from the one selected unit, the rejected slot's logits formed
+    # window by window from W_base h and B h
+    (I.CP, 3, 8, 64, 64, 16, 150, 1),
+    (I.HMM, 4, 8, 48, 64, 32, 140, 1),
+    (I.BTREE, 4, 4, 32, 64, 16, 200, 1),
+    (I.HMM_CTX, 3, 4, 320, 64, 16, 130, 1),
 ])
 def test_draft_and_accept_on_a_factored_low_rank_head(family, n, r, v, d, k, P, wpp):
     """App. G's shared unembeddings kept factored (U_ij = W_i + A_ij B_ij never formed): the few-position draft streams
