@@ -474,6 +474,25 @@ def measure_factored_draft(torch, wl, lowrank, peaks, P: int = 8, wpp: int = 16,
     e1.record()
     torch.cuda.synchronize()
     whole_ms = e0.elapsed_time(e1) / 5
+    # draft (with prefix marginals) + acceptance stage against synthetic target-model rows, whole batch
+    tp_all = torch.from_numpy(I.target_rows(I.BASE_SEED + 93, 9, (wl.T, s.n + 1, s.v))).cuda()
+    ua_all = torch.from_numpy(I.uniforms(I.BASE_SEED + 94, 10, (wl.T, s.n + 1))).cuda()
+    pre_all = torch.empty((wl.T, s.n), dtype=torch.float32, device="cuda")
+    acc_all = torch.empty(wl.T, dtype=torch.int32, device="cuda")
+    nxt_all = torch.empty(wl.T, dtype=torch.int32, device="cuda")
+
+    def cycle():
+        big.mtpc_draft_sample_prefix(hid_all, 1, u_all, ob_all, pre_all)
+        big.mtpc_speculative_accept(wl.T, 1, ob_all, pre_all, tp_all, ua_all, acc_all, nxt_all)
+    for _ in range(2):
+        cycle()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(5):
+        cycle()
+    e1.record()
+    torch.cuda.synchronize()
+    cycle_ms = e0.elapsed_time(e1) / 5
     status |= big.mtpc_get_status()
     big.mtpc_destroy()
     p50, g50 = statistics.median(lat), statistics.median(graph_lat)
@@ -484,6 +503,7 @@ def measure_factored_draft(torch, wl, lowrank, peaks, P: int = 8, wpp: int = 16,
             "weight_bytes": weight_bytes, "dense_weight_bytes": dense_bytes,
             "hbm_frac": weight_bytes / (g50 * 1e-3) / 1e9 / peaks["hbm_gbs"], "device_status": status,
             "whole_batch": {"windows": wl.T, "ms_per_call": whole_ms, "windows_per_s": wl.T / (whole_ms * 1e-3),
+                            "draft_plus_accept_ms": cycle_ms,
                             "note": "mtpc_draft_sample over all positions of the workload, one window each: log omega, latent draws, one unit's "
                                     "logits per (window, slot) from W_base h and B h, evidence by the factored projection, circuit"},
             "note": "weight pass (W_base, B, sum units) + logits from the two small products + per-slot kernel + circuit; "

@@ -296,11 +296,11 @@ int mtpc_lowrank_backward(int32_t n, int32_t r, int32_t v, int32_t d, int32_t k,
  *            of A in the layout the kernel reads (remade on every call, so A is always read as it is then) and, for
  *            v > 224, the per-panel partial log-sum-exps.
  * Such a head serves mtpc_window_logprob, mtpc_window_prefix_logprob, mtpc_window_loss, mtpc_window_logprob_host,
- * mtpc_draft_sample, mtpc_draft_sample_prefix and, after a draft of up to 128 positions, mtpc_speculative_accept: the
- * draft's weight pass streams W_base and B (n v + n r k rows) instead of n r v composed rows, and the logits are formed
- * from the two small products; longer drafts form, per (window, slot), the logits of the one unit the latent draw
- * selected (one window per position, v <= 512) or run 128 positions at a time, and keep no logits (the acceptance stage
- * then returns MTPC_ERR_STATE). Its training calls are mtpc_lowrank_window_logprob_backward and
+ * mtpc_draft_sample, mtpc_draft_sample_prefix and mtpc_speculative_accept: up to 128 positions, the draft's weight pass
+ * streams W_base and B (n v + n r k rows) instead of n r v composed rows and the logits are formed from the two small
+ * products; longer drafts with one window per position and v <= 512 form, per (window, slot), the logits of the one unit
+ * the latent draw selected, and the acceptance stage after them forms the rejected slot's logits the same way; other
+ * long drafts run 128 positions at a time and keep no logits (mtpc_speculative_accept then returns MTPC_ERR_STATE). Its training calls are mtpc_lowrank_window_logprob_backward and
  * mtpc_lowrank_window_loss_backward (below); mtpc_window_logprob_backward and mtpc_window_loss_backward return
  * MTPC_ERR_UNSUPPORTED on it (they produce the gradient of a composed tensor: mtpc_lowrank_compose + mtpc_create_head,
  * carried back by mtpc_lowrank_backward).
