@@ -109,11 +109,33 @@ __global__ void circuit_cp_kernel(const float* __restrict__ G, const float* __re
 // One sum layer seen from the parent: returns, for lane = parent value z, LSE_b(logOmega_c[z][b] + pc[b]).
 // tab: the child's r x r table in global memory; pc: r floats in shared memory (written before the call; the
 // function synchronises the warp); table: r * (r+1) floats of per-warp shared scratch.
+// An r x r table from global memory into a padded shared tile (row pitch r + 1), by one warp. ROWS > 1: that many rows'
+// loads are in flight before the first store - for a kernel where one warp walks many tables on its own (a load-store pair
+// per row costs one memory round trip per row); a kernel with many such warps per SM hides that latency and is better
+// off with the plain loop's few registers.
+template <int ROWS>
+__device__ __forceinline__ void btree_stage_table(const float* __restrict__ tab, float* table, int lane, int r) {
+  const bool has = lane < r;
+  if (ROWS == 1) {
+    for (int a = 0; a < r; ++a)
+      if (has) table[a * (r + 1) + lane] = tab[a * r + lane];
+    return;
+  }
+  for (int a0 = 0; a0 < r; a0 += ROWS) {
+    float t[ROWS];
+#pragma unroll
+    for (int q = 0; q < ROWS; ++q) t[q] = (has && a0 + q < r) ? tab[(a0 + q) * r + lane] : 0.f;
+#pragma unroll
+    for (int q = 0; q < ROWS; ++q)
+      if (has && a0 + q < r) table[(a0 + q) * (r + 1) + lane] = t[q];
+  }
+}
+
+template <int ROWS = 1>
 __device__ __forceinline__ float btree_sum_layer(const float* __restrict__ tab, const float* pc, float* table,
                                                  int lane, int r) {
   const bool has = lane < r;
-  for (int a = 0; a < r; ++a)                      // coalesced rows -> padded shared tile
-    if (has) table[a * (r + 1) + lane] = tab[a * r + lane];
+  btree_stage_table<ROWS>(tab, table, lane, r);    // coalesced rows -> padded shared tile
   __syncwarp();
   float res = 0.f;
   if (has) {

@@ -697,7 +697,7 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
         float acc = 0.f;
         for (int side = 0; side < 2; ++side) {
           const int ch = 2 * j + 1 + side;
-          const float sc = btree_sum_layer(lw + r + static_cast<size_t>(ch - 1) * r * r, prod + ch * r, table, lane, r);
+          const float sc = btree_sum_layer<16>(lw + r + static_cast<size_t>(ch - 1) * r * r, prod + ch * r, table, lane, r);
           if (has) S[ch * r + lane] = sc;
           acc += sc;
         }
@@ -715,11 +715,13 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
         const int sib = (child & 1) ? child + 1 : child - 1;
         if (has) cur[lane] = up + S[sib * r + lane];
         __syncwarp();
-        const float* tab = lw + r + static_cast<size_t>(child - 1) * r * r;   // [parent value z][own value b]
+        // the child's table [parent value z][own value b], staged into the padded shared tile first
+        btree_stage_table<16>(lw + r + static_cast<size_t>(child - 1) * r * r, table, lane, r);
+        __syncwarp();
         float m = -CUDART_INF_F;
-        for (int z = 0; z < r; ++z) m = fmaxf(m, has ? cur[z] + tab[z * r + lane] : -CUDART_INF_F);
+        for (int z = 0; z < r; ++z) m = fmaxf(m, has ? cur[z] + table[z * (r + 1) + lane] : -CUDART_INF_F);
         float acc = 0.f;
-        for (int z = 0; z < r; ++z) acc += has ? __expf(cur[z] + tab[z * r + lane] - m) : 0.f;
+        for (int z = 0; z < r; ++z) acc += has ? __expf(cur[z] + table[z * (r + 1) + lane] - m) : 0.f;
         up = has ? m + __logf(acc) : -CUDART_INF_F;
         __syncwarp();
         node = child;
