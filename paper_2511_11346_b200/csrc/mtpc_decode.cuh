@@ -678,7 +678,14 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_kernel(
         const float e = has ? __expf(alpha - m) : 0.f;
         const float* A = logA + static_cast<size_t>(pos) * logA_stride + static_cast<size_t>(i) * r * r;
         float acc = 0.f;
-        for (int a = 0; a < r; ++a) acc = fmaf(__shfl_sync(kFull, e, a), has ? __expf(__ldg(A + a * r + lane)) : 0.f, acc);
+        for (int a0 = 0; a0 < r; a0 += 16) {           // sixteen rows of the table in flight at a time
+          float tv[16];
+#pragma unroll
+          for (int q = 0; q < 16; ++q) tv[q] = (has && a0 + q < r) ? __ldg(A + (a0 + q) * r + lane) : -CUDART_INF_F;
+#pragma unroll
+          for (int q = 0; q < 16; ++q)
+            if (a0 + q < r) acc = fmaf(__shfl_sync(kFull, e, a0 + q), __expf(tv[q]), acc);
+        }
         alpha = has ? m + __logf(acc) : -CUDART_INF_F;
       }
       c = alpha;
